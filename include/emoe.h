@@ -1,0 +1,191 @@
+/*
+ * emoe — sparse MoE layer forward on per-expert mixed-bitwidth (INT2/INT4/INT8) packed
+ * weights, for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * Method: EdgeMoE (arXiv 2308.14352).  Section 3.2 stores every expert at its own
+ * bitwidth with channel-wise linear quantisation and a float16 scale channel, and
+ * decompresses (w~ = q * s) before use; Sections 1 and 2.1 define the layer: a router
+ * sends each token to its Top-K experts, each expert an independent FFN.  This library
+ * computes the same layer but forms q * s in registers: dequantised weights are never
+ * written to memory.
+ *
+ * Conventions
+ *   - Every function returns an int status: EMOE_OK (0) or a negative EMOE_ERR_* code.
+ *     No exceptions, no abort, nothing printed.
+ *   - Pointers are DEVICE pointers unless the parameter name starts with `host_`.
+ *     The library never takes ownership of caller memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Work is enqueued asynchronously; argument errors are reported synchronously,
+ *     before anything is enqueued.
+ *   - A context belongs to one device and must be used by one host thread at a time.
+ *     Calls that share a context share its workspace: they must be ordered on the GPU
+ *     (same stream, or explicit dependencies).
+ *   - Matrices: an expert matrix has N output channels (rows) and K inputs (columns).
+ *     ReLU experts:   m = 0  W_in [d_ff][d_model],  m = 1  W_out [d_model][d_ff].
+ *     SwiGLU experts: m = 0  w1 [d_ff][d_model], m = 1  w3 [d_ff][d_model],
+ *                     m = 2  w2 [d_model][d_ff].
+ *
+ * Storage format of a packed matrix (part of the ABI; Section 3.2 leaves it open)
+ *   qmax(b) = 2^(b-1) - 1.  Per output channel n and per group g of `group` consecutive
+ *   inputs (group = 0: the whole row):
+ *       amax  = max |w|,   s32 = amax / qmax (IEEE fp32 division),
+ *       s     = s32, or s32 rounded to fp16 (nearest even) when scale_dtype = F16,
+ *       q     = clamp(round_half_even(w / s), -qmax, qmax)   (fp32 division by the
+ *               STORED scale; q = 0 when s = 0).
+ *   Codes: b-bit two's-complement fields; element k of row n sits at bit offset
+ *   (k*b) mod 8 of byte n*(K*b/8) + (k*b)/8 (low bits first).  Scales: [N][K/group]
+ *   row-major in scale_dtype.
+ */
+#ifndef EMOE_H_
+#define EMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define EMOE_OK 0
+#define EMOE_ERR_INVALID_ARG (-1)  /* null pointer, non-positive size, top_k > E, group does not divide K ... */
+#define EMOE_ERR_UNSUPPORTED (-2)  /* bits not in {2,4,8}, unknown enum value, shape outside the kernels' limits */
+#define EMOE_ERR_ALIGNMENT (-3)    /* a pointer or row size is not 16-byte aligned */
+#define EMOE_ERR_WORKSPACE (-4)    /* the context's workspace is too small for this call */
+#define EMOE_ERR_CUDA (-5)         /* a CUDA call failed; emoe_last_cuda_error() gives its code */
+#define EMOE_ERR_DEVICE_CHECK (-6) /* a kernel found inconsistent data (e.g. an expert id out of range) */
+
+/* enums (plain ints in the ABI) */
+#define EMOE_DTYPE_F32 0
+#define EMOE_DTYPE_F16 1
+#define EMOE_DTYPE_BF16 2
+#define EMOE_ACT_RELU 0
+#define EMOE_ACT_SWIGLU 1
+#define EMOE_GATE_SOFTMAX 0        /* gate = softmax probability of the pick over all experts */
+#define EMOE_GATE_SOFTMAX_RENORM 1 /* gate = that probability / sum over the token's K picks */
+
+#define EMOE_MAX_EXPERTS 256
+#define EMOE_MAX_TOP_K 8
+
+typedef struct emoe_ctx emoe_ctx;
+
+/* One expert of a layer: its bitwidth and DEVICE pointers to its packed matrices and
+ * scale channels (Section 3.2: experts of one layer may differ in bitwidth).
+ * ReLU uses entries 0..1, SwiGLU 0..2 (order as listed above). */
+typedef struct emoe_expert {
+  int32_t bits; /* 2, 4 or 8 */
+  int32_t reserved;
+  const void* packed[3];
+  const void* scales[3];
+} emoe_expert;
+
+/* Static description of a layer. */
+typedef struct emoe_layer_desc {
+  int32_t d_model;
+  int32_t d_ff;
+  int32_t n_experts;   /* 1 .. EMOE_MAX_EXPERTS */
+  int32_t top_k;       /* 1 .. min(n_experts, EMOE_MAX_TOP_K) */
+  int32_t act;         /* EMOE_ACT_* */
+  int32_t gate_mode;   /* EMOE_GATE_* */
+  int32_t group;       /* 0 = one scale per output channel, else inputs per scale */
+  int32_t scale_dtype; /* EMOE_DTYPE_F32 | EMOE_DTYPE_F16 */
+  int32_t act_dtype;   /* EMOE_DTYPE_F32 | EMOE_DTYPE_BF16: type of x and of the hidden vector */
+} emoe_layer_desc;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Creates a context on `device` owning `workspace_bytes` of device scratch (intermediate
+ * results of a forward call: the paper's "working buffer", Section 3.1).  Returns NULL and
+ * sets *status on failure.  This is the only call (with emoe_destroy) that allocates or
+ * frees device memory. */
+emoe_ctx* emoe_create(int device, size_t workspace_bytes, int* status);
+int emoe_destroy(emoe_ctx* ctx);
+
+/* Scratch a forward call over T tokens needs; pass the maximum over your calls to
+ * emoe_create.  Returns 0 for an invalid description. */
+size_t emoe_workspace_bytes(const emoe_layer_desc* desc, int T);
+
+/* CUDA error code of the last failed CUDA call on this context (0 if none). */
+int emoe_last_cuda_error(const emoe_ctx* ctx);
+
+/* Reads (and clears) the device-side check word: EMOE_OK, or EMOE_ERR_DEVICE_CHECK if a
+ * kernel of an earlier call met inconsistent data.  Synchronises `stream`. */
+int emoe_device_status(emoe_ctx* ctx, void* stream);
+
+const char* emoe_status_string(int status);
+
+/* ---- sizes -------------------------------------------------------------------------- */
+
+size_t emoe_packed_bytes(int N, int K, int bits);                   /* N*K*bits/8, 0 if invalid */
+size_t emoe_scales_bytes(int N, int K, int group, int scale_dtype); /* N*(K/group)*sizeof, 0 if invalid */
+
+/* ---- Section 3.2: expert-wise quantisation ------------------------------------------- */
+
+/* Quantises and packs one matrix W[N][K] (fp32, row-major, rows = output channels) to
+ * `bits` in the storage format described at the top of this file.
+ *   group: 0 or a multiple of 4 that divides K;  K*bits must be a multiple of 32.
+ *   out_packed: emoe_packed_bytes(N,K,bits) bytes; out_scales: emoe_scales_bytes(...).
+ *   W and out_packed must be 16-byte aligned, out_scales 4-byte aligned.
+ * Bit-exact with the definition: IEEE division and round-half-even, no fast-math. */
+int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int group, int scale_dtype,
+                     void* out_packed, void* out_scales, void* stream);
+
+/* ---- Sections 1, 2.1: router and Top-K gating ----------------------------------------- */
+
+/* z[t][e] = sum_i x[t][i] * router_W[i][e] (+ bias), p = softmax(z) over all experts; the
+ * top_k largest logits are selected (ties: lower expert index) and listed in descending
+ * order of logit.
+ *   x: [T][d] in act_dtype (F32 or BF16); router_W: [d][E] fp32;
+ *   router_bias: NULL, or fp32 with bias[t*bias_token_stride + e]
+ *                (bias_token_stride = 0: one vector for all tokens; = E: one per token);
+ *   out_ids [T][top_k] int32, out_gates [T][top_k] fp32, out_logits NULL or [T][E] fp32.
+ * Accumulation is fp32. */
+int emoe_router_topk(emoe_ctx* ctx, const void* x, int act_dtype, int T, int d, const float* router_W,
+                     const float* router_bias, int bias_token_stride, int E, int top_k, int gate_mode,
+                     int32_t* out_ids, float* out_gates, float* out_logits, void* stream);
+
+/* Token -> expert permutation: stable counting sort of the pair indices p = t*top_k + j by
+ * expert id.  out_counts [E], out_off [E+1] (exclusive prefix sum), out_perm [n_pairs]
+ * (pair indices in expert order, increasing inside an expert), out_slot_of_pair [n_pairs]
+ * (the inverse: position of pair p in out_perm; may be NULL).  Ids outside [0,E) set the
+ * device check word and are dropped. */
+int emoe_permute(emoe_ctx* ctx, const int32_t* ids, int n_pairs, int E, int32_t* out_counts, int32_t* out_off,
+                 int32_t* out_perm, int32_t* out_slot_of_pair, void* stream);
+
+/* ---- the layer ------------------------------------------------------------------------ */
+
+/* Full layer forward (Sections 1, 2.1 on the Section 3.2 storage):
+ * router -> Top-K -> permutation -> expert FFNs on packed weights -> weighted combine.
+ *   ReLU:   h = max(0, x W~in^T),            o = h W~out^T
+ *   SwiGLU: h = silu(x W~1^T) * (x W~3^T),   o = h W~2^T
+ *   y[t] = sum_j gate[t][j] * o[pair (t,j)],  W~[n][k] = q[n][k] * s[n][k/group].
+ * With BF16 activations the hidden vector h is rounded once to bf16; with F32 it stays
+ * fp32.  Only the distinct activated experts' weights are read.
+ *   x [T][d_model] in desc->act_dtype; y [T][d_model] fp32.
+ *   host_experts: HOST array of desc->n_experts entries holding DEVICE pointers; the
+ *     library keeps a device copy per distinct table (by content), uploaded on `stream`
+ *     the first time a table is seen.
+ *   out_ids / out_gates ([T][top_k]) and out_perm ([T*top_k]) are optional (NULL) copies
+ *   of the routing decisions.
+ * Shape limits: d_model and d_ff multiples of 32 with K*bits/8 a multiple of 16 for every
+ * matrix; group 0 or a multiple of 32 (INT8), 32 (INT4), 64 (INT2) dividing K.
+ * Uses the context workspace (emoe_workspace_bytes). */
+int emoe_moe_forward(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int T, const float* router_W,
+                     const float* router_bias, int bias_token_stride, const emoe_expert* host_experts, float* y,
+                     int32_t* out_ids, float* out_gates, int32_t* out_perm, void* stream);
+
+/* Same layer with the routing decisions given (ids [T][top_k] in [0,E), gates [T][top_k]):
+ * runs the permutation, the expert FFNs and the combine only. */
+int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int T, const int32_t* ids,
+                            const float* gates, const emoe_expert* host_experts, float* y, int32_t* out_perm,
+                            void* stream);
+
+/* Selects the expert-FFN kernel family: 0 = automatic (default), 1 = force the CUDA-core
+ * grouped GEMV, 2 = force the tensor-core path where the shape allows it.  For tests and
+ * measurements. */
+int emoe_set_ffn_path(emoe_ctx* ctx, int path);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EMOE_H_ */

@@ -1,0 +1,173 @@
+"""ctypes binding of libemoe.so: one Python function per C entry point of include/emoe.h,
+same names, argument marshalling only.  Tensors are passed as raw device pointers
+(``tensor.data_ptr()``), streams as ``torch.cuda.Stream.cuda_stream`` integers.
+
+There is no fallback: if the library has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libemoe.so")
+
+OK = 0
+ERR_INVALID_ARG = -1
+ERR_UNSUPPORTED = -2
+ERR_ALIGNMENT = -3
+ERR_WORKSPACE = -4
+ERR_CUDA = -5
+ERR_DEVICE_CHECK = -6
+
+DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
+ACT_RELU, ACT_SWIGLU = 0, 1
+GATE_SOFTMAX, GATE_SOFTMAX_RENORM = 0, 1
+
+EXPORTS = (
+    "emoe_create", "emoe_destroy", "emoe_workspace_bytes", "emoe_last_cuda_error", "emoe_device_status",
+    "emoe_status_string", "emoe_packed_bytes", "emoe_scales_bytes", "emoe_pack_expert", "emoe_router_topk",
+    "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path",
+)
+
+
+class EmoeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+class emoe_expert(ctypes.Structure):
+    _fields_ = [("bits", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("packed", ctypes.c_void_p * 3), ("scales", ctypes.c_void_p * 3)]
+
+
+class emoe_layer_desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("d_model", "d_ff", "n_experts", "top_k", "act", "gate_mode", "group", "scale_dtype", "act_dtype")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library; raises if it is missing (no CPU fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2308_14352_b200.build` "
+                "(needs nvcc); this package has no fallback path")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.emoe_create.restype = vp
+        L.emoe_create.argtypes = [i32, sz, ctypes.POINTER(ctypes.c_int)]
+        L.emoe_destroy.argtypes = [vp]
+        L.emoe_workspace_bytes.restype = sz
+        L.emoe_workspace_bytes.argtypes = [ctypes.POINTER(emoe_layer_desc), i32]
+        L.emoe_last_cuda_error.argtypes = [vp]
+        L.emoe_device_status.argtypes = [vp, vp]
+        L.emoe_status_string.restype = ctypes.c_char_p
+        L.emoe_status_string.argtypes = [i32]
+        L.emoe_packed_bytes.restype = sz
+        L.emoe_packed_bytes.argtypes = [i32, i32, i32]
+        L.emoe_scales_bytes.restype = sz
+        L.emoe_scales_bytes.argtypes = [i32, i32, i32, i32]
+        L.emoe_pack_expert.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.emoe_router_topk.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.emoe_permute.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
+        L.emoe_moe_forward.argtypes = [vp, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp, i32,
+                                       ctypes.POINTER(emoe_expert), vp, vp, vp, vp, vp]
+        L.emoe_moe_forward_routed.argtypes = [vp, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
+                                              ctypes.POINTER(emoe_expert), vp, vp, vp]
+        L.emoe_set_ffn_path.argtypes = [vp, i32]
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise EmoeError(status, where)
+
+
+def status_string(status: int) -> str:
+    return lib().emoe_status_string(status).decode()
+
+
+def emoe_create(device: int, workspace_bytes: int) -> int:
+    st = ctypes.c_int(0)
+    ctx = lib().emoe_create(device, workspace_bytes, ctypes.byref(st))
+    if not ctx:
+        raise EmoeError(st.value, "emoe_create")
+    return ctx
+
+
+def emoe_destroy(ctx: int) -> None:
+    _check(lib().emoe_destroy(ctx), "emoe_destroy")
+
+
+def emoe_workspace_bytes(desc: emoe_layer_desc, T: int) -> int:
+    return int(lib().emoe_workspace_bytes(ctypes.byref(desc), T))
+
+
+def emoe_last_cuda_error(ctx: int) -> int:
+    return int(lib().emoe_last_cuda_error(ctx))
+
+
+def emoe_device_status(ctx: int, stream: int = 0) -> int:
+    return int(lib().emoe_device_status(ctx, stream))
+
+
+def emoe_packed_bytes(N: int, K: int, bits: int) -> int:
+    return int(lib().emoe_packed_bytes(N, K, bits))
+
+
+def emoe_scales_bytes(N: int, K: int, group: int, scale_dtype: int) -> int:
+    return int(lib().emoe_scales_bytes(N, K, group, scale_dtype))
+
+
+def emoe_pack_expert(ctx, W_ptr, N, K, bits, group, scale_dtype, out_packed_ptr, out_scales_ptr, stream=0) -> None:
+    _check(lib().emoe_pack_expert(ctx, W_ptr, N, K, bits, group, scale_dtype, out_packed_ptr, out_scales_ptr, stream),
+           "emoe_pack_expert")
+
+
+def emoe_router_topk(ctx, x_ptr, act_dtype, T, d, router_W_ptr, bias_ptr, bias_token_stride, E, top_k, gate_mode,
+                     out_ids_ptr, out_gates_ptr, out_logits_ptr=None, stream=0) -> None:
+    _check(lib().emoe_router_topk(ctx, x_ptr, act_dtype, T, d, router_W_ptr, bias_ptr, bias_token_stride, E, top_k,
+                                  gate_mode, out_ids_ptr, out_gates_ptr, out_logits_ptr, stream), "emoe_router_topk")
+
+
+def emoe_permute(ctx, ids_ptr, n_pairs, E, out_counts_ptr, out_off_ptr, out_perm_ptr, out_slot_of_pair_ptr=None,
+                 stream=0) -> None:
+    _check(lib().emoe_permute(ctx, ids_ptr, n_pairs, E, out_counts_ptr, out_off_ptr, out_perm_ptr,
+                              out_slot_of_pair_ptr, stream), "emoe_permute")
+
+
+def make_expert_table(entries: Sequence[tuple]):
+    """entries[e] = (bits, [packed ptrs], [scale ptrs]) -> ctypes array of emoe_expert."""
+    tab = (emoe_expert * len(entries))()
+    for e, (bits, packed, scales) in enumerate(entries):
+        tab[e].bits = bits
+        tab[e].reserved = 0
+        for m in range(3):
+            tab[e].packed[m] = packed[m] if m < len(packed) else None
+            tab[e].scales[m] = scales[m] if m < len(scales) else None
+    return tab
+
+
+def emoe_moe_forward(ctx, desc: emoe_layer_desc, x_ptr, T, router_W_ptr, bias_ptr, bias_token_stride, expert_table,
+                     y_ptr, out_ids_ptr=None, out_gates_ptr=None, out_perm_ptr=None, stream=0) -> None:
+    _check(lib().emoe_moe_forward(ctx, ctypes.byref(desc), x_ptr, T, router_W_ptr, bias_ptr, bias_token_stride,
+                                  expert_table, y_ptr, out_ids_ptr, out_gates_ptr, out_perm_ptr, stream),
+           "emoe_moe_forward")
+
+
+def emoe_moe_forward_routed(ctx, desc: emoe_layer_desc, x_ptr, T, ids_ptr, gates_ptr, expert_table, y_ptr,
+                            out_perm_ptr=None, stream=0) -> None:
+    _check(lib().emoe_moe_forward_routed(ctx, ctypes.byref(desc), x_ptr, T, ids_ptr, gates_ptr, expert_table, y_ptr,
+                                         out_perm_ptr, stream), "emoe_moe_forward_routed")
+
+
+def emoe_set_ffn_path(ctx, path: int) -> None:
+    _check(lib().emoe_set_ffn_path(ctx, path), "emoe_set_ffn_path")

@@ -1,0 +1,368 @@
+// C ABI of libemoe: context, argument checks, and the orchestration of one layer forward
+// (router -> Top-K -> permutation -> expert FFNs on packed weights -> combine).  All
+// arithmetic is in the kernels of the sibling files; nothing here touches tensor data on the
+// host.
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace emoe;
+
+namespace {
+
+constexpr int MAX_TABLES = 256;  // distinct expert tables a context can keep on the device
+
+struct TableEntry {
+  std::vector<emoe_expert> host;
+};
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+struct WorkspaceLayout {
+  size_t ids, gates, counts, off, perm, slot_of_pair, xs, hidden, o_part, total;
+  int ksplit;
+};
+
+bool make_dims(const emoe_layer_desc* d, LayerDims* L) {
+  if (!d) return false;
+  if (d->d_model <= 0 || d->d_ff <= 0) return false;
+  if (d->n_experts < 1 || d->n_experts > EMOE_MAX_EXPERTS) return false;
+  if (d->top_k < 1 || d->top_k > d->n_experts || d->top_k > EMOE_MAX_TOP_K) return false;
+  if (d->act != EMOE_ACT_RELU && d->act != EMOE_ACT_SWIGLU) return false;
+  if (d->gate_mode != EMOE_GATE_SOFTMAX && d->gate_mode != EMOE_GATE_SOFTMAX_RENORM) return false;
+  if (d->scale_dtype != EMOE_DTYPE_F32 && d->scale_dtype != EMOE_DTYPE_F16) return false;
+  if (d->act_dtype != EMOE_DTYPE_F32 && d->act_dtype != EMOE_DTYPE_BF16) return false;
+  if (d->group < 0) return false;
+  if (d->group > 0 && (d->d_model % d->group != 0 || d->d_ff % d->group != 0)) return false;
+  L->d_model = d->d_model;
+  L->d_ff = d->d_ff;
+  L->E = d->n_experts;
+  L->top_k = d->top_k;
+  L->act = d->act;
+  L->gate_mode = d->gate_mode;
+  L->group = d->group;
+  L->scale_f16 = d->scale_dtype == EMOE_DTYPE_F16;
+  L->act_bf16 = d->act_dtype == EMOE_DTYPE_BF16;
+  return true;
+}
+
+WorkspaceLayout make_layout(const LayerDims& L, int T) {
+  WorkspaceLayout w{};
+  const size_t P = static_cast<size_t>(T) * L.top_k;
+  w.ksplit = ffn_mma_supported(L) ? ffn_mma_ksplit(L, T) : 1;
+  size_t o = 0;
+  w.ids = o;          o += align_up(P * 4);
+  w.gates = o;        o += align_up(P * 4);
+  w.counts = o;       o += align_up(static_cast<size_t>(L.E) * 4);
+  w.off = o;          o += align_up(static_cast<size_t>(L.E + 1) * 4);
+  w.perm = o;         o += align_up(P * 4);
+  w.slot_of_pair = o; o += align_up(P * 4);
+  w.xs = o;           o += align_up(L.act_bf16 ? P * L.d_model * 2 : 0);
+  w.hidden = o;       o += align_up(P * L.d_ff * (L.act_bf16 ? 2 : 4));
+  w.o_part = o;       o += align_up(static_cast<size_t>(w.ksplit) * P * L.d_model * 4);
+  w.total = o;
+  return w;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace
+
+struct emoe_ctx {
+  int device = 0;
+  char* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  int* check_word = nullptr;        // device
+  int* check_host = nullptr;        // pinned
+  ExpertDev* tables_dev = nullptr;  // [MAX_TABLES][EMOE_MAX_EXPERTS]
+  ExpertDev* tables_pin = nullptr;  // pinned mirror, never rewritten once filled
+  std::vector<TableEntry> tables;
+  int last_cuda = 0;
+  int ffn_path = 0;
+};
+
+namespace {
+
+int cuda_fail(emoe_ctx* ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda = static_cast<int>(e);
+  return EMOE_ERR_CUDA;
+}
+
+#define EMOE_CUDA(ctx, call)                          \
+  do {                                                \
+    cudaError_t e__ = (call);                         \
+    if (e__ != cudaSuccess) return cuda_fail(ctx, e__); \
+  } while (0)
+
+// Device copy of a host expert table; uploaded on `st` the first time its content is seen.
+int get_table(emoe_ctx* ctx, const emoe_expert* host, int E, cudaStream_t st, const ExpertDev** out) {
+  for (size_t i = 0; i < ctx->tables.size(); ++i) {
+    const std::vector<emoe_expert>& h = ctx->tables[i].host;
+    if (static_cast<int>(h.size()) != E) continue;
+    bool same = true;
+    for (int e = 0; e < E && same; ++e) {
+      same = h[e].bits == host[e].bits;
+      for (int m = 0; m < 3 && same; ++m) same = h[e].packed[m] == host[e].packed[m] && h[e].scales[m] == host[e].scales[m];
+    }
+    if (same) {
+      *out = ctx->tables_dev + i * EMOE_MAX_EXPERTS;
+      return EMOE_OK;
+    }
+  }
+  if (ctx->tables.size() >= MAX_TABLES) return EMOE_ERR_WORKSPACE;
+  const size_t slot = ctx->tables.size();
+  ExpertDev* pin = ctx->tables_pin + slot * EMOE_MAX_EXPERTS;
+  for (int e = 0; e < E; ++e) {
+    pin[e].bits = host[e].bits;
+    pin[e].pad = 0;
+    for (int m = 0; m < 3; ++m) {
+      pin[e].packed[m] = static_cast<const uint8_t*>(host[e].packed[m]);
+      pin[e].scales[m] = host[e].scales[m];
+    }
+  }
+  ExpertDev* dev = ctx->tables_dev + slot * EMOE_MAX_EXPERTS;
+  EMOE_CUDA(ctx, cudaMemcpyAsync(dev, pin, sizeof(ExpertDev) * E, cudaMemcpyHostToDevice, st));
+  TableEntry te;
+  te.host.assign(host, host + E);
+  ctx->tables.push_back(std::move(te));
+  *out = dev;
+  return EMOE_OK;
+}
+
+int check_experts(const LayerDims& L, const emoe_expert* host) {
+  const int nmat = L.act == EMOE_ACT_RELU ? 2 : 3;
+  for (int e = 0; e < L.E; ++e) {
+    const int b = host[e].bits;
+    if (b != 2 && b != 4 && b != 8) return EMOE_ERR_UNSUPPORTED;
+    const int wpv = 128 / b;  // weights per 128-bit load
+    if (L.d_model % wpv != 0 || L.d_ff % wpv != 0) return EMOE_ERR_UNSUPPORTED;
+    if (L.group > 0 && L.group % wpv != 0) return EMOE_ERR_UNSUPPORTED;
+    for (int m = 0; m < nmat; ++m) {
+      if (!host[e].packed[m] || !host[e].scales[m]) return EMOE_ERR_INVALID_ARG;
+      if (!aligned(host[e].packed[m], 16)) return EMOE_ERR_ALIGNMENT;
+      if (!aligned(host[e].scales[m], L.scale_f16 ? 2 : 4)) return EMOE_ERR_ALIGNMENT;
+    }
+  }
+  return EMOE_OK;
+}
+
+int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int T, const float* router_W,
+                 const float* router_bias, int bias_token_stride, const int32_t* ids_in, const float* gates_in,
+                 const emoe_expert* host_experts, float* y, int32_t* out_ids, float* out_gates, int32_t* out_perm,
+                 cudaStream_t st) {
+  LayerDims L;
+  if (!ctx || !make_dims(desc, &L)) return EMOE_ERR_INVALID_ARG;
+  if (!x || !y || !host_experts || T <= 0) return EMOE_ERR_INVALID_ARG;
+  const bool routed = ids_in != nullptr;
+  if (routed ? gates_in == nullptr : router_W == nullptr) return EMOE_ERR_INVALID_ARG;
+  if (!routed && router_bias && bias_token_stride != 0 && bias_token_stride != L.E) return EMOE_ERR_INVALID_ARG;
+  if (L.d_model % 32 != 0 || L.d_ff % 32 != 0) return EMOE_ERR_UNSUPPORTED;
+  if (static_cast<long long>(T) * L.top_k > 0x7fffffffLL / 4) return EMOE_ERR_UNSUPPORTED;
+  if (!aligned(x, 16) || !aligned(y, 16)) return EMOE_ERR_ALIGNMENT;
+  int rc = check_experts(L, host_experts);
+  if (rc != EMOE_OK) return rc;
+  const WorkspaceLayout w = make_layout(L, T);
+  if (w.total > ctx->workspace_bytes) return EMOE_ERR_WORKSPACE;
+  EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+
+  const ExpertDev* table = nullptr;
+  rc = get_table(ctx, host_experts, L.E, st, &table);
+  if (rc != EMOE_OK) return rc;
+
+  char* ws = ctx->workspace;
+  const int P = T * L.top_k;
+  int32_t* ids = reinterpret_cast<int32_t*>(ws + w.ids);
+  float* gates = reinterpret_cast<float*>(ws + w.gates);
+  int32_t* counts = reinterpret_cast<int32_t*>(ws + w.counts);
+  int32_t* off = reinterpret_cast<int32_t*>(ws + w.off);
+  int32_t* perm = reinterpret_cast<int32_t*>(ws + w.perm);
+  int32_t* slot_of_pair = reinterpret_cast<int32_t*>(ws + w.slot_of_pair);
+  __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(ws + w.xs);
+  void* hidden = ws + w.hidden;
+  float* o_part = reinterpret_cast<float*>(ws + w.o_part);
+
+  const int32_t* ids_use = ids;
+  const float* gates_use = gates;
+  if (routed) {
+    ids_use = ids_in;
+    gates_use = gates_in;
+  } else {
+    EMOE_CUDA(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,
+                                      L.top_k, L.gate_mode == EMOE_GATE_SOFTMAX_RENORM, ids, gates, nullptr, st));
+  }
+  EMOE_CUDA(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
+
+  const bool use_mma = ffn_mma_supported(L) && ctx->ffn_path != 1;
+  if (ctx->ffn_path == 2 && !use_mma) return EMOE_ERR_UNSUPPORTED;
+  int ksplit = 1;
+  if (use_mma) {
+    ksplit = w.ksplit;
+    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, xs, P, st));
+    EMOE_CUDA(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
+    EMOE_CUDA(ctx, launch_ffn_mma(1, L, table, reinterpret_cast<const __nv_bfloat16*>(hidden), off,
+                                  reinterpret_cast<__nv_bfloat16*>(hidden), o_part, ksplit, P, T, st));
+  } else {
+    EMOE_CUDA(ctx, launch_ffn_gemv(0, L, table, x, perm, off, hidden, o_part, P, st));
+    EMOE_CUDA(ctx, launch_ffn_gemv(1, L, table, x, perm, off, hidden, o_part, P, st));
+  }
+  EMOE_CUDA(ctx, launch_combine(o_part, ksplit, static_cast<size_t>(P), gates_use, slot_of_pair, T, L.top_k, L.d_model,
+                                y, st));
+  if (out_ids) EMOE_CUDA(ctx, cudaMemcpyAsync(out_ids, ids_use, sizeof(int32_t) * P, cudaMemcpyDeviceToDevice, st));
+  if (out_gates) EMOE_CUDA(ctx, cudaMemcpyAsync(out_gates, gates_use, sizeof(float) * P, cudaMemcpyDeviceToDevice, st));
+  if (out_perm) EMOE_CUDA(ctx, cudaMemcpyAsync(out_perm, perm, sizeof(int32_t) * P, cudaMemcpyDeviceToDevice, st));
+  return EMOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+emoe_ctx* emoe_create(int device, size_t workspace_bytes, int* status) {
+  int dummy;
+  if (!status) status = &dummy;
+  *status = EMOE_OK;
+  emoe_ctx* ctx = new (std::nothrow) emoe_ctx();
+  if (!ctx) {
+    *status = EMOE_ERR_INVALID_ARG;
+    return nullptr;
+  }
+  ctx->device = device;
+  cudaError_t e = cudaSetDevice(device);
+  if (e == cudaSuccess && workspace_bytes > 0) e = cudaMalloc(&ctx->workspace, workspace_bytes);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->check_word, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(ctx->check_word, 0, sizeof(int));
+  if (e == cudaSuccess) e = cudaMallocHost(&ctx->check_host, sizeof(int));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->tables_dev, sizeof(ExpertDev) * MAX_TABLES * EMOE_MAX_EXPERTS);
+  if (e == cudaSuccess) e = cudaMallocHost(&ctx->tables_pin, sizeof(ExpertDev) * MAX_TABLES * EMOE_MAX_EXPERTS);
+  if (e != cudaSuccess) {
+    *status = EMOE_ERR_CUDA;
+    ctx->last_cuda = static_cast<int>(e);
+    emoe_destroy(ctx);
+    return nullptr;
+  }
+  ctx->workspace_bytes = workspace_bytes;
+  return ctx;
+}
+
+int emoe_destroy(emoe_ctx* ctx) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  if (ctx->workspace) cudaFree(ctx->workspace);
+  if (ctx->check_word) cudaFree(ctx->check_word);
+  if (ctx->check_host) cudaFreeHost(ctx->check_host);
+  if (ctx->tables_dev) cudaFree(ctx->tables_dev);
+  if (ctx->tables_pin) cudaFreeHost(ctx->tables_pin);
+  delete ctx;
+  return EMOE_OK;
+}
+
+size_t emoe_workspace_bytes(const emoe_layer_desc* desc, int T) {
+  LayerDims L;
+  if (!make_dims(desc, &L) || T <= 0) return 0;
+  return make_layout(L, T).total;
+}
+
+int emoe_last_cuda_error(const emoe_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int emoe_device_status(emoe_ctx* ctx, void* stream) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+  EMOE_CUDA(ctx, cudaMemcpyAsync(ctx->check_host, ctx->check_word, sizeof(int), cudaMemcpyDeviceToHost, st));
+  EMOE_CUDA(ctx, cudaMemsetAsync(ctx->check_word, 0, sizeof(int), st));
+  EMOE_CUDA(ctx, cudaStreamSynchronize(st));
+  return *ctx->check_host ? EMOE_ERR_DEVICE_CHECK : EMOE_OK;
+}
+
+const char* emoe_status_string(int status) {
+  switch (status) {
+    case EMOE_OK: return "ok";
+    case EMOE_ERR_INVALID_ARG: return "invalid argument";
+    case EMOE_ERR_UNSUPPORTED: return "unsupported bitwidth, enum value or shape";
+    case EMOE_ERR_ALIGNMENT: return "pointer or row size not sufficiently aligned";
+    case EMOE_ERR_WORKSPACE: return "context workspace (or expert-table cache) too small";
+    case EMOE_ERR_CUDA: return "CUDA call failed (see emoe_last_cuda_error)";
+    case EMOE_ERR_DEVICE_CHECK: return "a kernel found inconsistent data";
+    default: return "unknown status";
+  }
+}
+
+size_t emoe_packed_bytes(int N, int K, int bits) {
+  if (N <= 0 || K <= 0 || (bits != 2 && bits != 4 && bits != 8)) return 0;
+  if ((static_cast<long long>(K) * bits) % 8 != 0) return 0;
+  return static_cast<size_t>(N) * (static_cast<size_t>(K) * bits / 8);
+}
+
+size_t emoe_scales_bytes(int N, int K, int group, int scale_dtype) {
+  if (N <= 0 || K <= 0 || group < 0) return 0;
+  if (scale_dtype != EMOE_DTYPE_F32 && scale_dtype != EMOE_DTYPE_F16) return 0;
+  const int G = group > 0 ? group : K;
+  if (K % G != 0) return 0;
+  return static_cast<size_t>(N) * (K / G) * (scale_dtype == EMOE_DTYPE_F16 ? 2 : 4);
+}
+
+int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int group, int scale_dtype,
+                     void* out_packed, void* out_scales, void* stream) {
+  if (!ctx || !W || !out_packed || !out_scales || N <= 0 || K <= 0 || group < 0) return EMOE_ERR_INVALID_ARG;
+  if (bits != 2 && bits != 4 && bits != 8) return EMOE_ERR_UNSUPPORTED;
+  if (scale_dtype != EMOE_DTYPE_F32 && scale_dtype != EMOE_DTYPE_F16) return EMOE_ERR_UNSUPPORTED;
+  const int G = group > 0 ? group : K;
+  if (K % G != 0) return EMOE_ERR_INVALID_ARG;
+  if ((static_cast<long long>(G) * bits) % 32 != 0 || G % 4 != 0) return EMOE_ERR_UNSUPPORTED;
+  if (!aligned(W, 16) || !aligned(out_packed, 16) || !aligned(out_scales, 4)) return EMOE_ERR_ALIGNMENT;
+  EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+  EMOE_CUDA(ctx, launch_pack(W, N, K, bits, group, scale_dtype == EMOE_DTYPE_F16, static_cast<uint8_t*>(out_packed),
+                             out_scales, static_cast<cudaStream_t>(stream)));
+  return EMOE_OK;
+}
+
+int emoe_router_topk(emoe_ctx* ctx, const void* x, int act_dtype, int T, int d, const float* router_W,
+                     const float* router_bias, int bias_token_stride, int E, int top_k, int gate_mode,
+                     int32_t* out_ids, float* out_gates, float* out_logits, void* stream) {
+  if (!ctx || !x || !router_W || !out_ids || !out_gates || T <= 0 || d <= 0) return EMOE_ERR_INVALID_ARG;
+  if (E < 1 || E > EMOE_MAX_EXPERTS || top_k < 1 || top_k > E || top_k > EMOE_MAX_TOP_K) return EMOE_ERR_INVALID_ARG;
+  if (act_dtype != EMOE_DTYPE_F32 && act_dtype != EMOE_DTYPE_BF16) return EMOE_ERR_UNSUPPORTED;
+  if (gate_mode != EMOE_GATE_SOFTMAX && gate_mode != EMOE_GATE_SOFTMAX_RENORM) return EMOE_ERR_UNSUPPORTED;
+  if (router_bias && bias_token_stride != 0 && bias_token_stride != E) return EMOE_ERR_INVALID_ARG;
+  EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+  EMOE_CUDA(ctx, launch_router_topk(x, act_dtype == EMOE_DTYPE_BF16, T, d, router_W, router_bias, bias_token_stride, E,
+                                    top_k, gate_mode == EMOE_GATE_SOFTMAX_RENORM, out_ids, out_gates, out_logits,
+                                    static_cast<cudaStream_t>(stream)));
+  return EMOE_OK;
+}
+
+int emoe_permute(emoe_ctx* ctx, const int32_t* ids, int n_pairs, int E, int32_t* out_counts, int32_t* out_off,
+                 int32_t* out_perm, int32_t* out_slot_of_pair, void* stream) {
+  if (!ctx || !ids || !out_counts || !out_off || !out_perm || n_pairs <= 0) return EMOE_ERR_INVALID_ARG;
+  if (E < 1 || E > EMOE_MAX_EXPERTS) return EMOE_ERR_INVALID_ARG;
+  EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+  EMOE_CUDA(ctx, launch_permute(ids, n_pairs, E, out_counts, out_off, out_perm, out_slot_of_pair, ctx->check_word,
+                                static_cast<cudaStream_t>(stream)));
+  return EMOE_OK;
+}
+
+int emoe_moe_forward(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int T, const float* router_W,
+                     const float* router_bias, int bias_token_stride, const emoe_expert* host_experts, float* y,
+                     int32_t* out_ids, float* out_gates, int32_t* out_perm, void* stream) {
+  if (!router_W) return EMOE_ERR_INVALID_ARG;
+  return forward_impl(ctx, desc, x, T, router_W, router_bias, bias_token_stride, nullptr, nullptr, host_experts, y,
+                      out_ids, out_gates, out_perm, static_cast<cudaStream_t>(stream));
+}
+
+int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int T, const int32_t* ids,
+                            const float* gates, const emoe_expert* host_experts, float* y, int32_t* out_perm,
+                            void* stream) {
+  if (!ids || !gates) return EMOE_ERR_INVALID_ARG;
+  return forward_impl(ctx, desc, x, T, nullptr, nullptr, 0, ids, gates, host_experts, y, nullptr, nullptr, out_perm,
+                      static_cast<cudaStream_t>(stream));
+}
+
+int emoe_set_ffn_path(emoe_ctx* ctx, int path) {
+  if (!ctx || path < 0 || path > 2) return EMOE_ERR_INVALID_ARG;
+  ctx->ffn_path = path;
+  return EMOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,64 @@
+// Internal declarations shared by the .cu files of libemoe (not part of the ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/emoe.h"
+
+namespace emoe {
+
+// Device copy of one layer's expert table (one entry per expert).
+struct ExpertDev {
+  int32_t bits;
+  int32_t pad;
+  const uint8_t* packed[3];
+  const void* scales[3];
+};
+
+// Bits of the device-side check word.
+enum : int {
+  CHECK_BAD_EXPERT_ID = 1,
+};
+
+struct LayerDims {
+  int d_model, d_ff, E, top_k, act, gate_mode, group, scale_f16, act_bf16;
+};
+
+// ---- launchers (each enqueues on `st` and returns the launch error) ---------------------
+cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int scale_f16, uint8_t* packed,
+                        void* scales, cudaStream_t st);
+
+cudaError_t launch_router_topk(const void* x, int x_bf16, int T, int d, const float* Wr, const float* bias,
+                               int bias_stride, int E, int top_k, int renorm, int32_t* ids, float* gates,
+                               float* logits, cudaStream_t st);
+
+cudaError_t launch_permute(const int32_t* ids, int n_pairs, int E, int32_t* counts, int32_t* off, int32_t* perm,
+                           int32_t* slot_of_pair, int* check_word, cudaStream_t st);
+
+// Generic CUDA-core grouped GEMV.
+//   phase 0: hidden[slot][f] = act(x[token(slot)] . W~first)      (x gathered through perm)
+//   phase 1: o[slot][d]      = hidden[slot] . W~last
+// hidden is fp32 (act_bf16 = 0) or bf16 (act_bf16 = 1).
+cudaError_t launch_ffn_gemv(int phase, const LayerDims& L, const ExpertDev* experts, const void* x,
+                            const int32_t* perm, const int32_t* off, void* hidden, float* o, int n_pairs,
+                            cudaStream_t st);
+
+// Tensor-core (mma.sync bf16) grouped kernel for bf16 activations.
+// xs: x rows scattered into expert order with the per-bitwidth k-interleave, [n_pairs][d_model] bf16.
+// hidden: same interleave, [n_pairs][d_ff] bf16.  o_part: [ksplit][n_pairs][d_model] fp32.
+bool ffn_mma_supported(const LayerDims& L);
+int ffn_mma_ksplit(const LayerDims& L, int T);
+cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
+                             const int32_t* perm, __nv_bfloat16* xs, int n_pairs, cudaStream_t st);
+cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
+                           const int32_t* off, __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs,
+                           int T, cudaStream_t st);
+
+// y[t] = sum_j gates[t][j] * sum_z o_part[z][slot_of_pair[t*k+j]]
+// o_part holds ksplit partial results, each [n_pairs_stride][d].
+cudaError_t launch_combine(const float* o_part, int ksplit, size_t n_pairs_stride, const float* gates,
+                           const int32_t* slot_of_pair, int T, int top_k, int d, float* y, cudaStream_t st);
+
+}  // namespace emoe

@@ -1,0 +1,143 @@
+"""GPU parity: the whole layer (emoe_moe_forward / emoe_moe_forward_routed) against the CPU
+checker through the C ABI, on small layers that still span several tiles and ragged tails.
+Bars: permutation bit-exact; ids exact outside the 1e-4 logit margin; outputs within
+max|y - y_ref| / max|y_ref| <= 2e-3 (bf16 activations) or 1e-5 (fp32 activations).  The
+reference is always evaluated with the ids the GPU picked, so a legal tie-break difference
+does not leak into the output comparison."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2308_14352_b200 import binding as B, inputs, layer
+from tests.helpers import check_ids, oracle_pack_layer, output_tolerance, rel_to_max
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_case(shape, bits, T, seed, path, bias=None, std=0.02, max_tokens=None):
+    W = inputs.expert_set(seed, 0, shape, std)
+    x = inputs.activations(seed, 0, T, shape.d_model, shape.act_dtype)
+    Wr = inputs.router_weight(seed, 0, shape.d_model, shape.n_experts, std=0.05)
+    packed, scales = oracle_pack_layer(W, shape, bits)
+    with layer.MoELayer(shape, bits, max_tokens=max_tokens or T) as moe:
+        B.emoe_set_ffn_path(moe.ctx, path)
+        moe.pack_from_host(W)
+        for e in range(shape.n_experts):          # packed bytes and scales are bit-exact
+            for m in range(shape.n_matrices):
+                assert np.array_equal(moe.packed_host(e, m), packed[e][m])
+                assert np.array_equal(moe.scales_host(e, m).astype(np.float32), scales[e][m])
+        y, ids, gates, perm = moe.forward(x, Wr, bias)
+    renorm = shape.gate_mode == "softmax_renorm"
+    ids_ref, gates_ref, logits_ref = oracle.route(x, Wr, bias, shape.top_k, renorm)
+    check_ids(ids, logits_ref, shape.top_k)
+    same = np.all(ids == ids_ref, axis=1)
+    np.testing.assert_allclose(gates[same], gates_ref[same], rtol=2e-5, atol=1e-7)
+    _, _, perm_ref = oracle.permute(ids, shape.n_experts)
+    assert np.array_equal(perm, perm_ref)
+    y_ref = oracle.moe_ffn_combine(x, shape.d_ff, shape.act, shape.group, shape.act_dtype == "bf16", bits, packed,
+                                   scales, ids, gates)
+    err = rel_to_max(y, y_ref)
+    assert err <= output_tolerance(shape.act_dtype), err
+    return err
+
+
+GEMV_CASES = [
+    # act, act_dtype, group, scale_dtype, d, f, E, k, gate, bits, T
+    ("relu", "f32", 0, "f32", 128, 256, 4, 1, "softmax", [8, 4, 2, 4], 9),
+    ("relu", "f32", 64, "f32", 192, 320, 3, 2, "softmax_renorm", [2, 8, 4], 7),
+    ("swiglu", "f32", 0, "f16", 256, 448, 4, 2, "softmax_renorm", [4, 2, 8, 4], 11),
+    ("relu", "bf16", 32, "f16", 64, 160, 5, 1, "softmax", [8, 8, 4, 4, 8], 13),     # shapes the MMA path refuses
+    ("swiglu", "bf16", 64, "f16", 192, 320, 2, 2, "softmax", [4, 2], 5),
+    ("relu", "bf16", 128, "f16", 256, 512, 4, 1, "softmax", [2, 4, 8, 4], 10),
+]
+
+
+@pytest.mark.parametrize("act,adt,group,sdt,d,f,E,k,gate,bits,T", GEMV_CASES)
+def test_forward_cuda_core_path(act, adt, group, sdt, d, f, E, k, gate, bits, T):
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, adt)
+    _run_case(shape, bits, T, seed=21, path=1)
+
+
+MMA_CASES = [
+    ("relu", 128, "f16", 256, 512, 4, 1, "softmax", [2, 4, 8, 4], 10),
+    ("relu", 128, "f16", 768, 3072, 8, 1, "softmax", [8, 4, 2, 4, 8, 2, 4, 8], 64),
+    ("relu", 0, "f16", 384, 640, 4, 2, "softmax_renorm", [4, 2, 8, 2], 19),        # per-channel scales, ragged row tiles
+    ("relu", 128, "f32", 256, 1152, 3, 1, "softmax", [8, 2, 4], 37),                # 37 tokens: two 32-token passes possible
+    ("swiglu", 128, "f16", 512, 1408, 4, 2, "softmax_renorm", [4, 8, 2, 4], 16),
+    ("swiglu", 256, "f16", 1024, 2560, 8, 2, "softmax_renorm", [4, 4, 8, 2, 4, 8, 2, 4], 33),
+    ("swiglu", 128, "f16", 128, 128, 2, 2, "softmax", [2, 8], 1),
+    ("relu", 128, "f16", 128, 4224, 2, 1, "softmax", [4, 2], 3),                    # long K in the second projection: split-K
+]
+
+
+@pytest.mark.parametrize("act,group,sdt,d,f,E,k,gate,bits,T", MMA_CASES)
+def test_forward_tensor_core_path(act, group, sdt, d, f, E, k, gate, bits, T):
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, "bf16")
+    _run_case(shape, bits, T, seed=22, path=2)
+
+
+def test_both_paths_agree_and_default_picks_tensor_cores():
+    shape = inputs.LayerShape(256, 512, 4, 2, "swiglu", "softmax_renorm", 128, "f16", "bf16")
+    e_auto = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=0)
+    e_gemv = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=1)
+    e_mma = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=2)
+    assert e_auto == e_mma and e_gemv <= 2e-3
+
+
+def test_zipf_bias_and_many_tokens_on_one_expert():
+    """All tokens of a batch on one expert (several token passes) plus idle experts."""
+    shape = inputs.LayerShape(256, 512, 8, 1, "relu", "softmax", 128, "f16", "bf16")
+    bias = np.full(8, -30.0, dtype=np.float32)
+    bias[5] = 30.0
+    for path in (1, 2):
+        _run_case(shape, [2, 4, 8, 4, 2, 4, 8, 2], 70, seed=24, path=path, bias=bias)
+
+
+def test_forward_routed_and_unselected_experts():
+    shape = inputs.LayerShape(256, 384, 4, 2, "relu", "softmax", 128, "f16", "bf16")
+    bits = [4, 2, 8, 4]
+    W = inputs.expert_set(30, 0, shape)
+    x = inputs.activations(30, 0, 6, shape.d_model, "bf16")
+    ids = np.array([[0, 2], [2, 0], [0, 2], [2, 0], [0, 2], [2, 0]], dtype=np.int32)
+    gates = np.random.default_rng(0).random((6, 2)).astype(np.float32)
+    packed, scales = oracle_pack_layer(W, shape, bits)
+    y_ref = oracle.moe_ffn_combine(x, shape.d_ff, "relu", 128, True, bits, packed, scales, ids, gates)
+    for path in (1, 2):
+        with layer.MoELayer(shape, bits, max_tokens=6) as moe:
+            B.emoe_set_ffn_path(moe.ctx, path)
+            moe.pack_from_host(W)
+            y, perm = moe.forward_routed(x, ids, gates)
+            assert np.array_equal(perm, oracle.permute(ids, 4)[2])
+            assert rel_to_max(y, y_ref) <= 2e-3
+            # experts 1 and 3 are never selected: overwriting their weights changes nothing
+            moe.packed[1][0].fill_(0x5A)
+            moe.scales[3][1].fill_(3.0)
+            y2, _ = moe.forward_routed(x, ids, gates)
+            assert np.array_equal(y, y2)
+            # two runs are bit-identical
+            y3, _ = moe.forward_routed(x, ids, gates)
+            assert np.array_equal(y2, y3)
+
+
+def test_forward_argument_errors():
+    shape = inputs.LayerShape(256, 384, 4, 2, "relu", "softmax", 128, "f16", "bf16")
+    lib = B.lib()
+    with layer.MoELayer(shape, [4, 2, 8, 4], max_tokens=4) as moe:
+        x = torch.zeros(8, 256, dtype=torch.bfloat16, device="cuda")
+        Wr = torch.zeros(256, 4, device="cuda")
+        y = torch.zeros(8, 256, device="cuda")
+        import ctypes
+        fwd = lambda desc, T, tab, xp=x.data_ptr(): lib.emoe_moe_forward(
+            moe.ctx, ctypes.byref(desc), xp, T, Wr.data_ptr(), None, 0, tab, y.data_ptr(), None, None, None, None)
+        assert fwd(moe.desc, 8, moe.table) == B.ERR_WORKSPACE          # context sized for 4 tokens
+        assert fwd(moe.desc, 0, moe.table) == B.ERR_INVALID_ARG
+        assert fwd(moe.desc, 4, moe.table, x.data_ptr() + 2) == B.ERR_ALIGNMENT
+        bad = layer.make_desc(shape)
+        bad.top_k = 5
+        assert fwd(bad, 4, moe.table) == B.ERR_INVALID_ARG
+        tab = B.make_expert_table([(3, [t.data_ptr() for t in moe.packed[e]], [t.data_ptr() for t in moe.scales[e]])
+                                   for e in range(4)])
+        assert fwd(moe.desc, 4, tab) == B.ERR_UNSUPPORTED
+        assert fwd(moe.desc, 4, moe.table) == B.OK
+        torch.cuda.synchronize()
