@@ -1,0 +1,450 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse-MoE layer forward on mixed-bitwidth packed experts.
+
+One step = one forward pass of every MoE layer of the workload over one batch of tokens
+(router -> Top-K -> permutation -> expert FFNs on packed weights -> combine), each layer with
+its own seeded input batch.  Prints ONE JSON line (see --help for the arms).
+
+    python bench.py                                  # switch_base_decode, 64 tokens, 1 GPU
+    python bench.py --workload mixtral_decode --tokens 32
+    python bench.py --impl reference                 # the CPU checker timed on the host cores
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   # N replicas
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2308_14352_b200 import inputs  # noqa: E402
+
+METRIC = "MoE-layer tokens/s"
+UNIT = "tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="emoe", choices=["emoe", "reference"])
+    ap.add_argument("--workload", default="switch_base_decode", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--tokens", type=int, default=0, help="batch size (default: the workload's largest)")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
+    ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying a CUDA graph")
+    ap.add_argument("--ffn-path", type=int, default=0, help="0 auto, 1 CUDA-core GEMV, 2 tensor-core path")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(n_gpus: int):
+    """(rank, world, local_rank) and an initialised process group when launched by torchrun."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        if backend == "nccl":
+            torch.cuda.set_device(local)
+        dist.init_process_group(backend=backend)
+    return rank, world, local
+
+
+def reduce_max_and_sum(ms: float, units: float, world: int, device=None):
+    """Replicas only: the step time of the job is the max over ranks, its work the sum."""
+    if world <= 1:
+        return ms, units
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.barrier()
+
+
+def config_dict(w: inputs.Workload, T: int, n_layers: int, world: int, graph: bool):
+    sh = w.shape
+    return {
+        "workload": f"{w.name} T={T}",
+        "layers": n_layers, "tokens_per_step": T, "d_model": sh.d_model, "d_ff": sh.d_ff, "experts": sh.n_experts,
+        "top_k": sh.top_k, "act": sh.act, "bits": "per-expert INT2/4/8 (" + w.bits_rule + ")",
+        "scales": f"group-{sh.group or 'channel'} {sh.scale_dtype}", "activations": sh.act_dtype,
+        "tokens_counted": "tokens x layers per step (every layer forwards the whole batch)",
+        "l2": "each step streams the packed experts of all layers (larger than the 126 MB L2), nothing is flushed by hand",
+        "launch": "cuda-graph replay of the forward calls" if graph else "direct launches",
+        "parallelism": f"replicas x{world}",
+    }
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU checker, as it stands, on the host cores
+# ------------------------------------------------------------------------------------------------
+def oracle_layers(w: inputs.Workload, T: int, n_layers: int):
+    import oracle
+
+    sh = w.shape
+    layers = []
+    for l in range(n_layers):
+        bits = inputs.expert_bits(w, l)
+        x, Wr, bias = inputs.layer_tensors(w, l, T)
+        ids, gates, _ = oracle.route(x, Wr, bias, sh.top_k, sh.gate_mode == "softmax_renorm")
+        active = sorted(set(ids.reshape(-1).tolist()))
+        packed = [[None] * sh.n_matrices for _ in range(sh.n_experts)]
+        scales = [[None] * sh.n_matrices for _ in range(sh.n_experts)]
+        dummy_p, dummy_s = np.zeros((1, 16), np.uint8), np.zeros((1, 1), np.float32)
+        for e in range(sh.n_experts):
+            for m in range(sh.n_matrices):
+                if e in active:   # experts that are never activated are never read: skip generating them
+                    N, K = sh.matrix_shape(m)
+                    packed[e][m], scales[e][m] = oracle.pack_expert(
+                        inputs.expert_matrix(w.seed, l, e, m, N, K), bits[e], sh.group, sh.scale_dtype)
+                else:
+                    packed[e][m], scales[e][m] = dummy_p, dummy_s
+        layers.append((bits, x, Wr, bias, packed, scales))
+    return layers
+
+
+def time_oracle(w: inputs.Workload, T: int, n_layers: int, steps: int, warmup: int):
+    import oracle
+
+    sh = w.shape
+    layers = oracle_layers(w, T, n_layers)
+
+    def step():
+        for bits, x, Wr, bias, packed, scales in layers:
+            oracle.moe_forward(x, Wr, bias, sh.top_k, sh.gate_mode == "softmax_renorm", sh.d_ff, sh.act, sh.group,
+                               sh.act_dtype == "bf16", bits, packed, scales)
+
+    for _ in range(warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    return dt, oracle.num_threads()
+
+
+def run_reference(args, w, T, n_layers, rank, world):
+    if rank != 0:
+        return
+    # bounded sample: as many layers as keep one step near a second of CPU time
+    sample_layers = min(n_layers, 2 if w.shape.d_model <= 1024 else 1)
+    sample_T = T if w.shape.d_model <= 1024 else 1
+    steps = max(1, min(args.steps, 5))
+    warmup = max(0, min(args.warmup, 1))
+    dt, threads = time_oracle(w, sample_T, sample_layers, steps, warmup)
+    value = sample_T * sample_layers / dt
+    sample = f"{sample_layers} of {n_layers} layers at T={sample_T}, {steps} timed passes"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": config_dict(w, T, n_layers, 1, False),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------------
+def run_emoe(args, w, T, n_layers, rank, world, local):
+    import torch
+
+    from paper_2308_14352_b200 import binding as B, layer as L
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device for --impl emoe (there is no CPU path)")
+    B.lib()
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    sh = w.shape
+    desc = L.make_desc(sh)
+    ctx = B.emoe_create(local, B.emoe_workspace_bytes(desc, T))
+    B.emoe_set_ffn_path(ctx, args.ffn_path)
+
+    # ---- build the stack: seeded fp32 experts -> packed on the device by the library ------------
+    t_build = time.perf_counter()
+    layers, xs, Wrs, biases, ys = [], [], [], [], []
+    pack_bytes_in = 0
+    pack_ms = 0.0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    from concurrent.futures import ThreadPoolExecutor
+
+    pool = ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1))
+    for l in range(n_layers):
+        bits = inputs.expert_bits(w, l)
+        moe = L.MoELayer(sh, bits, device=local, max_tokens=T, ctx=ctx)
+        jobs = [(e, m) + sh.matrix_shape(m) for e in range(sh.n_experts) for m in range(sh.n_matrices)]
+        mats = pool.map(lambda j: inputs.expert_matrix(w.seed, l, j[0], j[1], j[2], j[3]), jobs)
+        for (e, m, N, K), Wh in zip(jobs, mats):
+            Wd = torch.from_numpy(Wh).to(dev)
+            ev0.record()
+            moe.pack_matrix(e, m, Wd)
+            ev1.record()
+            ev1.synchronize()
+            pack_ms += ev0.elapsed_time(ev1)
+            pack_bytes_in += N * K * 4
+            del Wd, Wh
+        x, Wr, bias = inputs.layer_tensors(w, l, T)
+        layers.append(moe)
+        xs.append(moe.to_device_x(x))
+        Wrs.append(torch.from_numpy(Wr).to(dev))
+        biases.append(None if bias is None else torch.from_numpy(bias).to(dev))
+        ys.append(torch.zeros(T, sh.d_model, dtype=torch.float32, device=dev))
+    torch.cuda.synchronize()
+    build_s = time.perf_counter() - t_build
+
+    ids_dev = [torch.zeros(T, sh.top_k, dtype=torch.int32, device=dev) for _ in range(n_layers)]
+    stream = torch.cuda.Stream(device=dev)
+
+    def forward_all(st, want_ids=False):
+        for l, moe in enumerate(layers):
+            moe.forward_device(xs[l], Wrs[l], biases[l], ys[l], ids_dev[l] if want_ids else None, None, None, st)
+
+    # first pass: uploads the expert tables, gives the routing decisions for the byte count
+    with torch.cuda.stream(stream):
+        forward_all(stream.cuda_stream, want_ids=True)
+    stream.synchronize()
+    if B.emoe_device_status(ctx, stream.cuda_stream) != B.OK:
+        raise RuntimeError("device-side check failed")
+
+    # algorithmic bytes: packed codes + scales of the distinct activated experts of every layer
+    scale_sz = 2 if sh.scale_dtype == "f16" else 4
+    expert_bytes_per_step = 0
+    for l, moe in enumerate(layers):
+        for e in set(ids_dev[l].cpu().numpy().reshape(-1).tolist()):
+            for m in range(sh.n_matrices):
+                N, K = sh.matrix_shape(m)
+                G = sh.group or K
+                expert_bytes_per_step += N * K * moe.bits[e] // 8 + N * (K // G) * scale_sz
+
+    use_graph = not args.no_graph
+    graph = None
+    if use_graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            forward_all(stream.cuda_stream)
+
+    def step():
+        if graph is not None:
+            graph.replay()
+        else:
+            forward_all(stream.cuda_stream)
+
+    kernels_per_layer = 6  # router+top-k, permute, scatter, two expert-FFN launches, combine
+    launches_per_step = kernels_per_layer * n_layers
+
+    # ---- device-resident timing ----------------------------------------------------------------
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step()
+        stream.synchronize()
+        barrier(world)
+        sampler = ClockSampler(local)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier(world)
+        clocks = sampler.stop()
+    ms_step = e0.elapsed_time(e1) / args.steps
+
+    # ---- the expert-FFN kernels alone, by CUDA events on the launching stream -------------------
+    B.emoe_set_timing(ctx, True)
+    with torch.cuda.stream(stream):
+        for _ in range(min(args.steps, 20)):
+            forward_all(stream.cuda_stream)
+        stream.synchronize()
+    ffn0_ms, ffn1_ms, calls = B.emoe_read_timing(ctx)
+    B.emoe_set_timing(ctx, False)
+    ffn_ms_per_step = (ffn0_ms + ffn1_ms) / calls * n_layers
+    peak, peak_kind = load_peaks()
+    achieved = expert_bytes_per_step / (ffn_ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the C ABI from host buffers ----------------------------------------
+    x_host = [torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in xs]
+    for h, d in zip(x_host, xs):
+        h.copy_(d.cpu())
+    y_host = [torch.empty(T, sh.d_model, dtype=torch.float32).pin_memory() for _ in range(n_layers)]
+    x_stage = [torch.empty_like(x) for x in xs]
+
+    def e2e_step():
+        for l, moe in enumerate(layers):
+            x_stage[l].copy_(x_host[l], non_blocking=True)
+            moe.forward_device(x_stage[l], Wrs[l], biases[l], ys[l], None, None, None, stream.cuda_stream)
+            y_host[l].copy_(ys[l], non_blocking=True)
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            e2e_step()
+        stream.synchronize()
+        barrier(world)
+        t0 = time.perf_counter()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record(stream)
+        for _ in range(args.steps):
+            e2e_step()
+        f1.record(stream)
+        stream.synchronize()
+        e2e_wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    e2e_ms = max(f0.elapsed_time(f1) / args.steps, e2e_wall_ms)
+    h2d = sum(x.numel() * x.element_size() for x in xs)
+    d2h = sum(y.numel() * y.element_size() for y in ys)
+
+    units = float(T * n_layers)
+    ms_job, units_job = reduce_max_and_sum(ms_step, units, world, dev)
+    e2e_job, _ = reduce_max_and_sum(e2e_ms, units, world, dev)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample_layers = min(n_layers, 2 if sh.d_model <= 1024 else 1)
+        sample_T = T if sh.d_model <= 1024 else 1
+        dt, threads = time_oracle(w, sample_T, sample_layers, 3, 1)
+        cpu = {"value": sample_T * sample_layers / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"{sample_layers} of {n_layers} layers at T={sample_T}, 3 timed passes"}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": units_job / (ms_job * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_job, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if sh.act_dtype == "bf16" else "f32", "data": "synthetic",
+            "config": config_dict(w, T, n_layers, world, use_graph),
+            "clocks": clocks,
+            "e2e": {"value": units_job / (e2e_job * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_job},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": {
+                "kernel": "expert-FFN kernels (both projections of every layer)", "bound": "hbm",
+                "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_8TBs": achieved / 8000.0, "traffic": None,
+                "algorithmic_bytes_per_step": expert_bytes_per_step, "kernel_ms_per_step": ffn_ms_per_step,
+                "first_projection_ms": ffn0_ms / calls * n_layers, "second_projection_ms": ffn1_ms / calls * n_layers,
+            },
+            "whole_step_gbs": expert_bytes_per_step / (ms_job * 1e-3) / 1e9,
+            "pack": {"gbs_fp32_in": pack_bytes_in / (pack_ms * 1e-3) / 1e9, "ms_total": pack_ms,
+                     "note": "expert quantise+pack kernel, fp32 bytes read per second, timed per matrix while building the stack"},
+            "build_seconds": build_s,
+        }
+        if cpu is not None:
+            out["cpu_baseline"] = cpu
+        print(json.dumps(out))
+    for moe in layers:
+        moe.close()
+    torch.cuda.synchronize()
+    B.emoe_destroy(ctx)
+
+
+def main():
+    args = parse_args()
+    w = inputs.WORKLOADS[args.workload]
+    T = args.tokens or max(t for t in w.tokens if t <= 64)
+    n_layers = args.layers or w.n_layers
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        run_reference(args, w, T, n_layers, rank, int(os.environ.get("WORLD_SIZE", "1")))
+        return
+    rank, world, local = dist_setup(args.gpus)
+    try:
+        run_emoe(args, w, T, n_layers, rank, world, local)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

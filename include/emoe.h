@@ -123,7 +123,8 @@ size_t emoe_scales_bytes(int N, int K, int group, int scale_dtype); /* N*(K/grou
 
 /* Quantises and packs one matrix W[N][K] (fp32, row-major, rows = output channels) to
  * `bits` in the storage format described at the top of this file.
- *   group: 0 or a multiple of 4 that divides K;  K*bits must be a multiple of 32.
+ *   group: 0 or a divisor of K; the scale run (group, or K when group = 0) must be a multiple
+ *   of 4 inputs and of 32 bits of codes (so 16 / 8 / 4 inputs at 2 / 4 / 8 bits).
  *   out_packed: emoe_packed_bytes(N,K,bits) bytes; out_scales: emoe_scales_bytes(...).
  *   W and out_packed must be 16-byte aligned, out_scales 4-byte aligned.
  * Bit-exact with the definition: IEEE division and round-half-even, no fast-math. */
@@ -184,6 +185,15 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
  * grouped GEMV, 2 = force the tensor-core path where the shape allows it.  For tests and
  * measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);
+
+/* Measurement aid (Section 4 of the paper times compute and loading separately; here the
+ * expert-FFN kernels are the part bound by weight streaming).  While enabled, every forward
+ * call records CUDA events on its stream around the first-projection and second-projection
+ * expert kernels.  emoe_read_timing waits for the recorded events, returns the summed device
+ * time of each projection (milliseconds) and the number of forward calls covered, and clears
+ * the record.  Off by default; not for use during stream capture. */
+int emoe_set_timing(emoe_ctx* ctx, int enabled);
+int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, int* out_calls);
 
 #ifdef __cplusplus
 }

@@ -28,7 +28,8 @@ GATE_SOFTMAX, GATE_SOFTMAX_RENORM = 0, 1
 EXPORTS = (
     "emoe_create", "emoe_destroy", "emoe_workspace_bytes", "emoe_last_cuda_error", "emoe_device_status",
     "emoe_status_string", "emoe_packed_bytes", "emoe_scales_bytes", "emoe_pack_expert", "emoe_router_topk",
-    "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path",
+    "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
+    "emoe_read_timing",
 )
 
 
@@ -82,6 +83,9 @@ def lib() -> ctypes.CDLL:
         L.emoe_moe_forward_routed.argtypes = [vp, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
                                               ctypes.POINTER(emoe_expert), vp, vp, vp]
         L.emoe_set_ffn_path.argtypes = [vp, i32]
+        L.emoe_set_timing.argtypes = [vp, i32]
+        L.emoe_read_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                       ctypes.POINTER(ctypes.c_int)]
         _lib = L
     return _lib
 
@@ -171,3 +175,14 @@ def emoe_moe_forward_routed(ctx, desc: emoe_layer_desc, x_ptr, T, ids_ptr, gates
 
 def emoe_set_ffn_path(ctx, path: int) -> None:
     _check(lib().emoe_set_ffn_path(ctx, path), "emoe_set_ffn_path")
+
+
+def emoe_set_timing(ctx, enabled: bool) -> None:
+    _check(lib().emoe_set_timing(ctx, int(enabled)), "emoe_set_timing")
+
+
+def emoe_read_timing(ctx):
+    """(first-projection ms, second-projection ms, forward calls covered) since the last read."""
+    a, b, n = ctypes.c_float(0), ctypes.c_float(0), ctypes.c_int(0)
+    _check(lib().emoe_read_timing(ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(n)), "emoe_read_timing")
+    return a.value, b.value, n.value

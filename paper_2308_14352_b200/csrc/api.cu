@@ -81,6 +81,9 @@ struct emoe_ctx {
   std::vector<TableEntry> tables;
   int last_cuda = 0;
   int ffn_path = 0;
+  bool timing = false;
+  std::vector<cudaEvent_t> events;  // triples (start, mid, end) per timed forward call
+  size_t events_used = 0;
 };
 
 namespace {
@@ -197,16 +200,31 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   const bool use_mma = ffn_mma_supported(L) && ctx->ffn_path != 1;
   if (ctx->ffn_path == 2 && !use_mma) return EMOE_ERR_UNSUPPORTED;
   int ksplit = 1;
+  cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+  if (ctx->timing) {
+    while (ctx->events.size() < ctx->events_used + 3) {
+      cudaEvent_t e;
+      EMOE_CUDA(ctx, cudaEventCreate(&e));
+      ctx->events.push_back(e);
+    }
+    for (int i = 0; i < 3; ++i) ev[i] = ctx->events[ctx->events_used + i];
+    ctx->events_used += 3;
+  }
   if (use_mma) {
     ksplit = w.ksplit;
     EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, xs, P, st));
+    if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_CUDA(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
+    if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
     EMOE_CUDA(ctx, launch_ffn_mma(1, L, table, reinterpret_cast<const __nv_bfloat16*>(hidden), off,
                                   reinterpret_cast<__nv_bfloat16*>(hidden), o_part, ksplit, P, T, st));
   } else {
+    if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_CUDA(ctx, launch_ffn_gemv(0, L, table, x, perm, off, hidden, o_part, P, st));
+    if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
     EMOE_CUDA(ctx, launch_ffn_gemv(1, L, table, x, perm, off, hidden, o_part, P, st));
   }
+  if (ev[2]) EMOE_CUDA(ctx, cudaEventRecord(ev[2], st));
   EMOE_CUDA(ctx, launch_combine(o_part, ksplit, static_cast<size_t>(P), gates_use, slot_of_pair, T, L.top_k, L.d_model,
                                 y, st));
   if (out_ids) EMOE_CUDA(ctx, cudaMemcpyAsync(out_ids, ids_use, sizeof(int32_t) * P, cudaMemcpyDeviceToDevice, st));
@@ -254,6 +272,7 @@ int emoe_destroy(emoe_ctx* ctx) {
   if (ctx->check_host) cudaFreeHost(ctx->check_host);
   if (ctx->tables_dev) cudaFree(ctx->tables_dev);
   if (ctx->tables_pin) cudaFreeHost(ctx->tables_pin);
+  for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
   delete ctx;
   return EMOE_OK;
 }
@@ -357,6 +376,32 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
   if (!ids || !gates) return EMOE_ERR_INVALID_ARG;
   return forward_impl(ctx, desc, x, T, nullptr, nullptr, 0, ids, gates, host_experts, y, nullptr, nullptr, out_perm,
                       static_cast<cudaStream_t>(stream));
+}
+
+int emoe_set_timing(emoe_ctx* ctx, int enabled) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  ctx->timing = enabled != 0;
+  ctx->events_used = 0;
+  return EMOE_OK;
+}
+
+int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, int* out_calls) {
+  if (!ctx || !out_first_ms || !out_second_ms || !out_calls) return EMOE_ERR_INVALID_ARG;
+  float a = 0.f, b = 0.f;
+  const size_t n = ctx->events_used / 3;
+  for (size_t i = 0; i < n; ++i) {
+    float ms = 0.f;
+    EMOE_CUDA(ctx, cudaEventSynchronize(ctx->events[3 * i + 2]));
+    EMOE_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->events[3 * i], ctx->events[3 * i + 1]));
+    a += ms;
+    EMOE_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->events[3 * i + 1], ctx->events[3 * i + 2]));
+    b += ms;
+  }
+  *out_first_ms = a;
+  *out_second_ms = b;
+  *out_calls = static_cast<int>(n);
+  ctx->events_used = 0;
+  return EMOE_OK;
 }
 
 int emoe_set_ffn_path(emoe_ctx* ctx, int path) {
