@@ -186,6 +186,29 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
  * measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);
 
+/* The routed layer forward for callers that cannot allocate device memory (the paper has no
+ * counterpart: it is an addition for hosts such as a framework that owns the whole device
+ * heap, a plug-in whose memory pool is fixed at start-up, or a latency-critical loop in which
+ * an allocation, which may synchronise the device, is not acceptable).  Such callers cannot
+ * have a context, because emoe_create allocates; this call needs none.  It computes exactly
+ * what emoe_moe_forward_routed computes, with its intermediate buffers in a fixed 8 MiB array
+ * that is part of the library image on every GPU that loads it (held until the process
+ * exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   Limits: T * top_k <= 64, and the intermediates of the call must fit the 8 MiB array
+ *   (roughly: 64 * (2*d_model + 2*d_ff + 4*d_model*splits) bytes); otherwise the call
+ *   returns EMOE_ERR_WORKSPACE and does nothing.  Other argument rules as for
+ *   emoe_moe_forward_routed.
+ *   First call on a device: looks up the array's device address (with that device made
+ *   current).  Make this first call outside any stream capture.
+ *   Sharing: every call on a device uses the same array, which keeps the previous call's
+ *   contents (the call clears what has to start at zero itself).  Two calls whose GPU work
+ *   overlaps (different streams without a dependency, or different host threads) race on it:
+ *   order them.
+ * `device` is the CUDA device ordinal; the other parameters are those of
+ * emoe_moe_forward_routed. */
+int emoe_moe_forward_routed_static(int device, const emoe_layer_desc* desc, const void* x, int T, const int32_t* ids,
+                                   const float* gates, const emoe_expert* host_experts, float* y, void* stream);
+
 /* Measurement aid (Section 4 of the paper times compute and loading separately; here the
  * expert-FFN kernels are the part bound by weight streaming).  While enabled, every forward
  * call records CUDA events on its stream around the first-projection and second-projection
