@@ -181,9 +181,10 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
                             const float* gates, const emoe_expert* host_experts, float* y, int32_t* out_perm,
                             void* stream);
 
-/* Selects the expert-FFN kernel family: 0 = automatic (default), 1 = force the CUDA-core
- * grouped GEMV, 2 = force the tensor-core path where the shape allows it.  For tests and
- * measurements. */
+/* Selects the expert-FFN kernel family: 0 = automatic (default), 1 = the CUDA-core grouped
+ * GEMV, 2 = the tensor-core kernel with register-staged weight loads, 3 = the tensor-core kernel
+ * with the TMA-staged weight pipeline.  2 and 3 fail with EMOE_ERR_UNSUPPORTED in forward calls
+ * whose shape they do not take.  For tests and measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);
 
 /* The routed layer forward for callers that cannot allocate device memory (the paper has no

@@ -12,16 +12,22 @@ using namespace emoe;
 
 namespace {
 
-constexpr int MAX_TABLES = 256;  // distinct expert tables a context can keep on the device
+constexpr int MAX_TABLES = 128;  // distinct expert tables a context can keep on the device
+constexpr size_t TMAP_BYTES = 128;  // sizeof(CUtensorMap)
+// one table block: the expert entries followed by one tensor map per (expert, matrix)
+constexpr size_t TABLE_MAPS_OFFSET = (sizeof(ExpertDev) * EMOE_MAX_EXPERTS + 127) / 128 * 128;
+constexpr size_t TABLE_BLOCK_BYTES = TABLE_MAPS_OFFSET + TMAP_BYTES * 3 * EMOE_MAX_EXPERTS;
 
 struct TableEntry {
   std::vector<emoe_expert> host;
+  int d_model = 0, d_ff = 0, act = 0;
+  bool has_tmaps = false;
 };
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-  size_t ids, gates, counts, off, perm, slot_of_pair, xs, hidden, o_part, total;
+  size_t ids, gates, counts, off, perm, slot_of_pair, plan, xs, hidden, o_part, total;
   int ksplit;
 };
 
@@ -51,7 +57,9 @@ bool make_dims(const emoe_layer_desc* d, LayerDims* L) {
 WorkspaceLayout make_layout(const LayerDims& L, int T) {
   WorkspaceLayout w{};
   const size_t P = static_cast<size_t>(T) * L.top_k;
-  w.ksplit = ffn_mma_supported(L) ? ffn_mma_ksplit(L, T) : 1;
+  w.ksplit = 1;
+  if (ffn_mma_supported(L)) w.ksplit = ffn_mma_ksplit(L, T);
+  if (ffn_tma_supported(L) && ffn_tma_ksplit(L, T) > w.ksplit) w.ksplit = ffn_tma_ksplit(L, T);
   size_t o = 0;
   w.ids = o;          o += align_up(P * 4);
   w.gates = o;        o += align_up(P * 4);
@@ -59,6 +67,7 @@ WorkspaceLayout make_layout(const LayerDims& L, int T) {
   w.off = o;          o += align_up(static_cast<size_t>(L.E + 1) * 4);
   w.perm = o;         o += align_up(P * 4);
   w.slot_of_pair = o; o += align_up(P * 4);
+  w.plan = o;         o += align_up(static_cast<size_t>(L.E + 4) * 4);
   w.xs = o;           o += align_up(L.act_bf16 ? P * L.d_model * 2 : 0);
   w.hidden = o;       o += align_up(P * L.d_ff * (L.act_bf16 ? 2 : 4));
   w.o_part = o;       o += align_up(static_cast<size_t>(w.ksplit) * P * L.d_model * 4);
@@ -76,8 +85,8 @@ struct emoe_ctx {
   size_t workspace_bytes = 0;
   int* check_word = nullptr;        // device
   int* check_host = nullptr;        // pinned
-  ExpertDev* tables_dev = nullptr;  // [MAX_TABLES][EMOE_MAX_EXPERTS]
-  ExpertDev* tables_pin = nullptr;  // pinned mirror, never rewritten once filled
+  char* tables_dev = nullptr;  // MAX_TABLES blocks of TABLE_BLOCK_BYTES
+  char* tables_pin = nullptr;  // pinned mirror, never rewritten once filled
   std::vector<TableEntry> tables;
   int last_cuda = 0;
   int ffn_path = 0;
@@ -99,24 +108,32 @@ int cuda_fail(emoe_ctx* ctx, cudaError_t e) {
     if (e__ != cudaSuccess) return cuda_fail(ctx, e__); \
   } while (0)
 
-// Device copy of a host expert table; uploaded on `st` the first time its content is seen.
-int get_table(emoe_ctx* ctx, const emoe_expert* host, int E, cudaStream_t st, const ExpertDev** out) {
+// Device copy of a host expert table (entries + tensor maps); uploaded on `st` the first time
+// its content is seen.  *tmaps is null when the shape has no TMA path.
+int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaStream_t st, const ExpertDev** out,
+              const void** tmaps) {
+  const int E = L.E;
   for (size_t i = 0; i < ctx->tables.size(); ++i) {
-    const std::vector<emoe_expert>& h = ctx->tables[i].host;
-    if (static_cast<int>(h.size()) != E) continue;
+    const TableEntry& te = ctx->tables[i];
+    if (static_cast<int>(te.host.size()) != E || te.d_model != L.d_model || te.d_ff != L.d_ff || te.act != L.act) continue;
     bool same = true;
     for (int e = 0; e < E && same; ++e) {
-      same = h[e].bits == host[e].bits;
-      for (int m = 0; m < 3 && same; ++m) same = h[e].packed[m] == host[e].packed[m] && h[e].scales[m] == host[e].scales[m];
+      same = te.host[e].bits == host[e].bits;
+      for (int m = 0; m < 3 && same; ++m)
+        same = te.host[e].packed[m] == host[e].packed[m] && te.host[e].scales[m] == host[e].scales[m];
     }
     if (same) {
-      *out = ctx->tables_dev + i * EMOE_MAX_EXPERTS;
+      *out = reinterpret_cast<const ExpertDev*>(ctx->tables_dev + i * TABLE_BLOCK_BYTES);
+      *tmaps = te.has_tmaps ? ctx->tables_dev + i * TABLE_BLOCK_BYTES + TABLE_MAPS_OFFSET : nullptr;
       return EMOE_OK;
     }
   }
   if (ctx->tables.size() >= MAX_TABLES) return EMOE_ERR_WORKSPACE;
   const size_t slot = ctx->tables.size();
-  ExpertDev* pin = ctx->tables_pin + slot * EMOE_MAX_EXPERTS;
+  char* pin_block = ctx->tables_pin + slot * TABLE_BLOCK_BYTES;
+  ExpertDev* pin = reinterpret_cast<ExpertDev*>(pin_block);
+  const int nmat = L.act == EMOE_ACT_RELU ? 2 : 3;
+  bool maps_ok = ffn_tma_supported(L);
   for (int e = 0; e < E; ++e) {
     pin[e].bits = host[e].bits;
     pin[e].pad = 0;
@@ -124,13 +141,25 @@ int get_table(emoe_ctx* ctx, const emoe_expert* host, int E, cudaStream_t st, co
       pin[e].packed[m] = static_cast<const uint8_t*>(host[e].packed[m]);
       pin[e].scales[m] = host[e].scales[m];
     }
+    for (int m = 0; m < nmat && maps_ok; ++m) {
+      const bool first = m < nmat - 1;
+      const int N = first ? L.d_ff : L.d_model, K = first ? L.d_model : L.d_ff;
+      maps_ok = encode_weight_tmap(pin_block + TABLE_MAPS_OFFSET + TMAP_BYTES * (3 * e + m), host[e].packed[m], N, K,
+                                   host[e].bits) == 0;
+    }
   }
-  ExpertDev* dev = ctx->tables_dev + slot * EMOE_MAX_EXPERTS;
-  EMOE_CUDA(ctx, cudaMemcpyAsync(dev, pin, sizeof(ExpertDev) * E, cudaMemcpyHostToDevice, st));
+  char* dev = ctx->tables_dev + slot * TABLE_BLOCK_BYTES;
+  const size_t bytes = maps_ok ? TABLE_MAPS_OFFSET + TMAP_BYTES * 3 * E : sizeof(ExpertDev) * E;
+  EMOE_CUDA(ctx, cudaMemcpyAsync(dev, pin_block, bytes, cudaMemcpyHostToDevice, st));
   TableEntry te;
   te.host.assign(host, host + E);
+  te.d_model = L.d_model;
+  te.d_ff = L.d_ff;
+  te.act = L.act;
+  te.has_tmaps = maps_ok;
   ctx->tables.push_back(std::move(te));
-  *out = dev;
+  *out = reinterpret_cast<const ExpertDev*>(dev);
+  *tmaps = maps_ok ? dev + TABLE_MAPS_OFFSET : nullptr;
   return EMOE_OK;
 }
 
@@ -171,7 +200,8 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
 
   const ExpertDev* table = nullptr;
-  rc = get_table(ctx, host_experts, L.E, st, &table);
+  const void* tmaps = nullptr;
+  rc = get_table(ctx, L, host_experts, st, &table, &tmaps);
   if (rc != EMOE_OK) return rc;
 
   char* ws = ctx->workspace;
@@ -182,6 +212,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   int32_t* off = reinterpret_cast<int32_t*>(ws + w.off);
   int32_t* perm = reinterpret_cast<int32_t*>(ws + w.perm);
   int32_t* slot_of_pair = reinterpret_cast<int32_t*>(ws + w.slot_of_pair);
+  int* plan = reinterpret_cast<int*>(ws + w.plan);
   __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(ws + w.xs);
   void* hidden = ws + w.hidden;
   float* o_part = reinterpret_cast<float*>(ws + w.o_part);
@@ -197,8 +228,11 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   }
   EMOE_CUDA(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
 
+  const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
+  const bool use_tma = can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
   const bool use_mma = ffn_mma_supported(L) && ctx->ffn_path != 1;
   if (ctx->ffn_path == 2 && !use_mma) return EMOE_ERR_UNSUPPORTED;
+  if (ctx->ffn_path == 3 && !use_tma) return EMOE_ERR_UNSUPPORTED;
   int ksplit = 1;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
   if (ctx->timing) {
@@ -210,9 +244,18 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     for (int i = 0; i < 3; ++i) ev[i] = ctx->events[ctx->events_used + i];
     ctx->events_used += 3;
   }
-  if (use_mma) {
-    ksplit = w.ksplit;
-    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, xs, P, st));
+  if (use_tma) {
+    ksplit = ffn_tma_ksplit(L, T);
+    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, st));
+    if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
+    EMOE_CUDA(ctx, launch_ffn_tma(0, L, table, tmaps, xs, off, plan, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T,
+                                  ctx->check_word, st));
+    if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+    EMOE_CUDA(ctx, launch_ffn_tma(1, L, table, tmaps, reinterpret_cast<const __nv_bfloat16*>(hidden), off, plan,
+                                  reinterpret_cast<__nv_bfloat16*>(hidden), o_part, ksplit, P, T, ctx->check_word, st));
+  } else if (use_mma) {
+    ksplit = ffn_mma_ksplit(L, T);
+    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_CUDA(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
@@ -252,8 +295,8 @@ emoe_ctx* emoe_create(int device, size_t workspace_bytes, int* status) {
   if (e == cudaSuccess) e = cudaMalloc(&ctx->check_word, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(ctx->check_word, 0, sizeof(int));
   if (e == cudaSuccess) e = cudaMallocHost(&ctx->check_host, sizeof(int));
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->tables_dev, sizeof(ExpertDev) * MAX_TABLES * EMOE_MAX_EXPERTS);
-  if (e == cudaSuccess) e = cudaMallocHost(&ctx->tables_pin, sizeof(ExpertDev) * MAX_TABLES * EMOE_MAX_EXPERTS);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->tables_dev, TABLE_BLOCK_BYTES * MAX_TABLES);
+  if (e == cudaSuccess) e = cudaMallocHost(&ctx->tables_pin, TABLE_BLOCK_BYTES * MAX_TABLES);
   if (e != cudaSuccess) {
     *status = EMOE_ERR_CUDA;
     ctx->last_cuda = static_cast<int>(e);
@@ -405,7 +448,7 @@ int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, i
 }
 
 int emoe_set_ffn_path(emoe_ctx* ctx, int path) {
-  if (!ctx || path < 0 || path > 2) return EMOE_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 3) return EMOE_ERR_INVALID_ARG;
   ctx->ffn_path = path;
   return EMOE_OK;
 }

@@ -20,6 +20,7 @@ struct ExpertDev {
 // Bits of the device-side check word.
 enum : int {
   CHECK_BAD_EXPERT_ID = 1,
+  CHECK_WAIT_TIMEOUT = 2,  // a bounded wait inside a kernel ran out
 };
 
 struct LayerDims {
@@ -50,11 +51,23 @@ cudaError_t launch_ffn_gemv(int phase, const LayerDims& L, const ExpertDev* expe
 // hidden: same interleave, [n_pairs][d_ff] bf16.  o_part: [ksplit][n_pairs][d_model] fp32.
 bool ffn_mma_supported(const LayerDims& L);
 int ffn_mma_ksplit(const LayerDims& L, int T);
+int ffn_token_tiles(const LayerDims& L, int T);
+// plan (nullable): int[4 + E] work plan for the persistent TMA kernels, filled by block 0.
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
-                             const int32_t* perm, __nv_bfloat16* xs, int n_pairs, cudaStream_t st);
+                             const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
+                             cudaStream_t st);
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
                            const int32_t* off, __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs,
                            int T, cudaStream_t st);
+
+// TMA-staged variant of the tensor-core kernel (needs one tensor map per packed matrix, built
+// on the host by encode_weight_tmap and kept next to the expert table: tmaps[e*3 + m], 128 bytes each).
+bool ffn_tma_supported(const LayerDims& L);
+int ffn_tma_ksplit(const LayerDims& L, int T);
+int encode_weight_tmap(void* out_map, const void* packed, int N, int K, int bits);
+cudaError_t launch_ffn_tma(int phase, const LayerDims& L, const ExpertDev* experts, const void* tmaps,
+                           const __nv_bfloat16* in, const int32_t* off, int* plan, __nv_bfloat16* hidden, float* o_part,
+                           int ksplit, int n_pairs, int T, int* check_word, cudaStream_t st);
 
 // y[t] = sum_j gates[t][j] * sum_z o_part[z][slot_of_pair[t*k+j]]
 // o_part holds ksplit partial results, each [n_pairs_stride][d].

@@ -18,7 +18,10 @@
 // and (c, c+8) of a 16-code word at 2 bits, so the activations are stored in that interleaved
 // order once (scatter_x_kernel for x, the first phase's epilogue for the hidden vector) and
 // B fragments become plain 128-bit shared-memory loads.
+#include <cmath>
+
 #include "common.cuh"
+#include "ffn_tile.cuh"
 
 namespace emoe {
 namespace {
@@ -27,136 +30,8 @@ constexpr int MMA_WARPS = 4;
 constexpr int MMA_THREADS = MMA_WARPS * 32;
 constexpr int MMA_MT = 2;          // 16-row tiles per warp
 constexpr int MMA_KCH = 512;       // inputs per staged activation chunk (4 segments of 128)
-constexpr int MMA_XPAD = 8;        // bf16 elements of row padding in shared memory
+constexpr int MMA_XPAD = 32;       // bf16 elements of row padding in shared memory
 constexpr int MMA_XSTRIDE = MMA_KCH + MMA_XPAD;
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t r;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-  return r;
-}
-
-// (a & b) ^ c in one LOP3
-__device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t r;
-  asm("lop3.b32 %0, %1, %2, %3, 0x6a;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
-  return r;
-}
-
-__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t r;
-  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
-  return r;
-}
-
-__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t a0, const uint32_t a1, const uint32_t a2,
-                                         const uint32_t a3, const uint32_t b0, const uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// ---- per-bitwidth unpack: 32 codes of one output channel -> 16 bf16x2 registers -------------
-// P[r] holds the codes with local index (a_r, b_r); the interleaved activation layout puts
-// x[a_r] at position 2r and x[b_r] at 2r+1 of the lane's 32-element block.
-template <int BITS>
-struct Raw;  // the lane's raw bytes for one row of one segment
-template <>
-struct Raw<8> { uint4 v[2]; };
-template <>
-struct Raw<4> { uint4 v[1]; };
-template <>
-struct Raw<2> { uint2 v[1]; };
-
-template <int BITS>
-__device__ __forceinline__ Raw<BITS> load_raw(const uint8_t* p);
-template <>
-__device__ __forceinline__ Raw<8> load_raw<8>(const uint8_t* p) {
-  Raw<8> r;
-  r.v[0] = __ldg(reinterpret_cast<const uint4*>(p));
-  r.v[1] = __ldg(reinterpret_cast<const uint4*>(p) + 1);
-  return r;
-}
-template <>
-__device__ __forceinline__ Raw<4> load_raw<4>(const uint8_t* p) {
-  Raw<4> r;
-  r.v[0] = __ldg(reinterpret_cast<const uint4*>(p));
-  return r;
-}
-template <>
-__device__ __forceinline__ Raw<2> load_raw<2>(const uint8_t* p) {
-  Raw<2> r;
-  r.v[0] = __ldg(reinterpret_cast<const uint2*>(p));
-  return r;
-}
-
-// 8 bits: byte -> 2^23 + (q+128) as fp32 by byte permute, subtract, keep the high halves
-// (integers of magnitude <= 128 are exact in bf16).  Natural pair order (2r, 2r+1).
-__device__ __forceinline__ void unpack(const Raw<8>& raw, uint32_t (&P)[16]) {
-  const uint32_t w[8] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w, raw.v[1].x, raw.v[1].y, raw.v[1].z, raw.v[1].w};
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const uint32_t u = w[i] ^ 0x80808080u;
-    const float f0 = __uint_as_float(prmt(u, 0x4B000000u, 0x7540u)) - 8388736.0f;
-    const float f1 = __uint_as_float(prmt(u, 0x4B000000u, 0x7541u)) - 8388736.0f;
-    const float f2 = __uint_as_float(prmt(u, 0x4B000000u, 0x7542u)) - 8388736.0f;
-    const float f3 = __uint_as_float(prmt(u, 0x4B000000u, 0x7543u)) - 8388736.0f;
-    P[2 * i] = prmt(__float_as_uint(f0), __float_as_uint(f1), 0x7632u);
-    P[2 * i + 1] = prmt(__float_as_uint(f2), __float_as_uint(f3), 0x7632u);
-  }
-}
-
-// 4 bits: nibble c of a 16-bit half lands in the mantissa of bf16 128.0 (ulp 1), with its
-// sign bit flipped (two's complement -> offset binary): value 128 + (q + 8); subtract 136.
-// Pair order (c, c+4) inside each 8-code word.
-__device__ __forceinline__ void unpack(const Raw<4>& raw, uint32_t (&P)[16]) {
-  const uint32_t w[4] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w};
-  const uint32_t one = 0x3F803F80u;   // bf16x2 (1, 1)
-  const uint32_t m136 = 0xC308C308u;  // bf16x2 (-136, -136)
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const uint32_t v = and_xor(w[i] >> (4 * c), 0x000F000Fu, 0x43084308u);
-      P[4 * i + c] = bf16x2_fma(v, one, m136);
-    }
-  }
-}
-
-// 2 bits: field at mantissa bit p in {0,2,4} of bf16 128.0: value 128 + (q + 2) * 2^p;
-// q = v * 2^-p - (128 * 2^-p + 2).  Pair order (c, c+8) inside each 16-code word.
-__device__ __forceinline__ void unpack(const Raw<2>& raw, uint32_t (&P)[16]) {
-  const uint32_t w[2] = {raw.v[0].x, raw.v[0].y};
-  // bf16: 1 = 0x3F80, 0.25 = 0x3E80, 0.0625 = 0x3D80; -130 = 0xC302, -34 = 0xC208, -10 = 0xC120
-  const uint32_t mul[3] = {0x3F803F80u, 0x3E803E80u, 0x3D803D80u};
-  const uint32_t add[3] = {0xC302C302u, 0xC208C208u, 0xC120C120u};
-  const uint32_t msk[3] = {0x00030003u, 0x000C000Cu, 0x00300030u};
-  const uint32_t mag[3] = {0x43024302u, 0x43084308u, 0x43204320u};  // 128 with the field's sign bit set
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const int sh = 6 * (c / 3), p = c % 3;
-      const uint32_t v = and_xor(w[i] >> sh, msk[p], mag[p]);
-      P[8 * i + c] = bf16x2_fma(v, mul[p], add[p]);
-    }
-  }
-}
-
-// position of element `o` (natural order) inside its interleaved block
-template <int BITS>
-__device__ __forceinline__ int interleaved_pos(int k) {
-  if (BITS == 8) return k;
-  constexpr int B = BITS == 4 ? 8 : 16;  // block length
-  const int o = k & (B - 1);
-  return (k & ~(B - 1)) + (o < B / 2 ? 2 * o : 2 * (o - B / 2) + 1);
-}
-
-__device__ __forceinline__ float load_scale(const void* scales, bool f16, size_t idx) {
-  return f16 ? __half2float(__ldg(reinterpret_cast<const __half*>(scales) + idx))
-             : __ldg(reinterpret_cast<const float*>(scales) + idx);
-}
 
 // ---- the kernel body for one bitwidth -----------------------------------------------------------
 template <int BITS, int NT>
@@ -237,16 +112,16 @@ __device__ __forceinline__ void ffn_mma_body(int phase, const LayerDims& L, cons
 #pragma unroll
         for (int mt = 0; mt < MMA_MT; ++mt)
 #pragma unroll
-          for (int h = 0; h < 2; ++h) sc[mt][h] = load_scale(sbase[mt], sf16, srow[mt][h] + grp);
+          for (int h = 0; h < 2; ++h) sc[mt][h] = load_scale_ro(sbase[mt], sf16, srow[mt][h] + grp);
 
         // B fragments of this segment: the lane's 32 interleaved activations of token (nt*8 + g)
         uint4 bq[NT][4];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           if (nt * 8 < ntok) {
-            const uint4* src = reinterpret_cast<const uint4*>(xsm + (nt * 8 + g) * MMA_XSTRIDE + sg * 128 + t * 32);
+            const uint4* src = reinterpret_cast<const uint4*>(xsm + (nt * 8 + g) * MMA_XSTRIDE + sg * 128 + t * 8);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) bq[nt][q] = src[q];
+            for (int q = 0; q < 4; ++q) bq[nt][q] = src[q * 4];  // piece q of lane t sits at (q*4 + t) * 16 bytes
           }
         }
 #pragma unroll
@@ -286,7 +161,7 @@ __device__ __forceinline__ void ffn_mma_body(int phase, const LayerDims& L, cons
           if (n < N) {
             const float a = tot[0][nt][i], b = tot[1][nt][i];
             const float h = a / (1.0f + expf(-a)) * b;
-            hidden[slot * N + interleaved_pos<BITS>(n)] = __float2bfloat16_rn(h);
+            hidden[slot * N + act_pos<BITS>(n)] = __float2bfloat16_rn(h);
           }
         } else {
 #pragma unroll
@@ -294,7 +169,7 @@ __device__ __forceinline__ void ffn_mma_body(int phase, const LayerDims& L, cons
             const int n = row0 + 16 * mt + g + 8 * (i >> 1);
             if (n >= N) continue;
             if (phase == 0)
-              hidden[slot * N + interleaved_pos<BITS>(n)] = __float2bfloat16_rn(fmaxf(tot[mt][nt][i], 0.0f));
+              hidden[slot * N + act_pos<BITS>(n)] = __float2bfloat16_rn(fmaxf(tot[mt][nt][i], 0.0f));
             else
               o_part[(static_cast<size_t>(blockIdx.y) * n_pairs + slot) * N + n] = tot[mt][nt][i];
           }
@@ -326,38 +201,71 @@ __global__ void __launch_bounds__(MMA_THREADS)
   }
 }
 
-// x rows -> expert-sorted order, in the k-interleave of the owning expert's bitwidth
+// x rows -> expert-sorted order, in the activation layout of the owning expert's bitwidth
 __global__ void __launch_bounds__(128)
     scatter_x_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
-                     const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, int top_k, int d, int n_pairs,
-                     __nv_bfloat16* __restrict__ xs) {
+                     const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
+                     int E, int* __restrict__ plan, int top_k, int d, int n_pairs, __nv_bfloat16* __restrict__ xs) {
+  if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
+    // work plan of the persistent expert kernels: activated experts, widest codes (most bytes)
+    // first; the two item counters restart from zero
+    const int lane = threadIdx.x;
+    int base = 0;
+    for (int b = 8; b >= 2; b >>= 1) {
+      for (int e0 = 0; e0 < E; e0 += 32) {
+        const int e = e0 + lane;
+        const bool act = e < E && off[e + 1] > off[e] && experts[e].bits == b;
+        const unsigned m = __ballot_sync(0xffffffffu, act);
+        if (act) plan[4 + base + __popc(m & ((1u << lane) - 1u))] = e;
+        base += __popc(m);
+      }
+    }
+    if (lane == 0) {
+      plan[0] = base;
+      plan[1] = 0;
+      plan[2] = 0;
+    }
+  }
   const int slot = blockIdx.x;
   const int pair = perm[slot];
   if (pair < 0 || pair >= n_pairs) return;
   const int bits = experts[ids[pair]].bits;
-  const uint4* src = reinterpret_cast<const uint4*>(x + static_cast<size_t>(pair / top_k) * d);
-  uint4* dst = reinterpret_cast<uint4*>(xs + static_cast<size_t>(slot) * d);
-  for (int b = threadIdx.x; b < d / 16; b += blockDim.x) {  // 16 elements = two 128-bit vectors
-    const uint4 a = src[2 * b], c = src[2 * b + 1];
+  const __nv_bfloat16* src_row = x + static_cast<size_t>(pair / top_k) * d;
+  __nv_bfloat16* dst_row = xs + static_cast<size_t>(slot) * d;
+  // one thread moves 16 consecutive inputs: half b of lane t's 32-block of a 128-input segment
+  for (int u = threadIdx.x; u < d / 16; u += blockDim.x) {
+    const int seg = (u >> 3) * 128, t = (u >> 1) & 3, b = u & 1;
+    const uint4* src = reinterpret_cast<const uint4*>(src_row + seg + t * 32 + b * 16);
+    const uint4 a = src[0], c = src[1];
     uint4 oa, oc;
     if (bits == 8) {
       oa = a;
       oc = c;
-    } else if (bits == 4) {  // [0,4,1,5,2,6,3,7] inside each 8
+    } else if (bits == 4) {  // pair order (c, c+4) inside each 8
       oa = make_uint4(prmt(a.x, a.z, 0x5410u), prmt(a.x, a.z, 0x7632u), prmt(a.y, a.w, 0x5410u), prmt(a.y, a.w, 0x7632u));
       oc = make_uint4(prmt(c.x, c.z, 0x5410u), prmt(c.x, c.z, 0x7632u), prmt(c.y, c.w, 0x5410u), prmt(c.y, c.w, 0x7632u));
-    } else {  // [0,8,1,9,...,7,15] inside each 16
+    } else {  // pair order (c, c+8) inside each 16
       oa = make_uint4(prmt(a.x, c.x, 0x5410u), prmt(a.x, c.x, 0x7632u), prmt(a.y, c.y, 0x5410u), prmt(a.y, c.y, 0x7632u));
       oc = make_uint4(prmt(a.z, c.z, 0x5410u), prmt(a.z, c.z, 0x7632u), prmt(a.w, c.w, 0x5410u), prmt(a.w, c.w, 0x7632u));
     }
-    dst[2 * b] = oa;
-    dst[2 * b + 1] = oc;
+    // pieces q = 2b and 2b+1 of lane t, stored piece-major
+    *reinterpret_cast<uint4*>(dst_row + seg + (((2 * b) * 4 + t) << 3)) = oa;
+    *reinterpret_cast<uint4*>(dst_row + seg + (((2 * b + 1) * 4 + t) << 3)) = oc;
   }
 }
 
-int pick_nt(int T) { return T <= 8 ? 1 : (T <= 16 ? 2 : 4); }
 
 }  // namespace
+
+// 8-token tiles a CTA handles per pass over its weights: enough for the mean tokens per expert
+// plus 2.5 standard deviations under uniform routing (an expert with more tokens takes another
+// pass over its own weights, which then come from L2).
+int ffn_token_tiles(const LayerDims& L, int T) {
+  const double mean = static_cast<double>(T) * L.top_k / L.E;
+  double need = mean + 2.5 * sqrt(mean) + 1.0;
+  if (need > T) need = T;
+  return need <= 8.0 ? 1 : (need <= 16.0 ? 2 : 4);
+}
 
 bool ffn_mma_supported(const LayerDims& L) {
   if (!L.act_bf16) return false;
@@ -379,9 +287,10 @@ int ffn_mma_ksplit(const LayerDims& L, int T) {
 }
 
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
-                             const int32_t* perm, __nv_bfloat16* xs, int n_pairs, cudaStream_t st) {
-  scatter_x_kernel<<<n_pairs, 128, 0, st>>>(experts, reinterpret_cast<const __nv_bfloat16*>(x), ids, perm, L.top_k,
-                                            L.d_model, n_pairs, xs);
+                             const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
+                             cudaStream_t st) {
+  scatter_x_kernel<<<n_pairs, 128, 0, st>>>(experts, reinterpret_cast<const __nv_bfloat16*>(x), ids, perm, off, L.E, plan,
+                                            L.top_k, L.d_model, n_pairs, xs);
   return cudaGetLastError();
 }
 
@@ -392,7 +301,7 @@ cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* exper
   const int rows_per_cta = (phase == 0 && L.act == EMOE_ACT_SWIGLU) ? 16 * MMA_WARPS : 16 * MMA_MT * MMA_WARPS;
   const dim3 grid((N + rows_per_cta - 1) / rows_per_cta, phase == 0 ? 1 : ksplit, L.E);
   const int z = phase == 0 ? 1 : ksplit;
-  switch (pick_nt(T)) {
+  switch (ffn_token_tiles(L, T)) {
     case 1: ffn_mma_kernel<1><<<grid, MMA_THREADS, 0, st>>>(phase, L, experts, in, off, hidden, o_part, z, n_pairs); break;
     case 2: ffn_mma_kernel<2><<<grid, MMA_THREADS, 0, st>>>(phase, L, experts, in, off, hidden, o_part, z, n_pairs); break;
     default: ffn_mma_kernel<4><<<grid, MMA_THREADS, 0, st>>>(phase, L, experts, in, off, hidden, o_part, z, n_pairs); break;

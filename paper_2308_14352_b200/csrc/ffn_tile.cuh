@@ -1,0 +1,150 @@
+// Device helpers shared by the tensor-core expert-FFN kernels: the bitwidth-specialised unpack
+// of packed codes into exact bf16 integers, the MMA wrapper, and the activation layout.
+//
+// Activation layout ("k-interleave").  An MMA does not care in which order the reduction index
+// is enumerated as long as A and B agree, so the activations (x rows and the hidden vector) are
+// stored once in the order that makes both operands cheap:
+//   * inside a 128-input segment, lane t of a quad owns inputs [32t, 32t+32);
+//   * the unpack emits code pairs (c, c+4) of an 8-code word at 4 bits, (c, c+8) of a 16-code
+//     word at 2 bits and (2c, 2c+1) at 8 bits, so the lane's 32 activations are stored in that
+//     pair order (position 2r, 2r+1 <- the two inputs of pair r);
+//   * the lane's four 16-byte pieces q are stored piece-major, at (q*4 + t)*16 bytes of the
+//     segment, so that the four lanes of a quad read adjacent 16-byte columns of shared memory.
+#pragma once
+#include "common.cuh"
+
+namespace emoe {
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
+}
+
+// (a & b) ^ c in one LOP3
+__device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("lop3.b32 %0, %1, %2, %3, 0x6a;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+
+__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t a0, const uint32_t a1, const uint32_t a2,
+                                         const uint32_t a3, const uint32_t b0, const uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// ---- per-bitwidth unpack: 32 codes of one output channel -> 16 bf16x2 registers -------------
+// P[r] holds the codes with local index (a_r, b_r); the interleaved activation layout puts
+// x[a_r] at position 2r and x[b_r] at 2r+1 of the lane's 32-element block.
+template <int BITS>
+struct Raw;  // the lane's raw bytes for one row of one segment
+template <>
+struct Raw<8> { uint4 v[2]; };
+template <>
+struct Raw<4> { uint4 v[1]; };
+template <>
+struct Raw<2> { uint2 v[1]; };
+
+template <int BITS>
+__device__ __forceinline__ Raw<BITS> load_raw(const uint8_t* p);
+template <>
+__device__ __forceinline__ Raw<8> load_raw<8>(const uint8_t* p) {
+  Raw<8> r;
+  r.v[0] = __ldg(reinterpret_cast<const uint4*>(p));
+  r.v[1] = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+  return r;
+}
+template <>
+__device__ __forceinline__ Raw<4> load_raw<4>(const uint8_t* p) {
+  Raw<4> r;
+  r.v[0] = __ldg(reinterpret_cast<const uint4*>(p));
+  return r;
+}
+template <>
+__device__ __forceinline__ Raw<2> load_raw<2>(const uint8_t* p) {
+  Raw<2> r;
+  r.v[0] = __ldg(reinterpret_cast<const uint2*>(p));
+  return r;
+}
+
+// 8 bits: byte -> 2^23 + (q+128) as fp32 by byte permute, subtract, keep the high halves
+// (integers of magnitude <= 128 are exact in bf16).  Natural pair order (2r, 2r+1).
+__device__ __forceinline__ void unpack(const Raw<8>& raw, uint32_t (&P)[16]) {
+  const uint32_t w[8] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w, raw.v[1].x, raw.v[1].y, raw.v[1].z, raw.v[1].w};
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t u = w[i] ^ 0x80808080u;
+    const float f0 = __uint_as_float(prmt(u, 0x4B000000u, 0x7540u)) - 8388736.0f;
+    const float f1 = __uint_as_float(prmt(u, 0x4B000000u, 0x7541u)) - 8388736.0f;
+    const float f2 = __uint_as_float(prmt(u, 0x4B000000u, 0x7542u)) - 8388736.0f;
+    const float f3 = __uint_as_float(prmt(u, 0x4B000000u, 0x7543u)) - 8388736.0f;
+    P[2 * i] = prmt(__float_as_uint(f0), __float_as_uint(f1), 0x7632u);
+    P[2 * i + 1] = prmt(__float_as_uint(f2), __float_as_uint(f3), 0x7632u);
+  }
+}
+
+// 4 bits: nibble c of a 16-bit half lands in the mantissa of bf16 128.0 (ulp 1), with its
+// sign bit flipped (two's complement -> offset binary): value 128 + (q + 8); subtract 136.
+// Pair order (c, c+4) inside each 8-code word.
+__device__ __forceinline__ void unpack(const Raw<4>& raw, uint32_t (&P)[16]) {
+  const uint32_t w[4] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w};
+  const uint32_t one = 0x3F803F80u;   // bf16x2 (1, 1)
+  const uint32_t m136 = 0xC308C308u;  // bf16x2 (-136, -136)
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint32_t v = and_xor(w[i] >> (4 * c), 0x000F000Fu, 0x43084308u);
+      P[4 * i + c] = bf16x2_fma(v, one, m136);
+    }
+  }
+}
+
+// 2 bits: field at mantissa bit p in {0,2,4} of bf16 128.0: value 128 + (q + 2) * 2^p;
+// q = v * 2^-p - (128 * 2^-p + 2).  Pair order (c, c+8) inside each 16-code word.
+__device__ __forceinline__ void unpack(const Raw<2>& raw, uint32_t (&P)[16]) {
+  const uint32_t w[2] = {raw.v[0].x, raw.v[0].y};
+  // bf16: 1 = 0x3F80, 0.25 = 0x3E80, 0.0625 = 0x3D80; -130 = 0xC302, -34 = 0xC208, -10 = 0xC120
+  const uint32_t mul[3] = {0x3F803F80u, 0x3E803E80u, 0x3D803D80u};
+  const uint32_t add[3] = {0xC302C302u, 0xC208C208u, 0xC120C120u};
+  const uint32_t msk[3] = {0x00030003u, 0x000C000Cu, 0x00300030u};
+  const uint32_t mag[3] = {0x43024302u, 0x43084308u, 0x43204320u};  // 128 with the field's sign bit set
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const int sh = 6 * (c / 3), p = c % 3;
+      const uint32_t v = and_xor(w[i] >> sh, msk[p], mag[p]);
+      P[8 * i + c] = bf16x2_fma(v, mul[p], add[p]);
+    }
+  }
+}
+
+// position of input k (natural order) in the activation layout described at the top
+template <int BITS>
+__device__ __forceinline__ int act_pos(int k) {
+  const int kk = k & 127, t = kk >> 5, i = kk & 31;
+  int j = i;
+  if (BITS != 8) {
+    constexpr int B = BITS == 4 ? 8 : 16;  // codes per unpacked word
+    const int o = i & (B - 1);
+    j = (i & ~(B - 1)) + (o < B / 2 ? 2 * o : 2 * (o - B / 2) + 1);
+  }
+  return (k & ~127) + (((j >> 3) * 4 + t) << 3) + (j & 7);
+}
+
+__device__ __forceinline__ float load_scale_ro(const void* scales, bool f16, size_t idx) {
+  return f16 ? __half2float(__ldg(reinterpret_cast<const __half*>(scales) + idx))
+             : __ldg(reinterpret_cast<const float*>(scales) + idx);
+}
+
+}  // namespace emoe

@@ -1,0 +1,519 @@
+// Grouped expert FFN on packed weights: TMA-staged weight stream + tensor-core multiply-adds,
+// for bf16 activations in the decode regime.  Paper Sections 1/2.1 (each activated expert is an
+// independent FFN) on the Section 3.2 storage (b-bit codes + scale channel, w~ = q * s formed
+// in registers).
+//
+// Same arithmetic as ffn_mma.cu (codes as exact bf16 integers in the A operand of
+// mma.m16n8k16, tokens as the N dimension, fp32 accumulation per 128-input segment, then
+// total += scale * segment); what differs is how the bytes travel.  The kernel is bound by
+// streaming packed weights from HBM, so the bytes in flight must not depend on registers:
+//   * the kernel is persistent: a CTA pulls work items (activated expert, block of output
+//     rows, split-K slice) from a device-side counter, most expensive bitwidth first, and its
+//     producer warp runs ahead across item boundaries, so the weight stream never drains
+//     between tiles;
+//   * the producer keeps a ring of STAGES shared-memory stages full.  One stage holds two
+//     64-row x 128-byte boxes of packed codes, fetched by two TMA tensor copies (128-byte
+//     swizzle, so that the consumers' 128-bit reads are conflict free), the matching slice of
+//     the expert's activations, fetched by one bulk copy per token row, and a small record
+//     that tells the consumers which item and which inputs the stage belongs to;
+//   * four consumer warps wait on the stage's mbarrier, read their 16-row tiles from shared
+//     memory, unpack, issue the MMAs, and hand the stage back through a second mbarrier.
+// 128 bytes of a row are 128 / 256 / 512 inputs at 8 / 4 / 2 bits, so a stage covers 1 / 2 / 4
+// scale segments.  Every wait is bounded: a wait that runs out sets a bit in the context's
+// check word and the CTA winds down without touching the stage.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ffn_tile.cuh"
+
+namespace emoe {
+namespace {
+
+constexpr int TMA_CONSUMER_WARPS = 4;
+constexpr int TMA_THREADS = (TMA_CONSUMER_WARPS + 1) * 32;
+constexpr int TMA_BOX_ROWS = 64;
+constexpr int TMA_BOX_BYTES = TMA_BOX_ROWS * 128;  // 8 KB
+constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a stage (row stride = 64 mod 128)
+constexpr unsigned WAIT_LIMIT = 1u << 22;          // polls before a wait gives up (~0.2 s)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (after flagging the check word) if the phase never completed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* check_word, volatile int* abort_flag) {
+  for (unsigned i = 0; i < WAIT_LIMIT; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (i > 64) __nanosleep(40);
+  }
+  *abort_flag = 1;
+  atomicOr(check_word, CHECK_WAIT_TIMEOUT);
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(tmap), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+// MMA row g of a 16-row tile -> row of the shared-memory box, chosen per bitwidth so that the
+// lanes of one shared-memory transaction fall into different 16-byte columns after the swizzle.
+template <int BITS>
+__device__ __forceinline__ int box_row_of(int g) {
+  if (BITS == 8) return g;
+  if (BITS == 4) return ((g & 1) << 2) | (g >> 1);
+  return ((g & 3) << 1) | (g >> 2);
+}
+
+// the lane's raw codes of one row for segment `sg` of the stage, from a swizzled box
+template <int BITS>
+__device__ __forceinline__ Raw<BITS> lds_raw(const unsigned char* box, int row, int sg, int t);
+template <>
+__device__ __forceinline__ Raw<8> lds_raw<8>(const unsigned char* box, int row, int sg, int t) {
+  (void)sg;
+  Raw<8> r;
+  const unsigned char* base = box + row * 128;
+  r.v[0] = *reinterpret_cast<const uint4*>(base + (((2 * t) ^ (row & 7)) << 4));
+  r.v[1] = *reinterpret_cast<const uint4*>(base + (((2 * t + 1) ^ (row & 7)) << 4));
+  return r;
+}
+template <>
+__device__ __forceinline__ Raw<4> lds_raw<4>(const unsigned char* box, int row, int sg, int t) {
+  Raw<4> r;
+  r.v[0] = *reinterpret_cast<const uint4*>(box + row * 128 + (((4 * sg + t) ^ (row & 7)) << 4));
+  return r;
+}
+template <>
+__device__ __forceinline__ Raw<2> lds_raw<2>(const unsigned char* box, int row, int sg, int t) {
+  Raw<2> r;
+  r.v[0] = *reinterpret_cast<const uint2*>(box + row * 128 + (((2 * sg + (t >> 1)) ^ (row & 7)) << 4) + ((t & 1) << 3));
+  return r;
+}
+
+// a stage = two weight boxes + the activation tile, padded so that every stage (and with it
+// every swizzled box) starts on a 1024-byte boundary
+__host__ __device__ constexpr int stage_bytes_for(int nt) { return 2 * TMA_BOX_BYTES + (nt * 8 * TMA_XROW_MAX + 1023) / 1024 * 1024; }
+
+struct TmaArgs {
+  int phase;
+  LayerDims L;
+  const ExpertDev* experts;
+  const CUtensorMap* tmaps;  // [E][3]
+  const __nv_bfloat16* in;
+  const int32_t* off;
+  int* plan;  // [0] activated experts, [1 + phase] item counter, [4...] their ids, widest codes first
+  __nv_bfloat16* hidden;
+  float* o_part;
+  int ksplit;
+  int row_blocks;
+  int n_pairs;
+  int* check_word;
+};
+
+// what a stage holds, written by the producer before it arms the stage's barrier
+struct StageMeta {
+  int e, rb, z, begin, p0, ntok, k0, bits;
+  int flags;  // 1 = first stage of an item pass, 2 = last, 4 = no more work, 8 = stage carries no inputs
+  int pad;
+  const void* scales[2];  // scale channel of the matrix behind each m-tile
+};
+constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8;
+
+template <int BITS, int NT>
+__device__ __forceinline__ void consume_stage(const TmaArgs& a, const StageMeta& m, const unsigned char* st, int warp,
+                                              int lane, float (&tot)[2][NT][4]) {
+  constexpr int KSPAN = 1024 / BITS;  // inputs per stage (128 bytes of a row)
+  constexpr int SEGS = KSPAN / 128;   // scale segments per stage
+  const LayerDims& L = a.L;
+  const int N = a.phase == 0 ? L.d_ff : L.d_model;
+  const int K = a.phase == 0 ? L.d_model : L.d_ff;
+  const int G = L.group > 0 ? L.group : K;
+  const int ngroups = K / G;
+  const bool swiglu_in = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const bool sf16 = L.scale_f16 != 0;
+  const int g = lane >> 2, t = lane & 3;
+  const int gp = box_row_of<BITS>(g);
+  const unsigned char* xt = st + 2 * TMA_BOX_BYTES;
+  const int nseg = min(SEGS, (K - m.k0) / 128);
+
+  int box_of[2], brow_of[2], nrow_of[2];
+#pragma unroll
+  for (int mt = 0; mt < 2; ++mt) {
+    if (swiglu_in) {
+      box_of[mt] = mt;
+      brow_of[mt] = 16 * warp;
+      nrow_of[mt] = m.rb * TMA_BOX_ROWS + 16 * warp;
+    } else {
+      box_of[mt] = warp >> 1;
+      brow_of[mt] = 32 * (warp & 1) + 16 * mt;
+      nrow_of[mt] = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt;
+    }
+  }
+  // all scales of the stage first, so that their latency hides behind the unpack work
+  float sc[SEGS][2][2];
+#pragma unroll
+  for (int sg = 0; sg < SEGS; ++sg)
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int n = min(nrow_of[mt] + gp + 8 * h, N - 1);
+        const int grp = min((m.k0 + sg * 128) / G, ngroups - 1);
+        sc[sg][mt][h] = load_scale_ro(m.scales[mt], sf16, static_cast<size_t>(n) * ngroups + grp);
+      }
+#pragma unroll
+  for (int sg = 0; sg < SEGS; ++sg) {
+    if (sg < nseg) {
+      // B fragments: piece q of lane t sits at (q*4 + t) * 16 bytes of the segment
+      uint4 bq[NT][4];
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        if (nt * 8 < m.ntok) {
+          const unsigned char* src = xt + (nt * 8 + g) * TMA_XROW_MAX + sg * 256 + t * 16;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) bq[nt][q] = *reinterpret_cast<const uint4*>(src + q * 64);
+        }
+      }
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const unsigned char* box = st + box_of[mt] * TMA_BOX_BYTES;
+        const int r0 = brow_of[mt] + gp, r1 = r0 + 8;
+        uint32_t P0[16], P1[16];
+        unpack(lds_raw<BITS>(box, r0, sg, t), P0);
+        unpack(lds_raw<BITS>(box, r1, sg, t), P1);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          if (nt * 8 < m.ntok) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              mma_bf16(acc, P0[4 * q], P1[4 * q], P0[4 * q + 1], P1[4 * q + 1], bq[nt][q].x, bq[nt][q].y);
+              mma_bf16(acc, P0[4 * q + 2], P1[4 * q + 2], P0[4 * q + 3], P1[4 * q + 3], bq[nt][q].z, bq[nt][q].w);
+            }
+            tot[mt][nt][0] = fmaf(sc[sg][mt][0], acc[0], tot[mt][nt][0]);
+            tot[mt][nt][1] = fmaf(sc[sg][mt][0], acc[1], tot[mt][nt][1]);
+            tot[mt][nt][2] = fmaf(sc[sg][mt][1], acc[2], tot[mt][nt][2]);
+            tot[mt][nt][3] = fmaf(sc[sg][mt][1], acc[3], tot[mt][nt][3]);
+          }
+        }
+      }
+    }
+  }
+}
+
+// results of one item pass: lane holds rows (gp, gp+8) x tokens (2t, 2t+1) of every tile
+template <int BITS, int NT>
+__device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m, int warp, int lane,
+                                           const float (&tot)[2][NT][4]) {
+  const LayerDims& L = a.L;
+  const int N = a.phase == 0 ? L.d_ff : L.d_model;
+  const bool swiglu_in = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const int g = lane >> 2, t = lane & 3;
+  const int gp = box_row_of<BITS>(g);
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int tok = nt * 8 + 2 * t + (i & 1);
+      if (tok >= m.ntok) continue;
+      const size_t slot = static_cast<size_t>(m.begin + m.p0 + tok);
+      if (swiglu_in) {
+        const int n = m.rb * TMA_BOX_ROWS + 16 * warp + gp + 8 * (i >> 1);
+        if (n < N) {
+          const float av = tot[0][nt][i], bv = tot[1][nt][i];
+          a.hidden[slot * N + act_pos<BITS>(n)] = __float2bfloat16_rn(av / (1.0f + expf(-av)) * bv);
+        }
+      } else {
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
+          if (n >= N) continue;
+          if (a.phase == 0)
+            a.hidden[slot * N + act_pos<BITS>(n)] = __float2bfloat16_rn(fmaxf(tot[mt][nt][i], 0.0f));
+          else
+            a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + slot) * N + n] = tot[mt][nt][i];
+        }
+      }
+    }
+  }
+}
+
+template <int NT>
+__host__ __device__ constexpr int stages_for() { return NT == 4 ? 3 : 4; }
+
+template <int NT>
+__host__ __device__ constexpr int smem_bytes_for() {
+  return stages_for<NT>() * stage_bytes_for(NT) + 1024;  // + slack to align the base to 1024
+}
+
+template <int NT>
+__global__ void __launch_bounds__(TMA_THREADS) ffn_tma_kernel(const TmaArgs a) {
+  constexpr int STAGES = stages_for<NT>();
+  constexpr int STAGE_BYTES = stage_bytes_for(NT);
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES];
+  __shared__ __align__(16) StageMeta meta[STAGES];
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(bars + s), 1);                            // full: the producer's arrival (+ copy bytes)
+      mbar_init(smem_u32(bars + STAGES + s), TMA_CONSUMER_WARPS);  // empty: one arrival per consumer warp
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // Token rows of a stage that no copy fills keep whatever shared memory held.  That is
+  // harmless: a column of the MMA result depends only on its own column of B, and columns past
+  // the expert's token count are never stored.
+  __syncthreads();
+
+  const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + STAGES);
+  const LayerDims& L = a.L;
+  const int K = a.phase == 0 ? L.d_model : L.d_ff;
+  const bool swiglu_in = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const int mat_first = a.phase == 0 ? 0 : (L.act == EMOE_ACT_SWIGLU ? 2 : 1);
+  const int rows_per_item = swiglu_in ? TMA_BOX_ROWS : 2 * TMA_BOX_ROWS;
+
+  if (warp == TMA_CONSUMER_WARPS) {
+    // ---------------- producer warp ----------------
+    const int n_items = a.plan[0] * a.row_blocks * a.ksplit;
+    int it = 0;
+    bool ok = true;
+    while (ok) {
+      int item = 0;
+      if (lane == 0) item = atomicAdd(a.plan + 1 + a.phase, 1);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      if (item >= n_items || *abort_flag) break;
+      const int z = item % a.ksplit;
+      const int rb = (item / a.ksplit) % a.row_blocks;
+      const int e = a.plan[4 + item / (a.ksplit * a.row_blocks)];
+      const int begin = a.off[e];
+      const int cnt = a.off[e + 1] - begin;
+      const ExpertDev ex = a.experts[e];
+      const CUtensorMap* maps = a.tmaps + static_cast<size_t>(e) * 3;
+      const int bits = ex.bits;
+      const int kspan = 1024 / bits;
+      const int steps_total = (K + kspan - 1) / kspan;
+      const int spz = (steps_total + a.ksplit - 1) / a.ksplit;
+      const int step_begin = z * spz;
+      const int nsteps = max(0, min(steps_total, step_begin + spz) - step_begin);
+      const int npass = (cnt + NT * 8 - 1) / (NT * 8);
+      const int row0 = rb * rows_per_item;
+      for (int pass = 0; pass < npass && ok; ++pass) {
+        const int p0 = pass * NT * 8;
+        const int ntok = min(NT * 8, cnt - p0);
+        const int nst = max(nsteps, 1);  // an empty split-K slice still has to store its zeros
+        for (int s = 0; s < nst; ++s, ++it) {
+          const int stage = it % STAGES;
+          const uint32_t par = (it / STAGES) & 1;
+          if (!mbar_wait(bar_empty + 8 * stage, par ^ 1, a.check_word, abort_flag)) {
+            ok = false;
+            break;
+          }
+          unsigned char* st = smem + stage * STAGE_BYTES;
+          const uint32_t full = bar_full + 8 * stage;
+          const int k0 = (step_begin + s) * kspan;
+          const int klen = nsteps > 0 ? min(kspan, K - k0) : 0;
+          if (lane == 0) {
+            StageMeta& m = meta[stage];
+            m.e = e; m.rb = rb; m.z = z; m.begin = begin; m.p0 = p0; m.ntok = ntok; m.k0 = k0; m.bits = bits;
+            m.flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0);
+            m.scales[0] = ex.scales[swiglu_in ? 0 : mat_first];
+            m.scales[1] = ex.scales[swiglu_in ? 1 : mat_first];
+            if (klen > 0) {
+              mbar_expect_tx(full, 2 * TMA_BOX_BYTES + ntok * klen * 2);
+              const int c0 = k0 * bits / 8;
+              if (swiglu_in) {
+                tma_load_2d(smem_u32(st), maps + 0, c0, row0, full);
+                tma_load_2d(smem_u32(st + TMA_BOX_BYTES), maps + 1, c0, row0, full);
+              } else {
+                tma_load_2d(smem_u32(st), maps + mat_first, c0, row0, full);
+                tma_load_2d(smem_u32(st + TMA_BOX_BYTES), maps + mat_first, c0, row0 + TMA_BOX_ROWS, full);
+              }
+            } else {
+              mbar_arrive(full);
+            }
+          }
+          __syncwarp();
+          if (klen > 0)
+            for (int r = lane; r < ntok; r += 32)
+              bulk_load(smem_u32(st + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
+                        a.in + static_cast<size_t>(begin + p0 + r) * K + k0, klen * 2, full);
+        }
+      }
+    }
+    if (ok && !*abort_flag) {  // tell the consumers that nothing else comes
+      const int stage = it % STAGES;
+      const uint32_t par = (it / STAGES) & 1;
+      if (mbar_wait(bar_empty + 8 * stage, par ^ 1, a.check_word, abort_flag) && lane == 0) {
+        meta[stage].flags = META_STOP;
+        mbar_arrive(bar_full + 8 * stage);
+      }
+    }
+  } else {
+    // ---------------- consumer warps ----------------
+    float tot[2][NT][4];
+    for (int it = 0;; ++it) {
+      const int stage = it % STAGES;
+      const uint32_t par = (it / STAGES) & 1;
+      if (!mbar_wait(bar_full + 8 * stage, par, a.check_word, abort_flag)) break;
+      const StageMeta m = meta[stage];
+      if (m.flags & META_STOP) break;
+      if (m.flags & META_FIRST) {
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) tot[mt][nt][i] = 0.0f;
+      }
+      const unsigned char* st = smem + stage * STAGE_BYTES;
+      if (!(m.flags & META_EMPTY)) {
+        switch (m.bits) {
+          case 2: consume_stage<2, NT>(a, m, st, warp, lane, tot); break;
+          case 4: consume_stage<4, NT>(a, m, st, warp, lane, tot); break;
+          default: consume_stage<8, NT>(a, m, st, warp, lane, tot); break;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
+      if (m.flags & META_LAST) {
+        switch (m.bits) {
+          case 2: store_item<2, NT>(a, m, warp, lane, tot); break;
+          case 4: store_item<4, NT>(a, m, warp, lane, tot); break;
+          default: store_item<8, NT>(a, m, warp, lane, tot); break;
+        }
+      }
+    }
+  }
+  if (*abort_flag) {
+    // a wait ran out: give copies that may still be in flight time to land before the CTA's
+    // shared memory is released
+    for (int i = 0; i < 2000; ++i) __nanosleep(100);
+  }
+}
+
+template <int NT>
+cudaError_t launch_nt(const TmaArgs& a, int max_items, cudaStream_t st) {
+  constexpr int SMEM = smem_bytes_for<NT>();
+  static int ctas_per_device[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!ctas_per_device[dev]) {
+    e = cudaFuncSetAttribute(ffn_tma_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0, sms = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ffn_tma_kernel<NT>, TMA_THREADS, SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    ctas_per_device[dev] = (per_sm > 0 ? per_sm : 1) * sms;
+  }
+  const int grid = max_items < ctas_per_device[dev] ? max_items : ctas_per_device[dev];
+  ffn_tma_kernel<NT><<<grid, TMA_THREADS, SMEM, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool ffn_tma_supported(const LayerDims& L) {
+  // tensor maps use 128-byte x 64-row boxes: every packed row must hold at least 128 bytes at
+  // the narrowest width (2 bits)
+  return ffn_mma_supported(L) && L.d_model >= 512 && L.d_ff >= 512;
+}
+
+int ffn_tma_ksplit(const LayerDims& L, int T) {
+  const int row_blocks = (L.d_model + 2 * TMA_BOX_ROWS - 1) / (2 * TMA_BOX_ROWS);
+  const long long pairs = static_cast<long long>(T) * L.top_k;
+  const long long active = pairs < L.E ? pairs : L.E;
+  const long long ctas = row_blocks * active;
+  const int steps_min = (L.d_ff + 511) / 512;  // stages at the widest span (2 bits)
+  long long z = (4 * 148 + ctas - 1) / ctas;
+  if (z > steps_min) z = steps_min;
+  if (z > 16) z = 16;
+  if (z < 1) z = 1;
+  return static_cast<int>(z);
+}
+
+cudaError_t launch_ffn_tma(int phase, const LayerDims& L, const ExpertDev* experts, const void* tmaps,
+                           const __nv_bfloat16* in, const int32_t* off, int* plan, __nv_bfloat16* hidden, float* o_part,
+                           int ksplit, int n_pairs, int T, int* check_word, cudaStream_t st) {
+  const int N = phase == 0 ? L.d_ff : L.d_model;
+  const int rows_per_item = (phase == 0 && L.act == EMOE_ACT_SWIGLU) ? TMA_BOX_ROWS : 2 * TMA_BOX_ROWS;
+  TmaArgs a;
+  a.phase = phase;
+  a.L = L;
+  a.experts = experts;
+  a.tmaps = static_cast<const CUtensorMap*>(tmaps);
+  a.in = in;
+  a.off = off;
+  a.plan = plan;
+  a.hidden = hidden;
+  a.o_part = o_part;
+  a.ksplit = phase == 0 ? 1 : ksplit;
+  a.row_blocks = (N + rows_per_item - 1) / rows_per_item;
+  a.n_pairs = n_pairs;
+  a.check_word = check_word;
+  const long long active_max = n_pairs < L.E ? n_pairs : L.E;
+  const long long items = active_max * a.row_blocks * a.ksplit;
+  const int max_items = items > (1 << 30) ? (1 << 30) : static_cast<int>(items);
+  const int nt = ffn_token_tiles(L, T);
+  if (nt == 1) return launch_nt<1>(a, max_items, st);
+  if (nt == 2) return launch_nt<2>(a, max_items, st);
+  return launch_nt<4>(a, max_items, st);
+}
+
+// One tensor map per packed matrix: a [N][row_bytes] byte image, 64-row x 128-byte boxes, 128-byte swizzle.
+int encode_weight_tmap(void* out_map, const void* packed, int N, int K, int bits) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || !p) return -1;
+    fn = reinterpret_cast<EncodeFn>(p);
+  }
+  const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * bits / 8;
+  if (row_bytes < 128 || row_bytes % 16 != 0 || N < TMA_BOX_ROWS) return -2;
+  const cuuint64_t dims[2] = {row_bytes, static_cast<cuuint64_t>(N)};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {128, TMA_BOX_ROWS};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(static_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(packed), dims,
+                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -3;
+}
+
+}  // namespace emoe

@@ -77,12 +77,39 @@ def test_forward_tensor_core_path(act, group, sdt, d, f, E, k, gate, bits, T):
     _run_case(shape, bits, T, seed=22, path=2)
 
 
+TMA_CASES = [
+    ("relu", 128, "f16", 768, 3072, 8, 1, "softmax", [8, 4, 2, 4, 8, 2, 4, 8], 64),   # 1.5 stages at 2 bits
+    ("relu", 128, "f16", 768, 3072, 8, 1, "softmax", [2, 2, 4, 4, 8, 8, 2, 4], 5),    # one 8-token tile
+    ("relu", 0, "f16", 512, 1152, 4, 2, "softmax_renorm", [4, 2, 8, 2], 9),           # per-channel scales, 16-token tiles
+    ("relu", 128, "f32", 640, 1664, 3, 1, "softmax", [8, 2, 4], 37),                  # K tails at every width, two passes
+    ("swiglu", 128, "f16", 512, 1408, 4, 2, "softmax_renorm", [4, 8, 2, 4], 16),
+    ("swiglu", 256, "f16", 1024, 2560, 8, 2, "softmax_renorm", [4, 4, 8, 2, 4, 8, 2, 4], 33),
+    ("swiglu", 128, "f16", 512, 512, 2, 2, "softmax", [2, 8], 1),
+    ("relu", 128, "f16", 512, 8704, 2, 1, "softmax", [4, 2], 3),                      # long K: split-K and many ring wraps
+]
+
+
+@pytest.mark.parametrize("act,group,sdt,d,f,E,k,gate,bits,T", TMA_CASES)
+def test_forward_tma_pipeline_path(act, group, sdt, d, f, E, k, gate, bits, T):
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, "bf16")
+    _run_case(shape, bits, T, seed=25, path=3)
+
+
+def test_tma_path_is_refused_for_narrow_rows():
+    shape = inputs.LayerShape(256, 512, 4, 1, "relu", "softmax", 128, "f16", "bf16")
+    with pytest.raises(B.EmoeError) as ei:
+        _run_case(shape, [2, 4, 8, 4], 4, seed=26, path=3)
+    assert ei.value.status == B.ERR_UNSUPPORTED
+
+
 def test_both_paths_agree_and_default_picks_tensor_cores():
     shape = inputs.LayerShape(256, 512, 4, 2, "swiglu", "softmax_renorm", 128, "f16", "bf16")
     e_auto = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=0)
     e_gemv = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=1)
     e_mma = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=2)
     assert e_auto == e_mma and e_gemv <= 2e-3
+    big = inputs.LayerShape(512, 1024, 4, 2, "swiglu", "softmax_renorm", 128, "f16", "bf16")
+    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=0) == _run_case(big, [2, 4, 8, 4], 12, seed=23, path=3)
 
 
 def test_zipf_bias_and_many_tokens_on_one_expert():
@@ -92,6 +119,8 @@ def test_zipf_bias_and_many_tokens_on_one_expert():
     bias[5] = 30.0
     for path in (1, 2):
         _run_case(shape, [2, 4, 8, 4, 2, 4, 8, 2], 70, seed=24, path=path, bias=bias)
+    wide = inputs.LayerShape(512, 1024, 8, 1, "relu", "softmax", 128, "f16", "bf16")
+    _run_case(wide, [2, 4, 8, 4, 2, 4, 8, 2], 70, seed=24, path=3, bias=bias)
 
 
 def test_forward_routed_and_unselected_experts():
