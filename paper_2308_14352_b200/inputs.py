@@ -173,22 +173,23 @@ def zipf_targets(n_experts: int, s: float) -> np.ndarray:
     return p / p.sum()
 
 
-def zipf_router_bias(x: np.ndarray, Wr: np.ndarray, s: float, iters: int = 200, eta: float = 0.5) -> np.ndarray:
-    """Additive per-expert router bias that makes the realised top-1 loads of the
-    seeded batch x follow Zipf(s).  This shapes an *input* (the bias vector); the
-    layer under test recomputes its own logits from x, Wr and this bias."""
+def zipf_router_bias(x: np.ndarray, Wr: np.ndarray, s: float, iters: int = 400, eta: float = 0.1) -> np.ndarray:
+    """Additive per-expert router bias that makes the realised top-1 loads of the seeded batch x
+    follow Zipf(s).  Damped fixed-point iteration b += eta * (log target - log observed); the
+    iterate with the smallest worst-case load error is kept.  This shapes an *input* (the bias
+    vector); the layer under test recomputes its own logits from x, Wr and this bias."""
     T, E = x.shape[0], Wr.shape[1]
     z = x.astype(np.float64) @ Wr.astype(np.float64)
-    target = zipf_targets(E, s)
-    b = np.log(target)
+    target = zipf_targets(E, s) * T
+    b = np.log(target / T)
+    best, best_err = b.copy(), np.inf
     for _ in range(iters):
         load = np.bincount(np.argmax(z + b, axis=1), minlength=E).astype(np.float64)
-        obs = (load + 0.5) / (T + 0.5 * E)
-        step = np.log(target) - np.log(obs)
-        if np.max(np.abs(load / T - target)) < 0.5 / T:
-            break
-        b = b + eta * step
-    return b.astype(np.float32)
+        err = np.max(np.abs(load - target))
+        if err < best_err:
+            best, best_err = b.copy(), err
+        b = b + eta * (np.log(target + 0.5) - np.log(load + 0.5))
+    return best.astype(np.float32)
 
 
 def transition_prior(seed: int, n_experts: int, concentration: float = 0.3) -> np.ndarray:
