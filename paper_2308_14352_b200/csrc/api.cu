@@ -67,7 +67,7 @@ WorkspaceLayout make_layout(const LayerDims& L, int T) {
   w.off = o;          o += align_up(static_cast<size_t>(L.E + 1) * 4);
   w.perm = o;         o += align_up(P * 4);
   w.slot_of_pair = o; o += align_up(P * 4);
-  w.plan = o;         o += align_up(static_cast<size_t>(L.E + 4) * 4);
+  w.plan = o;         o += align_up(plan_bytes(L.E));
   w.xs = o;           o += align_up(L.act_bf16 ? P * L.d_model * 2 : 0);
   w.hidden = o;       o += align_up(P * L.d_ff * (L.act_bf16 ? 2 : 4));
   w.o_part = o;       o += align_up(static_cast<size_t>(w.ksplit) * P * L.d_model * 4);

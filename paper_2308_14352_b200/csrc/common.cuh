@@ -23,6 +23,17 @@ enum : int {
   CHECK_WAIT_TIMEOUT = 2,  // a bounded wait inside a kernel ran out
 };
 
+// Work plan of the persistent expert kernels, built on the device after the permutation:
+// a 16-byte header {activated experts, item counter of the first projection, of the second, 0}
+// followed by one record per activated expert, widest codes first.
+struct PlanRec {
+  int32_t e, begin, cnt, bits;
+  const void* scales[3];
+  int64_t pad;
+};
+constexpr size_t PLAN_HEADER_BYTES = 16;
+inline size_t plan_bytes(int E) { return PLAN_HEADER_BYTES + sizeof(PlanRec) * static_cast<size_t>(E); }
+
 struct LayerDims {
   int d_model, d_ff, E, top_k, act, gate_mode, group, scale_f16, act_bf16;
 };
@@ -52,7 +63,7 @@ cudaError_t launch_ffn_gemv(int phase, const LayerDims& L, const ExpertDev* expe
 bool ffn_mma_supported(const LayerDims& L);
 int ffn_mma_ksplit(const LayerDims& L, int T);
 int ffn_token_tiles(const LayerDims& L, int T);
-// plan (nullable): int[4 + E] work plan for the persistent TMA kernels, filled by block 0.
+// plan (nullable): plan_bytes(E) bytes, the work plan for the persistent TMA kernels, filled by block 0.
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
                              cudaStream_t st);

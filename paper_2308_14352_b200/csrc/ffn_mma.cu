@@ -210,13 +210,23 @@ __global__ void __launch_bounds__(128)
     // work plan of the persistent expert kernels: activated experts, widest codes (most bytes)
     // first; the two item counters restart from zero
     const int lane = threadIdx.x;
+    PlanRec* recs = reinterpret_cast<PlanRec*>(reinterpret_cast<char*>(plan) + PLAN_HEADER_BYTES);
     int base = 0;
     for (int b = 8; b >= 2; b >>= 1) {
       for (int e0 = 0; e0 < E; e0 += 32) {
         const int e = e0 + lane;
         const bool act = e < E && off[e + 1] > off[e] && experts[e].bits == b;
         const unsigned m = __ballot_sync(0xffffffffu, act);
-        if (act) plan[4 + base + __popc(m & ((1u << lane) - 1u))] = e;
+        if (act) {
+          PlanRec& r = recs[base + __popc(m & ((1u << lane) - 1u))];
+          r.e = e;
+          r.begin = off[e];
+          r.cnt = off[e + 1] - off[e];
+          r.bits = b;
+          r.scales[0] = experts[e].scales[0];
+          r.scales[1] = experts[e].scales[1];
+          r.scales[2] = experts[e].scales[2];
+        }
         base += __popc(m);
       }
     }

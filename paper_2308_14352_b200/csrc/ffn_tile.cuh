@@ -36,7 +36,7 @@ __device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t 
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t a0, const uint32_t a1, const uint32_t a2,
                                          const uint32_t a3, const uint32_t b0, const uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -126,6 +126,42 @@ __device__ __forceinline__ void unpack(const Raw<2>& raw, uint32_t (&P)[16]) {
       const uint32_t v = and_xor(w[i] >> sh, msk[p], mag[p]);
       P[8 * i + c] = bf16x2_fma(v, mul[p], add[p]);
     }
+  }
+}
+
+// One k16-pair step of the unpack: the four registers (code pairs 4q .. 4q+3 of the lane's
+// row) that feed the two MMAs of step q, so that a tile can be consumed step by step without
+// holding all 16 registers of a row at once.
+__device__ __forceinline__ void unpack_step(const Raw<8>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[8] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w, raw.v[1].x, raw.v[1].y, raw.v[1].z, raw.v[1].w};
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const uint32_t u = w[2 * q + j] ^ 0x80808080u;
+    const float f0 = __uint_as_float(prmt(u, 0x4B000000u, 0x7540u)) - 8388736.0f;
+    const float f1 = __uint_as_float(prmt(u, 0x4B000000u, 0x7541u)) - 8388736.0f;
+    const float f2 = __uint_as_float(prmt(u, 0x4B000000u, 0x7542u)) - 8388736.0f;
+    const float f3 = __uint_as_float(prmt(u, 0x4B000000u, 0x7543u)) - 8388736.0f;
+    o[2 * j] = prmt(__float_as_uint(f0), __float_as_uint(f1), 0x7632u);
+    o[2 * j + 1] = prmt(__float_as_uint(f2), __float_as_uint(f3), 0x7632u);
+  }
+}
+__device__ __forceinline__ void unpack_step(const Raw<4>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[4] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w};
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+    o[c] = bf16x2_fma(and_xor(w[q] >> (4 * c), 0x000F000Fu, 0x43084308u), 0x3F803F80u, 0xC308C308u);
+}
+__device__ __forceinline__ void unpack_step(const Raw<2>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[2] = {raw.v[0].x, raw.v[0].y};
+  const uint32_t mul[3] = {0x3F803F80u, 0x3E803E80u, 0x3D803D80u};
+  const uint32_t add[3] = {0xC302C302u, 0xC208C208u, 0xC120C120u};
+  const uint32_t msk[3] = {0x00030003u, 0x000C000Cu, 0x00300030u};
+  const uint32_t mag[3] = {0x43024302u, 0x43084308u, 0x43204320u};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = 4 * (q & 1) + j;
+    const int sh = 6 * (c / 3), p = c % 3;
+    o[j] = bf16x2_fma(and_xor(w[q >> 1] >> sh, msk[p], mag[p]), mul[p], add[p]);
   }
 }
 

@@ -16,8 +16,12 @@
 //     swizzle, so that the consumers' 128-bit reads are conflict free), the matching slice of
 //     the expert's activations, fetched by one bulk copy per token row, and a small record
 //     that tells the consumers which item and which inputs the stage belongs to;
+//   * the producer's lanes also start small asynchronous copies (cp.async) of the stage's
+//     scales (128 rows x up to 4 segments, 16 bytes per row) that complete on the same
+//     mbarrier, so that no warp ever waits on a global load of a scale;
 //   * four consumer warps wait on the stage's mbarrier, read their 16-row tiles from shared
-//     memory, unpack, issue the MMAs, and hand the stage back through a second mbarrier.
+//     memory, unpack step by step, issue the MMAs, and hand the stage back through a second
+//     mbarrier.
 // 128 bytes of a row are 128 / 256 / 512 inputs at 8 / 4 / 2 bits, so a stage covers 1 / 2 / 4
 // scale segments.  Every wait is bounded: a wait that runs out sets a bit in the context's
 // check word and the CTA winds down without touching the stage.
@@ -30,10 +34,17 @@ namespace emoe {
 namespace {
 
 constexpr int TMA_CONSUMER_WARPS = 4;
-constexpr int TMA_THREADS = (TMA_CONSUMER_WARPS + 1) * 32;
+constexpr int TMA_THREADS = (TMA_CONSUMER_WARPS + 1) * 32;  // + the producer warp
+constexpr int TMA_SCALE_BYTES = 128 * 16;                   // raw scales of a stage: 16 bytes per row
 constexpr int TMA_BOX_ROWS = 64;
 constexpr int TMA_BOX_BYTES = TMA_BOX_ROWS * 128;  // 8 KB
 constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a stage (row stride = 64 mod 128)
+#ifndef EMOE_TMA_STAGES_NT1
+#define EMOE_TMA_STAGES_NT1 3
+#endif
+#ifndef EMOE_TMA_CTAS_NT1
+#define EMOE_TMA_CTAS_NT1 2
+#endif
 constexpr unsigned WAIT_LIMIT = 1u << 22;          // polls before a wait gives up (~0.2 s)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -115,7 +126,20 @@ __device__ __forceinline__ Raw<2> lds_raw<2>(const unsigned char* box, int row, 
 
 // a stage = two weight boxes + the activation tile, padded so that every stage (and with it
 // every swizzled box) starts on a 1024-byte boundary
-__host__ __device__ constexpr int stage_bytes_for(int nt) { return 2 * TMA_BOX_BYTES + (nt * 8 * TMA_XROW_MAX + 1023) / 1024 * 1024; }
+__host__ __device__ constexpr int stage_bytes_for(int nt) {
+  return 2 * TMA_BOX_BYTES + (nt * 8 * TMA_XROW_MAX + TMA_SCALE_BYTES + 1023) / 1024 * 1024;
+}
+__host__ __device__ constexpr int scale_tile_offset(int nt) { return 2 * TMA_BOX_BYTES + nt * 8 * TMA_XROW_MAX; }
+
+// The scales a stage needs from row n (groups of inputs k0 .. k0 + 128*segs) sit in one short
+// byte window of the scale channel; it is copied from its 4-byte-aligned start.
+__device__ __forceinline__ int scale_window_begin(int n, int ngroups, int g0, int ssz) {
+  return ((n * ngroups + g0) * ssz) & ~3;
+}
+// group index of input k (groups of G inputs, G a multiple of 128 or the whole row)
+__device__ __forceinline__ int group_of(int k, int G, int ngroups) {
+  return ngroups == 1 ? 0 : (G == 128 ? (k >> 7) : k / G);
+}
 
 struct TmaArgs {
   int phase;
@@ -124,7 +148,7 @@ struct TmaArgs {
   const CUtensorMap* tmaps;  // [E][3]
   const __nv_bfloat16* in;
   const int32_t* off;
-  int* plan;  // [0] activated experts, [1 + phase] item counter, [4...] their ids, widest codes first
+  int* plan;  // header {activated experts, item counters} + one PlanRec per activated expert
   __nv_bfloat16* hidden;
   float* o_part;
   int ksplit;
@@ -143,47 +167,24 @@ struct StageMeta {
 constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8;
 
 template <int BITS, int NT>
-__device__ __forceinline__ void consume_stage(const TmaArgs& a, const StageMeta& m, const unsigned char* st, int warp,
-                                              int lane, float (&tot)[2][NT][4]) {
+__device__ __forceinline__ void consume_stage(const TmaArgs& a, int rb, int k0, int ntok, const unsigned char* st,
+                                              int warp, int lane, uint32_t bar_empty, float (&tot)[2][NT][4]) {
   constexpr int KSPAN = 1024 / BITS;  // inputs per stage (128 bytes of a row)
   constexpr int SEGS = KSPAN / 128;   // scale segments per stage
   const LayerDims& L = a.L;
-  const int N = a.phase == 0 ? L.d_ff : L.d_model;
   const int K = a.phase == 0 ? L.d_model : L.d_ff;
-  const int G = L.group > 0 ? L.group : K;
-  const int ngroups = K / G;
   const bool swiglu_in = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
-  const bool sf16 = L.scale_f16 != 0;
   const int g = lane >> 2, t = lane & 3;
   const int gp = box_row_of<BITS>(g);
   const unsigned char* xt = st + 2 * TMA_BOX_BYTES;
-  const int nseg = min(SEGS, (K - m.k0) / 128);
-
-  int box_of[2], brow_of[2], nrow_of[2];
-#pragma unroll
-  for (int mt = 0; mt < 2; ++mt) {
-    if (swiglu_in) {
-      box_of[mt] = mt;
-      brow_of[mt] = 16 * warp;
-      nrow_of[mt] = m.rb * TMA_BOX_ROWS + 16 * warp;
-    } else {
-      box_of[mt] = warp >> 1;
-      brow_of[mt] = 32 * (warp & 1) + 16 * mt;
-      nrow_of[mt] = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt;
-    }
-  }
-  // all scales of the stage first, so that their latency hides behind the unpack work
-  float sc[SEGS][2][2];
-#pragma unroll
-  for (int sg = 0; sg < SEGS; ++sg)
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int n = min(nrow_of[mt] + gp + 8 * h, N - 1);
-        const int grp = min((m.k0 + sg * 128) / G, ngroups - 1);
-        sc[sg][mt][h] = load_scale_ro(m.scales[mt], sf16, static_cast<size_t>(n) * ngroups + grp);
-      }
+  const unsigned char* sct = st + scale_tile_offset(NT);
+  const int N = a.phase == 0 ? L.d_ff : L.d_model;
+  const int G = L.group > 0 ? L.group : K;
+  const int ngroups = K / G;
+  const int ssz = L.scale_f16 ? 2 : 4;
+  const int nrow0 = swiglu_in ? rb * TMA_BOX_ROWS + 16 * warp : rb * 2 * TMA_BOX_ROWS + 32 * warp;
+  const int nseg = min(SEGS, (K - k0) / 128);
+  const int g0 = group_of(k0, G, ngroups);
 #pragma unroll
   for (int sg = 0; sg < SEGS; ++sg) {
     if (sg < nseg) {
@@ -191,37 +192,68 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, const StageMeta&
       uint4 bq[NT][4];
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
-        if (nt * 8 < m.ntok) {
+        if (nt * 8 < ntok) {
           const unsigned char* src = xt + (nt * 8 + g) * TMA_XROW_MAX + sg * 256 + t * 16;
 #pragma unroll
           for (int q = 0; q < 4; ++q) bq[nt][q] = *reinterpret_cast<const uint4*>(src + q * 64);
         }
       }
+      // one 16-row tile at a time, one k16-pair step at a time: the unpacked codes of a step
+      // live in 8 registers and go straight into the MMAs.  The k-steps alternate between two
+      // partial accumulators so that consecutive MMAs do not depend on each other.
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        const unsigned char* box = st + box_of[mt] * TMA_BOX_BYTES;
-        const int r0 = brow_of[mt] + gp, r1 = r0 + 8;
-        uint32_t P0[16], P1[16];
-        unpack(lds_raw<BITS>(box, r0, sg, t), P0);
-        unpack(lds_raw<BITS>(box, r1, sg, t), P1);
+        const int box_i = swiglu_in ? mt : (warp >> 1);
+        const int r0 = (swiglu_in ? 16 * warp : 32 * (warp & 1) + 16 * mt) + gp;
+        const unsigned char* box = st + box_i * TMA_BOX_BYTES;
+        const Raw<BITS> raw0 = lds_raw<BITS>(box, r0, sg, t);
+        const Raw<BITS> raw1 = lds_raw<BITS>(box, r0 + 8, sg, t);
+        float s0, s1;
+        {
+          const int n0 = min(nrow0 + (swiglu_in ? 0 : 16 * mt) + gp, N - 1), n1 = min(n0 + 8, N - 1);
+          const int grp = group_of(k0 + sg * 128, G, ngroups);
+          const unsigned char* w0 = sct + (box_i * TMA_BOX_ROWS + r0) * 16 + (n0 * ngroups + grp) * ssz -
+                                    scale_window_begin(n0, ngroups, g0, ssz);
+          const unsigned char* w1 = sct + (box_i * TMA_BOX_ROWS + r0 + 8) * 16 + (n1 * ngroups + grp) * ssz -
+                                    scale_window_begin(n1, ngroups, g0, ssz);
+          if (ssz == 2) {
+            s0 = __half2float(*reinterpret_cast<const __half*>(w0));
+            s1 = __half2float(*reinterpret_cast<const __half*>(w1));
+          } else {
+            s0 = *reinterpret_cast<const float*>(w0);
+            s1 = *reinterpret_cast<const float*>(w1);
+          }
+        }
+        float pa[NT][4], pb[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) pa[nt][i] = pb[nt][i] = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t c0[4], c1[4];
+          unpack_step(raw0, q, c0);
+          unpack_step(raw1, q, c1);
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            if (nt * 8 < ntok) {
+              mma_bf16(pa[nt], c0[0], c1[0], c0[1], c1[1], bq[nt][q].x, bq[nt][q].y);
+              mma_bf16(pb[nt], c0[2], c1[2], c0[3], c1[3], bq[nt][q].z, bq[nt][q].w);
+            }
+        }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          if (nt * 8 < m.ntok) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              mma_bf16(acc, P0[4 * q], P1[4 * q], P0[4 * q + 1], P1[4 * q + 1], bq[nt][q].x, bq[nt][q].y);
-              mma_bf16(acc, P0[4 * q + 2], P1[4 * q + 2], P0[4 * q + 3], P1[4 * q + 3], bq[nt][q].z, bq[nt][q].w);
-            }
-            tot[mt][nt][0] = fmaf(sc[sg][mt][0], acc[0], tot[mt][nt][0]);
-            tot[mt][nt][1] = fmaf(sc[sg][mt][0], acc[1], tot[mt][nt][1]);
-            tot[mt][nt][2] = fmaf(sc[sg][mt][1], acc[2], tot[mt][nt][2]);
-            tot[mt][nt][3] = fmaf(sc[sg][mt][1], acc[3], tot[mt][nt][3]);
-          }
+          tot[mt][nt][0] = fmaf(s0, pa[nt][0] + pb[nt][0], tot[mt][nt][0]);
+          tot[mt][nt][1] = fmaf(s0, pa[nt][1] + pb[nt][1], tot[mt][nt][1]);
+          tot[mt][nt][2] = fmaf(s1, pa[nt][2] + pb[nt][2], tot[mt][nt][2]);
+          tot[mt][nt][3] = fmaf(s1, pa[nt][3] + pb[nt][3], tot[mt][nt][3]);
         }
       }
     }
   }
+  // shared memory of the stage is no longer needed
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar_empty);
 }
 
 // results of one item pass: lane holds rows (gp, gp+8) x tokens (2t, 2t+1) of every tile
@@ -261,8 +293,12 @@ __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m,
   }
 }
 
+// ring depth and CTAs per SM by token-tile count: more, smaller CTAs when registers allow, so
+// that every scheduler has several consumer warps to switch between
 template <int NT>
-__host__ __device__ constexpr int stages_for() { return NT == 4 ? 3 : 4; }
+__host__ __device__ constexpr int stages_for() { return NT == 1 ? EMOE_TMA_STAGES_NT1 : 3; }
+template <int NT>
+__host__ __device__ constexpr int ctas_per_sm_for() { return NT == 1 ? EMOE_TMA_CTAS_NT1 : (NT == 2 ? 2 : 1); }
 
 template <int NT>
 __host__ __device__ constexpr int smem_bytes_for() {
@@ -270,11 +306,11 @@ __host__ __device__ constexpr int smem_bytes_for() {
 }
 
 template <int NT>
-__global__ void __launch_bounds__(TMA_THREADS) ffn_tma_kernel(const TmaArgs a) {
+__global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_kernel(const TmaArgs a) {
   constexpr int STAGES = stages_for<NT>();
   constexpr int STAGE_BYTES = stage_bytes_for(NT);
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * STAGES];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES];  // full, empty
   __shared__ __align__(16) StageMeta meta[STAGES];
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
@@ -284,7 +320,7 @@ __global__ void __launch_bounds__(TMA_THREADS) ffn_tma_kernel(const TmaArgs a) {
   if (threadIdx.x == 0) {
     abort_word = 0;
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(bars + s), 1);                            // full: the producer's arrival (+ copy bytes)
+      mbar_init(smem_u32(bars + s), 33);  // full: lane 0's arrival (+ bulk-copy bytes) and every lane's scale copies
       mbar_init(smem_u32(bars + STAGES + s), TMA_CONSUMER_WARPS);  // empty: one arrival per consumer warp
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -303,22 +339,38 @@ __global__ void __launch_bounds__(TMA_THREADS) ffn_tma_kernel(const TmaArgs a) {
 
   if (warp == TMA_CONSUMER_WARPS) {
     // ---------------- producer warp ----------------
-    const int n_items = a.plan[0] * a.row_blocks * a.ksplit;
+    const int n_active = *reinterpret_cast<volatile const int*>(a.plan);
+    const int n_items = n_active * a.row_blocks * a.ksplit;
+    const PlanRec* recs = reinterpret_cast<const PlanRec*>(reinterpret_cast<const char*>(a.plan) + PLAN_HEADER_BYTES);
+    const int Nrows = a.phase == 0 ? L.d_ff : L.d_model;
+    const int Gk = L.group > 0 ? L.group : K;
+    const int ngroups_k = K / Gk;
+    const int ssz = L.scale_f16 ? 2 : 4;
+    const int per_expert = a.ksplit * a.row_blocks;
     int it = 0;
     bool ok = true;
+    // Item look-ahead of two: the counter increment for item i+2 and the expert record of item
+    // i+1 are issued before item i is streamed and only read after it, so that switching items
+    // costs no round trip to memory.  A CTA's first item is its own index; the counter hands
+    // out the items after those.
+    int item_cur = blockIdx.x, item_next = 0;
+    if (lane == 0) item_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
+    PlanRec rec_cur = recs[min(item_cur / per_expert, L.E - 1)];  // read before n_items is known: same latency
+    item_next = __shfl_sync(0xffffffffu, item_next, 0);
     while (ok) {
-      int item = 0;
-      if (lane == 0) item = atomicAdd(a.plan + 1 + a.phase, 1);
-      item = __shfl_sync(0xffffffffu, item, 0);
+      const int item = item_cur;
       if (item >= n_items || *abort_flag) break;
+      const PlanRec rec = rec_cur;
+      int raw_after_next = 0;
+      if (lane == 0) raw_after_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
+      const PlanRec rec_next = recs[item_next < n_items ? item_next / per_expert : 0];
       const int z = item % a.ksplit;
       const int rb = (item / a.ksplit) % a.row_blocks;
-      const int e = a.plan[4 + item / (a.ksplit * a.row_blocks)];
-      const int begin = a.off[e];
-      const int cnt = a.off[e + 1] - begin;
-      const ExpertDev ex = a.experts[e];
+      const int e = rec.e;
+      const int begin = rec.begin;
+      const int cnt = rec.cnt;
       const CUtensorMap* maps = a.tmaps + static_cast<size_t>(e) * 3;
-      const int bits = ex.bits;
+      const int bits = rec.bits;
       const int kspan = 1024 / bits;
       const int steps_total = (K + kspan - 1) / kspan;
       const int spz = (steps_total + a.ksplit - 1) / a.ksplit;
@@ -345,8 +397,8 @@ __global__ void __launch_bounds__(TMA_THREADS) ffn_tma_kernel(const TmaArgs a) {
             StageMeta& m = meta[stage];
             m.e = e; m.rb = rb; m.z = z; m.begin = begin; m.p0 = p0; m.ntok = ntok; m.k0 = k0; m.bits = bits;
             m.flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0);
-            m.scales[0] = ex.scales[swiglu_in ? 0 : mat_first];
-            m.scales[1] = ex.scales[swiglu_in ? 1 : mat_first];
+            m.scales[0] = swiglu_in ? rec.scales[0] : rec.scales[mat_first];
+            m.scales[1] = swiglu_in ? rec.scales[1] : rec.scales[mat_first];
             if (klen > 0) {
               mbar_expect_tx(full, 2 * TMA_BOX_BYTES + ntok * klen * 2);
               const int c0 = k0 * bits / 8;
@@ -362,18 +414,59 @@ __global__ void __launch_bounds__(TMA_THREADS) ffn_tma_kernel(const TmaArgs a) {
             }
           }
           __syncwarp();
-          if (klen > 0)
+          if (klen > 0) {
             for (int r = lane; r < ntok; r += 32)
               bulk_load(smem_u32(st + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
                         a.in + static_cast<size_t>(begin + p0 + r) * K + k0, klen * 2, full);
+            // scales: lane l copies the windows of rows 4l .. 4l+3 of the stage (box-major)
+            const int nseg = klen / 128;
+            const int g0 = group_of(k0, Gk, ngroups_k), g1 = group_of(k0 + (nseg - 1) * 128, Gk, ngroups_k);
+            const uint32_t sdst = smem_u32(st + scale_tile_offset(NT));
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              const int row = 4 * lane + r;
+              const int n = min(swiglu_in ? row0 + (row & 63) : row0 + row, Nrows - 1);
+              const char* sp = static_cast<const char*>(swiglu_in ? rec.scales[row >> 6] : rec.scales[mat_first]);
+              const int b0 = scale_window_begin(n, ngroups_k, g0, ssz);
+              const int b1 = (n * ngroups_k + g1 + 1) * ssz;
+              for (int w = 0; b0 + 4 * w < b1; ++w)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + row * 16 + 4 * w), "l"(sp + b0 + 4 * w)
+                             : "memory");
+            }
+            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full) : "memory");
+          } else {
+            mbar_arrive(full);  // with lane 0's arrival above: 33 in all
+          }
+        }
+      }
+      item_cur = item_next;
+      rec_cur = rec_next;
+      item_next = __shfl_sync(0xffffffffu, raw_after_next, 0);
+      if (item_cur < n_items) {
+        // pull the next item's scale rows towards L2 while its codes are still far away
+        const int rbn = (item_cur / a.ksplit) % a.row_blocks;
+        const int Nn = a.phase == 0 ? L.d_ff : L.d_model;
+        const int ngroups = L.group > 0 ? K / L.group : 1;
+        const int ssz = L.scale_f16 ? 2 : 4;
+        const int rows = min(rows_per_item, Nn - rbn * rows_per_item);
+        const int lines = (rows * ngroups * ssz + 127) / 128;
+        const size_t offs = static_cast<size_t>(rbn) * rows_per_item * ngroups * ssz;
+        const int nm = swiglu_in ? 2 : 1;
+        for (int i = lane; i < nm * lines; i += 32) {
+          const char* base = static_cast<const char*>(rec_cur.scales[swiglu_in ? i / lines : mat_first]) + offs;
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(base + static_cast<size_t>(i % lines) * 128));
         }
       }
     }
     if (ok && !*abort_flag) {  // tell the consumers that nothing else comes
       const int stage = it % STAGES;
       const uint32_t par = (it / STAGES) & 1;
-      if (mbar_wait(bar_empty + 8 * stage, par ^ 1, a.check_word, abort_flag) && lane == 0) {
-        meta[stage].flags = META_STOP;
+      if (mbar_wait(bar_empty + 8 * stage, par ^ 1, a.check_word, abort_flag)) {
+        if (lane == 0) {
+          meta[stage].flags = META_STOP;
+          mbar_arrive(bar_full + 8 * stage);  // lane 0 arrives twice: once for itself, once in place of a copy
+        }
+        __syncwarp();
         mbar_arrive(bar_full + 8 * stage);
       }
     }
@@ -397,13 +490,14 @@ __global__ void __launch_bounds__(TMA_THREADS) ffn_tma_kernel(const TmaArgs a) {
       const unsigned char* st = smem + stage * STAGE_BYTES;
       if (!(m.flags & META_EMPTY)) {
         switch (m.bits) {
-          case 2: consume_stage<2, NT>(a, m, st, warp, lane, tot); break;
-          case 4: consume_stage<4, NT>(a, m, st, warp, lane, tot); break;
-          default: consume_stage<8, NT>(a, m, st, warp, lane, tot); break;
+          case 2: consume_stage<2, NT>(a, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          case 4: consume_stage<4, NT>(a, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          default: consume_stage<8, NT>(a, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
         }
+      } else {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
       if (m.flags & META_LAST) {
         switch (m.bits) {
           case 2: store_item<2, NT>(a, m, warp, lane, tot); break;
