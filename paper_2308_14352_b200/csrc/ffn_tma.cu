@@ -42,6 +42,9 @@ constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a s
 #ifndef EMOE_TMA_STAGES_NT1
 #define EMOE_TMA_STAGES_NT1 3
 #endif
+#ifndef EMOE_TMA_LOOKAHEAD
+#define EMOE_TMA_LOOKAHEAD 0
+#endif
 #ifndef EMOE_TMA_CTAS_NT1
 #define EMOE_TMA_CTAS_NT1 2
 #endif
@@ -306,7 +309,11 @@ __host__ __device__ constexpr int smem_bytes_for() {
 }
 
 template <int NT>
+#ifdef EMOE_TMA_MAXNREG
+__global__ void __maxnreg__(EMOE_TMA_MAXNREG) ffn_tma_kernel(const TmaArgs a) {
+#else
 __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_kernel(const TmaArgs a) {
+#endif
   constexpr int STAGES = stages_for<NT>();
   constexpr int STAGE_BYTES = stage_bytes_for(NT);
   extern __shared__ unsigned char smem_raw[];
@@ -354,16 +361,20 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
     // costs no round trip to memory.  A CTA's first item is its own index; the counter hands
     // out the items after those.
     int item_cur = blockIdx.x, item_next = 0;
+#if EMOE_TMA_LOOKAHEAD
     if (lane == 0) item_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
+#endif
     PlanRec rec_cur = recs[min(item_cur / per_expert, L.E - 1)];  // read before n_items is known: same latency
     item_next = __shfl_sync(0xffffffffu, item_next, 0);
     while (ok) {
       const int item = item_cur;
       if (item >= n_items || *abort_flag) break;
       const PlanRec rec = rec_cur;
+#if EMOE_TMA_LOOKAHEAD
       int raw_after_next = 0;
       if (lane == 0) raw_after_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
       const PlanRec rec_next = recs[item_next < n_items ? item_next / per_expert : 0];
+#endif
       const int z = item % a.ksplit;
       const int rb = (item / a.ksplit) % a.row_blocks;
       const int e = rec.e;
@@ -439,9 +450,17 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           }
         }
       }
+#if EMOE_TMA_LOOKAHEAD
       item_cur = item_next;
       rec_cur = rec_next;
       item_next = __shfl_sync(0xffffffffu, raw_after_next, 0);
+#else
+      // the ring still holds several stages of work for the consumers: fetching the next item
+      // only now costs them nothing and no CTA sits on items it is not yet working on
+      if (lane == 0) item_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
+      item_cur = __shfl_sync(0xffffffffu, item_next, 0);
+      rec_cur = recs[item_cur < n_items ? item_cur / per_expert : 0];
+#endif
       if (item_cur < n_items) {
         // pull the next item's scale rows towards L2 while its codes are still far away
         const int rbn = (item_cur / a.ksplit) % a.row_blocks;
