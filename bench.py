@@ -36,8 +36,8 @@ UNIT = "tokens/s"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="emoe", choices=["emoe", "reference"])
     ap.add_argument("--workload", default="switch_base_decode", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--tokens", type=int, default=0, help="batch size (default: the workload's largest)")
