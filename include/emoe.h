@@ -183,8 +183,9 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
 
 /* Selects the expert-FFN kernel family: 0 = automatic (default), 1 = the CUDA-core grouped
  * GEMV, 2 = the tensor-core kernel with register-staged weight loads, 3 = the tensor-core kernel
- * with the TMA-staged weight pipeline.  2 and 3 fail with EMOE_ERR_UNSUPPORTED in forward calls
- * whose shape they do not take.  For tests and measurements. */
+ * with the TMA-staged weight pipeline, 4 = the tcgen05 grouped GEMM (fp16 operands; meant for
+ * many tokens per expert).  2, 3 and 4 fail with EMOE_ERR_UNSUPPORTED in forward calls whose shape
+ * they do not take.  For tests and measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);
 
 /* The routed layer forward for callers that cannot allocate device memory (the paper has no

@@ -229,10 +229,14 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   EMOE_CUDA(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
 
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
-  const bool use_tma = can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
+  const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
+  // many tokens per expert: the tcgen05 grouped GEMM; otherwise the weight-streaming kernels
+  const bool use_umma = can_umma && (ctx->ffn_path == 4 || (ctx->ffn_path == 0 && ffn_token_tiles(L, T) >= 4));
+  const bool use_tma = !use_umma && can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
   const bool use_mma = ffn_mma_supported(L) && ctx->ffn_path != 1;
   if (ctx->ffn_path == 2 && !use_mma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 3 && !use_tma) return EMOE_ERR_UNSUPPORTED;
+  if (ctx->ffn_path == 4 && !use_umma) return EMOE_ERR_UNSUPPORTED;
   int ksplit = 1;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
   if (ctx->timing) {
@@ -244,7 +248,13 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     for (int i = 0; i < 3; ++i) ev[i] = ctx->events[ctx->events_used + i];
     ctx->events_used += 3;
   }
-  if (use_tma) {
+  if (use_umma) {
+    EMOE_CUDA(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, st));
+    if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
+    EMOE_CUDA(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, P, ctx->check_word, st));
+    if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+    EMOE_CUDA(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
+  } else if (use_tma) {
     ksplit = ffn_tma_ksplit(L, T);
     EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
@@ -448,7 +458,7 @@ int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, i
 }
 
 int emoe_set_ffn_path(emoe_ctx* ctx, int path) {
-  if (!ctx || path < 0 || path > 3) return EMOE_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 4) return EMOE_ERR_INVALID_ARG;
   ctx->ffn_path = path;
   return EMOE_OK;
 }

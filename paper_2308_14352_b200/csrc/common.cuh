@@ -80,6 +80,18 @@ cudaError_t launch_ffn_tma(int phase, const LayerDims& L, const ExpertDev* exper
                            const __nv_bfloat16* in, const int32_t* off, int* plan, __nv_bfloat16* hidden, float* o_part,
                            int ksplit, int n_pairs, int T, int* check_word, cudaStream_t st);
 
+int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
+                   uint32_t box_inner, uint32_t box_outer);
+
+// tcgen05 grouped GEMM for experts with many tokens (fp16 operands, fp32 accumulation in tensor
+// memory).  xs16 / hidden16: activations in expert order, fp16, pair order; o: [n_pairs][d_model].
+bool ffn_umma_supported(const LayerDims& L);
+cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
+                               const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
+                               cudaStream_t st);
+cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
+                            void* hidden16, float* o, int n_pairs, int* check_word, cudaStream_t st);
+
 // y[t] = sum_j gates[t][j] * sum_z o_part[z][slot_of_pair[t*k+j]]
 // o_part holds ksplit partial results, each [n_pairs_stride][d].
 cudaError_t launch_combine(const float* o_part, int ksplit, size_t n_pairs_stride, const float* gates,

@@ -562,8 +562,11 @@ cudaError_t launch_ffn_tma(int phase, const LayerDims& L, const ExpertDev* exper
   return launch_nt<4>(a, max_items, st);
 }
 
-// One tensor map per packed matrix: a [N][row_bytes] byte image, 64-row x 128-byte boxes, 128-byte swizzle.
-int encode_weight_tmap(void* out_map, const void* packed, int N, int K, int bits) {
+// Host-side tensor-map encoder (driver entry point looked up once; no link against libcuda).
+// dtype: 0 = bytes, 1 = fp16.  2-D row-major image [outer][inner], box [box_outer][box_inner],
+// 128-byte swizzle (box_inner * element size must be 128 bytes or less).
+int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
+                   uint32_t box_inner, uint32_t box_outer) {
   typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -574,16 +577,22 @@ int encode_weight_tmap(void* out_map, const void* packed, int N, int K, int bits
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || !p) return -1;
     fn = reinterpret_cast<EncodeFn>(p);
   }
-  const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * bits / 8;
-  if (row_bytes < 128 || row_bytes % 16 != 0 || N < TMA_BOX_ROWS) return -2;
-  const cuuint64_t dims[2] = {row_bytes, static_cast<cuuint64_t>(N)};
-  const cuuint64_t strides[1] = {row_bytes};
-  const cuuint32_t box[2] = {128, TMA_BOX_ROWS};
+  if (row_stride_bytes % 16 != 0 || (reinterpret_cast<uintptr_t>(base) & 15) != 0) return -2;
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {row_stride_bytes};
+  const cuuint32_t box[2] = {box_inner, box_outer};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(static_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(packed), dims,
-                        strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  const CUresult r = fn(static_cast<CUtensorMap*>(out_map), dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
+                        2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : -3;
+}
+
+// One tensor map per packed matrix: a [N][row_bytes] byte image, 64-row x 128-byte boxes, 128-byte swizzle.
+int encode_weight_tmap(void* out_map, const void* packed, int N, int K, int bits) {
+  const uint64_t row_bytes = static_cast<uint64_t>(K) * bits / 8;
+  if (row_bytes < 128 || N < TMA_BOX_ROWS) return -2;
+  return encode_tmap_2d(out_map, 0, packed, row_bytes, static_cast<uint64_t>(N), row_bytes, 128, TMA_BOX_ROWS);
 }
 
 }  // namespace emoe

@@ -1,0 +1,552 @@
+// Grouped expert GEMM on packed weights with tcgen05 tensor-core MMAs, for experts that hold
+// many tokens (prefill, large decode batches).  Paper Sections 1/2.1 (each activated expert is
+// an independent FFN) on the Section 3.2 storage (b-bit codes + scale channel, w~ = q * s).
+//
+// Shape of one tile: 128 output channels (UMMA M, "swap-AB": the weight rows are the M side)
+// x 128 tokens of one expert (UMMA N) x all inputs, accumulated in tensor memory.
+//   warp 0    TMA producer: packed code boxes (128 rows x 128 bytes, the decode kernel's tensor
+//             maps) into a 2-deep raw ring, and the tokens' activations (128 tokens x 64 inputs,
+//             fp16, K-major, 128-byte swizzle) into a 3-deep operand ring;
+//   warps 2-5 one thread per output channel: read the channel's packed bytes from the raw ring,
+//             dequantise to fp16 (code -> exact fp16 integer by mantissa insertion, then one
+//             multiply by the group scale: |error| <= 2^-12 relative, the only approximation of
+//             this path), and write the row of the A operand in the canonical K-major
+//             swizzled layout; later the epilogue: tensor memory -> registers -> activation ->
+//             global memory;
+//   warp 1    one thread issues tcgen05.mma (M128 N128 K16, fp16 x fp16 -> fp32 in TMEM) per 16
+//             inputs and commits each stage back to the producers.
+// SwiGLU's first projection runs two accumulators (w1 and w3 rows of the same 128 channels
+// against the same activation tile), so that silu(a) * b needs no exchange between warps.
+// Activations travel as fp16 (exact for bf16 values inside the fp16 range, saturated outside);
+// the hidden vector is rounded to bf16 first, as the definition asks, then stored as fp16.
+// The reduction index is enumerated in the order the unpack emits code pairs; the activation
+// buffers are written in that same order (scatter_x16_kernel, first-projection epilogue).
+// Every wait is bounded (see pipe.cuh); tensor memory is always released before exit.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "ffn_tile.cuh"
+#include "pipe.cuh"
+
+namespace emoe {
+namespace {
+
+constexpr int UM_TOK = 128;                // tokens per tile (UMMA N)
+constexpr int UM_ROWS = 128;               // output channels per tile (UMMA M)
+constexpr int UM_BK = 64;                  // inputs per operand stage: one 128-byte row of fp16
+constexpr int UM_AB_STAGES = 3;
+constexpr int UM_RAW_STAGES = 2;
+constexpr int UM_TILE_BYTES = 128 * 128;   // a [128][64] fp16 operand tile, or a [128 rows][128 B] packed tile
+constexpr int UM_AB_STAGE_BYTES = 3 * UM_TILE_BYTES;   // A (first matrix), A (second matrix), B
+constexpr int UM_RAW_STAGE_BYTES = 2 * UM_TILE_BYTES;  // packed tiles of up to two matrices
+constexpr int UM_SMEM_BYTES = UM_RAW_STAGES * UM_RAW_STAGE_BYTES + UM_AB_STAGES * UM_AB_STAGE_BYTES + 1024;
+constexpr int UM_THREADS = 192;
+constexpr int UM_TMEM_COLS = 256;
+
+// position of input k in the activation buffers of this path: the unpack emits the code pairs
+// (c, c+4) of an 8-code word at 4 bits and (c, c+8) of a 16-code word at 2 bits
+template <int BITS>
+__device__ __forceinline__ int pair_pos(int k) {
+  if (BITS == 8) return k;
+  constexpr int B = BITS == 4 ? 8 : 16;
+  const int o = k & (B - 1);
+  return (k & ~(B - 1)) + (o < B / 2 ? 2 * o : 2 * (o - B / 2) + 1);
+}
+__device__ __forceinline__ int pair_pos_rt(int bits, int k) {
+  return bits == 8 ? k : (bits == 4 ? pair_pos<4>(k) : pair_pos<2>(k));
+}
+
+__device__ __forceinline__ uint32_t h2_fma(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t r;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+  return r;
+}
+__device__ __forceinline__ uint32_t h2_add(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("add.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+__device__ __forceinline__ uint32_t h2_mul(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// ---- dequantise one 16-byte chunk of a packed row to fp16 (q * s), 8 values per output chunk ----
+// 8 bits: 16 codes -> 2 chunks.  byte ^ 0x80 = q + 128 goes into the mantissa of 1024.
+__device__ __forceinline__ void dequant_chunk8(const uint4& raw, uint32_t s2, uint4 (&out)[2]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  uint32_t o[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t u = w[i] ^ 0x80808080u;
+    o[2 * i] = h2_mul(h2_add(prmt(u, 0x64646464u, 0x5140u), 0xE480E480u), s2);      // -(1024 + 128)
+    o[2 * i + 1] = h2_mul(h2_add(prmt(u, 0x64646464u, 0x5342u), 0xE480E480u), s2);
+  }
+  out[0] = make_uint4(o[0], o[1], o[2], o[3]);
+  out[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+// 4 bits: 32 codes -> 4 chunks (one per 8-code word, pair order (c, c+4)).
+__device__ __forceinline__ void dequant_chunk4(const uint4& raw, uint32_t s2, uint4 (&out)[4]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t hi = w[i] >> 8;
+    const uint32_t t0 = h2_add(and_xor(w[i], 0x000F000Fu, 0x64086408u), 0xE408E408u);               // v - 1032
+    const uint32_t t1 = h2_fma(and_xor(w[i], 0x00F000F0u, 0x64806480u), 0x2C002C00u, 0xD480D480u);  // v/16 - 72
+    const uint32_t t2 = h2_add(and_xor(hi, 0x000F000Fu, 0x64086408u), 0xE408E408u);
+    const uint32_t t3 = h2_fma(and_xor(hi, 0x00F000F0u, 0x64806480u), 0x2C002C00u, 0xD480D480u);
+    out[i] = make_uint4(h2_mul(t0, s2), h2_mul(t1, s2), h2_mul(t2, s2), h2_mul(t3, s2));
+  }
+}
+// 2 bits: 64 codes -> 8 chunks (two per 16-code word, pair order (c, c+8)).
+__device__ __forceinline__ void dequant_chunk2(const uint4& raw, uint32_t s2, uint4 (&out)[8]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  // field at mantissa bit p of 1024: v = 1024 + (q + 2) * 2^p;  q = v * 2^-p - (1024 * 2^-p + 2)
+  const uint32_t msk[5] = {0x00030003u, 0x000C000Cu, 0x00300030u, 0x00C000C0u, 0x03000300u};
+  const uint32_t mag[5] = {0x64026402u, 0x64086408u, 0x64206420u, 0x64806480u, 0x66006600u};
+  const uint32_t mul[5] = {0x3C003C00u, 0x34003400u, 0x2C002C00u, 0x24002400u, 0x1C001C00u};
+  const uint32_t add[5] = {0xE402E402u, 0xDC08DC08u, 0xD420D420u, 0xCC80CC80u, 0xC600C600u};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint32_t o[8];
+    const uint32_t hi = w[i] >> 10;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const int p = c < 5 ? c : c - 5;
+      const uint32_t src = c < 5 ? w[i] : hi;
+      o[c] = h2_mul(h2_fma(and_xor(src, msk[p], mag[p]), mul[p], add[p]), s2);
+    }
+    out[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+    out[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+  }
+}
+
+struct UmmaArgs {
+  int phase;
+  LayerDims L;
+  const CUtensorMap* wmaps;  // [E][3] packed-weight tensor maps (boxes of 64 rows x 128 bytes)
+  const int* plan;           // header + PlanRec per activated expert
+  __half* hidden16;          // first projection's output (fp16, pair order)
+  float* o;                  // second projection's output [n_pairs][d_model]
+  int* check_word;
+};
+
+// the tiles of this CTA: linear index = blockIdx.x, += gridDim.x over
+// (activated expert, token tile, row block) with the row block running fastest
+struct TileWalk {
+  const PlanRec* recs;
+  int n_active, row_blocks, lin, a, base;
+  PlanRec rec;
+  int tiles_of_a;
+  __device__ __forceinline__ void init(const int* plan, int rb) {
+    n_active = *reinterpret_cast<const volatile int*>(plan);
+    recs = reinterpret_cast<const PlanRec*>(reinterpret_cast<const char*>(plan) + PLAN_HEADER_BYTES);
+    row_blocks = rb;
+    lin = blockIdx.x;
+    a = -1;
+    base = 0;
+    tiles_of_a = 0;
+  }
+  // advances to the CTA's next tile; false when there is none
+  __device__ __forceinline__ bool next(int& tt, int& rb) {
+    while (a < 0 || lin >= base + tiles_of_a) {
+      base += tiles_of_a;
+      ++a;
+      if (a >= n_active) return false;
+      rec = recs[a];
+      tiles_of_a = row_blocks * ((rec.cnt + UM_TOK - 1) / UM_TOK);
+    }
+    const int local = lin - base;
+    tt = local / row_blocks;
+    rb = local - tt * row_blocks;
+    lin += gridDim.x;
+    return true;
+  }
+};
+
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  // K-major, 128-byte swizzle: 8-row groups 1024 bytes apart; descriptor version 1
+  return static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      :
+      : "r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(UM_THREADS, 1)
+    ffn_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_b) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * UM_RAW_STAGES + 3 * UM_AB_STAGES + 2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* raw_ring = smem;
+  unsigned char* ab_ring = smem + UM_RAW_STAGES * UM_RAW_STAGE_BYTES;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+  const uint32_t bar_raw_full = smem_u32(bars);
+  const uint32_t bar_raw_empty = smem_u32(bars + UM_RAW_STAGES);
+  const uint32_t bar_b_full = smem_u32(bars + 2 * UM_RAW_STAGES);
+  const uint32_t bar_a_full = smem_u32(bars + 2 * UM_RAW_STAGES + UM_AB_STAGES);
+  const uint32_t bar_ab_empty = smem_u32(bars + 2 * UM_RAW_STAGES + 2 * UM_AB_STAGES);
+  const uint32_t bar_acc_full = smem_u32(bars + 2 * UM_RAW_STAGES + 3 * UM_AB_STAGES);
+  const uint32_t bar_acc_empty = bar_acc_full + 8;
+
+  if (threadIdx.x == 0) {
+    abort_word = 0;
+    for (int s = 0; s < UM_RAW_STAGES; ++s) {
+      mbar_init(bar_raw_full + 8 * s, 1);
+      mbar_init(bar_raw_empty + 8 * s, 4);
+    }
+    for (int s = 0; s < UM_AB_STAGES; ++s) {
+      mbar_init(bar_b_full + 8 * s, 1);
+      mbar_init(bar_a_full + 8 * s, 4);
+      mbar_init(bar_ab_empty + 8 * s, 1);
+    }
+    mbar_init(bar_acc_full, 1);
+    mbar_init(bar_acc_empty, 4);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // tensor memory for the accumulators (two of 128 columns)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(UM_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const LayerDims& L = a.L;
+  const int N = a.phase == 0 ? L.d_ff : L.d_model;
+  const int K = a.phase == 0 ? L.d_model : L.d_ff;
+  const bool dual = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const int n_mats = dual ? 2 : 1;
+  const int mat_first = a.phase == 0 ? 0 : (L.act == EMOE_ACT_SWIGLU ? 2 : 1);
+  const int row_blocks = (N + UM_ROWS - 1) / UM_ROWS;
+  const int kb_total = K / UM_BK;
+
+  TileWalk walk;
+  walk.init(a.plan, row_blocks);
+  int tt, rb;
+
+  if (warp == 0) {
+    // ---------------- TMA producer (one lane) ----------------
+    if (lane == 0) {
+      int raw_it = 0, ab_it = 0;
+      bool ok = true;
+      while (ok && walk.next(tt, rb)) {
+        const PlanRec rec = walk.rec;
+        const CUtensorMap* maps = a.wmaps + static_cast<size_t>(rec.e) * 3;
+        const int kbs = (1024 / rec.bits) / UM_BK;  // operand stages per packed box (128 bytes of a row)
+        const int row0 = rb * UM_ROWS;
+        const int tok0 = rec.begin + tt * UM_TOK;
+        for (int kb = 0; kb < kb_total && ok;) {
+          const int rs = raw_it % UM_RAW_STAGES;
+          if (!mbar_wait(bar_raw_empty + 8 * rs, ((raw_it / UM_RAW_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
+            ok = false;
+            break;
+          }
+          const uint32_t rfull = bar_raw_full + 8 * rs;
+          mbar_expect_tx(rfull, n_mats * UM_TILE_BYTES);
+          const int c0 = (kb / kbs) * 128;
+          for (int m = 0; m < n_mats; ++m) {
+            const uint32_t dst = smem_u32(raw_ring + rs * UM_RAW_STAGE_BYTES + m * UM_TILE_BYTES);
+            const CUtensorMap* mp = maps + (dual ? m : mat_first);
+            tma_load_2d(dst, mp, c0, row0, rfull);
+            tma_load_2d(dst + UM_TILE_BYTES / 2, mp, c0, row0 + 64, rfull);
+          }
+          ++raw_it;
+          for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb) {
+            const int s = ab_it % UM_AB_STAGES;
+            if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_AB_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
+              ok = false;
+              break;
+            }
+            const uint32_t bfull = bar_b_full + 8 * s;
+            mbar_expect_tx(bfull, UM_TILE_BYTES);
+            tma_load_2d(smem_u32(ab_ring + s * UM_AB_STAGE_BYTES + 2 * UM_TILE_BYTES), &tmap_b, kb * UM_BK, tok0, bfull);
+            ++ab_it;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (one lane) ----------------
+    if (lane == 0) {
+      // kind::f16, fp16 x fp16 -> fp32, both operands K-major, M = 128, N = 128
+      const uint32_t idesc = (1u << 4) | ((UM_TOK >> 3) << 17) | ((UM_ROWS >> 4) << 24);
+      int ab_it = 0, tile_it = 0;
+      bool ok = true;
+      while (ok && walk.next(tt, rb)) {
+        if (!mbar_wait(bar_acc_empty, ((tile_it & 1) ^ 1), a.check_word, abort_flag)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        for (int kb = 0; kb < kb_total; ++kb, ++ab_it) {
+          const int s = ab_it % UM_AB_STAGES;
+          const uint32_t par = (ab_it / UM_AB_STAGES) & 1;
+          if (!mbar_wait(bar_a_full + 8 * s, par, a.check_word, abort_flag) ||
+              !mbar_wait(bar_b_full + 8 * s, par, a.check_word, abort_flag)) {
+            ok = false;
+            break;
+          }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t st = smem_u32(ab_ring + s * UM_AB_STAGE_BYTES);
+          const uint64_t da0 = umma_desc(st), da1 = umma_desc(st + UM_TILE_BYTES), db = umma_desc(st + 2 * UM_TILE_BYTES);
+#pragma unroll
+          for (int k4 = 0; k4 < UM_BK / 16; ++k4) {  // 16 inputs = 32 bytes = 2 descriptor units per step
+            const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
+            umma_f16(tmem_base, da0 + 2 * k4, db + 2 * k4, idesc, acc);
+            if (dual) umma_f16(tmem_base + UM_TOK, da1 + 2 * k4, db + 2 * k4, idesc, acc);
+          }
+          umma_commit(bar_ab_empty + 8 * s);  // the stage may be refilled once these MMAs have read it
+        }
+        if (ok) umma_commit(bar_acc_full);
+        ++tile_it;
+      }
+    }
+  } else {
+    // ---------------- dequantise (one thread per output channel), then epilogue ----------------
+    const int quarter = warp & 3;          // TMEM lanes this warp may read: 32 * quarter ...
+    const int r = 32 * quarter + lane;     // channel of the tile = row of the operand = TMEM lane
+    const int box = r >> 6, rin = r & 63;
+    const int G = L.group > 0 ? L.group : K;
+    const int ngroups = K / G;
+    const bool sf16 = L.scale_f16 != 0;
+    int raw_it = 0, ab_it = 0, tile_it = 0;
+    bool ok = true;
+    while (ok && walk.next(tt, rb)) {
+      const PlanRec rec = walk.rec;
+      const int bits = rec.bits;
+      const int kbs = (1024 / bits) / UM_BK;
+      const int n = min(rb * UM_ROWS + r, N - 1);
+      const void* sp[2] = {dual ? rec.scales[0] : rec.scales[mat_first], dual ? rec.scales[1] : rec.scales[mat_first]};
+      const size_t srow = static_cast<size_t>(n) * ngroups;
+      float sv[2], sv_next[2];
+      for (int m = 0; m < n_mats; ++m) sv[m] = load_scale_ro(sp[m], sf16, srow);
+      for (int kb = 0; kb < kb_total && ok;) {
+        const int rs = raw_it % UM_RAW_STAGES;
+        if (!mbar_wait(bar_raw_full + 8 * rs, (raw_it / UM_RAW_STAGES) & 1, a.check_word, abort_flag)) {
+          ok = false;
+          break;
+        }
+        for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb, ++ab_it) {
+          const int s = ab_it % UM_AB_STAGES;
+          if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_AB_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
+            ok = false;
+            break;
+          }
+          const int g_next = min(((kb + 1) * UM_BK) / G, ngroups - 1);
+          for (int m = 0; m < n_mats; ++m) sv_next[m] = load_scale_ro(sp[m], sf16, srow + g_next);
+          for (int m = 0; m < n_mats; ++m) {
+            const __half sh = __float2half_rn(sv[m]);
+            const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
+            const unsigned char* rrow = raw_ring + rs * UM_RAW_STAGE_BYTES + m * UM_TILE_BYTES + box * (UM_TILE_BYTES / 2) + rin * 128;
+            unsigned char* arow = ab_ring + s * UM_AB_STAGE_BYTES + m * UM_TILE_BYTES + r * 128;
+            if (bits == 8) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(rrow + (((4 * j + c) ^ (rin & 7)) << 4));
+                uint4 o[2];
+                dequant_chunk8(raw, s2, o);
+                *reinterpret_cast<uint4*>(arow + (((2 * c) ^ (r & 7)) << 4)) = o[0];
+                *reinterpret_cast<uint4*>(arow + (((2 * c + 1) ^ (r & 7)) << 4)) = o[1];
+              }
+            } else if (bits == 4) {
+#pragma unroll
+              for (int c = 0; c < 2; ++c) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(rrow + (((2 * j + c) ^ (rin & 7)) << 4));
+                uint4 o[4];
+                dequant_chunk4(raw, s2, o);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(arow + (((4 * c + i) ^ (r & 7)) << 4)) = o[i];
+              }
+            } else {
+              const uint4 raw = *reinterpret_cast<const uint4*>(rrow + ((j ^ (rin & 7)) << 4));
+              uint4 o[8];
+              dequant_chunk2(raw, s2, o);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) *reinterpret_cast<uint4*>(arow + ((i ^ (r & 7)) << 4)) = o[i];
+            }
+          }
+          for (int m = 0; m < n_mats; ++m) sv[m] = sv_next[m];
+          // generic-proxy writes of the operand must be visible to the tensor core's async reads
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_a_full + 8 * s);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_raw_empty + 8 * rs);
+        ++raw_it;
+      }
+      if (!ok) break;
+      // ---- epilogue: this warp's 32 channels x 128 tokens ----
+      if (!mbar_wait(bar_acc_full, tile_it & 1, a.check_word, abort_flag)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int nrow = rb * UM_ROWS + r;
+      const int tokens = min(UM_TOK, rec.cnt - tt * UM_TOK);
+      const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tt) * UM_TOK;
+      const int hpos = a.phase == 0 ? pair_pos_rt(bits, min(nrow, N - 1)) : 0;
+#pragma unroll 1
+      for (int cc = 0; cc < UM_TOK; cc += 32) {
+        uint32_t va[32], vb[32];
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + cc;
+        tmem_ld32(taddr, va);
+        if (dual) tmem_ld32(taddr + UM_TOK, vb);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (nrow < N) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (cc + j < tokens) {
+              const float x = __uint_as_float(va[j]);
+              if (a.phase == 0) {
+                float h;
+                if (dual) h = x / (1.0f + expf(-x)) * __uint_as_float(vb[j]);
+                else h = fmaxf(x, 0.0f);
+                h = __bfloat162float(__float2bfloat16_rn(h));  // the hidden vector is a bf16 tensor
+                h = fminf(fmaxf(h, -65504.0f), 65504.0f);
+                a.hidden16[(slot0 + cc + j) * N + hpos] = __float2half_rn(h);
+              } else {
+                a.o[(slot0 + cc + j) * N + nrow] = x;
+              }
+            }
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty);
+      ++tile_it;
+    }
+  }
+
+  // wind-down: everybody meets, then the allocating warp releases tensor memory
+  if (*abort_flag)
+    for (int i = 0; i < 2000; ++i) __nanosleep(100);  // let copies in flight land
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(UM_TMEM_COLS) : "memory");
+  }
+}
+
+// x rows -> expert order, fp16, pair order of the owning expert's bitwidth (saturating)
+__global__ void __launch_bounds__(128)
+    scatter_x16_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
+                       const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
+                       int E, int* __restrict__ plan, int top_k, int d, int n_pairs, __half* __restrict__ xs) {
+  if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
+    // work plan: activated experts, widest codes first
+    const int lane = threadIdx.x;
+    PlanRec* recs = reinterpret_cast<PlanRec*>(reinterpret_cast<char*>(plan) + PLAN_HEADER_BYTES);
+    int base = 0;
+    for (int b = 8; b >= 2; b >>= 1) {
+      for (int e0 = 0; e0 < E; e0 += 32) {
+        const int e = e0 + lane;
+        const bool act = e < E && off[e + 1] > off[e] && experts[e].bits == b;
+        const unsigned m = __ballot_sync(0xffffffffu, act);
+        if (act) {
+          PlanRec& r = recs[base + __popc(m & ((1u << lane) - 1u))];
+          r.e = e;
+          r.begin = off[e];
+          r.cnt = off[e + 1] - off[e];
+          r.bits = b;
+          r.scales[0] = experts[e].scales[0];
+          r.scales[1] = experts[e].scales[1];
+          r.scales[2] = experts[e].scales[2];
+        }
+        base += __popc(m);
+      }
+    }
+    if (lane == 0) {
+      plan[0] = base;
+      plan[1] = 0;
+      plan[2] = 0;
+    }
+  }
+  const int slot = blockIdx.x;
+  const int pair = perm[slot];
+  if (pair < 0 || pair >= n_pairs) return;
+  const int bits = experts[ids[pair]].bits;
+  const __nv_bfloat16* src = x + static_cast<size_t>(pair / top_k) * d;
+  __half* dst = xs + static_cast<size_t>(slot) * d;
+  for (int k = threadIdx.x; k < d; k += blockDim.x) {
+    const float v = fminf(fmaxf(__bfloat162float(src[k]), -65504.0f), 65504.0f);
+    dst[pair_pos_rt(bits, k)] = __float2half_rn(v);
+  }
+}
+
+}  // namespace
+
+bool ffn_umma_supported(const LayerDims& L) {
+  // the same tensor maps as the TMA path; K in whole 128-byte packed rows at every width
+  return ffn_tma_supported(L) && L.d_model % 512 == 0 && L.d_ff % 512 == 0;
+}
+
+cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
+                               const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
+                               cudaStream_t st) {
+  scatter_x16_kernel<<<n_pairs, 128, 0, st>>>(experts, reinterpret_cast<const __nv_bfloat16*>(x), ids, perm, off, L.E, plan,
+                                              L.top_k, L.d_model, n_pairs, reinterpret_cast<__half*>(xs16));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
+                            void* hidden16, float* o, int n_pairs, int* check_word, cudaStream_t st) {
+  const int N = phase == 0 ? L.d_ff : L.d_model;
+  const int K = phase == 0 ? L.d_model : L.d_ff;
+  CUtensorMap tmap_b;
+  if (encode_tmap_2d(&tmap_b, /*fp16*/ 1, in16, static_cast<uint64_t>(K), static_cast<uint64_t>(n_pairs),
+                     static_cast<uint64_t>(K) * 2, UM_BK, UM_TOK) != 0)
+    return cudaErrorInvalidValue;
+  static int sms_of_device[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!sms_of_device[dev]) {
+    e = cudaFuncSetAttribute(ffn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, UM_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&sms_of_device[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+  }
+  const long long row_blocks = (N + UM_ROWS - 1) / UM_ROWS;
+  // upper bound of the tile count: every pair alone in a token tile
+  long long tiles = row_blocks * (static_cast<long long>(n_pairs < L.E ? n_pairs : L.E) + n_pairs / UM_TOK);
+  const int grid = static_cast<int>(tiles < sms_of_device[dev] ? tiles : sms_of_device[dev]);
+  UmmaArgs a;
+  a.phase = phase;
+  a.L = L;
+  a.wmaps = static_cast<const CUtensorMap*>(wmaps);
+  a.plan = plan;
+  a.hidden16 = reinterpret_cast<__half*>(hidden16);
+  a.o = o;
+  a.check_word = check_word;
+  ffn_umma_kernel<<<grid, UM_THREADS, UM_SMEM_BYTES, st>>>(a, tmap_b);
+  return cudaGetLastError();
+}
+
+}  // namespace emoe

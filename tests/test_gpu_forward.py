@@ -95,6 +95,22 @@ def test_forward_tma_pipeline_path(act, group, sdt, d, f, E, k, gate, bits, T):
     _run_case(shape, bits, T, seed=25, path=3)
 
 
+UMMA_CASES = [
+    ("relu", 128, "f16", 512, 1024, 4, 1, "softmax", [8, 4, 2, 4], 200),              # ~50 tokens per expert
+    ("relu", 128, "f16", 512, 1024, 2, 1, "softmax", [4, 2], 300),                    # two token tiles per expert
+    ("relu", 0, "f16", 1024, 512, 3, 2, "softmax_renorm", [2, 8, 4], 97),             # per-channel scales
+    ("swiglu", 128, "f16", 512, 1536, 4, 2, "softmax_renorm", [4, 8, 2, 4], 150),     # two accumulators
+    ("swiglu", 256, "f32", 1024, 2048, 8, 2, "softmax_renorm", [4, 4, 8, 2, 4, 8, 2, 4], 64),
+    ("relu", 128, "f16", 512, 512, 2, 1, "softmax", [2, 8], 1),                       # a single token
+]
+
+
+@pytest.mark.parametrize("act,group,sdt,d,f,E,k,gate,bits,T", UMMA_CASES)
+def test_forward_tcgen05_path(act, group, sdt, d, f, E, k, gate, bits, T):
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, "bf16")
+    _run_case(shape, bits, T, seed=27, path=4)
+
+
 def test_tma_path_is_refused_for_narrow_rows():
     shape = inputs.LayerShape(256, 512, 4, 1, "relu", "softmax", 128, "f16", "bf16")
     with pytest.raises(B.EmoeError) as ei:
