@@ -430,7 +430,7 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
 def main():
     args = parse_args()
     w = inputs.WORKLOADS[args.workload]
-    T = args.tokens or max(t for t in w.tokens if t <= 64)
+    T = args.tokens or max([t for t in w.tokens if t <= 64] or list(w.tokens))
     n_layers = args.layers or w.n_layers
     if args.impl == "reference":
         rank = int(os.environ.get("RANK", "0"))

@@ -7,7 +7,7 @@
 //   warp 0    TMA producer: packed code boxes (128 rows x 128 bytes, the decode kernel's tensor
 //             maps) into a 2-deep raw ring, and the tokens' activations (128 tokens x 64 inputs,
 //             fp16, K-major, 128-byte swizzle) into a 3-deep operand ring;
-//   warps 2-5 one thread per output channel: read the channel's packed bytes from the raw ring,
+//   warps 2-9 two threads per output channel: read the channel's packed bytes from the raw ring,
 //             dequantise to fp16 (code -> exact fp16 integer by mantissa insertion, then one
 //             multiply by the group scale: |error| <= 2^-12 relative, the only approximation of
 //             this path), and write the row of the A operand in the canonical K-major
@@ -40,7 +40,8 @@ constexpr int UM_TILE_BYTES = 128 * 128;   // a [128][64] fp16 operand tile, or 
 constexpr int UM_AB_STAGE_BYTES = 3 * UM_TILE_BYTES;   // A (first matrix), A (second matrix), B
 constexpr int UM_RAW_STAGE_BYTES = 2 * UM_TILE_BYTES;  // packed tiles of up to two matrices
 constexpr int UM_SMEM_BYTES = UM_RAW_STAGES * UM_RAW_STAGE_BYTES + UM_AB_STAGES * UM_AB_STAGE_BYTES + 1024;
-constexpr int UM_THREADS = 192;
+constexpr int UM_UNPACK_WARPS = 8;         // two threads per output channel, each dequantises half of a stage
+constexpr int UM_THREADS = (2 + UM_UNPACK_WARPS) * 32;
 constexpr int UM_TMEM_COLS = 256;
 
 // position of input k in the activation buffers of this path: the unpack emits the code pairs
@@ -99,16 +100,17 @@ __device__ __forceinline__ void dequant_chunk4(const uint4& raw, uint32_t s2, ui
     out[i] = make_uint4(h2_mul(t0, s2), h2_mul(t1, s2), h2_mul(t2, s2), h2_mul(t3, s2));
   }
 }
-// 2 bits: 64 codes -> 8 chunks (two per 16-code word, pair order (c, c+8)).
-__device__ __forceinline__ void dequant_chunk2(const uint4& raw, uint32_t s2, uint4 (&out)[8]) {
-  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+// 2 bits: 64 codes -> 8 chunks (two per 16-code word, pair order (c, c+8)); this does the four
+// chunks of words 2*half and 2*half+1.
+__device__ __forceinline__ void dequant_chunk2_half(const uint4& raw, int half, uint32_t s2, uint4 (&out)[4]) {
+  const uint32_t w[2] = {half ? raw.z : raw.x, half ? raw.w : raw.y};
   // field at mantissa bit p of 1024: v = 1024 + (q + 2) * 2^p;  q = v * 2^-p - (1024 * 2^-p + 2)
   const uint32_t msk[5] = {0x00030003u, 0x000C000Cu, 0x00300030u, 0x00C000C0u, 0x03000300u};
   const uint32_t mag[5] = {0x64026402u, 0x64086408u, 0x64206420u, 0x64806480u, 0x66006600u};
   const uint32_t mul[5] = {0x3C003C00u, 0x34003400u, 0x2C002C00u, 0x24002400u, 0x1C001C00u};
   const uint32_t add[5] = {0xE402E402u, 0xDC08DC08u, 0xD420D420u, 0xCC80CC80u, 0xC600C600u};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
+  for (int i = 0; i < 2; ++i) {
     uint32_t o[8];
     const uint32_t hi = w[i] >> 10;
 #pragma unroll
@@ -218,15 +220,15 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
     abort_word = 0;
     for (int s = 0; s < UM_RAW_STAGES; ++s) {
       mbar_init(bar_raw_full + 8 * s, 1);
-      mbar_init(bar_raw_empty + 8 * s, 4);
+      mbar_init(bar_raw_empty + 8 * s, UM_UNPACK_WARPS);
     }
     for (int s = 0; s < UM_AB_STAGES; ++s) {
       mbar_init(bar_b_full + 8 * s, 1);
-      mbar_init(bar_a_full + 8 * s, 4);
+      mbar_init(bar_a_full + 8 * s, UM_UNPACK_WARPS);
       mbar_init(bar_ab_empty + 8 * s, 1);
     }
     mbar_init(bar_acc_full, 1);
-    mbar_init(bar_acc_empty, 4);
+    mbar_init(bar_acc_empty, UM_UNPACK_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {  // tensor memory for the accumulators (two of 128 columns)
@@ -330,6 +332,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
   } else {
     // ---------------- dequantise (one thread per output channel), then epilogue ----------------
     const int quarter = warp & 3;          // TMEM lanes this warp may read: 32 * quarter ...
+    const int half = (warp - 2) >> 2;      // which half of a stage's chunks (and of the token columns) is this warp's
     const int r = 32 * quarter + lane;     // channel of the tile = row of the operand = TMEM lane
     const int box = r >> 6, rin = r & 63;
     const int G = L.group > 0 ? L.group : K;
@@ -367,7 +370,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
             unsigned char* arow = ab_ring + s * UM_AB_STAGE_BYTES + m * UM_TILE_BYTES + r * 128;
             if (bits == 8) {
 #pragma unroll
-              for (int c = 0; c < 4; ++c) {
+              for (int c = 2 * half; c < 2 * half + 2; ++c) {
                 const uint4 raw = *reinterpret_cast<const uint4*>(rrow + (((4 * j + c) ^ (rin & 7)) << 4));
                 uint4 o[2];
                 dequant_chunk8(raw, s2, o);
@@ -375,8 +378,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
                 *reinterpret_cast<uint4*>(arow + (((2 * c + 1) ^ (r & 7)) << 4)) = o[1];
               }
             } else if (bits == 4) {
-#pragma unroll
-              for (int c = 0; c < 2; ++c) {
+              {
+                const int c = half;
                 const uint4 raw = *reinterpret_cast<const uint4*>(rrow + (((2 * j + c) ^ (rin & 7)) << 4));
                 uint4 o[4];
                 dequant_chunk4(raw, s2, o);
@@ -385,10 +388,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
               }
             } else {
               const uint4 raw = *reinterpret_cast<const uint4*>(rrow + ((j ^ (rin & 7)) << 4));
-              uint4 o[8];
-              dequant_chunk2(raw, s2, o);
+              uint4 o[4];
+              dequant_chunk2_half(raw, half, s2, o);
 #pragma unroll
-              for (int i = 0; i < 8; ++i) *reinterpret_cast<uint4*>(arow + ((i ^ (r & 7)) << 4)) = o[i];
+              for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(arow + (((4 * half + i) ^ (r & 7)) << 4)) = o[i];
             }
           }
           for (int m = 0; m < n_mats; ++m) sv[m] = sv_next[m];
@@ -402,7 +405,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
         ++raw_it;
       }
       if (!ok) break;
-      // ---- epilogue: this warp's 32 channels x 128 tokens ----
+      // ---- epilogue: this warp's 32 channels x 64 tokens ----
       if (!mbar_wait(bar_acc_full, tile_it & 1, a.check_word, abort_flag)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int nrow = rb * UM_ROWS + r;
@@ -410,7 +413,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tt) * UM_TOK;
       const int hpos = a.phase == 0 ? pair_pos_rt(bits, min(nrow, N - 1)) : 0;
 #pragma unroll 1
-      for (int cc = 0; cc < UM_TOK; cc += 32) {
+      for (int cc = 64 * half; cc < 64 * half + 64; cc += 32) {
         uint32_t va[32], vb[32];
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + cc;
         tmem_ld32(taddr, va);
