@@ -40,7 +40,11 @@ constexpr int UM_TILE_BYTES = 128 * 128;   // a [128][64] fp16 operand tile, or 
 constexpr int UM_AB_STAGE_BYTES = 3 * UM_TILE_BYTES;   // A (first matrix), A (second matrix), B
 constexpr int UM_RAW_STAGE_BYTES = 2 * UM_TILE_BYTES;  // packed tiles of up to two matrices
 constexpr int UM_SMEM_BYTES = UM_RAW_STAGES * UM_RAW_STAGE_BYTES + UM_AB_STAGES * UM_AB_STAGE_BYTES + 1024;
-constexpr int UM_UNPACK_WARPS = 8;         // two threads per output channel, each dequantises half of a stage
+#ifndef EMOE_UM_UNPACK_WARPS
+#define EMOE_UM_UNPACK_WARPS 8
+#endif
+constexpr int UM_UNPACK_WARPS = EMOE_UM_UNPACK_WARPS;  // 8 or 16: two or four threads per output channel
+constexpr int UM_PARTS = UM_UNPACK_WARPS / 4;            // each dequantises its share of a stage and reads its share of the columns
 constexpr int UM_THREADS = (2 + UM_UNPACK_WARPS) * 32;
 constexpr int UM_TMEM_COLS = 256;
 
@@ -87,40 +91,47 @@ __device__ __forceinline__ void dequant_chunk8(const uint4& raw, uint32_t s2, ui
   out[0] = make_uint4(o[0], o[1], o[2], o[3]);
   out[1] = make_uint4(o[4], o[5], o[6], o[7]);
 }
-// 4 bits: 32 codes -> 4 chunks (one per 8-code word, pair order (c, c+4)).
-__device__ __forceinline__ void dequant_chunk4(const uint4& raw, uint32_t s2, uint4 (&out)[4]) {
-  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint32_t hi = w[i] >> 8;
-    const uint32_t t0 = h2_add(and_xor(w[i], 0x000F000Fu, 0x64086408u), 0xE408E408u);               // v - 1032
-    const uint32_t t1 = h2_fma(and_xor(w[i], 0x00F000F0u, 0x64806480u), 0x2C002C00u, 0xD480D480u);  // v/16 - 72
-    const uint32_t t2 = h2_add(and_xor(hi, 0x000F000Fu, 0x64086408u), 0xE408E408u);
-    const uint32_t t3 = h2_fma(and_xor(hi, 0x00F000F0u, 0x64806480u), 0x2C002C00u, 0xD480D480u);
-    out[i] = make_uint4(h2_mul(t0, s2), h2_mul(t1, s2), h2_mul(t2, s2), h2_mul(t3, s2));
-  }
+// 4 bits: one 8-code word -> one chunk, pair order (c, c+4).
+__device__ __forceinline__ uint4 dequant_word4(uint32_t w, uint32_t s2) {
+  const uint32_t hi = w >> 8;
+  const uint32_t t0 = h2_add(and_xor(w, 0x000F000Fu, 0x64086408u), 0xE408E408u);               // v - 1032
+  const uint32_t t1 = h2_fma(and_xor(w, 0x00F000F0u, 0x64806480u), 0x2C002C00u, 0xD480D480u);  // v/16 - 72
+  const uint32_t t2 = h2_add(and_xor(hi, 0x000F000Fu, 0x64086408u), 0xE408E408u);
+  const uint32_t t3 = h2_fma(and_xor(hi, 0x00F000F0u, 0x64806480u), 0x2C002C00u, 0xD480D480u);
+  return make_uint4(h2_mul(t0, s2), h2_mul(t1, s2), h2_mul(t2, s2), h2_mul(t3, s2));
 }
-// 2 bits: 64 codes -> 8 chunks (two per 16-code word, pair order (c, c+8)); this does the four
-// chunks of words 2*half and 2*half+1.
-__device__ __forceinline__ void dequant_chunk2_half(const uint4& raw, int half, uint32_t s2, uint4 (&out)[4]) {
-  const uint32_t w[2] = {half ? raw.z : raw.x, half ? raw.w : raw.y};
+// 2 bits: one 16-code word -> two chunks, pair order (c, c+8).
+__device__ __forceinline__ void dequant_word2(uint32_t w, uint32_t s2, uint4 (&out)[2]) {
   // field at mantissa bit p of 1024: v = 1024 + (q + 2) * 2^p;  q = v * 2^-p - (1024 * 2^-p + 2)
   const uint32_t msk[5] = {0x00030003u, 0x000C000Cu, 0x00300030u, 0x00C000C0u, 0x03000300u};
   const uint32_t mag[5] = {0x64026402u, 0x64086408u, 0x64206420u, 0x64806480u, 0x66006600u};
   const uint32_t mul[5] = {0x3C003C00u, 0x34003400u, 0x2C002C00u, 0x24002400u, 0x1C001C00u};
   const uint32_t add[5] = {0xE402E402u, 0xDC08DC08u, 0xD420D420u, 0xCC80CC80u, 0xC600C600u};
+  uint32_t o[8];
+  const uint32_t hi = w >> 10;
 #pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    uint32_t o[8];
-    const uint32_t hi = w[i] >> 10;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const int p = c < 5 ? c : c - 5;
-      const uint32_t src = c < 5 ? w[i] : hi;
-      o[c] = h2_mul(h2_fma(and_xor(src, msk[p], mag[p]), mul[p], add[p]), s2);
-    }
-    out[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
-    out[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+  for (int c = 0; c < 8; ++c) {
+    const int p = c < 5 ? c : c - 5;
+    o[c] = h2_mul(h2_fma(and_xor(c < 5 ? w : hi, msk[p], mag[p]), mul[p], add[p]), s2);
+  }
+  out[0] = make_uint4(o[0], o[1], o[2], o[3]);
+  out[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+__device__ __forceinline__ uint32_t pick_word(const uint4& v, int i) {
+  return i == 0 ? v.x : (i == 1 ? v.y : (i == 2 ? v.z : v.w));
+}
+// Output chunks 2*pp and 2*pp+1 (16 inputs) of operand stage j of a packed row.
+__device__ __forceinline__ void dequant_pair(int bits, const unsigned char* rrow, int rin, int j, int pp, uint32_t s2,
+                                             uint4 (&out)[2]) {
+  if (bits == 8) {
+    dequant_chunk8(*reinterpret_cast<const uint4*>(rrow + (((4 * j + pp) ^ (rin & 7)) << 4)), s2, out);
+  } else if (bits == 4) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(rrow + (((2 * j + (pp >> 1)) ^ (rin & 7)) << 4));
+    out[0] = dequant_word4(pick_word(raw, 2 * (pp & 1)), s2);
+    out[1] = dequant_word4(pick_word(raw, 2 * (pp & 1) + 1), s2);
+  } else {
+    const uint4 raw = *reinterpret_cast<const uint4*>(rrow + ((j ^ (rin & 7)) << 4));
+    dequant_word2(pick_word(raw, pp), s2, out);
   }
 }
 
@@ -332,7 +343,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
   } else {
     // ---------------- dequantise (one thread per output channel), then epilogue ----------------
     const int quarter = warp & 3;          // TMEM lanes this warp may read: 32 * quarter ...
-    const int half = (warp - 2) >> 2;      // which half of a stage's chunks (and of the token columns) is this warp's
+    const int part = (warp - 2) >> 2;      // which share of a stage's chunks (and of the token columns) is this warp's
     const int r = 32 * quarter + lane;     // channel of the tile = row of the operand = TMEM lane
     const int box = r >> 6, rin = r & 63;
     const int G = L.group > 0 ? L.group : K;
@@ -368,30 +379,12 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
             const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
             const unsigned char* rrow = raw_ring + rs * UM_RAW_STAGE_BYTES + m * UM_TILE_BYTES + box * (UM_TILE_BYTES / 2) + rin * 128;
             unsigned char* arow = ab_ring + s * UM_AB_STAGE_BYTES + m * UM_TILE_BYTES + r * 128;
-            if (bits == 8) {
 #pragma unroll
-              for (int c = 2 * half; c < 2 * half + 2; ++c) {
-                const uint4 raw = *reinterpret_cast<const uint4*>(rrow + (((4 * j + c) ^ (rin & 7)) << 4));
-                uint4 o[2];
-                dequant_chunk8(raw, s2, o);
-                *reinterpret_cast<uint4*>(arow + (((2 * c) ^ (r & 7)) << 4)) = o[0];
-                *reinterpret_cast<uint4*>(arow + (((2 * c + 1) ^ (r & 7)) << 4)) = o[1];
-              }
-            } else if (bits == 4) {
-              {
-                const int c = half;
-                const uint4 raw = *reinterpret_cast<const uint4*>(rrow + (((2 * j + c) ^ (rin & 7)) << 4));
-                uint4 o[4];
-                dequant_chunk4(raw, s2, o);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(arow + (((4 * c + i) ^ (r & 7)) << 4)) = o[i];
-              }
-            } else {
-              const uint4 raw = *reinterpret_cast<const uint4*>(rrow + ((j ^ (rin & 7)) << 4));
-              uint4 o[4];
-              dequant_chunk2_half(raw, half, s2, o);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(arow + (((4 * half + i) ^ (r & 7)) << 4)) = o[i];
+            for (int pp = part * (4 / UM_PARTS); pp < (part + 1) * (4 / UM_PARTS); ++pp) {
+              uint4 o[2];
+              dequant_pair(bits, rrow, rin, j, pp, s2, o);
+              *reinterpret_cast<uint4*>(arow + (((2 * pp) ^ (r & 7)) << 4)) = o[0];
+              *reinterpret_cast<uint4*>(arow + (((2 * pp + 1) ^ (r & 7)) << 4)) = o[1];
             }
           }
           for (int m = 0; m < n_mats; ++m) sv[m] = sv_next[m];
@@ -405,7 +398,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
         ++raw_it;
       }
       if (!ok) break;
-      // ---- epilogue: this warp's 32 channels x 64 tokens ----
+      // ---- epilogue: this warp's 32 channels x its share of the token columns ----
       if (!mbar_wait(bar_acc_full, tile_it & 1, a.check_word, abort_flag)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int nrow = rb * UM_ROWS + r;
@@ -413,7 +406,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tt) * UM_TOK;
       const int hpos = a.phase == 0 ? pair_pos_rt(bits, min(nrow, N - 1)) : 0;
 #pragma unroll 1
-      for (int cc = 64 * half; cc < 64 * half + 64; cc += 32) {
+      for (int cc = (UM_TOK / UM_PARTS) * part; cc < (UM_TOK / UM_PARTS) * (part + 1); cc += 32) {
         uint32_t va[32], vb[32];
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + cc;
         tmem_ld32(taddr, va);
