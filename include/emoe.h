@@ -124,7 +124,7 @@ size_t emoe_scales_bytes(int N, int K, int group, int scale_dtype); /* N*(K/grou
 /* Quantises and packs one matrix W[N][K] (fp32, row-major, rows = output channels) to
  * `bits` in the storage format described at the top of this file.
  *   group: 0 or a divisor of K; the scale run (group, or K when group = 0) must be a multiple
- *   of 4 inputs and of 32 bits of codes (so 16 / 8 / 4 inputs at 2 / 4 / 8 bits).
+ *   of 4 inputs.
  *   out_packed: emoe_packed_bytes(N,K,bits) bytes; out_scales: emoe_scales_bytes(...).
  *   W and out_packed must be 16-byte aligned, out_scales 4-byte aligned.
  * Bit-exact with the definition: IEEE division and round-half-even, no fast-math. */

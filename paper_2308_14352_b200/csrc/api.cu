@@ -382,7 +382,7 @@ int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int 
   if (scale_dtype != EMOE_DTYPE_F32 && scale_dtype != EMOE_DTYPE_F16) return EMOE_ERR_UNSUPPORTED;
   const int G = group > 0 ? group : K;
   if (K % G != 0) return EMOE_ERR_INVALID_ARG;
-  if ((static_cast<long long>(G) * bits) % 32 != 0 || G % 4 != 0) return EMOE_ERR_UNSUPPORTED;
+  if (G % 4 != 0) return EMOE_ERR_UNSUPPORTED;
   if (!aligned(W, 16) || !aligned(out_packed, 16) || !aligned(out_scales, 4)) return EMOE_ERR_ALIGNMENT;
   EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
   EMOE_CUDA(ctx, launch_pack(W, N, K, bits, group, scale_dtype == EMOE_DTYPE_F16, static_cast<uint8_t*>(out_packed),

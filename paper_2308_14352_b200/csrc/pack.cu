@@ -1,7 +1,7 @@
 // Expert-wise quantisation kernel (paper Section 3.2, "Choosing the algorithm"):
 // channel-wise linear quantisation of an fp32 matrix to INT2/INT4/INT8 codes plus a scale
 // channel.  One warp owns one (output channel, group) unit: it finds the unit's max-abs,
-// derives the scale, then quantises and packs, each lane emitting whole 32-bit words of codes.
+// derives the scale, then quantises and packs, each lane emitting the codes of 4 consecutive weights.
 // HBM-bound: 4 bytes read and bits/8 bytes written per weight (the second read of a unit
 // comes from L1/L2).
 #include "common.cuh"
@@ -10,22 +10,36 @@ namespace emoe {
 namespace {
 
 template <int BITS>
+struct PackWord;  // the codes of 4 consecutive weights
+template <>
+struct PackWord<8> { typedef uint32_t type; };
+template <>
+struct PackWord<4> { typedef uint16_t type; };
+template <>
+struct PackWord<2> { typedef uint8_t type; };
+
+template <int BITS>
 __global__ void __launch_bounds__(256) pack_kernel(const float* __restrict__ W, int N, int K, int G, int ngroups,
                                                    int scale_f16, uint8_t* __restrict__ packed,
                                                    void* __restrict__ scales) {
-  constexpr int WPL = 32 / BITS;  // weights per 32-bit output word
+  typedef typename PackWord<BITS>::type word_t;
   constexpr int MASK = (1 << BITS) - 1;
   const float qmax = static_cast<float>((1 << (BITS - 1)) - 1);
   const int lane = threadIdx.x & 31;
-  const long long unit = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-  if (unit >= static_cast<long long>(N) * ngroups) return;
+  const long long n_units = static_cast<long long>(N) * ngroups;
+  const long long warps = (static_cast<long long>(gridDim.x) * blockDim.x) >> 5;
+  for (long long unit = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; unit < n_units; unit += warps) {
   const int n = static_cast<int>(unit / ngroups);
   const int g = static_cast<int>(unit % ngroups);
   const float* w = W + static_cast<size_t>(n) * K + static_cast<size_t>(g) * G;
 
+  // every lane owns 4 consecutive weights per 128-weight step; with 128-weight groups the
+  // weights stay in registers between the two passes
+  float4 first = make_float4(0.f, 0.f, 0.f, 0.f);
   float amax = 0.0f;
   for (int i = lane * 4; i < G; i += 128) {
     const float4 v = *reinterpret_cast<const float4*>(w + i);
+    if (i < 128) first = v;
     amax = fmaxf(amax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
   }
 #pragma unroll
@@ -41,26 +55,24 @@ __global__ void __launch_bounds__(256) pack_kernel(const float* __restrict__ W, 
     reinterpret_cast<float*>(scales)[unit] = s;
   }
 
-  uint32_t* out = reinterpret_cast<uint32_t*>(packed + static_cast<size_t>(n) * (static_cast<size_t>(K) * BITS / 8) +
-                                              static_cast<size_t>(g) * G * BITS / 8);
-  for (int i = lane * WPL; i < G; i += 32 * WPL) {
+  word_t* out = reinterpret_cast<word_t*>(packed + static_cast<size_t>(n) * (static_cast<size_t>(K) * BITS / 8) +
+                                          static_cast<size_t>(g) * G * BITS / 8);
+  for (int i = lane * 4; i < G; i += 128) {
+    const float4 v = i < 128 ? first : *reinterpret_cast<const float4*>(w + i);
+    const float e[4] = {v.x, v.y, v.z, v.w};
     uint32_t word = 0;
 #pragma unroll
-    for (int j = 0; j < WPL / 4; ++j) {
-      const float4 v = *reinterpret_cast<const float4*>(w + i + 4 * j);
-      const float e[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        int q = 0;
-        if (s != 0.0f) {
-          float r = rintf(__fdiv_rn(e[c], s));  // round half to even on the quotient by the stored scale
-          r = fminf(fmaxf(r, -qmax), qmax);
-          q = static_cast<int>(r);
-        }
-        word |= static_cast<uint32_t>(q & MASK) << (BITS * (4 * j + c));
+    for (int c = 0; c < 4; ++c) {
+      int q = 0;
+      if (s != 0.0f) {
+        float r = rintf(__fdiv_rn(e[c], s));  // round half to even on the quotient by the stored scale
+        r = fminf(fmaxf(r, -qmax), qmax);
+        q = static_cast<int>(r);
       }
+      word |= static_cast<uint32_t>(q & MASK) << (BITS * c);
     }
-    out[i / WPL] = word;
+    out[i >> 2] = static_cast<word_t>(word);
+  }
   }
 }
 
@@ -72,8 +84,9 @@ cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int s
   const int ngroups = K / G;
   const long long units = static_cast<long long>(N) * ngroups;
   const int threads = 256;
-  const long long blocks = (units * 32 + threads - 1) / threads;
-  if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+  long long blocks = (units * 32 + threads - 1) / threads;
+  const long long cap = 148LL * 8 * 4;  // a few waves of resident blocks; each warp then loops over its units
+  if (blocks > cap) blocks = cap;
   const dim3 grid(static_cast<unsigned>(blocks));
   switch (bits) {
     case 2: pack_kernel<2><<<grid, threads, 0, st>>>(W, N, K, G, ngroups, scale_f16, packed, scales); break;
