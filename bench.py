@@ -50,6 +50,7 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying a CUDA graph")
     ap.add_argument("--ffn-path", type=int, default=0, help="0 auto, 1 CUDA-core GEMV, 2 tensor-core path")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-pdl", action="store_true", help="switch programmatic dependent launch off")
     return ap.parse_args()
 
 
@@ -255,6 +256,7 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
     desc = L.make_desc(sh)
     ctx = B.emoe_create(local, B.emoe_workspace_bytes(desc, T))
     B.emoe_set_ffn_path(ctx, args.ffn_path)
+    B.emoe_set_dependent_launch(ctx, not args.no_pdl)
 
     # ---- build the stack: seeded fp32 experts -> packed on the device by the library ------------
     t_build = time.perf_counter()

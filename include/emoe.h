@@ -188,6 +188,11 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
  * they do not take.  For tests and measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);
 
+/* Programmatic dependent launch along the kernels of a forward call (on by default): each
+ * kernel may start its prologue while the one in front drains.  Results are identical either
+ * way; switch it off to compare timings or when a tool in use does not support the attribute. */
+int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled);
+
 /* The routed layer forward for callers that cannot allocate device memory (the paper has no
  * counterpart: it is an addition for hosts such as a framework that owns the whole device
  * heap, a plug-in whose memory pool is fixed at start-up, or a latency-critical loop in which

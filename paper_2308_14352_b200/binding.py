@@ -29,7 +29,7 @@ EXPORTS = (
     "emoe_create", "emoe_destroy", "emoe_workspace_bytes", "emoe_last_cuda_error", "emoe_device_status",
     "emoe_status_string", "emoe_packed_bytes", "emoe_scales_bytes", "emoe_pack_expert", "emoe_router_topk",
     "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
-    "emoe_read_timing", "emoe_moe_forward_routed_static",
+    "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_set_dependent_launch",
 )
 
 
@@ -84,6 +84,7 @@ def lib() -> ctypes.CDLL:
                                               ctypes.POINTER(emoe_expert), vp, vp, vp]
         L.emoe_set_ffn_path.argtypes = [vp, i32]
         L.emoe_set_timing.argtypes = [vp, i32]
+        L.emoe_set_dependent_launch.argtypes = [vp, i32]
         L.emoe_moe_forward_routed_static.argtypes = [i32, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
                                                      ctypes.POINTER(emoe_expert), vp, vp]
         L.emoe_read_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
@@ -196,3 +197,7 @@ def emoe_moe_forward_routed_static(device: int, desc: emoe_layer_desc, x_ptr, T,
     inside the library; T * top_k <= 64).  For callers that may not allocate."""
     _check(lib().emoe_moe_forward_routed_static(device, ctypes.byref(desc), x_ptr, T, ids_ptr, gates_ptr,
                                                 expert_table, y_ptr, stream), "emoe_moe_forward_routed_static")
+
+
+def emoe_set_dependent_launch(ctx, enabled: bool) -> None:
+    _check(lib().emoe_set_dependent_launch(ctx, int(enabled)), "emoe_set_dependent_launch")

@@ -10,6 +10,10 @@
 
 using namespace emoe;
 
+namespace emoe {
+thread_local bool g_pdl_enabled = false;
+}
+
 namespace {
 
 constexpr int MAX_TABLES = 128;  // distinct expert tables a context can keep on the device
@@ -90,6 +94,7 @@ struct emoe_ctx {
   std::vector<TableEntry> tables;
   int last_cuda = 0;
   int ffn_path = 0;
+  bool pdl = true;  // programmatic dependent launch along the kernel chain of a forward call
   bool timing = false;
   std::vector<cudaEvent_t> events;  // triples (start, mid, end) per timed forward call
   size_t events_used = 0;
@@ -198,6 +203,10 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   const WorkspaceLayout w = make_layout(L, T);
   if (w.total > ctx->workspace_bytes) return EMOE_ERR_WORKSPACE;
   EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+  struct PdlScope {
+    explicit PdlScope(bool on) { g_pdl_enabled = on; }
+    ~PdlScope() { g_pdl_enabled = false; }
+  } pdl_scope(ctx->pdl && !ctx->timing);
 
   const ExpertDev* table = nullptr;
   const void* tmaps = nullptr;
@@ -454,6 +463,12 @@ int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, i
   *out_second_ms = b;
   *out_calls = static_cast<int>(n);
   ctx->events_used = 0;
+  return EMOE_OK;
+}
+
+int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  ctx->pdl = enabled != 0;
   return EMOE_OK;
 }
 

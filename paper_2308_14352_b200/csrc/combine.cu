@@ -10,6 +10,8 @@ namespace {
 __global__ void __launch_bounds__(256)
     combine_kernel(const float* __restrict__ o_part, int ksplit, size_t part_stride, const float* __restrict__ gates,
                    const int32_t* __restrict__ slot_of_pair, int T, int top_k, int d, float* __restrict__ y) {
+  pdl_wait();
+  pdl_trigger();
   const int d4 = d >> 2;
   const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (idx >= static_cast<size_t>(T) * d4) return;
@@ -40,9 +42,8 @@ cudaError_t launch_combine(const float* o_part, int ksplit, size_t n_pairs_strid
                            const int32_t* slot_of_pair, int T, int top_k, int d, float* y, cudaStream_t st) {
   const size_t total = static_cast<size_t>(T) * (d >> 2);
   const unsigned blocks = static_cast<unsigned>((total + 255) / 256);
-  combine_kernel<<<blocks, 256, 0, st>>>(o_part, ksplit, n_pairs_stride * d * sizeof(float), gates, slot_of_pair, T,
-                                         top_k, d, y);
-  return cudaGetLastError();
+  return launch_chain(combine_kernel, dim3(blocks), dim3(256), 0, st, o_part, ksplit, n_pairs_stride * d * sizeof(float), gates,
+                      slot_of_pair, T, top_k, d, y);
 }
 
 }  // namespace emoe

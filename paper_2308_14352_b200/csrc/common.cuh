@@ -38,6 +38,37 @@ struct LayerDims {
   int d_model, d_ff, E, top_k, act, gate_mode, group, scale_f16, act_bf16;
 };
 
+// ---- programmatic dependent launch ---------------------------------------------------------
+// The kernels of a forward call form a chain on one stream.  When enabled (per host thread,
+// set by the forward call from its context), every launch carries the "programmatic stream
+// serialization" attribute: the next kernel of the chain may start its prologue (barrier set-up,
+// tensor-memory allocation, fetching weights that no kernel of the chain writes) while the
+// current one drains.  Device side, every kernel executes pdl_wait() before it touches anything
+// an earlier kernel of the chain wrote or read, and pdl_trigger() right after, which lets the
+// kernel behind it start.  Without the attribute both are no-ops.
+extern thread_local bool g_pdl_enabled;
+
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  if (g_pdl_enabled) {
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+  }
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- launchers (each enqueues on `st` and returns the launch error) ---------------------
 cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int scale_f16, uint8_t* packed,
                         void* scales, cudaStream_t st);

@@ -160,6 +160,8 @@ __global__ void __launch_bounds__(GEMV_WARPS * 32)
     ffn_gemv_kernel(int phase, LayerDims L, const ExpertDev* __restrict__ experts, const void* __restrict__ x,
                     const int32_t* __restrict__ perm, const int32_t* __restrict__ off, void* hidden,
                     float* __restrict__ o) {
+  pdl_wait();
+  pdl_trigger();
   const int e = blockIdx.y;
   const int begin = off[e];
   const int cnt = off[e + 1] - begin;
@@ -181,8 +183,7 @@ cudaError_t launch_ffn_gemv(int phase, const LayerDims& L, const ExpertDev* expe
   (void)n_pairs;
   const int N = phase == 0 ? L.d_ff : L.d_model;
   const dim3 grid((N + GEMV_WARPS - 1) / GEMV_WARPS, L.E);
-  ffn_gemv_kernel<<<grid, GEMV_WARPS * 32, 0, st>>>(phase, L, experts, x, perm, off, hidden, o);
-  return cudaGetLastError();
+  return launch_chain(ffn_gemv_kernel, grid, dim3(GEMV_WARPS * 32), 0, st, phase, L, experts, x, perm, off, hidden, o);
 }
 
 }  // namespace emoe

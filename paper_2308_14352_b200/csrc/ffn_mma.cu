@@ -185,6 +185,8 @@ __global__ void __launch_bounds__(MMA_THREADS)
                    const int32_t* __restrict__ off, __nv_bfloat16* __restrict__ hidden, float* __restrict__ o_part,
                    int ksplit, int n_pairs) {
   __shared__ __align__(16) __nv_bfloat16 xsm[NT * 8 * MMA_XSTRIDE];
+  pdl_wait();
+  pdl_trigger();
   const int e = blockIdx.z;
   const int begin = off[e];
   const int cnt = off[e + 1] - begin;
@@ -206,6 +208,8 @@ __global__ void __launch_bounds__(128)
     scatter_x_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
                      const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
                      int E, int* __restrict__ plan, int top_k, int d, int n_pairs, __nv_bfloat16* __restrict__ xs) {
+  pdl_wait();
+  pdl_trigger();
   if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
     // work plan of the persistent expert kernels: activated experts, widest codes (most bytes)
     // first; the two item counters restart from zero
@@ -299,9 +303,8 @@ int ffn_mma_ksplit(const LayerDims& L, int T) {
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
                              cudaStream_t st) {
-  scatter_x_kernel<<<n_pairs, 128, 0, st>>>(experts, reinterpret_cast<const __nv_bfloat16*>(x), ids, perm, off, L.E, plan,
-                                            L.top_k, L.d_model, n_pairs, xs);
-  return cudaGetLastError();
+  return launch_chain(scatter_x_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
+                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, xs);
 }
 
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
@@ -312,11 +315,10 @@ cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* exper
   const dim3 grid((N + rows_per_cta - 1) / rows_per_cta, phase == 0 ? 1 : ksplit, L.E);
   const int z = phase == 0 ? 1 : ksplit;
   switch (ffn_token_tiles(L, T)) {
-    case 1: ffn_mma_kernel<1><<<grid, MMA_THREADS, 0, st>>>(phase, L, experts, in, off, hidden, o_part, z, n_pairs); break;
-    case 2: ffn_mma_kernel<2><<<grid, MMA_THREADS, 0, st>>>(phase, L, experts, in, off, hidden, o_part, z, n_pairs); break;
-    default: ffn_mma_kernel<4><<<grid, MMA_THREADS, 0, st>>>(phase, L, experts, in, off, hidden, o_part, z, n_pairs); break;
+    case 1: return launch_chain(ffn_mma_kernel<1>, grid, dim3(MMA_THREADS), 0, st, phase, L, experts, in, off, hidden, o_part, z, n_pairs);
+    case 2: return launch_chain(ffn_mma_kernel<2>, grid, dim3(MMA_THREADS), 0, st, phase, L, experts, in, off, hidden, o_part, z, n_pairs);
+    default: return launch_chain(ffn_mma_kernel<4>, grid, dim3(MMA_THREADS), 0, st, phase, L, experts, in, off, hidden, o_part, z, n_pairs);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace emoe

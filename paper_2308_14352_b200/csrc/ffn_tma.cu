@@ -293,6 +293,12 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
   // harmless: a column of the MMA result depends only on its own column of B, and columns past
   // the expert's token count are never stored.
   __syncthreads();
+  // Everything above overlaps the tail of the kernel in front.  The first projection needs that
+  // kernel's results (the plan) at once; the second projection's plan, weights and scales are
+  // older than the kernel in front, so its producer starts fetching them and waits only before
+  // the first copy of a hidden vector (see `waited` below).
+  if (a.phase == 0) pdl_wait();
+  pdl_trigger();
 
   const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + STAGES);
   const LayerDims& L = a.L;
@@ -313,6 +319,9 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
     const int per_expert = a.ksplit * a.row_blocks;
     int it = 0;
     bool ok = true;
+    bool waited = a.phase == 0;  // false: copies of activation rows are parked until pdl_wait()
+    int n_parked = 0;
+    int park_stage[STAGES], park_row[STAGES], park_k0[STAGES], park_klen[STAGES], park_ntok[STAGES];
     // Item look-ahead of two: the counter increment for item i+2 and the expert record of item
     // i+1 are issued before item i is streamed and only read after it, so that switching items
     // costs no round trip to memory.  A CTA's first item is its own index; the counter hands
@@ -383,9 +392,18 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           }
           __syncwarp();
           if (klen > 0) {
-            for (int r = lane; r < ntok; r += 32)
-              bulk_load(smem_u32(st + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
-                        a.in + static_cast<size_t>(begin + p0 + r) * K + k0, klen * 2, full);
+            if (waited) {
+              for (int r = lane; r < ntok; r += 32)
+                bulk_load(smem_u32(st + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
+                          a.in + static_cast<size_t>(begin + p0 + r) * K + k0, klen * 2, full);
+            } else {
+              park_stage[n_parked] = stage;
+              park_row[n_parked] = begin + p0;
+              park_k0[n_parked] = k0;
+              park_klen[n_parked] = klen;
+              park_ntok[n_parked] = ntok;
+              ++n_parked;
+            }
             // scales: lane l copies the windows of rows 4l .. 4l+3 of the stage (box-major)
             const int nseg = klen / 128;
             const int g0 = group_of(k0, Gk, ngroups_k), g1 = group_of(k0 + (nseg - 1) * 128, Gk, ngroups_k);
@@ -404,6 +422,16 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full) : "memory");
           } else {
             mbar_arrive(full);  // with lane 0's arrival above: 33 in all
+          }
+          if (!waited && n_parked == STAGES) {  // the ring is full: nothing more can be fetched early
+            pdl_wait();
+            waited = true;
+            for (int i = 0; i < n_parked; ++i)
+              for (int r = lane; r < park_ntok[i]; r += 32)
+                bulk_load(smem_u32(smem + park_stage[i] * STAGE_BYTES + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
+                          a.in + static_cast<size_t>(park_row[i] + r) * K + park_k0[i], park_klen[i] * 2,
+                          bar_full + 8 * park_stage[i]);
+            n_parked = 0;
           }
         }
       }
@@ -433,6 +461,16 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           asm volatile("prefetch.global.L2 [%0];" ::"l"(base + static_cast<size_t>(i % lines) * 128));
         }
       }
+    }
+    if (!waited) {  // fewer stages than the ring holds: release the parked copies now
+      pdl_wait();
+      waited = true;
+      for (int i = 0; i < n_parked; ++i)
+        for (int r = lane; r < park_ntok[i]; r += 32)
+          bulk_load(smem_u32(smem + park_stage[i] * STAGE_BYTES + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
+                    a.in + static_cast<size_t>(park_row[i] + r) * K + park_k0[i], park_klen[i] * 2,
+                    bar_full + 8 * park_stage[i]);
+      n_parked = 0;
     }
     if (ok && !*abort_flag) {  // tell the consumers that nothing else comes
       const int stage = it % STAGES;
@@ -509,8 +547,7 @@ cudaError_t launch_nt(const TmaArgs& a, int max_items, cudaStream_t st) {
     ctas_per_device[dev] = (per_sm > 0 ? per_sm : 1) * sms;
   }
   const int grid = max_items < ctas_per_device[dev] ? max_items : ctas_per_device[dev];
-  ffn_tma_kernel<NT><<<grid, TMA_THREADS, SMEM, st>>>(a);
-  return cudaGetLastError();
+  return launch_chain(ffn_tma_kernel<NT>, dim3(grid), dim3(TMA_THREADS), SMEM, st, a);
 }
 
 }  // namespace

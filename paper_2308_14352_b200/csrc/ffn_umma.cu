@@ -252,6 +252,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = tmem_base_slot;
+  pdl_wait();  // barrier set-up and the tensor-memory allocation overlap the kernel in front
+  pdl_trigger();
 
   const LayerDims& L = a.L;
   const int N = a.phase == 0 ? L.d_ff : L.d_model;
@@ -454,6 +456,8 @@ __global__ void __launch_bounds__(128)
     scatter_x16_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
                        const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
                        int E, int* __restrict__ plan, int top_k, int d, int n_pairs, __half* __restrict__ xs) {
+  pdl_wait();
+  pdl_trigger();
   if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
     // work plan: activated experts, widest codes first
     const int lane = threadIdx.x;
@@ -505,9 +509,8 @@ bool ffn_umma_supported(const LayerDims& L) {
 cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
                                cudaStream_t st) {
-  scatter_x16_kernel<<<n_pairs, 128, 0, st>>>(experts, reinterpret_cast<const __nv_bfloat16*>(x), ids, perm, off, L.E, plan,
-                                              L.top_k, L.d_model, n_pairs, reinterpret_cast<__half*>(xs16));
-  return cudaGetLastError();
+  return launch_chain(scatter_x16_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
+                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, reinterpret_cast<__half*>(xs16));
 }
 
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
@@ -541,8 +544,7 @@ cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, co
   a.hidden16 = reinterpret_cast<__half*>(hidden16);
   a.o = o;
   a.check_word = check_word;
-  ffn_umma_kernel<<<grid, UM_THREADS, UM_SMEM_BYTES, st>>>(a, tmap_b);
-  return cudaGetLastError();
+  return launch_chain(ffn_umma_kernel, dim3(grid), dim3(UM_THREADS), UM_SMEM_BYTES, st, a, tmap_b);
 }
 
 }  // namespace emoe

@@ -36,6 +36,9 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
   const int S = ROUTER_THREADS >> ep_shift;
   const int t0 = blockIdx.x * TT;
 
+  // x and the router weights are inputs of the call: the logits are computed while the kernels
+  // in front drain; the wait comes before the first write (ids / gates may still be read there)
+  pdl_trigger();
   float acc[TT];
 #pragma unroll
   for (int tt = 0; tt < TT; ++tt) acc[tt] = 0.0f;
@@ -76,6 +79,7 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
 #pragma unroll
   for (int tt = 0; tt < TT; ++tt) red[(slice * TT + tt) * EP + e] = acc[tt];
   __syncthreads();
+  pdl_wait();
   for (int idx = tid; idx < TT * EP; idx += ROUTER_THREADS) {
     const int tt = idx >> ep_shift, ee = idx & (EP - 1);
     const int t = t0 + tt;
@@ -168,6 +172,8 @@ __global__ void __launch_bounds__(1024)
   int* wcnt = cursor + E; // [32][E]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+  pdl_wait();
+  pdl_trigger();
   for (int e = tid; e < E; e += 1024) cnt[e] = 0;
   __syncthreads();
   bool bad = false;
@@ -252,13 +258,13 @@ cudaError_t launch_router_topk(const void* x, int x_bf16, int T, int d, const fl
   if (T >= 8 * 64) {
     constexpr int TT = 8;
     const size_t smem = sizeof(float) * (TT * ROUTER_DC + ROUTER_THREADS * TT + TT * EP);  // <= 48 KB
-    router_topk_kernel<TT><<<(T + TT - 1) / TT, ROUTER_THREADS, smem, st>>>(x, x_bf16, T, d, Wr, bias, bias_stride, E, EP,
-                                                                          sh, top_k, renorm, ids, gates, logits);
+    return launch_chain(router_topk_kernel<TT>, dim3((T + TT - 1) / TT), dim3(ROUTER_THREADS), smem, st, x, x_bf16, T, d, Wr, bias,
+                        bias_stride, E, EP, sh, top_k, renorm, ids, gates, logits);
   } else {
     constexpr int TT = 1;
     const size_t smem = sizeof(float) * (TT * ROUTER_DC + ROUTER_THREADS * TT + TT * EP);
-    router_topk_kernel<TT><<<T, ROUTER_THREADS, smem, st>>>(x, x_bf16, T, d, Wr, bias, bias_stride, E, EP, sh, top_k,
-                                                          renorm, ids, gates, logits);
+    return launch_chain(router_topk_kernel<TT>, dim3(T), dim3(ROUTER_THREADS), smem, st, x, x_bf16, T, d, Wr, bias, bias_stride, E,
+                        EP, sh, top_k, renorm, ids, gates, logits);
   }
   return cudaGetLastError();
 }
@@ -266,8 +272,7 @@ cudaError_t launch_router_topk(const void* x, int x_bf16, int T, int d, const fl
 cudaError_t launch_permute(const int32_t* ids, int n_pairs, int E, int32_t* counts, int32_t* off, int32_t* perm,
                            int32_t* slot_of_pair, int* check_word, cudaStream_t st) {
   const size_t smem = sizeof(int) * (2 * E + 32 * E);
-  permute_kernel<<<1, 1024, smem, st>>>(ids, n_pairs, E, counts, off, perm, slot_of_pair, check_word);
-  return cudaGetLastError();
+  return launch_chain(permute_kernel, dim3(1), dim3(1024), smem, st, ids, n_pairs, E, counts, off, perm, slot_of_pair, check_word);
 }
 
 }  // namespace emoe
