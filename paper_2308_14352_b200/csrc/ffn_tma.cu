@@ -43,6 +43,9 @@ constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a s
 #ifndef EMOE_TMA_STAGES_NT1
 #define EMOE_TMA_STAGES_NT1 3
 #endif
+#ifndef EMOE_TMA_UNROLL_SEGS
+#define EMOE_TMA_UNROLL_SEGS 0
+#endif
 #ifndef EMOE_TMA_LOOKAHEAD
 #define EMOE_TMA_LOOKAHEAD 0
 #endif
@@ -145,7 +148,11 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, int rb, int k0, 
   const int nrow0 = swiglu_in ? rb * TMA_BOX_ROWS + 16 * warp : rb * 2 * TMA_BOX_ROWS + 32 * warp;
   const int nseg = min(SEGS, (K - k0) / 128);
   const int g0 = group_of(k0, G, ngroups);
+#if EMOE_TMA_UNROLL_SEGS
 #pragma unroll
+#else
+#pragma unroll 1
+#endif
   for (int sg = 0; sg < SEGS; ++sg) {
     if (sg < nseg) {
       // B fragments: piece q of lane t sits at (q*4 + t) * 16 bytes of the segment
