@@ -46,6 +46,9 @@ constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a s
 #ifndef EMOE_TMA_UNROLL_SEGS
 #define EMOE_TMA_UNROLL_SEGS 0
 #endif
+#ifndef EMOE_TMA_L2PROMO
+#define EMOE_TMA_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+#endif
 #ifndef EMOE_TMA_LOOKAHEAD
 #define EMOE_TMA_LOOKAHEAD 0
 #endif
@@ -628,7 +631,7 @@ int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, u
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(static_cast<CUtensorMap*>(out_map), dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
                         2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                        CU_TENSOR_MAP_SWIZZLE_128B, EMOE_TMA_L2PROMO, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : -3;
 }
 
