@@ -272,11 +272,12 @@ __global__ void __launch_bounds__(128)
 }  // namespace
 
 // 8-token tiles a CTA handles per pass over its weights: enough for the mean tokens per expert
-// plus 2.5 standard deviations under uniform routing (an expert with more tokens takes another
-// pass over its own weights, which then come from L2).
+// plus 2.5 standard deviations under uniform routing (a token picks an expert with probability
+// top_k / E); an expert with more tokens takes another pass over its own weights.
 int ffn_token_tiles(const LayerDims& L, int T) {
-  const double mean = static_cast<double>(T) * L.top_k / L.E;
-  double need = mean + 2.5 * sqrt(mean) + 1.0;
+  const double p = static_cast<double>(L.top_k) / L.E;
+  const double mean = T * p;
+  double need = mean + 2.5 * sqrt(T * p * (1.0 - p));
   if (need > T) need = T;
   return need <= 8.0 ? 1 : (need <= 16.0 ? 2 : 4);
 }
