@@ -51,6 +51,7 @@ def parse_args():
     ap.add_argument("--ffn-path", type=int, default=0, help="0 auto, 1 CUDA-core GEMV, 2 tensor-core path")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pdl", action="store_true", help="switch programmatic dependent launch off")
+    ap.add_argument("--no-fuse", action="store_true", help="run the two projections of the expert FFNs as two launches")
     return ap.parse_args()
 
 
@@ -257,6 +258,7 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
     ctx = B.emoe_create(local, B.emoe_workspace_bytes(desc, T))
     B.emoe_set_ffn_path(ctx, args.ffn_path)
     B.emoe_set_dependent_launch(ctx, not args.no_pdl)
+    B.emoe_set_fused_projections(ctx, not args.no_fuse)
 
     # ---- build the stack: seeded fp32 experts -> packed on the device by the library ------------
     t_build = time.perf_counter()

@@ -193,6 +193,13 @@ int emoe_set_ffn_path(emoe_ctx* ctx, int path);
  * way; switch it off to compare timings or when a tool in use does not support the attribute. */
 int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled);
 
+/* Both projections of the activated experts' FFNs (paper Section 2.1: an expert is one FFN) in a
+ * single launch of the weight-streaming kernel (on by default): an expert's second projection
+ * starts as soon as all of its hidden vectors are written, instead of after the first
+ * projection of every expert.  Results are identical either way; switch it off to run the two
+ * projections as two launches (to compare timings, or to time them separately). */
+int emoe_set_fused_projections(emoe_ctx* ctx, int enabled);
+
 /* The routed layer forward for callers that cannot allocate device memory (the paper has no
  * counterpart: it is an addition for hosts such as a framework that owns the whole device
  * heap, a plug-in whose memory pool is fixed at start-up, or a latency-critical loop in which

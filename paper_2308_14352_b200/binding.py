@@ -30,6 +30,7 @@ EXPORTS = (
     "emoe_status_string", "emoe_packed_bytes", "emoe_scales_bytes", "emoe_pack_expert", "emoe_router_topk",
     "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
     "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_set_dependent_launch",
+    "emoe_set_fused_projections",
 )
 
 
@@ -85,6 +86,7 @@ def lib() -> ctypes.CDLL:
         L.emoe_set_ffn_path.argtypes = [vp, i32]
         L.emoe_set_timing.argtypes = [vp, i32]
         L.emoe_set_dependent_launch.argtypes = [vp, i32]
+        L.emoe_set_fused_projections.argtypes = [vp, i32]
         L.emoe_moe_forward_routed_static.argtypes = [i32, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
                                                      ctypes.POINTER(emoe_expert), vp, vp]
         L.emoe_read_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
@@ -201,3 +203,7 @@ def emoe_moe_forward_routed_static(device: int, desc: emoe_layer_desc, x_ptr, T,
 
 def emoe_set_dependent_launch(ctx, enabled: bool) -> None:
     _check(lib().emoe_set_dependent_launch(ctx, int(enabled)), "emoe_set_dependent_launch")
+
+
+def emoe_set_fused_projections(ctx, enabled: bool) -> None:
+    _check(lib().emoe_set_fused_projections(ctx, int(enabled)), "emoe_set_fused_projections")

@@ -95,6 +95,7 @@ struct emoe_ctx {
   int last_cuda = 0;
   int ffn_path = 0;
   bool pdl = true;  // programmatic dependent launch along the kernel chain of a forward call
+  bool fuse_projections = true;  // weight-streaming kernel: both projections in one launch
   bool timing = false;
   std::vector<cudaEvent_t> events;  // triples (start, mid, end) per timed forward call
   size_t events_used = 0;
@@ -267,11 +268,16 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     ksplit = ffn_tma_ksplit(L, T);
     EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
-    EMOE_CUDA(ctx, launch_ffn_tma(0, L, table, tmaps, xs, off, plan, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T,
-                                  ctx->check_word, st));
-    if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-    EMOE_CUDA(ctx, launch_ffn_tma(1, L, table, tmaps, reinterpret_cast<const __nv_bfloat16*>(hidden), off, plan,
-                                  reinterpret_cast<__nv_bfloat16*>(hidden), o_part, ksplit, P, T, ctx->check_word, st));
+    __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
+    if (ctx->fuse_projections) {
+      // one launch: an expert's second projection starts when its hidden vectors are complete
+      EMOE_CUDA(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+    } else {
+      EMOE_CUDA(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+      EMOE_CUDA(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+    }
   } else if (use_mma) {
     ksplit = ffn_mma_ksplit(L, T);
     EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, st));
@@ -469,6 +475,12 @@ int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, i
 int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled) {
   if (!ctx) return EMOE_ERR_INVALID_ARG;
   ctx->pdl = enabled != 0;
+  return EMOE_OK;
+}
+
+int emoe_set_fused_projections(emoe_ctx* ctx, int enabled) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  ctx->fuse_projections = enabled != 0;
   return EMOE_OK;
 }
 

@@ -25,11 +25,14 @@ enum : int {
 
 // Work plan of the persistent expert kernels, built on the device after the permutation:
 // a 16-byte header {activated experts, item counter of the first projection, of the second, 0}
-// followed by one record per activated expert, widest codes first.
+// followed by one record per activated expert, widest codes first.  `done` counts the finished
+// pieces of the expert's first projection (zeroed with the plan): the fused expert kernel starts
+// an expert's second projection once the count is complete.
 struct PlanRec {
   int32_t e, begin, cnt, bits;
   const void* scales[3];
-  int64_t pad;
+  int32_t done;
+  int32_t pad;
 };
 constexpr size_t PLAN_HEADER_BYTES = 16;
 inline size_t plan_bytes(int E) { return PLAN_HEADER_BYTES + sizeof(PlanRec) * static_cast<size_t>(E); }
@@ -107,9 +110,12 @@ cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* exper
 bool ffn_tma_supported(const LayerDims& L);
 int ffn_tma_ksplit(const LayerDims& L, int T);
 int encode_weight_tmap(void* out_map, const void* packed, int N, int K, int bits);
-cudaError_t launch_ffn_tma(int phase, const LayerDims& L, const ExpertDev* experts, const void* tmaps,
-                           const __nv_bfloat16* in, const int32_t* off, int* plan, __nv_bfloat16* hidden, float* o_part,
-                           int ksplit, int n_pairs, int T, int* check_word, cudaStream_t st);
+// Phases [phase_begin, phase_end) of the FFN in one launch: (0,1) first projection, (1,2) second,
+// (0,2) both, the second projection of an expert starting as soon as its hidden vectors are complete.
+cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, const ExpertDev* experts,
+                           const void* tmaps, const __nv_bfloat16* xs, const int32_t* off, int* plan,
+                           __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs, int T, int* check_word,
+                           cudaStream_t st);
 
 int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
                    uint32_t box_inner, uint32_t box_outer);

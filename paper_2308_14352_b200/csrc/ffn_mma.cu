@@ -230,6 +230,7 @@ __global__ void __launch_bounds__(128)
           r.scales[0] = experts[e].scales[0];
           r.scales[1] = experts[e].scales[1];
           r.scales[2] = experts[e].scales[2];
+          r.done = 0;
         }
         base += __popc(m);
       }

@@ -108,43 +108,67 @@ __device__ __forceinline__ int group_of(int k, int G, int ngroups) {
 }
 
 struct TmaArgs {
-  int phase;
+  int phase_begin, phase_end;  // projections this launch runs: [0,1), [1,2) or both, [0,2)
   LayerDims L;
   const ExpertDev* experts;
   const CUtensorMap* tmaps;  // [E][3]
-  const __nv_bfloat16* in;
+  const __nv_bfloat16* xs;   // input of the first projection (tokens in expert order)
   const int32_t* off;
   int* plan;  // header {activated experts, item counters} + one PlanRec per activated expert
-  __nv_bfloat16* hidden;
+  __nv_bfloat16* hidden;  // output of the first projection, input of the second
   float* o_part;
-  int ksplit;
-  int row_blocks;
+  int ksplit;         // split-K slices of the second projection
+  int row_blocks[2];  // row blocks of an expert per projection
   int n_pairs;
   int* check_word;
 };
 
+// what differs between the two projections
+struct PhaseDims {
+  int K, N, rows_per_item, row_blocks, ksplit, mat_first;
+  bool swiglu_in;
+};
+__device__ __forceinline__ PhaseDims phase_dims(const TmaArgs& a, int phase) {
+  PhaseDims d;
+  d.K = phase == 0 ? a.L.d_model : a.L.d_ff;
+  d.N = phase == 0 ? a.L.d_ff : a.L.d_model;
+  d.swiglu_in = phase == 0 && a.L.act == EMOE_ACT_SWIGLU;
+  d.rows_per_item = d.swiglu_in ? TMA_BOX_ROWS : 2 * TMA_BOX_ROWS;
+  d.row_blocks = a.row_blocks[phase];
+  d.ksplit = phase == 0 ? 1 : a.ksplit;
+  d.mat_first = phase == 0 ? 0 : (a.L.act == EMOE_ACT_SWIGLU ? 2 : 1);
+  return d;
+}
+
 // what a stage holds, written by the producer before it arms the stage's barrier
 struct StageMeta {
   int e, rb, z, begin, p0, ntok, k0, bits;
-  int flags;  // 1 = first stage of an item pass, 2 = last, 4 = no more work, 8 = stage carries no inputs
-  int pad;
+  int flags;  // 1 = first stage of an item pass, 2 = last, 4 = no more work, 8 = stage carries no inputs,
+              // 16 = last stage of a first-projection item whose completion the second projection waits for
+  int phase;
   const void* scales[2];  // scale channel of the matrix behind each m-tile
+  int ai;                 // index of the expert's plan record
+  int pad;
 };
-constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8;
+constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8, META_DONE = 16;
+
+// How long the second projection of an expert waits for its hidden vectors (polls of ~0.1 us).
+constexpr unsigned DEP_WAIT_LIMIT = 1u << 20;
 
 template <int BITS, int NT>
-__device__ __forceinline__ void consume_stage(const TmaArgs& a, int rb, int k0, int ntok, const unsigned char* st,
-                                              int warp, int lane, uint32_t bar_empty, float (&tot)[2][NT][4]) {
+__device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int rb, int k0, int ntok,
+                                              const unsigned char* st, int warp, int lane, uint32_t bar_empty,
+                                              float (&tot)[2][NT][4]) {
   constexpr int KSPAN = 1024 / BITS;  // inputs per stage (128 bytes of a row)
   constexpr int SEGS = KSPAN / 128;   // scale segments per stage
   const LayerDims& L = a.L;
-  const int K = a.phase == 0 ? L.d_model : L.d_ff;
-  const bool swiglu_in = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const int K = phase == 0 ? L.d_model : L.d_ff;
+  const bool swiglu_in = phase == 0 && L.act == EMOE_ACT_SWIGLU;
   const int g = lane >> 2, t = lane & 3;
   const int gp = box_row_of<BITS>(g);
   const unsigned char* xt = st + 2 * TMA_BOX_BYTES;
   const unsigned char* sct = st + scale_tile_offset(NT);
-  const int N = a.phase == 0 ? L.d_ff : L.d_model;
+  const int N = phase == 0 ? L.d_ff : L.d_model;
   const int G = L.group > 0 ? L.group : K;
   const int ngroups = K / G;
   const int ssz = L.scale_f16 ? 2 : 4;
@@ -231,8 +255,8 @@ template <int BITS, int NT>
 __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m, int warp, int lane,
                                            const float (&tot)[2][NT][4]) {
   const LayerDims& L = a.L;
-  const int N = a.phase == 0 ? L.d_ff : L.d_model;
-  const bool swiglu_in = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const int N = m.phase == 0 ? L.d_ff : L.d_model;
+  const bool swiglu_in = m.phase == 0 && L.act == EMOE_ACT_SWIGLU;
   const int g = lane >> 2, t = lane & 3;
   const int gp = box_row_of<BITS>(g);
 #pragma unroll
@@ -253,7 +277,7 @@ __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m,
         for (int mt = 0; mt < 2; ++mt) {
           const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
           if (n >= N) continue;
-          if (a.phase == 0)
+          if (m.phase == 0)
             a.hidden[slot * N + act_pos<BITS>(n)] = __float2bfloat16_rn(fmaxf(tot[mt][nt][i], 0.0f));
           else
             a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + slot) * N + n] = tot[mt][nt][i];
@@ -277,9 +301,9 @@ __host__ __device__ constexpr int smem_bytes_for() {
 
 template <int NT>
 #ifdef EMOE_TMA_MAXNREG
-__global__ void __maxnreg__(EMOE_TMA_MAXNREG) ffn_tma_kernel(const TmaArgs a) {
+__global__ void __maxnreg__(EMOE_TMA_MAXNREG) ffn_tma_kernel(const __grid_constant__ TmaArgs a) {
 #else
-__global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_kernel(const TmaArgs a) {
+__global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_kernel(const __grid_constant__ TmaArgs a) {
 #endif
   constexpr int STAGES = stages_for<NT>();
   constexpr int STAGE_BYTES = stage_bytes_for(NT);
@@ -303,56 +327,57 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
   // harmless: a column of the MMA result depends only on its own column of B, and columns past
   // the expert's token count are never stored.
   __syncthreads();
-  // Everything above overlaps the tail of the kernel in front.  The first projection needs that
-  // kernel's results (the plan) at once; the second projection's plan, weights and scales are
-  // older than the kernel in front, so its producer starts fetching them and waits only before
-  // the first copy of a hidden vector (see `waited` below).
-  if (a.phase == 0) pdl_wait();
+  // Everything above overlaps the tail of the kernel in front.  A launch that starts with the
+  // first projection needs that kernel's results (the plan) at once; a launch of the second
+  // projection alone finds plan, weights and scales older than the kernel in front, so its
+  // producer starts fetching them and waits only before the first copy of a hidden vector (see
+  // `waited` below).
+  if (a.phase_begin == 0) pdl_wait();
   pdl_trigger();
 
   const uint32_t bar_full = smem_u32(bars), bar_empty = smem_u32(bars + STAGES);
   const LayerDims& L = a.L;
-  const int K = a.phase == 0 ? L.d_model : L.d_ff;
-  const bool swiglu_in = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
-  const int mat_first = a.phase == 0 ? 0 : (L.act == EMOE_ACT_SWIGLU ? 2 : 1);
-  const int rows_per_item = swiglu_in ? TMA_BOX_ROWS : 2 * TMA_BOX_ROWS;
+  PlanRec* recs = reinterpret_cast<PlanRec*>(reinterpret_cast<char*>(a.plan) + PLAN_HEADER_BYTES);
+  // both projections in this launch: an item of the second projection waits until the expert's
+  // hidden vectors are complete (PlanRec::done, raised by the consumers of the first projection)
+  const bool fused = a.phase_begin == 0 && a.phase_end == 2;
 
   if (warp == TMA_CONSUMER_WARPS) {
     // ---------------- producer warp ----------------
+    // the record the CTA's first item most likely needs, requested together with the header
+    const int ai_guess = min(static_cast<int>(blockIdx.x) / (a.phase_begin == 0 ? a.row_blocks[0] : a.row_blocks[1] * a.ksplit),
+                             L.E - 1);
+    const PlanRec rec_guess = recs[ai_guess];
     const int n_active = *reinterpret_cast<volatile const int*>(a.plan);
-    const int n_items = n_active * a.row_blocks * a.ksplit;
-    const PlanRec* recs = reinterpret_cast<const PlanRec*>(reinterpret_cast<const char*>(a.plan) + PLAN_HEADER_BYTES);
-    const int Nrows = a.phase == 0 ? L.d_ff : L.d_model;
-    const int Gk = L.group > 0 ? L.group : K;
-    const int ngroups_k = K / Gk;
+    // items: the first projection's (expert, row block), then the second's (expert, row block,
+    // split-K slice), each list expert-major in plan order
+    const int n_items0 = a.phase_begin == 0 ? n_active * a.row_blocks[0] : 0;
+    const int n_items1 = a.phase_end == 2 ? n_active * a.row_blocks[1] * a.ksplit : 0;
+    const int n_items = n_items0 + n_items1;
     const int ssz = L.scale_f16 ? 2 : 4;
-    const int per_expert = a.ksplit * a.row_blocks;
     int it = 0;
     bool ok = true;
-    bool waited = a.phase == 0;  // false: copies of activation rows are parked until pdl_wait()
+    bool waited = a.phase_begin == 0;  // false: copies of activation rows are parked until pdl_wait()
     int n_parked = 0;
     int park_stage[STAGES], park_row[STAGES], park_k0[STAGES], park_klen[STAGES], park_ntok[STAGES];
-    // Item look-ahead of two: the counter increment for item i+2 and the expert record of item
-    // i+1 are issued before item i is streamed and only read after it, so that switching items
-    // costs no round trip to memory.  A CTA's first item is its own index; the counter hands
-    // out the items after those.
+    // A CTA's first item is its own index; the counter hands out the items after those.
     int item_cur = blockIdx.x, item_next = 0;
-#if EMOE_TMA_LOOKAHEAD
-    if (lane == 0) item_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
-#endif
-    PlanRec rec_cur = recs[min(item_cur / per_expert, L.E - 1)];  // read before n_items is known: same latency
-    item_next = __shfl_sync(0xffffffffu, item_next, 0);
     while (ok) {
       const int item = item_cur;
       if (item >= n_items || *abort_flag) break;
-      const PlanRec rec = rec_cur;
-#if EMOE_TMA_LOOKAHEAD
-      int raw_after_next = 0;
-      if (lane == 0) raw_after_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
-      const PlanRec rec_next = recs[item_next < n_items ? item_next / per_expert : 0];
-#endif
-      const int z = item % a.ksplit;
-      const int rb = (item / a.ksplit) % a.row_blocks;
+      const int phase = item < n_items0 ? 0 : 1;
+      const int li = item - (phase == 0 ? 0 : n_items0);
+      const PhaseDims pd = phase_dims(a, phase);
+      const int K = pd.K;
+      const bool swiglu_in = pd.swiglu_in;
+      const int mat_first = pd.mat_first;
+      const int Gk = L.group > 0 ? L.group : K;
+      const int ngroups_k = K / Gk;
+      const int ai = li / (pd.ksplit * pd.row_blocks);
+      const PlanRec rec = (it == 0 && ai == ai_guess) ? rec_guess : recs[ai];
+      const __nv_bfloat16* in = phase == 0 ? a.xs : a.hidden;
+      const int z = li % pd.ksplit;
+      const int rb = (li / pd.ksplit) % pd.row_blocks;
       const int e = rec.e;
       const int begin = rec.begin;
       const int cnt = rec.cnt;
@@ -360,11 +385,12 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
       const int bits = rec.bits;
       const int kspan = 1024 / bits;
       const int steps_total = (K + kspan - 1) / kspan;
-      const int spz = (steps_total + a.ksplit - 1) / a.ksplit;
+      const int spz = (steps_total + pd.ksplit - 1) / pd.ksplit;
       const int step_begin = z * spz;
       const int nsteps = max(0, min(steps_total, step_begin + spz) - step_begin);
       const int npass = (cnt + NT * 8 - 1) / (NT * 8);
-      const int row0 = rb * rows_per_item;
+      const int row0 = rb * pd.rows_per_item;
+      bool need_dep = fused && phase == 1;
       for (int pass = 0; pass < npass && ok; ++pass) {
         const int p0 = pass * NT * 8;
         const int ntok = min(NT * 8, cnt - p0);
@@ -383,7 +409,10 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           if (lane == 0) {
             StageMeta& m = meta[stage];
             m.e = e; m.rb = rb; m.z = z; m.begin = begin; m.p0 = p0; m.ntok = ntok; m.k0 = k0; m.bits = bits;
-            m.flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0);
+            m.phase = phase;
+            m.ai = ai;
+            m.flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0) |
+                      (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0);
             m.scales[0] = swiglu_in ? rec.scales[0] : rec.scales[mat_first];
             m.scales[1] = swiglu_in ? rec.scales[1] : rec.scales[mat_first];
             if (klen > 0) {
@@ -402,18 +431,6 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           }
           __syncwarp();
           if (klen > 0) {
-            if (waited) {
-              for (int r = lane; r < ntok; r += 32)
-                bulk_load(smem_u32(st + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
-                          a.in + static_cast<size_t>(begin + p0 + r) * K + k0, klen * 2, full);
-            } else {
-              park_stage[n_parked] = stage;
-              park_row[n_parked] = begin + p0;
-              park_k0[n_parked] = k0;
-              park_klen[n_parked] = klen;
-              park_ntok[n_parked] = ntok;
-              ++n_parked;
-            }
             // scales: lane l copies the windows of rows 4l .. 4l+3 of the stage (box-major)
             const int nseg = klen / 128;
             const int g0 = group_of(k0, Gk, ngroups_k), g1 = group_of(k0 + (nseg - 1) * 128, Gk, ngroups_k);
@@ -421,7 +438,7 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
               const int row = 4 * lane + r;
-              const int n = min(swiglu_in ? row0 + (row & 63) : row0 + row, Nrows - 1);
+              const int n = min(swiglu_in ? row0 + (row & 63) : row0 + row, pd.N - 1);
               const char* sp = static_cast<const char*>(swiglu_in ? rec.scales[row >> 6] : rec.scales[mat_first]);
               const int b0 = scale_window_begin(n, ngroups_k, g0, ssz);
               const int b1 = (n * ngroups_k + g1 + 1) * ssz;
@@ -430,6 +447,43 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
                              : "memory");
             }
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full) : "memory");
+            if (need_dep) {
+              // The codes and scales of the stage are on their way; the hidden vectors may still be
+              // in the making on other SMs.  Every lane acquires the counter itself, so that its
+              // own copies below are ordered behind the writers' stores.
+              need_dep = false;
+              const int expect = a.row_blocks[0] * TMA_CONSUMER_WARPS;
+              const int* done = &recs[ai].done;
+              bool ready = false;
+              for (unsigned i = 0; i < DEP_WAIT_LIMIT; ++i) {
+                int v;
+                asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(done) : "memory");
+                ready = __all_sync(0xffffffffu, v >= expect);
+                if (ready || *abort_flag) break;
+                __nanosleep(100);
+              }
+              if (!ready) {
+                if (lane == 0) {
+                  *abort_flag = 1;
+                  atomicOr(a.check_word, CHECK_WAIT_TIMEOUT);
+                }
+                ok = false;
+                break;
+              }
+              asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores -> bulk-copy reads
+            }
+            if (waited) {
+              for (int r = lane; r < ntok; r += 32)
+                bulk_load(smem_u32(st + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
+                          in + static_cast<size_t>(begin + p0 + r) * K + k0, klen * 2, full);
+            } else {
+              park_stage[n_parked] = stage;
+              park_row[n_parked] = begin + p0;
+              park_k0[n_parked] = k0;
+              park_klen[n_parked] = klen;
+              park_ntok[n_parked] = ntok;
+              ++n_parked;
+            }
           } else {
             mbar_arrive(full);  // with lane 0's arrival above: 33 in all
           }
@@ -439,35 +493,30 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
             for (int i = 0; i < n_parked; ++i)
               for (int r = lane; r < park_ntok[i]; r += 32)
                 bulk_load(smem_u32(smem + park_stage[i] * STAGE_BYTES + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
-                          a.in + static_cast<size_t>(park_row[i] + r) * K + park_k0[i], park_klen[i] * 2,
+                          a.hidden + static_cast<size_t>(park_row[i] + r) * K + park_k0[i], park_klen[i] * 2,
                           bar_full + 8 * park_stage[i]);
             n_parked = 0;
           }
         }
       }
-#if EMOE_TMA_LOOKAHEAD
-      item_cur = item_next;
-      rec_cur = rec_next;
-      item_next = __shfl_sync(0xffffffffu, raw_after_next, 0);
-#else
       // the ring still holds several stages of work for the consumers: fetching the next item
       // only now costs them nothing and no CTA sits on items it is not yet working on
-      if (lane == 0) item_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase, 1);
+      if (lane == 0) item_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase_begin, 1);
       item_cur = __shfl_sync(0xffffffffu, item_next, 0);
-      rec_cur = recs[item_cur < n_items ? item_cur / per_expert : 0];
-#endif
       if (item_cur < n_items) {
         // pull the next item's scale rows towards L2 while its codes are still far away
-        const int rbn = (item_cur / a.ksplit) % a.row_blocks;
-        const int Nn = a.phase == 0 ? L.d_ff : L.d_model;
-        const int ngroups = L.group > 0 ? K / L.group : 1;
-        const int ssz = L.scale_f16 ? 2 : 4;
-        const int rows = min(rows_per_item, Nn - rbn * rows_per_item);
+        const int phn = item_cur < n_items0 ? 0 : 1;
+        const int lin = item_cur - (phn == 0 ? 0 : n_items0);
+        const PhaseDims pn = phase_dims(a, phn);
+        const PlanRec rn = recs[lin / (pn.ksplit * pn.row_blocks)];
+        const int rbn = (lin / pn.ksplit) % pn.row_blocks;
+        const int ngroups = L.group > 0 ? pn.K / L.group : 1;
+        const int rows = min(pn.rows_per_item, pn.N - rbn * pn.rows_per_item);
         const int lines = (rows * ngroups * ssz + 127) / 128;
-        const size_t offs = static_cast<size_t>(rbn) * rows_per_item * ngroups * ssz;
-        const int nm = swiglu_in ? 2 : 1;
+        const size_t offs = static_cast<size_t>(rbn) * pn.rows_per_item * ngroups * ssz;
+        const int nm = pn.swiglu_in ? 2 : 1;
         for (int i = lane; i < nm * lines; i += 32) {
-          const char* base = static_cast<const char*>(rec_cur.scales[swiglu_in ? i / lines : mat_first]) + offs;
+          const char* base = static_cast<const char*>(rn.scales[pn.swiglu_in ? i / lines : pn.mat_first]) + offs;
           asm volatile("prefetch.global.L2 [%0];" ::"l"(base + static_cast<size_t>(i % lines) * 128));
         }
       }
@@ -478,7 +527,7 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
       for (int i = 0; i < n_parked; ++i)
         for (int r = lane; r < park_ntok[i]; r += 32)
           bulk_load(smem_u32(smem + park_stage[i] * STAGE_BYTES + 2 * TMA_BOX_BYTES + r * TMA_XROW_MAX),
-                    a.in + static_cast<size_t>(park_row[i] + r) * K + park_k0[i], park_klen[i] * 2,
+                    a.hidden + static_cast<size_t>(park_row[i] + r) * L.d_ff + park_k0[i], park_klen[i] * 2,
                     bar_full + 8 * park_stage[i]);
       n_parked = 0;
     }
@@ -514,9 +563,9 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
       const unsigned char* st = smem + stage * STAGE_BYTES;
       if (!(m.flags & META_EMPTY)) {
         switch (m.bits) {
-          case 2: consume_stage<2, NT>(a, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
-          case 4: consume_stage<4, NT>(a, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
-          default: consume_stage<8, NT>(a, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          case 2: consume_stage<2, NT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          case 4: consume_stage<4, NT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          default: consume_stage<8, NT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
         }
       } else {
         __syncwarp();
@@ -527,6 +576,16 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           case 2: store_item<2, NT>(a, m, warp, lane, tot); break;
           case 4: store_item<4, NT>(a, m, warp, lane, tot); break;
           default: store_item<8, NT>(a, m, warp, lane, tot); break;
+        }
+        if (m.flags & META_DONE) {
+          // this warp's share of the expert's hidden vectors is written: make it visible to the
+          // bulk copies of other SMs, then count it
+          asm volatile("fence.proxy.async;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            __threadfence();
+            atomicAdd(&recs[m.ai].done, 1);
+          }
         }
       }
     }
@@ -581,27 +640,33 @@ int ffn_tma_ksplit(const LayerDims& L, int T) {
   return static_cast<int>(z);
 }
 
-cudaError_t launch_ffn_tma(int phase, const LayerDims& L, const ExpertDev* experts, const void* tmaps,
-                           const __nv_bfloat16* in, const int32_t* off, int* plan, __nv_bfloat16* hidden, float* o_part,
-                           int ksplit, int n_pairs, int T, int* check_word, cudaStream_t st) {
-  const int N = phase == 0 ? L.d_ff : L.d_model;
-  const int rows_per_item = (phase == 0 && L.act == EMOE_ACT_SWIGLU) ? TMA_BOX_ROWS : 2 * TMA_BOX_ROWS;
+cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, const ExpertDev* experts,
+                           const void* tmaps, const __nv_bfloat16* xs, const int32_t* off, int* plan,
+                           __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs, int T, int* check_word,
+                           cudaStream_t st) {
+  if (phase_begin < 0 || phase_end > 2 || phase_begin >= phase_end) return cudaErrorInvalidValue;
+  const int rows_first = L.act == EMOE_ACT_SWIGLU ? TMA_BOX_ROWS : 2 * TMA_BOX_ROWS;
   TmaArgs a;
-  a.phase = phase;
+  a.phase_begin = phase_begin;
+  a.phase_end = phase_end;
   a.L = L;
   a.experts = experts;
   a.tmaps = static_cast<const CUtensorMap*>(tmaps);
-  a.in = in;
+  a.xs = xs;
   a.off = off;
   a.plan = plan;
   a.hidden = hidden;
   a.o_part = o_part;
-  a.ksplit = phase == 0 ? 1 : ksplit;
-  a.row_blocks = (N + rows_per_item - 1) / rows_per_item;
+  a.ksplit = ksplit;
+  a.row_blocks[0] = (L.d_ff + rows_first - 1) / rows_first;
+  a.row_blocks[1] = (L.d_model + 2 * TMA_BOX_ROWS - 1) / (2 * TMA_BOX_ROWS);
   a.n_pairs = n_pairs;
   a.check_word = check_word;
   const long long active_max = n_pairs < L.E ? n_pairs : L.E;
-  const long long items = active_max * a.row_blocks * a.ksplit;
+  long long per_expert = 0;
+  if (phase_begin == 0) per_expert += a.row_blocks[0];
+  if (phase_end == 2) per_expert += static_cast<long long>(a.row_blocks[1]) * ksplit;
+  const long long items = active_max * per_expert;
   const int max_items = items > (1 << 30) ? (1 << 30) : static_cast<int>(items);
   const int nt = ffn_token_tiles(L, T);
   if (nt == 1) return launch_nt<1>(a, max_items, st);

@@ -15,13 +15,14 @@ from tests.helpers import check_ids, oracle_pack_layer, output_tolerance, rel_to
 pytestmark = pytest.mark.gpu
 
 
-def _run_case(shape, bits, T, seed, path, bias=None, std=0.02, max_tokens=None):
+def _run_case(shape, bits, T, seed, path, bias=None, std=0.02, max_tokens=None, fused=True, want_y=False):
     W = inputs.expert_set(seed, 0, shape, std)
     x = inputs.activations(seed, 0, T, shape.d_model, shape.act_dtype)
     Wr = inputs.router_weight(seed, 0, shape.d_model, shape.n_experts, std=0.05)
     packed, scales = oracle_pack_layer(W, shape, bits)
     with layer.MoELayer(shape, bits, max_tokens=max_tokens or T) as moe:
         B.emoe_set_ffn_path(moe.ctx, path)
+        B.emoe_set_fused_projections(moe.ctx, fused)
         moe.pack_from_host(W)
         for e in range(shape.n_experts):          # packed bytes and scales are bit-exact
             for m in range(shape.n_matrices):
@@ -39,7 +40,7 @@ def _run_case(shape, bits, T, seed, path, bias=None, std=0.02, max_tokens=None):
                                    scales, ids, gates)
     err = rel_to_max(y, y_ref)
     assert err <= output_tolerance(shape.act_dtype), err
-    return err
+    return (err, y) if want_y else err
 
 
 GEMV_CASES = [
@@ -91,8 +92,12 @@ TMA_CASES = [
 
 @pytest.mark.parametrize("act,group,sdt,d,f,E,k,gate,bits,T", TMA_CASES)
 def test_forward_tma_pipeline_path(act, group, sdt, d, f, E, k, gate, bits, T):
+    """Both projections in one launch (the default) and as two launches: each within the bar, and
+    bit-identical to each other (same arithmetic in the same order, only the scheduling differs)."""
     shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, "bf16")
-    _run_case(shape, bits, T, seed=25, path=3)
+    _, y_fused = _run_case(shape, bits, T, seed=25, path=3, want_y=True)
+    _, y_split = _run_case(shape, bits, T, seed=25, path=3, fused=False, want_y=True)
+    assert np.array_equal(y_fused, y_split)
 
 
 UMMA_CASES = [
