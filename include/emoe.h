@@ -71,7 +71,8 @@ typedef struct emoe_ctx emoe_ctx;
 
 /* One expert of a layer: its bitwidth and DEVICE pointers to its packed matrices and
  * scale channels (Section 3.2: experts of one layer may differ in bitwidth).
- * ReLU uses entries 0..1, SwiGLU 0..2 (order as listed above). */
+ * ReLU uses entries 0..1, SwiGLU 0..2 (order as listed above).  Packed matrices must be
+ * 16-byte aligned, scale channels 4-byte aligned (whatever their type). */
 typedef struct emoe_expert {
   int32_t bits; /* 2, 4 or 8 */
   int32_t reserved;

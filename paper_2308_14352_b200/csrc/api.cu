@@ -180,7 +180,7 @@ int check_experts(const LayerDims& L, const emoe_expert* host) {
     for (int m = 0; m < nmat; ++m) {
       if (!host[e].packed[m] || !host[e].scales[m]) return EMOE_ERR_INVALID_ARG;
       if (!aligned(host[e].packed[m], 16)) return EMOE_ERR_ALIGNMENT;
-      if (!aligned(host[e].scales[m], L.scale_f16 ? 2 : 4)) return EMOE_ERR_ALIGNMENT;
+      if (!aligned(host[e].scales[m], 4)) return EMOE_ERR_ALIGNMENT;
     }
   }
   return EMOE_OK;
@@ -266,7 +266,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     EMOE_CUDA(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
   } else if (use_tma) {
     ksplit = ffn_tma_ksplit(L, T);
-    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, st));
+    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
     if (ctx->fuse_projections) {
@@ -280,7 +280,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     }
   } else if (use_mma) {
     ksplit = ffn_mma_ksplit(L, T);
-    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, st));
+    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, false, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_CUDA(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));

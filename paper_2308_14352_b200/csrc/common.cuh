@@ -98,9 +98,10 @@ bool ffn_mma_supported(const LayerDims& L);
 int ffn_mma_ksplit(const LayerDims& L, int T);
 int ffn_token_tiles(const LayerDims& L, int T);
 // plan (nullable): plan_bytes(E) bytes, the work plan for the persistent TMA kernels, filled by block 0.
+// to_f16: store the rows as fp16 (saturating) instead of bf16, same layout (the TMA-staged kernel's input).
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
-                             cudaStream_t st);
+                             bool to_f16, cudaStream_t st);
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
                            const int32_t* off, __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs,
                            int T, cudaStream_t st);

@@ -207,7 +207,8 @@ __global__ void __launch_bounds__(MMA_THREADS)
 __global__ void __launch_bounds__(128)
     scatter_x_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
                      const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
-                     int E, int* __restrict__ plan, int top_k, int d, int n_pairs, __nv_bfloat16* __restrict__ xs) {
+                     int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int to_f16,
+                     __nv_bfloat16* __restrict__ xs) {
   pdl_wait();
   pdl_trigger();
   if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
@@ -251,7 +252,11 @@ __global__ void __launch_bounds__(128)
   for (int u = threadIdx.x; u < d / 16; u += blockDim.x) {
     const int seg = (u >> 3) * 128, t = (u >> 1) & 3, b = u & 1;
     const uint4* src = reinterpret_cast<const uint4*>(src_row + seg + t * 32 + b * 16);
-    const uint4 a = src[0], c = src[1];
+    uint4 a = src[0], c = src[1];
+    if (to_f16) {  // the streaming kernel multiplies in fp16: same layout, 16-bit values converted in place
+      a = make_uint4(bf16x2_to_f16x2_sat(a.x), bf16x2_to_f16x2_sat(a.y), bf16x2_to_f16x2_sat(a.z), bf16x2_to_f16x2_sat(a.w));
+      c = make_uint4(bf16x2_to_f16x2_sat(c.x), bf16x2_to_f16x2_sat(c.y), bf16x2_to_f16x2_sat(c.z), bf16x2_to_f16x2_sat(c.w));
+    }
     uint4 oa, oc;
     if (bits == 8) {
       oa = a;
@@ -304,9 +309,9 @@ int ffn_mma_ksplit(const LayerDims& L, int T) {
 
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
-                             cudaStream_t st) {
+                             bool to_f16, cudaStream_t st) {
   return launch_chain(scatter_x_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
-                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, xs);
+                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, to_f16 ? 1 : 0, xs);
 }
 
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,

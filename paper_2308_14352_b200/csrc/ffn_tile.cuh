@@ -165,6 +165,120 @@ __device__ __forceinline__ void unpack_step(const Raw<2>& raw, int q, uint32_t (
   }
 }
 
+// ---- offset codes: the unpack of the streaming kernel -------------------------------------------
+// fp16 has a 10-bit mantissa, so a code field that sits at bit p of a 16-bit half can be read in
+// place as mantissa bits of the fp16 number 2^(10-p) (whose mantissa bit p weighs 1): masking the
+// field, flipping its sign bit (two's complement -> offset binary) and setting the exponent is
+// ONE logic instruction, and the result is the exact fp16 integer c + q with the constant
+// c = 2^(10-p) + 2^(b-1).  The constant is not subtracted per code:
+//   sum_k (c + q_k) x_k  =  sum_k q_k x_k  +  c * sum_k x_k,
+// and the second sum does not depend on the output channel, so one extra MMA per step, with the
+// constants as its A operand, yields it for all channels of the warp at once.  Products of two
+// fp16 numbers are exact in fp32; what the subtraction costs is cancellation inside the tensor
+// core's accumulation, which grows with c / rms(q).  The fields are therefore moved (one shift
+// per word of fields) to the highest position that holds them, where c is smallest:
+//   8 bits: no constant is carried: byte ^ 0x80 under the exponent byte 0x64 is 1152 + q, and one
+//           fp16x2 subtraction makes it q (the only position that holds 8 bits is p = 0, where
+//           c = 1152 costs more accuracy than the subtraction costs time), pairs (2c, 2c+1);
+//   4 bits: pairs (c, c+4) of an 8-code word, every field at p = 4: 72 + q;
+//   2 bits: pairs (c, c+8) of a 16-code word, odd c at p = 8 (6 + q), even c at p = 6 (18 + q),
+//           two neighbouring pairs per shifted word.
+__device__ __forceinline__ void mma_f16(float (&d)[4], const uint32_t a0, const uint32_t a1, const uint32_t a2,
+                                        const uint32_t a3, const uint32_t b0, const uint32_t b1) {
+  asm(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t f16x2_sub(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// fp16x2 constant c of register j (0..3) of a step, per bitwidth (both halves equal)
+template <int BITS>
+__device__ __forceinline__ constexpr uint32_t offset_const(int j) {
+  if (BITS == 8) return 0u;                      // exact codes, nothing to take out
+  if (BITS == 4) return 0x54805480u;             // 72
+  return (j & 1) ? 0x46004600u : 0x4C804C80u;    // odd pair: 6, even pair: 18
+}
+
+// the four registers (code pairs 4q .. 4q+3 of the lane's row) of step q as offset codes
+__device__ __forceinline__ void unpack_step_off(const Raw<8>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[8] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w, raw.v[1].x, raw.v[1].y, raw.v[1].z, raw.v[1].w};
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const uint32_t u = w[2 * q + j] ^ 0x80808080u;
+    o[2 * j] = f16x2_sub(prmt(u, 0x64646464u, 0x4140u), 0x64806480u);
+    o[2 * j + 1] = f16x2_sub(prmt(u, 0x64646464u, 0x4342u), 0x64806480u);
+  }
+}
+__device__ __forceinline__ void unpack_step_off(const Raw<4>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[4] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w};
+  const uint32_t v = w[q];  // nibble c of each half goes to bits 4..7
+  o[0] = and_xor(v << 4, 0x00F000F0u, 0x54805480u);
+  o[1] = and_xor(v, 0x00F000F0u, 0x54805480u);
+  o[2] = and_xor(v >> 4, 0x00F000F0u, 0x54805480u);
+  o[3] = and_xor(v >> 8, 0x00F000F0u, 0x54805480u);
+}
+__device__ __forceinline__ void unpack_step_off(const Raw<2>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[2] = {raw.v[0].x, raw.v[0].y};
+  const uint32_t v = w[q >> 1];
+  // pairs c = 4(q&1) + j; field c of each half to bits 8..9 (odd c) or 6..7 (even c): the
+  // shift that puts an odd c at bit 8 puts c - 1 at bit 6
+  uint32_t s01, s23;  // fields (c0, c0+1) and (c0+2, c0+3) in place
+  if ((q & 1) == 0) {
+    s01 = v << 6;
+    s23 = v << 2;
+  } else {
+    s01 = v >> 2;
+    s23 = v >> 6;
+  }
+  o[0] = and_xor(s01, 0x00C000C0u, 0x4C804C80u);
+  o[1] = and_xor(s01, 0x03000300u, 0x46004600u);
+  o[2] = and_xor(s23, 0x00C000C0u, 0x4C804C80u);
+  o[3] = and_xor(s23, 0x03000300u, 0x46004600u);
+}
+
+// The same registers as exact fp16 integers q (the constant subtracted per pair): one more
+// instruction per pair and no extra MMAs, the better trade when a pass multiplies every code
+// with several token tiles.  Fields are read where they sit (p = 0 / 4 at 4 bits, p = 0..8 at 2
+// bits: the subtraction is exact whatever the constant).
+__device__ __forceinline__ void unpack_step_exact(const Raw<8>& raw, int q, uint32_t (&o)[4]) { unpack_step_off(raw, q, o); }
+__device__ __forceinline__ void unpack_step_exact(const Raw<4>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[4] = {raw.v[0].x, raw.v[0].y, raw.v[0].z, raw.v[0].w};
+  const uint32_t lo = w[q], hi = lo >> 8;
+  o[0] = f16x2_sub(and_xor(lo, 0x000F000Fu, 0x64086408u), 0x64086408u);  // 1032 + q
+  o[1] = f16x2_sub(and_xor(lo, 0x00F000F0u, 0x54805480u), 0x54805480u);  // 72 + q
+  o[2] = f16x2_sub(and_xor(hi, 0x000F000Fu, 0x64086408u), 0x64086408u);
+  o[3] = f16x2_sub(and_xor(hi, 0x00F000F0u, 0x54805480u), 0x54805480u);
+}
+__device__ __forceinline__ void unpack_step_exact(const Raw<2>& raw, int q, uint32_t (&o)[4]) {
+  const uint32_t w[2] = {raw.v[0].x, raw.v[0].y};
+  const uint32_t lo = w[q >> 1], hi = lo >> 10;
+  // 2^(10-p) + 2 as fp16 for p = 0, 2, 4, 6, 8: 1026, 258, 66, 18, 6
+  const uint32_t mag[5] = {0x64026402u, 0x5C085C08u, 0x54205420u, 0x4C804C80u, 0x46004600u};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = 4 * (q & 1) + j;  // pair (c, c+8) of the 16-code word
+    const int pi = c < 5 ? c : c - 5;
+    o[j] = f16x2_sub(and_xor(c < 5 ? lo : hi, 0x00030003u << (2 * pi), mag[pi]), mag[pi]);
+  }
+}
+
+// two bf16 values -> two fp16 values (exact inside the fp16 range, saturating outside)
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2_sat(uint32_t v) {
+  const float lo = fminf(fmaxf(__uint_as_float(v << 16), -65504.0f), 65504.0f);
+  const float hi = fminf(fmaxf(__uint_as_float(v & 0xffff0000u), -65504.0f), 65504.0f);
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ __half f32_to_f16_sat(float v) {
+  return __float2half_rn(fminf(fmaxf(v, -65504.0f), 65504.0f));
+}
+
 // position of input k (natural order) in the activation layout described at the top
 template <int BITS>
 __device__ __forceinline__ int act_pos(int k) {

@@ -3,10 +3,13 @@
 // independent FFN) on the Section 3.2 storage (b-bit codes + scale channel, w~ = q * s formed
 // in registers).
 //
-// Same arithmetic as ffn_mma.cu (codes as exact bf16 integers in the A operand of
+// Same shape of arithmetic as ffn_mma.cu (codes as exact small integers in the A operand of
 // mma.m16n8k16, tokens as the N dimension, fp32 accumulation per 128-input segment, then
-// total += scale * segment); what differs is how the bytes travel.  The kernel is bound by
-// streaming packed weights from HBM, so the bytes in flight must not depend on registers:
+// total += scale * segment), with two differences.  The operands are fp16: the codes are read
+// as offset codes c + q with one logic instruction per pair and the constant is taken out
+// again per segment (ffn_tile.cuh), and the activations (bf16 values) travel as fp16, exact
+// inside the fp16 range and saturated outside.  And the bytes travel differently: the kernel is
+// bound by streaming packed weights from HBM, so the bytes in flight must not depend on registers:
 //   * the kernel is persistent: a CTA pulls work items (activated expert, block of output
 //     rows, split-K slice) from a device-side counter, most expensive bitwidth first, and its
 //     producer warp runs ahead across item boundaries, so the weight stream never drains
@@ -41,7 +44,7 @@ constexpr int TMA_BOX_ROWS = 64;
 constexpr int TMA_BOX_BYTES = TMA_BOX_ROWS * 128;  // 8 KB
 constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a stage (row stride = 64 mod 128)
 #ifndef EMOE_TMA_STAGES_NT1
-#define EMOE_TMA_STAGES_NT1 3
+#define EMOE_TMA_STAGES_NT1 2
 #endif
 #ifndef EMOE_TMA_UNROLL_SEGS
 #define EMOE_TMA_UNROLL_SEGS 0
@@ -53,7 +56,7 @@ constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a s
 #define EMOE_TMA_LOOKAHEAD 0
 #endif
 #ifndef EMOE_TMA_CTAS_NT1
-#define EMOE_TMA_CTAS_NT1 2
+#define EMOE_TMA_CTAS_NT1 3
 #endif
 
 // MMA row g of a 16-row tile -> row of the shared-memory box, chosen per bitwidth so that the
@@ -65,28 +68,28 @@ __device__ __forceinline__ int box_row_of(int g) {
   return ((g & 3) << 1) | (g >> 2);
 }
 
-// the lane's raw codes of one row for segment `sg` of the stage, from a swizzled box
+// the lane's raw codes of one row for segment `sg` of the stage: `row` points at the row's 128
+// bytes inside a swizzled box, `swz` is the row's swizzle term (row index mod 8)
 template <int BITS>
-__device__ __forceinline__ Raw<BITS> lds_raw(const unsigned char* box, int row, int sg, int t);
+__device__ __forceinline__ Raw<BITS> lds_raw(const unsigned char* row, int swz, int sg, int t);
 template <>
-__device__ __forceinline__ Raw<8> lds_raw<8>(const unsigned char* box, int row, int sg, int t) {
+__device__ __forceinline__ Raw<8> lds_raw<8>(const unsigned char* row, int swz, int sg, int t) {
   (void)sg;
   Raw<8> r;
-  const unsigned char* base = box + row * 128;
-  r.v[0] = *reinterpret_cast<const uint4*>(base + (((2 * t) ^ (row & 7)) << 4));
-  r.v[1] = *reinterpret_cast<const uint4*>(base + (((2 * t + 1) ^ (row & 7)) << 4));
+  r.v[0] = *reinterpret_cast<const uint4*>(row + (((2 * t) ^ swz) << 4));
+  r.v[1] = *reinterpret_cast<const uint4*>(row + (((2 * t + 1) ^ swz) << 4));
   return r;
 }
 template <>
-__device__ __forceinline__ Raw<4> lds_raw<4>(const unsigned char* box, int row, int sg, int t) {
+__device__ __forceinline__ Raw<4> lds_raw<4>(const unsigned char* row, int swz, int sg, int t) {
   Raw<4> r;
-  r.v[0] = *reinterpret_cast<const uint4*>(box + row * 128 + (((4 * sg + t) ^ (row & 7)) << 4));
+  r.v[0] = *reinterpret_cast<const uint4*>(row + (((4 * sg + t) ^ swz) << 4));
   return r;
 }
 template <>
-__device__ __forceinline__ Raw<2> lds_raw<2>(const unsigned char* box, int row, int sg, int t) {
+__device__ __forceinline__ Raw<2> lds_raw<2>(const unsigned char* row, int swz, int sg, int t) {
   Raw<2> r;
-  r.v[0] = *reinterpret_cast<const uint2*>(box + row * 128 + (((2 * sg + (t >> 1)) ^ (row & 7)) << 4) + ((t & 1) << 3));
+  r.v[0] = *reinterpret_cast<const uint2*>(row + (((2 * sg + (t >> 1)) ^ swz) << 4) + ((t & 1) << 3));
   return r;
 }
 
@@ -98,13 +101,11 @@ __host__ __device__ constexpr int stage_bytes_for(int nt) {
 __host__ __device__ constexpr int scale_tile_offset(int nt) { return 2 * TMA_BOX_BYTES + nt * 8 * TMA_XROW_MAX; }
 
 // The scales a stage needs from row n (groups of inputs k0 .. k0 + 128*segs) sit in one short
-// byte window of the scale channel; it is copied from its 4-byte-aligned start.
-__device__ __forceinline__ int scale_window_begin(int n, int ngroups, int g0, int ssz) {
-  return ((n * ngroups + g0) * ssz) & ~3;
-}
-// group index of input k (groups of G inputs, G a multiple of 128 or the whole row)
-__device__ __forceinline__ int group_of(int k, int G, int ngroups) {
-  return ngroups == 1 ? 0 : (G == 128 ? (k >> 7) : k / G);
+// byte window of the scale channel; it is copied from the 4-byte boundary at or below its start.
+// group index of input k (groups of G inputs, G a multiple of 128 or the whole row);
+// gshift = log2(G) when G is a power of two, else -1
+__device__ __forceinline__ int group_of(int k, int gshift, int G, int ngroups) {
+  return ngroups == 1 ? 0 : (gshift >= 0 ? (k >> gshift) : k / G);
 }
 
 struct TmaArgs {
@@ -112,13 +113,15 @@ struct TmaArgs {
   LayerDims L;
   const ExpertDev* experts;
   const CUtensorMap* tmaps;  // [E][3]
-  const __nv_bfloat16* xs;   // input of the first projection (tokens in expert order)
+  const __half* xs;          // input of the first projection (tokens in expert order, fp16)
   const int32_t* off;
   int* plan;  // header {activated experts, item counters} + one PlanRec per activated expert
-  __nv_bfloat16* hidden;  // output of the first projection, input of the second
+  __half* hidden;         // output of the first projection, input of the second (bf16 values as fp16)
   float* o_part;
   int ksplit;         // split-K slices of the second projection
   int row_blocks[2];  // row blocks of an expert per projection
+  int ngroups[2];     // scale groups per row, per projection
+  int gshift;         // log2(group size) if it is a power of two, else -1
   int n_pairs;
   int* check_word;
 };
@@ -146,8 +149,7 @@ struct StageMeta {
   int flags;  // 1 = first stage of an item pass, 2 = last, 4 = no more work, 8 = stage carries no inputs,
               // 16 = last stage of a first-projection item whose completion the second projection waits for
   int phase;
-  const void* scales[2];  // scale channel of the matrix behind each m-tile
-  int ai;                 // index of the expert's plan record
+  int ai;  // index of the expert's plan record
   int pad;
 };
 constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8, META_DONE = 16;
@@ -161,20 +163,34 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int r
                                               float (&tot)[2][NT][4]) {
   constexpr int KSPAN = 1024 / BITS;  // inputs per stage (128 bytes of a row)
   constexpr int SEGS = KSPAN / 128;   // scale segments per stage
+  // one token tile: offset codes (fewest instructions per code); more: exact codes (no MMAs for
+  // the constants, which would have to be repeated per token tile)
+  constexpr bool OFFSET_CODES = NT == 1 && BITS != 8;
   const LayerDims& L = a.L;
   const int K = phase == 0 ? L.d_model : L.d_ff;
   const bool swiglu_in = phase == 0 && L.act == EMOE_ACT_SWIGLU;
   const int g = lane >> 2, t = lane & 3;
   const int gp = box_row_of<BITS>(g);
-  const unsigned char* xt = st + 2 * TMA_BOX_BYTES;
-  const unsigned char* sct = st + scale_tile_offset(NT);
   const int N = phase == 0 ? L.d_ff : L.d_model;
-  const int G = L.group > 0 ? L.group : K;
-  const int ngroups = K / G;
+  const int ngroups = a.ngroups[phase];
   const int ssz = L.scale_f16 ? 2 : 4;
-  const int nrow0 = swiglu_in ? rb * TMA_BOX_ROWS + 16 * warp : rb * 2 * TMA_BOX_ROWS + 32 * warp;
   const int nseg = min(SEGS, (K - k0) / 128);
-  const int g0 = group_of(k0, G, ngroups);
+  const int g0 = group_of(k0, a.gshift, L.group, ngroups);
+  // Everything that does not depend on the segment, once per stage.  The lane's four rows (2
+  // tiles x rows gp, gp+8) sit at fixed distances from the first one, in the boxes (128 bytes
+  // per row) and in the scale tile (16 bytes per row): tile 1 is the other box (gated
+  // projection) or 16 rows further down, rows gp+8 are 8 rows further down.  A row's scale
+  // window starts at the 4-byte boundary at or below its first scale of the stage; the rows of a
+  // lane are an even number of rows apart, so the distance to that boundary is the same for all.
+  const int swz = gp & 7;  // swizzle term of all four rows (they differ by multiples of 8)
+  const int box_first = swiglu_in ? 0 : (warp >> 1);
+  const int r_first = (swiglu_in ? 16 * warp : 32 * (warp & 1)) + gp;
+  const int nrow = (swiglu_in ? rb * TMA_BOX_ROWS + 16 * warp : rb * 2 * TMA_BOX_ROWS + 32 * warp) + gp;
+  const int dmt = swiglu_in ? TMA_BOX_BYTES : 16 * 128;
+  const unsigned char* row_base = st + box_first * TMA_BOX_BYTES + r_first * 128;
+  const unsigned char* sc_base = st + scale_tile_offset(NT) + (box_first * TMA_BOX_ROWS + r_first) * 16 +
+                                 (((min(nrow, N - 1) * ngroups + g0) * ssz) & 3);
+  const unsigned char* xlane = st + 2 * TMA_BOX_BYTES + g * TMA_XROW_MAX + t * 16;
 #if EMOE_TMA_UNROLL_SEGS
 #pragma unroll
 #else
@@ -187,52 +203,70 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int r
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         if (nt * 8 < ntok) {
-          const unsigned char* src = xt + (nt * 8 + g) * TMA_XROW_MAX + sg * 256 + t * 16;
+          const unsigned char* src = xlane + nt * 8 * TMA_XROW_MAX + sg * 256;
 #pragma unroll
           for (int q = 0; q < 4; ++q) bq[nt][q] = *reinterpret_cast<const uint4*>(src + q * 64);
         }
       }
-      // one 16-row tile at a time, one k16-pair step at a time: the unpacked codes of a step
-      // live in 8 registers and go straight into the MMAs.  The k-steps alternate between two
-      // partial accumulators so that consecutive MMAs do not depend on each other.
+      // - sum_k c_k x_k of the segment (see ffn_tile.cuh): the same for every output channel, so
+      // one pair of MMAs per step, with the constants as A operand, serves both 16-row tiles
+      float osum[NT][2];  // per token (2t, 2t+1)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        float da[4] = {0.0f, 0.0f, 0.0f, 0.0f}, db[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (OFFSET_CODES && nt * 8 < ntok) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            mma_f16(da, offset_const<BITS>(0), offset_const<BITS>(0), offset_const<BITS>(1), offset_const<BITS>(1),
+                    bq[nt][q].x, bq[nt][q].y);
+            mma_f16(db, offset_const<BITS>(2), offset_const<BITS>(2), offset_const<BITS>(3), offset_const<BITS>(3),
+                    bq[nt][q].z, bq[nt][q].w);
+          }
+        }
+        osum[nt][0] = -(da[0] + db[0]);
+        osum[nt][1] = -(da[1] + db[1]);
+      }
+      const int sdelta = (group_of(k0 + sg * 128, a.gshift, L.group, ngroups) - g0) * ssz;
+      // one 16-row tile at a time, one k16-pair step at a time: the codes of a step live in 8
+      // registers and go straight into the MMAs.  The k-steps alternate between two partial
+      // accumulators so that consecutive MMAs do not depend on each other; the first starts from
+      // the constant's share.
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        const int box_i = swiglu_in ? mt : (warp >> 1);
-        const int r0 = (swiglu_in ? 16 * warp : 32 * (warp & 1) + 16 * mt) + gp;
-        const unsigned char* box = st + box_i * TMA_BOX_BYTES;
-        const Raw<BITS> raw0 = lds_raw<BITS>(box, r0, sg, t);
-        const Raw<BITS> raw1 = lds_raw<BITS>(box, r0 + 8, sg, t);
+        const Raw<BITS> raw0 = lds_raw<BITS>(row_base + mt * dmt, swz, sg, t);
+        const Raw<BITS> raw1 = lds_raw<BITS>(row_base + mt * dmt + 8 * 128, swz, sg, t);
+        const unsigned char* sc = sc_base + mt * (dmt >> 3) + sdelta;
         float s0, s1;
-        {
-          const int n0 = min(nrow0 + (swiglu_in ? 0 : 16 * mt) + gp, N - 1), n1 = min(n0 + 8, N - 1);
-          const int grp = group_of(k0 + sg * 128, G, ngroups);
-          const unsigned char* w0 = sct + (box_i * TMA_BOX_ROWS + r0) * 16 + (n0 * ngroups + grp) * ssz -
-                                    scale_window_begin(n0, ngroups, g0, ssz);
-          const unsigned char* w1 = sct + (box_i * TMA_BOX_ROWS + r0 + 8) * 16 + (n1 * ngroups + grp) * ssz -
-                                    scale_window_begin(n1, ngroups, g0, ssz);
-          if (ssz == 2) {
-            s0 = __half2float(*reinterpret_cast<const __half*>(w0));
-            s1 = __half2float(*reinterpret_cast<const __half*>(w1));
-          } else {
-            s0 = *reinterpret_cast<const float*>(w0);
-            s1 = *reinterpret_cast<const float*>(w1);
-          }
+        if (ssz == 2) {
+          s0 = __half2float(*reinterpret_cast<const __half*>(sc));
+          s1 = __half2float(*reinterpret_cast<const __half*>(sc + 8 * 16));
+        } else {
+          s0 = *reinterpret_cast<const float*>(sc);
+          s1 = *reinterpret_cast<const float*>(sc + 8 * 16);
         }
         float pa[NT][4], pb[NT][4];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int nt = 0; nt < NT; ++nt) {
+          pa[nt][0] = pa[nt][2] = osum[nt][0];
+          pa[nt][1] = pa[nt][3] = osum[nt][1];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) pa[nt][i] = pb[nt][i] = 0.0f;
+          for (int i = 0; i < 4; ++i) pb[nt][i] = 0.0f;
+        }
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           uint32_t c0[4], c1[4];
-          unpack_step(raw0, q, c0);
-          unpack_step(raw1, q, c1);
+          if (OFFSET_CODES) {
+            unpack_step_off(raw0, q, c0);
+            unpack_step_off(raw1, q, c1);
+          } else {
+            unpack_step_exact(raw0, q, c0);
+            unpack_step_exact(raw1, q, c1);
+          }
 #pragma unroll
           for (int nt = 0; nt < NT; ++nt)
             if (nt * 8 < ntok) {
-              mma_bf16(pa[nt], c0[0], c1[0], c0[1], c1[1], bq[nt][q].x, bq[nt][q].y);
-              mma_bf16(pb[nt], c0[2], c1[2], c0[3], c1[3], bq[nt][q].z, bq[nt][q].w);
+              mma_f16(pa[nt], c0[0], c1[0], c0[1], c1[1], bq[nt][q].x, bq[nt][q].y);
+              mma_f16(pb[nt], c0[2], c1[2], c0[3], c1[3], bq[nt][q].z, bq[nt][q].w);
             }
         }
 #pragma unroll
@@ -249,6 +283,20 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int r
   __syncwarp();
   if (lane == 0) mbar_arrive(bar_empty);
 }
+
+// This warp's share of an expert's hidden vectors is written: make it visible to the bulk copies
+// of other SMs (release), then count it.
+__device__ __forceinline__ void count_item_done(PlanRec* recs, int ai, int lane) {
+  asm volatile("fence.proxy.async;" ::: "memory");
+  __syncwarp();
+  if (lane == 0) {
+    __threadfence();
+    atomicAdd(&recs[ai].done, 1);
+  }
+}
+
+// the hidden vector is rounded to bf16 (the layer's activation type), then carried as fp16
+__device__ __forceinline__ __half hidden_value(float h) { return f32_to_f16_sat(__bfloat162float(__float2bfloat16_rn(h))); }
 
 // results of one item pass: lane holds rows (gp, gp+8) x tokens (2t, 2t+1) of every tile
 template <int BITS, int NT>
@@ -270,7 +318,7 @@ __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m,
         const int n = m.rb * TMA_BOX_ROWS + 16 * warp + gp + 8 * (i >> 1);
         if (n < N) {
           const float av = tot[0][nt][i], bv = tot[1][nt][i];
-          a.hidden[slot * N + act_pos<BITS>(n)] = __float2bfloat16_rn(av / (1.0f + expf(-av)) * bv);
+          a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(av / (1.0f + expf(-av)) * bv);
         }
       } else {
 #pragma unroll
@@ -278,7 +326,7 @@ __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m,
           const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
           if (n >= N) continue;
           if (m.phase == 0)
-            a.hidden[slot * N + act_pos<BITS>(n)] = __float2bfloat16_rn(fmaxf(tot[mt][nt][i], 0.0f));
+            a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(fmaxf(tot[mt][nt][i], 0.0f));
           else
             a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + slot) * N + n] = tot[mt][nt][i];
         }
@@ -300,11 +348,7 @@ __host__ __device__ constexpr int smem_bytes_for() {
 }
 
 template <int NT>
-#ifdef EMOE_TMA_MAXNREG
-__global__ void __maxnreg__(EMOE_TMA_MAXNREG) ffn_tma_kernel(const __grid_constant__ TmaArgs a) {
-#else
 __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_kernel(const __grid_constant__ TmaArgs a) {
-#endif
   constexpr int STAGES = stages_for<NT>();
   constexpr int STAGE_BYTES = stage_bytes_for(NT);
   extern __shared__ unsigned char smem_raw[];
@@ -371,11 +415,10 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
       const int K = pd.K;
       const bool swiglu_in = pd.swiglu_in;
       const int mat_first = pd.mat_first;
-      const int Gk = L.group > 0 ? L.group : K;
-      const int ngroups_k = K / Gk;
+      const int ngroups_k = a.ngroups[phase];
       const int ai = li / (pd.ksplit * pd.row_blocks);
       const PlanRec rec = (it == 0 && ai == ai_guess) ? rec_guess : recs[ai];
-      const __nv_bfloat16* in = phase == 0 ? a.xs : a.hidden;
+      const __half* in = phase == 0 ? a.xs : a.hidden;
       const int z = li % pd.ksplit;
       const int rb = (li / pd.ksplit) % pd.row_blocks;
       const int e = rec.e;
@@ -391,6 +434,17 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
       const int npass = (cnt + NT * 8 - 1) / (NT * 8);
       const int row0 = rb * pd.rows_per_item;
       bool need_dep = fused && phase == 1;
+      // scale rows of the item this lane copies (rows 4l .. 4l+3 of a stage, box-major): start
+      // of each row's scale channel as a byte offset from its 4-byte-aligned matrix base
+      const char* srow_base[4];
+      int srow_off[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int row = 4 * lane + r;
+        const int n = min(swiglu_in ? row0 + (row & 63) : row0 + row, pd.N - 1);
+        srow_base[r] = static_cast<const char*>(swiglu_in ? rec.scales[row >> 6] : rec.scales[mat_first]);
+        srow_off[r] = n * ngroups_k * ssz;
+      }
       for (int pass = 0; pass < npass && ok; ++pass) {
         const int p0 = pass * NT * 8;
         const int ntok = min(NT * 8, cnt - p0);
@@ -407,14 +461,13 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           const int k0 = (step_begin + s) * kspan;
           const int klen = nsteps > 0 ? min(kspan, K - k0) : 0;
           if (lane == 0) {
-            StageMeta& m = meta[stage];
-            m.e = e; m.rb = rb; m.z = z; m.begin = begin; m.p0 = p0; m.ntok = ntok; m.k0 = k0; m.bits = bits;
-            m.phase = phase;
-            m.ai = ai;
-            m.flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0) |
-                      (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0);
-            m.scales[0] = swiglu_in ? rec.scales[0] : rec.scales[mat_first];
-            m.scales[1] = swiglu_in ? rec.scales[1] : rec.scales[mat_first];
+            const int flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0) |
+                              (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0);
+            // the record as three 16-byte stores (field order of StageMeta)
+            uint4* mq = reinterpret_cast<uint4*>(&meta[stage]);
+            mq[0] = make_uint4(e, rb, z, begin);
+            mq[1] = make_uint4(p0, ntok, k0, bits);
+            mq[2] = make_uint4(flags, phase, ai, 0);
             if (klen > 0) {
               mbar_expect_tx(full, 2 * TMA_BOX_BYTES + ntok * klen * 2);
               const int c0 = k0 * bits / 8;
@@ -433,17 +486,17 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           if (klen > 0) {
             // scales: lane l copies the windows of rows 4l .. 4l+3 of the stage (box-major)
             const int nseg = klen / 128;
-            const int g0 = group_of(k0, Gk, ngroups_k), g1 = group_of(k0 + (nseg - 1) * 128, Gk, ngroups_k);
+            const int g0 = group_of(k0, a.gshift, L.group, ngroups_k),
+                      g1 = group_of(k0 + (nseg - 1) * 128, a.gshift, L.group, ngroups_k);
             const uint32_t sdst = smem_u32(st + scale_tile_offset(NT));
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
-              const int row = 4 * lane + r;
-              const int n = min(swiglu_in ? row0 + (row & 63) : row0 + row, pd.N - 1);
-              const char* sp = static_cast<const char*>(swiglu_in ? rec.scales[row >> 6] : rec.scales[mat_first]);
-              const int b0 = scale_window_begin(n, ngroups_k, g0, ssz);
-              const int b1 = (n * ngroups_k + g1 + 1) * ssz;
+              const int b0 = (srow_off[r] + g0 * ssz) & ~3;
+              const int b1 = srow_off[r] + (g1 + 1) * ssz;
+#pragma unroll 1
               for (int w = 0; b0 + 4 * w < b1; ++w)
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + row * 16 + 4 * w), "l"(sp + b0 + 4 * w)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + (4 * lane + r) * 16 + 4 * w),
+                             "l"(srow_base[r] + b0 + 4 * w)
                              : "memory");
             }
             asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full) : "memory");
@@ -510,7 +563,7 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
         const PhaseDims pn = phase_dims(a, phn);
         const PlanRec rn = recs[lin / (pn.ksplit * pn.row_blocks)];
         const int rbn = (lin / pn.ksplit) % pn.row_blocks;
-        const int ngroups = L.group > 0 ? pn.K / L.group : 1;
+        const int ngroups = a.ngroups[phn];
         const int rows = min(pn.rows_per_item, pn.N - rbn * pn.rows_per_item);
         const int lines = (rows * ngroups * ssz + 127) / 128;
         const size_t offs = static_cast<size_t>(rbn) * pn.rows_per_item * ngroups * ssz;
@@ -546,9 +599,17 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
   } else {
     // ---------------- consumer warps ----------------
     float tot[2][NT][4];
+    // A finished first-projection item is counted one stage late: by then its stores have long
+    // been acknowledged and the fence in front of the count costs nothing.  It is never held back
+    // across a wait, because the stage waited for may be the one that waits for this count.
+    int pending_ai = -1;
     for (int it = 0;; ++it) {
       const int stage = it % STAGES;
       const uint32_t par = (it / STAGES) & 1;
+      if (pending_ai >= 0 && !__shfl_sync(0xffffffffu, mbar_try_wait(bar_full + 8 * stage, par) ? 1 : 0, 0)) {
+        count_item_done(recs, pending_ai, lane);
+        pending_ai = -1;
+      }
       if (!mbar_wait(bar_full + 8 * stage, par, a.check_word, abort_flag)) break;
       const StageMeta m = meta[stage];
       if (m.flags & META_STOP) break;
@@ -577,22 +638,19 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           case 4: store_item<4, NT>(a, m, warp, lane, tot); break;
           default: store_item<8, NT>(a, m, warp, lane, tot); break;
         }
-        if (m.flags & META_DONE) {
-          // this warp's share of the expert's hidden vectors is written: make it visible to the
-          // bulk copies of other SMs, then count it
-          asm volatile("fence.proxy.async;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) {
-            __threadfence();
-            atomicAdd(&recs[m.ai].done, 1);
-          }
-        }
       }
+      if (pending_ai >= 0) {
+        count_item_done(recs, pending_ai, lane);
+        pending_ai = -1;
+      }
+      if ((m.flags & META_LAST) && (m.flags & META_DONE)) pending_ai = m.ai;
     }
+    if (pending_ai >= 0) count_item_done(recs, pending_ai, lane);
   }
   if (*abort_flag) {
     // a wait ran out: give copies that may still be in flight time to land before the CTA's
     // shared memory is released
+#pragma unroll 1
     for (int i = 0; i < 2000; ++i) __nanosleep(100);
   }
 }
@@ -652,14 +710,19 @@ cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, c
   a.L = L;
   a.experts = experts;
   a.tmaps = static_cast<const CUtensorMap*>(tmaps);
-  a.xs = xs;
+  a.xs = reinterpret_cast<const __half*>(xs);
   a.off = off;
   a.plan = plan;
-  a.hidden = hidden;
+  a.hidden = reinterpret_cast<__half*>(hidden);
   a.o_part = o_part;
   a.ksplit = ksplit;
   a.row_blocks[0] = (L.d_ff + rows_first - 1) / rows_first;
   a.row_blocks[1] = (L.d_model + 2 * TMA_BOX_ROWS - 1) / (2 * TMA_BOX_ROWS);
+  a.ngroups[0] = L.group > 0 ? L.d_model / L.group : 1;
+  a.ngroups[1] = L.group > 0 ? L.d_ff / L.group : 1;
+  a.gshift = -1;
+  for (int b = 7; b < 31; ++b)
+    if (L.group == (1 << b)) a.gshift = b;
   a.n_pairs = n_pairs;
   a.check_word = check_word;
   const long long active_max = n_pairs < L.E ? n_pairs : L.E;
