@@ -691,7 +691,9 @@ int ffn_tma_ksplit(const LayerDims& L, int T) {
   const long long active = pairs < L.E ? pairs : L.E;
   const long long ctas = row_blocks * active;
   const int steps_min = (L.d_ff + 511) / 512;  // stages at the widest span (2 bits)
-  long long z = (4 * 148 + ctas - 1) / ctas;
+  // enough slices that the second projection's items outnumber the resident CTAs (3 per SM)
+  // about twice: short items at the end of the launch keep its tail short
+  long long z = (8 * 148 + ctas - 1) / ctas;
   if (z > steps_min) z = steps_min;
   if (z > 16) z = 16;
   if (z < 1) z = 1;
