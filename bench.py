@@ -29,10 +29,10 @@ if ROOT not in sys.path:
 
 from paper_2308_14352_b200 import inputs  # noqa: E402
 
-# DRAM bytes (read + write) of the two expert-FFN launches of one layer from the ncu capture
-# summarised in profiles/ffn_tma_kernel_switch_base_decode_T64.md; reported as `traffic` for
-# that workload only, and to be set back to None whenever that kernel changes.
-NCU_DRAM_BYTES_PER_LAYER = {("switch_base_decode", 64): 71.0e6}
+# DRAM bytes (read + write) of the expert-FFN launch of one layer (mean of the two layers of the ncu
+# capture summarised in profiles/ffn_tma_kernel_switch_base_decode_T64.md); reported as `traffic`
+# for that workload only, and to be set back to None whenever that kernel changes.
+NCU_DRAM_BYTES_PER_LAYER = {("switch_base_decode", 64): 75.0e6}
 
 METRIC = "MoE-layer tokens/s"
 UNIT = "tokens/s"
@@ -334,7 +334,8 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
         else:
             forward_all(stream.cuda_stream)
 
-    kernels_per_layer = 6  # router+top-k, permute, scatter, two expert-FFN launches, combine
+    # router+top-k, permute, scatter, expert FFNs (one launch or two), combine: as counted by the library
+    kernels_per_layer = B.emoe_kernels_last_forward(ctx)
     launches_per_step = kernels_per_layer * n_layers
 
     # ---- device-resident timing ----------------------------------------------------------------

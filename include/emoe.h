@@ -201,6 +201,11 @@ int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled);
  * projections as two launches (to compare timings, or to time them separately). */
 int emoe_set_fused_projections(emoe_ctx* ctx, int enabled);
 
+/* Number of kernels the last emoe_moe_forward / emoe_moe_forward_routed call on this context
+ * enqueued (router + Top-K, permutation, scatter, expert FFNs, combine: Sections 2.1 and 3.2 name
+ * the steps, the count depends on the kernel family the shape takes).  0 before the first call. */
+int emoe_kernels_last_forward(const emoe_ctx* ctx);
+
 /* The routed layer forward for callers that cannot allocate device memory (the paper has no
  * counterpart: it is an addition for hosts such as a framework that owns the whole device
  * heap, a plug-in whose memory pool is fixed at start-up, or a latency-critical loop in which
@@ -229,7 +234,9 @@ int emoe_moe_forward_routed_static(int device, const emoe_layer_desc* desc, cons
  * call records CUDA events on its stream around the first-projection and second-projection
  * expert kernels.  emoe_read_timing waits for the recorded events, returns the summed device
  * time of each projection (milliseconds) and the number of forward calls covered, and clears
- * the record.  Off by default; not for use during stream capture. */
+ * the record.  Where both projections run as one launch (see emoe_set_fused_projections) the
+ * whole time is returned as the first value and the second is 0.  Off by default; not for use
+ * during stream capture. */
 int emoe_set_timing(emoe_ctx* ctx, int enabled);
 int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, int* out_calls);
 

@@ -30,7 +30,7 @@ EXPORTS = (
     "emoe_status_string", "emoe_packed_bytes", "emoe_scales_bytes", "emoe_pack_expert", "emoe_router_topk",
     "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
     "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_set_dependent_launch",
-    "emoe_set_fused_projections",
+    "emoe_set_fused_projections", "emoe_kernels_last_forward",
 )
 
 
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.emoe_set_timing.argtypes = [vp, i32]
         L.emoe_set_dependent_launch.argtypes = [vp, i32]
         L.emoe_set_fused_projections.argtypes = [vp, i32]
+        L.emoe_kernels_last_forward.argtypes = [vp]
         L.emoe_moe_forward_routed_static.argtypes = [i32, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
                                                      ctypes.POINTER(emoe_expert), vp, vp]
         L.emoe_read_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
@@ -207,3 +208,7 @@ def emoe_set_dependent_launch(ctx, enabled: bool) -> None:
 
 def emoe_set_fused_projections(ctx, enabled: bool) -> None:
     _check(lib().emoe_set_fused_projections(ctx, int(enabled)), "emoe_set_fused_projections")
+
+
+def emoe_kernels_last_forward(ctx) -> int:
+    return int(lib().emoe_kernels_last_forward(ctx))

@@ -97,8 +97,10 @@ struct emoe_ctx {
   bool pdl = true;  // programmatic dependent launch along the kernel chain of a forward call
   bool fuse_projections = true;  // weight-streaming kernel: both projections in one launch
   bool timing = false;
+  int kernels_last = 0;  // kernels the last forward call enqueued
   std::vector<cudaEvent_t> events;  // triples (start, mid, end) per timed forward call
   size_t events_used = 0;
+  std::vector<char> events_one_launch;  // per triple: both projections ran as one launch (no second interval)
 };
 
 namespace {
@@ -112,6 +114,13 @@ int cuda_fail(emoe_ctx* ctx, cudaError_t e) {
   do {                                                \
     cudaError_t e__ = (call);                         \
     if (e__ != cudaSuccess) return cuda_fail(ctx, e__); \
+  } while (0)
+
+// a kernel launch of a forward call: counted, so that callers can report how many kernels ran
+#define EMOE_LAUNCH(ctx, call) \
+  do {                         \
+    EMOE_CUDA(ctx, call);      \
+    ++(ctx)->kernels_last;     \
   } while (0)
 
 // Device copy of a host expert table (entries + tensor maps); uploaded on `st` the first time
@@ -209,6 +218,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     ~PdlScope() { g_pdl_enabled = false; }
   } pdl_scope(ctx->pdl && !ctx->timing);
 
+  ctx->kernels_last = 0;
   const ExpertDev* table = nullptr;
   const void* tmaps = nullptr;
   rc = get_table(ctx, L, host_experts, st, &table, &tmaps);
@@ -233,10 +243,10 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     ids_use = ids_in;
     gates_use = gates_in;
   } else {
-    EMOE_CUDA(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,
+    EMOE_LAUNCH(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,
                                       L.top_k, L.gate_mode == EMOE_GATE_SOFTMAX_RENORM, ids, gates, nullptr, st));
   }
-  EMOE_CUDA(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
+  EMOE_LAUNCH(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
 
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
   const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
@@ -256,44 +266,50 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       ctx->events.push_back(e);
     }
     for (int i = 0; i < 3; ++i) ev[i] = ctx->events[ctx->events_used + i];
+    if (ctx->events_one_launch.size() < ctx->events_used / 3 + 1) ctx->events_one_launch.resize(ctx->events_used / 3 + 1);
+    ctx->events_one_launch[ctx->events_used / 3] = 0;
     ctx->events_used += 3;
   }
   if (use_umma) {
-    EMOE_CUDA(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
-    EMOE_CUDA(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, P, ctx->check_word, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-    EMOE_CUDA(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
   } else if (use_tma) {
     ksplit = ffn_tma_ksplit(L, T);
-    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
     if (ctx->fuse_projections) {
       // one launch: an expert's second projection starts when its hidden vectors are complete
-      EMOE_CUDA(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
-      if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      if (ev[1]) {  // one interval only: the end event of the triple stays unused
+        EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+        ctx->events_one_launch[ctx->events_used / 3 - 1] = 1;
+        ev[2] = nullptr;
+      }
     } else {
-      EMOE_CUDA(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
       if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-      EMOE_CUDA(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
     }
   } else if (use_mma) {
     ksplit = ffn_mma_ksplit(L, T);
-    EMOE_CUDA(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, false, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, false, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
-    EMOE_CUDA(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
+    EMOE_LAUNCH(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-    EMOE_CUDA(ctx, launch_ffn_mma(1, L, table, reinterpret_cast<const __nv_bfloat16*>(hidden), off,
+    EMOE_LAUNCH(ctx, launch_ffn_mma(1, L, table, reinterpret_cast<const __nv_bfloat16*>(hidden), off,
                                   reinterpret_cast<__nv_bfloat16*>(hidden), o_part, ksplit, P, T, st));
   } else {
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
-    EMOE_CUDA(ctx, launch_ffn_gemv(0, L, table, x, perm, off, hidden, o_part, P, st));
+    EMOE_LAUNCH(ctx, launch_ffn_gemv(0, L, table, x, perm, off, hidden, o_part, P, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-    EMOE_CUDA(ctx, launch_ffn_gemv(1, L, table, x, perm, off, hidden, o_part, P, st));
+    EMOE_LAUNCH(ctx, launch_ffn_gemv(1, L, table, x, perm, off, hidden, o_part, P, st));
   }
   if (ev[2]) EMOE_CUDA(ctx, cudaEventRecord(ev[2], st));
-  EMOE_CUDA(ctx, launch_combine(o_part, ksplit, static_cast<size_t>(P), gates_use, slot_of_pair, T, L.top_k, L.d_model,
+  EMOE_LAUNCH(ctx, launch_combine(o_part, ksplit, static_cast<size_t>(P), gates_use, slot_of_pair, T, L.top_k, L.d_model,
                                 y, st));
   if (out_ids) EMOE_CUDA(ctx, cudaMemcpyAsync(out_ids, ids_use, sizeof(int32_t) * P, cudaMemcpyDeviceToDevice, st));
   if (out_gates) EMOE_CUDA(ctx, cudaMemcpyAsync(out_gates, gates_use, sizeof(float) * P, cudaMemcpyDeviceToDevice, st));
@@ -459,11 +475,14 @@ int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, i
   const size_t n = ctx->events_used / 3;
   for (size_t i = 0; i < n; ++i) {
     float ms = 0.f;
-    EMOE_CUDA(ctx, cudaEventSynchronize(ctx->events[3 * i + 2]));
+    const bool one = ctx->events_one_launch[i] != 0;
+    EMOE_CUDA(ctx, cudaEventSynchronize(ctx->events[3 * i + (one ? 1 : 2)]));
     EMOE_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->events[3 * i], ctx->events[3 * i + 1]));
     a += ms;
-    EMOE_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->events[3 * i + 1], ctx->events[3 * i + 2]));
-    b += ms;
+    if (!one) {
+      EMOE_CUDA(ctx, cudaEventElapsedTime(&ms, ctx->events[3 * i + 1], ctx->events[3 * i + 2]));
+      b += ms;
+    }
   }
   *out_first_ms = a;
   *out_second_ms = b;
@@ -477,6 +496,8 @@ int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled) {
   ctx->pdl = enabled != 0;
   return EMOE_OK;
 }
+
+int emoe_kernels_last_forward(const emoe_ctx* ctx) { return ctx ? ctx->kernels_last : 0; }
 
 int emoe_set_fused_projections(emoe_ctx* ctx, int enabled) {
   if (!ctx) return EMOE_ERR_INVALID_ARG;
