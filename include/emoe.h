@@ -185,8 +185,10 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
 /* Selects the expert-FFN kernel family: 0 = automatic (default), 1 = the CUDA-core grouped
  * GEMV, 2 = the tensor-core kernel with register-staged weight loads, 3 = the tensor-core kernel
  * with the TMA-staged weight pipeline, 4 = the tcgen05 grouped GEMM (fp16 operands; meant for
- * many tokens per expert).  2, 3 and 4 fail with EMOE_ERR_UNSUPPORTED in forward calls whose shape
- * they do not take.  For tests and measurements. */
+ * many tokens per expert), 5 = both of the last two in one call: experts with at most 32 tokens
+ * take the streaming kernel, the others the grouped GEMM (what 0 picks for large batches).
+ * 2 to 5 fail with EMOE_ERR_UNSUPPORTED in forward calls whose shape they do not take.  For tests
+ * and measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);
 
 /* Programmatic dependent launch along the kernels of a forward call (on by default): each

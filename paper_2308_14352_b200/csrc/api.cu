@@ -2,6 +2,7 @@
 // (router -> Top-K -> permutation -> expert FFNs on packed weights -> combine).  All
 // arithmetic is in the kernels of the sibling files; nothing here touches tensor data on the
 // host.
+#include <climits>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -71,7 +72,7 @@ WorkspaceLayout make_layout(const LayerDims& L, int T) {
   w.off = o;          o += align_up(static_cast<size_t>(L.E + 1) * 4);
   w.perm = o;         o += align_up(P * 4);
   w.slot_of_pair = o; o += align_up(P * 4);
-  w.plan = o;         o += align_up(plan_bytes(L.E));
+  w.plan = o;         o += 2 * align_up(plan_bytes(L.E));  // two plans: one per kernel family of a forward call
   w.xs = o;           o += align_up(L.act_bf16 ? P * L.d_model * 2 : 0);
   w.hidden = o;       o += align_up(P * L.d_ff * (L.act_bf16 ? 2 : 4));
   w.o_part = o;       o += align_up(static_cast<size_t>(w.ksplit) * P * L.d_model * 4);
@@ -251,12 +252,17 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
   const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
   // many tokens per expert: the tcgen05 grouped GEMM; otherwise the weight-streaming kernels
-  const bool use_umma = can_umma && (ctx->ffn_path == 4 || (ctx->ffn_path == 0 && ffn_token_tiles(L, T) >= 4));
-  const bool use_tma = !use_umma && can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
+  const bool many_tokens = ffn_token_tiles(L, T) >= 4;
+  // skewed loads: experts with few tokens stream through the TMA kernel, the others take the
+  // tcgen05 grouped GEMM, in the same forward call
+  const bool use_hybrid = can_umma && can_tma && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens));
+  const bool use_umma = !use_hybrid && can_umma && (ctx->ffn_path == 4 || (ctx->ffn_path == 0 && many_tokens));
+  const bool use_tma = !use_hybrid && !use_umma && can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
   const bool use_mma = ffn_mma_supported(L) && ctx->ffn_path != 1;
   if (ctx->ffn_path == 2 && !use_mma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 3 && !use_tma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 4 && !use_umma) return EMOE_ERR_UNSUPPORTED;
+  if (ctx->ffn_path == 5 && !use_hybrid) return EMOE_ERR_UNSUPPORTED;
   int ksplit = 1;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
   if (ctx->timing) {
@@ -270,33 +276,68 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     ctx->events_one_launch[ctx->events_used / 3] = 0;
     ctx->events_used += 3;
   }
-  if (use_umma) {
-    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, st));
+  if (use_hybrid) {
+    // experts with up to HYBRID_STREAM_TOKENS tokens: one or two passes of 16-token tiles through the
+    // streaming kernel (measured best on a Zipf(1.1) load over 128 experts: 16 .. 128 tokens all within
+    // 10 %); the others: 128-token tiles on tcgen05.  Each family has its own plan and writes only
+    // its own slots of xs / hidden / o_part.
+#ifndef EMOE_HYBRID_TOKENS
+#define EMOE_HYBRID_TOKENS 32
+#endif
+#ifndef EMOE_HYBRID_TILES
+#define EMOE_HYBRID_TILES 2
+#endif
+    constexpr int HYBRID_STREAM_TOKENS = EMOE_HYBRID_TOKENS;
+    int* plan_heavy = reinterpret_cast<int*>(reinterpret_cast<char*>(plan) + align_up(plan_bytes(L.E)));
+    __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
+    ksplit = ffn_tma_ksplit(L, T);
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, 1, HYBRID_STREAM_TOKENS, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan_heavy, xs, P, HYBRID_STREAM_TOKENS + 1, INT_MAX, st));
+    if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
+    // the tcgen05 kernel writes plane 0 only: the other split-K planes of its slots must read as zero
+    if (ksplit > 1)
+      EMOE_CUDA(ctx, cudaMemsetAsync(o_part + static_cast<size_t>(P) * L.d_model, 0,
+                                     static_cast<size_t>(ksplit - 1) * P * L.d_model * sizeof(float), st));
+    if (ctx->fuse_projections) {
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
+    } else {
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
+    }
+    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, P, ctx->check_word, st));
+    if (ev[1]) {  // one interval for the whole expert stage
+      EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+      ctx->events_one_launch[ctx->events_used / 3 - 1] = 1;
+      ev[2] = nullptr;
+    }
+  } else if (use_umma) {
+    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, 1, INT_MAX, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, P, ctx->check_word, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
     EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
   } else if (use_tma) {
     ksplit = ffn_tma_ksplit(L, T);
-    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, 1, INT_MAX, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
     if (ctx->fuse_projections) {
       // one launch: an expert's second projection starts when its hidden vectors are complete
-      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, 0, ctx->check_word, st));
       if (ev[1]) {  // one interval only: the end event of the triple stays unused
         EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
         ctx->events_one_launch[ctx->events_used / 3 - 1] = 1;
         ev[2] = nullptr;
       }
     } else {
-      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, 0, ctx->check_word, st));
       if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-      EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, 0, ctx->check_word, st));
     }
   } else if (use_mma) {
     ksplit = ffn_mma_ksplit(L, T);
-    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, false, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, false, 1, INT_MAX, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_LAUNCH(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
@@ -506,7 +547,7 @@ int emoe_set_fused_projections(emoe_ctx* ctx, int enabled) {
 }
 
 int emoe_set_ffn_path(emoe_ctx* ctx, int path) {
-  if (!ctx || path < 0 || path > 4) return EMOE_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 5) return EMOE_ERR_INVALID_ARG;
   ctx->ffn_path = path;
   return EMOE_OK;
 }

@@ -99,9 +99,11 @@ int ffn_mma_ksplit(const LayerDims& L, int T);
 int ffn_token_tiles(const LayerDims& L, int T);
 // plan (nullable): plan_bytes(E) bytes, the work plan for the persistent TMA kernels, filled by block 0.
 // to_f16: store the rows as fp16 (saturating) instead of bf16, same layout (the TMA-staged kernel's input).
+// cnt_lo .. cnt_hi: only experts with that many tokens are listed in the plan and have their rows
+// written (1 .. INT_MAX: all activated experts); lets two kernel families share one forward call.
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
-                             bool to_f16, cudaStream_t st);
+                             bool to_f16, int cnt_lo, int cnt_hi, cudaStream_t st);
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
                            const int32_t* off, __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs,
                            int T, cudaStream_t st);
@@ -113,10 +115,11 @@ int ffn_tma_ksplit(const LayerDims& L, int T);
 int encode_weight_tmap(void* out_map, const void* packed, int N, int K, int bits);
 // Phases [phase_begin, phase_end) of the FFN in one launch: (0,1) first projection, (1,2) second,
 // (0,2) both, the second projection of an expert starting as soon as its hidden vectors are complete.
+// token_tiles: 8-token tiles per pass (1, 2 or 4), 0 = by the routing statistics of (L, T).
 cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, const ExpertDev* experts,
                            const void* tmaps, const __nv_bfloat16* xs, const int32_t* off, int* plan,
-                           __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs, int T, int* check_word,
-                           cudaStream_t st);
+                           __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs, int T, int token_tiles,
+                           int* check_word, cudaStream_t st);
 
 int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
                    uint32_t box_inner, uint32_t box_outer);
@@ -126,7 +129,7 @@ int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, u
 bool ffn_umma_supported(const LayerDims& L);
 cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
-                               cudaStream_t st);
+                               int cnt_lo, int cnt_hi, cudaStream_t st);
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
                             void* hidden16, float* o, int n_pairs, int* check_word, cudaStream_t st);
 

@@ -702,8 +702,8 @@ int ffn_tma_ksplit(const LayerDims& L, int T) {
 
 cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, const ExpertDev* experts,
                            const void* tmaps, const __nv_bfloat16* xs, const int32_t* off, int* plan,
-                           __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs, int T, int* check_word,
-                           cudaStream_t st) {
+                           __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs, int T, int token_tiles,
+                           int* check_word, cudaStream_t st) {
   if (phase_begin < 0 || phase_end > 2 || phase_begin >= phase_end) return cudaErrorInvalidValue;
   const int rows_first = L.act == EMOE_ACT_SWIGLU ? TMA_BOX_ROWS : 2 * TMA_BOX_ROWS;
   TmaArgs a;
@@ -733,7 +733,7 @@ cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, c
   if (phase_end == 2) per_expert += static_cast<long long>(a.row_blocks[1]) * ksplit;
   const long long items = active_max * per_expert;
   const int max_items = items > (1 << 30) ? (1 << 30) : static_cast<int>(items);
-  const int nt = ffn_token_tiles(L, T);
+  const int nt = token_tiles > 0 ? token_tiles : ffn_token_tiles(L, T);
   if (nt == 1) return launch_nt<1>(a, max_items, st);
   if (nt == 2) return launch_nt<2>(a, max_items, st);
   return launch_nt<4>(a, max_items, st);

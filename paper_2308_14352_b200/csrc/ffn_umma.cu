@@ -455,7 +455,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
 __global__ void __launch_bounds__(128)
     scatter_x16_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
                        const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
-                       int E, int* __restrict__ plan, int top_k, int d, int n_pairs, __half* __restrict__ xs) {
+                       int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int cnt_lo, int cnt_hi,
+                       __half* __restrict__ xs) {
   pdl_wait();
   pdl_trigger();
   if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
@@ -466,13 +467,14 @@ __global__ void __launch_bounds__(128)
     for (int b = 8; b >= 2; b >>= 1) {
       for (int e0 = 0; e0 < E; e0 += 32) {
         const int e = e0 + lane;
-        const bool act = e < E && off[e + 1] > off[e] && experts[e].bits == b;
+        const int cnt = e < E ? off[e + 1] - off[e] : 0;
+        const bool act = cnt >= cnt_lo && cnt <= cnt_hi && experts[e].bits == b;
         const unsigned m = __ballot_sync(0xffffffffu, act);
         if (act) {
           PlanRec& r = recs[base + __popc(m & ((1u << lane) - 1u))];
           r.e = e;
           r.begin = off[e];
-          r.cnt = off[e + 1] - off[e];
+          r.cnt = cnt;
           r.bits = b;
           r.scales[0] = experts[e].scales[0];
           r.scales[1] = experts[e].scales[1];
@@ -491,7 +493,10 @@ __global__ void __launch_bounds__(128)
   const int slot = blockIdx.x;
   const int pair = perm[slot];
   if (pair < 0 || pair >= n_pairs) return;
-  const int bits = experts[ids[pair]].bits;
+  const int e_slot = ids[pair];
+  const int cnt_slot = off[e_slot + 1] - off[e_slot];
+  if (cnt_slot < cnt_lo || cnt_slot > cnt_hi) return;  // this expert's rows belong to another kernel family
+  const int bits = experts[e_slot].bits;
   const __nv_bfloat16* src = x + static_cast<size_t>(pair / top_k) * d;
   __half* dst = xs + static_cast<size_t>(slot) * d;
   for (int k = threadIdx.x; k < d; k += blockDim.x) {
@@ -509,9 +514,9 @@ bool ffn_umma_supported(const LayerDims& L) {
 
 cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
-                               cudaStream_t st) {
+                               int cnt_lo, int cnt_hi, cudaStream_t st) {
   return launch_chain(scatter_x16_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
-                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, reinterpret_cast<__half*>(xs16));
+                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, cnt_lo, cnt_hi, reinterpret_cast<__half*>(xs16));
 }
 
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,

@@ -12,6 +12,7 @@
 // The array below is that scratch.  In host code its name is only a handle of the host-side
 // shadow of the symbol, never a device address; the device address is obtained once per
 // device with cudaGetSymbolAddress and that pointer is what the kernels receive.
+#include <climits>
 #include <cstring>
 
 #include "common.cuh"
@@ -145,7 +146,7 @@ extern "C" int emoe_moe_forward_routed_static(int device, const emoe_layer_desc*
   EMOE_TRY(cudaMemsetAsync(check, 0, sizeof(int), st));
   EMOE_TRY(launch_permute(ids, P, L.E, counts, off, perm, slot_of_pair, check, st));
   if (ffn_mma_supported(L)) {
-    EMOE_TRY(launch_scatter_x(L, table, x, ids, perm, off, nullptr, xs, P, false, st));
+    EMOE_TRY(launch_scatter_x(L, table, x, ids, perm, off, nullptr, xs, P, false, 1, INT_MAX, st));
     EMOE_TRY(launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     EMOE_TRY(launch_ffn_mma(1, L, table, reinterpret_cast<const __nv_bfloat16*>(hidden), off,
                             reinterpret_cast<__nv_bfloat16*>(hidden), o_part, w.ksplit, P, T, st));

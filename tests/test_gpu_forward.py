@@ -116,6 +116,32 @@ def test_forward_tcgen05_path(act, group, sdt, d, f, E, k, gate, bits, T):
     _run_case(shape, bits, T, seed=27, path=4)
 
 
+HYBRID_CASES = [
+    # loads shaped by a router bias so that some experts hold more than 32 tokens and others fewer
+    ("relu", 128, "f16", 512, 1024, 8, 1, "softmax", [8, 4, 2, 4, 2, 8, 4, 2], 220, 1.1),
+    ("swiglu", 128, "f16", 512, 1536, 6, 2, "softmax_renorm", [4, 8, 2, 4, 2, 8], 90, 1.3),
+    ("relu", 0, "f32", 1024, 512, 5, 1, "softmax", [2, 8, 4, 4, 8], 64, 1.5),
+    ("relu", 128, "f16", 512, 512, 4, 1, "softmax", [2, 8, 4, 4], 12, 0.0),          # nobody above 32 tokens
+]
+
+
+@pytest.mark.parametrize("act,group,sdt,d,f,E,k,gate,bits,T,zipf", HYBRID_CASES)
+def test_forward_both_kernel_families_in_one_call(act, group, sdt, d, f, E, k, gate, bits, T, zipf):
+    """Skewed loads: experts with few tokens stream, the others run on tcgen05, one forward call."""
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, "bf16")
+    bias = None
+    if zipf > 0:
+        bias = (-zipf * 2.0 * np.log(np.arange(1, E + 1))).astype(np.float32)  # strongly decreasing loads
+    x = inputs.activations(29, 0, T, d, "bf16")
+    Wr = inputs.router_weight(29, 0, d, E, std=0.05)
+    ids, _, _ = oracle.route(x, Wr, bias, k, gate == "softmax_renorm")
+    counts = np.bincount(ids.reshape(-1), minlength=E)
+    if zipf > 0:
+        assert counts.max() > 32 and 0 < counts[counts > 0].min() <= 32, counts   # the case covers both families
+    _run_case(shape, bits, T, seed=29, path=5, bias=bias)
+    _run_case(shape, bits, T, seed=29, path=5, bias=bias, fused=False)
+
+
 def test_tma_path_is_refused_for_narrow_rows():
     shape = inputs.LayerShape(256, 512, 4, 1, "relu", "softmax", 128, "f16", "bf16")
     with pytest.raises(B.EmoeError) as ei:
