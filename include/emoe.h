@@ -54,6 +54,7 @@ extern "C" {
 #define EMOE_ERR_WORKSPACE (-4)    /* the context's workspace is too small for this call */
 #define EMOE_ERR_CUDA (-5)         /* a CUDA call failed; emoe_last_cuda_error() gives its code */
 #define EMOE_ERR_DEVICE_CHECK (-6) /* a kernel found inconsistent data (e.g. an expert id out of range) */
+#define EMOE_ERR_CACHE_FULL (-7)   /* every slot of the expert cache is in use by an unfinished call */
 
 /* enums (plain ints in the ABI) */
 #define EMOE_DTYPE_F32 0
@@ -241,6 +242,86 @@ int emoe_moe_forward_routed_static(int device, const emoe_layer_desc* desc, cons
  * during stream capture. */
 int emoe_set_timing(emoe_ctx* ctx, int enabled);
 int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, int* out_calls);
+
+/* ---- expert cache and prefetch ------------------------------------------------------------
+ * Section 3.3 of the paper keeps the experts in slow storage, holds a buffer of fixed size in
+ * fast memory, preloads the experts it predicts from the previous layers' activations while the
+ * current layer computes, and evicts by activation frequency and layer distance.  Here slow
+ * storage is PINNED HOST memory (owned by the caller, registered once), fast memory is
+ * `n_slots` equal HBM slots owned by the context, loads are asynchronous copies on a copy
+ * stream, and the compute stream is made to wait (on the device, never on the host) for a
+ * slot's contents.  Typical layer:  ids = router (emoe_router_topk, read back);
+ * emoe_prefetch_experts(predicted experts of the next layer);  emoe_cache_acquire(ids) -> device
+ * pointers for the expert table;  emoe_moe_forward_routed;  emoe_cache_release(ids). */
+
+#define EMOE_EVICT_FORWARD 0 /* score -f/D, D = layers until the expert's layer runs again: (i - I) mod S */
+#define EMOE_EVICT_PRINTED 1 /* score -f/D with D = (S - i + I) mod S as the formula is printed */
+#define EMOE_EVICT_LRU 2     /* least recently used */
+
+typedef struct emoe_cache_stats {
+  int64_t hits;               /* acquire found the expert in a slot (loaded or loading) */
+  int64_t misses;             /* acquire had to start the load itself */
+  int64_t prefetch_hits;      /* hits on an expert whose load a prefetch started and nobody used since */
+  int64_t prefetched;         /* loads started by prefetch calls */
+  int64_t prefetch_redundant; /* prefetch requests for experts already in a slot */
+  int64_t prefetch_refused;   /* prefetch requests dropped because every slot was in use */
+  int64_t evictions;
+  int64_t bytes_copied;       /* host -> device bytes of all loads started */
+} emoe_cache_stats;
+
+/* Allocates the cache of a context: n_slots x slot_bytes of device memory and two events per
+ * slot (the only allocating call besides emoe_create; freed by emoe_destroy).  n_layers = S of
+ * the eviction score; policy = EMOE_EVICT_*. */
+int emoe_cache_create(emoe_ctx* ctx, int n_slots, size_t slot_bytes, int n_layers, int policy);
+
+/* Registers an expert of layer `layer` under a caller-chosen id.  host_pinned_packed[3] /
+ * host_pinned_scales[3]: its matrices in pinned host memory (null with 0 bytes for an absent
+ * third matrix), bytes[6] their sizes (packed 0..2, then scales 0..2).  The memory stays the
+ * caller's and must outlive the cache.  Packed matrices must be 16-byte aligned; inside a slot
+ * every matrix starts on a 256-byte boundary. */
+int emoe_register_expert(emoe_ctx* ctx, int64_t id, int layer, int bits, const void* const* host_pinned_packed,
+                         const void* const* host_pinned_scales, const size_t* bytes);
+
+/* Starts loading the listed experts (most likely first) on copy_stream unless they are in a slot
+ * already; evicts by the policy; drops requests when every slot is in use.  current_layer = I of
+ * the score.  Never blocks the host and never makes the compute stream wait. */
+int emoe_prefetch_experts(emoe_ctx* ctx, const int64_t* ids, int n, int current_layer, void* copy_stream);
+
+/* The listed experts are about to be used on compute_stream: experts not in a slot are loaded
+ * now (on copy_stream), compute_stream waits on the device for each slot's contents, the slots
+ * are protected from eviction until emoe_cache_release, activation counts go up by one, and
+ * out_experts[i] receives the device pointers of ids[i] (valid until the release).
+ * EMOE_ERR_CACHE_FULL if a load finds every slot protected. */
+int emoe_cache_acquire(emoe_ctx* ctx, const int64_t* ids, int n, int current_layer, void* compute_stream,
+                       void* copy_stream, emoe_expert* out_experts);
+
+/* Call after the last kernel that reads the experts has been enqueued on compute_stream: a later
+ * load into one of these slots waits (on the device) until that point of the stream. */
+int emoe_cache_release(emoe_ctx* ctx, const int64_t* ids, int n, void* compute_stream);
+
+/* Slot that holds the expert, -1 if none. */
+int emoe_cache_slot_of(emoe_ctx* ctx, int64_t id);
+int emoe_cache_get_stats(emoe_ctx* ctx, emoe_cache_stats* out);
+
+/* The cache's bookkeeping alone, without a device (same code as behind the calls above): for
+ * checking slot assignment, eviction order and counters on a host without a GPU.
+ * emoe_policy_prefetch returns the slot a load would go to (-1: none), emoe_policy_acquire the
+ * slot (-1: every slot protected) with *loaded = 1 on a miss; *evicted_id = id that left, or -1. */
+typedef struct emoe_policy emoe_policy;
+emoe_policy* emoe_policy_create(int n_slots, int n_layers, int policy);
+void emoe_policy_destroy(emoe_policy* p);
+int emoe_policy_register(emoe_policy* p, int64_t id, int layer, int64_t bytes);
+int emoe_policy_prefetch(emoe_policy* p, int64_t id, int current_layer, int64_t* evicted_id);
+int emoe_policy_acquire(emoe_policy* p, int64_t id, int current_layer, int* loaded, int64_t* evicted_id);
+int emoe_policy_release(emoe_policy* p, int64_t id);
+int emoe_policy_get_stats(emoe_policy* p, emoe_cache_stats* out);
+
+/* Ranks the experts of the next layer from a first-order layer-transition prior (Section 3.3,
+ * "Estimating expert activation a priori", with one previous layer as key): prior is a host
+ * array [n_experts][n_experts], row p = distribution of the next layer's expert given pick p;
+ * score[e] = sum over prev_ids of prior[p][e]; out_order (host, n_experts entries) lists the
+ * experts by descending score, ties by lower index. */
+int emoe_rank_experts(const float* prior, int n_experts, const int32_t* prev_ids, int n_prev, int32_t* out_order);
 
 #ifdef __cplusplus
 }

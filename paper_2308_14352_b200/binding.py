@@ -20,6 +20,8 @@ ERR_ALIGNMENT = -3
 ERR_WORKSPACE = -4
 ERR_CUDA = -5
 ERR_DEVICE_CHECK = -6
+ERR_CACHE_FULL = -7
+EVICT_FORWARD, EVICT_PRINTED, EVICT_LRU = 0, 1, 2
 
 DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
 ACT_RELU, ACT_SWIGLU = 0, 1
@@ -31,6 +33,9 @@ EXPORTS = (
     "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
     "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_set_dependent_launch",
     "emoe_set_fused_projections", "emoe_kernels_last_forward",
+    "emoe_cache_create", "emoe_register_expert", "emoe_prefetch_experts", "emoe_cache_acquire", "emoe_cache_release",
+    "emoe_cache_slot_of", "emoe_cache_get_stats", "emoe_policy_create", "emoe_policy_destroy", "emoe_policy_register",
+    "emoe_policy_prefetch", "emoe_policy_acquire", "emoe_policy_release", "emoe_policy_get_stats", "emoe_rank_experts",
 )
 
 
@@ -48,6 +53,15 @@ class emoe_expert(ctypes.Structure):
 class emoe_layer_desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("d_model", "d_ff", "n_experts", "top_k", "act", "gate_mode", "group", "scale_dtype", "act_dtype")]
+
+
+class emoe_cache_stats(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in
+                ("hits", "misses", "prefetch_hits", "prefetched", "prefetch_redundant", "prefetch_refused", "evictions",
+                 "bytes_copied")]
+
+    def as_dict(self):
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
 
 
 _lib = None
@@ -88,6 +102,25 @@ def lib() -> ctypes.CDLL:
         L.emoe_set_dependent_launch.argtypes = [vp, i32]
         L.emoe_set_fused_projections.argtypes = [vp, i32]
         L.emoe_kernels_last_forward.argtypes = [vp]
+        i64 = ctypes.c_int64
+        L.emoe_cache_create.argtypes = [vp, i32, sz, i32, i32]
+        L.emoe_register_expert.argtypes = [vp, i64, i32, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(sz)]
+        L.emoe_prefetch_experts.argtypes = [vp, ctypes.POINTER(i64), i32, i32, vp]
+        L.emoe_cache_acquire.argtypes = [vp, ctypes.POINTER(i64), i32, i32, vp, vp, ctypes.POINTER(emoe_expert)]
+        L.emoe_cache_release.argtypes = [vp, ctypes.POINTER(i64), i32, vp]
+        L.emoe_cache_slot_of.argtypes = [vp, i64]
+        L.emoe_cache_get_stats.argtypes = [vp, ctypes.POINTER(emoe_cache_stats)]
+        L.emoe_policy_create.restype = vp
+        L.emoe_policy_create.argtypes = [i32, i32, i32]
+        L.emoe_policy_destroy.restype = None
+        L.emoe_policy_destroy.argtypes = [vp]
+        L.emoe_policy_register.argtypes = [vp, i64, i32, i64]
+        L.emoe_policy_prefetch.argtypes = [vp, i64, i32, ctypes.POINTER(i64)]
+        L.emoe_policy_acquire.argtypes = [vp, i64, i32, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(i64)]
+        L.emoe_policy_release.argtypes = [vp, i64]
+        L.emoe_policy_get_stats.argtypes = [vp, ctypes.POINTER(emoe_cache_stats)]
+        L.emoe_rank_experts.argtypes = [ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(ctypes.c_int32), i32,
+                                        ctypes.POINTER(ctypes.c_int32)]
         L.emoe_moe_forward_routed_static.argtypes = [i32, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
                                                      ctypes.POINTER(emoe_expert), vp, vp]
         L.emoe_read_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
@@ -212,3 +245,106 @@ def emoe_set_fused_projections(ctx, enabled: bool) -> None:
 
 def emoe_kernels_last_forward(ctx) -> int:
     return int(lib().emoe_kernels_last_forward(ctx))
+
+
+# ---- expert cache and prefetch ------------------------------------------------------------------
+def _i64_array(ids):
+    arr = (ctypes.c_int64 * len(ids))(*[int(i) for i in ids])
+    return arr
+
+
+def emoe_cache_create(ctx, n_slots: int, slot_bytes: int, n_layers: int, policy: int = EVICT_FORWARD) -> None:
+    _check(lib().emoe_cache_create(ctx, n_slots, slot_bytes, n_layers, policy), "emoe_cache_create")
+
+
+def emoe_register_expert(ctx, expert_id: int, layer: int, bits: int, host_packed, host_scales, nbytes) -> None:
+    """host_packed / host_scales: 3 host addresses each (0 for an absent matrix); nbytes: 6 sizes."""
+    vp = ctypes.c_void_p
+    hp = (vp * 3)(*[vp(int(a)) if a else vp(None) for a in host_packed])
+    hs = (vp * 3)(*[vp(int(a)) if a else vp(None) for a in host_scales])
+    nb = (ctypes.c_size_t * 6)(*[int(b) for b in nbytes])
+    _check(lib().emoe_register_expert(ctx, expert_id, layer, bits, hp, hs, nb), "emoe_register_expert")
+
+
+def emoe_prefetch_experts(ctx, ids, current_layer: int, copy_stream: int) -> None:
+    if len(ids) == 0:
+        return
+    _check(lib().emoe_prefetch_experts(ctx, _i64_array(ids), len(ids), current_layer, copy_stream), "emoe_prefetch_experts")
+
+
+def emoe_cache_acquire(ctx, ids, current_layer: int, compute_stream: int, copy_stream: int):
+    out = (emoe_expert * len(ids))()
+    _check(lib().emoe_cache_acquire(ctx, _i64_array(ids), len(ids), current_layer, compute_stream, copy_stream, out),
+           "emoe_cache_acquire")
+    return out
+
+
+def emoe_cache_release(ctx, ids, compute_stream: int) -> None:
+    _check(lib().emoe_cache_release(ctx, _i64_array(ids), len(ids), compute_stream), "emoe_cache_release")
+
+
+def emoe_cache_slot_of(ctx, expert_id: int) -> int:
+    return int(lib().emoe_cache_slot_of(ctx, expert_id))
+
+
+def emoe_cache_get_stats(ctx) -> dict:
+    st = emoe_cache_stats()
+    _check(lib().emoe_cache_get_stats(ctx, ctypes.byref(st)), "emoe_cache_get_stats")
+    return st.as_dict()
+
+
+def emoe_policy_create(n_slots: int, n_layers: int, policy: int = EVICT_FORWARD):
+    h = lib().emoe_policy_create(n_slots, n_layers, policy)
+    if not h:
+        raise EmoeError(ERR_INVALID_ARG, "emoe_policy_create")
+    return h
+
+
+def emoe_policy_destroy(h) -> None:
+    lib().emoe_policy_destroy(h)
+
+
+def emoe_policy_register(h, expert_id: int, layer: int, nbytes: int = 0) -> None:
+    _check(lib().emoe_policy_register(h, expert_id, layer, nbytes), "emoe_policy_register")
+
+
+def emoe_policy_prefetch(h, expert_id: int, current_layer: int):
+    """-> (slot the load goes to or -1, id that was evicted or -1)"""
+    ev = ctypes.c_int64(-1)
+    s = lib().emoe_policy_prefetch(h, expert_id, current_layer, ctypes.byref(ev))
+    if s == -2:
+        raise EmoeError(ERR_INVALID_ARG, "emoe_policy_prefetch")
+    return int(s), int(ev.value)
+
+
+def emoe_policy_acquire(h, expert_id: int, current_layer: int):
+    """-> (slot or -1 when every slot is protected, loaded now?, id that was evicted or -1)"""
+    ev = ctypes.c_int64(-1)
+    loaded = ctypes.c_int(0)
+    s = lib().emoe_policy_acquire(h, expert_id, current_layer, ctypes.byref(loaded), ctypes.byref(ev))
+    if s == -2:
+        raise EmoeError(ERR_INVALID_ARG, "emoe_policy_acquire")
+    return int(s), bool(loaded.value), int(ev.value)
+
+
+def emoe_policy_release(h, expert_id: int) -> int:
+    return int(lib().emoe_policy_release(h, expert_id))
+
+
+def emoe_policy_get_stats(h) -> dict:
+    st = emoe_cache_stats()
+    _check(lib().emoe_policy_get_stats(h, ctypes.byref(st)), "emoe_policy_get_stats")
+    return st.as_dict()
+
+
+def emoe_rank_experts(prior, prev_ids):
+    import numpy as np
+
+    prior = np.ascontiguousarray(prior, dtype=np.float32)
+    prev = np.ascontiguousarray(prev_ids, dtype=np.int32).reshape(-1)
+    E = prior.shape[0]
+    out = np.empty(E, dtype=np.int32)
+    _check(lib().emoe_rank_experts(prior.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), E,
+                                   prev.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), len(prev),
+                                   out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "emoe_rank_experts")
+    return out

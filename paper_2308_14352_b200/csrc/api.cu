@@ -99,6 +99,10 @@ struct emoe_ctx {
   bool fuse_projections = true;  // weight-streaming kernel: both projections in one launch
   bool timing = false;
   int kernels_last = 0;  // kernels the last forward call enqueued
+  ExpertCache* cache = nullptr;  // expert cache (cache.cu), optional
+  std::vector<cudaEvent_t> table_events;  // per table block: its upload has left the pinned mirror
+  std::vector<uint64_t> table_used;       // per table block: last use (for recycling)
+  uint64_t table_clock = 0;
   std::vector<cudaEvent_t> events;  // triples (start, mid, end) per timed forward call
   size_t events_used = 0;
   std::vector<char> events_one_launch;  // per triple: both projections ran as one launch (no second interval)
@@ -139,13 +143,23 @@ int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaSt
         same = te.host[e].packed[m] == host[e].packed[m] && te.host[e].scales[m] == host[e].scales[m];
     }
     if (same) {
+      ctx->table_used[i] = ++ctx->table_clock;
       *out = reinterpret_cast<const ExpertDev*>(ctx->tables_dev + i * TABLE_BLOCK_BYTES);
       *tmaps = te.has_tmaps ? ctx->tables_dev + i * TABLE_BLOCK_BYTES + TABLE_MAPS_OFFSET : nullptr;
       return EMOE_OK;
     }
   }
-  if (ctx->tables.size() >= MAX_TABLES) return EMOE_ERR_WORKSPACE;
-  const size_t slot = ctx->tables.size();
+  // A new table: the next unused block, or (tables that change from call to call, e.g. pointers
+  // into an expert cache) the block that was used longest ago, once its upload has left the
+  // pinned mirror.  Kernels that read the old device copy were enqueued earlier on the stream.
+  size_t slot = ctx->tables.size();
+  const bool recycle = slot >= MAX_TABLES;
+  if (recycle) {
+    slot = 0;
+    for (size_t i = 1; i < ctx->tables.size(); ++i)
+      if (ctx->table_used[i] < ctx->table_used[slot]) slot = i;
+    EMOE_CUDA(ctx, cudaEventSynchronize(ctx->table_events[slot]));
+  }
   char* pin_block = ctx->tables_pin + slot * TABLE_BLOCK_BYTES;
   ExpertDev* pin = reinterpret_cast<ExpertDev*>(pin_block);
   const int nmat = L.act == EMOE_ACT_RELU ? 2 : 3;
@@ -173,7 +187,17 @@ int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaSt
   te.d_ff = L.d_ff;
   te.act = L.act;
   te.has_tmaps = maps_ok;
-  ctx->tables.push_back(std::move(te));
+  if (recycle) {
+    ctx->tables[slot] = std::move(te);
+  } else {
+    ctx->tables.push_back(std::move(te));
+    cudaEvent_t ev;
+    EMOE_CUDA(ctx, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    ctx->table_events.push_back(ev);
+    ctx->table_used.push_back(0);
+  }
+  EMOE_CUDA(ctx, cudaEventRecord(ctx->table_events[slot], st));
+  ctx->table_used[slot] = ++ctx->table_clock;
   *out = reinterpret_cast<const ExpertDev*>(dev);
   *tmaps = maps_ok ? dev + TABLE_MAPS_OFFSET : nullptr;
   return EMOE_OK;
@@ -360,6 +384,12 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
 
 }  // namespace
 
+namespace emoe {
+ExpertCache*& ctx_cache(emoe_ctx* ctx) { return ctx->cache; }
+int ctx_device(const emoe_ctx* ctx) { return ctx->device; }
+int ctx_cuda_fail(emoe_ctx* ctx, cudaError_t e) { return cuda_fail(ctx, e); }
+}  // namespace emoe
+
 extern "C" {
 
 emoe_ctx* emoe_create(int device, size_t workspace_bytes, int* status) {
@@ -398,6 +428,8 @@ int emoe_destroy(emoe_ctx* ctx) {
   if (ctx->tables_dev) cudaFree(ctx->tables_dev);
   if (ctx->tables_pin) cudaFreeHost(ctx->tables_pin);
   for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
+  for (cudaEvent_t e : ctx->table_events) cudaEventDestroy(e);
+  cache_destroy(ctx->cache);
   delete ctx;
   return EMOE_OK;
 }
@@ -429,6 +461,7 @@ const char* emoe_status_string(int status) {
     case EMOE_ERR_WORKSPACE: return "context workspace (or expert-table cache) too small";
     case EMOE_ERR_CUDA: return "CUDA call failed (see emoe_last_cuda_error)";
     case EMOE_ERR_DEVICE_CHECK: return "a kernel found inconsistent data";
+    case EMOE_ERR_CACHE_FULL: return "every slot of the expert cache is in use";
     default: return "unknown status";
   }
 }

@@ -72,6 +72,10 @@ inline cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block,
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// expert cache of a context (cache.cu)
+struct ExpertCache;
+void cache_destroy(ExpertCache* c);
+
 // ---- launchers (each enqueues on `st` and returns the launch error) ---------------------
 cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int scale_f16, uint8_t* packed,
                         void* scales, cudaStream_t st);

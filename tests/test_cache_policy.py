@@ -1,0 +1,87 @@
+"""The library's cache bookkeeping (emoe_policy_*: the same host code that drives the device
+cache) against the plain model, operation by operation, on random traces: slots, evictions and
+counters are integer work and must agree exactly.  Runs without a GPU."""
+import random
+
+import numpy as np
+import pytest
+
+from oracle.cache_sim import ExpertBufferModel, rank_experts
+from paper_2308_14352_b200 import binding as B
+
+RULES = [("forward", B.EVICT_FORWARD), ("printed", B.EVICT_PRINTED), ("lru", B.EVICT_LRU)]
+
+
+@pytest.mark.parametrize("rule,code", RULES)
+@pytest.mark.parametrize("n_slots,n_layers,per_layer,seed", [(3, 4, 2, 0), (8, 6, 4, 1), (16, 12, 8, 2), (5, 32, 8, 3)])
+def test_random_traces_agree(rule, code, n_slots, n_layers, per_layer, seed):
+    rng = random.Random(seed)
+    model = ExpertBufferModel(n_slots, n_layers, rule)
+    h = B.emoe_policy_create(n_slots, n_layers, code)
+    try:
+        ids = []
+        for layer in range(n_layers):
+            for j in range(per_layer):
+                eid = 1000 * layer + j
+                nbytes = rng.randrange(1, 1 << 20)
+                model.register(eid, layer, nbytes)
+                B.emoe_policy_register(h, eid, layer, nbytes)
+                ids.append(eid)
+        held = []
+        for step in range(3000):
+            layer = step % n_layers
+            op = rng.random()
+            if op < 0.35:
+                eid = rng.choice(ids)
+                s_ref, ev_ref = model.prefetch(eid, layer)
+                s, ev = B.emoe_policy_prefetch(h, eid, layer)
+                assert (s, ev) == (-1 if s_ref is None else s_ref, -1 if ev_ref is None else ev_ref), step
+            elif op < 0.8:
+                eid = rng.choice([e for e in ids if e // 1000 == layer])    # activations come from the current layer
+                s_ref, ld_ref, ev_ref = model.acquire(eid, layer)
+                s, ld, ev = B.emoe_policy_acquire(h, eid, layer)
+                assert (s, ld, ev) == (-1 if s_ref is None else s_ref, ld_ref, -1 if ev_ref is None else ev_ref), step
+                if s_ref is not None:
+                    held.append(eid)
+            elif held:
+                eid = held.pop(rng.randrange(len(held)))
+                assert B.emoe_policy_release(h, eid) == model.release(eid)
+            if len(held) >= n_slots - 1:                                 # keep the trace moving
+                eid = held.pop(0)
+                assert B.emoe_policy_release(h, eid) == model.release(eid)
+            if step % 97 == 0:
+                assert B.emoe_policy_get_stats(h) == model.counters
+        assert B.emoe_policy_get_stats(h) == model.counters
+        assert model.counters["evictions"] > 0
+    finally:
+        B.emoe_policy_destroy(h)
+
+
+def test_policy_argument_errors():
+    with pytest.raises(B.EmoeError):
+        B.emoe_policy_create(0, 4, B.EVICT_FORWARD)
+    with pytest.raises(B.EmoeError):
+        B.emoe_policy_create(4, 4, 17)
+    h = B.emoe_policy_create(2, 4, B.EVICT_LRU)
+    try:
+        B.emoe_policy_register(h, 5, 1, 10)
+        with pytest.raises(B.EmoeError):
+            B.emoe_policy_register(h, 5, 2, 10)       # same id twice
+        with pytest.raises(B.EmoeError):
+            B.emoe_policy_acquire(h, 6, 0)            # unknown id
+        assert B.emoe_policy_release(h, 5) == -1      # not held
+    finally:
+        B.emoe_policy_destroy(h)
+
+
+def test_rank_experts_matches_the_model():
+    rng = np.random.default_rng(3)
+    for E, k in ((8, 2), (8, 1), (32, 4), (5, 5)):
+        prior = rng.random((E, E)).astype(np.float32)
+        prior /= prior.sum(axis=1, keepdims=True)
+        prior[1] = prior[0]                                   # equal rows: ties within a sum stay possible
+        prior[:, 3] = prior[:, 2]                             # equal columns: exact ties between experts 2 and 3
+        for _ in range(20):
+            prev = rng.integers(0, E, size=k)
+            got = B.emoe_rank_experts(prior, prev)
+            assert got.tolist() == rank_experts(prior.tolist(), prev.tolist())

@@ -1,0 +1,141 @@
+"""Pins of the expert-buffer model (oracle/cache_sim.py) against things that are not itself:
+hand-worked scores of the eviction formula (Section 3.3), a textbook LRU, closed-form special
+cases, and brute force over tiny traces."""
+import itertools
+import random
+from collections import OrderedDict
+
+import pytest
+
+from oracle.cache_sim import ExpertBufferModel, rank_experts
+
+
+def _fill(m, ids, layer_fn, acquires):
+    for e in ids:
+        m.register(e, layer_fn(e), 100)
+    for e, n in acquires:
+        for _ in range(n):
+            s, _, _ = m.acquire(e, 0)
+            assert s is not None
+            m.release(e)
+
+
+def test_hand_worked_scores_forward_reading():
+    # S = 12 layers, current layer I = 3.  Experts: id = 10*layer + j.
+    # e41 (layer 4, f=2): D = 1,  L = -2        e21 (layer 2, f=2): D = 11, L = -2/11
+    # e91 (layer 9, f=6): D = 6,  L = -1        e31 (layer 3, f=0): D = 0, protected
+    # highest L leaves first: e21 (-0.18), then e91 (-1), then e41 (-2), last the protected e31
+    m = ExpertBufferModel(4, 12, "forward")
+    _fill(m, [41, 21, 91, 31], lambda e: e // 10, [(41, 2), (21, 2), (91, 6)])
+    m.prefetch(31, 0)
+    order = [m.slot_content[s] for s in m.eviction_order(3)]
+    assert order == [21, 91, 41, 31]
+
+
+def test_hand_worked_scores_printed_reading():
+    # same buffer, printed distance (S - i + I) mod S at I = 3:
+    # e41: D = 11, L = -2/11   e21: D = 1, L = -2   e91: D = 6, L = -1   e31: D = 0 protected
+    m = ExpertBufferModel(4, 12, "printed")
+    _fill(m, [41, 21, 91, 31], lambda e: e // 10, [(41, 2), (21, 2), (91, 6)])
+    m.prefetch(31, 0)
+    order = [m.slot_content[s] for s in m.eviction_order(3)]
+    assert order == [41, 91, 21, 31]
+
+
+def test_never_used_experts_leave_first_and_ties_go_to_the_lowest_slot():
+    m = ExpertBufferModel(3, 8, "forward")
+    for e, layer in ((1, 5), (2, 6), (3, 7)):
+        m.register(e, layer)
+        m.prefetch(e, 0)                   # f = 0 for all: L = 0 for all, a three-way tie
+    assert m.eviction_order(0) == [0, 1, 2]
+    m.register(4, 1)
+    s, ev = m.prefetch(4, 0)
+    assert (s, ev) == (0, 1)
+
+
+def test_lru_rule_is_textbook_lru():
+    rng = random.Random(5)
+    m = ExpertBufferModel(4, 6, "lru")
+    for e in range(12):
+        m.register(e, e % 6)
+    book = OrderedDict()
+    for step in range(400):
+        e = rng.randrange(12)
+        s, loaded, ev = m.acquire(e, step % 6)
+        m.release(e)
+        if e in book:
+            assert not loaded and ev is None
+            book.move_to_end(e)
+        else:
+            assert loaded
+            if len(book) == 4:
+                oldest, _ = book.popitem(last=False)
+                assert ev == oldest
+            else:
+                assert ev is None
+            book[e] = True
+    assert set(m.where) == set(book)
+    assert m.counters["hits"] + m.counters["misses"] == 400
+
+
+@pytest.mark.parametrize("rule", ["forward", "printed", "lru"])
+def test_no_eviction_when_everything_fits_and_counters_add_up(rule):
+    rng = random.Random(7)
+    m = ExpertBufferModel(16, 4, rule)
+    for e in range(16):
+        m.register(e, e % 4, 10 + e)
+    for step in range(200):
+        e = rng.randrange(16)
+        if rng.random() < 0.3:
+            m.prefetch(e, step % 4)
+        else:
+            assert m.acquire(e, step % 4)[0] is not None
+            m.release(e)
+    c = m.counters
+    assert c["evictions"] == 0
+    assert c["misses"] + c["prefetched"] == len(m.where)             # every expert was loaded exactly once
+    assert c["bytes_copied"] == sum(10 + e for e in m.where)
+    assert c["prefetch_hits"] <= c["prefetched"]
+
+
+def test_experts_in_use_are_never_evicted_and_a_full_buffer_refuses():
+    m = ExpertBufferModel(2, 4, "forward")
+    for e in range(4):
+        m.register(e, e)
+    assert m.acquire(0, 0)[0] == 0 and m.acquire(1, 0)[0] == 1      # both slots in use
+    assert m.prefetch(2, 0) == (None, None) and m.counters["prefetch_refused"] == 1
+    assert m.acquire(3, 0) == (None, False, None)
+    m.release(1)
+    s, loaded, ev = m.acquire(3, 0)
+    assert (s, loaded, ev) == (1, True, 1)
+
+
+def test_victim_maximises_the_score_brute_force():
+    """For every small configuration: the evicted expert has the highest L = -f/D among the
+    candidates with D > 0 (computed here directly from the formula with floats)."""
+    for layers, freqs, current in itertools.product(itertools.permutations(range(1, 5), 3), [(0, 1, 5), (3, 3, 1), (2, 7, 4)], range(5)):
+        m = ExpertBufferModel(3, 5, "forward")
+        for j, (layer, f) in enumerate(zip(layers, freqs)):
+            m.register(j, layer)
+            m.prefetch(j, 0)
+            for _ in range(f):
+                m.acquire(j, 0)
+                m.release(j)
+        m.register(99, 0)
+        s, ev = m.prefetch(99, current)
+        scores = {}
+        for j, (layer, f) in enumerate(zip(layers, freqs)):
+            D = (layer - current) % 5
+            if D:
+                scores[j] = -f / D
+        if scores:
+            best = max(scores.values())
+            assert scores[ev] == pytest.approx(best)
+            assert ev == min(j for j, v in scores.items() if v == pytest.approx(best))
+
+
+def test_rank_experts():
+    prior = [[0.7, 0.2, 0.1], [0.1, 0.1, 0.8], [0.3, 0.3, 0.4]]
+    assert rank_experts(prior, [0]) == [0, 1, 2]
+    assert rank_experts(prior, [1]) == [2, 0, 1]            # tie between 0 and 1: lower index first
+    assert rank_experts(prior, [0, 1]) == [2, 0, 1]         # sums 0.8, 0.3, 0.9
