@@ -17,7 +17,9 @@ Readings where the paper is silent or at odds with itself (all listed in DESIGN.
   soon" kept, which is (i - I) mod S.  Both exist: `forward` (default) and `printed`.
 * D = 0 (an expert of the current layer): the formula divides by zero; such experts are
   protected and leave only when no other candidate exists (then lowest f first).
-* f: running count of activations (acquire calls) of that expert.
+* f: the paper's f comes from an offline profile; there is none here, so f = 1 + the running
+  count of activations (acquire calls) of that expert: a preloaded expert that has not been used
+  yet is then ranked by its layer distance instead of leaving first with L = 0.
 * ties: the lowest slot index leaves.
 * an expert in use (acquired, not released) is never evicted; a preload that finds no
   candidate is dropped; an activation that finds none is an error.
@@ -62,7 +64,7 @@ class ExpertBufferModel:
             D = self.distance(eid, current_layer)
             if D == 0:                      # protected: after everybody else, lowest count first
                 return (1, Fraction(self.freq[eid]), s)
-            return (0, Fraction(self.freq[eid], D), s)   # highest L = -f/D first  <=>  smallest f/D first
+            return (0, Fraction(self.freq[eid] + 1, D), s)   # highest L = -f/D first  <=>  smallest f/D first
         return sorted(cands, key=key)
 
     def _put(self, eid, current_layer):

@@ -59,9 +59,12 @@ class CachePolicy {
   emoe_cache_stats& stats() { return stats_; }
 
   // Eviction order (Section 3.3, "Cache eviction policy"): the expert with the highest score
-  // L = -f / D leaves first, f its activation count, D the distance of its layer from the
-  // current one.  EMOE_EVICT_FORWARD takes D as the number of layers until the expert's layer runs
-  // again, (i - I) mod S, which is what the text asks for (layers about to run are kept);
+  // L = -f / D leaves first, f its activation frequency, D the distance of its layer from the
+  // current one.  The paper takes f from an offline profile; here it is the running activation
+  // count plus one, so that an expert that was preloaded but not used yet (count 0) is still
+  // ranked by its layer distance instead of being the first to go.  EMOE_EVICT_FORWARD takes D as
+  // the number of layers until the expert's layer runs again, (i - I) mod S, which is what the
+  // text asks for (layers about to run are kept);
   // EMOE_EVICT_PRINTED takes the printed (S - i + I) mod S.  D = 0 (the current layer) is
   // protected: such an expert goes only when nothing else can.  EMOE_EVICT_LRU: least recently
   // touched first.  Ties: lowest slot.
@@ -75,8 +78,8 @@ class CachePolicy {
     const int da = distance(a.layer, current_layer), db = distance(b.layer, current_layer);
     if ((da == 0) != (db == 0)) return db == 0;  // the unprotected one
     if (da == 0) return a.freq != b.freq ? a.freq < b.freq : sa < sb;
-    // -fa/da > -fb/db  <=>  fa * db < fb * da   (exact in integers)
-    const int64_t lhs = a.freq * db, rhs = b.freq * da;
+    // -fa/da > -fb/db  <=>  fa * db < fb * da   (exact in integers), f = count + 1
+    const int64_t lhs = (a.freq + 1) * db, rhs = (b.freq + 1) * da;
     return lhs != rhs ? lhs < rhs : sa < sb;
   }
   int distance(int layer, int current_layer) const {

@@ -22,9 +22,10 @@ def _fill(m, ids, layer_fn, acquires):
 
 def test_hand_worked_scores_forward_reading():
     # S = 12 layers, current layer I = 3.  Experts: id = 10*layer + j.
-    # e41 (layer 4, f=2): D = 1,  L = -2        e21 (layer 2, f=2): D = 11, L = -2/11
-    # e91 (layer 9, f=6): D = 6,  L = -1        e31 (layer 3, f=0): D = 0, protected
-    # highest L leaves first: e21 (-0.18), then e91 (-1), then e41 (-2), last the protected e31
+    # f = activations + 1.
+    # e41 (layer 4, 2 activations): D = 1,  L = -3        e21 (layer 2, 2): D = 11, L = -3/11
+    # e91 (layer 9, 6 activations): D = 6,  L = -7/6      e31 (layer 3, 0): D = 0, protected
+    # highest L leaves first: e21 (-0.27), then e91 (-1.17), then e41 (-3), last the protected e31
     m = ExpertBufferModel(4, 12, "forward")
     _fill(m, [41, 21, 91, 31], lambda e: e // 10, [(41, 2), (21, 2), (91, 6)])
     m.prefetch(31, 0)
@@ -34,7 +35,7 @@ def test_hand_worked_scores_forward_reading():
 
 def test_hand_worked_scores_printed_reading():
     # same buffer, printed distance (S - i + I) mod S at I = 3:
-    # e41: D = 11, L = -2/11   e21: D = 1, L = -2   e91: D = 6, L = -1   e31: D = 0 protected
+    # e41: D = 11, L = -3/11   e21: D = 1, L = -3   e91: D = 6, L = -7/6   e31: D = 0 protected
     m = ExpertBufferModel(4, 12, "printed")
     _fill(m, [41, 21, 91, 31], lambda e: e // 10, [(41, 2), (21, 2), (91, 6)])
     m.prefetch(31, 0)
@@ -42,15 +43,20 @@ def test_hand_worked_scores_printed_reading():
     assert order == [41, 91, 21, 31]
 
 
-def test_never_used_experts_leave_first_and_ties_go_to_the_lowest_slot():
+def test_unused_preloads_rank_by_distance_and_ties_go_to_the_lowest_slot():
     m = ExpertBufferModel(3, 8, "forward")
     for e, layer in ((1, 5), (2, 6), (3, 7)):
         m.register(e, layer)
-        m.prefetch(e, 0)                   # f = 0 for all: L = 0 for all, a three-way tie
-    assert m.eviction_order(0) == [0, 1, 2]
+        m.prefetch(e, 0)                   # never activated: L = -1/5, -1/6, -1/7: the farthest layer leaves first
+    assert m.eviction_order(0) == [2, 1, 0]
     m.register(4, 1)
     s, ev = m.prefetch(4, 0)
-    assert (s, ev) == (0, 1)
+    assert (s, ev) == (2, 3)
+    t = ExpertBufferModel(3, 8, "forward")
+    for e in (1, 2, 3):
+        t.register(e, 5)
+        t.prefetch(e, 0)                   # same layer, same count: a three-way tie
+    assert t.eviction_order(0) == [0, 1, 2]
 
 
 def test_lru_rule_is_textbook_lru():
@@ -127,7 +133,7 @@ def test_victim_maximises_the_score_brute_force():
         for j, (layer, f) in enumerate(zip(layers, freqs)):
             D = (layer - current) % 5
             if D:
-                scores[j] = -f / D
+                scores[j] = -(f + 1) / D
         if scores:
             best = max(scores.values())
             assert scores[ev] == pytest.approx(best)
