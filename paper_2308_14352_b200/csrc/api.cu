@@ -276,7 +276,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
   const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
   // many tokens per expert: the tcgen05 grouped GEMM; otherwise the weight-streaming kernels
-  const bool many_tokens = ffn_token_tiles(L, T) >= 4;
+  const bool many_tokens = ffn_many_tokens(L, T);
   // skewed loads: experts with few tokens stream through the TMA kernel, the others take the
   // tcgen05 grouped GEMM, in the same forward call
   const bool use_hybrid = can_umma && can_tma && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens));
@@ -301,15 +301,14 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     ctx->events_used += 3;
   }
   if (use_hybrid) {
-    // experts with up to HYBRID_STREAM_TOKENS tokens: one or two passes of 16-token tiles through the
-    // streaming kernel (measured best on a Zipf(1.1) load over 128 experts: 16 .. 128 tokens all within
-    // 10 %); the others: 128-token tiles on tcgen05.  Each family has its own plan and writes only
+    // experts with up to HYBRID_STREAM_TOKENS tokens: passes of 8-token tiles through the streaming
+    // kernel; the others: 128-token tiles on tcgen05.  Each family has its own plan and writes only
     // its own slots of xs / hidden / o_part.
 #ifndef EMOE_HYBRID_TOKENS
 #define EMOE_HYBRID_TOKENS 32
 #endif
 #ifndef EMOE_HYBRID_TILES
-#define EMOE_HYBRID_TILES 2
+#define EMOE_HYBRID_TILES 1
 #endif
     constexpr int HYBRID_STREAM_TOKENS = EMOE_HYBRID_TOKENS;
     int* plan_heavy = reinterpret_cast<int*>(reinterpret_cast<char*>(plan) + align_up(plan_bytes(L.E)));

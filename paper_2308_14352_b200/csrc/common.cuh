@@ -101,6 +101,7 @@ cudaError_t launch_ffn_gemv(int phase, const LayerDims& L, const ExpertDev* expe
 bool ffn_mma_supported(const LayerDims& L);
 int ffn_mma_ksplit(const LayerDims& L, int T);
 int ffn_token_tiles(const LayerDims& L, int T);
+bool ffn_many_tokens(const LayerDims& L, int T);
 // plan (nullable): plan_bytes(E) bytes, the work plan for the persistent TMA kernels, filled by block 0.
 // to_f16: store the rows as fp16 (saturating) instead of bf16, same layout (the TMA-staged kernel's input).
 // cnt_lo .. cnt_hi: only experts with that many tokens are listed in the plan and have their rows

@@ -281,16 +281,19 @@ __global__ void __launch_bounds__(128)
 
 }  // namespace
 
-// 8-token tiles a CTA handles per pass over its weights: enough for the mean tokens per expert
-// plus 2.5 standard deviations under uniform routing (a token picks an expert with probability
-// top_k / E); an expert with more tokens takes another pass over its own weights.
+// 8-token tiles a CTA handles per pass over its weights.  A pass with one tile is the cheapest
+// per byte by far (measured on the streaming kernel: 1 : 1.6 for one against two tiles), and an
+// expert with more tokens simply takes another pass over its own weights (from L2), so one tile
+// wins as long as the mean tokens per expert under uniform routing stay below about 12 (expected
+// passes below 1.6); beyond that two tiles.  Four tiles only on request.
 int ffn_token_tiles(const LayerDims& L, int T) {
-  const double p = static_cast<double>(L.top_k) / L.E;
-  const double mean = T * p;
-  double need = mean + 2.5 * sqrt(T * p * (1.0 - p));
-  if (need > T) need = T;
-  return need <= 8.0 ? 1 : (need <= 16.0 ? 2 : 4);
+  const double mean = static_cast<double>(T) * L.top_k / L.E;
+  return mean <= 12.0 ? 1 : 2;
 }
+
+// Enough tokens per expert (mean of 16 under uniform routing) that the experts with many tokens
+// are a dense contraction: those go to the tcgen05 grouped GEMM.
+bool ffn_many_tokens(const LayerDims& L, int T) { return static_cast<double>(T) * L.top_k / L.E >= 16.0; }
 
 bool ffn_mma_supported(const LayerDims& L) {
   if (!L.act_bf16) return false;
