@@ -3,10 +3,13 @@
 // an independent FFN) on the Section 3.2 storage (b-bit codes + scale channel, w~ = q * s).
 //
 // Shape of one tile: 128 output channels (UMMA M, "swap-AB": the weight rows are the M side)
-// x 128 tokens of one expert (UMMA N) x all inputs, accumulated in tensor memory.
+// x a group of up to three 128-token tiles of one expert (UMMA N = 128 each, one accumulator in
+// tensor memory per token tile; two token tiles with two accumulators each for a gated first
+// projection) x all inputs.  The dequantised A stage, the expensive part, is shared by the whole
+// group: up to 384 tokens per dequantisation.
 //   warp 0    TMA producer: packed code boxes (128 rows x 128 bytes, the decode kernel's tensor
-//             maps) into a 2-deep raw ring, and the tokens' activations (128 tokens x 64 inputs,
-//             fp16, K-major, 128-byte swizzle) into a 3-deep operand ring;
+//             maps) into a 2-deep raw ring, and the tokens' activations (one box of 128 tokens x
+//             64 inputs per token tile, fp16, K-major, 128-byte swizzle) into a 2- or 3-deep operand ring;
 //   warps 2-9 two threads per output channel: read the channel's packed bytes from the raw ring,
 //             dequantise to fp16 (code -> exact fp16 integer by mantissa insertion, then one
 //             multiply by the group scale: |error| <= 2^-12 relative, the only approximation of
@@ -14,7 +17,7 @@
 //             swizzled layout; later the epilogue: tensor memory -> registers -> activation ->
 //             global memory;
 //   warp 1    one thread issues tcgen05.mma (M128 N128 K16, fp16 x fp16 -> fp32 in TMEM) per 16
-//             inputs and commits each stage back to the producers.
+//             inputs and token tile and commits each stage back to the producers.
 // SwiGLU's first projection runs two accumulators (w1 and w3 rows of the same 128 channels
 // against the same activation tile), so that silu(a) * b needs no exchange between warps.
 // Activations travel as fp16 (exact for bf16 values inside the fp16 range, saturated outside);
@@ -34,19 +37,29 @@ namespace {
 constexpr int UM_TOK = 128;                // tokens per tile (UMMA N)
 constexpr int UM_ROWS = 128;               // output channels per tile (UMMA M)
 constexpr int UM_BK = 64;                  // inputs per operand stage: one 128-byte row of fp16
-constexpr int UM_AB_STAGES = 3;
+constexpr int UM_AB_STAGES_MAX = 3;
 constexpr int UM_RAW_STAGES = 2;
 constexpr int UM_TILE_BYTES = 128 * 128;   // a [128][64] fp16 operand tile, or a [128 rows][128 B] packed tile
-constexpr int UM_AB_STAGE_BYTES = 3 * UM_TILE_BYTES;   // A (first matrix), A (second matrix), B
-constexpr int UM_RAW_STAGE_BYTES = 2 * UM_TILE_BYTES;  // packed tiles of up to two matrices
-constexpr int UM_SMEM_BYTES = UM_RAW_STAGES * UM_RAW_STAGE_BYTES + UM_AB_STAGES * UM_AB_STAGE_BYTES + 1024;
+// One dequantised A stage is multiplied with a group of token tiles (each its own accumulator in
+// tensor memory), so that the dequantisation, the slowest step, is shared by up to 384 tokens
+// (256 with the two accumulators per token tile of a gated first projection).  Shared memory
+// decides the shapes: an operand stage holds the A tiles (1 or 2 matrices) and the group's B
+// tiles, a raw stage the packed tiles of 1 or 2 matrices.
+//   one matrix:   group 3, 3 operand stages of 4 tiles + 2 raw stages of 1 tile = 224 KB
+//   two matrices: group 2, 2 operand stages of 4 tiles + 2 raw stages of 2 tiles = 192 KB
+constexpr int UM_GROUP_SINGLE = 3;
+constexpr int UM_GROUP_DUAL = 2;
+constexpr int UM_STAGES_SINGLE = 3;
+constexpr int UM_STAGES_DUAL = 2;
+constexpr int UM_AB_STAGE_BYTES = 4 * UM_TILE_BYTES;
+constexpr int UM_SMEM_BYTES = 14 * UM_TILE_BYTES + 1024;
 #ifndef EMOE_UM_UNPACK_WARPS
 #define EMOE_UM_UNPACK_WARPS 8
 #endif
 constexpr int UM_UNPACK_WARPS = EMOE_UM_UNPACK_WARPS;  // 8 or 16: two or four threads per output channel
 constexpr int UM_PARTS = UM_UNPACK_WARPS / 4;            // each dequantises its share of a stage and reads its share of the columns
 constexpr int UM_THREADS = (2 + UM_UNPACK_WARPS) * 32;
-constexpr int UM_TMEM_COLS = 256;
+constexpr int UM_TMEM_COLS = 512;
 
 // position of input k in the activation buffers of this path: the unpack emits the code pairs
 // (c, c+4) of an 8-code word at 4 bits and (c, c+8) of a 16-code word at 2 bits
@@ -146,29 +159,41 @@ struct UmmaArgs {
 };
 
 // the tiles of this CTA: linear index = blockIdx.x, += gridDim.x over
-// (activated expert, token tile, row block) with the row block running fastest
+// (activated expert, group of `group` token tiles, row block) with the row block running fastest
 struct TileWalk {
   const PlanRec* recs;
-  int n_active, row_blocks, lin, a, base;
+  int n_active, row_blocks, lin, a, base, group;
   PlanRec rec;
   int tiles_of_a;
-  __device__ __forceinline__ void init(const int* plan, int rb) {
+  __device__ __forceinline__ void init(const int* plan, int rb, int token_tiles_per_group) {
     n_active = *reinterpret_cast<const volatile int*>(plan);
     recs = reinterpret_cast<const PlanRec*>(reinterpret_cast<const char*>(plan) + PLAN_HEADER_BYTES);
     row_blocks = rb;
+    // Grouping token tiles shares the dequantisation but makes fewer, longer work units: take the
+    // largest group (up to the limit) that still leaves every CTA of the grid a unit.  Every
+    // thread that walks the tiles computes the same answer from the plan.
+    group = 1;
+    for (int g = token_tiles_per_group; g > 1; --g) {
+      long long units = 0;
+      for (int i = 0; i < n_active; ++i) units += (recs[i].cnt + g * UM_TOK - 1) / (g * UM_TOK);
+      if (units * rb >= static_cast<long long>(gridDim.x)) {
+        group = g;
+        break;
+      }
+    }
     lin = blockIdx.x;
     a = -1;
     base = 0;
     tiles_of_a = 0;
   }
-  // advances to the CTA's next tile; false when there is none
+  // advances to the CTA's next tile (tt = index of its token group); false when there is none
   __device__ __forceinline__ bool next(int& tt, int& rb) {
     while (a < 0 || lin >= base + tiles_of_a) {
       base += tiles_of_a;
       ++a;
       if (a >= n_active) return false;
       rec = recs[a];
-      tiles_of_a = row_blocks * ((rec.cnt + UM_TOK - 1) / UM_TOK);
+      tiles_of_a = row_blocks * ((rec.cnt + group * UM_TOK - 1) / (group * UM_TOK));
     }
     const int local = lin - base;
     tt = local / row_blocks;
@@ -210,21 +235,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __global__ void __launch_bounds__(UM_THREADS, 1)
     ffn_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_b) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * UM_RAW_STAGES + 3 * UM_AB_STAGES + 2];
+  __shared__ __align__(8) uint64_t bars[2 * UM_RAW_STAGES + 3 * UM_AB_STAGES_MAX + 2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* raw_ring = smem;
-  unsigned char* ab_ring = smem + UM_RAW_STAGES * UM_RAW_STAGE_BYTES;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   const uint32_t bar_raw_full = smem_u32(bars);
   const uint32_t bar_raw_empty = smem_u32(bars + UM_RAW_STAGES);
   const uint32_t bar_b_full = smem_u32(bars + 2 * UM_RAW_STAGES);
-  const uint32_t bar_a_full = smem_u32(bars + 2 * UM_RAW_STAGES + UM_AB_STAGES);
-  const uint32_t bar_ab_empty = smem_u32(bars + 2 * UM_RAW_STAGES + 2 * UM_AB_STAGES);
-  const uint32_t bar_acc_full = smem_u32(bars + 2 * UM_RAW_STAGES + 3 * UM_AB_STAGES);
+  const uint32_t bar_a_full = smem_u32(bars + 2 * UM_RAW_STAGES + UM_AB_STAGES_MAX);
+  const uint32_t bar_ab_empty = smem_u32(bars + 2 * UM_RAW_STAGES + 2 * UM_AB_STAGES_MAX);
+  const uint32_t bar_acc_full = smem_u32(bars + 2 * UM_RAW_STAGES + 3 * UM_AB_STAGES_MAX);
   const uint32_t bar_acc_empty = bar_acc_full + 8;
 
   if (threadIdx.x == 0) {
@@ -233,7 +257,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       mbar_init(bar_raw_full + 8 * s, 1);
       mbar_init(bar_raw_empty + 8 * s, UM_UNPACK_WARPS);
     }
-    for (int s = 0; s < UM_AB_STAGES; ++s) {
+    for (int s = 0; s < UM_AB_STAGES_MAX; ++s) {
       mbar_init(bar_b_full + 8 * s, 1);
       mbar_init(bar_a_full + 8 * s, UM_UNPACK_WARPS);
       mbar_init(bar_ab_empty + 8 * s, 1);
@@ -264,8 +288,14 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
   const int row_blocks = (N + UM_ROWS - 1) / UM_ROWS;
   const int kb_total = K / UM_BK;
 
+  const int group_max = dual ? UM_GROUP_DUAL : UM_GROUP_SINGLE;  // token tiles that may share one dequantised A stage
+  const int ab_stages = dual ? UM_STAGES_DUAL : UM_STAGES_SINGLE;
+  const int raw_stage_bytes = n_mats * UM_TILE_BYTES;
+  unsigned char* ab_ring = smem + UM_RAW_STAGES * raw_stage_bytes;
+  const int b_off = n_mats * UM_TILE_BYTES;                   // B tiles follow the A tiles inside an operand stage
   TileWalk walk;
-  walk.init(a.plan, row_blocks);
+  walk.init(a.plan, row_blocks, group_max);
+  const int group = walk.group;
   int tt, rb;
 
   if (warp == 0) {
@@ -278,7 +308,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
         const CUtensorMap* maps = a.wmaps + static_cast<size_t>(rec.e) * 3;
         const int kbs = (1024 / rec.bits) / UM_BK;  // operand stages per packed box (128 bytes of a row)
         const int row0 = rb * UM_ROWS;
-        const int tok0 = rec.begin + tt * UM_TOK;
+        const int tok0 = rec.begin + tt * group * UM_TOK;
+        const int ntt = min(group, (rec.cnt - tt * group * UM_TOK + UM_TOK - 1) / UM_TOK);  // token tiles of this group
         for (int kb = 0; kb < kb_total && ok;) {
           const int rs = raw_it % UM_RAW_STAGES;
           if (!mbar_wait(bar_raw_empty + 8 * rs, ((raw_it / UM_RAW_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
@@ -289,21 +320,23 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
           mbar_expect_tx(rfull, n_mats * UM_TILE_BYTES);
           const int c0 = (kb / kbs) * 128;
           for (int m = 0; m < n_mats; ++m) {
-            const uint32_t dst = smem_u32(raw_ring + rs * UM_RAW_STAGE_BYTES + m * UM_TILE_BYTES);
+            const uint32_t dst = smem_u32(raw_ring + rs * raw_stage_bytes + m * UM_TILE_BYTES);
             const CUtensorMap* mp = maps + (dual ? m : mat_first);
             tma_load_2d(dst, mp, c0, row0, rfull);
             tma_load_2d(dst + UM_TILE_BYTES / 2, mp, c0, row0 + 64, rfull);
           }
           ++raw_it;
           for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb) {
-            const int s = ab_it % UM_AB_STAGES;
-            if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_AB_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
+            const int s = ab_it % ab_stages;
+            if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / ab_stages) & 1) ^ 1, a.check_word, abort_flag)) {
               ok = false;
               break;
             }
             const uint32_t bfull = bar_b_full + 8 * s;
-            mbar_expect_tx(bfull, UM_TILE_BYTES);
-            tma_load_2d(smem_u32(ab_ring + s * UM_AB_STAGE_BYTES + 2 * UM_TILE_BYTES), &tmap_b, kb * UM_BK, tok0, bfull);
+            mbar_expect_tx(bfull, ntt * UM_TILE_BYTES);
+            for (int j = 0; j < ntt; ++j)
+              tma_load_2d(smem_u32(ab_ring + s * UM_AB_STAGE_BYTES + b_off + j * UM_TILE_BYTES), &tmap_b, kb * UM_BK,
+                          tok0 + j * UM_TOK, bfull);
             ++ab_it;
           }
         }
@@ -317,11 +350,12 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       int ab_it = 0, tile_it = 0;
       bool ok = true;
       while (ok && walk.next(tt, rb)) {
+        const int ntt = min(group, (walk.rec.cnt - tt * group * UM_TOK + UM_TOK - 1) / UM_TOK);
         if (!mbar_wait(bar_acc_empty, ((tile_it & 1) ^ 1), a.check_word, abort_flag)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         for (int kb = 0; kb < kb_total; ++kb, ++ab_it) {
-          const int s = ab_it % UM_AB_STAGES;
-          const uint32_t par = (ab_it / UM_AB_STAGES) & 1;
+          const int s = ab_it % ab_stages;
+          const uint32_t par = (ab_it / ab_stages) & 1;
           if (!mbar_wait(bar_a_full + 8 * s, par, a.check_word, abort_flag) ||
               !mbar_wait(bar_b_full + 8 * s, par, a.check_word, abort_flag)) {
             ok = false;
@@ -329,12 +363,17 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
           }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t st = smem_u32(ab_ring + s * UM_AB_STAGE_BYTES);
-          const uint64_t da0 = umma_desc(st), da1 = umma_desc(st + UM_TILE_BYTES), db = umma_desc(st + 2 * UM_TILE_BYTES);
+          const uint64_t da0 = umma_desc(st), da1 = umma_desc(st + UM_TILE_BYTES);
+          // accumulator of token tile j: columns j*128 (one matrix) or j*256 and j*256 + 128 (two)
+          for (int j = 0; j < ntt; ++j) {
+            const uint64_t db = umma_desc(st + b_off + j * UM_TILE_BYTES);
+            const uint32_t acc_col = tmem_base + j * n_mats * UM_TOK;
 #pragma unroll
-          for (int k4 = 0; k4 < UM_BK / 16; ++k4) {  // 16 inputs = 32 bytes = 2 descriptor units per step
-            const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
-            umma_f16(tmem_base, da0 + 2 * k4, db + 2 * k4, idesc, acc);
-            if (dual) umma_f16(tmem_base + UM_TOK, da1 + 2 * k4, db + 2 * k4, idesc, acc);
+            for (int k4 = 0; k4 < UM_BK / 16; ++k4) {  // 16 inputs = 32 bytes = 2 descriptor units per step
+              const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
+              umma_f16(acc_col, da0 + 2 * k4, db + 2 * k4, idesc, acc);
+              if (dual) umma_f16(acc_col + UM_TOK, da1 + 2 * k4, db + 2 * k4, idesc, acc);
+            }
           }
           umma_commit(bar_ab_empty + 8 * s);  // the stage may be refilled once these MMAs have read it
         }
@@ -369,8 +408,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
           break;
         }
         for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb, ++ab_it) {
-          const int s = ab_it % UM_AB_STAGES;
-          if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_AB_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
+          const int s = ab_it % ab_stages;
+          if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / ab_stages) & 1) ^ 1, a.check_word, abort_flag)) {
             ok = false;
             break;
           }
@@ -379,7 +418,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
           for (int m = 0; m < n_mats; ++m) {
             const __half sh = __float2half_rn(sv[m]);
             const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
-            const unsigned char* rrow = raw_ring + rs * UM_RAW_STAGE_BYTES + m * UM_TILE_BYTES + box * (UM_TILE_BYTES / 2) + rin * 128;
+            const unsigned char* rrow = raw_ring + rs * raw_stage_bytes + m * UM_TILE_BYTES + box * (UM_TILE_BYTES / 2) + rin * 128;
             unsigned char* arow = ab_ring + s * UM_AB_STAGE_BYTES + m * UM_TILE_BYTES + r * 128;
 #pragma unroll
             for (int pp = part * (4 / UM_PARTS); pp < (part + 1) * (4 / UM_PARTS); ++pp) {
@@ -404,13 +443,18 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       if (!mbar_wait(bar_acc_full, tile_it & 1, a.check_word, abort_flag)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int nrow = rb * UM_ROWS + r;
-      const int tokens = min(UM_TOK, rec.cnt - tt * UM_TOK);
-      const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tt) * UM_TOK;
+      const int tok_first = tt * group * UM_TOK;
+      const int ntt = min(group, (rec.cnt - tok_first + UM_TOK - 1) / UM_TOK);
       const int hpos = a.phase == 0 ? pair_pos_rt(bits, min(nrow, N - 1)) : 0;
 #pragma unroll 1
-      for (int cc = (UM_TOK / UM_PARTS) * part; cc < (UM_TOK / UM_PARTS) * (part + 1); cc += 32) {
+      for (int jc = 0; jc < ntt * (UM_TOK / UM_PARTS / 32); ++jc) {
+        // token tile j of the group, 32 columns from cc on (this warp's share of the tile's columns)
+        const int j = jc / (UM_TOK / UM_PARTS / 32);
+        const int cc = (UM_TOK / UM_PARTS) * part + 32 * (jc % (UM_TOK / UM_PARTS / 32));
+        const int tokens = min(UM_TOK, rec.cnt - tok_first - j * UM_TOK);
+        const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tok_first) + static_cast<size_t>(j) * UM_TOK;
         uint32_t va[32], vb[32];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + cc;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + j * n_mats * UM_TOK + cc;
         tmem_ld32(taddr, va);
         if (dual) tmem_ld32(taddr + UM_TOK, vb);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
