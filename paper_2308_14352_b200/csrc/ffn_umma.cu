@@ -347,6 +347,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
     if (lane == 0) {
       // kind::f16, fp16 x fp16 -> fp32, both operands K-major, M = 128, N = 128
       const uint32_t idesc = (1u << 4) | ((UM_TOK >> 3) << 17) | ((UM_ROWS >> 4) << 24);
+      // two neighbouring token tiles as one N = 256 MMA: the A tile is read from shared memory once
+      // for both (at N = 128 the operand reads alone take the whole shared-memory bandwidth)
+      const uint32_t idesc2 = (1u << 4) | (((2 * UM_TOK) >> 3) << 17) | ((UM_ROWS >> 4) << 24);
       int ab_it = 0, tile_it = 0;
       bool ok = true;
       while (ok && walk.next(tt, rb)) {
@@ -364,15 +367,18 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t st = smem_u32(ab_ring + s * UM_AB_STAGE_BYTES);
           const uint64_t da0 = umma_desc(st), da1 = umma_desc(st + UM_TILE_BYTES);
-          // accumulator of token tile j: columns j*128 (one matrix) or j*256 and j*256 + 128 (two)
-          for (int j = 0; j < ntt; ++j) {
+          // accumulator of token tile j of matrix m: columns (m * group + j) * 128; the B tiles of a
+          // group lie back to back, so tiles j and j+1 form one 256-token operand
+          for (int j = 0; j < ntt; j += 2) {
+            const bool two = j + 1 < ntt;
             const uint64_t db = umma_desc(st + b_off + j * UM_TILE_BYTES);
-            const uint32_t acc_col = tmem_base + j * n_mats * UM_TOK;
+            const uint32_t acc_col = tmem_base + j * UM_TOK;
+            const uint32_t id = two ? idesc2 : idesc;
 #pragma unroll
             for (int k4 = 0; k4 < UM_BK / 16; ++k4) {  // 16 inputs = 32 bytes = 2 descriptor units per step
               const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
-              umma_f16(acc_col, da0 + 2 * k4, db + 2 * k4, idesc, acc);
-              if (dual) umma_f16(acc_col + UM_TOK, da1 + 2 * k4, db + 2 * k4, idesc, acc);
+              umma_f16(acc_col, da0 + 2 * k4, db + 2 * k4, id, acc);
+              if (dual) umma_f16(acc_col + group * UM_TOK, da1 + 2 * k4, db + 2 * k4, id, acc);
             }
           }
           umma_commit(bar_ab_empty + 8 * s);  // the stage may be refilled once these MMAs have read it
@@ -454,9 +460,9 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
         const int tokens = min(UM_TOK, rec.cnt - tok_first - j * UM_TOK);
         const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tok_first) + static_cast<size_t>(j) * UM_TOK;
         uint32_t va[32], vb[32];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + j * n_mats * UM_TOK + cc;
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + j * UM_TOK + cc;
         tmem_ld32(taddr, va);
-        if (dual) tmem_ld32(taddr + UM_TOK, vb);
+        if (dual) tmem_ld32(taddr + group * UM_TOK, vb);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (nrow < N) {
 #pragma unroll
