@@ -122,6 +122,8 @@ HYBRID_CASES = [
     ("swiglu", 128, "f16", 512, 1536, 6, 2, "softmax_renorm", [4, 8, 2, 4, 2, 8], 90, 1.3),
     ("relu", 0, "f32", 1024, 512, 5, 1, "softmax", [2, 8, 4, 4, 8], 64, 1.5),
     ("relu", 128, "f16", 512, 512, 4, 1, "softmax", [2, 8, 4, 4], 12, 0.0),          # nobody above 32 tokens
+    ("relu", 128, "f16", 512, 1024, 2, 1, "softmax", [4, 2], 300, 0.0),               # everybody above 32 tokens
+    ("swiglu", 128, "f16", 512, 512, 2, 2, "softmax_renorm", [8, 2], 700, 0.0),       # 700 tokens per expert: several token groups
 ]
 
 
