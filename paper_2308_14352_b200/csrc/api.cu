@@ -271,8 +271,6 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     EMOE_LAUNCH(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,
                                       L.top_k, L.gate_mode == EMOE_GATE_SOFTMAX_RENORM, ids, gates, nullptr, st));
   }
-  EMOE_LAUNCH(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
-
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
   const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
   // many tokens per expert: the tcgen05 grouped GEMM; otherwise the weight-streaming kernels
@@ -287,6 +285,10 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   if (ctx->ffn_path == 3 && !use_tma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 4 && !use_umma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 5 && !use_hybrid) return EMOE_ERR_UNSUPPORTED;
+  // small batches on the streaming kernel: permutation, scatter and plan in one launch
+  const bool one_launch_permute = use_tma && ctx->fuse_projections && permute_scatter_supported(L, P);
+  if (!one_launch_permute)
+    EMOE_LAUNCH(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
   int ksplit = 1;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
   if (ctx->timing) {
@@ -342,7 +344,11 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
   } else if (use_tma) {
     ksplit = ffn_tma_ksplit(L, T);
-    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, 1, INT_MAX, st));
+    if (one_launch_permute)
+      EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, P, true,
+                                              ctx->check_word, st));
+    else
+      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, 1, INT_MAX, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
     if (ctx->fuse_projections) {

@@ -109,6 +109,11 @@ bool ffn_many_tokens(const LayerDims& L, int T);
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
                              bool to_f16, int cnt_lo, int cnt_hi, cudaStream_t st);
+// Permutation + scatter + plan in one launch (one CTA per pair) for batches of at most 1024 pairs.
+bool permute_scatter_supported(const LayerDims& L, int n_pairs);
+cudaError_t launch_permute_scatter(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
+                                   int32_t* counts, int32_t* off, int32_t* perm, int32_t* slot_of_pair, int* plan,
+                                   __nv_bfloat16* xs, int n_pairs, bool to_f16, int* check_word, cudaStream_t st);
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
                            const int32_t* off, __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs,
                            int T, cudaStream_t st);

@@ -203,55 +203,43 @@ __global__ void __launch_bounds__(MMA_THREADS)
   }
 }
 
-// x rows -> expert-sorted order, in the activation layout of the owning expert's bitwidth
-__global__ void __launch_bounds__(128)
-    scatter_x_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
-                     const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
-                     int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int to_f16, int cnt_lo, int cnt_hi,
-                     __nv_bfloat16* __restrict__ xs) {
-  pdl_wait();
-  pdl_trigger();
-  if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
-    // work plan of the persistent expert kernels: activated experts, widest codes (most bytes)
-    // first; the two item counters restart from zero
-    const int lane = threadIdx.x;
-    PlanRec* recs = reinterpret_cast<PlanRec*>(reinterpret_cast<char*>(plan) + PLAN_HEADER_BYTES);
-    int base = 0;
-    for (int b = 8; b >= 2; b >>= 1) {
-      for (int e0 = 0; e0 < E; e0 += 32) {
-        const int e = e0 + lane;
-        const int cnt = e < E ? off[e + 1] - off[e] : 0;
-        const bool act = cnt >= cnt_lo && cnt <= cnt_hi && experts[e].bits == b;
-        const unsigned m = __ballot_sync(0xffffffffu, act);
-        if (act) {
-          PlanRec& r = recs[base + __popc(m & ((1u << lane) - 1u))];
-          r.e = e;
-          r.begin = off[e];
-          r.cnt = cnt;
-          r.bits = b;
-          r.scales[0] = experts[e].scales[0];
-          r.scales[1] = experts[e].scales[1];
-          r.scales[2] = experts[e].scales[2];
-          r.done = 0;
-        }
-        base += __popc(m);
+// Work plan of the persistent expert kernels, written by one warp: activated experts whose token
+// count lies in [cnt_lo, cnt_hi], widest codes (most bytes) first; the item counters restart from
+// zero.  off: exclusive offsets of the experts' slots (global or shared memory).
+__device__ __forceinline__ void build_plan(int* plan, const ExpertDev* __restrict__ experts, const int32_t* off, int E,
+                                           int cnt_lo, int cnt_hi, int lane) {
+  PlanRec* recs = reinterpret_cast<PlanRec*>(reinterpret_cast<char*>(plan) + PLAN_HEADER_BYTES);
+  int base = 0;
+  for (int b = 8; b >= 2; b >>= 1) {
+    for (int e0 = 0; e0 < E; e0 += 32) {
+      const int e = e0 + lane;
+      const int cnt = e < E ? off[e + 1] - off[e] : 0;
+      const bool act = cnt >= cnt_lo && cnt <= cnt_hi && experts[e].bits == b;
+      const unsigned m = __ballot_sync(0xffffffffu, act);
+      if (act) {
+        PlanRec& r = recs[base + __popc(m & ((1u << lane) - 1u))];
+        r.e = e;
+        r.begin = off[e];
+        r.cnt = cnt;
+        r.bits = b;
+        r.scales[0] = experts[e].scales[0];
+        r.scales[1] = experts[e].scales[1];
+        r.scales[2] = experts[e].scales[2];
+        r.done = 0;
       }
-    }
-    if (lane == 0) {
-      plan[0] = base;
-      plan[1] = 0;
-      plan[2] = 0;
+      base += __popc(m);
     }
   }
-  const int slot = blockIdx.x;
-  const int pair = perm[slot];
-  if (pair < 0 || pair >= n_pairs) return;
-  const int e_slot = ids[pair];
-  const int cnt_slot = off[e_slot + 1] - off[e_slot];
-  if (cnt_slot < cnt_lo || cnt_slot > cnt_hi) return;  // this expert's rows belong to another kernel family
-  const int bits = experts[e_slot].bits;
-  const __nv_bfloat16* src_row = x + static_cast<size_t>(pair / top_k) * d;
-  __nv_bfloat16* dst_row = xs + static_cast<size_t>(slot) * d;
+  if (lane == 0) {
+    plan[0] = base;
+    plan[1] = 0;
+    plan[2] = 0;
+  }
+}
+
+// One activation row into the layout of the owning expert's bitwidth (optionally as fp16).
+__device__ __forceinline__ void scatter_row(const __nv_bfloat16* __restrict__ src_row, __nv_bfloat16* __restrict__ dst_row,
+                                            int d, int bits, int to_f16) {
   // one thread moves 16 consecutive inputs: half b of lane t's 32-block of a 128-input segment
   for (int u = threadIdx.x; u < d / 16; u += blockDim.x) {
     const int seg = (u >> 3) * 128, t = (u >> 1) & 3, b = u & 1;
@@ -276,6 +264,98 @@ __global__ void __launch_bounds__(128)
     *reinterpret_cast<uint4*>(dst_row + seg + (((2 * b) * 4 + t) << 3)) = oa;
     *reinterpret_cast<uint4*>(dst_row + seg + (((2 * b + 1) * 4 + t) << 3)) = oc;
   }
+}
+
+// x rows -> expert-sorted order, in the activation layout of the owning expert's bitwidth
+__global__ void __launch_bounds__(128)
+    scatter_x_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
+                     const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
+                     int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int to_f16, int cnt_lo, int cnt_hi,
+                     __nv_bfloat16* __restrict__ xs) {
+  pdl_wait();
+  pdl_trigger();
+  if (plan && blockIdx.x == 0 && threadIdx.x < 32) build_plan(plan, experts, off, E, cnt_lo, cnt_hi, threadIdx.x);
+  const int slot = blockIdx.x;
+  const int pair = perm[slot];
+  if (pair < 0 || pair >= n_pairs) return;
+  const int e_slot = ids[pair];
+  const int cnt_slot = off[e_slot + 1] - off[e_slot];
+  if (cnt_slot < cnt_lo || cnt_slot > cnt_hi) return;  // this expert's rows belong to another kernel family
+  scatter_row(x + static_cast<size_t>(pair / top_k) * d, xs + static_cast<size_t>(slot) * d, d, experts[e_slot].bits, to_f16);
+}
+
+// Permutation and scatter in one launch for small batches (at most PS_MAX_PAIRS pairs): one CTA
+// per pair.  Every CTA reads all expert ids and works out its own pair's slot (pairs with a lower
+// expert id come first, then pairs of the same expert with a lower index: the stable counting
+// sort of the definition), writes perm / slot_of_pair for it and copies its row; CTA 0 also
+// writes counts, offsets and the work plan.  No CTA waits for another.
+constexpr int PS_MAX_PAIRS = 1024;
+__global__ void __launch_bounds__(128)
+    permute_scatter_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
+                           const int32_t* __restrict__ ids, int E, int top_k, int d, int n_pairs, int to_f16,
+                           int32_t* __restrict__ counts, int32_t* __restrict__ off, int32_t* __restrict__ perm,
+                           int32_t* __restrict__ slot_of_pair, int* __restrict__ plan, int* __restrict__ check_word,
+                           __nv_bfloat16* __restrict__ xs) {
+  __shared__ int s_ids[PS_MAX_PAIRS];
+  __shared__ int s_off[EMOE_MAX_EXPERTS + 1];
+  __shared__ int s_red[2][4];
+  pdl_wait();
+  pdl_trigger();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int q = tid; q < n_pairs; q += blockDim.x) s_ids[q] = ids[q];
+  __syncthreads();
+  const int p = blockIdx.x;
+  const int e = s_ids[p];
+  const bool valid = e >= 0 && e < E;
+  // pairs in front of this one in expert order
+  int before = 0, same = 0;
+  for (int q = tid; q < n_pairs; q += blockDim.x) {
+    const int eq = s_ids[q];
+    before += (eq >= 0 && eq < e) || (eq == e && q < p);
+    same += eq == e;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    before += __shfl_xor_sync(0xffffffffu, before, o);
+    same += __shfl_xor_sync(0xffffffffu, same, o);
+  }
+  if (lane == 0) {
+    s_red[0][warp] = before;
+    s_red[1][warp] = same;
+  }
+  __syncthreads();
+  const int slot = s_red[0][0] + s_red[0][1] + s_red[0][2] + s_red[0][3];
+  if (p == 0) {
+    // counts, offsets, plan (this CTA only); invalid ids are reported and own no slot
+    for (int ee = tid; ee <= E; ee += blockDim.x) s_off[ee] = 0;
+    __syncthreads();
+    bool bad = false;
+    for (int q = tid; q < n_pairs; q += blockDim.x) {
+      const int eq = s_ids[q];
+      if (eq >= 0 && eq < E) atomicAdd(&s_off[eq + 1], 1);
+      else bad = true;
+    }
+    if (bad) atomicOr(check_word, CHECK_BAD_EXPERT_ID);
+    __syncthreads();
+    if (tid == 0) {
+      for (int ee = 0; ee < E; ++ee) {
+        counts[ee] = s_off[ee + 1];
+        s_off[ee + 1] += s_off[ee];
+      }
+    }
+    __syncthreads();
+    for (int ee = tid; ee <= E; ee += blockDim.x) off[ee] = s_off[ee];
+    if (warp == 0) build_plan(plan, experts, s_off, E, 1, 0x7fffffff, lane);
+  }
+  if (!valid) {
+    if (tid == 0) slot_of_pair[p] = -1;
+    return;
+  }
+  if (tid == 0) {
+    perm[slot] = p;
+    slot_of_pair[p] = slot;
+  }
+  scatter_row(x + static_cast<size_t>(p / top_k) * d, xs + static_cast<size_t>(slot) * d, d, experts[e].bits, to_f16);
 }
 
 
@@ -319,6 +399,16 @@ cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const
                              bool to_f16, int cnt_lo, int cnt_hi, cudaStream_t st) {
   return launch_chain(scatter_x_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
                       perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, to_f16 ? 1 : 0, cnt_lo, cnt_hi, xs);
+}
+
+bool permute_scatter_supported(const LayerDims& L, int n_pairs) { return n_pairs <= PS_MAX_PAIRS && L.E <= EMOE_MAX_EXPERTS; }
+
+cudaError_t launch_permute_scatter(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
+                                   int32_t* counts, int32_t* off, int32_t* perm, int32_t* slot_of_pair, int* plan,
+                                   __nv_bfloat16* xs, int n_pairs, bool to_f16, int* check_word, cudaStream_t st) {
+  return launch_chain(permute_scatter_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x),
+                      ids, L.E, L.top_k, L.d_model, n_pairs, to_f16 ? 1 : 0, counts, off, perm, slot_of_pair, plan, check_word,
+                      xs);
 }
 
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
