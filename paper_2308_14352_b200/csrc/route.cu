@@ -59,16 +59,18 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
     }
     __syncthreads();
     if (e < E) {
-      // 8 independent router-weight loads in flight per thread (the loop is L2-latency bound)
-      for (int i = slice; i < dc; i += 8 * S) {
-        float w[8];
+      // many independent router-weight loads in flight per thread (the loop is L2-latency bound;
+      // with one token per CTA the registers allow 24)
+      constexpr int U = TT == 1 ? 24 : 8;
+      for (int i = slice; i < dc; i += U * S) {
+        float w[U];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < U; ++u) {
           const int ii = i + u * S;
           w[u] = ii < dc ? __ldg(Wr + static_cast<size_t>(c0 + ii) * E + e) : 0.0f;
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < U; ++u) {
           const int ii = min(i + u * S, dc - 1);
 #pragma unroll
           for (int tt = 0; tt < TT; ++tt) acc[tt] = fmaf(xs[tt * ROUTER_DC + ii], w[u], acc[tt]);
