@@ -10,10 +10,13 @@
 // again per segment (ffn_tile.cuh), and the activations (bf16 values) travel as fp16, exact
 // inside the fp16 range and saturated outside.  And the bytes travel differently: the kernel is
 // bound by streaming packed weights from HBM, so the bytes in flight must not depend on registers:
-//   * the kernel is persistent: a CTA pulls work items (activated expert, block of output
-//     rows, split-K slice) from a device-side counter, most expensive bitwidth first, and its
+//   * the kernel is persistent and runs BOTH projections of a layer: a CTA pulls work items
+//     (activated expert, block of output rows[, split-K slice]) from a device-side counter, the
+//     first projection's items before the second's, most expensive bitwidth first, and its
 //     producer warp runs ahead across item boundaries, so the weight stream never drains
-//     between tiles;
+//     between tiles; an item of the second projection waits until the consumers of the first
+//     have counted the expert's hidden vectors complete (release / acquire on a counter in
+//     the expert's plan record);
 //   * the producer keeps a ring of STAGES shared-memory stages full.  One stage holds two
 //     64-row x 128-byte boxes of packed codes, fetched by two TMA tensor copies (128-byte
 //     swizzle, so that the consumers' 128-bit reads are conflict free), the matching slice of
@@ -51,9 +54,6 @@ constexpr int TMA_XROW_MAX = 512 * 2 + 64;         // bytes per token row of a s
 #endif
 #ifndef EMOE_TMA_L2PROMO
 #define EMOE_TMA_L2PROMO CU_TENSOR_MAP_L2_PROMOTION_L2_256B
-#endif
-#ifndef EMOE_TMA_LOOKAHEAD
-#define EMOE_TMA_LOOKAHEAD 0
 #endif
 #ifndef EMOE_TMA_CTAS_NT1
 #define EMOE_TMA_CTAS_NT1 3
