@@ -376,6 +376,13 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
   // projection alone finds plan, weights and scales older than the kernel in front, so its
   // producer starts fetching them and waits only before the first copy of a hidden vector (see
   // `waited` below).
+  if (warp == TMA_CONSUMER_WARPS) {
+    // The tensor maps are older than every kernel of the chain: pull them towards L2 now, so that
+    // the first copy of an expert's matrix does not wait for its descriptor to come from HBM.
+    const int n_maps = 3 * a.L.E;
+    const int i = (static_cast<int>(blockIdx.x) * 32 + lane) % ((n_maps + 31) / 32 * 32);
+    if (i < n_maps) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.tmaps + i));
+  }
   if (a.phase_begin == 0) pdl_wait();
   pdl_trigger();
 
