@@ -112,6 +112,17 @@ def pack_expert(W: np.ndarray, bits: int, group: int, scale_dtype: str) -> Tuple
     return pack(q, bits), s
 
 
+def requantize(packed: np.ndarray, scales: np.ndarray, K: int, bits_in: int, bits_out: int, group: int,
+               scale_dtype: str) -> Tuple[np.ndarray, np.ndarray]:
+    """An expert matrix stored at `bits_in` moved to `bits_out` without the original weights
+    (paper Section 3.2: the bitwidth selection lowers the width of chosen experts): decompress
+    to FP32 as the paper does (w~ = q * s, rounded once to fp32; exact with fp16 scales, which
+    have 11 significant bits against the codes' 8), then the same channel-wise linear
+    quantisation as for an fp32 matrix.  Returns (packed bytes, stored scales)."""
+    Wt = dequantize(packed, scales, K, bits_in, group)
+    return pack_expert(Wt.astype(np.float32), bits_out, group, scale_dtype)
+
+
 def scales_storage(scales: np.ndarray, scale_dtype: str) -> np.ndarray:
     """The scale channel in its storage type (values are already representable)."""
     return scales.astype(np.float16) if scale_dtype == "f16" else scales.astype(np.float32)

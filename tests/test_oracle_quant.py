@@ -132,3 +132,75 @@ def test_fp16_and_bf16_rounding_against_library_types():
     assert oracle.round_bf16(tie) == 1.0
     assert oracle.round_bf16(tie + 2.0 ** -40) == 1.0078125
     assert oracle.round_bf16(3.0 * 2.0 ** -134) == 2.0 ** -132   # subnormal tie: 1.5 quanta -> 2
+
+
+# ---- moving a stored matrix to another bitwidth (Section 3.2, bitwidth selection) -------------
+REQUANT_GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "requant_rows.txt")
+
+
+def _requant_rows():
+    rows = []
+    with open(REQUANT_GOLDEN) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            bi, bo, group, sdt, b_in, s_in, q_out, s_out, b_out = [p.strip() for p in line.split("|")]
+            rows.append((int(bi), int(bo), int(group), sdt,
+                         np.array([int(v, 16) for v in b_in.split()], dtype=np.uint8),
+                         np.array(s_in.split(), dtype=np.float64).astype(np.float32),
+                         np.array(q_out.split(), dtype=np.int64),
+                         np.array(s_out.split(), dtype=np.float64),
+                         np.array([int(v, 16) for v in b_out.split()], dtype=np.uint8)))
+    return rows
+
+
+@pytest.mark.parametrize("row", _requant_rows(), ids=lambda r: f"int{r[0]}_to_int{r[1]}_g{r[2]}_{r[3]}")
+def test_requantize_hand_computed_rows(row):
+    bi, bo, group, sdt, b_in, s_in, q_exp, s_exp, b_exp = row
+    K = b_in.size * 8 // bi
+    packed, scales = oracle.requantize(b_in[None, :], s_in[None, :], K, bi, bo, group, sdt)
+    assert np.array_equal(oracle.unpack(packed, K, bo)[0].astype(np.int64), q_exp)
+    assert np.array_equal(scales[0].astype(np.float64), s_exp)
+    assert np.array_equal(packed[0], b_exp)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("group", [0, 32])
+def test_requantize_to_the_same_width_is_the_identity(bits, group):
+    """Every non-zero group of a stored matrix holds a code of magnitude qmax, so its max-abs is
+    qmax * s exactly (fp16 scale: 11 + 7 significant bits) and the new scale (qmax * s) / qmax is s
+    again; the quotients (q * s) / s are the codes themselves."""
+    rng = np.random.default_rng(5 + bits)
+    W = (rng.standard_normal((24, 128)) * 0.02).astype(np.float32)
+    W[3, :] = 0.0  # an all-zero channel stays all zero
+    packed, scales = oracle.pack_expert(W, bits, group, "f16")
+    packed2, scales2 = oracle.requantize(packed, scales, 128, bits, bits, group, "f16")
+    assert np.array_equal(packed2, packed)
+    assert np.array_equal(scales2, scales)
+
+
+@pytest.mark.parametrize("bits_in,bits_out", [(8, 4), (8, 2), (4, 2), (2, 4), (4, 8)])
+@pytest.mark.parametrize("sdt", ["f16", "f32"])
+def test_requantize_closed_forms(bits_in, bits_out, sdt):
+    """The largest stored weight of a group maps to +-qmax of the new width, the new scale is the
+    group's largest decompressed magnitude over that qmax, and no weight moves by more than half
+    a new step (plus the fp16 rounding of the scale)."""
+    rng = np.random.default_rng(11 * bits_in + bits_out)
+    N, K, G = 16, 256, 128
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    packed, scales = oracle.pack_expert(W, bits_in, G, sdt)
+    Wt = oracle.dequantize(packed, scales, K, bits_in, G).astype(np.float32).astype(np.float64)
+    packed2, scales2 = oracle.requantize(packed, scales, K, bits_in, bits_out, G, sdt)
+    q2 = oracle.unpack(packed2, K, bits_out).astype(np.int64)
+    qmax = (1 << (bits_out - 1)) - 1
+    amax = np.abs(Wt).reshape(N, K // G, G).max(axis=2)
+    s32 = (amax.astype(np.float32) / np.float32(qmax)).astype(np.float32)
+    expect_s = s32.astype(np.float16).astype(np.float32) if sdt == "f16" else s32
+    assert np.array_equal(scales2, expect_s)
+    Wt2 = q2 * np.repeat(scales2.astype(np.float64), G, axis=1)
+    assert np.all(np.abs(q2) <= qmax)
+    at_max = np.abs(Wt) == np.repeat(amax, G, axis=1)
+    assert np.all(np.abs(q2[at_max & (np.repeat(amax, G, axis=1) > 0)]) == qmax)
+    slack = np.repeat(amax, G, axis=1) * 2.0 ** -11 if sdt == "f16" else 0.0
+    assert np.all(np.abs(Wt2 - Wt) <= np.repeat(scales2.astype(np.float64), G, axis=1) / 2 + slack + 1e-12)
