@@ -133,6 +133,23 @@ size_t emoe_scales_bytes(int N, int K, int group, int scale_dtype); /* N*(K/grou
 int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int group, int scale_dtype,
                      void* out_packed, void* out_scales, void* stream);
 
+/* Moves one stored matrix [N][K] from `bits_in` to `bits_out` without the fp32 original
+ * (Section 3.2, "Choosing the bitwidth": the selection puts the least important experts at
+ * the lower width and widens or narrows the set until the loss target is met; an expert that
+ * changes its width is re-quantised).  Each weight is decompressed in registers
+ * (w~ = q * s, rounded once to fp32; exact with fp16 scales) and quantised again with the
+ * arithmetic of emoe_pack_expert: the result equals emoe_pack_expert on the decompressed matrix,
+ * bit for bit.  Input and output use the same `group` and `scale_dtype`; any pair of widths is
+ * allowed (the same width reproduces the input when the scales are fp16).
+ *   in_packed / in_scales: device buffers in the storage format, emoe_packed_bytes(N,K,bits_in)
+ *   and emoe_scales_bytes(...) bytes; out_packed / out_scales: emoe_packed_bytes(N,K,bits_out)
+ *   and emoe_scales_bytes(...) bytes, owned by the caller, distinct from the inputs (not in
+ *   place).  Packed buffers 16-byte aligned, scale buffers 4-byte aligned.
+ * Errors as for emoe_pack_expert; asynchronous on `stream`. */
+int emoe_requantize_expert(emoe_ctx* ctx, const void* in_packed, const void* in_scales, int N, int K, int bits_in,
+                           int bits_out, int group, int scale_dtype, void* out_packed, void* out_scales,
+                           void* stream);
+
 /* ---- Sections 1, 2.1: router and Top-K gating ----------------------------------------- */
 
 /* z[t][e] = sum_i x[t][i] * router_W[i][e] (+ bias), p = softmax(z) over all experts; the

@@ -500,6 +500,27 @@ int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int 
   return EMOE_OK;
 }
 
+int emoe_requantize_expert(emoe_ctx* ctx, const void* in_packed, const void* in_scales, int N, int K, int bits_in,
+                           int bits_out, int group, int scale_dtype, void* out_packed, void* out_scales,
+                           void* stream) {
+  if (!ctx || !in_packed || !in_scales || !out_packed || !out_scales || N <= 0 || K <= 0 || group < 0)
+    return EMOE_ERR_INVALID_ARG;
+  if (bits_in != 2 && bits_in != 4 && bits_in != 8) return EMOE_ERR_UNSUPPORTED;
+  if (bits_out != 2 && bits_out != 4 && bits_out != 8) return EMOE_ERR_UNSUPPORTED;
+  if (scale_dtype != EMOE_DTYPE_F32 && scale_dtype != EMOE_DTYPE_F16) return EMOE_ERR_UNSUPPORTED;
+  const int G = group > 0 ? group : K;
+  if (K % G != 0) return EMOE_ERR_INVALID_ARG;
+  if (G % 4 != 0) return EMOE_ERR_UNSUPPORTED;
+  if (in_packed == out_packed || in_scales == out_scales) return EMOE_ERR_INVALID_ARG;  // not in place
+  if (!aligned(in_packed, 16) || !aligned(out_packed, 16) || !aligned(in_scales, 4) || !aligned(out_scales, 4))
+    return EMOE_ERR_ALIGNMENT;
+  EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+  EMOE_CUDA(ctx, launch_requant(static_cast<const uint8_t*>(in_packed), in_scales, N, K, bits_in, bits_out, group,
+                                scale_dtype == EMOE_DTYPE_F16, static_cast<uint8_t*>(out_packed), out_scales,
+                                static_cast<cudaStream_t>(stream)));
+  return EMOE_OK;
+}
+
 int emoe_router_topk(emoe_ctx* ctx, const void* x, int act_dtype, int T, int d, const float* router_W,
                      const float* router_bias, int bias_token_stride, int E, int top_k, int gate_mode,
                      int32_t* out_ids, float* out_gates, float* out_logits, void* stream) {
