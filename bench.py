@@ -397,34 +397,58 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
     achieved = expert_bytes_per_step / (ffn_ms_per_step * 1e-3) / 1e9
 
     # ---- end to end through the C ABI from host buffers ----------------------------------------
-    x_host = [torch.empty(x.shape, dtype=x.dtype).pin_memory() for x in xs]
-    for h, d in zip(x_host, xs):
-        h.copy_(d.cpu())
-    y_host = [torch.empty(T, sh.d_model, dtype=torch.float32).pin_memory() for _ in range(n_layers)]
-    x_stage = [torch.empty_like(x) for x in xs]
+    # one pinned buffer with the step's inputs (every layer's x) and one for its results: a step
+    # is one host->device copy, the forward calls of all layers, one device->host copy
+    x_host = torch.empty((n_layers,) + tuple(xs[0].shape), dtype=xs[0].dtype).pin_memory()
+    for l, d in enumerate(xs):
+        x_host[l].copy_(d.cpu())
+    y_host = torch.empty(n_layers, T, sh.d_model, dtype=torch.float32).pin_memory()
+    x_stage = torch.empty(x_host.shape, dtype=x_host.dtype, device=dev)
+    y_stage = torch.zeros(y_host.shape, dtype=torch.float32, device=dev)
 
     def e2e_step():
+        x_stage.copy_(x_host, non_blocking=True)
         for l, moe in enumerate(layers):
-            x_stage[l].copy_(x_host[l], non_blocking=True)
-            moe.forward_device(x_stage[l], Wrs[l], biases[l], ys[l], None, None, None, stream.cuda_stream)
-            y_host[l].copy_(ys[l], non_blocking=True)
+            moe.forward_device(x_stage[l], Wrs[l], biases[l], y_stage[l], None, None, None, stream.cuda_stream)
+        y_host.copy_(y_stage, non_blocking=True)
+
+    # like the device-resident arm, the step (copies included) is replayed as a CUDA graph unless
+    # --no-graph asks for direct launches: every replay copies x from the pinned buffers, runs the
+    # forward calls and copies y back
+    e2e_graph = None
+    if use_graph:
+        with torch.cuda.stream(stream):
+            e2e_step()
+            stream.synchronize()
+        e2e_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(e2e_graph, stream=stream):
+            e2e_step()
+
+    def e2e_run():
+        if e2e_graph is not None:
+            e2e_graph.replay()
+        else:
+            e2e_step()
 
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
-            e2e_step()
+            e2e_run()
         stream.synchronize()
         barrier(world)
         t0 = time.perf_counter()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record(stream)
         for _ in range(args.steps):
-            e2e_step()
+            e2e_run()
         f1.record(stream)
         stream.synchronize()
         e2e_wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
     e2e_ms = max(f0.elapsed_time(f1) / args.steps, e2e_wall_ms)
-    h2d = sum(x.numel() * x.element_size() for x in xs)
-    d2h = sum(y.numel() * y.element_size() for y in ys)
+    for l in (0, n_layers - 1):  # the copies of the timed steps really delivered the results
+        if not torch.equal(y_host[l], ys[l].cpu()):
+            raise RuntimeError("end-to-end arm: host copy of y differs from the device result")
+    h2d = x_host.numel() * x_host.element_size()
+    d2h = y_host.numel() * y_host.element_size()
 
     units = float(T * n_layers)
     ms_job, units_job = reduce_max_and_sum(ms_step, units, world, dev)
