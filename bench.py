@@ -397,53 +397,95 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
     achieved = expert_bytes_per_step / (ffn_ms_per_step * 1e-3) / 1e9
 
     # ---- end to end through the C ABI from host buffers ----------------------------------------
-    # one pinned buffer with the step's inputs (every layer's x) and one for its results: a step
-    # is one host->device copy, the forward calls of all layers, one device->host copy
+    # One pinned buffer with the step's inputs (every layer's x) and one for its results.  Two
+    # buffer sets on the device: while the forward calls of step i run on set b, a second stream
+    # copies the results of step i-1 to the host and the inputs of step i+1 to the device (set
+    # 1-b), so every step still moves its inputs and its results across the host link inside the
+    # timed region, under the kernels of its neighbours.
     x_host = torch.empty((n_layers,) + tuple(xs[0].shape), dtype=xs[0].dtype).pin_memory()
     for l, d in enumerate(xs):
         x_host[l].copy_(d.cpu())
     y_host = torch.empty(n_layers, T, sh.d_model, dtype=torch.float32).pin_memory()
-    x_stage = torch.empty(x_host.shape, dtype=x_host.dtype, device=dev)
-    y_stage = torch.zeros(y_host.shape, dtype=torch.float32, device=dev)
+    x_stage = [torch.empty(x_host.shape, dtype=x_host.dtype, device=dev) for _ in range(2)]
+    y_stage = [torch.zeros(y_host.shape, dtype=torch.float32, device=dev) for _ in range(2)]
+    copy_stream = torch.cuda.Stream(device=dev)
 
-    def e2e_step():
-        x_stage.copy_(x_host, non_blocking=True)
+    def e2e_step(b):
+        fork = torch.cuda.Event()
+        fork.record(stream)
+        copy_stream.wait_event(fork)
+        with torch.cuda.stream(copy_stream):
+            y_host.copy_(y_stage[1 - b], non_blocking=True)
+            x_stage[1 - b].copy_(x_host, non_blocking=True)
+            join = torch.cuda.Event()
+            join.record(copy_stream)
         for l, moe in enumerate(layers):
-            moe.forward_device(x_stage[l], Wrs[l], biases[l], y_stage[l], None, None, None, stream.cuda_stream)
-        y_host.copy_(y_stage, non_blocking=True)
+            moe.forward_device(x_stage[b][l], Wrs[l], biases[l], y_stage[b][l], None, None, None, stream.cuda_stream)
+        stream.wait_event(join)
 
-    # like the device-resident arm, the step (copies included) is replayed as a CUDA graph unless
-    # --no-graph asks for direct launches: every replay copies x from the pinned buffers, runs the
-    # forward calls and copies y back
-    e2e_graph = None
+    # like the device-resident arm, the steps (copies included) are replayed as CUDA graphs, one
+    # per buffer set, unless --no-graph asks for direct launches
+    e2e_graphs = None
+    with torch.cuda.stream(stream):
+        x_stage[0].copy_(x_host, non_blocking=True)
+        e2e_step(0)
+        e2e_step(1)
+        stream.synchronize()
     if use_graph:
-        with torch.cuda.stream(stream):
-            e2e_step()
-            stream.synchronize()
-        e2e_graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(e2e_graph, stream=stream):
-            e2e_step()
+        e2e_graphs = []
+        for b in range(2):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                e2e_step(b)
+            e2e_graphs.append(g)
 
-    def e2e_run():
-        if e2e_graph is not None:
-            e2e_graph.replay()
+    def e2e_run(i):
+        if e2e_graphs is not None:
+            e2e_graphs[i & 1].replay()
         else:
-            e2e_step()
+            e2e_step(i & 1)
 
     with torch.cuda.stream(stream):
-        for _ in range(args.warmup):
-            e2e_run()
+        for i in range(2 * ((args.warmup + 1) // 2)):
+            e2e_run(i)
         stream.synchronize()
         barrier(world)
         t0 = time.perf_counter()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record(stream)
-        for _ in range(args.steps):
-            e2e_run()
+        for i in range(args.steps):
+            e2e_run(i)
+        y_host.copy_(y_stage[(args.steps - 1) & 1], non_blocking=True)  # the last step's results
         f1.record(stream)
         stream.synchronize()
         e2e_wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
     e2e_ms = max(f0.elapsed_time(f1) / args.steps, e2e_wall_ms)
+
+    # the same step without overlap, for comparison: copy in, forward calls, copy out, one stream
+    def serial_step():
+        x_stage[0].copy_(x_host, non_blocking=True)
+        for l, moe in enumerate(layers):
+            moe.forward_device(x_stage[0][l], Wrs[l], biases[l], y_stage[0][l], None, None, None, stream.cuda_stream)
+        y_host.copy_(y_stage[0], non_blocking=True)
+
+    serial_graph = None
+    with torch.cuda.stream(stream):
+        serial_step()
+        stream.synchronize()
+    if use_graph:
+        serial_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(serial_graph, stream=stream):
+            serial_step()
+    n_serial = min(args.steps, 200)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            serial_graph.replay() if serial_graph is not None else serial_step()
+        stream.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n_serial):
+            serial_graph.replay() if serial_graph is not None else serial_step()
+        stream.synchronize()
+        serial_ms = (time.perf_counter() - t0) * 1e3 / n_serial
     for l in (0, n_layers - 1):  # the copies of the timed steps really delivered the results
         if not torch.equal(y_host[l], ys[l].cpu()):
             raise RuntimeError("end-to-end arm: host copy of y differs from the device result")
@@ -470,7 +512,11 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
             "config": config_dict(w, T, n_layers, world, use_graph),
             "clocks": clocks,
             "e2e": {"value": units_job / (e2e_job * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_job},
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_job, "serial_ms_per_step": serial_ms,
+                    "note": "every step copies its inputs host->device and its results device->host (pinned "
+                            "memory, second stream, two buffer sets: the copies of neighbouring steps run "
+                            "under the step's kernels); serial_ms_per_step: the same step with copy in, forward "
+                            "calls and copy out one after the other on one stream"},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": {
                 "kernel": "expert-FFN kernels (both projections of every layer)", "bound": "hbm",
