@@ -88,6 +88,26 @@ class MoELayer:
                 self.pack_matrix(e, m, w)
         torch.cuda.synchronize(self.device)
 
+    def change_width(self, e: int, bits_out: int, stream: int = 0) -> None:
+        """Moves expert `e` to `bits_out` on the device, from its stored codes and scales (no fp32
+        original needed), and points the expert table at the new buffers."""
+        b_in = self.bits[e]
+        new_packed, new_scales = [], []
+        for m in range(self.shape.n_matrices):
+            N, K = self.shape.matrix_shape(m)
+            p = torch.empty(N * K * bits_out // 8, dtype=torch.uint8, device=self.device)
+            s = torch.empty_like(self.scales[e][m])
+            B.emoe_requantize_expert(self.ctx, self.packed[e][m].data_ptr(), self.scales[e][m].data_ptr(), N, K, b_in,
+                                     bits_out, self.shape.group, _SDT[self.shape.scale_dtype], p.data_ptr(),
+                                     s.data_ptr(), stream)
+            new_packed.append(p)
+            new_scales.append(s)
+        torch.cuda.synchronize(self.device)  # the old buffers are released below
+        self.packed[e], self.scales[e], self.bits[e] = new_packed, new_scales, bits_out
+        self.table = B.make_expert_table([
+            (self.bits[i], [t.data_ptr() for t in self.packed[i]], [t.data_ptr() for t in self.scales[i]])
+            for i in range(self.shape.n_experts)])
+
     def packed_host(self, e: int, m: int) -> np.ndarray:
         N, K = self.shape.matrix_shape(m)
         return self.packed[e][m].cpu().numpy().reshape(N, K * self.bits[e] // 8)

@@ -113,3 +113,39 @@ def test_requantize_argument_errors(ctx):
     assert call(*bad(0, pin.data_ptr() + 4)) == B.ERR_ALIGNMENT
     assert call(*bad(7, B.DTYPE_BF16)) == B.ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+def test_forward_after_lowering_the_width_of_two_experts():
+    """The bitwidth adaptation end to end: a layer packed at INT8, two experts then moved to INT4
+    and INT2 on the device; packed bytes and scales equal the checker's, and the forward on the
+    new storage equals the checker's forward on it."""
+    from paper_2308_14352_b200 import inputs, layer
+    from tests.helpers import rel_to_max
+
+    shape = inputs.LayerShape(512, 1024, 4, 2, "swiglu", "softmax_renorm", 128, "f16", "bf16")
+    bits = [8, 8, 8, 8]
+    W = inputs.expert_set(41, 0, shape)
+    x = inputs.activations(41, 0, 12, shape.d_model, "bf16")
+    Wr = inputs.router_weight(41, 0, shape.d_model, shape.n_experts, std=0.05)
+    packed, scales = [], []
+    for e in range(4):
+        ps = [oracle.pack_expert(W[e][m], 8, 128, "f16") for m in range(3)]
+        packed.append([p for p, _ in ps])
+        scales.append([s for _, s in ps])
+    new_bits = [8, 4, 8, 2]
+    for e in (1, 3):
+        for m in range(3):
+            K = shape.matrix_shape(m)[1]
+            packed[e][m], scales[e][m] = oracle.requantize(packed[e][m], scales[e][m], K, 8, new_bits[e], 128, "f16")
+    with layer.MoELayer(shape, bits, max_tokens=12) as moe:
+        moe.pack_from_host(W)
+        moe.change_width(1, 4)
+        moe.change_width(3, 2)
+        assert moe.bits == new_bits
+        for e in range(4):
+            for m in range(3):
+                assert np.array_equal(moe.packed_host(e, m), packed[e][m])
+                assert np.array_equal(moe.scales_host(e, m).astype(np.float32), scales[e][m])
+        y, ids, gates, _ = moe.forward(x, Wr)
+    y_ref = oracle.moe_ffn_combine(x, shape.d_ff, "swiglu", 128, True, new_bits, packed, scales, ids, gates)
+    assert rel_to_max(y, y_ref) <= 2e-3
