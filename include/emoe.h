@@ -103,8 +103,8 @@ typedef struct emoe_layer_desc {
 emoe_ctx* emoe_create(int device, size_t workspace_bytes, int* status);
 int emoe_destroy(emoe_ctx* ctx);
 
-/* Scratch a forward call over T tokens needs; pass the maximum over your calls to
- * emoe_create.  Returns 0 for an invalid description. */
+/* Scratch that forward calls over at most T tokens need; pass the maximum over the layer
+ * descriptions you use to emoe_create.  Returns 0 for an invalid description. */
 size_t emoe_workspace_bytes(const emoe_layer_desc* desc, int T);
 
 /* CUDA error code of the last failed CUDA call on this context (0 if none). */

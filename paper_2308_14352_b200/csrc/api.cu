@@ -442,7 +442,14 @@ int emoe_destroy(emoe_ctx* ctx) {
 size_t emoe_workspace_bytes(const emoe_layer_desc* desc, int T) {
   LayerDims L;
   if (!make_dims(desc, &L) || T <= 0) return 0;
-  return make_layout(L, T).total;
+  // enough for every call of up to T tokens: a call with very few tokens splits the second
+  // projection finer and may need more partial-sum rows per token than a larger one
+  size_t need = make_layout(L, T).total;
+  for (int t = 1; t < T && t <= 256; ++t) {
+    const size_t n = make_layout(L, t).total;
+    if (n > need) need = n;
+  }
+  return need;
 }
 
 int emoe_last_cuda_error(const emoe_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }

@@ -701,7 +701,13 @@ int ffn_tma_ksplit(const LayerDims& L, int T) {
   // enough slices that the second projection's items outnumber the resident CTAs (3 per SM)
   // about twice: short items at the end of the launch keep its tail short
   long long z = (8 * 148 + ctas - 1) / ctas;
-  if (z > steps_min) z = steps_min;
+  // A handful of tokens leaves most SMs without an item: the slices are then cut as fine as the
+  // 8-bit stages allow (narrower experts get empty slices, which only store zeros), so that the
+  // second projection of the one or two activated experts is a short step on many SMs instead
+  // of a chain of stages on a few (single token, Switch-base-like layer: 8 % off the launch).
+  const int steps_max = (L.d_ff + 127) / 128;
+  const int cap = ctas * 4 <= 148 ? steps_max : steps_min;
+  if (z > cap) z = cap;
   if (z > 16) z = 16;
   if (z < 1) z = 1;
   return static_cast<int>(z);
