@@ -289,10 +289,8 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int r
 __device__ __forceinline__ void count_item_done(PlanRec* recs, int ai, int lane) {
   asm volatile("fence.proxy.async;" ::: "memory");
   __syncwarp();
-  if (lane == 0) {
-    __threadfence();
-    atomicAdd(&recs[ai].done, 1);
-  }
+  if (lane == 0)  // release: the hidden values this warp stored are visible before the count is
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(&recs[ai].done), "r"(1) : "memory");
 }
 
 // the hidden vector is rounded to bf16 (the layer's activation type), then carried as fp16
