@@ -32,7 +32,7 @@ from paper_2308_14352_b200 import inputs  # noqa: E402
 # DRAM bytes (read + write) of the expert-FFN launch of one layer (mean of the two layers of the ncu
 # capture summarised in profiles/ffn_tma_kernel_switch_base_decode_T64.md); reported as `traffic`
 # for that workload only, and to be set back to None whenever that kernel changes.
-NCU_DRAM_BYTES_PER_LAYER = {("switch_base_decode", 64): 74.9e6}
+NCU_DRAM_BYTES_PER_LAYER = {("switch_base_decode", 64): 74.7e6}
 
 METRIC = "MoE-layer tokens/s"
 UNIT = "tokens/s"
