@@ -55,6 +55,7 @@ extern "C" {
 #define EMOE_ERR_CUDA (-5)         /* a CUDA call failed; emoe_last_cuda_error() gives its code */
 #define EMOE_ERR_DEVICE_CHECK (-6) /* a kernel found inconsistent data (e.g. an expert id out of range) */
 #define EMOE_ERR_CACHE_FULL (-7)   /* every slot of the expert cache is in use by an unfinished call */
+#define EMOE_ERR_TIMEOUT (-8)      /* a bounded wait inside a kernel ran out; the kernel gave up and returned */
 
 /* enums (plain ints in the ABI) */
 #define EMOE_DTYPE_F32 0
@@ -110,8 +111,10 @@ size_t emoe_workspace_bytes(const emoe_layer_desc* desc, int T);
 /* CUDA error code of the last failed CUDA call on this context (0 if none). */
 int emoe_last_cuda_error(const emoe_ctx* ctx);
 
-/* Reads (and clears) the device-side check word: EMOE_OK, or EMOE_ERR_DEVICE_CHECK if a
- * kernel of an earlier call met inconsistent data.  Synchronises `stream`. */
+/* Reads (and clears) the device-side check word: EMOE_OK; EMOE_ERR_TIMEOUT if a bounded wait
+ * inside a kernel of an earlier call ran out (the kernel gave up and returned; results of that
+ * call are undefined, the context stays usable); else EMOE_ERR_DEVICE_CHECK if a kernel met
+ * inconsistent data (an expert id out of range).  Synchronises `stream`. */
 int emoe_device_status(emoe_ctx* ctx, void* stream);
 
 const char* emoe_status_string(int status);
@@ -239,7 +242,11 @@ int emoe_kernels_last_forward(const emoe_ctx* ctx);
  *   returns EMOE_ERR_WORKSPACE and does nothing.  Other argument rules as for
  *   emoe_moe_forward_routed.
  *   First call on a device: looks up the array's device address (with that device made
- *   current).  Make this first call outside any stream capture.
+ *   current).  Make this first call outside any stream capture.  Every call only enqueues
+ *   kernels (the expert table travels as launch parameters, no host buffer is referenced after
+ *   the call returns).
+ *   Expert ids outside [0, n_experts) are dropped from the result and set a check word inside
+ *   the array; emoe_static_device_status reads it.
  *   Sharing: every call on a device uses the same array, which keeps the previous call's
  *   contents (the call clears what has to start at zero itself).  Two calls whose GPU work
  *   overlaps (different streams without a dependency, or different host threads) race on it:
@@ -248,6 +255,12 @@ int emoe_kernels_last_forward(const emoe_ctx* ctx);
  * emoe_moe_forward_routed. */
 int emoe_moe_forward_routed_static(int device, const emoe_layer_desc* desc, const void* x, int T, const int32_t* ids,
                                    const float* gates, const emoe_expert* host_experts, float* y, void* stream);
+
+/* Status of the calls of emoe_moe_forward_routed_static enqueued so far on `device` (the paper
+ * has no counterpart): synchronises `stream`, then returns EMOE_OK, EMOE_ERR_DEVICE_CHECK (an
+ * expert id was out of range) or EMOE_ERR_TIMEOUT.  The word is cleared by the next forward call,
+ * not by this one.  Allocates nothing. */
+int emoe_static_device_status(int device, void* stream);
 
 /* Measurement aid (Section 4 of the paper times compute and loading separately; here the
  * expert-FFN kernels are the part bound by weight streaming).  While enabled, every forward

@@ -21,6 +21,7 @@ ERR_WORKSPACE = -4
 ERR_CUDA = -5
 ERR_DEVICE_CHECK = -6
 ERR_CACHE_FULL = -7
+ERR_TIMEOUT = -8
 EVICT_FORWARD, EVICT_PRINTED, EVICT_LRU = 0, 1, 2
 
 DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
@@ -32,7 +33,7 @@ EXPORTS = (
     "emoe_status_string", "emoe_packed_bytes", "emoe_scales_bytes", "emoe_pack_expert", "emoe_requantize_expert",
     "emoe_router_topk",
     "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
-    "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_set_dependent_launch",
+    "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_static_device_status", "emoe_set_dependent_launch",
     "emoe_set_fused_projections", "emoe_kernels_last_forward",
     "emoe_cache_create", "emoe_register_expert", "emoe_prefetch_experts", "emoe_cache_acquire", "emoe_cache_release",
     "emoe_cache_slot_of", "emoe_cache_get_stats", "emoe_policy_create", "emoe_policy_destroy", "emoe_policy_register",
@@ -125,6 +126,7 @@ def lib() -> ctypes.CDLL:
                                         ctypes.POINTER(ctypes.c_int32)]
         L.emoe_moe_forward_routed_static.argtypes = [i32, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
                                                      ctypes.POINTER(emoe_expert), vp, vp]
+        L.emoe_static_device_status.argtypes = [i32, vp]
         L.emoe_read_timing.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
                                        ctypes.POINTER(ctypes.c_int)]
         _lib = L
@@ -241,6 +243,11 @@ def emoe_moe_forward_routed_static(device: int, desc: emoe_layer_desc, x_ptr, T,
     inside the library; T * top_k <= 64).  For callers that may not allocate."""
     _check(lib().emoe_moe_forward_routed_static(device, ctypes.byref(desc), x_ptr, T, ids_ptr, gates_ptr,
                                                 expert_table, y_ptr, stream), "emoe_moe_forward_routed_static")
+
+
+def emoe_static_device_status(device: int, stream: int = 0) -> int:
+    """Status word of the context-free forward calls enqueued so far on `device` (synchronises)."""
+    return int(lib().emoe_static_device_status(device, stream))
 
 
 def emoe_set_dependent_launch(ctx, enabled: bool) -> None:

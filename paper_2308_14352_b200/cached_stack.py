@@ -43,7 +43,8 @@ class CachedStack:
         self.compute = torch.cuda.Stream(device=self.dev)
         self.copy = torch.cuda.Stream(device=self.dev)
         E = shape.n_experts
-        gen = torch.Generator(device=self.dev)
+        self.seed = seed
+        self._gen = torch.Generator(device=self.dev)
         sdt = torch.float16 if shape.scale_dtype == "f16" else torch.float32
         # experts: seeded N(0, 0.02^2) fp32 on the device -> packed by the library -> pinned host memory
         self.host: List[List[tuple]] = []
@@ -56,8 +57,7 @@ class CachedStack:
                 for m in range(shape.n_matrices):
                     N, K = shape.matrix_shape(m)
                     G = shape.group if shape.group > 0 else K
-                    gen.manual_seed((seed << 32) ^ (l << 16) ^ (e << 4) ^ m)
-                    W = torch.randn(N, K, generator=gen, device=self.dev, dtype=torch.float32) * 0.02
+                    W = self.draw_matrix(l, e, m)
                     p = torch.empty(N * K * self.bits[e] // 8, dtype=torch.uint8, device=self.dev)
                     s = torch.empty(N * (K // G), dtype=sdt, device=self.dev)
                     B.emoe_pack_expert(self.ctx, W.data_ptr(), N, K, self.bits[e], shape.group, _SDT[shape.scale_dtype],
@@ -92,6 +92,12 @@ class CachedStack:
         self.y = torch.empty(max_tokens, shape.d_model, dtype=torch.float32, device=self.dev)
         torch.cuda.synchronize(self.dev)
 
+    def draw_matrix(self, l: int, e: int, m: int) -> torch.Tensor:
+        """The fp32 weight matrix m of expert e of layer l (seeded N(0, 0.02^2), drawn on the device)."""
+        N, K = self.shape.matrix_shape(m)
+        self._gen.manual_seed((self.seed << 32) ^ (l << 16) ^ (e << 4) ^ m)
+        return torch.randn(N, K, generator=self._gen, device=self.dev, dtype=torch.float32) * 0.02
+
     @staticmethod
     def _nbytes(pm, sm):
         nb = [t.numel() * t.element_size() for t in pm] + [0] * (3 - len(pm))
@@ -120,11 +126,13 @@ class CachedStack:
         e1.synchronize()
         return 4 * src.numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9
 
-    def forward_stack(self, xs: Sequence[torch.Tensor], measure: bool = False, prefetch: bool = True):
+    def forward_stack(self, xs: Sequence[torch.Tensor], measure: bool = False, prefetch: bool = True,
+                      outputs: Optional[list] = None):
         """One pass of the token batch through all layers.  xs[l]: [T][d] bf16 on the device.
         Returns the picks of every layer (host arrays).  With measure=True every acquire is
         bracketed by two events on the compute stream: their distance is the time the compute
-        stream stood still for a load (the exposed copy time)."""
+        stream stood still for a load (the exposed copy time).  If `outputs` is a list, every
+        layer appends (gates, y) of the batch to it (device copies)."""
         sh, E = self.shape, self.shape.n_experts
         T = xs[0].shape[0]
         cs, cps = self.compute.cuda_stream, self.copy.cuda_stream
@@ -160,14 +168,19 @@ class CachedStack:
                 first = acq[0]
                 table = (B.emoe_expert * E)()
                 for e in range(E):
-                    src = by_e.get(e, first)    # entries of experts nobody picked are never read
-                    table[e].bits = self.bits[e]
+                    # entries of experts nobody picked are never read; they borrow an acquired expert
+                    # whole (pointers AND width, so that whatever is derived from an entry stays
+                    # inside that expert's slot)
+                    src = by_e.get(e, first)
+                    table[e].bits = self.bits[e] if e in by_e else self.bits[active[0]]
                     for m in range(3):
                         table[e].packed[m] = src.packed[m]
                         table[e].scales[m] = src.scales[m]
                 B.emoe_moe_forward_routed(self.ctx, self.desc, xs[l].data_ptr(), T, self.ids.data_ptr(), self.gates.data_ptr(),
                                           table, self.y.data_ptr(), None, cs)
                 B.emoe_cache_release(self.ctx, eids, cs)
+                if outputs is not None:
+                    outputs.append((self.gates[:T].clone(), self.y[:T].clone()))
                 prev = ids
         return picks
 

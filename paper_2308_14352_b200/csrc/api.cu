@@ -461,6 +461,7 @@ int emoe_device_status(emoe_ctx* ctx, void* stream) {
   EMOE_CUDA(ctx, cudaMemcpyAsync(ctx->check_host, ctx->check_word, sizeof(int), cudaMemcpyDeviceToHost, st));
   EMOE_CUDA(ctx, cudaMemsetAsync(ctx->check_word, 0, sizeof(int), st));
   EMOE_CUDA(ctx, cudaStreamSynchronize(st));
+  if (*ctx->check_host & CHECK_WAIT_TIMEOUT) return EMOE_ERR_TIMEOUT;
   return *ctx->check_host ? EMOE_ERR_DEVICE_CHECK : EMOE_OK;
 }
 
@@ -474,6 +475,7 @@ const char* emoe_status_string(int status) {
     case EMOE_ERR_CUDA: return "CUDA call failed (see emoe_last_cuda_error)";
     case EMOE_ERR_DEVICE_CHECK: return "a kernel found inconsistent data";
     case EMOE_ERR_CACHE_FULL: return "every slot of the expert cache is in use";
+    case EMOE_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
     default: return "unknown status";
   }
 }

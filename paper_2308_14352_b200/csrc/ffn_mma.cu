@@ -279,6 +279,7 @@ __global__ void __launch_bounds__(128)
   const int pair = perm[slot];
   if (pair < 0 || pair >= n_pairs) return;
   const int e_slot = ids[pair];
+  if (e_slot < 0 || e_slot >= E) return;  // a slot the permutation did not write (stale entry behind a dropped pair)
   const int cnt_slot = off[e_slot + 1] - off[e_slot];
   if (cnt_slot < cnt_lo || cnt_slot > cnt_hi) return;  // this expert's rows belong to another kernel family
   scatter_row(x + static_cast<size_t>(pair / top_k) * d, xs + static_cast<size_t>(slot) * d, d, experts[e_slot].bits, to_f16);

@@ -41,6 +41,7 @@ bool dims_from_desc(const emoe_layer_desc* d, LayerDims* L) {
   if (d->n_experts < 1 || d->n_experts > EMOE_MAX_EXPERTS) return false;
   if (d->top_k < 1 || d->top_k > d->n_experts || d->top_k > EMOE_MAX_TOP_K) return false;
   if (d->act != EMOE_ACT_RELU && d->act != EMOE_ACT_SWIGLU) return false;
+  if (d->gate_mode != EMOE_GATE_SOFTMAX && d->gate_mode != EMOE_GATE_SOFTMAX_RENORM) return false;
   if (d->scale_dtype != EMOE_DTYPE_F32 && d->scale_dtype != EMOE_DTYPE_F16) return false;
   if (d->act_dtype != EMOE_DTYPE_F32 && d->act_dtype != EMOE_DTYPE_BF16) return false;
   if (d->group < 0 || (d->group > 0 && (d->d_model % d->group != 0 || d->d_ff % d->group != 0))) return false;
@@ -78,6 +79,20 @@ StaticLayout layout_for(const LayerDims& L, int T) {
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// The expert table reaches the scratch array as kernel parameters, 64 entries (3.5 KB) per
+// launch: parameters are copied when the launch is enqueued (or captured), so no copy node ever
+// keeps the address of a host buffer that has gone out of scope, and no pageable copy stalls
+// the calling thread behind earlier work on the stream.
+constexpr int TABLE_CHUNK = 64;
+struct TableChunk {
+  ExpertDev e[TABLE_CHUNK];
+};
+__global__ void write_table_kernel(const __grid_constant__ TableChunk c, ExpertDev* dst, int n, int* check_word) {
+  const int i = threadIdx.x;
+  if (i < n) dst[i] = c.e[i];
+  if (check_word && i == 0) *check_word = 0;  // the array keeps the previous call's contents
+}
+
 }  // namespace
 
 extern "C" int emoe_moe_forward_routed_static(int device, const emoe_layer_desc* desc, const void* x, int T,
@@ -97,6 +112,7 @@ extern "C" int emoe_moe_forward_routed_static(int device, const emoe_layer_desc*
     for (int m = 0; m < nmat; ++m) {
       if (!host_experts[e].packed[m] || !host_experts[e].scales[m]) return EMOE_ERR_INVALID_ARG;
       if (!aligned(host_experts[e].packed[m], 16)) return EMOE_ERR_ALIGNMENT;
+      if (!aligned(host_experts[e].scales[m], 4)) return EMOE_ERR_ALIGNMENT;
     }
   }
   // the fixed array bounds the problem size: refuse anything that does not fit
@@ -115,16 +131,6 @@ extern "C" int emoe_moe_forward_routed_static(int device, const emoe_layer_desc*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int P = T * L.top_k;
 
-  // the expert table goes through a small host staging copy into the scratch array
-  ExpertDev host_tab[EMOE_MAX_EXPERTS];
-  for (int e = 0; e < L.E; ++e) {
-    host_tab[e].bits = host_experts[e].bits;
-    host_tab[e].pad = 0;
-    for (int m = 0; m < 3; ++m) {
-      host_tab[e].packed[m] = static_cast<const uint8_t*>(host_experts[e].packed[m]);
-      host_tab[e].scales[m] = host_experts[e].scales[m];
-    }
-  }
   ExpertDev* table = reinterpret_cast<ExpertDev*>(ws + w.table);
   int* check = reinterpret_cast<int*>(ws + w.check);
   int32_t* counts = reinterpret_cast<int32_t*>(ws + w.counts);
@@ -139,11 +145,23 @@ extern "C" int emoe_moe_forward_routed_static(int device, const emoe_layer_desc*
   do {                 \
     if ((call) != cudaSuccess) return EMOE_ERR_CUDA; \
   } while (0)
-  // pageable source: the copy is staged by the driver before the call returns, so the
-  // stack array may go out of scope
-  EMOE_TRY(cudaMemcpyAsync(table, host_tab, sizeof(ExpertDev) * L.E, cudaMemcpyHostToDevice, st));
-  // the array keeps whatever the previous call left: the check word must start at zero
-  EMOE_TRY(cudaMemsetAsync(check, 0, sizeof(int), st));
+  // the expert table travels as launch parameters; the first chunk's kernel also clears the check
+  // word (the array keeps whatever the previous call left)
+  for (int e0 = 0; e0 < L.E; e0 += TABLE_CHUNK) {
+    TableChunk chunk;
+    const int n = L.E - e0 < TABLE_CHUNK ? L.E - e0 : TABLE_CHUNK;
+    for (int i = 0; i < n; ++i) {
+      chunk.e[i].bits = host_experts[e0 + i].bits;
+      chunk.e[i].pad = 0;
+      for (int m = 0; m < 3; ++m) {
+        chunk.e[i].packed[m] = static_cast<const uint8_t*>(host_experts[e0 + i].packed[m]);
+        chunk.e[i].scales[m] = host_experts[e0 + i].scales[m];
+      }
+    }
+    for (int i = n; i < TABLE_CHUNK; ++i) chunk.e[i] = ExpertDev{};
+    write_table_kernel<<<1, TABLE_CHUNK, 0, st>>>(chunk, table + e0, n, e0 == 0 ? check : nullptr);
+    EMOE_TRY(cudaGetLastError());
+  }
   EMOE_TRY(launch_permute(ids, P, L.E, counts, off, perm, slot_of_pair, check, st));
   if (ffn_mma_supported(L)) {
     EMOE_TRY(launch_scatter_x(L, table, x, ids, perm, off, nullptr, xs, P, false, 1, INT_MAX, st));
@@ -158,4 +176,17 @@ extern "C" int emoe_moe_forward_routed_static(int device, const emoe_layer_desc*
   }
 #undef EMOE_TRY
   return EMOE_OK;
+}
+
+extern "C" int emoe_static_device_status(int device, void* stream) {
+  if (device < 0 || device >= MAX_DEVICES) return EMOE_ERR_INVALID_ARG;
+  if (cudaSetDevice(device) != cudaSuccess) return EMOE_ERR_CUDA;
+  if (!g_scratch_addr[device]) return EMOE_OK;  // no call has run on this device yet
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  // the check word is the first thing in the scratch array (StaticLayout::check == 0)
+  if (cudaMemcpyAsync(&word, g_scratch_addr[device], sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return EMOE_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return EMOE_ERR_CUDA;
+  if (word & CHECK_WAIT_TIMEOUT) return EMOE_ERR_TIMEOUT;
+  return word ? EMOE_ERR_DEVICE_CHECK : EMOE_OK;
 }

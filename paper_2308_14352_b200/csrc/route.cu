@@ -212,6 +212,8 @@ __global__ void __launch_bounds__(1024)
     if (lane == 31) off[E] = incl;
   }
   __syncthreads();
+  // pairs with an id outside [0, E) own no slot: the slots behind the last valid one read as "no pair"
+  for (int p = off[E] + tid; p < n; p += 1024) perm[p] = -1;
 
   for (int base = 0; base < n; base += 1024) {
     for (int i = tid; i < 32 * E; i += 1024) wcnt[i] = 0;

@@ -68,6 +68,8 @@ def _table_from(acquired, ids_active, bits):
     entries = []
     for e, b in enumerate(bits):
         src = by_e.get(e, first)
+        if e not in by_e:
+            b = bits[ids_active[0]]      # a borrowed entry carries the width of the expert it borrows from
         entries.append((b, [src.packed[m] for m in range(3) if src.packed[m]], [src.scales[m] for m in range(3) if src.scales[m]]))
     return B.make_expert_table(entries)
 
@@ -224,3 +226,67 @@ def test_cache_argument_errors():
     finally:
         torch.cuda.synchronize()
         B.emoe_destroy(ctx)
+
+
+def test_cached_stack_two_layers_at_the_mixtral_shape():
+    """The cached pipeline at the full layer shape (two layers of the Mixtral-like stack): a
+    2048-token prefill, then single-token decode steps.  Weights are drawn on the device by the
+    stack's seeded generator; the checker packs the same matrices itself (compared byte for byte
+    with what the stack staged in host memory) and evaluates sampled outputs."""
+    from paper_2308_14352_b200.cached_stack import CachedStack
+
+    w = inputs.WORKLOADS["mixtral_stack_cached"]
+    sh, bits = w.shape, list(w.fixed_bits)
+    T = 2048
+    stack = CachedStack(sh, 2, bits, n_slots=12, max_tokens=T, seed=w.seed)
+    try:
+        def oracle_expert(l, e):
+            ps = [oracle.pack_expert(stack.draw_matrix(l, e, m).cpu().numpy(), bits[e], sh.group, sh.scale_dtype)
+                  for m in range(sh.n_matrices)]
+            for m, (p, s_) in enumerate(ps):     # the staged copy is the library's packing of the same matrix
+                assert np.array_equal(stack.host[l][e][0][m].numpy().reshape(p.shape), p)
+                assert np.array_equal(stack.host[l][e][1][m].numpy().astype(np.float32).reshape(s_.shape), s_)
+            return [p for p, _ in ps], [s_ for _, s_ in ps]
+
+        def check(l, x, ids, gates, y, tokens, channels):
+            worst, cache = 0.0, {}
+            for t in tokens:
+                acc = np.zeros(len(channels))
+                for j in range(sh.top_k):
+                    e = int(ids[t, j])
+                    if e not in cache:
+                        cache[e] = oracle_expert(l, e)
+                    p, s_ = cache[e]
+                    h = oracle.hidden_for_pair(x[t], sh.d_ff, sh.act, sh.group, True, bits[e], p, s_)
+                    acc += float(gates[t, j]) * oracle.output_channels(h, sh.group, bits[e], p[2], s_[2], channels)
+                worst = max(worst, float(np.abs(y[t, channels] - acc).max()))
+            return worst / float(np.abs(y).max())
+
+        channels = np.arange(3, sh.d_model, 131, dtype=np.int32)
+        # prefill
+        x_host = [inputs.activations(w.seed, l, T, sh.d_model, "bf16") for l in range(2)]
+        xs = [torch.from_numpy(x).to(stack.dev).to(torch.bfloat16) for x in x_host]
+        outs = []
+        picks = stack.forward_stack(xs, outputs=outs)
+        stack.compute.synchronize()
+        assert B.emoe_device_status(stack.ctx, stack.compute.cuda_stream) == B.OK
+        gates, y = outs[1][0].cpu().numpy(), outs[1][1].cpu().numpy()
+        assert np.isfinite(y).all()
+        e1 = int(picks[1][0, 0])
+        owners = [t for t in range(T) if e1 in picks[1][t]]
+        assert check(1, x_host[1], picks[1], gates, y, [owners[2], owners[-2]], channels) <= 2e-3
+        # decode: three single-token steps, the last one checked on both layers
+        for step in range(3):
+            x_host = [inputs.activations(w.seed, l, 1, sh.d_model, "bf16", batch_tag=10 + step) for l in range(2)]
+            xs = [torch.from_numpy(x).to(stack.dev).to(torch.bfloat16) for x in x_host]
+            outs = []
+            picks = stack.forward_stack(xs, outputs=outs)
+        stack.compute.synchronize()
+        assert B.emoe_device_status(stack.ctx, stack.compute.cuda_stream) == B.OK
+        for l in range(2):
+            gates, y = outs[l][0].cpu().numpy(), outs[l][1].cpu().numpy()
+            assert check(l, x_host[l], picks[l], gates, y, [0], channels) <= 2e-3
+        st = B.emoe_cache_get_stats(stack.ctx)
+        assert st["bytes_copied"] > 0 and st["hits"] + st["misses"] > 0
+    finally:
+        stack.close()

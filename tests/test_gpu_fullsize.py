@@ -108,7 +108,14 @@ def _sampled_output_check(w, layer_idx, bits, x, ids, gates, y, tokens, channels
     return worst / float(np.abs(y).max())
 
 
-@pytest.mark.parametrize("T", [1, 16])
+def _rank_in_expert(ids, t, j):
+    """Position of pair (t, j) among the pairs of its expert in permutation order."""
+    flat = ids.reshape(-1)
+    p = t * ids.shape[1] + j
+    return int(np.count_nonzero(flat[:p] == flat[p]))
+
+
+@pytest.mark.parametrize("T", [1, 4, 16, 32])
 def test_mixtral_decode_sampled_outputs(T):
     w = inputs.WORKLOADS["mixtral_decode"]
     sh, bits = w.shape, inputs.expert_bits(w, 0)
@@ -125,8 +132,46 @@ def test_mixtral_decode_sampled_outputs(T):
     np.testing.assert_allclose(gates.sum(axis=1), 1.0, rtol=1e-5)
     rng = np.random.default_rng(T)
     tokens = [0] if T == 1 else [0, int(rng.integers(1, T))]
+    if T == 32:
+        # a pair that sits behind the first eight of its expert: it is served by a later pass (or
+        # a later token tile) than the expert's first tokens
+        ranks = [(max(_rank_in_expert(ids, t, j) for j in range(sh.top_k)), t) for t in range(T)]
+        deep_rank, deep_t = max(ranks)
+        assert deep_rank >= 8, ranks
+        tokens = [0, deep_t]
     channels = np.concatenate([[0, 1, 4095], rng.integers(0, sh.d_model, 29)]).astype(np.int32)
     assert _sampled_output_check(w, 0, bits, x, ids, gates, y, tokens, channels) <= 2e-3
+    assert np.isfinite(y).all()
+
+
+def test_mixtral_shape_prefill_2048_tokens_sampled_outputs():
+    """The Mixtral-like layer with 2048 tokens (about 512 per expert) on the automatic path: the
+    many-token grouped GEMM at its full shape.  Routing and permutation in full, one expert byte
+    for byte, outputs of tokens that sit in different token groups of one expert, on channels
+    spread over the 128-row blocks."""
+    w = inputs.WORKLOADS["mixtral_decode"]
+    sh, bits, T = w.shape, inputs.expert_bits(w, 0), 2048
+    x, Wr, _ = inputs.layer_tensors(w, 0, T, batch_tag=5)
+    with layer.MoELayer(sh, bits, max_tokens=T) as moe:
+        _pack_layer_on_gpu(moe, w, 0)
+        y, ids, gates, perm = moe.forward(x, Wr)
+        e0 = int(ids[0, 0])
+        p_ref, s_ref = _oracle_expert(w, 0, e0, bits[e0])
+        for m in range(3):
+            assert np.array_equal(moe.packed_host(e0, m), p_ref[m])
+            assert np.array_equal(moe.scales_host(e0, m).astype(np.float32), s_ref[m])
+    strict = _check_routing(w, x, Wr, None, ids, gates, perm)
+    assert strict >= 0.9 * T
+    assert np.isfinite(y).all()
+    # two tokens of expert e0 far apart in its token list (ranks 3 and 300+: different 128-token
+    # tiles and different tile groups), plus one more token sharing an expert with them
+    owners = [(t, j) for t in range(T) for j in range(sh.top_k) if ids[t, j] == e0]
+    assert len(owners) > 320, len(owners)
+    t_near, t_far = owners[3][0], owners[310][0]
+    assert _rank_in_expert(ids, *owners[310]) == 310
+    channels = np.arange(5, sh.d_model, 97, dtype=np.int32)     # every 128-row block is hit
+    assert len(set((channels // 128).tolist())) == sh.d_model // 128
+    assert _sampled_output_check(w, 0, bits, x, ids, gates, y, [t_near, t_far], channels) <= 2e-3
 
 
 def test_switch_large_prefill_zipf_sampled_outputs():

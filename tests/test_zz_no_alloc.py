@@ -2,8 +2,8 @@
 allocate device memory (a framework that owns the device heap, a plug-in with a fixed pool,
 a latency-critical loop).  It takes no context and keeps its intermediates in a fixed array
 inside the library, so this test builds the inputs with plain torch tensors, never creates an
-emoe context for the call under test, and checks the result against the ordinary
-emoe_moe_forward_routed on the same inputs.  Two calls in a row with different inputs show
+emoe context for the call under test, and checks the result against the CPU checker and
+against the ordinary emoe_moe_forward_routed on the same inputs.  Two calls in a row with different inputs show
 that what the first call left in the shared array does not leak into the second.
 
 The file name sorts last on purpose: a run that stops at the first failure has then already
@@ -14,7 +14,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2308_14352_b200 import binding as B, inputs, layer
+from tests.helpers import oracle_pack_layer, rel_to_max
 
 pytestmark = pytest.mark.gpu
 
@@ -36,6 +38,7 @@ def test_static_entry_point_matches_the_context_one_twice_in_a_row(act, adt, gro
     with layer.MoELayer(shape, bits, max_tokens=16) as moe:        # only to pack weights and for the reference
         W, _, _, _ = _case(shape, bits, 1, 40)
         moe.pack_from_host(W)
+        packed, scales = oracle_pack_layer(W, shape, bits)
         for call, (T, seed) in enumerate([(16, 41), (5, 42)]):
             _, x, ids, gates = _case(shape, bits, T, seed)
             y_ref, _ = moe.forward_routed(x, ids, gates)
@@ -48,8 +51,41 @@ def test_static_entry_point_matches_the_context_one_twice_in_a_row(act, adt, gro
             torch.cuda.synchronize()
             y = y.cpu().numpy()
             assert np.isfinite(y).all()
+            y_cpu = oracle.moe_ffn_combine(x, shape.d_ff, shape.act, shape.group, adt == "bf16", bits, packed, scales,
+                                           ids, gates)
+            assert rel_to_max(y, y_cpu) <= tol, (call, rel_to_max(y, y_cpu))     # against the CPU checker
             err = np.abs(y - y_ref).max() / np.abs(y_ref).max()
-            assert err <= tol, (call, err)
+            assert err <= tol, (call, err)                                       # against the context entry point
+            assert B.emoe_static_device_status(0) == B.OK
+
+
+def test_static_entry_point_reports_an_expert_id_out_of_range():
+    """Ids outside [0, E) are dropped (their terms are missing from y) and leave a flag that the
+    status call returns; the next call clears it."""
+    shape = inputs.LayerShape(256, 512, 4, 2, "relu", "softmax", 128, "f16", "bf16")
+    bits = [4, 2, 8, 4]
+    with layer.MoELayer(shape, bits, max_tokens=8) as moe:
+        W, x, ids, gates = _case(shape, bits, 6, 43)
+        moe.pack_from_host(W)
+        packed, scales = oracle_pack_layer(W, shape, bits)
+        xd = moe.to_device_x(x)
+        gd = torch.from_numpy(gates).cuda()
+        y = torch.zeros((6, shape.d_model), dtype=torch.float32, device="cuda")
+        bad = ids.copy()
+        bad[2, 1] = 7                      # E = 4
+        idd = torch.from_numpy(bad).cuda()
+        B.emoe_moe_forward_routed_static(0, moe.desc, xd.data_ptr(), 6, idd.data_ptr(), gd.data_ptr(), moe.table,
+                                         y.data_ptr(), 0)
+        assert B.emoe_static_device_status(0) == B.ERR_DEVICE_CHECK
+        # the dropped pair contributes nothing: same as a zero gate on a valid expert
+        ids_eq, gates_eq = ids.copy(), gates.copy()
+        gates_eq[2, 1] = 0.0
+        y_cpu = oracle.moe_ffn_combine(x, shape.d_ff, "relu", 128, True, bits, packed, scales, ids_eq, gates_eq)
+        assert rel_to_max(y.cpu().numpy(), y_cpu) <= 2e-3
+        idd = torch.from_numpy(ids).cuda()
+        B.emoe_moe_forward_routed_static(0, moe.desc, xd.data_ptr(), 6, idd.data_ptr(), gd.data_ptr(), moe.table,
+                                         y.data_ptr(), 0)
+        assert B.emoe_static_device_status(0) == B.OK
 
 
 def test_static_entry_point_rejects_what_does_not_fit():
