@@ -204,13 +204,28 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
                             void* stream);
 
 /* Selects the expert-FFN kernel family: 0 = automatic (default), 1 = the CUDA-core grouped
- * GEMV, 2 = the tensor-core kernel with register-staged weight loads, 3 = the tensor-core kernel
- * with the TMA-staged weight pipeline, 4 = the tcgen05 grouped GEMM (fp16 operands; meant for
- * many tokens per expert), 5 = both of the last two in one call: experts with at most 32 tokens
- * take the streaming kernel, the others the grouped GEMM (what 0 picks for large batches).
- * 2 to 5 fail with EMOE_ERR_UNSUPPORTED in forward calls whose shape they do not take.  For tests
+ * GEMV, 2 = the tensor-core kernel with register-staged weight loads, 3 = the fp16 mma.sync
+ * kernel with the TMA-staged weight pipeline, 4 = the tcgen05 grouped GEMM (fp16 operands; meant
+ * for many tokens per expert), 6 = the weight-streaming kernel on 8-bit integer tcgen05 operands
+ * (what 0 picks for decode batches), 5 = 6 and 4 in one call: experts with at most 32 tokens take
+ * the streaming kernel, the others the grouped GEMM (what 0 picks for large batches).
+ * 2 to 6 fail with EMOE_ERR_UNSUPPORTED in forward calls whose shape they do not take.  For tests
  * and measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);
+
+/* Every wait inside the weight-streaming kernel (on a pipeline stage, on tensor memory, on the
+ * completion of an expert's hidden vectors) is bounded: after `polls` unsuccessful polls the
+ * kernel records the failure, lets its copies in flight land, releases what it holds and
+ * returns; emoe_device_status then reports EMOE_ERR_TIMEOUT and the context stays usable.  This
+ * is the library's form of failure detection (the paper's only failure path is a mispredicted
+ * preload, Section 3.3, which is corrected by loading the right expert).  polls = 0 restores the
+ * default (about 0.2 s).  Applies to the forward calls that follow. */
+int emoe_set_wait_limit(emoe_ctx* ctx, unsigned polls);
+
+/* Test hook for the above: the second projection of every expert waits for `extra` more
+ * completions of its first projection than will ever be counted, so that its bounded wait runs
+ * out.  0 (the default) in any real use.  No counterpart in the paper. */
+int emoe_debug_expect_extra_completions(emoe_ctx* ctx, int extra);
 
 /* Programmatic dependent launch along the kernels of a forward call (on by default): each
  * kernel may start its prologue while the one in front drains.  Results are identical either

@@ -32,7 +32,7 @@ struct TableEntry {
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-  size_t ids, gates, counts, off, perm, slot_of_pair, plan, xs, hidden, o_part, total;
+  size_t ids, gates, counts, off, perm, slot_of_pair, plan, xs, hidden, xsc, hsc, o_part, total;
   int ksplit;
 };
 
@@ -65,6 +65,7 @@ WorkspaceLayout make_layout(const LayerDims& L, int T) {
   w.ksplit = 1;
   if (ffn_mma_supported(L)) w.ksplit = ffn_mma_ksplit(L, T);
   if (ffn_tma_supported(L) && ffn_tma_ksplit(L, T) > w.ksplit) w.ksplit = ffn_tma_ksplit(L, T);
+  if (ffn_i8_supported(L) && ffn_i8_ksplit(L, T) > w.ksplit) w.ksplit = ffn_i8_ksplit(L, T);
   size_t o = 0;
   w.ids = o;          o += align_up(P * 4);
   w.gates = o;        o += align_up(P * 4);
@@ -75,6 +76,9 @@ WorkspaceLayout make_layout(const LayerDims& L, int T) {
   w.plan = o;         o += 2 * align_up(plan_bytes(L.E));  // two plans: one per kernel family of a forward call
   w.xs = o;           o += align_up(L.act_bf16 ? P * L.d_model * 2 : 0);
   w.hidden = o;       o += align_up(P * L.d_ff * (L.act_bf16 ? 2 : 4));
+  // block scales of the integer activations (int8 tensor-core kernel): one fp32 per 128 inputs
+  w.xsc = o;          o += align_up(ffn_i8_supported(L) ? P * (L.d_model / 128) * 4 : 0);
+  w.hsc = o;          o += align_up(ffn_i8_supported(L) ? P * (L.d_ff / 128) * 4 : 0);
   w.o_part = o;       o += align_up(static_cast<size_t>(w.ksplit) * P * L.d_model * 4);
   w.total = o;
   return w;
@@ -98,6 +102,8 @@ struct emoe_ctx {
   bool pdl = true;  // programmatic dependent launch along the kernel chain of a forward call
   bool fuse_projections = true;  // weight-streaming kernel: both projections in one launch
   bool timing = false;
+  unsigned wait_limit = 0;  // polls before a wait inside the int8 streaming kernel gives up (0 = its default)
+  int dep_extra = 0;        // test hook: extra completions the second projection waits for
   int kernels_last = 0;  // kernels the last forward call enqueued
   ExpertCache* cache = nullptr;  // expert cache (cache.cu), optional
   std::vector<cudaEvent_t> table_events;  // per table block: its upload has left the pinned mirror
@@ -260,6 +266,8 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   int* plan = reinterpret_cast<int*>(ws + w.plan);
   __nv_bfloat16* xs = reinterpret_cast<__nv_bfloat16*>(ws + w.xs);
   void* hidden = ws + w.hidden;
+  float* xsc = reinterpret_cast<float*>(ws + w.xsc);
+  float* hsc = reinterpret_cast<float*>(ws + w.hsc);
   float* o_part = reinterpret_cast<float*>(ws + w.o_part);
 
   const int32_t* ids_use = ids;
@@ -272,21 +280,25 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
                                       L.top_k, L.gate_mode == EMOE_GATE_SOFTMAX_RENORM, ids, gates, nullptr, st));
   }
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
+  const bool can_i8 = ffn_i8_supported(L) && tmaps != nullptr;
   const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
   // many tokens per expert: the tcgen05 grouped GEMM; otherwise the weight-streaming kernels
   const bool many_tokens = ffn_many_tokens(L, T);
   // skewed loads: experts with few tokens stream through the TMA kernel, the others take the
   // tcgen05 grouped GEMM, in the same forward call
-  const bool use_hybrid = can_umma && can_tma && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens));
+  const bool use_hybrid = can_umma && can_i8 && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens));
   const bool use_umma = !use_hybrid && can_umma && (ctx->ffn_path == 4 || (ctx->ffn_path == 0 && many_tokens));
-  const bool use_tma = !use_hybrid && !use_umma && can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
+  // the weight-streaming kernels: int8 tensor-core operands by default, the fp16 mma.sync one on request
+  const bool use_i8 = !use_hybrid && !use_umma && can_i8 && (ctx->ffn_path == 0 || ctx->ffn_path == 6);
+  const bool use_tma = !use_hybrid && !use_umma && !use_i8 && can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
   const bool use_mma = ffn_mma_supported(L) && ctx->ffn_path != 1;
   if (ctx->ffn_path == 2 && !use_mma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 3 && !use_tma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 4 && !use_umma) return EMOE_ERR_UNSUPPORTED;
   if (ctx->ffn_path == 5 && !use_hybrid) return EMOE_ERR_UNSUPPORTED;
-  // small batches on the streaming kernel: permutation, scatter and plan in one launch
-  const bool one_launch_permute = use_tma && ctx->fuse_projections && permute_scatter_supported(L, P);
+  if (ctx->ffn_path == 6 && !use_i8) return EMOE_ERR_UNSUPPORTED;
+  // small batches on the streaming kernels: permutation, scatter and plan in one launch
+  const bool one_launch_permute = (use_tma || use_i8) && ctx->fuse_projections && permute_scatter_supported(L, P);
   if (!one_launch_permute)
     EMOE_LAUNCH(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
   int ksplit = 1;
@@ -309,14 +321,13 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
 #ifndef EMOE_HYBRID_TOKENS
 #define EMOE_HYBRID_TOKENS 32
 #endif
-#ifndef EMOE_HYBRID_TILES
-#define EMOE_HYBRID_TILES 1
+#ifndef EMOE_HYBRID_TILE
+#define EMOE_HYBRID_TILE 16  // tokens per pass of the streaming family
 #endif
     constexpr int HYBRID_STREAM_TOKENS = EMOE_HYBRID_TOKENS;
     int* plan_heavy = reinterpret_cast<int*>(reinterpret_cast<char*>(plan) + align_up(plan_bytes(L.E)));
-    __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
-    ksplit = ffn_tma_ksplit(L, T);
-    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, 1, HYBRID_STREAM_TOKENS, st));
+    ksplit = ffn_i8_ksplit(L, T);
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, xsc, P, 2, 1, HYBRID_STREAM_TOKENS, st));
     EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan_heavy, xs, P, HYBRID_STREAM_TOKENS + 1, INT_MAX, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     // the tcgen05 kernel writes plane 0 only: the other split-K planes of its slots must read as zero
@@ -324,10 +335,10 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       EMOE_CUDA(ctx, cudaMemsetAsync(o_part + static_cast<size_t>(P) * L.d_model, 0,
                                      static_cast<size_t>(ksplit - 1) * P * L.d_model * sizeof(float), st));
     if (ctx->fuse_projections) {
-      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, ctx->dep_extra, ctx->check_word, st));
     } else {
-      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
-      EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 1, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_i8(1, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
     }
     EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, P, ctx->check_word, st));
     EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, P, ctx->check_word, st));
@@ -342,13 +353,37 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, P, ctx->check_word, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
     EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
+  } else if (use_i8) {
+    ksplit = ffn_i8_ksplit(L, T);
+    if (one_launch_permute)
+      EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, xsc, P, 2,
+                                              ctx->check_word, st));
+    else
+      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, xsc, P, 2, 1, INT_MAX, st));
+    if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
+    if (ctx->fuse_projections) {
+      // one launch: an expert's second projection starts when its hidden vectors are complete
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit,
+                                     ctx->dep_extra, ctx->check_word, st));
+      if (ev[1]) {  // one interval only: the end event of the triple stays unused
+        EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+        ctx->events_one_launch[ctx->events_used / 3 - 1] = 1;
+        ev[2] = nullptr;
+      }
+    } else {
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 1, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit, 0,
+                                     ctx->check_word, st));
+      if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+      EMOE_LAUNCH(ctx, launch_ffn_i8(1, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit, 0,
+                                     ctx->check_word, st));
+    }
   } else if (use_tma) {
     ksplit = ffn_tma_ksplit(L, T);
     if (one_launch_permute)
-      EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, P, true,
+      EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, nullptr, P, 1,
                                               ctx->check_word, st));
     else
-      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, P, true, 1, INT_MAX, st));
+      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, nullptr, P, 1, 1, INT_MAX, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
     if (ctx->fuse_projections) {
@@ -366,7 +401,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     }
   } else if (use_mma) {
     ksplit = ffn_mma_ksplit(L, T);
-    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, P, false, 1, INT_MAX, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, nullptr, P, 0, 1, INT_MAX, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_LAUNCH(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
@@ -614,8 +649,20 @@ int emoe_set_fused_projections(emoe_ctx* ctx, int enabled) {
   return EMOE_OK;
 }
 
+int emoe_set_wait_limit(emoe_ctx* ctx, unsigned polls) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  ctx->wait_limit = polls;
+  return EMOE_OK;
+}
+
+int emoe_debug_expect_extra_completions(emoe_ctx* ctx, int extra) {
+  if (!ctx || extra < 0) return EMOE_ERR_INVALID_ARG;
+  ctx->dep_extra = extra;
+  return EMOE_OK;
+}
+
 int emoe_set_ffn_path(emoe_ctx* ctx, int path) {
-  if (!ctx || path < 0 || path > 5) return EMOE_ERR_INVALID_ARG;
+  if (!ctx || path < 0 || path > 6) return EMOE_ERR_INVALID_ARG;
   ctx->ffn_path = path;
   return EMOE_OK;
 }

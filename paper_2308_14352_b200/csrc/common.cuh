@@ -105,17 +105,18 @@ int ffn_mma_ksplit(const LayerDims& L, int T);
 int ffn_token_tiles(const LayerDims& L, int T);
 bool ffn_many_tokens(const LayerDims& L, int T);
 // plan (nullable): plan_bytes(E) bytes, the work plan for the persistent TMA kernels, filled by block 0.
-// to_f16: store the rows as fp16 (saturating) instead of bf16, same layout (the TMA-staged kernel's input).
+// fmt: 0 = bf16, 1 = fp16 (saturating; same layout: the TMA-staged kernel's input), 2 = two-limb
+// block-scaled integers (act_q.cuh: the int8 tensor-core kernel's input; xsc receives the block scales).
 // cnt_lo .. cnt_hi: only experts with that many tokens are listed in the plan and have their rows
 // written (1 .. INT_MAX: all activated experts); lets two kernel families share one forward call.
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
-                             const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
-                             bool to_f16, int cnt_lo, int cnt_hi, cudaStream_t st);
+                             const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, float* xsc, int n_pairs,
+                             int fmt, int cnt_lo, int cnt_hi, cudaStream_t st);
 // Permutation + scatter + plan in one launch (one CTA per pair) for batches of at most 1024 pairs.
 bool permute_scatter_supported(const LayerDims& L, int n_pairs);
 cudaError_t launch_permute_scatter(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                    int32_t* counts, int32_t* off, int32_t* perm, int32_t* slot_of_pair, int* plan,
-                                   __nv_bfloat16* xs, int n_pairs, bool to_f16, int* check_word, cudaStream_t st);
+                                   __nv_bfloat16* xs, float* xsc, int n_pairs, int fmt, int* check_word, cudaStream_t st);
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,
                            const int32_t* off, __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs,
                            int T, cudaStream_t st);
@@ -132,6 +133,18 @@ cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, c
                            const void* tmaps, const __nv_bfloat16* xs, const int32_t* off, int* plan,
                            __nv_bfloat16* hidden, float* o_part, int ksplit, int n_pairs, int T, int token_tiles,
                            int* check_word, cudaStream_t st);
+
+// The weight-streaming kernel on 8-bit integer tensor-core operands (tcgen05 kind::i8, accumulators
+// and unpacked codes in tensor memory).  xq / hq: activations as two-limb block-scaled integers
+// [n_pairs][2][K] with block scales xsc / hsc [n_pairs][K/128] (act_q.cuh).  token_tile: tokens
+// per pass (8, 16 or 32), 0 = by the routing statistics of (L, T).  wait_limit: polls before a
+// wait inside the kernel gives up (0 = default); dep_extra: test hook, 0 in production.
+bool ffn_i8_supported(const LayerDims& L);
+int ffn_i8_ksplit(const LayerDims& L, int T);
+int ffn_i8_token_tile(const LayerDims& L, int T);
+cudaError_t launch_ffn_i8(int phase_begin, int phase_end, const LayerDims& L, const void* wmaps, const void* xq,
+                          const float* xsc, int* plan, void* hq, float* hsc, float* o_part, int ksplit, int n_pairs,
+                          int T, int token_tile, unsigned wait_limit, int dep_extra, int* check_word, cudaStream_t st);
 
 int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
                    uint32_t box_inner, uint32_t box_outer);

@@ -21,6 +21,7 @@
 #include <cmath>
 
 #include "common.cuh"
+#include "act_q.cuh"
 #include "ffn_tile.cuh"
 
 namespace emoe {
@@ -266,12 +267,26 @@ __device__ __forceinline__ void scatter_row(const __nv_bfloat16* __restrict__ sr
   }
 }
 
+// One activation row into slot `slot` of the activation buffer, in the format the expert kernel
+// wants: fmt 0 = bf16 and 1 = fp16 in the k-interleaved layout (ffn_tile.cuh), 2 = two-limb
+// block-scaled integers with their block scales (act_q.cuh; the slot's two limb rows take the
+// same 2 * d bytes as a 16-bit row).
+__device__ __forceinline__ void scatter_any(const __nv_bfloat16* __restrict__ src_row, __nv_bfloat16* __restrict__ xs,
+                                            float* __restrict__ xsc, int slot, int d, int bits, int fmt) {
+  if (fmt == 2) {
+    int8_t* q = reinterpret_cast<int8_t*>(xs) + static_cast<size_t>(slot) * 2 * d;
+    act_q_row(src_row, q, q + d, xsc + static_cast<size_t>(slot) * (d / 128), d, bits);
+  } else {
+    scatter_row(src_row, xs + static_cast<size_t>(slot) * d, d, bits, fmt);
+  }
+}
+
 // x rows -> expert-sorted order, in the activation layout of the owning expert's bitwidth
 __global__ void __launch_bounds__(128)
     scatter_x_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
                      const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
-                     int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int to_f16, int cnt_lo, int cnt_hi,
-                     __nv_bfloat16* __restrict__ xs) {
+                     int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int fmt, int cnt_lo, int cnt_hi,
+                     __nv_bfloat16* __restrict__ xs, float* __restrict__ xsc) {
   pdl_wait();
   pdl_trigger();
   if (plan && blockIdx.x == 0 && threadIdx.x < 32) build_plan(plan, experts, off, E, cnt_lo, cnt_hi, threadIdx.x);
@@ -282,7 +297,7 @@ __global__ void __launch_bounds__(128)
   if (e_slot < 0 || e_slot >= E) return;  // a slot the permutation did not write (stale entry behind a dropped pair)
   const int cnt_slot = off[e_slot + 1] - off[e_slot];
   if (cnt_slot < cnt_lo || cnt_slot > cnt_hi) return;  // this expert's rows belong to another kernel family
-  scatter_row(x + static_cast<size_t>(pair / top_k) * d, xs + static_cast<size_t>(slot) * d, d, experts[e_slot].bits, to_f16);
+  scatter_any(x + static_cast<size_t>(pair / top_k) * d, xs, xsc, slot, d, experts[e_slot].bits, fmt);
 }
 
 // Permutation and scatter in one launch for small batches (at most PS_MAX_PAIRS pairs): one CTA
@@ -293,10 +308,10 @@ __global__ void __launch_bounds__(128)
 constexpr int PS_MAX_PAIRS = 1024;
 __global__ void __launch_bounds__(128)
     permute_scatter_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
-                           const int32_t* __restrict__ ids, int E, int top_k, int d, int n_pairs, int to_f16,
+                           const int32_t* __restrict__ ids, int E, int top_k, int d, int n_pairs, int fmt,
                            int32_t* __restrict__ counts, int32_t* __restrict__ off, int32_t* __restrict__ perm,
                            int32_t* __restrict__ slot_of_pair, int* __restrict__ plan, int* __restrict__ check_word,
-                           __nv_bfloat16* __restrict__ xs) {
+                           __nv_bfloat16* __restrict__ xs, float* __restrict__ xsc) {
   __shared__ int s_ids[PS_MAX_PAIRS];
   __shared__ int s_off[EMOE_MAX_EXPERTS + 1];
   __shared__ int s_red[2][4];
@@ -356,7 +371,7 @@ __global__ void __launch_bounds__(128)
     perm[slot] = p;
     slot_of_pair[p] = slot;
   }
-  scatter_row(x + static_cast<size_t>(p / top_k) * d, xs + static_cast<size_t>(slot) * d, d, experts[e].bits, to_f16);
+  scatter_any(x + static_cast<size_t>(p / top_k) * d, xs, xsc, slot, d, experts[e].bits, fmt);
 }
 
 
@@ -396,20 +411,20 @@ int ffn_mma_ksplit(const LayerDims& L, int T) {
 }
 
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
-                             const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, int n_pairs,
-                             bool to_f16, int cnt_lo, int cnt_hi, cudaStream_t st) {
+                             const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, float* xsc, int n_pairs,
+                             int fmt, int cnt_lo, int cnt_hi, cudaStream_t st) {
   return launch_chain(scatter_x_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
-                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, to_f16 ? 1 : 0, cnt_lo, cnt_hi, xs);
+                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, fmt, cnt_lo, cnt_hi, xs, xsc);
 }
 
 bool permute_scatter_supported(const LayerDims& L, int n_pairs) { return n_pairs <= PS_MAX_PAIRS && L.E <= EMOE_MAX_EXPERTS; }
 
 cudaError_t launch_permute_scatter(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                    int32_t* counts, int32_t* off, int32_t* perm, int32_t* slot_of_pair, int* plan,
-                                   __nv_bfloat16* xs, int n_pairs, bool to_f16, int* check_word, cudaStream_t st) {
+                                   __nv_bfloat16* xs, float* xsc, int n_pairs, int fmt, int* check_word, cudaStream_t st) {
   return launch_chain(permute_scatter_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x),
-                      ids, L.E, L.top_k, L.d_model, n_pairs, to_f16 ? 1 : 0, counts, off, perm, slot_of_pair, plan, check_word,
-                      xs);
+                      ids, L.E, L.top_k, L.d_model, n_pairs, fmt, counts, off, perm, slot_of_pair, plan, check_word,
+                      xs, xsc);
 }
 
 cudaError_t launch_ffn_mma(int phase, const LayerDims& L, const ExpertDev* experts, const __nv_bfloat16* in,

@@ -100,6 +100,44 @@ def test_forward_tma_pipeline_path(act, group, sdt, d, f, E, k, gate, bits, T):
     assert np.array_equal(y_fused, y_split)
 
 
+I8_CASES = TMA_CASES + [
+    ("relu", 128, "f16", 768, 3072, 32, 1, "softmax", [2, 4, 8, 4] * 8, 64),                # many experts, 2 tokens each
+    ("swiglu", 128, "f16", 512, 1024, 8, 2, "softmax_renorm", [8, 8, 4, 4, 2, 2, 4, 8], 4),
+    ("relu", 256, "f16", 1024, 512, 2, 1, "softmax", [2, 4], 40),                          # 32-token tiles, two passes
+]
+
+
+@pytest.mark.parametrize("act,group,sdt,d,f,E,k,gate,bits,T", I8_CASES)
+def test_forward_int8_tensor_core_streaming_path(act, group, sdt, d, f, E, k, gate, bits, T):
+    """The decode kernel (codes as 8-bit integer tcgen05 operands, activations as two-limb block-scaled
+    integers): both projections in one launch and as two launches, each within the bar and
+    bit-identical to each other."""
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, "bf16")
+    _, y_fused = _run_case(shape, bits, T, seed=25, path=6, want_y=True)
+    _, y_split = _run_case(shape, bits, T, seed=25, path=6, fused=False, want_y=True)
+    assert np.array_equal(y_fused, y_split)
+
+
+def test_int8_streaming_path_keeps_the_bf16_range():
+    """Activations far outside the fp16 range (|x| up to 3e38 would overflow a 16-bit float operand)
+    and weights whose products are tiny: the block-scaled integer operands follow the bf16
+    exponent range, so the result stays inside the bar."""
+    shape = inputs.LayerShape(512, 1024, 4, 1, "relu", "softmax", 128, "f16", "bf16")
+    bits = [8, 4, 2, 4]
+    for scale_x, std in ((3.0e4, 0.02), (1.0e-3, 1.0e-4), (1.0e6, 1.0e-3)):
+        W = inputs.expert_set(28, 0, shape, std)
+        x = inputs.to_bf16_valued(inputs.activations(28, 0, 9, shape.d_model, "bf16") * np.float32(scale_x))
+        Wr = inputs.router_weight(28, 0, shape.d_model, shape.n_experts, std=0.05 / scale_x)
+        packed, scales = oracle_pack_layer(W, shape, bits)
+        with layer.MoELayer(shape, bits, max_tokens=9) as moe:
+            B.emoe_set_ffn_path(moe.ctx, 6)
+            moe.pack_from_host(W)
+            y, ids, gates, _ = moe.forward(x, Wr)
+        y_ref = oracle.moe_ffn_combine(x, shape.d_ff, shape.act, shape.group, True, bits, packed, scales, ids, gates)
+        assert np.isfinite(y).all() and np.abs(y_ref).max() > 0
+        assert rel_to_max(y, y_ref) <= 2e-3, (scale_x, std, rel_to_max(y, y_ref))
+
+
 UMMA_CASES = [
     ("relu", 128, "f16", 512, 1024, 4, 1, "softmax", [8, 4, 2, 4], 200),              # ~50 tokens per expert
     ("relu", 128, "f16", 512, 1024, 2, 1, "softmax", [4, 2], 300),                    # two token tiles per expert
