@@ -54,7 +54,7 @@ def parse_args():
     ap.add_argument("--no-fuse", action="store_true", help="run the two projections of the expert FFNs as two launches")
     ap.add_argument("--slots", type=int, default=0, help="mixtral_stack_cached: slots of the HBM expert cache (default: a quarter of the experts)")
     ap.add_argument("--prefetch", type=int, default=-1, help="mixtral_stack_cached: experts of the next layer preloaded per decode step (default: top_k)")
-    ap.add_argument("--evict", default="forward", choices=["forward", "printed", "lru"], help="mixtral_stack_cached: eviction rule")
+    ap.add_argument("--evict", default="forward", choices=["forward", "printed", "lru", "lfu", "fifo"], help="mixtral_stack_cached: eviction rule")
     return ap.parse_args()
 
 
@@ -570,7 +570,8 @@ def run_cached(args, w, rank, world, local):
     T_prefill, T_decode = w.tokens
     steps = 128 if args.steps == 1000 else args.steps
     warmup = min(args.warmup, 8)
-    policy = {"forward": B.EVICT_FORWARD, "printed": B.EVICT_PRINTED, "lru": B.EVICT_LRU}[args.evict]
+    policy = {"forward": B.EVICT_FORWARD, "printed": B.EVICT_PRINTED, "lru": B.EVICT_LRU, "lfu": B.EVICT_LFU,
+              "fifo": B.EVICT_FIFO}[args.evict]
     t0 = time.perf_counter()
     stack = CachedStack(sh, n_layers, bits, n_slots, device=local, max_tokens=T_prefill, seed=w.seed, policy=policy,
                         n_prefetch=None if args.prefetch < 0 else args.prefetch)

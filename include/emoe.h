@@ -302,6 +302,8 @@ int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, i
 #define EMOE_EVICT_FORWARD 0 /* score -f/D, D = layers until the expert's layer runs again: (i - I) mod S */
 #define EMOE_EVICT_PRINTED 1 /* score -f/D with D = (S - i + I) mod S as the formula is printed */
 #define EMOE_EVICT_LRU 2     /* least recently used */
+#define EMOE_EVICT_LFU 3     /* fewest activations so far; ties: loaded earliest */
+#define EMOE_EVICT_FIFO 4    /* loaded earliest */
 
 typedef struct emoe_cache_stats {
   int64_t hits;               /* acquire found the expert in a slot (loaded or loading) */

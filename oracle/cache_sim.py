@@ -12,7 +12,12 @@ What it follows (EdgeMoE, arXiv 2308.14352, Section 3.3):
 * "Estimating expert activation a priori": the probability estimate comes from a table keyed by
   earlier layers' activations (here: one previous layer, as the workload definition asks).
 
-Readings where the paper is silent or at odds with itself (all listed in the design doc):
+Two more textbook rules are modelled for comparison, as in the paper's evaluation of eviction
+policies (its cache-hit-ratio figure compares five): `lfu` (the expert with the fewest activations
+so far leaves; ties: the one loaded earliest, then the lowest slot) and `fifo` (the expert loaded
+earliest leaves, whatever its use).
+
+Readings where the paper is silent or at odds with itself:
 * D: the printed formula is (S - i + I) mod S; the text wants layers "going to be executed
   soon" kept, which is (i - I) mod S.  Both exist: `forward` (default) and `printed`.
 * D = 0 (an expert of the current layer): the formula divides by zero; such experts are
@@ -29,7 +34,7 @@ from fractions import Fraction
 
 class ExpertBufferModel:
     def __init__(self, n_slots, n_layers, rule="forward"):
-        assert rule in ("forward", "printed", "lru")
+        assert rule in ("forward", "printed", "lru", "lfu", "fifo")
         self.n_slots, self.S, self.rule = n_slots, n_layers, rule
         self.layer_of, self.bytes_of = {}, {}
         self.slot_content = [None] * n_slots     # expert id or None
@@ -38,6 +43,7 @@ class ExpertBufferModel:
         self.in_use = {}                         # expert id -> acquire count not yet released
         self.fresh_from_preload = set()
         self.touched = [0] * n_slots
+        self.loaded_at = [0] * n_slots           # tick at which the slot's present content was put there
         self.tick = 0
         self.counters = dict(hits=0, misses=0, prefetch_hits=0, prefetched=0, prefetch_redundant=0,
                              prefetch_refused=0, evictions=0, bytes_copied=0)
@@ -58,6 +64,10 @@ class ExpertBufferModel:
                  if self.slot_content[s] is not None and self.in_use[self.slot_content[s]] == 0]
         if self.rule == "lru":
             return sorted(cands, key=lambda s: (self.touched[s], s))
+        if self.rule == "fifo":
+            return sorted(cands, key=lambda s: (self.loaded_at[s], s))
+        if self.rule == "lfu":
+            return sorted(cands, key=lambda s: (self.freq[self.slot_content[s]], self.loaded_at[s], s))
 
         def key(s):
             eid = self.slot_content[s]
@@ -86,6 +96,7 @@ class ExpertBufferModel:
         self.where[eid] = s
         self.tick += 1
         self.touched[s] = self.tick
+        self.loaded_at[s] = self.tick
         self.counters["bytes_copied"] += self.bytes_of[eid]
         return s, evicted
 

@@ -14,7 +14,8 @@ import numpy as np
 
 from . import binding as B
 
-RULES = (("forward", B.EVICT_FORWARD), ("printed", B.EVICT_PRINTED), ("lru", B.EVICT_LRU))
+RULES = (("forward", B.EVICT_FORWARD), ("printed", B.EVICT_PRINTED), ("lru", B.EVICT_LRU), ("lfu", B.EVICT_LFU),
+         ("fifo", B.EVICT_FIFO))
 
 
 def make_trace(n_layers: int, n_experts: int, top_k: int, steps: int, beta: float, seed: int):

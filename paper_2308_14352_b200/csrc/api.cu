@@ -21,12 +21,15 @@ constexpr int MAX_TABLES = 128;  // distinct expert tables a context can keep on
 constexpr size_t TMAP_BYTES = 128;  // sizeof(CUtensorMap)
 // one table block: the expert entries followed by one tensor map per (expert, matrix)
 constexpr size_t TABLE_MAPS_OFFSET = (sizeof(ExpertDev) * EMOE_MAX_EXPERTS + 127) / 128 * 128;
-constexpr size_t TABLE_BLOCK_BYTES = TABLE_MAPS_OFFSET + TMAP_BYTES * 3 * EMOE_MAX_EXPERTS;
+// ... followed by one tensor map per (expert, scale channel) for the int8 streaming kernel's scale windows
+constexpr size_t TABLE_SMAPS_OFFSET = TABLE_MAPS_OFFSET + TMAP_BYTES * 3 * EMOE_MAX_EXPERTS;
+constexpr size_t TABLE_BLOCK_BYTES = TABLE_SMAPS_OFFSET + TMAP_BYTES * 3 * EMOE_MAX_EXPERTS;
 
 struct TableEntry {
   std::vector<emoe_expert> host;
   int d_model = 0, d_ff = 0, act = 0;
   bool has_tmaps = false;
+  bool scales16 = false;  // every scale channel is 16-byte aligned (bulk copies of scales are possible)
 };
 
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
@@ -137,7 +140,7 @@ int cuda_fail(emoe_ctx* ctx, cudaError_t e) {
 // Device copy of a host expert table (entries + tensor maps); uploaded on `st` the first time
 // its content is seen.  *tmaps is null when the shape has no TMA path.
 int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaStream_t st, const ExpertDev** out,
-              const void** tmaps) {
+              const void** tmaps, const void** smaps) {
   const int E = L.E;
   for (size_t i = 0; i < ctx->tables.size(); ++i) {
     const TableEntry& te = ctx->tables[i];
@@ -152,6 +155,7 @@ int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaSt
       ctx->table_used[i] = ++ctx->table_clock;
       *out = reinterpret_cast<const ExpertDev*>(ctx->tables_dev + i * TABLE_BLOCK_BYTES);
       *tmaps = te.has_tmaps ? ctx->tables_dev + i * TABLE_BLOCK_BYTES + TABLE_MAPS_OFFSET : nullptr;
+      *smaps = te.has_tmaps && te.scales16 ? ctx->tables_dev + i * TABLE_BLOCK_BYTES + TABLE_SMAPS_OFFSET : nullptr;
       return EMOE_OK;
     }
   }
@@ -170,6 +174,8 @@ int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaSt
   ExpertDev* pin = reinterpret_cast<ExpertDev*>(pin_block);
   const int nmat = L.act == EMOE_ACT_RELU ? 2 : 3;
   bool maps_ok = ffn_tma_supported(L);
+  bool scales16 = true;
+  const int ssz = L.scale_f16 ? 2 : 4;
   for (int e = 0; e < E; ++e) {
     pin[e].bits = host[e].bits;
     pin[e].pad = 0;
@@ -182,17 +188,29 @@ int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaSt
       const int N = first ? L.d_ff : L.d_model, K = first ? L.d_model : L.d_ff;
       maps_ok = encode_weight_tmap(pin_block + TABLE_MAPS_OFFSET + TMAP_BYTES * (3 * e + m), host[e].packed[m], N, K,
                                    host[e].bits) == 0;
+      // the scale channel's map, where its rows allow one (long rows in multiples of 16 bytes)
+      const int row_bytes = (L.group > 0 ? K / L.group : 1) * ssz;
+      char* smap = pin_block + TABLE_SMAPS_OFFSET + TMAP_BYTES * (3 * e + m);
+      if (!aligned(host[e].scales[m], 16)) scales16 = false;
+      else if (encode_scale_tmap(smap, host[e].scales[m], N, row_bytes) != 0) std::memset(smap, 0, TMAP_BYTES);
     }
   }
   char* dev = ctx->tables_dev + slot * TABLE_BLOCK_BYTES;
-  const size_t bytes = maps_ok ? TABLE_MAPS_OFFSET + TMAP_BYTES * 3 * E : sizeof(ExpertDev) * E;
-  EMOE_CUDA(ctx, cudaMemcpyAsync(dev, pin_block, bytes, cudaMemcpyHostToDevice, st));
+  if (maps_ok) {  // entries + weight maps in one copy, the scale maps (behind the unused weight maps) in another
+    EMOE_CUDA(ctx, cudaMemcpyAsync(dev, pin_block, TABLE_MAPS_OFFSET + TMAP_BYTES * 3 * E, cudaMemcpyHostToDevice, st));
+    if (scales16)
+      EMOE_CUDA(ctx, cudaMemcpyAsync(dev + TABLE_SMAPS_OFFSET, pin_block + TABLE_SMAPS_OFFSET, TMAP_BYTES * 3 * E,
+                                     cudaMemcpyHostToDevice, st));
+  } else {
+    EMOE_CUDA(ctx, cudaMemcpyAsync(dev, pin_block, sizeof(ExpertDev) * E, cudaMemcpyHostToDevice, st));
+  }
   TableEntry te;
   te.host.assign(host, host + E);
   te.d_model = L.d_model;
   te.d_ff = L.d_ff;
   te.act = L.act;
   te.has_tmaps = maps_ok;
+  te.scales16 = scales16;
   if (recycle) {
     ctx->tables[slot] = std::move(te);
   } else {
@@ -206,6 +224,7 @@ int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaSt
   ctx->table_used[slot] = ++ctx->table_clock;
   *out = reinterpret_cast<const ExpertDev*>(dev);
   *tmaps = maps_ok ? dev + TABLE_MAPS_OFFSET : nullptr;
+  *smaps = maps_ok && scales16 ? dev + TABLE_SMAPS_OFFSET : nullptr;
   return EMOE_OK;
 }
 
@@ -252,7 +271,8 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   ctx->kernels_last = 0;
   const ExpertDev* table = nullptr;
   const void* tmaps = nullptr;
-  rc = get_table(ctx, L, host_experts, st, &table, &tmaps);
+  const void* smaps = nullptr;
+  rc = get_table(ctx, L, host_experts, st, &table, &tmaps, &smaps);
   if (rc != EMOE_OK) return rc;
 
   char* ws = ctx->workspace;
@@ -335,10 +355,10 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       EMOE_CUDA(ctx, cudaMemsetAsync(o_part + static_cast<size_t>(P) * L.d_model, 0,
                                      static_cast<size_t>(ksplit - 1) * P * L.d_model * sizeof(float), st));
     if (ctx->fuse_projections) {
-      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, ctx->dep_extra, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 2, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, ctx->dep_extra, ctx->check_word, st));
     } else {
-      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 1, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
-      EMOE_LAUNCH(ctx, launch_ffn_i8(1, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 1, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_i8(1, 2, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
     }
     EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, P, ctx->check_word, st));
     EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, P, ctx->check_word, st));
@@ -363,7 +383,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     if (ctx->fuse_projections) {
       // one launch: an expert's second projection starts when its hidden vectors are complete
-      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit,
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 2, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit,
                                      ctx->dep_extra, ctx->check_word, st));
       if (ev[1]) {  // one interval only: the end event of the triple stays unused
         EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
@@ -371,10 +391,10 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
         ev[2] = nullptr;
       }
     } else {
-      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 1, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit, 0,
+      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 1, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit, 0,
                                      ctx->check_word, st));
       if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-      EMOE_LAUNCH(ctx, launch_ffn_i8(1, 2, L, tmaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit, 0,
+      EMOE_LAUNCH(ctx, launch_ffn_i8(1, 2, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, 0, ctx->wait_limit, 0,
                                      ctx->check_word, st));
     }
   } else if (use_tma) {
@@ -660,6 +680,13 @@ int emoe_debug_expect_extra_completions(emoe_ctx* ctx, int extra) {
   ctx->dep_extra = extra;
   return EMOE_OK;
 }
+
+#ifdef EMOE_I8_PROFILE
+int emoe_debug_set_profile_buffer(void* dev_buffer) {
+  g_i8_profile = static_cast<long long*>(dev_buffer);
+  return EMOE_OK;
+}
+#endif
 
 int emoe_set_ffn_path(emoe_ctx* ctx, int path) {
   if (!ctx || path < 0 || path > 6) return EMOE_ERR_INVALID_ARG;

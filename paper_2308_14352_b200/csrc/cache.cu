@@ -35,12 +35,13 @@ struct CacheSlot {
   int expert;  // index into experts, -1 = free
   int pins;    // acquired and not yet released
   int64_t last_touch;
+  int64_t loaded_at;  // clock value when the present content was placed
 };
 
 class CachePolicy {
  public:
   CachePolicy(int n_slots, int n_layers, int policy) : n_layers_(n_layers), policy_(policy), clock_(0) {
-    slots_.assign(static_cast<size_t>(n_slots), CacheSlot{-1, 0, 0});
+    slots_.assign(static_cast<size_t>(n_slots), CacheSlot{-1, 0, 0, 0});
     std::memset(&stats_, 0, sizeof(stats_));
   }
   int add(const CacheExpert& e) {
@@ -66,14 +67,21 @@ class CachePolicy {
   // the number of layers until the expert's layer runs again, (i - I) mod S, which is what the
   // text asks for (layers about to run are kept);
   // EMOE_EVICT_PRINTED takes the printed (S - i + I) mod S.  D = 0 (the current layer) is
-  // protected: such an expert goes only when nothing else can.  EMOE_EVICT_LRU: least recently
-  // touched first.  Ties: lowest slot.
+  // protected: such an expert goes only when nothing else can.  For comparison (the paper's
+  // evaluation sets its rule against the textbook ones): EMOE_EVICT_LRU, least recently touched
+  // first; EMOE_EVICT_FIFO, loaded earliest first; EMOE_EVICT_LFU, fewest activations first (ties:
+  // loaded earliest).  Remaining ties: lowest slot.
   bool better_victim(int sa, int sb, int current_layer) const {  // is slot sa a better victim than sb?
     const CacheExpert& a = experts_[static_cast<size_t>(slots_[static_cast<size_t>(sa)].expert)];
     const CacheExpert& b = experts_[static_cast<size_t>(slots_[static_cast<size_t>(sb)].expert)];
     if (policy_ == EMOE_EVICT_LRU) {
       const int64_t ta = slots_[static_cast<size_t>(sa)].last_touch, tb = slots_[static_cast<size_t>(sb)].last_touch;
       return ta != tb ? ta < tb : sa < sb;
+    }
+    if (policy_ == EMOE_EVICT_FIFO || policy_ == EMOE_EVICT_LFU) {
+      if (policy_ == EMOE_EVICT_LFU && a.freq != b.freq) return a.freq < b.freq;
+      const int64_t la = slots_[static_cast<size_t>(sa)].loaded_at, lb = slots_[static_cast<size_t>(sb)].loaded_at;
+      return la != lb ? la < lb : sa < sb;
     }
     const int da = distance(a.layer, current_layer), db = distance(b.layer, current_layer);
     if ((da == 0) != (db == 0)) return db == 0;  // the unprotected one
@@ -109,6 +117,7 @@ class CachePolicy {
     }
     slots_[static_cast<size_t>(best)].expert = ei;
     slots_[static_cast<size_t>(best)].last_touch = ++clock_;
+    slots_[static_cast<size_t>(best)].loaded_at = clock_;
     experts_[static_cast<size_t>(ei)].slot = best;
     for (int m = 0; m < 6; ++m) stats_.bytes_copied += static_cast<int64_t>(experts_[static_cast<size_t>(ei)].bytes[m]);
     return best;
@@ -248,7 +257,7 @@ extern "C" {
 
 int emoe_cache_create(emoe_ctx* ctx, int n_slots, size_t slot_bytes, int n_layers, int policy) {
   if (!ctx || n_slots <= 0 || slot_bytes == 0 || n_layers <= 0) return EMOE_ERR_INVALID_ARG;
-  if (policy != EMOE_EVICT_FORWARD && policy != EMOE_EVICT_PRINTED && policy != EMOE_EVICT_LRU) return EMOE_ERR_UNSUPPORTED;
+  if (policy < EMOE_EVICT_FORWARD || policy > EMOE_EVICT_FIFO) return EMOE_ERR_UNSUPPORTED;
   if (ctx_cache(ctx)) return EMOE_ERR_INVALID_ARG;  // one cache per context
   ExpertCache* c = new (std::nothrow) ExpertCache(n_slots, n_layers, policy);
   if (!c) return EMOE_ERR_INVALID_ARG;
@@ -308,22 +317,34 @@ int emoe_cache_acquire(emoe_ctx* ctx, const int64_t* ids, int n, int current_lay
   ExpertCache* c = ctx_cache(ctx);
   cudaError_t err = cudaSetDevice(c->device);
   if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
-  for (int i = 0; i < n; ++i) {
-    const int ei = c->policy.find(ids[i]);
-    if (ei < 0) return EMOE_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i)  // nothing is touched unless every id is known
+    if (c->policy.find(ids[i]) < 0) return EMOE_ERR_INVALID_ARG;
+  int rc = EMOE_OK, done = 0;
+  for (; done < n && rc == EMOE_OK; ++done) {
+    const int ei = c->policy.find(ids[done]);
     int load, evicted;
     const int s = c->policy.acquire(ei, current_layer, &load, &evicted);
-    if (s < 0) return EMOE_ERR_CACHE_FULL;
+    if (s < 0) {
+      rc = EMOE_ERR_CACHE_FULL;
+      break;
+    }
     if (load) {
       err = load_into_slot(c, c->policy.expert(ei), s, static_cast<cudaStream_t>(copy_stream));
-      if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
+      if (err != cudaSuccess) rc = ctx_cuda_fail(ctx, err);
     }
     // the compute stream goes on when the slot's contents are complete (no host wait)
-    err = cudaStreamWaitEvent(static_cast<cudaStream_t>(compute_stream), c->ready[static_cast<size_t>(s)], 0);
-    if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
-    expert_pointers(c, c->policy.expert(ei), &out_experts[i]);
+    if (rc == EMOE_OK) {
+      err = cudaStreamWaitEvent(static_cast<cudaStream_t>(compute_stream), c->ready[static_cast<size_t>(s)], 0);
+      if (err != cudaSuccess) rc = ctx_cuda_fail(ctx, err);
+    }
+    if (rc == EMOE_OK) expert_pointers(c, c->policy.expert(ei), &out_experts[done]);
   }
-  return EMOE_OK;
+  if (rc != EMOE_OK) {
+    // all or nothing: the experts acquired so far by this call are let go again, so that a failed
+    // call leaves no slot protected (their activation counts keep the increment)
+    for (int i = 0; i < done; ++i) c->policy.release(c->policy.find(ids[i]));
+  }
+  return rc;
 }
 
 int emoe_cache_release(emoe_ctx* ctx, const int64_t* ids, int n, void* compute_stream) {
@@ -331,16 +352,20 @@ int emoe_cache_release(emoe_ctx* ctx, const int64_t* ids, int n, void* compute_s
   ExpertCache* c = ctx_cache(ctx);
   cudaError_t err = cudaSetDevice(c->device);
   if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
-  for (int i = 0; i < n; ++i) {
-    const int ei = c->policy.find(ids[i]);
-    if (ei < 0) return EMOE_ERR_INVALID_ARG;
-    const int s = c->policy.release(ei);
-    if (s < 0) return EMOE_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i)
+    if (c->policy.find(ids[i]) < 0) return EMOE_ERR_INVALID_ARG;
+  int rc = EMOE_OK;
+  for (int i = 0; i < n; ++i) {  // an id that is not held does not keep the others from being released
+    const int s = c->policy.release(c->policy.find(ids[i]));
+    if (s < 0) {
+      rc = EMOE_ERR_INVALID_ARG;
+      continue;
+    }
     err = cudaEventRecord(c->idle[static_cast<size_t>(s)], static_cast<cudaStream_t>(compute_stream));
     if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
     c->idle_valid[static_cast<size_t>(s)] = 1;
   }
-  return EMOE_OK;
+  return rc;
 }
 
 int emoe_cache_slot_of(emoe_ctx* ctx, int64_t id) {
@@ -364,7 +389,7 @@ struct emoe_policy {
 
 emoe_policy* emoe_policy_create(int n_slots, int n_layers, int policy) {
   if (n_slots <= 0 || n_layers <= 0) return nullptr;
-  if (policy != EMOE_EVICT_FORWARD && policy != EMOE_EVICT_PRINTED && policy != EMOE_EVICT_LRU) return nullptr;
+  if (policy < EMOE_EVICT_FORWARD || policy > EMOE_EVICT_FIFO) return nullptr;
   return new (std::nothrow) emoe_policy(n_slots, n_layers, policy);
 }
 void emoe_policy_destroy(emoe_policy* p) { delete p; }

@@ -139,15 +139,19 @@ cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, c
 // [n_pairs][2][K] with block scales xsc / hsc [n_pairs][K/128] (act_q.cuh).  token_tile: tokens
 // per pass (8, 16 or 32), 0 = by the routing statistics of (L, T).  wait_limit: polls before a
 // wait inside the kernel gives up (0 = default); dep_extra: test hook, 0 in production.
+extern long long* g_i8_profile;  // device buffer [CTAs][16] for the timers of a profiling build (null otherwise)
 bool ffn_i8_supported(const LayerDims& L);
 int ffn_i8_ksplit(const LayerDims& L, int T);
 int ffn_i8_token_tile(const LayerDims& L, int T);
-cudaError_t launch_ffn_i8(int phase_begin, int phase_end, const LayerDims& L, const void* wmaps, const void* xq,
+// smaps: [E][3] tensor maps of the scale channels (encode_scale_tmap), or null when a channel is not 16-byte aligned.
+int encode_scale_tmap(void* out_map, const void* scales, int N, int row_bytes);
+cudaError_t launch_ffn_i8(int phase_begin, int phase_end, const LayerDims& L, const void* wmaps, const void* smaps, const void* xq,
                           const float* xsc, int* plan, void* hq, float* hsc, float* o_part, int ksplit, int n_pairs,
                           int T, int token_tile, unsigned wait_limit, int dep_extra, int* check_word, cudaStream_t st);
 
+// swizzle128: the 128-byte swizzle (operand tiles) or none (plain rows)
 int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
-                   uint32_t box_inner, uint32_t box_outer);
+                   uint32_t box_inner, uint32_t box_outer, bool swizzle128 = true);
 
 // tcgen05 grouped GEMM for experts with many tokens (fp16 operands, fp32 accumulation in tensor
 // memory).  xs16 / hidden16: activations in expert order, fp16, pair order; o: [n_pairs][d_model].

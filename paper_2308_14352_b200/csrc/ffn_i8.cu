@@ -23,11 +23,24 @@
 // Shape of the work: persistent CTAs, one per SM, pull items (activated expert, block of 128
 // output rows[, split-K slice]) of the first projection, then of the second, from a device
 // counter; an item of the second projection waits (bounded) until the expert's hidden vectors
-// are complete.  Warp roles: 4 epilogue warps (one thread per output row = tensor-memory lane),
-// 2 x 4 unpack warps (alternating A tiles, one thread per row), one TMA producer warp, one
-// MMA-issuing warp.  Rings: shared-memory stages (codes + activation tile + scales), two A
-// tiles and a ring of accumulators in tensor memory, each with full/empty mbarriers.  Every
-// wait is bounded: a wait that runs out sets CHECK_WAIT_TIMEOUT and the CTA winds down.
+// are complete.
+// Warp roles and rings (every ring has full/empty mbarriers, every wait is bounded: a wait that
+// runs out sets CHECK_WAIT_TIMEOUT and the CTA winds down):
+//   producer warp     TMA: weight boxes and the tokens' limb rows into the STAGE ring (shared
+//                     memory, 128 bytes of every row of 1 or 2 matrices per stage); a record of
+//                     what the stage holds plus the tokens' block scales into the deeper SIDE ring;
+//   unpack warps      2 x 4 warps, one thread per row: a 4- or 2-bit stage, one 128-input segment
+//                     at a time, into the A ring (8 segments of 32 columns in tensor memory);
+//   MMA warp          one thread: four K=32 MMAs per segment into the accumulator ring (groups of
+//                     up to four segments of one matrix), commits release A segments, stages and
+//                     publish accumulator groups;
+//   scale warp        follows the side ring and copies (cp.async) the weight scales every stage
+//                     needs, a short window per row, into the SCALE ring: under load a global load
+//                     takes a microsecond, so the scales travel as far ahead as the weights do;
+//   epilogue warps    4 warps, one thread per output row (= tensor-memory lane): accumulator
+//                     groups -> registers -> scaled fp32 totals.  They work from the side and scale
+//                     rings only, so a stage's shared memory is free again as soon as its MMAs
+//                     have read it, however far the epilogue lags.
 #include <cuda.h>
 
 #include "act_q.cuh"
@@ -45,35 +58,46 @@ constexpr int I8_MAT_BYTES = 2 * I8_BOX_BYTES;       // 128 rows x 128 bytes of 
 constexpr int I8_WARP_UNPACK0 = 4;                   // warps 0-3 epilogue, 4-7 and 8-11 unpack
 constexpr int I8_WARP_PRODUCER = 12;
 constexpr int I8_WARP_MMA = 13;
-constexpr int I8_THREADS = 14 * 32;
+constexpr int I8_WARP_SCALES = 14;
+constexpr int I8_THREADS = 15 * 32;
 constexpr int I8_MAX_STAGES = 8;
+constexpr int I8_SIDE = 16;                          // entries of the side ring
+// Weight scales travel ahead of their use in one of three ways, chosen per projection on the host:
+//   SCALE_BLOCK   a row's whole scale channel is at most 32 bytes: the 128 rows of an item are one
+//                 contiguous block, fetched by one bulk copy per matrix and item pass;
+//   SCALE_WINDOW  longer rows whose length is a multiple of 16 bytes: 32-byte windows of the 128 rows
+//                 (16 fp16 scales = 2048 inputs), one TMA box per matrix whenever the inputs move
+//                 into the next window;
+//   SCALE_STAGE   anything else (odd row lengths, unaligned channels, group sizes that are not a
+//                 power of two): a warp copies each stage's few bytes per row with cp.async.
+// The first two cost one instruction per matrix and thousands of inputs; the third is the slow,
+// general path.
+constexpr int SCALE_BLOCK = 0, SCALE_WINDOW = 1, SCALE_STAGE = 2;
+constexpr int I8_CHUNKS = 4;                         // entries of the scale ring in the first two modes
+constexpr int I8_CHUNK_ROW = 32;                     // bytes per row of an entry
+constexpr int I8_CHUNK_BYTES = I8_ROWS * I8_CHUNK_ROW;  // one matrix of one entry: 4 KB
+constexpr int I8_SCALE_RING = 8;                     // entries of the ring in the third mode
+constexpr int I8_SCALE_TILE = I8_ROWS * 16;          // one matrix of one stage: a 16-byte window per row
 constexpr int I8_TMEM_COLS = 512;
-constexpr int I8_A_COLS = 128;                       // an unpacked A tile: 128 rows x 512 bytes = 128 columns
-constexpr int I8_D_COL0 = 2 * I8_A_COLS;             // accumulators behind the two A tiles
-constexpr int I8_D_COLS = I8_TMEM_COLS - I8_D_COL0;  // 256 columns of accumulators
-constexpr int I8_MAX_DBUF = 16;
-constexpr int I8_SCALE_BYTES = I8_ROWS * 16;         // raw scales of a stage: a 16-byte window per row
-constexpr int I8_SX_BYTES = 4 * 32 * 4;              // activation block scales of a stage: [4 segments][32 tokens]
+constexpr int I8_A_SLOTS = 8;                        // A ring: unpacked 128-input segments, 32 columns each
+constexpr int I8_A_SLOT_COLS = 32;
+constexpr int I8_D_COL0 = I8_A_SLOTS * I8_A_SLOT_COLS;  // accumulators behind the A ring
+constexpr int I8_D_COLS = I8_TMEM_COLS - I8_D_COL0;     // 256 columns of accumulators
+constexpr int I8_MAX_GROUPS = 4;
 constexpr int I8_SMEM_LIMIT = 227 * 1024;
+constexpr int I8_STATIC_SMEM = 12 * 1024;            // barriers, side ring, exchange buffer (upper bound)
 
-// a shared-memory stage: weight boxes of 1 or 2 matrices | activation tiles of up to 4 segments
-// (2*NT rows x 128 bytes each) | weight-scale windows | activation block scales
-struct StageLayout {
-  int b_off, sc_off, sx_off, bytes;
-};
-__host__ __device__ inline StageLayout stage_layout(int nt, int nmat) {
-  StageLayout s;
-  s.b_off = nmat * I8_MAT_BYTES;
-  s.sc_off = s.b_off + 4 * (2 * nt) * 128;
-  s.sx_off = s.sc_off + nmat * I8_SCALE_BYTES;
-  s.bytes = (s.sx_off + I8_SX_BYTES + 1023) / 1024 * 1024;
-  return s;
-}
+// a shared-memory stage: weight boxes of 1 or 2 matrices | limb tiles of up to 4 segments
+// (2*NT rows x 128 bytes each)
+__host__ __device__ constexpr int stage_b_off(int nmat) { return nmat * I8_MAT_BYTES; }
+__host__ __device__ constexpr int stage_bytes(int nt, int nmat) { return nmat * I8_MAT_BYTES + 4 * (2 * nt) * 128; }
 
 struct I8Args {
   int phase_begin, phase_end;  // projections this launch runs: [0,1), [1,2) or both, [0,2)
   LayerDims L;
   const CUtensorMap* wmaps;  // [E][3] packed-weight maps: byte image [N][K*bits/8], boxes 64 rows x 128 bytes
+  const CUtensorMap* smaps;  // [E][3] scale-channel maps: byte image [N][row bytes], boxes 128 rows x 32 bytes (SCALE_WINDOW)
+  int scale_mode[2];         // per projection: SCALE_BLOCK / SCALE_WINDOW / SCALE_STAGE
   int* plan;                 // header {activated experts, item counters} + one PlanRec per activated expert
   const float* xsc;          // block scales of the first projection's input [P][d/128]
   int8_t* hq;                // hidden vectors as limbs [P][2][f] (written by the first projection)
@@ -89,6 +113,7 @@ struct I8Args {
   unsigned dep_wait_limit;  // polls (~0.1 us each) before the wait for an expert's hidden vectors gives up
   int dep_extra;            // test hook: completions expected beyond the real count (0 in production)
   int* check_word;
+  long long* prof;          // per-CTA timers of a profiling build, else null
 };
 
 struct PhaseDims {
@@ -106,13 +131,23 @@ __device__ __forceinline__ PhaseDims phase_dims(const I8Args& a, int phase) {
   return d;
 }
 
-// what a stage holds, written by the producer before it arms the stage's barrier
+// what a stage holds, written by the producer before it publishes the stage
 struct StageMeta {
   int e, rb, z, begin;
   int p0, ntok, k0, bits;
   int flags, phase, ai, nseg;
+  const void* scales[2];  // scale channels of the stage's matrices
+  int chunk, win0, pitch, pad;  // scale-ring entry of the stage, first byte of a row it holds, bytes per row in it
 };
 constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8, META_DONE = 16;
+constexpr int META_NEW_CHUNK = 32;  // the stage is the first to use its scale-ring entry
+constexpr int META_END_CHUNK = 64;  // ... the last
+
+// an entry of the side ring: the record of a stage and the block scales of its tokens' limbs
+struct SideEntry {
+  StageMeta m;
+  float sx[4][32];  // [segment][token]
+};
 
 __device__ __forceinline__ int group_of(int k, int gshift, int G, int ngroups) {
   return ngroups == 1 ? 0 : (gshift >= 0 ? (k >> gshift) : k / G);
@@ -120,10 +155,13 @@ __device__ __forceinline__ int group_of(int k, int gshift, int G, int ngroups) {
 
 __device__ __forceinline__ bool wait_lim(uint32_t bar, uint32_t parity, unsigned limit, int* check_word,
                                          volatile int* abort_flag) {
+  // every poll may park the thread for up to a microsecond (it resumes at once when the phase
+  // completes): the many warps of a CTA that wait at any time must not crowd the shared-memory pipe
+  // of the few that work
+  if (mbar_try_wait(bar, parity)) return true;
   for (unsigned i = 0; i < limit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_parked(bar, parity, 1000u)) return true;
     if (*abort_flag) return false;
-    if (i > 64) __nanosleep(40);
   }
   *abort_flag = 1;
   atomicOr(check_word, CHECK_WAIT_TIMEOUT);
@@ -157,6 +195,29 @@ __device__ __forceinline__ void unpack2(const uint4& v, uint32_t (&o)[16]) {
   }
 }
 
+// Optional per-CTA timers (build with -DEMOE_I8_PROFILE; the buffer is set by
+// emoe_debug_set_profile_buffer): cycles each role spends in its waits, read with clock64.
+#ifdef EMOE_I8_PROFILE
+#define PROF_DECL long long prof_t0 = 0, prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}
+#define PROF_BEGIN prof_t0 = clock64()
+#define PROF_END(i) prof_acc[i] += clock64() - prof_t0
+#define PROF_STORE(base, n)                                                     \
+  if (a.prof && lane == 0)                                                      \
+    for (int pi = 0; pi < (n); ++pi) a.prof[blockIdx.x * 32 + (base) + pi] = prof_acc[pi]
+#define PROF_LAP(i)                    \
+  {                                    \
+    const long long now__ = clock64(); \
+    prof_acc[i] += now__ - prof_t0;    \
+    prof_t0 = now__;                   \
+  }
+#else
+#define PROF_DECL
+#define PROF_BEGIN
+#define PROF_END(i)
+#define PROF_STORE(base, n)
+#define PROF_LAP(i)
+#endif
+
 // a ring position and the parity of its current round
 struct Ring {
   int i;
@@ -174,42 +235,65 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
     ffn_i8_kernel(const __grid_constant__ I8Args a, const __grid_constant__ CUtensorMap tmap_x,
                   const __grid_constant__ CUtensorMap tmap_h) {
   constexpr int NMAT_MAX = DUAL ? 2 : 1;
-  constexpr int NCOL = 2 * NT;                  // accumulator columns of one segment: hi and lo limb of NT tokens
-  constexpr int NDBUF = I8_D_COLS / NCOL;       // accumulators in the ring
-  constexpr int B_SEG_BYTES = NCOL * 128;       // activation tile of one segment
-  static_assert(NDBUF <= I8_MAX_DBUF && NDBUF >= 4, "accumulator ring");
+  constexpr int NCOL = 2 * NT;                 // accumulator columns of one segment: hi and lo limb of NT tokens
+  constexpr int GSEGS = NT == 32 ? 2 : 4;      // segments of one accumulator group
+  constexpr int GCOLS = GSEGS * NCOL;          // 64 / 128 / 128 columns
+  constexpr int NGRP = I8_D_COLS / GCOLS;      // groups in the ring: 4 / 2 / 2
+  constexpr int B_SEG_BYTES = NCOL * 128;      // limb tile of one segment
+  constexpr int STAGE_BYTES = stage_bytes(NT, NMAT_MAX);
+  constexpr int B_OFF = stage_b_off(NMAT_MAX);
+  static_assert(NGRP >= 2 && NGRP <= I8_MAX_GROUPS, "accumulator ring");
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * I8_MAX_STAGES + 4 + 2 * I8_MAX_DBUF + 1];
-  __shared__ __align__(16) StageMeta meta[I8_MAX_STAGES];
+  __shared__ __align__(8) uint64_t bars[2 * I8_MAX_STAGES + 2 * I8_SIDE + 2 * I8_A_SLOTS + 2 * I8_MAX_GROUPS + 1 + 2 * I8_SCALE_RING +
+                                        2 * I8_CHUNKS];
+  __shared__ __align__(16) SideEntry side[I8_SIDE];
   __shared__ __align__(16) uint32_t s_max[2][32][4];  // [item parity][token][epilogue warp]: largest |h| of the warp's rows
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const StageLayout SL = stage_layout(NT, NMAT_MAX);
   const int STAGES = a.stages;
 
   const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * I8_MAX_STAGES;
-  const uint32_t bar_afull = bar_empty + 8 * I8_MAX_STAGES, bar_aempty = bar_afull + 16;
-  const uint32_t bar_dfull = bar_aempty + 16, bar_dempty = bar_dfull + 8 * I8_MAX_DBUF;
-  const uint32_t bar_xchg = bar_dempty + 8 * I8_MAX_DBUF;
+  const uint32_t bar_sfull = bar_empty + 8 * I8_MAX_STAGES, bar_sempty = bar_sfull + 8 * I8_SIDE;
+  const uint32_t bar_afull = bar_sempty + 8 * I8_SIDE, bar_aempty = bar_afull + 8 * I8_A_SLOTS;
+  const uint32_t bar_dfull = bar_aempty + 8 * I8_A_SLOTS, bar_dempty = bar_dfull + 8 * I8_MAX_GROUPS;
+  const uint32_t bar_xchg = bar_dempty + 8 * I8_MAX_GROUPS;
+  const uint32_t bar_wfull = bar_xchg + 8, bar_wempty = bar_wfull + 8 * I8_SCALE_RING;
+  const uint32_t bar_cfull = bar_wempty + 8 * I8_SCALE_RING, bar_cempty = bar_cfull + 8 * I8_CHUNKS;
+  // the scale ring sits behind the stages in dynamic shared memory (entries of either kind)
+  unsigned char* scale_ring = smem + STAGES * STAGE_BYTES;
+  constexpr int SCALE_ENTRY = NMAT_MAX * I8_SCALE_TILE;
+  constexpr int CHUNK_ENTRY = NMAT_MAX * I8_CHUNK_BYTES;
 
   if (threadIdx.x == 0) {
     abort_word = 0;
     for (int s = 0; s < I8_MAX_STAGES; ++s) {
-      mbar_init(bar_full + 8 * s, 33);  // the producer's lane 0 (+ TMA bytes) and every lane's small copies
-      mbar_init(bar_empty + 8 * s, 5);  // the MMAs that read the stage (one commit) + the four epilogue warps
+      mbar_init(bar_full + 8 * s, 1);   // the producer's lane 0 (+ the bytes of its TMA copies)
+      mbar_init(bar_empty + 8 * s, 9);  // commit of the MMAs that read the stage + the eight unpack warps
     }
-    for (int w = 0; w < 2; ++w) {
-      mbar_init(bar_afull + 8 * w, 4);   // the four warps of the unpack group
-      mbar_init(bar_aempty + 8 * w, 1);  // commit of the MMAs that read the tile
+    for (int s = 0; s < I8_SIDE; ++s) {
+      mbar_init(bar_sfull + 8 * s, 33);  // the producer's lane 0 (record written) and every lane's small copies
+      mbar_init(bar_sempty + 8 * s, 4);  // the four epilogue warps
     }
-    for (int d = 0; d < I8_MAX_DBUF; ++d) {
-      mbar_init(bar_dfull + 8 * d, 1);   // commit of the segment's MMAs
+    for (int s = 0; s < I8_A_SLOTS; ++s) {
+      mbar_init(bar_afull + 8 * s, 4);   // the four warps of the unpack group that owns the slot
+      mbar_init(bar_aempty + 8 * s, 1);  // commit of the MMAs that read the segment
+    }
+    for (int d = 0; d < I8_MAX_GROUPS; ++d) {
+      mbar_init(bar_dfull + 8 * d, 1);   // commit of the group's MMAs
       mbar_init(bar_dempty + 8 * d, 4);  // the four epilogue warps have read it
     }
     mbar_init(bar_xchg, 4);
+    for (int w = 0; w < I8_SCALE_RING; ++w) {
+      mbar_init(bar_wfull + 8 * w, 32);   // every lane of the scale warp, after its copies
+      mbar_init(bar_wempty + 8 * w, 4);   // the four epilogue warps
+    }
+    for (int c = 0; c < I8_CHUNKS; ++c) {
+      mbar_init(bar_cfull + 8 * c, 1);    // the producer's lane 0 (+ the bytes of its copies)
+      mbar_init(bar_cempty + 8 * c, 4);   // the four epilogue warps
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == I8_WARP_MMA) tmem_alloc(smem_u32(&tmem_base_slot), I8_TMEM_COLS);
@@ -225,7 +309,6 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
   const LayerDims& L = a.L;
   PlanRec* recs = reinterpret_cast<PlanRec*>(reinterpret_cast<char*>(a.plan) + PLAN_HEADER_BYTES);
   const bool fused = a.phase_begin == 0 && a.phase_end == 2;
-  const int ssz = L.scale_f16 ? 2 : 4;
 
   if (warp == I8_WARP_PRODUCER) {
     // ---------------- producer warp ----------------
@@ -233,8 +316,13 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
     const int n_items0 = a.phase_begin == 0 ? n_active * a.row_blocks[0] : 0;
     const int n_items1 = a.phase_end == 2 ? n_active * a.row_blocks[1] * a.ksplit : 0;
     const int n_items = n_items0 + n_items1;
-    Ring ring{0, 0};
+    Ring ring{0, 0}, sring{0, 0}, cring{0, 0};
     bool ok = true;
+    const int ssz = L.scale_f16 ? 2 : 4;
+    PROF_DECL;
+#ifdef EMOE_I8_PROFILE
+    const long long prof_start = clock64();
+#endif
     int item = blockIdx.x;  // a CTA's first item is its own index; the counter hands out the rest
     while (ok) {
       if (item >= n_items || __any_sync(0xffffffffu, *abort_flag != 0)) break;
@@ -242,7 +330,6 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       const int li = item - (phase == 0 ? 0 : n_items0);
       const PhaseDims pd = phase_dims<DUAL>(a, phase);
       const int K = pd.K;
-      const int ngroups_k = a.ngroups[phase];
       const int ai = li / (pd.ksplit * pd.row_blocks);
       const PlanRec rec = recs[ai];
       const int z = li % pd.ksplit;
@@ -260,32 +347,80 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       const int npass = (rec.cnt + NT - 1) / NT;
       const int row0 = rb * I8_ROWS;
       bool need_dep = fused && phase == 1;
-      // scale rows this lane copies (rows 4l .. 4l+3 of every matrix of the stage): byte offset of
-      // the row's scale channel from its 4-byte-aligned base
-      int srow_off[4];
-#pragma unroll
-      for (int r = 0; r < 4; ++r) srow_off[r] = min(row0 + 4 * lane + r, pd.N - 1) * ngroups_k * ssz;
+      const int smode = a.scale_mode[phase];
+      const int ngroups_k = a.ngroups[phase];
+      const int row_bytes = ngroups_k * ssz;  // a row's scale channel
       for (int pass = 0; pass < npass && ok; ++pass) {
         const int p0 = pass * NT;
         const int ntok = min(NT, rec.cnt - p0);
         const int nst = max(nsteps, 1);  // an empty split-K slice still has to store its zeros
+        int cur_win = -1, cur_chunk = 0;
         for (int s = 0; s < nst; ++s) {
-          if (!wait_warp(bar_empty + 8 * ring.i, ring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
+          PROF_BEGIN;
+          if (!wait_warp(bar_empty + 8 * ring.i, ring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag) ||
+              !wait_warp(bar_sempty + 8 * sring.i, sring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
             ok = false;
             break;
           }
-          unsigned char* st = smem + ring.i * SL.bytes;
-          const uint32_t full = bar_full + 8 * ring.i;
+          PROF_END(0);
+          unsigned char* st = smem + ring.i * STAGE_BYTES;
+          const uint32_t full = bar_full + 8 * ring.i, sfull = bar_sfull + 8 * sring.i;
+          SideEntry* se = &side[sring.i];
           const int k0 = (step_begin + s) * kspan;
           const int klen = nsteps > 0 ? min(kspan, K - k0) : 0;
           const int nseg = klen / 128;
+          // the scale-ring entry of the stage: the item's block, or the 32-byte window its inputs fall into
+          int cflags = 0, stage_win0 = 0;
+          if (klen > 0 && smode != SCALE_STAGE) {
+            const int win = smode == SCALE_BLOCK ? 0 : (group_of(k0, a.gshift, L.group, ngroups_k) * ssz) / I8_CHUNK_ROW;
+            stage_win0 = win * I8_CHUNK_ROW;
+            if (win != cur_win) {
+              if (!wait_warp(bar_cempty + 8 * cring.i, cring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
+                ok = false;
+                break;
+              }
+              if (lane == 0) {
+                const uint32_t cfull = bar_cfull + 8 * cring.i;
+                unsigned char* cdst = scale_ring + cring.i * CHUNK_ENTRY;
+                if (smode == SCALE_BLOCK) {
+                  mbar_expect_tx(cfull, pd.nmat * I8_ROWS * row_bytes);
+                  for (int m = 0; m < pd.nmat; ++m)
+                    bulk_load(smem_u32(cdst + m * I8_CHUNK_BYTES),
+                              static_cast<const char*>(rec.scales[pd.mat_first + m]) + static_cast<size_t>(row0) * row_bytes,
+                              I8_ROWS * row_bytes, cfull);
+                } else {
+                  mbar_expect_tx(cfull, pd.nmat * I8_CHUNK_BYTES);
+                  for (int m = 0; m < pd.nmat; ++m)
+                    tma_load_2d(smem_u32(cdst + m * I8_CHUNK_BYTES), a.smaps + static_cast<size_t>(rec.e) * 3 + pd.mat_first + m,
+                                win * I8_CHUNK_ROW, row0, cfull);
+                }
+              }
+              cur_win = win;
+              cur_chunk = cring.i;
+              cring.next(I8_CHUNKS);
+              cflags |= META_NEW_CHUNK;
+            }
+            const int k0n = k0 + kspan;
+            const bool last = s == nst - 1 || k0n >= K ||
+                              (smode == SCALE_WINDOW && (group_of(k0n, a.gshift, L.group, ngroups_k) * ssz) / I8_CHUNK_ROW != win);
+            if (last) {
+              cflags |= META_END_CHUNK;
+              cur_win = -1;
+            }
+          }
           if (lane == 0) {
             const int flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0) |
-                              (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0);
-            uint4* mq = reinterpret_cast<uint4*>(&meta[ring.i]);
+                              (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0) | cflags;
+            uint4* mq = reinterpret_cast<uint4*>(&se->m);
             mq[0] = make_uint4(rec.e, rb, z, rec.begin);
             mq[1] = make_uint4(p0, ntok, k0, bits);
             mq[2] = make_uint4(flags, phase, ai, nseg);
+            se->m.scales[0] = rec.scales[pd.mat_first];
+            se->m.scales[1] = rec.scales[pd.mat_first + pd.nmat - 1];
+            se->m.chunk = cur_chunk;
+            se->m.win0 = stage_win0;
+            se->m.pitch = smode == SCALE_BLOCK ? row_bytes : I8_CHUNK_ROW;
+            mbar_arrive(sfull);  // the record is written (the other 32 arrivals follow the small copies)
             if (klen > 0) {
               mbar_expect_tx(full, pd.nmat * I8_MAT_BYTES + nseg * B_SEG_BYTES);
               const int c0 = k0 * bits / 8;
@@ -300,28 +435,12 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
           }
           __syncwarp();
           if (klen > 0) {
-            // weight scales: lane l copies the windows of rows 4l .. 4l+3 of every matrix
-            const int g0 = group_of(k0, a.gshift, L.group, ngroups_k),
-                      g1 = group_of(k0 + (nseg - 1) * 128, a.gshift, L.group, ngroups_k);
-            const uint32_t sdst = smem_u32(st + SL.sc_off);
-            for (int m = 0; m < pd.nmat; ++m) {
-              const char* sbase = static_cast<const char*>(rec.scales[pd.mat_first + m]);
-#pragma unroll
-              for (int r = 0; r < 4; ++r) {
-                const int b0 = (srow_off[r] + g0 * ssz) & ~3;
-                const int b1 = srow_off[r] + (g1 + 1) * ssz;
-#pragma unroll 1
-                for (int w = 0; b0 + 4 * w < b1; ++w)
-                  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + (m * I8_ROWS + 4 * lane + r) * 16 + 4 * w),
-                               "l"(sbase + b0 + 4 * w)
-                               : "memory");
-              }
-            }
             if (need_dep) {
-              // codes and scales of the stage are on their way; the hidden vectors may still be in the
+              // the codes of the stage are on their way; the hidden vectors may still be in the
               // making on other SMs.  Every lane acquires the counter itself, so that its own copies
               // below are ordered behind the writers' stores.
               need_dep = false;
+              PROF_BEGIN;
               const int expect = a.row_blocks[0] * 4 + a.dep_extra;
               const int* done = &recs[ai].done;
               bool ready = false;
@@ -338,29 +457,31 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
                   atomicOr(a.check_word, CHECK_WAIT_TIMEOUT);
                 }
                 ok = false;
-                // the stage's barrier stays incomplete: nobody consumes it, the copies already issued
+                // the stage's barriers stay incomplete: nobody consumes it, the copies already issued
                 // land in the CTA's own shared memory during the wind-down pause
                 break;
               }
               asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores -> TMA reads
+              PROF_END(1);
             }
-            // activation block scales of the tile's tokens
+            // block scales of the tile's tokens
             if (lane < ntok) {
               const float* src = act_scale + static_cast<size_t>(rec.begin + p0 + lane) * nblk + k0 / 128;
-              const uint32_t xdst = smem_u32(st + SL.sx_off) + lane * 4;
+              const uint32_t xdst = smem_u32(&se->sx[0][lane]);
               for (int sg = 0; sg < nseg; ++sg)
                 asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(xdst + sg * 128), "l"(src + sg) : "memory");
             }
-            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(full) : "memory");
+            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(sfull) : "memory");
             if (lane == 0) {
               // the tokens' limb rows: rows 2*slot (hi) and 2*slot+1 (lo) of the activation image
               for (int sg = 0; sg < nseg; ++sg)
-                tma_load_2d(smem_u32(st + SL.b_off + sg * B_SEG_BYTES), bmap, k0 + sg * 128, 2 * (rec.begin + p0), full);
+                tma_load_2d(smem_u32(st + B_OFF + sg * B_SEG_BYTES), bmap, k0 + sg * 128, 2 * (rec.begin + p0), full);
             }
           } else {
-            mbar_arrive(full);  // with lane 0's arrival above: 33 in all
+            mbar_arrive(sfull);  // with lane 0's arrival above: 33 in all
           }
           ring.next(STAGES);
+          sring.next(I8_SIDE);
         }
       }
       // the ring still holds several stages of work: fetching the next item only now costs nothing
@@ -369,139 +490,221 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       if (lane == 0) item_next = gridDim.x + atomicAdd(a.plan + 1 + a.phase_begin, 1);
       item = __shfl_sync(0xffffffffu, item_next, 0);
     }
+#ifdef EMOE_I8_PROFILE
+    prof_acc[2] = clock64() - prof_start;
+#endif
+    PROF_STORE(0, 3);
     if (ok && !__any_sync(0xffffffffu, *abort_flag != 0)) {  // tell the others that nothing else comes
-      if (wait_warp(bar_empty + 8 * ring.i, ring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
+      if (wait_warp(bar_empty + 8 * ring.i, ring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag) &&
+          wait_warp(bar_sempty + 8 * sring.i, sring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
         if (lane == 0) {
-          meta[ring.i].flags = META_STOP;
-          mbar_arrive(bar_full + 8 * ring.i);  // lane 0 arrives twice: once for itself, once in place of a copy
+          side[sring.i].m.flags = META_STOP;
+          mbar_arrive(bar_sfull + 8 * sring.i);
         }
         __syncwarp();
-        mbar_arrive(bar_full + 8 * ring.i);
+        mbar_arrive(bar_sfull + 8 * sring.i);
+        if (lane == 0) mbar_arrive(bar_full + 8 * ring.i);
       }
     }
+  } else if (warp == I8_WARP_SCALES) {
+    // ---------------- scale warp: weight scales of every stage into the scale ring ----------------
+    // (SCALE_STAGE projections only; in the other modes the producer's bulk copies bring the scales.)
+    // Lane l copies the windows of rows 4l .. 4l+3 of every matrix of the stage.  The scales a
+    // stage needs from a row (groups of inputs k0 .. k0 + 128 * segments) are a few neighbouring
+    // bytes of the row's scale channel; they are copied in 4-byte words from the 4-byte boundary at or
+    // below the first one, into a 16-byte window per row.
+    const int ssz = L.scale_f16 ? 2 : 4;
+    Ring sring{0, 0}, wring{0, 0};
+    while (true) {
+      if (!wait_warp(bar_sfull + 8 * sring.i, sring.ph, a.wait_limit, a.check_word, abort_flag)) break;
+      const StageMeta m = side[sring.i].m;
+      if (m.flags & META_STOP) break;
+      if (!(m.flags & META_EMPTY) && a.scale_mode[m.phase] == SCALE_STAGE) {
+        if (!wait_warp(bar_wempty + 8 * wring.i, wring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) break;
+        const int N = m.phase == 0 ? L.d_ff : L.d_model;
+        const int ngroups = a.ngroups[m.phase];
+        const int nmat = (DUAL && m.phase == 0) ? 2 : 1;
+        const int g0 = group_of(m.k0, a.gshift, L.group, ngroups),
+                  g1 = group_of(m.k0 + (m.nseg - 1) * 128, a.gshift, L.group, ngroups);
+        const uint32_t sdst = smem_u32(scale_ring + wring.i * SCALE_ENTRY);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int row = 4 * lane + r;
+          const int off = min(m.rb * I8_ROWS + row, N - 1) * ngroups * ssz;
+          const int b0 = (off + g0 * ssz) & ~3;
+          const int b1 = off + (g1 + 1) * ssz;
+          for (int mt = 0; mt < nmat; ++mt) {
+            const char* sbase = static_cast<const char*>(m.scales[mt]);
+#pragma unroll 1
+            for (int w = 0; b0 + 4 * w < b1; ++w)
+              asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + (mt * I8_ROWS + row) * 16 + 4 * w),
+                           "l"(sbase + b0 + 4 * w)
+                           : "memory");
+          }
+        }
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_wfull + 8 * wring.i) : "memory");
+        wring.next(I8_SCALE_RING);
+      }
+      sring.next(I8_SIDE);
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");  // nothing of this warp is in flight when the CTA ends
   } else if (warp == I8_WARP_MMA) {
     // ---------------- MMA issuer (one lane) ----------------
     if (lane == 0) {
       // kind::i8: s8 x s8 -> s32, both operands K-major, M = 128, N = 2 * NT
       const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((static_cast<uint32_t>(NCOL) >> 3) << 17) |
                              ((static_cast<uint32_t>(I8_ROWS) >> 4) << 24);
-      Ring ring{0, 0}, dring{0, 0};
-      uint32_t q = 0;  // A tiles that went through tensor memory so far
+      Ring ring{0, 0}, sring{0, 0}, gring{0, 0};
+      uint32_t qs = 0;  // segments that went through the A ring so far
       bool ok = true;
+      PROF_DECL;
       while (ok) {
+        PROF_BEGIN;
         if (!wait_lim(bar_full + 8 * ring.i, ring.ph, a.wait_limit, a.check_word, abort_flag)) break;
+        PROF_END(0);
         tc_fence_after();
-        const StageMeta m = meta[ring.i];
+        const StageMeta m = side[sring.i].m;
         if (m.flags & META_STOP) break;
         if (m.flags & META_EMPTY) {
           mbar_arrive(bar_empty + 8 * ring.i);
           ring.next(STAGES);
+          sring.next(I8_SIDE);
           continue;
         }
-        const uint32_t st = smem_u32(smem + ring.i * SL.bytes);
+        const uint32_t st = smem_u32(smem + ring.i * STAGE_BYTES);
         const int nmat = (DUAL && m.phase == 0) ? 2 : 1;
         for (int mt = 0; mt < nmat && ok; ++mt) {
-          const uint32_t abuf = q & 1u;
-          if (m.bits != 8) {
-            if (!wait_lim(bar_afull + 8 * abuf, (q >> 1) & 1u, a.wait_limit, a.check_word, abort_flag)) {
-              ok = false;
-              break;
-            }
-            tc_fence_after();
-          }
           const uint64_t adesc = umma_desc(st + mt * I8_MAT_BYTES);
-          for (int sg = 0; sg < m.nseg; ++sg) {
-            if (!wait_lim(bar_dempty + 8 * dring.i, dring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
+          for (int sg0 = 0; sg0 < m.nseg && ok; sg0 += GSEGS) {
+            PROF_BEGIN;
+            if (!wait_lim(bar_dempty + 8 * gring.i, gring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
               ok = false;
               break;
             }
+            PROF_END(2);
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + I8_D_COL0 + dring.i * NCOL;
-            const uint64_t bdesc = umma_desc(st + SL.b_off + sg * B_SEG_BYTES);
+            const int sg1 = min(m.nseg, sg0 + GSEGS);
+            for (int sg = sg0; sg < sg1; ++sg) {
+              const uint32_t d_tmem = tmem_base + I8_D_COL0 + gring.i * GCOLS + (sg - sg0) * NCOL;
+              const uint64_t bdesc = umma_desc(st + B_OFF + sg * B_SEG_BYTES);
+              if (m.bits == 8) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {  // 32 inputs per MMA
-              if (m.bits == 8)
-                umma_i8_ss(d_tmem, adesc + 2 * j, bdesc + 2 * j, idesc, j > 0 ? 1u : 0u);
-              else
-                umma_i8_ts(d_tmem, tmem_base + abuf * I8_A_COLS + sg * 32 + j * 8, bdesc + 2 * j, idesc, j > 0 ? 1u : 0u);
+                for (int j = 0; j < 4; ++j)  // 32 inputs per MMA
+                  umma_i8_ss(d_tmem, adesc + 2 * j, bdesc + 2 * j, idesc, j > 0 ? 1u : 0u);
+              } else {
+                const uint32_t slot = qs & (I8_A_SLOTS - 1);
+                PROF_BEGIN;
+                if (!wait_lim(bar_afull + 8 * slot, (qs / I8_A_SLOTS) & 1u, a.wait_limit, a.check_word, abort_flag)) {
+                  ok = false;
+                  break;
+                }
+                PROF_END(1);
+                tc_fence_after();
+                const uint32_t a_tmem = tmem_base + slot * I8_A_SLOT_COLS;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                  umma_i8_ts(d_tmem, a_tmem + 8 * j, bdesc + 2 * j, idesc, j > 0 ? 1u : 0u);
+                umma_commit(bar_aempty + 8 * slot);
+                ++qs;
+              }
             }
-            umma_commit(bar_dfull + 8 * dring.i);
-            dring.next(NDBUF);
-          }
-          if (!ok) break;
-          if (m.bits != 8) {
-            umma_commit(bar_aempty + 8 * abuf);
-            ++q;
+            if (!ok) break;
+            umma_commit(bar_dfull + 8 * gring.i);
+            gring.next(NGRP);
           }
         }
         if (!ok) break;
         umma_commit(bar_empty + 8 * ring.i);  // the stage's shared memory may be refilled once these MMAs have read it
         ring.next(STAGES);
+        sring.next(I8_SIDE);
       }
+      PROF_STORE(3, 3);
     }
   } else if (warp >= I8_WARP_UNPACK0) {
     // ---------------- unpack warps: packed codes -> int8 rows in tensor memory ----------------
-    const uint32_t wg = static_cast<uint32_t>(warp - I8_WARP_UNPACK0) >> 2;  // 0 or 1: which A tile is ours
-    const int r = 32 * (warp & 3) + lane;                                    // row of the item = tensor-memory lane
-    const uint32_t a_tmem = tmem_base + (static_cast<uint32_t>(32 * (warp & 3)) << 16) + wg * I8_A_COLS;
+    // segment number qs of the kernel goes to slot qs % 8 of the A ring; even segments are this
+    // group's if wg = 0, odd ones if wg = 1
+    const uint32_t wg = static_cast<uint32_t>(warp - I8_WARP_UNPACK0) >> 2;
+    const int r = 32 * (warp & 3) + lane;  // row of the item = tensor-memory lane
+    const uint32_t a_tmem0 = tmem_base + (static_cast<uint32_t>(32 * (warp & 3)) << 16);
     const int row_off = (r >> 6) * I8_BOX_BYTES + (r & 63) * 128;
     const int swz = r & 7;
-    Ring ring{0, 0};
-    uint32_t q = 0, uses = 0;
+    Ring ring{0, 0}, sring{0, 0};
+    uint32_t qs = 0;
     bool ok = true;
+    PROF_DECL;
     while (ok) {
+      PROF_BEGIN;
       if (!wait_warp(bar_full + 8 * ring.i, ring.ph, a.wait_limit, a.check_word, abort_flag)) break;
-      const int flags = meta[ring.i].flags;
+      PROF_END(0);
+      const int flags = side[sring.i].m.flags;
       if (flags & META_STOP) break;
-      const int bits = meta[ring.i].bits, nseg = meta[ring.i].nseg, phase = meta[ring.i].phase;
+      const int bits = side[sring.i].m.bits, nseg = side[sring.i].m.nseg, phase = side[sring.i].m.phase;
       if (!(flags & META_EMPTY) && bits != 8) {
         const int nmat = (DUAL && phase == 0) ? 2 : 1;
-        for (int mt = 0; mt < nmat; ++mt, ++q) {
-          if ((q & 1u) != wg) continue;
-          if (!wait_warp(bar_aempty + 8 * wg, (uses & 1u) ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const unsigned char* row = smem + ring.i * SL.bytes + mt * I8_MAT_BYTES + row_off;
-          if (bits == 4) {
-            // a 16-byte chunk = 32 codes = 8 columns; 4 chunks per 128-input segment
-#pragma unroll 2
-            for (int c = 0; c < 4 * nseg; ++c) {
-              uint32_t o[8];
-              unpack4(*reinterpret_cast<const uint4*>(row + ((c ^ swz) << 4)), o);
-              tmem_st8(a_tmem + 8 * c, o);
+        for (int mt = 0; mt < nmat && ok; ++mt) {
+          const unsigned char* row = smem + ring.i * STAGE_BYTES + mt * I8_MAT_BYTES + row_off;
+          for (int sg = 0; sg < nseg; ++sg, ++qs) {
+            if ((qs & 1u) != wg) continue;
+            const uint32_t slot = qs & (I8_A_SLOTS - 1);
+            PROF_BEGIN;
+            if (!wait_warp(bar_aempty + 8 * slot, ((qs / I8_A_SLOTS) & 1u) ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
+              ok = false;
+              break;
             }
-          } else {
-            // a 16-byte chunk = 64 codes = 16 columns; 2 chunks per segment
-#pragma unroll 2
-            for (int c = 0; c < 2 * nseg; ++c) {
-              uint32_t o[16];
-              unpack2(*reinterpret_cast<const uint4*>(row + ((c ^ swz) << 4)), o);
-              tmem_st16(a_tmem + 16 * c, o);
+            PROF_END(1);
+            PROF_BEGIN;
+            tc_fence_after();
+            const uint32_t a_tmem = a_tmem0 + slot * I8_A_SLOT_COLS;
+            if (bits == 4) {
+              // a 16-byte chunk = 32 codes = 8 columns; 4 chunks per segment
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                uint32_t o[8];
+                unpack4(*reinterpret_cast<const uint4*>(row + (((4 * sg + c) ^ swz) << 4)), o);
+                tmem_st8(a_tmem + 8 * c, o);
+              }
+            } else {
+              // a 16-byte chunk = 64 codes = 16 columns; 2 chunks per segment
+#pragma unroll
+              for (int c = 0; c < 2; ++c) {
+                uint32_t o[16];
+                unpack2(*reinterpret_cast<const uint4*>(row + (((2 * sg + c) ^ swz) << 4)), o);
+                tmem_st16(a_tmem + 16 * c, o);
+              }
             }
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_afull + 8 * slot);
+            PROF_END(2);
           }
-          tmem_st_wait();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_afull + 8 * wg);
-          ++uses;
         }
       }
+      // this warp is through with the stage (its codes and its record), whatever the width
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + 8 * ring.i);
       ring.next(STAGES);
+      sring.next(I8_SIDE);
     }
+    if (warp == I8_WARP_UNPACK0) { PROF_STORE(6, 3); }
   } else {
     // ---------------- epilogue warps: one thread per output row ----------------
     const int r = 32 * warp + lane;
     const uint32_t d_tmem0 = tmem_base + (static_cast<uint32_t>(32 * warp) << 16) + I8_D_COL0;
     float tot[NMAT_MAX][NT];
-    Ring ring{0, 0}, dring{0, 0};
+    Ring sring{0, 0}, gring{0, 0}, wring{0, 0}, cring{0, 0};
     uint32_t exchanges = 0;  // first-projection items finished so far (each uses the exchange barrier once)
     bool ok = true;
+    PROF_DECL;
     while (ok) {
-      if (!wait_warp(bar_full + 8 * ring.i, ring.ph, a.wait_limit, a.check_word, abort_flag)) break;
-      const StageMeta m = meta[ring.i];
+      PROF_BEGIN;
+      if (!wait_warp(bar_sfull + 8 * sring.i, sring.ph, a.wait_limit, a.check_word, abort_flag)) break;
+      PROF_END(0);
+      const SideEntry& se = side[sring.i];
+      const StageMeta m = se.m;
       if (m.flags & META_STOP) break;
+      PROF_BEGIN;
       if (m.flags & META_FIRST) {
 #pragma unroll
         for (int mt = 0; mt < NMAT_MAX; ++mt)
@@ -511,57 +714,112 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       const int N = m.phase == 0 ? L.d_ff : L.d_model;
       const int n = m.rb * I8_ROWS + r;
       if (!(m.flags & META_EMPTY)) {
-        const unsigned char* st = smem + ring.i * SL.bytes;
         const int nmat = (DUAL && m.phase == 0) ? 2 : 1;
+        // this row's weight scales of the stage, from the scale ring
+        float sw[NMAT_MAX][4];
         const int ngroups = a.ngroups[m.phase];
-        const int g0 = group_of(m.k0, a.gshift, L.group, ngroups);
-        // the row's scale window starts at the 4-byte boundary at or below its first scale of the stage
-        const unsigned char* sc_row = st + SL.sc_off + r * 16 + (((min(n, N - 1) * ngroups + g0) * ssz) & 3);
+        const int ssz = L.scale_f16 ? 2 : 4;
         const float unit = m.bits == 8 ? 1.0f : (m.bits == 4 ? 0.0625f : 0.015625f);  // codes arrive as 16 q / 64 q
+        const bool per_stage = a.scale_mode[m.phase] == SCALE_STAGE;
+        const unsigned char* sc_row;  // where the scale of the row's group 0 would sit
+        int mat_stride;
+        if (per_stage) {
+          if (!wait_warp(bar_wfull + 8 * wring.i, wring.ph, a.wait_limit, a.check_word, abort_flag)) break;
+          // the row's window starts at the 4-byte boundary at or below its first scale of the stage
+          const int g0 = group_of(m.k0, a.gshift, L.group, ngroups);
+          sc_row = scale_ring + wring.i * SCALE_ENTRY + r * 16 + (((min(n, N - 1) * ngroups + g0) * ssz) & 3) - g0 * ssz;
+          mat_stride = I8_SCALE_TILE;
+        } else {
+          PROF_LAP(6);
+          if (m.flags & META_NEW_CHUNK) {
+            if (!wait_warp(bar_cfull + 8 * cring.i, cring.ph, a.wait_limit, a.check_word, abort_flag)) break;
+            cring.next(I8_CHUNKS);
+          }
+          PROF_LAP(7);
+          sc_row = scale_ring + m.chunk * CHUNK_ENTRY + r * m.pitch - m.win0;
+          mat_stride = I8_CHUNK_BYTES;
+        }
+#pragma unroll
+        for (int mt = 0; mt < NMAT_MAX; ++mt)
+#pragma unroll
+          for (int sg = 0; sg < 4; ++sg) {
+            sw[mt][sg] = 0.0f;
+            if (mt < nmat && sg < m.nseg) {
+              const unsigned char* sc = sc_row + mt * mat_stride + group_of(m.k0 + sg * 128, a.gshift, L.group, ngroups) * ssz;
+              sw[mt][sg] = unit * (ssz == 2 ? __half2float(*reinterpret_cast<const __half*>(sc))
+                                            : *reinterpret_cast<const float*>(sc));
+            }
+          }
+        __syncwarp();
+        if (per_stage) {
+          if (lane == 0) mbar_arrive(bar_wempty + 8 * wring.i);
+          wring.next(I8_SCALE_RING);
+        } else if (m.flags & META_END_CHUNK) {
+          if (lane == 0) mbar_arrive(bar_cempty + 8 * m.chunk);
+        }
+        PROF_LAP(3);
 #pragma unroll
         for (int mt = 0; mt < NMAT_MAX; ++mt) {
           if (mt >= nmat || !ok) break;
-#pragma unroll 1
-          for (int sg = 0; sg < m.nseg; ++sg) {
-            if (!wait_warp(bar_dfull + 8 * dring.i, dring.ph, a.wait_limit, a.check_word, abort_flag)) {
+#pragma unroll
+          for (int g = 0; g < 4 / GSEGS; ++g) {
+            if (g * GSEGS >= m.nseg) break;
+            PROF_BEGIN;
+            if (!wait_warp(bar_dfull + 8 * gring.i, gring.ph, a.wait_limit, a.check_word, abort_flag)) {
               ok = false;
               break;
             }
+            PROF_LAP(1);
             tc_fence_after();
-            const unsigned char* sc = sc_row + mt * I8_SCALE_BYTES + (group_of(m.k0 + sg * 128, a.gshift, L.group, ngroups) - g0) * ssz;
-            const float sw = unit * (ssz == 2 ? __half2float(*reinterpret_cast<const __half*>(sc))
-                                              : *reinterpret_cast<const float*>(sc));
-            const float* sx = reinterpret_cast<const float*>(st + SL.sx_off) + sg * 32;
-            const uint32_t d_tmem = d_tmem0 + dring.i * NCOL;
+            const uint32_t d_tmem = d_tmem0 + gring.i * GCOLS;
+            // the group in chunks of 32 columns (2 segments at NT = 8, 1 at 16, half a segment at 32);
+            // the next chunk is requested before the current one is worked on
+            constexpr int NCHUNK = GCOLS / 32;
+            constexpr int TOK_PER_CHUNK = NT < 16 ? NT : 16;  // tokens of one segment inside a chunk
+            const int ncols = min(GSEGS, m.nseg - g * GSEGS) * NCOL;
+            uint32_t acc[2][32];
+            tmem_ld32(d_tmem, acc[0]);
 #pragma unroll
-            for (int half = 0; half < (NT + 15) / 16; ++half) {
-              constexpr int TT = NT < 16 ? NT : 16;  // tokens per read
-              uint32_t acc[2 * TT];
-              if constexpr (TT == 8) tmem_ld16(d_tmem, acc);
-              else tmem_ld32(d_tmem + half * 32, acc);
+            for (int c = 0; c < NCHUNK; ++c) {
+              if (c * 32 >= ncols) break;
               tmem_ld_wait();
-              if (half == (NT + 15) / 16 - 1) {  // the accumulator may be overwritten
+              const bool more = (c + 1) * 32 < ncols;
+              if (c + 1 < NCHUNK && more) tmem_ld32(d_tmem + (c + 1) * 32, acc[(c + 1) & 1]);
+              if (!more) {  // the last chunk is in registers: the accumulators may be overwritten
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_dempty + 8 * dring.i);
+                if (lane == 0) mbar_arrive(bar_dempty + 8 * gring.i);
               }
+              PROF_LAP(4);
 #pragma unroll
-              for (int t = 0; t < TT; ++t) {
-                if (half * 16 + t < m.ntok) {
-                  const int v = static_cast<int>(acc[2 * t]) * 128 + static_cast<int>(acc[2 * t + 1]);
-                  tot[mt][half * 16 + t] = fmaf(static_cast<float>(v), sw * sx[half * 16 + t], tot[mt][half * 16 + t]);
+              for (int u = 0; u < 32 / (2 * TOK_PER_CHUNK); ++u) {  // segments (or half segments) inside the chunk
+                const int col0 = c * 32 + u * 2 * TOK_PER_CHUNK;    // first column of this piece in the group
+                const int sg = g * GSEGS + col0 / NCOL;              // its segment in the stage
+                const int t0 = (col0 % NCOL) / 2;                    // its first token
+                if (sg < m.nseg) {
+                  const float s = sw[mt][sg < 4 ? sg : 3];
+#pragma unroll
+                  for (int t = 0; t < TOK_PER_CHUNK; ++t) {
+                    if (t0 + t < m.ntok) {
+                      const int v = static_cast<int>(acc[c & 1][u * 2 * TOK_PER_CHUNK + 2 * t]) * 128 +
+                                    static_cast<int>(acc[c & 1][u * 2 * TOK_PER_CHUNK + 2 * t + 1]);
+                      tot[mt][t0 + t] = fmaf(static_cast<float>(v), s * se.sx[sg < 4 ? sg : 3][t0 + t], tot[mt][t0 + t]);
+                    }
+                  }
                 }
               }
             }
-            dring.next(NDBUF);
+            PROF_LAP(5);
+            gring.next(NGRP);
           }
         }
         if (!ok) break;
       }
-      // the stage's scales are no longer needed
+      // the side entry is no longer needed
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_empty + 8 * ring.i);
+      if (lane == 0) mbar_arrive(bar_sempty + 8 * sring.i);
       if (m.flags & META_LAST) {
+        PROF_BEGIN;
         if (m.phase == 0) {
           // hidden values of this row: activation, rounded to bf16 (the hidden vector is a bf16
           // tensor), then to limbs under the block scale of the item's 128 rows
@@ -613,9 +871,11 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
             if (t < m.ntok)
               a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + (m.begin + m.p0 + t)) * N + n] = tot[0][t];
         }
+        PROF_END(2);
       }
-      ring.next(STAGES);
+      sring.next(I8_SIDE);
     }
+    if (warp == 0) { PROF_STORE(9, 8); }
   }
 
   // wind-down: after a wait that ran out, give copies and MMAs in flight time to land before the
@@ -633,8 +893,8 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
 }
 
 int stages_for(int nt, int nmat) {
-  const StageLayout sl = stage_layout(nt, nmat);
-  int s = (I8_SMEM_LIMIT - 1024 /*alignment slack*/ - 3072 /*static*/) / sl.bytes;
+  static_assert(I8_CHUNKS * I8_CHUNK_BYTES == I8_SCALE_RING * I8_SCALE_TILE, "both kinds of scale ring take the same room");
+  int s = (I8_SMEM_LIMIT - 1024 /*alignment slack*/ - I8_STATIC_SMEM - I8_SCALE_RING * nmat * I8_SCALE_TILE) / stage_bytes(nt, nmat);
   return s > I8_MAX_STAGES ? I8_MAX_STAGES : s;
 }
 
@@ -644,7 +904,7 @@ cudaError_t launch_variant(const I8Args& a_in, const CUtensorMap& tx, const CUte
   I8Args a = a_in;
   a.stages = stages_for(NT, DUAL ? 2 : 1);
   if (a.stages < 3) return cudaErrorInvalidValue;
-  const int smem = a.stages * stage_layout(NT, DUAL ? 2 : 1).bytes + 1024;
+  const int smem = a.stages * stage_bytes(NT, DUAL ? 2 : 1) + I8_SCALE_RING * (DUAL ? 2 : 1) * I8_SCALE_TILE + 1024;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -665,6 +925,8 @@ cudaError_t launch_variant(const I8Args& a_in, const CUtensorMap& tx, const CUte
 }
 
 }  // namespace
+
+long long* g_i8_profile = nullptr;
 
 bool ffn_i8_supported(const LayerDims& L) {
   // bf16 activations, inputs in whole 128-blocks, scale groups of whole blocks; the tensor maps use
@@ -696,7 +958,7 @@ int ffn_i8_ksplit(const LayerDims& L, int T) {
   return static_cast<int>(z);
 }
 
-cudaError_t launch_ffn_i8(int phase_begin, int phase_end, const LayerDims& L, const void* wmaps, const void* xq,
+cudaError_t launch_ffn_i8(int phase_begin, int phase_end, const LayerDims& L, const void* wmaps, const void* smaps, const void* xq,
                           const float* xsc, int* plan, void* hq, float* hsc, float* o_part, int ksplit, int n_pairs,
                           int T, int token_tile, unsigned wait_limit, int dep_extra, int* check_word, cudaStream_t st) {
   if (phase_begin < 0 || phase_end > 2 || phase_begin >= phase_end) return cudaErrorInvalidValue;
@@ -706,6 +968,7 @@ cudaError_t launch_ffn_i8(int phase_begin, int phase_end, const LayerDims& L, co
   a.phase_end = phase_end;
   a.L = L;
   a.wmaps = static_cast<const CUtensorMap*>(wmaps);
+  a.smaps = static_cast<const CUtensorMap*>(smaps);
   a.plan = plan;
   a.xsc = xsc;
   a.hq = static_cast<int8_t*>(hq);
@@ -719,12 +982,25 @@ cudaError_t launch_ffn_i8(int phase_begin, int phase_end, const LayerDims& L, co
   a.gshift = -1;
   for (int b = 7; b < 31; ++b)
     if (L.group == (1 << b)) a.gshift = b;
+  // how the weight scales travel (smaps is null when a scale channel of the table is not 16-byte aligned)
+  for (int p = 0; p < 2; ++p) {
+    const int row_bytes = a.ngroups[p] * (L.scale_f16 ? 2 : 4);
+    const bool pow2_groups = a.ngroups[p] == 1 || a.gshift >= 0;
+    a.scale_mode[p] = !smaps || !pow2_groups ? SCALE_STAGE
+                      : row_bytes <= I8_CHUNK_ROW ? SCALE_BLOCK
+                      : row_bytes % 16 == 0 ? SCALE_WINDOW
+                                            : SCALE_STAGE;
+  }
+  // both kinds of ring entry share one region of shared memory: one projection on the general path
+  // puts the other there too
+  if (a.scale_mode[0] == SCALE_STAGE || a.scale_mode[1] == SCALE_STAGE) a.scale_mode[0] = a.scale_mode[1] = SCALE_STAGE;
   a.n_pairs = n_pairs;
   a.stages = 0;
-  a.wait_limit = wait_limit ? wait_limit : PIPE_WAIT_LIMIT;
+  a.wait_limit = wait_limit ? wait_limit : (1u << 20);  // polls of up to a microsecond each
   a.dep_wait_limit = wait_limit ? wait_limit : (1u << 20);
   a.dep_extra = dep_extra;
   a.check_word = check_word;
+  a.prof = g_i8_profile;
   // activation images: [2 * n_pairs rows][K bytes], boxes of 2*nt rows x 128 bytes, 128-byte swizzle
   CUtensorMap tx, th;
   if (encode_tmap_2d(&tx, 0, xq, static_cast<uint64_t>(L.d_model), 2ull * n_pairs, static_cast<uint64_t>(L.d_model), 128, 2 * nt) != 0)

@@ -754,7 +754,7 @@ cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, c
 // dtype: 0 = bytes, 1 = fp16.  2-D row-major image [outer][inner], box [box_outer][box_inner],
 // 128-byte swizzle (box_inner * element size must be 128 bytes or less).
 int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_bytes,
-                   uint32_t box_inner, uint32_t box_outer) {
+                   uint32_t box_inner, uint32_t box_outer, bool swizzle128) {
   typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -772,8 +772,17 @@ int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, u
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = fn(static_cast<CUtensorMap*>(out_map), dtype == 1 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
                         2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, EMOE_TMA_L2PROMO, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                        swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, EMOE_TMA_L2PROMO,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? 0 : -3;
+}
+
+// One tensor map per scale channel whose rows are a multiple of 16 bytes: a [N][row_bytes] byte image,
+// boxes of 128 rows x 32 bytes, no swizzle (the int8 streaming kernel's scale windows).
+int encode_scale_tmap(void* out_map, const void* scales, int N, int row_bytes) {
+  if (row_bytes < 32 || row_bytes % 16 != 0 || N < 128) return -2;
+  return encode_tmap_2d(out_map, 0, scales, static_cast<uint64_t>(row_bytes), static_cast<uint64_t>(N),
+                        static_cast<uint64_t>(row_bytes), 32, 128, false);
 }
 
 // One tensor map per packed matrix: a [N][row_bytes] byte image, 64-row x 128-byte boxes, 128-byte swizzle.

@@ -28,6 +28,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same test, but the hardware may park the thread until the phase completes or `ns` nanoseconds
+// have passed: a waiting warp then costs neither issue slots nor shared-memory traffic, and it
+// resumes as soon as the phase completes.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false (after flagging the check word) if the phase never completed.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* check_word, volatile int* abort_flag) {
   for (unsigned i = 0; i < PIPE_WAIT_LIMIT; ++i) {

@@ -9,7 +9,8 @@ import pytest
 from oracle.cache_sim import ExpertBufferModel, rank_experts
 from paper_2308_14352_b200 import binding as B
 
-RULES = [("forward", B.EVICT_FORWARD), ("printed", B.EVICT_PRINTED), ("lru", B.EVICT_LRU)]
+RULES = [("forward", B.EVICT_FORWARD), ("printed", B.EVICT_PRINTED), ("lru", B.EVICT_LRU), ("lfu", B.EVICT_LFU),
+         ("fifo", B.EVICT_FIFO)]
 
 
 @pytest.mark.parametrize("rule,code", RULES)

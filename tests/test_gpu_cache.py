@@ -223,6 +223,14 @@ def test_cache_argument_errors():
         B.emoe_cache_release(ctx, [7], 0)
         B.emoe_cache_acquire(ctx, [8], 1, 0, 0)
         B.emoe_cache_release(ctx, [8], 0)
+        # a list that does not fit fails as a whole: the expert it had already taken is let go again
+        with pytest.raises(B.EmoeError) as ei:
+            B.emoe_cache_acquire(ctx, [7, 8], 0, 0, 0)
+        assert ei.value.status == B.ERR_CACHE_FULL
+        B.emoe_cache_acquire(ctx, [8], 1, 0, 0)                     # the only slot is free for it
+        B.emoe_cache_release(ctx, [8], 0)
+        with pytest.raises(B.EmoeError):
+            B.emoe_cache_release(ctx, [7, 8], 0)                    # neither is held
     finally:
         torch.cuda.synchronize()
         B.emoe_destroy(ctx)

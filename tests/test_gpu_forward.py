@@ -138,6 +138,35 @@ def test_int8_streaming_path_keeps_the_bf16_range():
         assert rel_to_max(y, y_ref) <= 2e-3, (scale_x, std, rel_to_max(y, y_ref))
 
 
+def test_bounded_wait_inside_the_kernel_runs_out_and_the_context_stays_usable():
+    """Failure detection without a fault: the second projection is told to expect one more
+    completion of the first than will ever be counted, with a short wait limit.  The wait must give
+    up, the kernels must return, the status call must say "timeout", and the next ordinary forward
+    on the same context must be right again."""
+    shape = inputs.LayerShape(512, 1024, 4, 1, "relu", "softmax", 128, "f16", "bf16")
+    bits, T = [8, 4, 2, 4], 6
+    W = inputs.expert_set(35, 0, shape)
+    x = inputs.activations(35, 0, T, shape.d_model, "bf16")
+    Wr = inputs.router_weight(35, 0, shape.d_model, shape.n_experts, std=0.05)
+    packed, scales = oracle_pack_layer(W, shape, bits)
+    with layer.MoELayer(shape, bits, max_tokens=T) as moe:
+        B.emoe_set_ffn_path(moe.ctx, 6)
+        moe.pack_from_host(W)
+        y, ids, gates, _ = moe.forward(x, Wr)
+        y_ref = oracle.moe_ffn_combine(x, shape.d_ff, shape.act, shape.group, True, bits, packed, scales, ids, gates)
+        assert rel_to_max(y, y_ref) <= 2e-3
+        B.emoe_set_wait_limit(moe.ctx, 20000)
+        B.emoe_debug_expect_extra_completions(moe.ctx, 1)
+        with pytest.raises(B.EmoeError) as ei:
+            moe.forward(x, Wr)                      # returns (no hang); the device check reports the timeout
+        assert ei.value.status == B.ERR_TIMEOUT
+        assert B.emoe_device_status(moe.ctx) == B.OK   # the word was cleared by the read above
+        B.emoe_debug_expect_extra_completions(moe.ctx, 0)
+        B.emoe_set_wait_limit(moe.ctx, 0)
+        y2, ids2, gates2, _ = moe.forward(x, Wr)
+        assert np.array_equal(ids2, ids) and np.array_equal(y2, y)
+
+
 UMMA_CASES = [
     ("relu", 128, "f16", 512, 1024, 4, 1, "softmax", [8, 4, 2, 4], 200),              # ~50 tokens per expert
     ("relu", 128, "f16", 512, 1024, 2, 1, "softmax", [4, 2], 300),                    # two token tiles per expert
@@ -196,7 +225,9 @@ def test_both_paths_agree_and_default_picks_tensor_cores():
     e_mma = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=2)
     assert e_auto == e_mma and e_gemv <= 2e-3
     big = inputs.LayerShape(512, 1024, 4, 2, "swiglu", "softmax_renorm", 128, "f16", "bf16")
-    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=0) == _run_case(big, [2, 4, 8, 4], 12, seed=23, path=3)
+    # wide enough for the weight-streaming kernels: the default is the int8 tensor-core one
+    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=0) == _run_case(big, [2, 4, 8, 4], 12, seed=23, path=6)
+    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=3) <= 2e-3
 
 
 def test_zipf_bias_and_many_tokens_on_one_expert():

@@ -84,7 +84,67 @@ def test_lru_rule_is_textbook_lru():
     assert m.counters["hits"] + m.counters["misses"] == 400
 
 
-@pytest.mark.parametrize("rule", ["forward", "printed", "lru"])
+def test_fifo_and_lfu_orders_worked_by_hand():
+    """Three slots, experts A B C D of one layer.  Loads: A, B, C (in that order); uses afterwards:
+    C twice, A once, B never again.  Every expert was activated once when it was loaded, so the
+    counts are A 2, B 1, C 3.
+      FIFO: the one loaded first leaves: A, then B, then C, whatever their use.
+      LFU: fewest activations first: B (1), then A (2), then C (3).
+      LRU for contrast: the touches in order are A, B, C, C, C, A, so the least recently touched
+      is B, then C, then A."""
+    def filled(rule):
+        m = ExpertBufferModel(3, 1, rule)
+        for e in "ABCD":
+            m.register(e, 0)
+        for e in "ABC":
+            m.acquire(e, 0)
+            m.release(e)
+        for e in "CCA":
+            assert m.acquire(e, 0)[1] is False
+            m.release(e)
+        return m
+    name = lambda m, order: [m.slot_content[s] for s in order]
+    assert name(filled("fifo"), filled("fifo").eviction_order(0)) == ["A", "B", "C"]
+    assert name(filled("lfu"), filled("lfu").eviction_order(0)) == ["B", "A", "C"]
+    assert name(filled("lru"), filled("lru").eviction_order(0)) == ["B", "C", "A"]
+    # and the eviction really takes the head of the order
+    m = filled("fifo")
+    assert m.acquire("D", 0) == (0, True, "A")
+    m = filled("lfu")
+    assert m.acquire("D", 0) == (1, True, "B")
+    # LFU ties (equal counts) go to the expert loaded earliest
+    t = ExpertBufferModel(2, 1, "lfu")
+    for e in "XYZ":
+        t.register(e, 0)
+    for e in "YX":
+        t.acquire(e, 0)
+        t.release(e)
+    assert t.acquire("Z", 0) == (0, True, "Y")
+
+
+def test_fifo_rule_is_a_textbook_queue():
+    rng = random.Random(9)
+    m = ExpertBufferModel(4, 6, "fifo")
+    for e in range(12):
+        m.register(e, e % 6)
+    queue = []
+    for step in range(400):
+        e = rng.randrange(12)
+        s, loaded, ev = m.acquire(e, step % 6)
+        m.release(e)
+        if e in queue:
+            assert not loaded and ev is None
+        else:
+            assert loaded
+            if len(queue) == 4:
+                assert ev == queue.pop(0)
+            else:
+                assert ev is None
+            queue.append(e)
+    assert set(m.where) == set(queue)
+
+
+@pytest.mark.parametrize("rule", ["forward", "printed", "lru", "lfu", "fifo"])
 def test_no_eviction_when_everything_fits_and_counters_add_up(rule):
     rng = random.Random(7)
     m = ExpertBufferModel(16, 4, rule)
