@@ -56,6 +56,7 @@ extern "C" {
 #define EMOE_ERR_DEVICE_CHECK (-6) /* a kernel found inconsistent data (e.g. an expert id out of range) */
 #define EMOE_ERR_CACHE_FULL (-7)   /* every slot of the expert cache is in use by an unfinished call */
 #define EMOE_ERR_TIMEOUT (-8)      /* a bounded wait inside a kernel ran out; the kernel gave up and returned */
+#define EMOE_ERR_RANGE (-9)        /* a value left the fp16 range of the selected kernel's operands (see emoe_moe_forward) */
 
 /* enums (plain ints in the ABI) */
 #define EMOE_DTYPE_F32 0
@@ -114,7 +115,8 @@ int emoe_last_cuda_error(const emoe_ctx* ctx);
 /* Reads (and clears) the device-side check word: EMOE_OK; EMOE_ERR_TIMEOUT if a bounded wait
  * inside a kernel of an earlier call ran out (the kernel gave up and returned; results of that
  * call are undefined, the context stays usable); else EMOE_ERR_DEVICE_CHECK if a kernel met
- * inconsistent data (an expert id out of range).  Synchronises `stream`. */
+ * inconsistent data (an expert id out of range); else EMOE_ERR_RANGE (see emoe_moe_forward:
+ * "Range").  Synchronises `stream`. */
 int emoe_device_status(emoe_ctx* ctx, void* stream);
 
 const char* emoe_status_string(int status);
@@ -190,6 +192,12 @@ int emoe_permute(emoe_ctx* ctx, const int32_t* ids, int n_pairs, int E, int32_t*
  *     the first time a table is seen.
  *   out_ids / out_gates ([T][top_k]) and out_perm ([T*top_k]) are optional (NULL) copies
  *   of the routing decisions.
+ * Range: with BF16 activations the default tensor-core kernels carry x and the hidden vector as
+ * fp16 operands (exact for bf16 values up to 65504 in magnitude) and the many-token grouped GEMM also
+ * rounds q * s to fp16.  A value beyond 65504 is saturated, and a scale below 2^-14 in the grouped
+ * GEMM loses bits: both set a flag that emoe_device_status reports as EMOE_ERR_RANGE, and y is then
+ * not within the usual bound of the definition.  Kernel family 6 (emoe_set_ffn_path) and the
+ * CUDA-core family 1 have no such limit: they follow the full bf16 exponent range.
  * Shape limits: d_model and d_ff multiples of 32 with K*bits/8 a multiple of 16 for every
  * matrix; group 0 or a multiple of 32 (INT8), 32 (INT4), 64 (INT2) dividing K.
  * Uses the context workspace (emoe_workspace_bytes). */
@@ -205,10 +213,11 @@ int emoe_moe_forward_routed(emoe_ctx* ctx, const emoe_layer_desc* desc, const vo
 
 /* Selects the expert-FFN kernel family: 0 = automatic (default), 1 = the CUDA-core grouped
  * GEMV, 2 = the tensor-core kernel with register-staged weight loads, 3 = the fp16 mma.sync
- * kernel with the TMA-staged weight pipeline, 4 = the tcgen05 grouped GEMM (fp16 operands; meant
- * for many tokens per expert), 6 = the weight-streaming kernel on 8-bit integer tcgen05 operands
- * (what 0 picks for decode batches), 5 = 6 and 4 in one call: experts with at most 32 tokens take
- * the streaming kernel, the others the grouped GEMM (what 0 picks for large batches).
+ * kernel with the TMA-staged weight pipeline (what 0 picks for decode batches), 4 = the tcgen05
+ * grouped GEMM (fp16 operands; meant for many tokens per expert), 5 = 3 and 4 in one call: experts
+ * with at most 32 tokens take the streaming kernel, the others the grouped GEMM (what 0 picks for
+ * large batches), 6 = the weight-streaming kernel on 8-bit integer tcgen05 operands with block-scaled
+ * integer activations (no fp16 range limit; at present slower than 3).
  * 2 to 6 fail with EMOE_ERR_UNSUPPORTED in forward calls whose shape they do not take.  For tests
  * and measurements. */
 int emoe_set_ffn_path(emoe_ctx* ctx, int path);

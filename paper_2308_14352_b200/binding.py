@@ -22,6 +22,7 @@ ERR_CUDA = -5
 ERR_DEVICE_CHECK = -6
 ERR_CACHE_FULL = -7
 ERR_TIMEOUT = -8
+ERR_RANGE = -9
 EVICT_FORWARD, EVICT_PRINTED, EVICT_LRU, EVICT_LFU, EVICT_FIFO = 0, 1, 2, 3, 4
 
 DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2

@@ -306,10 +306,11 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   const bool many_tokens = ffn_many_tokens(L, T);
   // skewed loads: experts with few tokens stream through the TMA kernel, the others take the
   // tcgen05 grouped GEMM, in the same forward call
-  const bool use_hybrid = can_umma && can_i8 && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens));
+  const bool use_hybrid = can_umma && can_tma && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens));
   const bool use_umma = !use_hybrid && can_umma && (ctx->ffn_path == 4 || (ctx->ffn_path == 0 && many_tokens));
-  // the weight-streaming kernels: int8 tensor-core operands by default, the fp16 mma.sync one on request
-  const bool use_i8 = !use_hybrid && !use_umma && can_i8 && (ctx->ffn_path == 0 || ctx->ffn_path == 6);
+  // the weight-streaming kernels: the fp16 mma.sync one by default (the faster of the two as measured), the
+  // one on int8 tcgen05 operands on request
+  const bool use_i8 = !use_hybrid && !use_umma && can_i8 && ctx->ffn_path == 6;
   const bool use_tma = !use_hybrid && !use_umma && !use_i8 && can_tma && (ctx->ffn_path == 0 || ctx->ffn_path == 3);
   const bool use_mma = ffn_mma_supported(L) && ctx->ffn_path != 1;
   if (ctx->ffn_path == 2 && !use_mma) return EMOE_ERR_UNSUPPORTED;
@@ -341,24 +342,25 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
 #ifndef EMOE_HYBRID_TOKENS
 #define EMOE_HYBRID_TOKENS 32
 #endif
-#ifndef EMOE_HYBRID_TILE
-#define EMOE_HYBRID_TILE 16  // tokens per pass of the streaming family
+#ifndef EMOE_HYBRID_TILES
+#define EMOE_HYBRID_TILES 1  // 8-token tiles per pass of the streaming family
 #endif
     constexpr int HYBRID_STREAM_TOKENS = EMOE_HYBRID_TOKENS;
     int* plan_heavy = reinterpret_cast<int*>(reinterpret_cast<char*>(plan) + align_up(plan_bytes(L.E)));
-    ksplit = ffn_i8_ksplit(L, T);
-    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, xsc, P, 2, 1, HYBRID_STREAM_TOKENS, st));
-    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan_heavy, xs, P, HYBRID_STREAM_TOKENS + 1, INT_MAX, st));
+    __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
+    ksplit = ffn_tma_ksplit(L, T);
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, nullptr, P, 1, 1, HYBRID_STREAM_TOKENS, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan_heavy, xs, P, HYBRID_STREAM_TOKENS + 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     // the tcgen05 kernel writes plane 0 only: the other split-K planes of its slots must read as zero
     if (ksplit > 1)
       EMOE_CUDA(ctx, cudaMemsetAsync(o_part + static_cast<size_t>(P) * L.d_model, 0,
                                      static_cast<size_t>(ksplit - 1) * P * L.d_model * sizeof(float), st));
     if (ctx->fuse_projections) {
-      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 2, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, ctx->dep_extra, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
     } else {
-      EMOE_LAUNCH(ctx, launch_ffn_i8(0, 1, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
-      EMOE_LAUNCH(ctx, launch_ffn_i8(1, 2, L, tmaps, smaps, xs, xsc, plan, hidden, hsc, o_part, ksplit, P, T, EMOE_HYBRID_TILE, ctx->wait_limit, 0, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
+      EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
     }
     EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, P, ctx->check_word, st));
     EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, P, ctx->check_word, st));
@@ -368,7 +370,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       ev[2] = nullptr;
     }
   } else if (use_umma) {
-    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, 1, INT_MAX, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, P, ctx->check_word, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
@@ -379,7 +381,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, xsc, P, 2,
                                               ctx->check_word, st));
     else
-      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, xsc, P, 2, 1, INT_MAX, st));
+      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, xsc, P, 2, 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     if (ctx->fuse_projections) {
       // one launch: an expert's second projection starts when its hidden vectors are complete
@@ -403,7 +405,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, nullptr, P, 1,
                                               ctx->check_word, st));
     else
-      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, nullptr, P, 1, 1, INT_MAX, st));
+      EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, nullptr, P, 1, 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
     if (ctx->fuse_projections) {
@@ -421,7 +423,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     }
   } else if (use_mma) {
     ksplit = ffn_mma_ksplit(L, T);
-    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, nullptr, P, 0, 1, INT_MAX, st));
+    EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, nullptr, xs, nullptr, P, 0, 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
     EMOE_LAUNCH(ctx, launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
@@ -517,6 +519,8 @@ int emoe_device_status(emoe_ctx* ctx, void* stream) {
   EMOE_CUDA(ctx, cudaMemsetAsync(ctx->check_word, 0, sizeof(int), st));
   EMOE_CUDA(ctx, cudaStreamSynchronize(st));
   if (*ctx->check_host & CHECK_WAIT_TIMEOUT) return EMOE_ERR_TIMEOUT;
+  if (*ctx->check_host & CHECK_BAD_EXPERT_ID) return EMOE_ERR_DEVICE_CHECK;
+  if (*ctx->check_host & CHECK_F16_RANGE) return EMOE_ERR_RANGE;
   return *ctx->check_host ? EMOE_ERR_DEVICE_CHECK : EMOE_OK;
 }
 
@@ -531,6 +535,7 @@ const char* emoe_status_string(int status) {
     case EMOE_ERR_DEVICE_CHECK: return "a kernel found inconsistent data";
     case EMOE_ERR_CACHE_FULL: return "every slot of the expert cache is in use";
     case EMOE_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case EMOE_ERR_RANGE: return "a value left the fp16 range of the selected kernel's operands";
     default: return "unknown status";
   }
 }

@@ -21,6 +21,7 @@ struct ExpertDev {
 enum : int {
   CHECK_BAD_EXPERT_ID = 1,
   CHECK_WAIT_TIMEOUT = 2,  // a bounded wait inside a kernel ran out
+  CHECK_F16_RANGE = 4,     // a kernel that carries activations as fp16 met a value outside the fp16 range
 };
 
 // Work plan of the persistent expert kernels, built on the device after the permutation:
@@ -111,7 +112,7 @@ bool ffn_many_tokens(const LayerDims& L, int T);
 // written (1 .. INT_MAX: all activated experts); lets two kernel families share one forward call.
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, float* xsc, int n_pairs,
-                             int fmt, int cnt_lo, int cnt_hi, cudaStream_t st);
+                             int fmt, int cnt_lo, int cnt_hi, int* check_word, cudaStream_t st);
 // Permutation + scatter + plan in one launch (one CTA per pair) for batches of at most 1024 pairs.
 bool permute_scatter_supported(const LayerDims& L, int n_pairs);
 cudaError_t launch_permute_scatter(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
@@ -158,7 +159,7 @@ int encode_tmap_2d(void* out_map, int dtype, const void* base, uint64_t inner, u
 bool ffn_umma_supported(const LayerDims& L);
 cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
-                               int cnt_lo, int cnt_hi, cudaStream_t st);
+                               int cnt_lo, int cnt_hi, int* check_word, cudaStream_t st);
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
                             void* hidden16, float* o, int n_pairs, int* check_word, cudaStream_t st);
 

@@ -26,21 +26,33 @@
 // are complete.
 // Warp roles and rings (every ring has full/empty mbarriers, every wait is bounded: a wait that
 // runs out sets CHECK_WAIT_TIMEOUT and the CTA winds down):
-//   producer warp     TMA: weight boxes and the tokens' limb rows into the STAGE ring (shared
-//                     memory, 128 bytes of every row of 1 or 2 matrices per stage); a record of
-//                     what the stage holds plus the tokens' block scales into the deeper SIDE ring;
+//   producer warp     walks the items; per stage: a record of what the stage holds into the deeper
+//                     SIDE ring, then the weight boxes by TMA into the STAGE ring (shared memory,
+//                     128 bytes of every row of 1 or 2 matrices per stage);
+//   feeder warp       follows the records: the tokens' limb rows (TMA, into the stage) and their
+//                     block scales (into the side ring); it is the one that waits for an expert's
+//                     hidden vectors, so the weights never wait for them.  (Every step of these
+//                     chains is a shared-memory or copy-engine operation of a hundred cycles and
+//                     more under load: one warp doing all of it could not fill a stage in time.)
 //   unpack warps      2 x 4 warps, one thread per row: a 4- or 2-bit stage, one 128-input segment
 //                     at a time, into the A ring (8 segments of 32 columns in tensor memory);
-//   MMA warp          one thread: four K=32 MMAs per segment into the accumulator ring (groups of
-//                     up to four segments of one matrix), commits release A segments, stages and
-//                     publish accumulator groups;
-//   scale warp        follows the side ring and copies (cp.async) the weight scales every stage
-//                     needs, a short window per row, into the SCALE ring: under load a global load
-//                     takes a microsecond, so the scales travel as far ahead as the weights do;
-//   epilogue warps    4 warps, one thread per output row (= tensor-memory lane): accumulator
-//                     groups -> registers -> scaled fp32 totals.  They work from the side and scale
-//                     rings only, so a stage's shared memory is free again as soon as its MMAs
-//                     have read it, however far the epilogue lags.
+//   MMA warps         one thread each: four K=32 MMAs per segment into the accumulator ring (groups
+//                     of up to four segments of one matrix), commits release A segments, stages
+//                     and publish accumulator groups.  Issuing an MMA costs the thread some fifty
+//                     cycles and a 2-bit stream needs one every sixty, so two threads take the
+//                     accumulator groups in turn (each feeds one group of epilogue warps);
+//                     In the general scale mode (SCALE_STAGE) it also copies, with cp.async, the few
+//                     bytes of weight scales every row needs for the stage into the SCALE ring: under
+//                     load a global load takes a microsecond, so the scales travel as far ahead as
+//                     the weights do;
+//   epilogue warps    2 x 4 warps, one thread per output row (= tensor-memory lane) in each group of
+//                     four: accumulator groups -> registers -> scaled fp32 totals.  The two groups
+//                     of warps take the accumulator groups in turn (their per-group work is a chain
+//                     of dependent steps: waits, a tensor-memory load, a few multiply-adds, so two
+//                     such chains per scheduler run twice as fast as one); at the end of an item the
+//                     second hands its partial totals to the first through shared memory.  They
+//                     work from the side and scale rings only, so a stage's shared memory is free
+//                     again as soon as its MMAs have read it, however far the epilogue lags.
 #include <cuda.h>
 
 #include "act_q.cuh"
@@ -55,11 +67,12 @@ constexpr int I8_ROWS = 128;                         // output rows of an item =
 constexpr int I8_BOX_ROWS = 64;                      // rows of one weight box (the tensor maps' box)
 constexpr int I8_BOX_BYTES = I8_BOX_ROWS * 128;      // 8 KB
 constexpr int I8_MAT_BYTES = 2 * I8_BOX_BYTES;       // 128 rows x 128 bytes of one matrix
-constexpr int I8_WARP_UNPACK0 = 4;                   // warps 0-3 epilogue, 4-7 and 8-11 unpack
-constexpr int I8_WARP_PRODUCER = 12;
-constexpr int I8_WARP_MMA = 13;
-constexpr int I8_WARP_SCALES = 14;
-constexpr int I8_THREADS = 15 * 32;
+constexpr int I8_WARP_UNPACK0 = 8;                   // warps 0-3 and 4-7 epilogue, 8-11 and 12-15 unpack
+constexpr int I8_WARP_PRODUCER = 16;
+constexpr int I8_WARP_MMA = 17;
+constexpr int I8_WARP_MMA1 = 18;                     // the second MMA-issuing warp
+constexpr int I8_WARP_FEEDER = 19;                   // the activation feeder
+constexpr int I8_THREADS = 20 * 32;
 constexpr int I8_MAX_STAGES = 8;
 constexpr int I8_SIDE = 16;                          // entries of the side ring
 // Weight scales travel ahead of their use in one of three ways, chosen per projection on the host:
@@ -137,11 +150,15 @@ struct StageMeta {
   int p0, ntok, k0, bits;
   int flags, phase, ai, nseg;
   const void* scales[2];  // scale channels of the stage's matrices
-  int chunk, win0, pitch, pad;  // scale-ring entry of the stage, first byte of a row it holds, bytes per row in it
+  int chunk, win0, pitch;  // scale-ring entry of the stage, first byte of a row it holds, bytes per row in it
+  uint32_t sc_rel;         // byte distance of the scale of segment 0..3 from that of segment 0, 8 bits each
+  uint32_t sc_addr;        // shared-memory address of row 0's scale of segment 0 (block and window modes)
+  int pad[3];
 };
 constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8, META_DONE = 16;
 constexpr int META_NEW_CHUNK = 32;  // the stage is the first to use its scale-ring entry
 constexpr int META_END_CHUNK = 64;  // ... the last
+constexpr int META_DEP = 128;       // the stage's activations are hidden vectors that may still be in the making
 
 // an entry of the side ring: the record of a stage and the block scales of its tokens' limbs
 struct SideEntry {
@@ -155,13 +172,16 @@ __device__ __forceinline__ int group_of(int k, int gshift, int G, int ngroups) {
 
 __device__ __forceinline__ bool wait_lim(uint32_t bar, uint32_t parity, unsigned limit, int* check_word,
                                          volatile int* abort_flag) {
-  // every poll may park the thread for up to a microsecond (it resumes at once when the phase
-  // completes): the many warps of a CTA that wait at any time must not crowd the shared-memory pipe
-  // of the few that work
+  // Most of a CTA's warps wait at any time.  A warp that polls in a tight loop takes issue slots
+  // and shared-memory cycles from the few that work (measured: a third of all issue slots), so a
+  // wait that is not over at once backs off: sleeps of 32, 64, ... up to 1024 ns between polls.
   if (mbar_try_wait(bar, parity)) return true;
+  unsigned ns = 32;
   for (unsigned i = 0; i < limit; ++i) {
-    if (mbar_try_wait_parked(bar, parity, 1000u)) return true;
-    if (*abort_flag) return false;
+    __nanosleep(ns);
+    if (ns < 1024) ns += ns;
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 3u) == 3u && *abort_flag) return false;
   }
   *abort_flag = 1;
   atomicOr(check_word, CHECK_WAIT_TIMEOUT);
@@ -245,7 +265,7 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
   static_assert(NGRP >= 2 && NGRP <= I8_MAX_GROUPS, "accumulator ring");
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * I8_MAX_STAGES + 2 * I8_SIDE + 2 * I8_A_SLOTS + 2 * I8_MAX_GROUPS + 1 + 2 * I8_SCALE_RING +
-                                        2 * I8_CHUNKS];
+                                        2 * I8_CHUNKS + 2 + I8_SIDE];
   __shared__ __align__(16) SideEntry side[I8_SIDE];
   __shared__ __align__(16) uint32_t s_max[2][32][4];  // [item parity][token][epilogue warp]: largest |h| of the warp's rows
   __shared__ uint32_t tmem_base_slot;
@@ -262,20 +282,25 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
   const uint32_t bar_xchg = bar_dempty + 8 * I8_MAX_GROUPS;
   const uint32_t bar_wfull = bar_xchg + 8, bar_wempty = bar_wfull + 8 * I8_SCALE_RING;
   const uint32_t bar_cfull = bar_wempty + 8 * I8_SCALE_RING, bar_cempty = bar_cfull + 8 * I8_CHUNKS;
+  const uint32_t bar_xfull = bar_cempty + 8 * I8_CHUNKS, bar_xempty = bar_xfull + 8;
+  const uint32_t bar_mready = bar_xempty + 8;
   // the scale ring sits behind the stages in dynamic shared memory (entries of either kind)
   unsigned char* scale_ring = smem + STAGES * STAGE_BYTES;
   constexpr int SCALE_ENTRY = NMAT_MAX * I8_SCALE_TILE;
   constexpr int CHUNK_ENTRY = NMAT_MAX * I8_CHUNK_BYTES;
+  // behind it: the partial totals the second group of epilogue warps hands to the first, [matrix][token][row]
+  float* xbuf = reinterpret_cast<float*>(scale_ring + I8_SCALE_RING * SCALE_ENTRY);
 
   if (threadIdx.x == 0) {
     abort_word = 0;
     for (int s = 0; s < I8_MAX_STAGES; ++s) {
       mbar_init(bar_full + 8 * s, 1);   // the producer's lane 0 (+ the bytes of its TMA copies)
-      mbar_init(bar_empty + 8 * s, 9);  // commit of the MMAs that read the stage + the eight unpack warps
+      mbar_init(bar_empty + 8 * s, 10);  // the two MMA warps (a commit each, or a plain arrival) + the eight unpack warps
     }
     for (int s = 0; s < I8_SIDE; ++s) {
-      mbar_init(bar_sfull + 8 * s, 33);  // the producer's lane 0 (record written) and every lane's small copies
-      mbar_init(bar_sempty + 8 * s, 4);  // the four epilogue warps
+      mbar_init(bar_sfull + 8 * s, 32);   // every lane of the feeder warp, after its small copies
+      mbar_init(bar_mready + 8 * s, 1);   // the producer: the record is written
+      mbar_init(bar_sempty + 8 * s, 8);  // the eight epilogue warps
     }
     for (int s = 0; s < I8_A_SLOTS; ++s) {
       mbar_init(bar_afull + 8 * s, 4);   // the four warps of the unpack group that owns the slot
@@ -283,17 +308,19 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
     }
     for (int d = 0; d < I8_MAX_GROUPS; ++d) {
       mbar_init(bar_dfull + 8 * d, 1);   // commit of the group's MMAs
-      mbar_init(bar_dempty + 8 * d, 4);  // the four epilogue warps have read it
+      mbar_init(bar_dempty + 8 * d, 4);  // the four epilogue warps that own the group have read it
     }
     mbar_init(bar_xchg, 4);
     for (int w = 0; w < I8_SCALE_RING; ++w) {
       mbar_init(bar_wfull + 8 * w, 32);   // every lane of the scale warp, after its copies
-      mbar_init(bar_wempty + 8 * w, 4);   // the four epilogue warps
+      mbar_init(bar_wempty + 8 * w, 8);   // the eight epilogue warps
     }
     for (int c = 0; c < I8_CHUNKS; ++c) {
       mbar_init(bar_cfull + 8 * c, 1);    // the producer's lane 0 (+ the bytes of its copies)
-      mbar_init(bar_cempty + 8 * c, 4);   // the four epilogue warps
+      mbar_init(bar_cempty + 8 * c, 8);   // the eight epilogue warps
     }
+    mbar_init(bar_xfull, 4);   // the second group of epilogue warps has written its partial totals
+    mbar_init(bar_xempty, 4);  // the first has read them
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == I8_WARP_MMA) tmem_alloc(smem_u32(&tmem_base_slot), I8_TMEM_COLS);
@@ -335,9 +362,6 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       const int z = li % pd.ksplit;
       const int rb = (li / pd.ksplit) % pd.row_blocks;
       const CUtensorMap* maps = a.wmaps + static_cast<size_t>(rec.e) * 3;
-      const CUtensorMap* bmap = phase == 0 ? &tmap_x : &tmap_h;
-      const float* act_scale = phase == 0 ? a.xsc : a.hsc;
-      const int nblk = K / 128;  // activation blocks per row
       const int bits = rec.bits;
       const int kspan = 1024 / bits;
       const int steps_total = (K + kspan - 1) / kspan;
@@ -346,6 +370,9 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       const int nsteps = max(0, min(steps_total, step_begin + spz) - step_begin);
       const int npass = (rec.cnt + NT - 1) / NT;
       const int row0 = rb * I8_ROWS;
+      // scale channels of the item's matrices (picked with constant indices: the record stays in registers)
+      const void* const sc_m0 = phase == 0 ? rec.scales[0] : (DUAL ? rec.scales[2] : rec.scales[1]);
+      const void* const sc_m1 = (DUAL && phase == 0) ? rec.scales[1] : sc_m0;
       bool need_dep = fused && phase == 1;
       const int smode = a.scale_mode[phase];
       const int ngroups_k = a.ngroups[phase];
@@ -364,7 +391,7 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
           }
           PROF_END(0);
           unsigned char* st = smem + ring.i * STAGE_BYTES;
-          const uint32_t full = bar_full + 8 * ring.i, sfull = bar_sfull + 8 * sring.i;
+          const uint32_t full = bar_full + 8 * ring.i;
           SideEntry* se = &side[sring.i];
           const int k0 = (step_begin + s) * kspan;
           const int klen = nsteps > 0 ? min(kspan, K - k0) : 0;
@@ -386,7 +413,7 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
                   mbar_expect_tx(cfull, pd.nmat * I8_ROWS * row_bytes);
                   for (int m = 0; m < pd.nmat; ++m)
                     bulk_load(smem_u32(cdst + m * I8_CHUNK_BYTES),
-                              static_cast<const char*>(rec.scales[pd.mat_first + m]) + static_cast<size_t>(row0) * row_bytes,
+                              static_cast<const char*>(m == 0 ? sc_m0 : sc_m1) + static_cast<size_t>(row0) * row_bytes,
                               I8_ROWS * row_bytes, cfull);
                 } else {
                   mbar_expect_tx(cfull, pd.nmat * I8_CHUNK_BYTES);
@@ -410,75 +437,38 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
           }
           if (lane == 0) {
             const int flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0) |
-                              (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0) | cflags;
+                              (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0) | cflags |
+                              (need_dep && klen > 0 ? META_DEP : 0);
             uint4* mq = reinterpret_cast<uint4*>(&se->m);
             mq[0] = make_uint4(rec.e, rb, z, rec.begin);
             mq[1] = make_uint4(p0, ntok, k0, bits);
             mq[2] = make_uint4(flags, phase, ai, nseg);
-            se->m.scales[0] = rec.scales[pd.mat_first];
-            se->m.scales[1] = rec.scales[pd.mat_first + pd.nmat - 1];
+            se->m.scales[0] = sc_m0;
+            se->m.scales[1] = sc_m1;
             se->m.chunk = cur_chunk;
             se->m.win0 = stage_win0;
             se->m.pitch = smode == SCALE_BLOCK ? row_bytes : I8_CHUNK_ROW;
-            mbar_arrive(sfull);  // the record is written (the other 32 arrivals follow the small copies)
-            if (klen > 0) {
-              mbar_expect_tx(full, pd.nmat * I8_MAT_BYTES + nseg * B_SEG_BYTES);
-              const int c0 = k0 * bits / 8;
-              for (int m = 0; m < pd.nmat; ++m) {
-                const CUtensorMap* mp = maps + pd.mat_first + m;
-                tma_load_2d(smem_u32(st + m * I8_MAT_BYTES), mp, c0, row0, full);
-                tma_load_2d(smem_u32(st + m * I8_MAT_BYTES + I8_BOX_BYTES), mp, c0, row0 + I8_BOX_ROWS, full);
-              }
-            } else {
-              mbar_arrive(full);
+            {
+              const int g0 = group_of(k0, a.gshift, L.group, ngroups_k);
+              uint32_t rel = 0;
+              for (int sg = 0; sg < 4; ++sg)
+                rel |= static_cast<uint32_t>((group_of(k0 + min(sg, max(nseg, 1) - 1) * 128, a.gshift, L.group, ngroups_k) - g0) * ssz)
+                       << (8 * sg);
+              se->m.sc_rel = rel;
+              se->m.sc_addr = smem_u32(scale_ring) + cur_chunk * CHUNK_ENTRY + g0 * ssz - stage_win0;
             }
+            // all bytes the stage will receive (the feeder's limb rows included), then the record is published
+            if (klen > 0) mbar_expect_tx(full, pd.nmat * I8_MAT_BYTES + nseg * B_SEG_BYTES);
+            else mbar_arrive(full);
+            mbar_arrive(bar_mready + 8 * sring.i);
           }
+          if (klen > 0) need_dep = false;
           __syncwarp();
-          if (klen > 0) {
-            if (need_dep) {
-              // the codes of the stage are on their way; the hidden vectors may still be in the
-              // making on other SMs.  Every lane acquires the counter itself, so that its own copies
-              // below are ordered behind the writers' stores.
-              need_dep = false;
-              PROF_BEGIN;
-              const int expect = a.row_blocks[0] * 4 + a.dep_extra;
-              const int* done = &recs[ai].done;
-              bool ready = false;
-              for (unsigned i = 0; i < a.dep_wait_limit; ++i) {
-                int v;
-                asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(done) : "memory");
-                ready = __all_sync(0xffffffffu, v >= expect);
-                if (ready || __any_sync(0xffffffffu, *abort_flag != 0)) break;
-                __nanosleep(100);
-              }
-              if (!ready) {
-                if (lane == 0) {
-                  *abort_flag = 1;
-                  atomicOr(a.check_word, CHECK_WAIT_TIMEOUT);
-                }
-                ok = false;
-                // the stage's barriers stay incomplete: nobody consumes it, the copies already issued
-                // land in the CTA's own shared memory during the wind-down pause
-                break;
-              }
-              asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores -> TMA reads
-              PROF_END(1);
-            }
-            // block scales of the tile's tokens
-            if (lane < ntok) {
-              const float* src = act_scale + static_cast<size_t>(rec.begin + p0 + lane) * nblk + k0 / 128;
-              const uint32_t xdst = smem_u32(&se->sx[0][lane]);
-              for (int sg = 0; sg < nseg; ++sg)
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(xdst + sg * 128), "l"(src + sg) : "memory");
-            }
-            asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(sfull) : "memory");
-            if (lane == 0) {
-              // the tokens' limb rows: rows 2*slot (hi) and 2*slot+1 (lo) of the activation image
-              for (int sg = 0; sg < nseg; ++sg)
-                tma_load_2d(smem_u32(st + B_OFF + sg * B_SEG_BYTES), bmap, k0 + sg * 128, 2 * (rec.begin + p0), full);
-            }
-          } else {
-            mbar_arrive(sfull);  // with lane 0's arrival above: 33 in all
+          // the weight boxes: lane l fetches box l (matrix l / 2, upper or lower 64 rows), one instruction for all
+          if (klen > 0 && lane < 2 * pd.nmat) {
+            const int mtx = lane >> 1, half = lane & 1;
+            tma_load_2d(smem_u32(st + mtx * I8_MAT_BYTES + half * I8_BOX_BYTES), maps + pd.mat_first + mtx, k0 * bits / 8,
+                        row0 + half * I8_BOX_ROWS, full);
           }
           ring.next(STAGES);
           sring.next(I8_SIDE);
@@ -499,63 +489,118 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
           wait_warp(bar_sempty + 8 * sring.i, sring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
         if (lane == 0) {
           side[sring.i].m.flags = META_STOP;
-          mbar_arrive(bar_sfull + 8 * sring.i);
+          mbar_arrive(bar_full + 8 * ring.i);
+          mbar_arrive(bar_mready + 8 * sring.i);
         }
-        __syncwarp();
-        mbar_arrive(bar_sfull + 8 * sring.i);
-        if (lane == 0) mbar_arrive(bar_full + 8 * ring.i);
       }
     }
-  } else if (warp == I8_WARP_SCALES) {
-    // ---------------- scale warp: weight scales of every stage into the scale ring ----------------
-    // (SCALE_STAGE projections only; in the other modes the producer's bulk copies bring the scales.)
-    // Lane l copies the windows of rows 4l .. 4l+3 of every matrix of the stage.  The scales a
-    // stage needs from a row (groups of inputs k0 .. k0 + 128 * segments) are a few neighbouring
-    // bytes of the row's scale channel; they are copied in 4-byte words from the 4-byte boundary at or
-    // below the first one, into a 16-byte window per row.
-    const int ssz = L.scale_f16 ? 2 : 4;
-    Ring sring{0, 0}, wring{0, 0};
+  } else if (warp == I8_WARP_FEEDER) {
+    // ---------------- feeder warp: the tokens' limb rows and block scales of every stage ----------------
+    Ring ring{0, 0}, sring{0, 0}, wring{0, 0};
     while (true) {
-      if (!wait_warp(bar_sfull + 8 * sring.i, sring.ph, a.wait_limit, a.check_word, abort_flag)) break;
-      const StageMeta m = side[sring.i].m;
-      if (m.flags & META_STOP) break;
-      if (!(m.flags & META_EMPTY) && a.scale_mode[m.phase] == SCALE_STAGE) {
-        if (!wait_warp(bar_wempty + 8 * wring.i, wring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) break;
-        const int N = m.phase == 0 ? L.d_ff : L.d_model;
-        const int ngroups = a.ngroups[m.phase];
-        const int nmat = (DUAL && m.phase == 0) ? 2 : 1;
-        const int g0 = group_of(m.k0, a.gshift, L.group, ngroups),
-                  g1 = group_of(m.k0 + (m.nseg - 1) * 128, a.gshift, L.group, ngroups);
-        const uint32_t sdst = smem_u32(scale_ring + wring.i * SCALE_ENTRY);
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int row = 4 * lane + r;
-          const int off = min(m.rb * I8_ROWS + row, N - 1) * ngroups * ssz;
-          const int b0 = (off + g0 * ssz) & ~3;
-          const int b1 = off + (g1 + 1) * ssz;
-          for (int mt = 0; mt < nmat; ++mt) {
-            const char* sbase = static_cast<const char*>(m.scales[mt]);
-#pragma unroll 1
-            for (int w = 0; b0 + 4 * w < b1; ++w)
-              asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + (mt * I8_ROWS + row) * 16 + 4 * w),
-                           "l"(sbase + b0 + 4 * w)
-                           : "memory");
-          }
-        }
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_wfull + 8 * wring.i) : "memory");
-        wring.next(I8_SCALE_RING);
+      if (!wait_warp(bar_mready + 8 * sring.i, sring.ph, a.wait_limit, a.check_word, abort_flag)) break;
+      SideEntry* se = &side[sring.i];
+      const uint4 m0 = *reinterpret_cast<const uint4*>(&se->m.e);       // e, rb, z, begin
+      const uint4 m1 = *reinterpret_cast<const uint4*>(&se->m.p0);      // p0, ntok, k0, bits
+      const uint4 m2 = *reinterpret_cast<const uint4*>(&se->m.flags);   // flags, phase, ai, nseg
+      const int flags = static_cast<int>(m2.x), phase = static_cast<int>(m2.y), ai = static_cast<int>(m2.z),
+                nseg = static_cast<int>(m2.w);
+      const uint32_t sfull = bar_sfull + 8 * sring.i;
+      if (flags & META_STOP) {
+        mbar_arrive(sfull);
+        break;
       }
+      if (!(flags & META_EMPTY)) {
+        const int begin = static_cast<int>(m0.w), p0 = static_cast<int>(m1.x), ntok = static_cast<int>(m1.y),
+                  k0 = static_cast<int>(m1.z);
+        if (flags & META_DEP) {
+          // The hidden vectors may still be in the making on other SMs.  Every lane acquires the
+          // counter itself, so that its own copies below are ordered behind the writers' stores.
+          const int expect = a.row_blocks[0] * 4 + a.dep_extra;
+          const int* done = &recs[ai].done;
+          bool ready = false;
+          for (unsigned i = 0; i < a.dep_wait_limit; ++i) {
+            int v;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(done) : "memory");
+            ready = __all_sync(0xffffffffu, v >= expect);
+            if (ready || __any_sync(0xffffffffu, *abort_flag != 0)) break;
+            __nanosleep(100);
+          }
+          if (!ready) {
+            // the stage's barriers stay incomplete: nobody consumes it; the weight copies already
+            // issued land in the CTA's own shared memory during the wind-down pause
+            if (lane == 0) {
+              *abort_flag = 1;
+              atomicOr(a.check_word, CHECK_WAIT_TIMEOUT);
+            }
+            break;
+          }
+          asm volatile("fence.proxy.async;" ::: "memory");  // generic-proxy stores -> TMA reads
+        }
+        const int K = phase == 0 ? L.d_model : L.d_ff;
+        if (a.scale_mode[phase] == SCALE_STAGE) {
+          // General scale mode: lane l copies the windows of rows 4l .. 4l+3 of every matrix of the stage.
+          // The scales a stage needs from a row (groups of inputs k0 .. k0 + 128 * segments) are a few
+          // neighbouring bytes of the row's scale channel; they are copied in 4-byte words from the
+          // 4-byte boundary at or below the first one, into a 16-byte window per row.
+          if (!wait_warp(bar_wempty + 8 * wring.i, wring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) break;
+          const int ssz = L.scale_f16 ? 2 : 4;
+          const int N = phase == 0 ? L.d_ff : L.d_model;
+          const int ngroups = a.ngroups[phase];
+          const int nmat = (DUAL && phase == 0) ? 2 : 1;
+          const int rb = static_cast<int>(m0.y);
+          const int g0 = group_of(k0, a.gshift, L.group, ngroups), g1 = group_of(k0 + (nseg - 1) * 128, a.gshift, L.group, ngroups);
+          const uint32_t sdst = smem_u32(scale_ring + wring.i * SCALE_ENTRY);
+          const char* const sb0 = static_cast<const char*>(se->m.scales[0]);
+          const char* const sb1 = static_cast<const char*>(se->m.scales[1]);
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            const int row = 4 * lane + r;
+            const int off = min(rb * I8_ROWS + row, N - 1) * ngroups * ssz;
+            const int b0 = (off + g0 * ssz) & ~3;
+            const int b1 = off + (g1 + 1) * ssz;
+            for (int mt = 0; mt < nmat; ++mt) {
+              const char* sbase = mt == 0 ? sb0 : sb1;
+#pragma unroll 1
+              for (int w = 0; b0 + 4 * w < b1; ++w)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + (mt * I8_ROWS + row) * 16 + 4 * w),
+                             "l"(sbase + b0 + 4 * w)
+                             : "memory");
+            }
+          }
+          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_wfull + 8 * wring.i) : "memory");
+          wring.next(I8_SCALE_RING);
+        }
+        // block scales of the tile's tokens
+        if (lane < ntok) {
+          const float* src = (phase == 0 ? a.xsc : a.hsc) + static_cast<size_t>(begin + p0 + lane) * (K / 128) + k0 / 128;
+          const uint32_t xdst = smem_u32(&se->sx[0][lane]);
+          for (int sg = 0; sg < nseg; ++sg)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(xdst + sg * 128), "l"(src + sg) : "memory");
+        }
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(sfull) : "memory");
+        // the tokens' limb rows: rows 2*slot (hi) and 2*slot+1 (lo) of the activation image; lane l fetches segment l
+        if (lane < nseg)
+          tma_load_2d(smem_u32(smem + ring.i * STAGE_BYTES + B_OFF + lane * B_SEG_BYTES), phase == 0 ? &tmap_x : &tmap_h,
+                      k0 + lane * 128, 2 * (begin + p0), bar_full + 8 * ring.i);
+      } else {
+        mbar_arrive(sfull);
+      }
+      ring.next(STAGES);
       sring.next(I8_SIDE);
     }
     asm volatile("cp.async.wait_all;" ::: "memory");  // nothing of this warp is in flight when the CTA ends
-  } else if (warp == I8_WARP_MMA) {
-    // ---------------- MMA issuer (one lane) ----------------
+  } else if (warp == I8_WARP_MMA || warp == I8_WARP_MMA1) {
+    // ---------------- MMA issuers (one lane of each of the two warps) ----------------
     if (lane == 0) {
+      const uint32_t mi = warp == I8_WARP_MMA ? 0u : 1u;  // even or odd accumulator groups
       // kind::i8: s8 x s8 -> s32, both operands K-major, M = 128, N = 2 * NT
       const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((static_cast<uint32_t>(NCOL) >> 3) << 17) |
                              ((static_cast<uint32_t>(I8_ROWS) >> 4) << 24);
-      Ring ring{0, 0}, sring{0, 0}, gring{0, 0};
+      Ring ring{0, 0}, sring{0, 0};
       uint32_t qs = 0;  // segments that went through the A ring so far
+      uint32_t gq = 0;  // accumulator groups so far: group gq lives in slot gq % NGRP, even ones belong to the
+                        // first group of epilogue warps, odd ones to the second
       bool ok = true;
       PROF_DECL;
       while (ok) {
@@ -573,11 +618,19 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
         }
         const uint32_t st = smem_u32(smem + ring.i * STAGE_BYTES);
         const int nmat = (DUAL && m.phase == 0) ? 2 : 1;
+        bool issued = false;
         for (int mt = 0; mt < nmat && ok; ++mt) {
           const uint64_t adesc = umma_desc(st + mt * I8_MAT_BYTES);
           for (int sg0 = 0; sg0 < m.nseg && ok; sg0 += GSEGS) {
+            if ((gq & 1u) != mi) {  // the other warp's group: only keep the counters in step
+              if (m.bits != 8) qs += min(m.nseg, sg0 + GSEGS) - sg0;
+              ++gq;
+              continue;
+            }
+            issued = true;
+            const uint32_t gslot = gq % NGRP;
             PROF_BEGIN;
-            if (!wait_lim(bar_dempty + 8 * gring.i, gring.ph ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
+            if (!wait_lim(bar_dempty + 8 * gslot, ((gq / NGRP) & 1u) ^ 1u, a.wait_limit, a.check_word, abort_flag)) {
               ok = false;
               break;
             }
@@ -585,12 +638,14 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
             tc_fence_after();
             const int sg1 = min(m.nseg, sg0 + GSEGS);
             for (int sg = sg0; sg < sg1; ++sg) {
-              const uint32_t d_tmem = tmem_base + I8_D_COL0 + gring.i * GCOLS + (sg - sg0) * NCOL;
+              const uint32_t d_tmem = tmem_base + I8_D_COL0 + gslot * GCOLS + (sg - sg0) * NCOL;
               const uint64_t bdesc = umma_desc(st + B_OFF + sg * B_SEG_BYTES);
               if (m.bits == 8) {
+                PROF_BEGIN;
 #pragma unroll
                 for (int j = 0; j < 4; ++j)  // 32 inputs per MMA
                   umma_i8_ss(d_tmem, adesc + 2 * j, bdesc + 2 * j, idesc, j > 0 ? 1u : 0u);
+                PROF_END(3);
               } else {
                 const uint32_t slot = qs & (I8_A_SLOTS - 1);
                 PROF_BEGIN;
@@ -601,24 +656,38 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
                 PROF_END(1);
                 tc_fence_after();
                 const uint32_t a_tmem = tmem_base + slot * I8_A_SLOT_COLS;
+                PROF_BEGIN;
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
                   umma_i8_ts(d_tmem, a_tmem + 8 * j, bdesc + 2 * j, idesc, j > 0 ? 1u : 0u);
+                PROF_END(3);
+                PROF_BEGIN;
                 umma_commit(bar_aempty + 8 * slot);
+                PROF_END(4);
                 ++qs;
               }
             }
             if (!ok) break;
-            umma_commit(bar_dfull + 8 * gring.i);
-            gring.next(NGRP);
+            PROF_BEGIN;
+            umma_commit(bar_dfull + 8 * gslot);
+            PROF_END(4);
+            ++gq;
           }
         }
         if (!ok) break;
-        umma_commit(bar_empty + 8 * ring.i);  // the stage's shared memory may be refilled once these MMAs have read it
+        // the stage's shared memory may be refilled once the MMAs of both warps have read it
+        if (issued) umma_commit(bar_empty + 8 * ring.i);
+        else mbar_arrive(bar_empty + 8 * ring.i);
         ring.next(STAGES);
         sring.next(I8_SIDE);
       }
-      PROF_STORE(3, 3);
+#ifdef EMOE_I8_PROFILE
+      if (a.prof && mi == 0) {
+        for (int pi = 0; pi < 3; ++pi) a.prof[blockIdx.x * 32 + 3 + pi] = prof_acc[pi];
+        a.prof[blockIdx.x * 32 + 28] = prof_acc[3];
+        a.prof[blockIdx.x * 32 + 29] = prof_acc[4];
+      }
+#endif
     }
   } else if (warp >= I8_WARP_UNPACK0) {
     // ---------------- unpack warps: packed codes -> int8 rows in tensor memory ----------------
@@ -689,11 +758,15 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
     }
     if (warp == I8_WARP_UNPACK0) { PROF_STORE(6, 3); }
   } else {
-    // ---------------- epilogue warps: one thread per output row ----------------
-    const int r = 32 * warp + lane;
-    const uint32_t d_tmem0 = tmem_base + (static_cast<uint32_t>(32 * warp) << 16) + I8_D_COL0;
-    float tot[NMAT_MAX][NT];
-    Ring sring{0, 0}, gring{0, 0}, wring{0, 0}, cring{0, 0};
+    // ---------------- epilogue warps: one thread per output row in each group of four warps ----------------
+    const uint32_t ew = static_cast<uint32_t>(warp) >> 2;  // which of the two groups
+    const int wq = warp & 3;                               // the warp's quarter of the tensor-memory lanes
+    const int r = 32 * wq + lane;
+    const uint32_t d_tmem0 = tmem_base + (static_cast<uint32_t>(32 * wq) << 16) + I8_D_COL0;
+    float tot[NMAT_MAX][NT];  // this group's share of the row's totals
+    Ring sring{0, 0}, wring{0, 0}, cring{0, 0};
+    uint32_t gq = 0;         // accumulator groups so far (as the MMA warp counts them)
+    uint32_t items = 0;      // items finished so far
     uint32_t exchanges = 0;  // first-projection items finished so far (each uses the exchange barrier once)
     bool ok = true;
     PROF_DECL;
@@ -702,124 +775,183 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       if (!wait_warp(bar_sfull + 8 * sring.i, sring.ph, a.wait_limit, a.check_word, abort_flag)) break;
       PROF_END(0);
       const SideEntry& se = side[sring.i];
-      const StageMeta m = se.m;
-      if (m.flags & META_STOP) break;
+      // Under load a shared-memory load takes a hundred cycles and more and every instruction of
+      // this chain waits for the one before, so the record is read in one batch, nothing branches
+      // on a loaded value where a batch of loads can be issued instead, and what does not depend
+      // on the row (offsets, addresses) was worked out once by the producer.
+      const uint4 q1 = *reinterpret_cast<const uint4*>(&se.m.p0);     // p0, ntok, k0, bits
+      const uint4 q2 = *reinterpret_cast<const uint4*>(&se.m.flags);  // flags, phase, ai, nseg
+      const uint4 q4 = *reinterpret_cast<const uint4*>(&se.m.chunk);  // chunk, win0, pitch, sc_rel
+      const uint32_t sc_addr0 = se.m.sc_addr;
+      const int flags = static_cast<int>(q2.x), phase = static_cast<int>(q2.y), nseg = static_cast<int>(q2.w);
+      const int ntok = static_cast<int>(q1.y);
+      if (flags & META_STOP) break;
       PROF_BEGIN;
-      if (m.flags & META_FIRST) {
+      if (flags & META_FIRST) {
 #pragma unroll
         for (int mt = 0; mt < NMAT_MAX; ++mt)
 #pragma unroll
           for (int t = 0; t < NT; ++t) tot[mt][t] = 0.0f;
       }
-      const int N = m.phase == 0 ? L.d_ff : L.d_model;
-      const int n = m.rb * I8_ROWS + r;
-      if (!(m.flags & META_EMPTY)) {
-        const int nmat = (DUAL && m.phase == 0) ? 2 : 1;
-        // this row's weight scales of the stage, from the scale ring
-        float sw[NMAT_MAX][4];
-        const int ngroups = a.ngroups[m.phase];
+      if (!(flags & META_EMPTY)) {
+        const int nmat = (DUAL && phase == 0) ? 2 : 1;
         const int ssz = L.scale_f16 ? 2 : 4;
-        const float unit = m.bits == 8 ? 1.0f : (m.bits == 4 ? 0.0625f : 0.015625f);  // codes arrive as 16 q / 64 q
-        const bool per_stage = a.scale_mode[m.phase] == SCALE_STAGE;
-        const unsigned char* sc_row;  // where the scale of the row's group 0 would sit
+        const bool per_stage = a.scale_mode[phase] == SCALE_STAGE;
+        uint32_t sc_row;  // shared-memory address of this row's scale of segment 0, first matrix
         int mat_stride;
         if (per_stage) {
           if (!wait_warp(bar_wfull + 8 * wring.i, wring.ph, a.wait_limit, a.check_word, abort_flag)) break;
           // the row's window starts at the 4-byte boundary at or below its first scale of the stage
-          const int g0 = group_of(m.k0, a.gshift, L.group, ngroups);
-          sc_row = scale_ring + wring.i * SCALE_ENTRY + r * 16 + (((min(n, N - 1) * ngroups + g0) * ssz) & 3) - g0 * ssz;
+          const int N = phase == 0 ? L.d_ff : L.d_model;
+          const int ngroups = a.ngroups[phase];
+          const int g0 = group_of(static_cast<int>(q1.z), a.gshift, L.group, ngroups);
+          const int n = se.m.rb * I8_ROWS + r;
+          sc_row = smem_u32(scale_ring) + wring.i * SCALE_ENTRY + r * 16 + (((min(n, N - 1) * ngroups + g0) * ssz) & 3);
           mat_stride = I8_SCALE_TILE;
         } else {
           PROF_LAP(6);
-          if (m.flags & META_NEW_CHUNK) {
+          if (flags & META_NEW_CHUNK) {
             if (!wait_warp(bar_cfull + 8 * cring.i, cring.ph, a.wait_limit, a.check_word, abort_flag)) break;
             cring.next(I8_CHUNKS);
           }
           PROF_LAP(7);
-          sc_row = scale_ring + m.chunk * CHUNK_ENTRY + r * m.pitch - m.win0;
+          sc_row = sc_addr0 + r * static_cast<int>(q4.z);
           mat_stride = I8_CHUNK_BYTES;
         }
+        uint32_t sraw[NMAT_MAX][4];  // the stage's scales of this row as stored (fp16 or fp32 bits)
 #pragma unroll
-        for (int mt = 0; mt < NMAT_MAX; ++mt)
+        for (int sg = 0; sg < 4; ++sg) {
+          const uint32_t off = (q4.w >> (8 * sg)) & 0xffu;
 #pragma unroll
-          for (int sg = 0; sg < 4; ++sg) {
-            sw[mt][sg] = 0.0f;
-            if (mt < nmat && sg < m.nseg) {
-              const unsigned char* sc = sc_row + mt * mat_stride + group_of(m.k0 + sg * 128, a.gshift, L.group, ngroups) * ssz;
-              sw[mt][sg] = unit * (ssz == 2 ? __half2float(*reinterpret_cast<const __half*>(sc))
-                                            : *reinterpret_cast<const float*>(sc));
-            }
+          for (int mt = 0; mt < NMAT_MAX; ++mt) {
+            const uint32_t ad = sc_row + (mt < nmat ? mt : 0) * mat_stride + off;
+            if (ssz == 2) asm volatile("ld.shared.u16 %0, [%1];" : "=r"(sraw[mt][sg]) : "r"(ad));
+            else asm volatile("ld.shared.u32 %0, [%1];" : "=r"(sraw[mt][sg]) : "r"(ad));
           }
+        }
         __syncwarp();
         if (per_stage) {
           if (lane == 0) mbar_arrive(bar_wempty + 8 * wring.i);
           wring.next(I8_SCALE_RING);
-        } else if (m.flags & META_END_CHUNK) {
-          if (lane == 0) mbar_arrive(bar_cempty + 8 * m.chunk);
+        } else if (flags & META_END_CHUNK) {
+          if (lane == 0) mbar_arrive(bar_cempty + 8 * static_cast<int>(q4.x));
         }
         PROF_LAP(3);
+        const uint32_t sx_addr = smem_u32(&se.sx[0][0]);
 #pragma unroll
         for (int mt = 0; mt < NMAT_MAX; ++mt) {
           if (mt >= nmat || !ok) break;
 #pragma unroll
           for (int g = 0; g < 4 / GSEGS; ++g) {
-            if (g * GSEGS >= m.nseg) break;
+            if (g * GSEGS >= nseg) break;
+            const uint32_t gslot = gq % NGRP, gpar = (gq / NGRP) & 1u;
+            const bool mine = (gq & 1u) == ew;
+            ++gq;
+            if (!mine) continue;
             PROF_BEGIN;
-            if (!wait_warp(bar_dfull + 8 * gring.i, gring.ph, a.wait_limit, a.check_word, abort_flag)) {
+            if (!wait_warp(bar_dfull + 8 * gslot, gpar, a.wait_limit, a.check_word, abort_flag)) {
               ok = false;
               break;
             }
             PROF_LAP(1);
             tc_fence_after();
-            const uint32_t d_tmem = d_tmem0 + gring.i * GCOLS;
-            // the group in chunks of 32 columns (2 segments at NT = 8, 1 at 16, half a segment at 32);
-            // the next chunk is requested before the current one is worked on
+            const uint32_t d_tmem = d_tmem0 + gslot * GCOLS;
+            // the group in chunks of 32 columns (2 segments at NT = 8, 1 at 16, half a segment at 32)
             constexpr int NCHUNK = GCOLS / 32;
             constexpr int TOK_PER_CHUNK = NT < 16 ? NT : 16;  // tokens of one segment inside a chunk
-            const int ncols = min(GSEGS, m.nseg - g * GSEGS) * NCOL;
-            uint32_t acc[2][32];
-            tmem_ld32(d_tmem, acc[0]);
+            constexpr int PIECES = 32 / (2 * TOK_PER_CHUNK);  // segments (or half segments) inside a chunk
+            const int ncols = min(GSEGS, nseg - g * GSEGS) * NCOL;
 #pragma unroll
             for (int c = 0; c < NCHUNK; ++c) {
               if (c * 32 >= ncols) break;
+              uint32_t acc[32];
+              tmem_ld32(d_tmem + c * 32, acc);
+              // the tokens' block scales of the chunk's pieces, requested under the tensor-memory load
+              float sxv[PIECES][TOK_PER_CHUNK];
+#pragma unroll
+              for (int u = 0; u < PIECES; ++u) {
+                const int col0 = c * 32 + u * 2 * TOK_PER_CHUNK;
+                const int sg = min(g * GSEGS + col0 / NCOL, 3), t0 = (col0 % NCOL) / 2;
+#pragma unroll
+                for (int t = 0; t < TOK_PER_CHUNK; t += 4)
+                  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                               : "=f"(sxv[u][t]), "=f"(sxv[u][t + 1]), "=f"(sxv[u][t + 2]), "=f"(sxv[u][t + 3])
+                               : "r"(sx_addr + (sg * 32 + t0 + t) * 4));
+              }
               tmem_ld_wait();
               const bool more = (c + 1) * 32 < ncols;
-              if (c + 1 < NCHUNK && more) tmem_ld32(d_tmem + (c + 1) * 32, acc[(c + 1) & 1]);
               if (!more) {  // the last chunk is in registers: the accumulators may be overwritten
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_dempty + 8 * gring.i);
+                if (lane == 0) mbar_arrive(bar_dempty + 8 * gslot);
               }
               PROF_LAP(4);
 #pragma unroll
-              for (int u = 0; u < 32 / (2 * TOK_PER_CHUNK); ++u) {  // segments (or half segments) inside the chunk
-                const int col0 = c * 32 + u * 2 * TOK_PER_CHUNK;    // first column of this piece in the group
-                const int sg = g * GSEGS + col0 / NCOL;              // its segment in the stage
-                const int t0 = (col0 % NCOL) / 2;                    // its first token
-                if (sg < m.nseg) {
-                  const float s = sw[mt][sg < 4 ? sg : 3];
+              for (int u = 0; u < PIECES; ++u) {
+                const int col0 = c * 32 + u * 2 * TOK_PER_CHUNK;  // first column of this piece in the group
+                const int sg = g * GSEGS + col0 / NCOL;            // its segment in the stage
+                const int t0 = (col0 % NCOL) / 2;                  // its first token
+                // (the factor 16 or 64 of the unpacked codes is taken out once, at the end of the item)
+                const uint32_t raw = sraw[mt][sg < 4 ? sg : 3];
+                const float sv = ssz == 2 ? __half2float(__ushort_as_half(static_cast<unsigned short>(raw))) : __uint_as_float(raw);
+                const float s = sv;
+                // tokens in pairs: a pair past the expert's tokens is skipped, inside a pair nothing branches;
+                // a segment past the stage's last is skipped too (its token scales are whatever the entry held)
 #pragma unroll
-                  for (int t = 0; t < TOK_PER_CHUNK; ++t) {
-                    if (t0 + t < m.ntok) {
-                      const int v = static_cast<int>(acc[c & 1][u * 2 * TOK_PER_CHUNK + 2 * t]) * 128 +
-                                    static_cast<int>(acc[c & 1][u * 2 * TOK_PER_CHUNK + 2 * t + 1]);
-                      tot[mt][t0 + t] = fmaf(static_cast<float>(v), s * se.sx[sg < 4 ? sg : 3][t0 + t], tot[mt][t0 + t]);
+                for (int t = 0; t < TOK_PER_CHUNK; t += 2) {
+                  if (sg < nseg && t0 + t < ntok) {
+#pragma unroll
+                    for (int tt = t; tt < t + 2; ++tt) {
+                      const int v = static_cast<int>(acc[u * 2 * TOK_PER_CHUNK + 2 * tt]) * 128 +
+                                    static_cast<int>(acc[u * 2 * TOK_PER_CHUNK + 2 * tt + 1]);
+                      tot[mt][t0 + tt] = fmaf(static_cast<float>(v), s * sxv[u][tt], tot[mt][t0 + tt]);
                     }
                   }
                 }
               }
             }
             PROF_LAP(5);
-            gring.next(NGRP);
           }
         }
         if (!ok) break;
       }
-      // the side entry is no longer needed
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_sempty + 8 * sring.i);
-      if (m.flags & META_LAST) {
+      if (!(flags & META_LAST)) {
+        // the side entry is no longer needed
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_sempty + 8 * sring.i);
+      } else {
+        // end of an item: the whole record is needed once more, then the entry is released
+        const StageMeta m = se.m;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_sempty + 8 * sring.i);
+        const int N = m.phase == 0 ? L.d_ff : L.d_model;
+        const int n = m.rb * I8_ROWS + r;
+        // 4- and 2-bit codes were multiplied as 16 q and 64 q: taken out here, once per item
+        const float unit = m.bits == 8 ? 1.0f : (m.bits == 4 ? 0.0625f : 0.015625f);
         PROF_BEGIN;
+        // the two groups of warps put their shares of the totals together: the second writes, the first adds
+        const uint32_t ipar = items & 1u;
+        ++items;
+        if (ew == 1) {
+          if (!wait_warp(bar_xempty, ipar ^ 1u, a.wait_limit, a.check_word, abort_flag)) break;
+#pragma unroll
+          for (int mt = 0; mt < NMAT_MAX; ++mt)
+#pragma unroll
+            for (int t = 0; t < NT; ++t)
+              if (t < m.ntok) xbuf[(mt * NT + t) * I8_ROWS + r] = tot[mt][t];  // (scaled by the reader)
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_xfull);
+          sring.next(I8_SIDE);
+          continue;
+        }
+        if (!wait_warp(bar_xfull, ipar, a.wait_limit, a.check_word, abort_flag)) break;
+#pragma unroll
+        for (int mt = 0; mt < NMAT_MAX; ++mt)
+#pragma unroll
+          for (int t = 0; t < NT; ++t)
+            if (t < m.ntok) tot[mt][t] = unit * (tot[mt][t] + xbuf[(mt * NT + t) * I8_ROWS + r]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_xempty);
         if (m.phase == 0) {
           // hidden values of this row: activation, rounded to bf16 (the hidden vector is a bf16
           // tensor), then to limbs under the block scale of the item's 128 rows
@@ -837,7 +969,7 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
             }
             h[t] = (t < m.ntok && n < N) ? __bfloat162float(__float2bfloat16_rn(v)) : 0.0f;
             const uint32_t mx = redux_max_u32(__float_as_uint(h[t]) & 0x7fffffffu);
-            if (lane == 0) s_max[par][t][warp] = mx;
+            if (lane == 0) s_max[par][t][wq] = mx;
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_xchg);
@@ -876,6 +1008,7 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
       sring.next(I8_SIDE);
     }
     if (warp == 0) { PROF_STORE(9, 8); }
+    if (warp == 4) { PROF_STORE(20, 8); }
   }
 
   // wind-down: after a wait that ran out, give copies and MMAs in flight time to land before the
@@ -894,7 +1027,8 @@ __global__ void __launch_bounds__(I8_THREADS, 1)
 
 int stages_for(int nt, int nmat) {
   static_assert(I8_CHUNKS * I8_CHUNK_BYTES == I8_SCALE_RING * I8_SCALE_TILE, "both kinds of scale ring take the same room");
-  int s = (I8_SMEM_LIMIT - 1024 /*alignment slack*/ - I8_STATIC_SMEM - I8_SCALE_RING * nmat * I8_SCALE_TILE) / stage_bytes(nt, nmat);
+  int s = (I8_SMEM_LIMIT - 1024 /*alignment slack*/ - I8_STATIC_SMEM - I8_SCALE_RING * nmat * I8_SCALE_TILE - nmat * nt * I8_ROWS * 4) /
+          stage_bytes(nt, nmat);
   return s > I8_MAX_STAGES ? I8_MAX_STAGES : s;
 }
 
@@ -904,7 +1038,8 @@ cudaError_t launch_variant(const I8Args& a_in, const CUtensorMap& tx, const CUte
   I8Args a = a_in;
   a.stages = stages_for(NT, DUAL ? 2 : 1);
   if (a.stages < 3) return cudaErrorInvalidValue;
-  const int smem = a.stages * stage_bytes(NT, DUAL ? 2 : 1) + I8_SCALE_RING * (DUAL ? 2 : 1) * I8_SCALE_TILE + 1024;
+  const int smem = a.stages * stage_bytes(NT, DUAL ? 2 : 1) + I8_SCALE_RING * (DUAL ? 2 : 1) * I8_SCALE_TILE +
+                   (DUAL ? 2 : 1) * NT * I8_ROWS * 4 + 1024;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;

@@ -240,13 +240,16 @@ __device__ __forceinline__ void build_plan(int* plan, const ExpertDev* __restric
 
 // One activation row into the layout of the owning expert's bitwidth (optionally as fp16).
 __device__ __forceinline__ void scatter_row(const __nv_bfloat16* __restrict__ src_row, __nv_bfloat16* __restrict__ dst_row,
-                                            int d, int bits, int to_f16) {
+                                            int d, int bits, int to_f16, int* __restrict__ check_word) {
+  bool beyond = false;
   // one thread moves 16 consecutive inputs: half b of lane t's 32-block of a 128-input segment
   for (int u = threadIdx.x; u < d / 16; u += blockDim.x) {
     const int seg = (u >> 3) * 128, t = (u >> 1) & 3, b = u & 1;
     const uint4* src = reinterpret_cast<const uint4*>(src_row + seg + t * 32 + b * 16);
     uint4 a = src[0], c = src[1];
     if (to_f16) {  // the streaming kernel multiplies in fp16: same layout, 16-bit values converted in place
+      beyond |= bf16x2_beyond_f16(a.x) | bf16x2_beyond_f16(a.y) | bf16x2_beyond_f16(a.z) | bf16x2_beyond_f16(a.w) |
+                bf16x2_beyond_f16(c.x) | bf16x2_beyond_f16(c.y) | bf16x2_beyond_f16(c.z) | bf16x2_beyond_f16(c.w);
       a = make_uint4(bf16x2_to_f16x2_sat(a.x), bf16x2_to_f16x2_sat(a.y), bf16x2_to_f16x2_sat(a.z), bf16x2_to_f16x2_sat(a.w));
       c = make_uint4(bf16x2_to_f16x2_sat(c.x), bf16x2_to_f16x2_sat(c.y), bf16x2_to_f16x2_sat(c.z), bf16x2_to_f16x2_sat(c.w));
     }
@@ -265,6 +268,8 @@ __device__ __forceinline__ void scatter_row(const __nv_bfloat16* __restrict__ sr
     *reinterpret_cast<uint4*>(dst_row + seg + (((2 * b) * 4 + t) << 3)) = oa;
     *reinterpret_cast<uint4*>(dst_row + seg + (((2 * b + 1) * 4 + t) << 3)) = oc;
   }
+  // a value the fp16 operand cannot hold was saturated: the result is no longer the definition's
+  if (beyond && check_word) atomicOr(check_word, CHECK_F16_RANGE);
 }
 
 // One activation row into slot `slot` of the activation buffer, in the format the expert kernel
@@ -272,12 +277,13 @@ __device__ __forceinline__ void scatter_row(const __nv_bfloat16* __restrict__ sr
 // block-scaled integers with their block scales (act_q.cuh; the slot's two limb rows take the
 // same 2 * d bytes as a 16-bit row).
 __device__ __forceinline__ void scatter_any(const __nv_bfloat16* __restrict__ src_row, __nv_bfloat16* __restrict__ xs,
-                                            float* __restrict__ xsc, int slot, int d, int bits, int fmt) {
+                                            float* __restrict__ xsc, int slot, int d, int bits, int fmt,
+                                            int* __restrict__ check_word) {
   if (fmt == 2) {
     int8_t* q = reinterpret_cast<int8_t*>(xs) + static_cast<size_t>(slot) * 2 * d;
     act_q_row(src_row, q, q + d, xsc + static_cast<size_t>(slot) * (d / 128), d, bits);
   } else {
-    scatter_row(src_row, xs + static_cast<size_t>(slot) * d, d, bits, fmt);
+    scatter_row(src_row, xs + static_cast<size_t>(slot) * d, d, bits, fmt, check_word);
   }
 }
 
@@ -286,7 +292,7 @@ __global__ void __launch_bounds__(128)
     scatter_x_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
                      const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
                      int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int fmt, int cnt_lo, int cnt_hi,
-                     __nv_bfloat16* __restrict__ xs, float* __restrict__ xsc) {
+                     __nv_bfloat16* __restrict__ xs, float* __restrict__ xsc, int* __restrict__ check_word) {
   pdl_wait();
   pdl_trigger();
   if (plan && blockIdx.x == 0 && threadIdx.x < 32) build_plan(plan, experts, off, E, cnt_lo, cnt_hi, threadIdx.x);
@@ -297,7 +303,7 @@ __global__ void __launch_bounds__(128)
   if (e_slot < 0 || e_slot >= E) return;  // a slot the permutation did not write (stale entry behind a dropped pair)
   const int cnt_slot = off[e_slot + 1] - off[e_slot];
   if (cnt_slot < cnt_lo || cnt_slot > cnt_hi) return;  // this expert's rows belong to another kernel family
-  scatter_any(x + static_cast<size_t>(pair / top_k) * d, xs, xsc, slot, d, experts[e_slot].bits, fmt);
+  scatter_any(x + static_cast<size_t>(pair / top_k) * d, xs, xsc, slot, d, experts[e_slot].bits, fmt, check_word);
 }
 
 // Permutation and scatter in one launch for small batches (at most PS_MAX_PAIRS pairs): one CTA
@@ -371,7 +377,7 @@ __global__ void __launch_bounds__(128)
     perm[slot] = p;
     slot_of_pair[p] = slot;
   }
-  scatter_any(x + static_cast<size_t>(p / top_k) * d, xs, xsc, slot, d, experts[e].bits, fmt);
+  scatter_any(x + static_cast<size_t>(p / top_k) * d, xs, xsc, slot, d, experts[e].bits, fmt, check_word);
 }
 
 
@@ -412,9 +418,9 @@ int ffn_mma_ksplit(const LayerDims& L, int T) {
 
 cudaError_t launch_scatter_x(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                              const int32_t* perm, const int32_t* off, int* plan, __nv_bfloat16* xs, float* xsc, int n_pairs,
-                             int fmt, int cnt_lo, int cnt_hi, cudaStream_t st) {
+                             int fmt, int cnt_lo, int cnt_hi, int* check_word, cudaStream_t st) {
   return launch_chain(scatter_x_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
-                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, fmt, cnt_lo, cnt_hi, xs, xsc);
+                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, fmt, cnt_lo, cnt_hi, xs, xsc, check_word);
 }
 
 bool permute_scatter_supported(const LayerDims& L, int n_pairs) { return n_pairs <= PS_MAX_PAIRS && L.E <= EMOE_MAX_EXPERTS; }

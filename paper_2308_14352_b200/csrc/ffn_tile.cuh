@@ -268,6 +268,12 @@ __device__ __forceinline__ void unpack_step_exact(const Raw<2>& raw, int q, uint
   }
 }
 
+// is the fp32 value outside what fp16 can hold (it would be saturated)?
+__device__ __forceinline__ bool beyond_f16(float v) { return fabsf(v) > 65504.0f; }
+// do both bf16 halves fit fp16?  (exponent field above that of 65504 = 2^15 * 1.999: bf16 exponent >= 143)
+__device__ __forceinline__ bool bf16x2_beyond_f16(uint32_t v) {
+  return ((v >> 7) & 0xffu) >= 143u || ((v >> 23) & 0xffu) >= 143u;
+}
 // two bf16 values -> two fp16 values (exact inside the fp16 range, saturating outside)
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2_sat(uint32_t v) {
   const float lo = fminf(fmaxf(__uint_as_float(v << 16), -65504.0f), 65504.0f);

@@ -294,7 +294,11 @@ __device__ __forceinline__ void count_item_done(PlanRec* recs, int ai, int lane)
 }
 
 // the hidden vector is rounded to bf16 (the layer's activation type), then carried as fp16
-__device__ __forceinline__ __half hidden_value(float h) { return f32_to_f16_sat(__bfloat162float(__float2bfloat16_rn(h))); }
+__device__ __forceinline__ __half hidden_value(float h, int* check_word) {
+  const float hb = __bfloat162float(__float2bfloat16_rn(h));
+  if (beyond_f16(hb)) atomicOr(check_word, CHECK_F16_RANGE);  // saturated below: reported, not silent
+  return f32_to_f16_sat(hb);
+}
 
 // results of one item pass: lane holds rows (gp, gp+8) x tokens (2t, 2t+1) of every tile
 template <int BITS, int NT>
@@ -316,7 +320,7 @@ __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m,
         const int n = m.rb * TMA_BOX_ROWS + 16 * warp + gp + 8 * (i >> 1);
         if (n < N) {
           const float av = tot[0][nt][i], bv = tot[1][nt][i];
-          a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(av / (1.0f + expf(-av)) * bv);
+          a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(av / (1.0f + expf(-av)) * bv, a.check_word);
         }
       } else {
 #pragma unroll
@@ -324,7 +328,7 @@ __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m,
           const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
           if (n >= N) continue;
           if (m.phase == 0)
-            a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(fmaxf(tot[mt][nt][i], 0.0f));
+            a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(fmaxf(tot[mt][nt][i], 0.0f), a.check_word);
           else
             a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + slot) * N + n] = tot[mt][nt][i];
         }

@@ -379,6 +379,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       const size_t srow = static_cast<size_t>(n) * ngroups;
       float sv[2], sv_next[2];
       for (int m = 0; m < n_mats; ++m) sv[m] = load_scale_ro(sp[m], sf16, srow);
+      bool tiny_scale = false;  // q * s below the smallest normal fp16 number would lose bits in the fp16 operand
       for (int kb = 0; kb < kb_total && ok;) {
         const int rs = raw_it % UM_RAW_STAGES;
         if (!mbar_wait(bar_raw_full + 8 * rs, (raw_it / UM_RAW_STAGES) & 1, a.check_word, abort_flag)) {
@@ -392,7 +393,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
             break;
           }
           const int g_next = min(((kb + 1) * UM_BK) / G, ngroups - 1);
-          for (int m = 0; m < n_mats; ++m) sv_next[m] = load_scale_ro(sp[m], sf16, srow + g_next);
+          for (int m = 0; m < n_mats; ++m) {
+            sv_next[m] = load_scale_ro(sp[m], sf16, srow + g_next);
+            tiny_scale |= sv[m] != 0.0f && fabsf(sv[m]) < 6.104e-5f;
+          }
           for (int m = 0; m < n_mats; ++m) {
             const __half sh = __float2half_rn(sv[m]);
             const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
@@ -417,6 +421,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
         ++raw_it;
       }
       if (!ok) break;
+      if (tiny_scale) atomicOr(a.check_word, CHECK_F16_RANGE);
       // ---- epilogue: this warp's 32 channels x its share of the token columns ----
       if (!mbar_wait(bar_acc_full, tile_it & 1, a.check_word, abort_flag)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -446,6 +451,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
                 if (dual) h = x / (1.0f + expf(-x)) * __uint_as_float(vb[j]);
                 else h = fmaxf(x, 0.0f);
                 h = __bfloat162float(__float2bfloat16_rn(h));  // the hidden vector is a bf16 tensor
+                if (beyond_f16(h)) atomicOr(a.check_word, CHECK_F16_RANGE);  // saturated below: reported, not silent
                 h = fminf(fmaxf(h, -65504.0f), 65504.0f);
                 a.hidden16[(slot0 + cc + j) * N + hpos] = __float2half_rn(h);
               } else {
@@ -478,7 +484,7 @@ __global__ void __launch_bounds__(128)
     scatter_x16_kernel(const ExpertDev* __restrict__ experts, const __nv_bfloat16* __restrict__ x,
                        const int32_t* __restrict__ ids, const int32_t* __restrict__ perm, const int32_t* __restrict__ off,
                        int E, int* __restrict__ plan, int top_k, int d, int n_pairs, int cnt_lo, int cnt_hi,
-                       __half* __restrict__ xs) {
+                       __half* __restrict__ xs, int* __restrict__ check_word) {
   pdl_wait();
   pdl_trigger();
   if (plan && blockIdx.x == 0 && threadIdx.x < 32) {
@@ -522,10 +528,13 @@ __global__ void __launch_bounds__(128)
   const int bits = experts[e_slot].bits;
   const __nv_bfloat16* src = x + static_cast<size_t>(pair / top_k) * d;
   __half* dst = xs + static_cast<size_t>(slot) * d;
+  bool beyond = false;
   for (int k = threadIdx.x; k < d; k += blockDim.x) {
-    const float v = fminf(fmaxf(__bfloat162float(src[k]), -65504.0f), 65504.0f);
-    dst[pair_pos_rt(bits, k)] = __float2half_rn(v);
+    const float xv = __bfloat162float(src[k]);
+    beyond |= beyond_f16(xv);
+    dst[pair_pos_rt(bits, k)] = __float2half_rn(fminf(fmaxf(xv, -65504.0f), 65504.0f));
   }
+  if (beyond) atomicOr(check_word, CHECK_F16_RANGE);  // saturated: reported, not silent
 }
 
 }  // namespace
@@ -537,9 +546,9 @@ bool ffn_umma_supported(const LayerDims& L) {
 
 cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
-                               int cnt_lo, int cnt_hi, cudaStream_t st) {
+                               int cnt_lo, int cnt_hi, int* check_word, cudaStream_t st) {
   return launch_chain(scatter_x16_kernel, dim3(n_pairs), dim3(128), 0, st, experts, reinterpret_cast<const __nv_bfloat16*>(x), ids,
-                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, cnt_lo, cnt_hi, reinterpret_cast<__half*>(xs16));
+                      perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, cnt_lo, cnt_hi, reinterpret_cast<__half*>(xs16), check_word);
 }
 
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,

@@ -164,7 +164,7 @@ extern "C" int emoe_moe_forward_routed_static(int device, const emoe_layer_desc*
   }
   EMOE_TRY(launch_permute(ids, P, L.E, counts, off, perm, slot_of_pair, check, st));
   if (ffn_mma_supported(L)) {
-    EMOE_TRY(launch_scatter_x(L, table, x, ids, perm, off, nullptr, xs, nullptr, P, 0, 1, INT_MAX, st));
+    EMOE_TRY(launch_scatter_x(L, table, x, ids, perm, off, nullptr, xs, nullptr, P, 0, 1, INT_MAX, check, st));
     EMOE_TRY(launch_ffn_mma(0, L, table, xs, off, reinterpret_cast<__nv_bfloat16*>(hidden), o_part, 1, P, T, st));
     EMOE_TRY(launch_ffn_mma(1, L, table, reinterpret_cast<const __nv_bfloat16*>(hidden), off,
                             reinterpret_cast<__nv_bfloat16*>(hidden), o_part, w.ksplit, P, T, st));

@@ -167,6 +167,34 @@ def test_bounded_wait_inside_the_kernel_runs_out_and_the_context_stays_usable():
         assert np.array_equal(ids2, ids) and np.array_equal(y2, y)
 
 
+@pytest.mark.parametrize("path", [0, 3, 4])
+def test_fp16_operand_kernels_report_values_outside_their_range(path):
+    """The default tensor-core kernels carry activations as fp16.  Inputs (or hidden values) beyond
+    65504 are saturated there, and the many-token kernel also loses bits of q * s below 2^-14: neither
+    may pass silently.  The device status must say so; the same inputs on kernel family 6 stay
+    inside the bar (previous test)."""
+    shape = inputs.LayerShape(512, 1024, 4, 1, "relu", "softmax", 128, "f16", "bf16")
+    bits, T = [8, 4, 2, 4], 9
+    cases = [(3.0e4, 0.02)]                    # x beyond 65504
+    if path == 4:
+        cases.append((1.0, 1.0e-5))            # scales below 2^-14: q * s is subnormal as fp16
+    for scale_x, std in cases:
+        W = inputs.expert_set(28, 0, shape, std)
+        x = inputs.to_bf16_valued(inputs.activations(28, 0, T, shape.d_model, "bf16") * np.float32(scale_x))
+        Wr = inputs.router_weight(28, 0, shape.d_model, shape.n_experts, std=0.05 / scale_x)
+        with layer.MoELayer(shape, bits, max_tokens=T) as moe:
+            B.emoe_set_ffn_path(moe.ctx, path)
+            moe.pack_from_host(W)
+            with pytest.raises(B.EmoeError) as ei:
+                moe.forward(x, Wr)
+            assert ei.value.status == B.ERR_RANGE, (path, scale_x)
+            # ordinary inputs afterwards: no flag is left over
+            x_ok = inputs.activations(28, 0, T, shape.d_model, "bf16")
+            W_ok = inputs.expert_set(28, 0, shape, 0.02)
+            moe.pack_from_host(W_ok)
+            moe.forward(x_ok, inputs.router_weight(28, 0, shape.d_model, shape.n_experts, std=0.05))
+
+
 UMMA_CASES = [
     ("relu", 128, "f16", 512, 1024, 4, 1, "softmax", [8, 4, 2, 4], 200),              # ~50 tokens per expert
     ("relu", 128, "f16", 512, 1024, 2, 1, "softmax", [4, 2], 300),                    # two token tiles per expert
@@ -225,9 +253,9 @@ def test_both_paths_agree_and_default_picks_tensor_cores():
     e_mma = _run_case(shape, [2, 4, 8, 4], 12, seed=23, path=2)
     assert e_auto == e_mma and e_gemv <= 2e-3
     big = inputs.LayerShape(512, 1024, 4, 2, "swiglu", "softmax_renorm", 128, "f16", "bf16")
-    # wide enough for the weight-streaming kernels: the default is the int8 tensor-core one
-    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=0) == _run_case(big, [2, 4, 8, 4], 12, seed=23, path=6)
-    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=3) <= 2e-3
+    # wide enough for the weight-streaming kernels: the default is the TMA-staged mma.sync one
+    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=0) == _run_case(big, [2, 4, 8, 4], 12, seed=23, path=3)
+    assert _run_case(big, [2, 4, 8, 4], 12, seed=23, path=6) <= 2e-3
 
 
 def test_zipf_bias_and_many_tokens_on_one_expert():
