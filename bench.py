@@ -29,10 +29,25 @@ if ROOT not in sys.path:
 
 from paper_2308_14352_b200 import inputs  # noqa: E402
 
-# DRAM bytes (read + write) of the expert-FFN launch of one layer (mean of the two layers of the ncu
-# capture summarised in profiles/ffn_tma_kernel_switch_base_decode_T64.md); reported as `traffic`
-# for that workload only, and to be set back to None whenever that kernel changes.
-NCU_DRAM_BYTES_PER_LAYER = {("switch_base_decode", 64): 74.7e6}
+
+
+def ncu_traffic_per_layer(workload: str, T: int):
+    """DRAM bytes (read + write) per expert-FFN launch from the last ncu capture, or None when the kernel's
+    source changed since (profiles/ncu_traffic.json records the capture and the hash of the source it saw)."""
+    import hashlib
+
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as fh:
+        rec = json.load(fh).get(f"{workload}:{T}")
+    if not rec:
+        return None
+    src = os.path.join(ROOT, "paper_2308_14352_b200", "csrc", rec["source"])
+    with open(src, "rb") as fh:
+        if hashlib.sha256(fh.read()).hexdigest()[:16] != rec["source_sha16"]:
+            return None
+    return float(rec["dram_bytes_per_launch"])
 
 METRIC = "MoE-layer tokens/s"
 UNIT = "tokens/s"
@@ -50,6 +65,7 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying a CUDA graph")
     ap.add_argument("--ffn-path", type=int, default=0, help="0 auto, 1 CUDA-core GEMV, 2 tensor-core path")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short measurements of the other workloads")
     ap.add_argument("--no-pdl", action="store_true", help="switch programmatic dependent launch off")
     ap.add_argument("--no-fuse", action="store_true", help="run the two projections of the expert FFNs as two launches")
     ap.add_argument("--slots", type=int, default=0, help="mixtral_stack_cached: slots of the HBM expert cache (default: a quarter of the experts)")
@@ -65,6 +81,15 @@ def load_peaks():
             d = json.load(fh)
         return float(d["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def load_tensor_peak():
+    """Measured dense bf16 rate (burst) of this machine's B200s, else the earlier measurement on this machine."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            return float(json.load(fh)["bf16_tflops"]), "measured"
+    return 1590.0, "fallback"
 
 
 class ClockSampler:
@@ -244,6 +269,190 @@ def run_reference(args, w, T, n_layers, rank, world):
 
 
 # ------------------------------------------------------------------------------------------------
+# offline kernels (quantise + pack, width change) and the short runs of the other workloads
+# ------------------------------------------------------------------------------------------------
+def time_offline_kernels(ctx, dev):
+    """The two offline kernels on ONE large matrix (14336 x 4096 fp32 = 235 MB, larger than L2), 20 launches
+    back to back between two events, nothing else running: quantise + pack at each width, and the width
+    change 8 -> 4 and 4 -> 2 of the stored matrix."""
+    import torch
+
+    from paper_2308_14352_b200 import binding as B
+
+    peak, _ = load_peaks()
+    N, K, G, reps = 14336, 4096, 128, 20
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(99)
+    W = torch.randn(N, K, generator=gen, device=dev) * 0.02
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    out = {"matrix": f"{N}x{K} fp32, group-{G} fp16 scales, {reps} launches back to back", "pack": {}, "requantize": {}}
+    stored = {}
+    for bits in (8, 4, 2):
+        p = torch.empty(N * K * bits // 8, dtype=torch.uint8, device=dev)
+        sc = torch.empty(N * (K // G), dtype=torch.float16, device=dev)
+        B.emoe_pack_expert(ctx, W.data_ptr(), N, K, bits, G, B.DTYPE_F16, p.data_ptr(), sc.data_ptr(), 0)
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(reps):
+            B.emoe_pack_expert(ctx, W.data_ptr(), N, K, bits, G, B.DTYPE_F16, p.data_ptr(), sc.data_ptr(), 0)
+        ev1.record()
+        ev1.synchronize()
+        gbs = reps * (N * K * 4 + N * K * bits // 8 + sc.numel() * 2) / (ev0.elapsed_time(ev1) * 1e-3) / 1e9
+        out["pack"][f"int{bits}"] = {"gbs": gbs, "frac_of_hbm_peak": gbs / peak}
+        stored[bits] = (p, sc)
+    for b_in, b_out in ((8, 4), (4, 2)):
+        p_in, s_in = stored[b_in]
+        p_out = torch.empty(N * K * b_out // 8, dtype=torch.uint8, device=dev)
+        s_out = torch.empty_like(s_in)
+        B.emoe_requantize_expert(ctx, p_in.data_ptr(), s_in.data_ptr(), N, K, b_in, b_out, G, B.DTYPE_F16, p_out.data_ptr(),
+                                 s_out.data_ptr(), 0)
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(reps):
+            B.emoe_requantize_expert(ctx, p_in.data_ptr(), s_in.data_ptr(), N, K, b_in, b_out, G, B.DTYPE_F16,
+                                     p_out.data_ptr(), s_out.data_ptr(), 0)
+        ev1.record()
+        ev1.synchronize()
+        gbs = reps * (N * K * (b_in + b_out) // 8 + 2 * s_out.numel() * 2) / (ev0.elapsed_time(ev1) * 1e-3) / 1e9
+        out["requantize"][f"int{b_in}_to_int{b_out}"] = {"gbs": gbs, "frac_of_hbm_peak": gbs / peak}
+    out["note"] = ("offline stage (Section 3.2), not part of the step; bytes = fp32 read + packed and scale bytes written "
+                   "(pack), packed and scale bytes read and written (width change)")
+    return out
+
+
+PER_CONFIG = (
+    # (label, workload, tokens, copies of the layer so that the weights of a step exceed L2)
+    ("cfg0", "switch_tiny_fp32", 16, 8),
+    ("cfg1 T=1", "switch_base_decode", 1, 12),
+    ("cfg1 T=8", "switch_base_decode", 8, 12),
+    ("cfg2", "switch_large_prefill", 2048, 2),
+    ("cfg3 T=1", "mixtral_decode", 1, 2),
+    ("cfg3 T=4", "mixtral_decode", 4, 2),
+    ("cfg3 T=16", "mixtral_decode", 16, 2),
+    ("cfg3 T=32", "mixtral_decode", 32, 2),
+    ("mixtral-shape prefill T=2048 (the dense load of cfg4)", "mixtral_decode", 2048, 1),
+)
+
+
+def measure_config(label, wname, T, copies, local, steps):
+    """One short measurement: `copies` independent layers of the workload's shape (weights drawn on the
+    device, seeded; packed by the library), the step = the forward of all of them, replayed as a CUDA graph."""
+    import torch
+
+    from paper_2308_14352_b200 import binding as B, layer as L
+
+    w = inputs.WORKLOADS[wname]
+    sh = w.shape
+    dev = torch.device("cuda", local)
+    ctx = B.emoe_create(local, B.emoe_workspace_bytes(L.make_desc(sh), T))
+    gen = torch.Generator(device=dev)
+    layers, xs, Wrs, biases, ys, ids_dev = [], [], [], [], [], []
+    try:
+        for c in range(copies):
+            l_idx = c % max(1, w.n_layers)
+            bits = inputs.expert_bits(w, l_idx)
+            moe = L.MoELayer(sh, bits, device=local, max_tokens=T, ctx=ctx)
+            for e in range(sh.n_experts):
+                for m in range(sh.n_matrices):
+                    N, K = sh.matrix_shape(m)
+                    gen.manual_seed((w.seed << 40) ^ (c << 24) ^ (e << 8) ^ m)
+                    Wd = torch.randn(N, K, generator=gen, device=dev) * 0.02
+                    moe.pack_matrix(e, m, Wd)
+                    del Wd
+            x, Wr, bias = inputs.layer_tensors(w, l_idx, T, batch_tag=c)
+            layers.append(moe)
+            xs.append(moe.to_device_x(x))
+            Wrs.append(torch.from_numpy(Wr).to(dev))
+            biases.append(None if bias is None else torch.from_numpy(bias).to(dev))
+            ys.append(torch.zeros(T, sh.d_model, dtype=torch.float32, device=dev))
+            ids_dev.append(torch.zeros(T, sh.top_k, dtype=torch.int32, device=dev))
+        torch.cuda.synchronize()
+        stream = torch.cuda.Stream(device=dev)
+
+        def fwd(want_ids=False):
+            for l, moe in enumerate(layers):
+                moe.forward_device(xs[l], Wrs[l], biases[l], ys[l], ids_dev[l] if want_ids else None, None, None,
+                                   stream.cuda_stream)
+
+        with torch.cuda.stream(stream):
+            fwd(True)
+        stream.synchronize()
+        status = B.emoe_device_status(ctx, stream.cuda_stream)
+        if status != B.OK:
+            return {"config": label, "error": B.status_string(status)}
+        ssz = 2 if sh.scale_dtype == "f16" else 4
+        nbytes, flops, heavy_flops = 0, 0, 0
+        per_expert_weights = sum(sh.matrix_shape(m)[0] * sh.matrix_shape(m)[1] for m in range(sh.n_matrices))
+        for l, moe in enumerate(layers):
+            picks = ids_dev[l].cpu().numpy().reshape(-1)
+            counts = np.bincount(picks, minlength=sh.n_experts)
+            for e in np.flatnonzero(counts):
+                for m in range(sh.n_matrices):
+                    N, K = sh.matrix_shape(m)
+                    nbytes += N * K * moe.bits[e] // 8 + N * (K // (sh.group or K)) * ssz
+                flops += 2 * int(counts[e]) * per_expert_weights
+                # experts above the ridge of the roofline (tokens x 2 flops per weight against bits / 8 bytes per weight)
+                if counts[e] > 32:
+                    heavy_flops += 2 * int(counts[e]) * per_expert_weights
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            fwd()
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        B.emoe_set_timing(ctx, True)
+        with torch.cuda.stream(stream):
+            for _ in range(5):
+                fwd()
+            stream.synchronize()
+        a, b, calls = B.emoe_read_timing(ctx)
+        B.emoe_set_timing(ctx, False)
+        kms = (a + b) / calls * copies
+        hbm, _ = load_peaks()
+        tf_peak, _ = load_tensor_peak()
+        t_hbm, t_tensor = nbytes / (hbm * 1e9), flops / (tf_peak * 1e12)
+        tensor_bound = t_tensor > t_hbm
+        out = {
+            "config": label, "workload": f"{wname} T={T}", "layers_in_step": copies, "ms_per_step": ms,
+            "tokens_per_s": T * copies / (ms * 1e-3), "expert_kernel_ms_per_step": kms,
+            "kernels_per_layer": B.emoe_kernels_last_forward(ctx),
+            "roofline": ({"bound": "tensor", "achieved": flops / (kms * 1e-3) / 1e12, "peak": tf_peak, "unit": "TFLOP/s",
+                          "frac": flops / (kms * 1e-3) / 1e12 / tf_peak, "flops": flops} if tensor_bound else
+                         {"bound": "hbm", "achieved": nbytes / (kms * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s",
+                          "frac": nbytes / (kms * 1e-3) / 1e9 / hbm, "algorithmic_bytes": nbytes}),
+            "frac_of_roofline_time": max(t_hbm, t_tensor) / (kms * 1e-3),
+        }
+        if heavy_flops and not tensor_bound:
+            # the dense-contraction subset of a skewed load: its flops against the time of the WHOLE expert stage
+            # (a lower bound of the tensor rate of that subset, the light experts' streaming time is in it)
+            out["experts_above_ridge"] = {"flops": heavy_flops, "tflops_lower_bound": heavy_flops / (kms * 1e-3) / 1e12,
+                                          "frac_of_bf16_peak_lower_bound": heavy_flops / (kms * 1e-3) / 1e12 / tf_peak}
+        return out
+    finally:
+        for moe in layers:
+            moe.close()
+        torch.cuda.synchronize()
+        B.emoe_destroy(ctx)
+
+
+def run_per_config(local, steps):
+    out = []
+    for label, wname, T, copies in PER_CONFIG:
+        try:
+            out.append(measure_config(label, wname, T, copies, local, steps))
+        except Exception as exc:  # a failing side measurement must not lose the headline line
+            out.append({"config": label, "error": repr(exc)[:200]})
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
 # the CUDA arm
 # ------------------------------------------------------------------------------------------------
 def run_emoe(args, w, T, n_layers, rank, world, local):
@@ -266,8 +475,6 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
     # ---- build the stack: seeded fp32 experts -> packed on the device by the library ------------
     t_build = time.perf_counter()
     layers, xs, Wrs, biases, ys = [], [], [], [], []
-    pack_bytes_in = 0
-    pack_ms = 0.0
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     from concurrent.futures import ThreadPoolExecutor
 
@@ -280,16 +487,6 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
         for (e, m, N, K), Wh in zip(jobs, mats):
             Wd = torch.from_numpy(Wh).to(dev)
             moe.pack_matrix(e, m, Wd)
-            if l == 0 and e < 4:
-                # quantise+pack kernel timed on its own: the same matrix packed 10 times back to back
-                torch.cuda.synchronize()
-                ev0.record()
-                for _ in range(10):
-                    moe.pack_matrix(e, m, Wd)
-                ev1.record()
-                ev1.synchronize()
-                pack_ms += ev0.elapsed_time(ev1)
-                pack_bytes_in += 10 * (N * K * 4 + N * K * bits[e] // 8)
             del Wd, Wh
         x, Wr, bias = inputs.layer_tensors(w, l, T)
         layers.append(moe)
@@ -298,31 +495,9 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
         biases.append(None if bias is None else torch.from_numpy(bias).to(dev))
         ys.append(torch.zeros(T, sh.d_model, dtype=torch.float32, device=dev))
     torch.cuda.synchronize()
-    # width-lowering kernel timed on its own: the stored matrices of the first layer's experts moved one
-    # width down (8 -> 4, 4 -> 2) into scratch buffers, 10 times back to back
-    requant_bytes, requant_ms = 0, 0.0
-    moe0 = layers[0]
-    sdt_code = B.DTYPE_F16 if sh.scale_dtype == "f16" else B.DTYPE_F32
-    for e in range(min(8, sh.n_experts)):
-        b_in = moe0.bits[e]
-        if b_in == 2:
-            continue
-        b_out = b_in // 2
-        for m in range(sh.n_matrices):
-            N, K = sh.matrix_shape(m)
-            p_out = torch.empty(N * K * b_out // 8, dtype=torch.uint8, device=dev)
-            s_out = torch.empty_like(moe0.scales[e][m])
-            torch.cuda.synchronize()
-            ev0.record()
-            for _ in range(10):
-                B.emoe_requantize_expert(ctx, moe0.packed[e][m].data_ptr(), moe0.scales[e][m].data_ptr(), N, K, b_in, b_out,
-                                         sh.group, sdt_code, p_out.data_ptr(), s_out.data_ptr(), 0)
-            ev1.record()
-            ev1.synchronize()
-            requant_ms += ev0.elapsed_time(ev1)
-            requant_bytes += 10 * (N * K * (b_in + b_out) // 8 + 2 * s_out.numel() * s_out.element_size())
-            del p_out, s_out
+    pool.shutdown(wait=True)
     build_s = time.perf_counter() - t_build
+    offline = time_offline_kernels(ctx, dev) if (rank == 0 and world == 1) else None
 
     ids_dev = [torch.zeros(T, sh.top_k, dtype=torch.int32, device=dev) for _ in range(n_layers)]
     stream = torch.cuda.Stream(device=dev)
@@ -522,30 +697,28 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
                 "kernel": "expert-FFN kernels (both projections of every layer)", "bound": "hbm",
                 "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_8TBs": achieved / 8000.0,
-                "traffic": (NCU_DRAM_BYTES_PER_LAYER[(w.name, T)] * n_layers
-                            if (w.name, T) in NCU_DRAM_BYTES_PER_LAYER and args.ffn_path == 0 else None),
+                "traffic": (ncu_traffic_per_layer(w.name, T) * n_layers
+                            if args.ffn_path == 0 and ncu_traffic_per_layer(w.name, T) is not None else None),
                 "per": "bench step (all layers); achieved = algorithmic bytes per step / kernel ms per step",
                 "algorithmic_bytes_per_step": expert_bytes_per_step, "kernel_ms_per_step": ffn_ms_per_step,
                 "first_projection_ms": ffn0_ms / calls * n_layers, "second_projection_ms": ffn1_ms / calls * n_layers,
             },
             "whole_step_gbs": expert_bytes_per_step / (ms_job * 1e-3) / 1e9,
-            "pack": {"gbs": pack_bytes_in / (pack_ms * 1e-3) / 1e9, "frac_of_hbm_peak": pack_bytes_in / (pack_ms * 1e-3) / 1e9 / peak,
-                     "note": "expert quantise+pack kernel (offline stage, not part of the step): fp32 bytes read + packed "
-                             "bytes written per second, matrices of the first experts packed 10 times back to back"},
-            "requantize": (None if requant_ms == 0.0 else
-                           {"gbs": requant_bytes / (requant_ms * 1e-3) / 1e9,
-                            "frac_of_hbm_peak": requant_bytes / (requant_ms * 1e-3) / 1e9 / peak,
-                            "note": "stored experts moved one width down (8 -> 4, 4 -> 2) without the fp32 original "
-                                    "(offline stage, not part of the step): packed + scale bytes read and written per second"}),
+            "offline_kernels": offline,
             "build_seconds": build_s,
         }
         if cpu is not None:
             out["cpu_baseline"] = cpu
-        print(json.dumps(out))
     for moe in layers:
         moe.close()
     torch.cuda.synchronize()
     B.emoe_destroy(ctx)
+    if rank == 0:
+        if world == 1 and not args.no_per_config and w.name == "switch_base_decode":
+            del layers, xs, Wrs, ys, x_stage, y_stage
+            torch.cuda.empty_cache()
+            out["per_config"] = run_per_config(local, max(5, min(args.steps, 20)))
+        print(json.dumps(out))
 
 
 # ------------------------------------------------------------------------------------------------
