@@ -233,7 +233,9 @@ int emoe_set_wait_limit(emoe_ctx* ctx, unsigned polls);
 
 /* Test hook for the above: the second projection of every expert waits for `extra` more
  * completions of its first projection than will ever be counted, so that its bounded wait runs
- * out.  0 (the default) in any real use.  No counterpart in the paper. */
+ * out; the grid-wide wait of the one-launch routing kernel (emoe_set_fused_routing) likewise
+ * waits for `extra` more arrivals than the grid has CTAs.  0 (the default) in any real use.  No
+ * counterpart in the paper. */
 int emoe_debug_expect_extra_completions(emoe_ctx* ctx, int extra);
 
 /* Programmatic dependent launch along the kernels of a forward call (on by default): each
@@ -247,6 +249,16 @@ int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled);
  * projection of every expert.  Results are identical either way; switch it off to run the two
  * projections as two launches (to compare timings, or to time them separately). */
 int emoe_set_fused_projections(emoe_ctx* ctx, int enabled);
+
+/* Router, Top-K, permutation, scatter and work plan (Section 2.1: every token goes to its Top-K
+ * experts) in ONE launch for batches of at most 1024 token-expert pairs on the weight-streaming
+ * kernels: one CTA per token; the CTAs meet at a bounded grid-wide wait on an arrival counter
+ * (all of them are resident: the library checks the grid against the device's capacity), after
+ * which each places its own pairs.  A forward call is then three launches.  Off by default: as
+ * measured, the chain of dependent launches is a little faster than the grid-wide wait.  ids,
+ * gates, permutation and outputs are identical either way.  A wait that runs out reports
+ * EMOE_ERR_TIMEOUT through emoe_device_status (limit: emoe_set_wait_limit). */
+int emoe_set_fused_routing(emoe_ctx* ctx, int enabled);
 
 /* Number of kernels the last emoe_moe_forward / emoe_moe_forward_routed call on this context
  * enqueued (router + Top-K, permutation, scatter, expert FFNs, combine: Sections 2.1 and 3.2 name

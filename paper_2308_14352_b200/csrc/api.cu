@@ -104,9 +104,11 @@ struct emoe_ctx {
   int ffn_path = 0;
   bool pdl = true;  // programmatic dependent launch along the kernel chain of a forward call
   bool fuse_projections = true;  // weight-streaming kernel: both projections in one launch
+  bool fuse_routing = false;     // router + Top-K + permutation + scatter + plan in one launch (small batches)
   bool timing = false;
   unsigned wait_limit = 0;  // polls before a wait inside the int8 streaming kernel gives up (0 = its default)
   int dep_extra = 0;        // test hook: extra completions the second projection waits for
+  int resident_route_ctas = -1;  // CTAs of the one-launch routing kernel the device holds at once (-1 = not asked yet)
   int kernels_last = 0;  // kernels the last forward call enqueued
   ExpertCache* cache = nullptr;  // expert cache (cache.cu), optional
   std::vector<cudaEvent_t> table_events;  // per table block: its upload has left the pinned mirror
@@ -290,15 +292,8 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   float* hsc = reinterpret_cast<float*>(ws + w.hsc);
   float* o_part = reinterpret_cast<float*>(ws + w.o_part);
 
-  const int32_t* ids_use = ids;
-  const float* gates_use = gates;
-  if (routed) {
-    ids_use = ids_in;
-    gates_use = gates_in;
-  } else {
-    EMOE_LAUNCH(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,
-                                      L.top_k, L.gate_mode == EMOE_GATE_SOFTMAX_RENORM, ids, gates, nullptr, st));
-  }
+  const int32_t* ids_use = routed ? ids_in : ids;
+  const float* gates_use = routed ? gates_in : gates;
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
   const bool can_i8 = ffn_i8_supported(L) && tmaps != nullptr;
   const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
@@ -320,6 +315,15 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   if (ctx->ffn_path == 6 && !use_i8) return EMOE_ERR_UNSUPPORTED;
   // small batches on the streaming kernels: permutation, scatter and plan in one launch
   const bool one_launch_permute = (use_tma || use_i8) && ctx->fuse_projections && permute_scatter_supported(L, P);
+  // ... and, when the router runs here too, router and Top-K in that same launch
+  if (ctx->resident_route_ctas < 0) ctx->resident_route_ctas = route_permute_scatter_resident_ctas(ctx->device);
+  const bool one_launch_route =
+      ctx->fuse_routing && one_launch_permute && !routed && route_permute_scatter_supported(L, T, ctx->resident_route_ctas);
+  if (!routed && !one_launch_route)
+    EMOE_LAUNCH(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,
+                                      L.top_k, L.gate_mode == EMOE_GATE_SOFTMAX_RENORM, ids, gates, nullptr, st));
+  unsigned* route_sync = reinterpret_cast<unsigned*>(ctx->check_word + 1);
+  const unsigned route_wait = ctx->wait_limit ? ctx->wait_limit : (1u << 22);
   if (!one_launch_permute)
     EMOE_LAUNCH(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
   int ksplit = 1;
@@ -377,7 +381,11 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
   } else if (use_i8) {
     ksplit = ffn_i8_ksplit(L, T);
-    if (one_launch_permute)
+    if (one_launch_route)
+      EMOE_LAUNCH(ctx, launch_route_permute_scatter(L, table, x, T, router_W, router_bias, bias_token_stride, ids, gates, counts,
+                                                    off, perm, slot_of_pair, plan, xs, xsc, 2, route_sync, route_wait,
+                                                    ctx->dep_extra, ctx->check_word, st));
+    else if (one_launch_permute)
       EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, xsc, P, 2,
                                               ctx->check_word, st));
     else
@@ -401,7 +409,11 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     }
   } else if (use_tma) {
     ksplit = ffn_tma_ksplit(L, T);
-    if (one_launch_permute)
+    if (one_launch_route)
+      EMOE_LAUNCH(ctx, launch_route_permute_scatter(L, table, x, T, router_W, router_bias, bias_token_stride, ids, gates, counts,
+                                                    off, perm, slot_of_pair, plan, xs, nullptr, 1, route_sync, route_wait,
+                                                    ctx->dep_extra, ctx->check_word, st));
+    else if (one_launch_permute)
       EMOE_LAUNCH(ctx, launch_permute_scatter(L, table, x, ids_use, counts, off, perm, slot_of_pair, plan, xs, nullptr, P, 1,
                                               ctx->check_word, st));
     else
@@ -466,8 +478,8 @@ emoe_ctx* emoe_create(int device, size_t workspace_bytes, int* status) {
   ctx->device = device;
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess && workspace_bytes > 0) e = cudaMalloc(&ctx->workspace, workspace_bytes);
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->check_word, sizeof(int));
-  if (e == cudaSuccess) e = cudaMemset(ctx->check_word, 0, sizeof(int));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->check_word, 4 * sizeof(int));  // + the routing kernel's two grid counters
+  if (e == cudaSuccess) e = cudaMemset(ctx->check_word, 0, 4 * sizeof(int));
   if (e == cudaSuccess) e = cudaMallocHost(&ctx->check_host, sizeof(int));
   if (e == cudaSuccess) e = cudaMalloc(&ctx->tables_dev, TABLE_BLOCK_BYTES * MAX_TABLES);
   if (e == cudaSuccess) e = cudaMallocHost(&ctx->tables_pin, TABLE_BLOCK_BYTES * MAX_TABLES);
@@ -516,7 +528,7 @@ int emoe_device_status(emoe_ctx* ctx, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
   EMOE_CUDA(ctx, cudaMemcpyAsync(ctx->check_host, ctx->check_word, sizeof(int), cudaMemcpyDeviceToHost, st));
-  EMOE_CUDA(ctx, cudaMemsetAsync(ctx->check_word, 0, sizeof(int), st));
+  EMOE_CUDA(ctx, cudaMemsetAsync(ctx->check_word, 0, 4 * sizeof(int), st));  // also the grid counters a timed-out wait left behind
   EMOE_CUDA(ctx, cudaStreamSynchronize(st));
   if (*ctx->check_host & CHECK_WAIT_TIMEOUT) return EMOE_ERR_TIMEOUT;
   if (*ctx->check_host & CHECK_BAD_EXPERT_ID) return EMOE_ERR_DEVICE_CHECK;
@@ -671,6 +683,12 @@ int emoe_kernels_last_forward(const emoe_ctx* ctx) { return ctx ? ctx->kernels_l
 int emoe_set_fused_projections(emoe_ctx* ctx, int enabled) {
   if (!ctx) return EMOE_ERR_INVALID_ARG;
   ctx->fuse_projections = enabled != 0;
+  return EMOE_OK;
+}
+
+int emoe_set_fused_routing(emoe_ctx* ctx, int enabled) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  ctx->fuse_routing = enabled != 0;
   return EMOE_OK;
 }
 

@@ -1073,7 +1073,9 @@ bool ffn_i8_supported(const LayerDims& L) {
 // tile, an expert with more tokens than the tile takes another pass over its weights (from L2)
 int ffn_i8_token_tile(const LayerDims& L, int T) {
   const double mean = static_cast<double>(T) * L.top_k / L.E;
-  return mean <= 6.0 ? 8 : (mean <= 12.0 ? 16 : 32);
+  // a gated layer's stage carries two weight boxes: with 32-token tiles fewer than three stages fit
+  const int widest = L.act == EMOE_ACT_SWIGLU ? 16 : 32;
+  return mean <= 6.0 ? 8 : (mean <= 12.0 ? 16 : widest);
 }
 
 int ffn_i8_ksplit(const LayerDims& L, int T) {

@@ -13,6 +13,7 @@
 #include <math_constants.h>
 
 #include "common.cuh"
+#include "scatter.cuh"
 
 namespace emoe {
 namespace {
@@ -20,13 +21,13 @@ namespace {
 constexpr int ROUTER_THREADS = 256;
 constexpr int ROUTER_DC = 1024;  // d_model chunk held in shared memory
 
+// Logits of the CTA's TT tokens into zs[TT][EP] (shared memory).  x and the router weights are
+// inputs of the call: the logits are computed while the kernels in front drain; the wait on
+// them comes before the first write to global memory (ids / gates may still be read there).
 template <int TT>
-__global__ void __launch_bounds__(ROUTER_THREADS)
-    router_topk_kernel(const void* __restrict__ x, int x_bf16, int T, int d, const float* __restrict__ Wr,
-                       const float* __restrict__ bias, int bias_stride, int E, int EP, int ep_shift, int top_k,
-                       int renorm, int32_t* __restrict__ ids, float* __restrict__ gates,
-                       float* __restrict__ logits) {
-  extern __shared__ float smem[];
+__device__ __forceinline__ void router_logits(float* smem, const void* __restrict__ x, int x_bf16, int T, int d,
+                                              const float* __restrict__ Wr, const float* __restrict__ bias,
+                                              int bias_stride, int E, int EP, int ep_shift, float* __restrict__ logits) {
   float* xs = smem;                          // [TT][ROUTER_DC]
   float* red = xs + TT * ROUTER_DC;          // [S][TT][EP]
   float* zs = red + ROUTER_THREADS * TT;     // [TT][EP]
@@ -36,9 +37,6 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
   const int S = ROUTER_THREADS >> ep_shift;
   const int t0 = blockIdx.x * TT;
 
-  // x and the router weights are inputs of the call: the logits are computed while the kernels
-  // in front drain; the wait comes before the first write (ids / gates may still be read there)
-  pdl_trigger();
   float acc[TT];
 #pragma unroll
   for (int tt = 0; tt < TT; ++tt) acc[tt] = 0.0f;
@@ -94,19 +92,19 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
     zs[idx] = z;
   }
   __syncthreads();
+}
 
-  const int warp = tid >> 5, lane = tid & 31;
-  if (warp >= TT) return;
-  const int t = t0 + warp;
-  if (t >= T) return;
-
+// Softmax and Top-K of one token by one warp from its row of logits zrow[EP] (shared memory):
+// K rounds of arg-max, ties to the lower expert index.  Lane r < top_k returns the r-th pick.
+__device__ __forceinline__ void router_pick(const float* zrow, int E, int top_k, int renorm, int lane, int& out_id,
+                                            float& out_gate) {
   constexpr int MAXJ = EMOE_MAX_EXPERTS / 32;
   float zv[MAXJ], pe[MAXJ];
   float m = -CUDART_INF_F;
 #pragma unroll
   for (int j = 0; j < MAXJ; ++j) {
     const int ee = lane + 32 * j;
-    zv[j] = ee < E ? zs[warp * EP + ee] : -CUDART_INF_F;
+    zv[j] = ee < E ? zrow[ee] : -CUDART_INF_F;
     m = fmaxf(m, zv[j]);
   }
 #pragma unroll
@@ -158,9 +156,140 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
       my_p = p;
     }
   }
+  out_id = my_id;
+  out_gate = renorm ? my_p / psel : my_p;
+}
+
+template <int TT>
+__global__ void __launch_bounds__(ROUTER_THREADS)
+    router_topk_kernel(const void* __restrict__ x, int x_bf16, int T, int d, const float* __restrict__ Wr,
+                       const float* __restrict__ bias, int bias_stride, int E, int EP, int ep_shift, int top_k,
+                       int renorm, int32_t* __restrict__ ids, float* __restrict__ gates,
+                       float* __restrict__ logits) {
+  extern __shared__ float smem[];
+  pdl_trigger();
+  router_logits<TT>(smem, x, x_bf16, T, d, Wr, bias, bias_stride, E, EP, ep_shift, logits);
+  const float* zs = smem + TT * ROUTER_DC + ROUTER_THREADS * TT;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp >= TT) return;
+  const int t = blockIdx.x * TT + warp;
+  if (t >= T) return;
+  int my_id;
+  float my_gate;
+  router_pick(zs + warp * EP, E, top_k, renorm, lane, my_id, my_gate);
   if (lane < top_k) {
     ids[static_cast<size_t>(t) * top_k + lane] = my_id;
-    gates[static_cast<size_t>(t) * top_k + lane] = renorm ? my_p / psel : my_p;
+    gates[static_cast<size_t>(t) * top_k + lane] = my_gate;
+  }
+}
+
+// Router, Top-K, permutation, scatter and work plan in one launch for small batches: one CTA per
+// token.  A CTA computes its token's picks, publishes them, and waits until every CTA of the grid
+// has done so (an arrival counter in global memory; the host launches this kernel only with a
+// grid that is resident at once, and the wait is bounded).  Then it works out the slots of its
+// own pairs exactly as permute_scatter_kernel does and copies its row into them; CTA 0 also
+// writes counts, offsets and the plan.  sync[0] counts arrivals, sync[1] departures; the last CTA
+// to leave sets both back to zero for the next launch.
+constexpr int RPS_MAX_PAIRS = 1024;
+__global__ void __launch_bounds__(ROUTER_THREADS)
+    route_permute_scatter_kernel(const __nv_bfloat16* __restrict__ x, int T, int d, const float* __restrict__ Wr,
+                                 const float* __restrict__ bias, int bias_stride, int E, int EP, int ep_shift, int top_k,
+                                 int renorm, int32_t* ids, float* __restrict__ gates,
+                                 const ExpertDev* __restrict__ experts, int fmt, int32_t* __restrict__ counts,
+                                 int32_t* __restrict__ off, int32_t* __restrict__ perm,
+                                 int32_t* __restrict__ slot_of_pair, int* __restrict__ plan, int* __restrict__ check_word,
+                                 __nv_bfloat16* __restrict__ xs_out, float* __restrict__ xsc, unsigned* sync,
+                                 unsigned wait_limit, int extra_arrivals) {
+  extern __shared__ float smem[];
+  __shared__ int s_ids[RPS_MAX_PAIRS];
+  __shared__ int s_off[EMOE_MAX_EXPERTS + 1];
+  __shared__ int s_red[2][ROUTER_THREADS / 32];
+  __shared__ int s_ok;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t = blockIdx.x;
+  const int n_pairs = T * top_k;
+  // The next kernel of the chain is scheduled once every CTA of this grid has executed this, i.e.
+  // once the whole grid is resident: it cannot take the room of a CTA the wait below needs.
+  pdl_trigger();
+  router_logits<1>(smem, x, 1, T, d, Wr, bias, bias_stride, E, EP, ep_shift, nullptr);  // waits on the kernels in front
+  // should this CTA's wait run out, the expert kernel behind must find an empty plan, not an old one
+  if (t == 0 && tid == 0) plan[0] = 0;
+  if (warp == 0) {
+    int my_id;
+    float my_gate;
+    router_pick(smem + ROUTER_DC + ROUTER_THREADS, E, top_k, renorm, lane, my_id, my_gate);
+    if (lane < top_k) {
+      ids[static_cast<size_t>(t) * top_k + lane] = my_id;
+      gates[static_cast<size_t>(t) * top_k + lane] = my_gate;
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && gridDim.x == 1) s_ok = 1;  // a single CTA has nobody to wait for
+  if (tid == 0 && gridDim.x > 1) {
+    __threadfence();
+    atomicAdd(&sync[0], 1u);
+    unsigned seen = 0, polls = 0;
+    int ok = 1;
+    for (;;) {
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(sync) : "memory");
+      if (seen >= static_cast<unsigned>(T + extra_arrivals)) break;
+      if (++polls > wait_limit) {
+        ok = 0;
+        break;
+      }
+    }
+    if (ok) {
+      if (atomicAdd(&sync[1], 1u) == static_cast<unsigned>(T) - 1u) {  // every CTA has passed its wait
+        sync[0] = 0;
+        sync[1] = 0;
+        __threadfence();
+      }
+    } else {
+      atomicOr(check_word, CHECK_WAIT_TIMEOUT);
+    }
+    s_ok = ok;
+  }
+  __syncthreads();
+  if (!s_ok) return;
+  for (int q = tid; q < n_pairs; q += ROUTER_THREADS) s_ids[q] = __ldcg(ids + q);
+  __syncthreads();
+  if (t == 0) {
+    // counts, offsets, plan (this CTA only); invalid ids cannot occur here: the picks lie in [0, E)
+    for (int ee = tid; ee <= E; ee += ROUTER_THREADS) s_off[ee] = 0;
+    __syncthreads();
+    for (int q = tid; q < n_pairs; q += ROUTER_THREADS) atomicAdd(&s_off[s_ids[q] + 1], 1);
+    __syncthreads();
+    if (tid == 0) {
+      for (int ee = 0; ee < E; ++ee) {
+        counts[ee] = s_off[ee + 1];
+        s_off[ee + 1] += s_off[ee];
+      }
+    }
+    __syncthreads();
+    for (int ee = tid; ee <= E; ee += ROUTER_THREADS) off[ee] = s_off[ee];
+    if (warp == 0) build_plan(plan, experts, s_off, E, 1, 0x7fffffff, lane);
+  }
+  for (int j = 0; j < top_k; ++j) {
+    const int p = t * top_k + j;
+    const int e = s_ids[p];
+    int before = 0;
+    for (int q = tid; q < n_pairs; q += ROUTER_THREADS) {
+      const int eq = s_ids[q];
+      before += eq < e || (eq == e && q < p);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+    __syncthreads();  // s_red of the previous pair has been read
+    if (lane == 0) s_red[0][warp] = before;
+    __syncthreads();
+    int slot = 0;
+#pragma unroll
+    for (int w = 0; w < ROUTER_THREADS / 32; ++w) slot += s_red[0][w];
+    if (tid == 0) {
+      perm[slot] = p;
+      slot_of_pair[p] = slot;
+    }
+    scatter_any(x + static_cast<size_t>(t) * d, xs_out, xsc, slot, d, experts[e].bits, fmt, check_word);
   }
 }
 
@@ -271,6 +400,35 @@ cudaError_t launch_router_topk(const void* x, int x_bf16, int T, int d, const fl
                         EP, sh, top_k, renorm, ids, gates, logits);
   }
   return cudaGetLastError();
+}
+
+bool route_permute_scatter_supported(const LayerDims& L, int T, int resident_ctas) {
+  return L.act_bf16 && T * L.top_k <= RPS_MAX_PAIRS && L.E <= EMOE_MAX_EXPERTS && 2 * T <= resident_ctas;
+}
+
+int route_permute_scatter_resident_ctas(int device) {
+  int per_sm = 0, sms = 0;
+  const size_t smem = sizeof(float) * (ROUTER_DC + ROUTER_THREADS + EMOE_MAX_EXPERTS);
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, route_permute_scatter_kernel, ROUTER_THREADS, smem) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return 0;
+  return per_sm * sms;
+}
+
+cudaError_t launch_route_permute_scatter(const LayerDims& L, const ExpertDev* experts, const void* x, int T, const float* Wr,
+                                         const float* bias, int bias_stride, int32_t* ids, float* gates, int32_t* counts,
+                                         int32_t* off, int32_t* perm, int32_t* slot_of_pair, int* plan, __nv_bfloat16* xs,
+                                         float* xsc, int fmt, unsigned* sync, unsigned wait_limit, int extra_arrivals,
+                                         int* check_word, cudaStream_t st) {
+  int EP = 1, sh = 0;
+  while (EP < L.E) {
+    EP <<= 1;
+    ++sh;
+  }
+  const size_t smem = sizeof(float) * (ROUTER_DC + ROUTER_THREADS + EP);
+  return launch_chain(route_permute_scatter_kernel, dim3(T), dim3(ROUTER_THREADS), smem, st,
+                      reinterpret_cast<const __nv_bfloat16*>(x), T, L.d_model, Wr, bias, bias_stride, L.E, EP, sh, L.top_k,
+                      static_cast<int>(L.gate_mode == EMOE_GATE_SOFTMAX_RENORM), ids, gates, experts, fmt, counts, off, perm,
+                      slot_of_pair, plan, check_word, xs, xsc, sync, wait_limit, extra_arrivals);
 }
 
 cudaError_t launch_permute(const int32_t* ids, int n_pairs, int E, int32_t* counts, int32_t* off, int32_t* perm,

@@ -138,6 +138,75 @@ def test_int8_streaming_path_keeps_the_bf16_range():
         assert rel_to_max(y, y_ref) <= 2e-3, (scale_x, std, rel_to_max(y, y_ref))
 
 
+ROUTE_CASES = [
+    # act, d, f, E, k, gate, T list (one context, calls back to back: the grid counters must come back to zero)
+    ("relu", 768, 3072, 32, 1, "softmax", [64, 1, 7, 64]),
+    ("swiglu", 512, 1024, 8, 2, "softmax_renorm", [4, 33, 1, 128]),
+    ("relu", 512, 512, 128, 1, "softmax", [96, 3]),
+]
+
+
+@pytest.mark.parametrize("act,d,f,E,k,gate,Ts", ROUTE_CASES)
+@pytest.mark.parametrize("path", [3, 6])
+def test_router_topk_permutation_and_scatter_in_one_launch(act, d, f, E, k, gate, Ts, path):
+    """Small batches take router, Top-K, permutation, scatter and plan in one launch (three launches
+    per layer with the expert kernel and the combine).  Its ids, gates, permutation and outputs are
+    bit-identical to those of the path with one launch per step, call after call on one context."""
+    shape = inputs.LayerShape(d, f, E, k, act, gate, 128, "f16", "bf16")
+    bits = ([8, 4, 2, 4] * E)[:E]
+    W = inputs.expert_set(41, 0, shape)
+    Wr = inputs.router_weight(41, 0, d, E, std=0.05)
+    with layer.MoELayer(shape, bits, max_tokens=max(Ts)) as moe:
+        B.emoe_set_ffn_path(moe.ctx, path)
+        moe.pack_from_host(W)
+        for i, T in enumerate(Ts):
+            x = inputs.activations(41, i, T, d, "bf16")
+            B.emoe_set_fused_projections(moe.ctx, True)
+            B.emoe_set_fused_routing(moe.ctx, True)
+            one = moe.forward(x, Wr)
+            assert B.emoe_kernels_last_forward(moe.ctx) == 3
+            B.emoe_set_fused_routing(moe.ctx, False)
+            chain = moe.forward(x, Wr)
+            assert B.emoe_kernels_last_forward(moe.ctx) == 4
+            B.emoe_set_fused_projections(moe.ctx, False)
+            many = moe.forward(x, Wr)
+            assert B.emoe_kernels_last_forward(moe.ctx) >= 6
+            for a, b in zip(one, chain):
+                assert np.array_equal(a, b)
+            for a, b in zip(one, many):
+                assert np.array_equal(a, b)
+            ids_ref, _, logits_ref = oracle.route(x, Wr, None, k, gate == "softmax_renorm")
+            check_ids(one[1], logits_ref, k)
+            _, _, perm_ref = oracle.permute(one[1], E)
+            assert np.array_equal(one[3], perm_ref)
+
+
+def test_grid_wide_wait_of_the_one_launch_routing_runs_out_without_a_hang():
+    """The CTAs are told to wait for one more arrival than the grid has, with a short limit: every
+    wait gives up, every kernel still returns, the status call says "timeout", and the next call on
+    the context is right again."""
+    shape = inputs.LayerShape(512, 1024, 8, 1, "relu", "softmax", 128, "f16", "bf16")
+    bits, T = [8, 4, 2, 4] * 2, 128
+    W = inputs.expert_set(43, 0, shape)
+    x = inputs.activations(43, 0, T, shape.d_model, "bf16")
+    Wr = inputs.router_weight(43, 0, shape.d_model, shape.n_experts, std=0.05)
+    with layer.MoELayer(shape, bits, max_tokens=T) as moe:
+        B.emoe_set_ffn_path(moe.ctx, 3)
+        moe.pack_from_host(W)
+        good = moe.forward(x, Wr)
+        B.emoe_set_fused_routing(moe.ctx, True)
+        B.emoe_set_wait_limit(moe.ctx, 2000)
+        B.emoe_debug_expect_extra_completions(moe.ctx, 1)
+        with pytest.raises(B.EmoeError) as ei:
+            moe.forward(x, Wr)
+        assert ei.value.status == B.ERR_TIMEOUT
+        B.emoe_set_wait_limit(moe.ctx, 0)
+        B.emoe_debug_expect_extra_completions(moe.ctx, 0)
+        again = moe.forward(x, Wr)
+        for a, b in zip(good, again):
+            assert np.array_equal(a, b)
+
+
 def test_bounded_wait_inside_the_kernel_runs_out_and_the_context_stays_usable():
     """Failure detection without a fault: the second projection is told to expect one more
     completion of the first than will ever be counted, with a short wait limit.  The wait must give
