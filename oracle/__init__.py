@@ -62,16 +62,18 @@ def round_bf16(v: float) -> float:
     return float(_load().orc_round_bf16(ctypes.c_double(v)))
 
 
-def quantize(W: np.ndarray, bits: int, group: int, scale_dtype: str) -> Tuple[np.ndarray, np.ndarray]:
-    """Codes q[N][K] (int8) and stored scales [N][K/G] (fp32 values)."""
+def quantize(W: np.ndarray, bits: int, group: int, scale_dtype: str, full_range: bool = False) -> Tuple[np.ndarray, np.ndarray]:
+    """Codes q[N][K] (int8) and stored scales [N][K/G] (fp32 values).  full_range: the reading of
+    Section 3.2's "range expressible by the bitwidth" that uses every code of the field
+    (-2^(b-1) .. 2^(b-1)-1, scale = max-abs / 2^(b-1)) instead of the symmetric one."""
     W = _c(W, np.float32)
     N, K = W.shape
     G = group if group > 0 else K
     q = np.empty((N, K), dtype=np.int8)
     s = np.empty((N, K // G), dtype=np.float32)
-    rc = _load().orc_quantize(_p(W), N, K, bits, group, int(scale_dtype == "f16"), _p(q), _p(s))
+    rc = _load().orc_quantize_mode(_p(W), N, K, bits, group, int(scale_dtype == "f16"), int(full_range), _p(q), _p(s))
     if rc != 0:
-        raise ValueError(f"orc_quantize failed ({rc})")
+        raise ValueError(f"orc_quantize_mode failed ({rc})")
     return q, s
 
 
@@ -106,21 +108,21 @@ def dequantize(packed: np.ndarray, scales: np.ndarray, K: int, bits: int, group:
     return Wt
 
 
-def pack_expert(W: np.ndarray, bits: int, group: int, scale_dtype: str) -> Tuple[np.ndarray, np.ndarray]:
+def pack_expert(W: np.ndarray, bits: int, group: int, scale_dtype: str, full_range: bool = False) -> Tuple[np.ndarray, np.ndarray]:
     """quantise + pack one matrix: (packed bytes [N][K*b/8], stored scales fp32 [N][K/G])."""
-    q, s = quantize(W, bits, group, scale_dtype)
+    q, s = quantize(W, bits, group, scale_dtype, full_range)
     return pack(q, bits), s
 
 
 def requantize(packed: np.ndarray, scales: np.ndarray, K: int, bits_in: int, bits_out: int, group: int,
-               scale_dtype: str) -> Tuple[np.ndarray, np.ndarray]:
+               scale_dtype: str, full_range: bool = False) -> Tuple[np.ndarray, np.ndarray]:
     """An expert matrix stored at `bits_in` moved to `bits_out` without the original weights
     (paper Section 3.2: the bitwidth selection lowers the width of chosen experts): decompress
     to FP32 as the paper does (w~ = q * s, rounded once to fp32; exact with fp16 scales, which
     have 11 significant bits against the codes' 8), then the same channel-wise linear
     quantisation as for an fp32 matrix.  Returns (packed bytes, stored scales)."""
     Wt = dequantize(packed, scales, K, bits_in, group)
-    return pack_expert(Wt.astype(np.float32), bits_out, group, scale_dtype)
+    return pack_expert(Wt.astype(np.float32), bits_out, group, scale_dtype, full_range)
 
 
 def scales_storage(scales: np.ndarray, scale_dtype: str) -> np.ndarray:

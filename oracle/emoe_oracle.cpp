@@ -94,20 +94,28 @@ extern "C" {
 // group == 0: one scale per row; otherwise one scale per `group` consecutive inputs.
 // q_out[N][K] receives the integer codes, scales_out[N][K/G] the scales *as stored*
 // (after the optional fp16 rounding), widened to fp32.
+//
+// full_range == 0 (the library's default reading of "the range expressible by the bitwidth"):
+//   symmetric codes, -qmax .. qmax with qmax = 2^(b-1) - 1, scale = max-abs / qmax.
+// full_range != 0 (the other reading): every code of the two's-complement field is used,
+//   -2^(b-1) .. 2^(b-1) - 1, scale = max-abs / 2^(b-1); a weight equal to +max-abs is clamped to
+//   the largest positive code.  At 2 bits this gives four levels (-2, -1, 0, 1) instead of three.
 // ---------------------------------------------------------------------------------------
-int orc_quantize(const float* W, int N, int K, int bits, int group, int scale_is_f16,
-                 int8_t* q_out, float* scales_out) {
+int orc_quantize_mode(const float* W, int N, int K, int bits, int group, int scale_is_f16, int full_range,
+                      int8_t* q_out, float* scales_out) {
   if (bits != 2 && bits != 4 && bits != 8) return -1;
   const int G = group > 0 ? group : K;
   if (K % G != 0) return -2;
   const int ngroups = K / G;
   const int qmax = qmax_of(bits);
+  const int qmin = full_range ? -(1 << (bits - 1)) : -qmax;
+  const int range = full_range ? (1 << (bits - 1)) : qmax;  // max-abs is divided by this
   for (int n = 0; n < N; ++n) {
     for (int g = 0; g < ngroups; ++g) {
       const float* w = W + static_cast<size_t>(n) * K + static_cast<size_t>(g) * G;
       float amax = 0.0f;
       for (int k = 0; k < G; ++k) amax = std::max(amax, std::fabs(w[k]));
-      float s = amax / static_cast<float>(qmax);
+      float s = amax / static_cast<float>(range);
       if (scale_is_f16) s = round_to_f16(s);
       scales_out[static_cast<size_t>(n) * ngroups + g] = s;
       int8_t* q = q_out + static_cast<size_t>(n) * K + static_cast<size_t>(g) * G;
@@ -115,7 +123,7 @@ int orc_quantize(const float* W, int N, int K, int bits, int group, int scale_is
         int code = 0;
         if (s != 0.0f) {
           const float r = std::nearbyintf(w[k] / s);  // round half to even
-          code = static_cast<int>(std::min(std::max(r, static_cast<float>(-qmax)),
+          code = static_cast<int>(std::min(std::max(r, static_cast<float>(qmin)),
                                            static_cast<float>(qmax)));
         }
         q[k] = static_cast<int8_t>(code);
@@ -123,6 +131,11 @@ int orc_quantize(const float* W, int N, int K, int bits, int group, int scale_is
     }
   }
   return 0;
+}
+
+int orc_quantize(const float* W, int N, int K, int bits, int group, int scale_is_f16, int8_t* q_out,
+                 float* scales_out) {
+  return orc_quantize_mode(W, N, K, bits, group, scale_is_f16, 0, q_out, scales_out);
 }
 
 // Storage format: element k of row n is a b-bit two's-complement field at bit offset

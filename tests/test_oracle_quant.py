@@ -204,3 +204,98 @@ def test_requantize_closed_forms(bits_in, bits_out, sdt):
     assert np.all(np.abs(q2[at_max & (np.repeat(amax, G, axis=1) > 0)]) == qmax)
     slack = np.repeat(amax, G, axis=1) * 2.0 ** -11 if sdt == "f16" else 0.0
     assert np.all(np.abs(Wt2 - Wt) <= np.repeat(scales2.astype(np.float64), G, axis=1) / 2 + slack + 1e-12)
+
+
+# ---- the full-range reading of the code range (Section 3.2) -----------------------------------
+FULL_RANGE_GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "full_range_rows.txt")
+
+
+def _full_range_rows(kind):
+    rows = []
+    with open(FULL_RANGE_GOLDEN) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            parts = [p.strip() for p in line.split("|")]
+            if parts[0] == kind:
+                rows.append(parts[1:])
+    return rows
+
+
+@pytest.mark.parametrize("row", _full_range_rows("pack"), ids=lambda r: f"int{r[0]}_g{r[1]}_{r[2]}")
+def test_full_range_hand_computed_rows(row):
+    bits, group, sdt = int(row[0]), int(row[1]), row[2]
+    w = np.array(row[3].split(), dtype=np.float64).astype(np.float32)
+    q_exp = np.array(row[4].split(), dtype=np.int64)
+    s_exp = np.array(row[5].split(), dtype=np.float64)
+    bytes_exp = np.array([int(v, 16) for v in row[6].split()], dtype=np.uint8)
+    q, s = oracle.quantize(w[None, :], bits, group, sdt, full_range=True)
+    assert np.array_equal(q[0].astype(np.int64), q_exp)
+    assert np.array_equal(s[0].astype(np.float64), s_exp)
+    packed, s2 = oracle.pack_expert(w[None, :], bits, group, sdt, full_range=True)
+    assert np.array_equal(packed[0], bytes_exp) and np.array_equal(s2, s)
+    assert np.array_equal(oracle.unpack(packed, w.size, bits)[0].astype(np.int64), q_exp)
+
+
+@pytest.mark.parametrize("row", _full_range_rows("requant"), ids=lambda r: f"int{r[0]}_to_int{r[1]}")
+def test_full_range_requantize_hand_computed_rows(row):
+    bi, bo, group, sdt = int(row[0]), int(row[1]), int(row[2]), row[3]
+    b_in = np.array([int(v, 16) for v in row[4].split()], dtype=np.uint8)
+    s_in = np.array(row[5].split(), dtype=np.float64).astype(np.float32)
+    q_exp = np.array(row[6].split(), dtype=np.int64)
+    s_exp = np.array(row[7].split(), dtype=np.float64)
+    b_exp = np.array([int(v, 16) for v in row[8].split()], dtype=np.uint8)
+    K = b_in.size * 8 // bi
+    packed, scales = oracle.requantize(b_in[None, :], s_in[None, :], K, bi, bo, group, sdt, full_range=True)
+    assert np.array_equal(oracle.unpack(packed, K, bo)[0].astype(np.int64), q_exp)
+    assert np.array_equal(scales[0].astype(np.float64), s_exp)
+    assert np.array_equal(packed[0], b_exp)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("group", [0, 32])
+def test_full_range_properties(bits, group):
+    """What the definition fixes at any size: codes lie in [-2^(b-1), 2^(b-1)-1]; the scale is
+    max-abs / 2^(b-1); a channel's most negative weight of magnitude max-abs takes the extra code;
+    the reconstruction error of a weight that is not clamped is at most half a step; and a matrix
+    whose weights are whole multiples of the step comes back exactly except +max-abs."""
+    rng = np.random.default_rng(11 + bits)
+    W = (rng.standard_normal((16, 128)) * 0.05).astype(np.float32)
+    W[5, :] = 0.0
+    half = 1 << (bits - 1)
+    q, s = oracle.quantize(W, bits, group, "f32", full_range=True)
+    G = group or 128
+    assert q.min() >= -half and q.max() <= half - 1
+    amax = np.abs(W.reshape(16, 128 // G, G)).max(axis=2)
+    assert np.array_equal(s, (amax / np.float32(half)).astype(np.float32))
+    step = np.repeat(s, G, axis=1).astype(np.float64)
+    Wt = q.astype(np.float64) * step
+    clamped = (W.astype(np.float64) > (half - 1 + 0.5) * step)
+    err = np.abs(Wt - W.astype(np.float64))
+    assert np.all(err[~clamped] <= 0.5 * step[~clamped] * (1 + 1e-6) + 1e-12)
+    # the negative extreme of a group maps to -2^(b-1) exactly
+    Wg = W.reshape(16, 128 // G, G)
+    qg = q.reshape(16, 128 // G, G)
+    for n in range(16):
+        for g in range(128 // G):
+            k = int(np.argmax(np.abs(Wg[n, g])))
+            if Wg[n, g, k] < 0:
+                assert qg[n, g, k] == -half
+    # symmetric and full-range agree on what they share: same codes wherever the symmetric scale
+    # is used with the symmetric clamp (sanity: the default did not change)
+    q0, s0 = oracle.quantize(W, bits, group, "f32")
+    assert q0.min() >= -(half - 1) and np.array_equal(s0, (amax / np.float32(half - 1)).astype(np.float32))
+
+
+def test_full_range_int2_has_four_levels_and_lower_error_on_gaussian_weights():
+    """Ternary INT2 (the default reading) maps most of a Gaussian group to 0; the four-level reading
+    halves the step.  On seeded Gaussian weights with groups of 128 its mean squared error is lower."""
+    rng = np.random.default_rng(3)
+    W = (rng.standard_normal((64, 512)) * 0.02).astype(np.float32)
+    q3, s3 = oracle.quantize(W, 2, 128, "f16")
+    q4, s4 = oracle.quantize(W, 2, 128, "f16", full_range=True)
+    assert set(np.unique(q3)) == {-1, 0, 1} and set(np.unique(q4)) == {-2, -1, 0, 1}
+    e3 = np.mean((q3 * np.repeat(s3, 128, axis=1) - W) ** 2)
+    e4 = np.mean((q4 * np.repeat(s4, 128, axis=1) - W) ** 2)
+    assert e4 < e3
