@@ -67,6 +67,9 @@ extern "C" {
 #define EMOE_GATE_SOFTMAX 0        /* gate = softmax probability of the pick over all experts */
 #define EMOE_GATE_SOFTMAX_RENORM 1 /* gate = that probability / sum over the token's K picks */
 
+#define EMOE_RANGE_SYMMETRIC 0 /* codes -qmax .. qmax, qmax = 2^(b-1) - 1 (the storage format above) */
+#define EMOE_RANGE_FULL 1      /* every code of the field: -2^(b-1) .. 2^(b-1) - 1, scale = amax / 2^(b-1) */
+
 #define EMOE_MAX_EXPERTS 256
 #define EMOE_MAX_TOP_K 8
 
@@ -154,6 +157,20 @@ int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int 
 int emoe_requantize_expert(emoe_ctx* ctx, const void* in_packed, const void* in_scales, int N, int K, int bits_in,
                            int bits_out, int group, int scale_dtype, void* out_packed, void* out_scales,
                            void* stream);
+
+/* The same two calls with the reading of "the range expressible by the bitwidth" (Section 3.2)
+ * as an argument.  EMOE_RANGE_SYMMETRIC is the storage format at the top of this file (what the
+ * calls above use).  EMOE_RANGE_FULL uses every code of the two's-complement field:
+ *       s32 = amax / 2^(b-1),  q = clamp(round_half_even(w / s), -2^(b-1), 2^(b-1) - 1),
+ * so that INT2 has four levels (-2, -1, 0, 1) instead of three; a weight equal to +amax is
+ * clamped to the largest positive code.  Storage layout, scale channel and every forward call are
+ * unchanged: the expert kernels decode whole two's-complement fields.  Everything else as above;
+ * an unknown range_mode returns EMOE_ERR_UNSUPPORTED. */
+int emoe_pack_expert_mode(emoe_ctx* ctx, const float* W, int N, int K, int bits, int group, int scale_dtype,
+                          int range_mode, void* out_packed, void* out_scales, void* stream);
+int emoe_requantize_expert_mode(emoe_ctx* ctx, const void* in_packed, const void* in_scales, int N, int K, int bits_in,
+                                int bits_out, int group, int scale_dtype, int range_mode, void* out_packed,
+                                void* out_scales, void* stream);
 
 /* ---- Sections 1, 2.1: router and Top-K gating ----------------------------------------- */
 

@@ -28,10 +28,12 @@ EVICT_FORWARD, EVICT_PRINTED, EVICT_LRU, EVICT_LFU, EVICT_FIFO = 0, 1, 2, 3, 4
 DTYPE_F32, DTYPE_F16, DTYPE_BF16 = 0, 1, 2
 ACT_RELU, ACT_SWIGLU = 0, 1
 GATE_SOFTMAX, GATE_SOFTMAX_RENORM = 0, 1
+RANGE_SYMMETRIC, RANGE_FULL = 0, 1
 
 EXPORTS = (
     "emoe_create", "emoe_destroy", "emoe_workspace_bytes", "emoe_last_cuda_error", "emoe_device_status",
     "emoe_status_string", "emoe_packed_bytes", "emoe_scales_bytes", "emoe_pack_expert", "emoe_requantize_expert",
+    "emoe_pack_expert_mode", "emoe_requantize_expert_mode",
     "emoe_router_topk",
     "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
     "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_static_device_status", "emoe_set_dependent_launch",
@@ -96,6 +98,8 @@ def lib() -> ctypes.CDLL:
         L.emoe_scales_bytes.argtypes = [i32, i32, i32, i32]
         L.emoe_pack_expert.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
         L.emoe_requantize_expert.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.emoe_pack_expert_mode.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.emoe_requantize_expert_mode.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp]
         L.emoe_router_topk.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
         L.emoe_permute.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp]
         L.emoe_moe_forward.argtypes = [vp, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp, i32,
@@ -182,6 +186,19 @@ def emoe_scales_bytes(N: int, K: int, group: int, scale_dtype: int) -> int:
 def emoe_pack_expert(ctx, W_ptr, N, K, bits, group, scale_dtype, out_packed_ptr, out_scales_ptr, stream=0) -> None:
     _check(lib().emoe_pack_expert(ctx, W_ptr, N, K, bits, group, scale_dtype, out_packed_ptr, out_scales_ptr, stream),
            "emoe_pack_expert")
+
+
+def emoe_pack_expert_mode(ctx, W_ptr, N, K, bits, group, scale_dtype, range_mode, out_packed_ptr, out_scales_ptr,
+                          stream=0) -> None:
+    _check(lib().emoe_pack_expert_mode(ctx, W_ptr, N, K, bits, group, scale_dtype, range_mode, out_packed_ptr,
+                                       out_scales_ptr, stream), "emoe_pack_expert_mode")
+
+
+def emoe_requantize_expert_mode(ctx, in_packed_ptr, in_scales_ptr, N, K, bits_in, bits_out, group, scale_dtype,
+                                range_mode, out_packed_ptr, out_scales_ptr, stream=0) -> None:
+    _check(lib().emoe_requantize_expert_mode(ctx, in_packed_ptr, in_scales_ptr, N, K, bits_in, bits_out, group,
+                                             scale_dtype, range_mode, out_packed_ptr, out_scales_ptr, stream),
+           "emoe_requantize_expert_mode")
 
 
 def emoe_requantize_expert(ctx, in_packed_ptr, in_scales_ptr, N, K, bits_in, bits_out, group, scale_dtype,

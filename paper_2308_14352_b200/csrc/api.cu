@@ -568,6 +568,12 @@ size_t emoe_scales_bytes(int N, int K, int group, int scale_dtype) {
 
 int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int group, int scale_dtype,
                      void* out_packed, void* out_scales, void* stream) {
+  return emoe_pack_expert_mode(ctx, W, N, K, bits, group, scale_dtype, EMOE_RANGE_SYMMETRIC, out_packed, out_scales, stream);
+}
+
+int emoe_pack_expert_mode(emoe_ctx* ctx, const float* W, int N, int K, int bits, int group, int scale_dtype,
+                          int range_mode, void* out_packed, void* out_scales, void* stream) {
+  if (range_mode != EMOE_RANGE_SYMMETRIC && range_mode != EMOE_RANGE_FULL) return EMOE_ERR_UNSUPPORTED;
   if (!ctx || !W || !out_packed || !out_scales || N <= 0 || K <= 0 || group < 0) return EMOE_ERR_INVALID_ARG;
   if (bits != 2 && bits != 4 && bits != 8) return EMOE_ERR_UNSUPPORTED;
   if (scale_dtype != EMOE_DTYPE_F32 && scale_dtype != EMOE_DTYPE_F16) return EMOE_ERR_UNSUPPORTED;
@@ -576,7 +582,7 @@ int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int 
   if (G % 4 != 0) return EMOE_ERR_UNSUPPORTED;
   if (!aligned(W, 16) || !aligned(out_packed, 16) || !aligned(out_scales, 4)) return EMOE_ERR_ALIGNMENT;
   EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
-  EMOE_CUDA(ctx, launch_pack(W, N, K, bits, group, scale_dtype == EMOE_DTYPE_F16, static_cast<uint8_t*>(out_packed),
+  EMOE_CUDA(ctx, launch_pack(W, N, K, bits, group, scale_dtype == EMOE_DTYPE_F16, range_mode == EMOE_RANGE_FULL, static_cast<uint8_t*>(out_packed),
                              out_scales, static_cast<cudaStream_t>(stream)));
   return EMOE_OK;
 }
@@ -584,6 +590,14 @@ int emoe_pack_expert(emoe_ctx* ctx, const float* W, int N, int K, int bits, int 
 int emoe_requantize_expert(emoe_ctx* ctx, const void* in_packed, const void* in_scales, int N, int K, int bits_in,
                            int bits_out, int group, int scale_dtype, void* out_packed, void* out_scales,
                            void* stream) {
+  return emoe_requantize_expert_mode(ctx, in_packed, in_scales, N, K, bits_in, bits_out, group, scale_dtype,
+                                     EMOE_RANGE_SYMMETRIC, out_packed, out_scales, stream);
+}
+
+int emoe_requantize_expert_mode(emoe_ctx* ctx, const void* in_packed, const void* in_scales, int N, int K, int bits_in,
+                                int bits_out, int group, int scale_dtype, int range_mode, void* out_packed,
+                                void* out_scales, void* stream) {
+  if (range_mode != EMOE_RANGE_SYMMETRIC && range_mode != EMOE_RANGE_FULL) return EMOE_ERR_UNSUPPORTED;
   if (!ctx || !in_packed || !in_scales || !out_packed || !out_scales || N <= 0 || K <= 0 || group < 0)
     return EMOE_ERR_INVALID_ARG;
   if (bits_in != 2 && bits_in != 4 && bits_in != 8) return EMOE_ERR_UNSUPPORTED;
@@ -597,7 +611,7 @@ int emoe_requantize_expert(emoe_ctx* ctx, const void* in_packed, const void* in_
     return EMOE_ERR_ALIGNMENT;
   EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
   EMOE_CUDA(ctx, launch_requant(static_cast<const uint8_t*>(in_packed), in_scales, N, K, bits_in, bits_out, group,
-                                scale_dtype == EMOE_DTYPE_F16, static_cast<uint8_t*>(out_packed), out_scales,
+                                scale_dtype == EMOE_DTYPE_F16, range_mode == EMOE_RANGE_FULL, static_cast<uint8_t*>(out_packed), out_scales,
                                 static_cast<cudaStream_t>(stream)));
   return EMOE_OK;
 }

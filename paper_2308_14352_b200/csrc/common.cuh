@@ -78,10 +78,10 @@ struct ExpertCache;
 void cache_destroy(ExpertCache* c);
 
 // ---- launchers (each enqueues on `st` and returns the launch error) ---------------------
-cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int scale_f16, uint8_t* packed,
+cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int scale_f16, int full_range, uint8_t* packed,
                         void* scales, cudaStream_t st);
 cudaError_t launch_requant(const uint8_t* in_packed, const void* in_scales, int N, int K, int bits_in, int bits_out,
-                           int group, int scale_f16, uint8_t* packed, void* scales, cudaStream_t st);
+                           int group, int scale_f16, int full_range, uint8_t* packed, void* scales, cudaStream_t st);
 
 cudaError_t launch_router_topk(const void* x, int x_bf16, int T, int d, const float* Wr, const float* bias,
                                int bias_stride, int E, int top_k, int renorm, int32_t* ids, float* gates,

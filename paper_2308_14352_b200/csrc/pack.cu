@@ -5,9 +5,22 @@
 // experts; the weight is decompressed in registers, w~ = q * s rounded once to fp32, and the fp32
 // original is not needed).  One warp owns one (output channel, group) unit at a time: it finds
 // the unit's max-abs, derives the scale, then quantises and packs, each lane emitting the codes
-// of 4 consecutive weights.  Groups of 128 weights, the usual case, are taken UNITS at a time so
-// that a warp has several independent loads in flight.  HBM-bound by definition: 4 (or
+// of 4 consecutive weights.  Groups of 128 weights, the usual case, take another route: the
+// matrix is dense, so its units follow each other in memory; a warp takes four consecutive units
+// at a time, eight lanes per unit and sixteen consecutive weights per lane (64 bytes read, 4 / 8 /
+// 16 bytes written by one store), two such steps in flight.  HBM-bound by definition: 4 (or
 // b_in / 8) bytes read and b_out / 8 bytes written per weight.
+//
+// Two readings of "the range expressible by the bitwidth" (Section 3.2): symmetric codes
+// -qmax .. qmax with qmax = 2^(b-1) - 1 and scale = max-abs / qmax (the default), or every code of
+// the field, -2^(b-1) .. 2^(b-1) - 1, with scale = max-abs / 2^(b-1) ("full range": four levels at
+// 2 bits instead of three).
+//
+// The quotient w / s is an IEEE division in the definition.  The kernels multiply by 1 / s
+// instead and keep the result when it cannot differ from the definition's: the product lies
+// within 1.8e-7 relative of the rounded quotient, so unless it comes within 1e-4 of a half-integer
+// (or leaves the range where that bound holds) both round to the same integer; otherwise the
+// division is carried out.  Bit-exact with the definition either way.
 #include "common.cuh"
 
 namespace emoe {
@@ -29,6 +42,18 @@ struct SourceF32 {
   int K;
   __device__ __forceinline__ float4 load4(int n, int k, long long) const {
     return *reinterpret_cast<const float4*>(W + static_cast<size_t>(n) * K + k);
+  }
+  // 16 consecutive weights from linear index w0 (a multiple of 16) of the dense matrix
+  __device__ __forceinline__ void load16(long long w0, long long, float (&v)[16]) const {
+    const float4* p = reinterpret_cast<const float4*>(W + w0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 f = p[i];
+      v[4 * i] = f.x;
+      v[4 * i + 1] = f.y;
+      v[4 * i + 2] = f.z;
+      v[4 * i + 3] = f.w;
+    }
   }
 };
 template <int BIN>
@@ -52,37 +77,75 @@ struct SourcePacked {
     }
     return make_float4(v[0], v[1], v[2], v[3]);
   }
+  __device__ __forceinline__ void load16(long long w0, long long unit, float (&v)[16]) const {
+    uint32_t w[4];  // the 16 codes, low fields first
+    const uint8_t* p = packed + w0 * BIN / 8;
+    if (BIN == 8) {
+      const uint4 q = *reinterpret_cast<const uint4*>(p);
+      w[0] = q.x, w[1] = q.y, w[2] = q.z, w[3] = q.w;
+    } else if (BIN == 4) {
+      const uint2 q = *reinterpret_cast<const uint2*>(p);
+      w[0] = q.x, w[1] = q.y;
+    } else {
+      w[0] = *reinterpret_cast<const uint32_t*>(p);
+    }
+    const float s = scale_f16 ? __half2float(reinterpret_cast<const __half*>(scales)[unit])
+                              : reinterpret_cast<const float*>(scales)[unit];
+    constexpr int PER_WORD = 32 / BIN;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      const uint32_t word = w[c / PER_WORD];
+      const int q = static_cast<int>(word << (32 - BIN * (c % PER_WORD + 1))) >> (32 - BIN);
+      v[c] = __fmul_rn(static_cast<float>(q), s);
+    }
+  }
 };
 
 // scale = max-abs / representable range, IEEE division; stored in the scale channel's type
-__device__ __forceinline__ float store_scale(float amax, float qmax, int scale_f16, void* scales, long long unit, int lane) {
-  float s = __fdiv_rn(amax, qmax);
+__device__ __forceinline__ float store_scale(float amax, float range, int scale_f16, void* scales, long long unit, bool writer) {
+  float s = __fdiv_rn(amax, range);
   if (scale_f16) {
     const __half h = __float2half_rn(s);
     s = __half2float(h);
-    if (lane == 0) reinterpret_cast<__half*>(scales)[unit] = h;
-  } else if (lane == 0) {
+    if (writer) reinterpret_cast<__half*>(scales)[unit] = h;
+  } else if (writer) {
     reinterpret_cast<float*>(scales)[unit] = s;
   }
   return s;
 }
 
+// What the codes of one unit are made with: the stored scale, its reciprocal for the fast
+// quotient (NaN where the error bound of the product does not hold: the division then decides
+// every code), and the clamp.
+struct QuantParams {
+  float s, r, qlo, qhi;
+};
+__device__ __forceinline__ QuantParams quant_params(float s, float qlo, float qhi) {
+  QuantParams p;
+  p.s = s;
+  p.r = (s > 1e-30f && s < 1e30f) ? __frcp_rn(s) : __int_as_float(0x7fc00000);
+  p.qlo = qlo;
+  p.qhi = qhi;
+  return p;
+}
+// one code: round-half-even of the fp32 quotient e / s, clamped (0 when the scale is 0)
+__device__ __forceinline__ int quantise1(float e, const QuantParams& p) {
+  const float t = e * p.r;
+  float q = rintf(t);
+  const float d = fabsf(fabsf(t - q) - 0.5f);
+  if (!(d >= 1e-4f) || !(fabsf(t) < 200.0f)) q = rintf(__fdiv_rn(e, p.s));
+  q = fminf(fmaxf(q, p.qlo), p.qhi);
+  return p.s != 0.0f ? static_cast<int>(q) : 0;
+}
+
 // codes of 4 weights: round half to even on the quotient by the stored scale, clamp, pack
 template <int BITS>
-__device__ __forceinline__ uint32_t quantise4(const float4& v, float s, float qmax) {
+__device__ __forceinline__ uint32_t quantise4(const float4& v, const QuantParams& p) {
   constexpr int MASK = (1 << BITS) - 1;
   const float e[4] = {v.x, v.y, v.z, v.w};
   uint32_t word = 0;
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    int q = 0;
-    if (s != 0.0f) {
-      float r = rintf(__fdiv_rn(e[c], s));
-      r = fminf(fmaxf(r, -qmax), qmax);
-      q = static_cast<int>(r);
-    }
-    word |= static_cast<uint32_t>(q & MASK) << (BITS * c);
-  }
+  for (int c = 0; c < 4; ++c) word |= static_cast<uint32_t>(quantise1(e[c], p) & MASK) << (BITS * c);
   return word;
 }
 
@@ -90,13 +153,17 @@ __device__ __forceinline__ float amax4(const float4& v) {
   return fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
 }
 
-constexpr int UNITS = 4;  // 128-weight units a warp works on at once
+constexpr int STEPS = 2;  // four-unit steps a warp has in flight (groups of 128)
 
 template <int BITS, typename Source>
 __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, int K, int G, int ngroups, int scale_f16,
-                                                       uint8_t* __restrict__ packed, void* __restrict__ scales) {
+                                                       int full_range, uint8_t* __restrict__ packed,
+                                                       void* __restrict__ scales) {
   typedef typename PackWord<BITS>::type word_t;
-  const float qmax = static_cast<float>((1 << (BITS - 1)) - 1);
+  constexpr int MASK = (1 << BITS) - 1;
+  const float qhi = static_cast<float>((1 << (BITS - 1)) - 1);
+  const float qlo = full_range ? -static_cast<float>(1 << (BITS - 1)) : -qhi;
+  const float range = full_range ? static_cast<float>(1 << (BITS - 1)) : qhi;  // max-abs is divided by this
   const int lane = threadIdx.x & 31;
   const long long n_units = static_cast<long long>(N) * ngroups;
   const long long warps = (static_cast<long long>(gridDim.x) * blockDim.x) >> 5;
@@ -104,30 +171,44 @@ __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, 
   const size_t row_bytes = static_cast<size_t>(K) * BITS / 8;
 
   if (G == 128) {
-    // one step per unit: the unit's weights stay in registers, UNITS units in flight
-    for (long long u0 = warp * UNITS; u0 < n_units; u0 += warps * UNITS) {
-      float4 v[UNITS];
-      float amax[UNITS];
+    // K is a whole number of units, so unit u holds the weights 128 u .. 128 u + 127 of the dense
+    // matrix and the bytes 16 b u .. of the packed one, whatever its row
+    const long long n_steps = (n_units + 3) >> 2;
+    for (long long st0 = warp * STEPS; st0 < n_steps; st0 += warps * STEPS) {
+      float v[STEPS][16];
+      float amax[STEPS];
 #pragma unroll
-      for (int u = 0; u < UNITS; ++u) {
-        const long long unit = u0 + u;
-        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (unit < n_units)
-          v[u] = src.load4(static_cast<int>(unit / ngroups), static_cast<int>(unit % ngroups) * 128 + lane * 4, unit);
-        amax[u] = amax4(v[u]);
+      for (int u = 0; u < STEPS; ++u) {
+        const long long unit = (st0 + u) * 4 + (lane >> 3);
+        if (unit < n_units) {
+          src.load16(unit * 128 + (lane & 7) * 16, unit, v[u]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) v[u][c] = 0.0f;
+        }
+        float m = 0.0f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) m = fmaxf(m, fabsf(v[u][c]));
+        amax[u] = m;
       }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1)
+      for (int o = 4; o > 0; o >>= 1)
 #pragma unroll
-        for (int u = 0; u < UNITS; ++u) amax[u] = fmaxf(amax[u], __shfl_xor_sync(0xffffffffu, amax[u], o));
+        for (int u = 0; u < STEPS; ++u) amax[u] = fmaxf(amax[u], __shfl_xor_sync(0xffffffffu, amax[u], o));
 #pragma unroll
-      for (int u = 0; u < UNITS; ++u) {
-        const long long unit = u0 + u;
-        if (unit >= n_units) break;
-        const float s = store_scale(amax[u], qmax, scale_f16, scales, unit, lane);
-        word_t* out = reinterpret_cast<word_t*>(packed + static_cast<size_t>(unit / ngroups) * row_bytes +
-                                                static_cast<size_t>(unit % ngroups) * 128 * BITS / 8);
-        out[lane] = static_cast<word_t>(quantise4<BITS>(v[u], s, qmax));
+      for (int u = 0; u < STEPS; ++u) {
+        const long long unit = (st0 + u) * 4 + (lane >> 3);
+        if (unit >= n_units) continue;
+        const QuantParams p = quant_params(store_scale(amax[u], range, scale_f16, scales, unit, (lane & 7) == 0), qlo, qhi);
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        constexpr int PER_WORD = 32 / BITS;
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          w[c / PER_WORD] |= static_cast<uint32_t>(quantise1(v[u][c], p) & MASK) << (BITS * (c % PER_WORD));
+        uint8_t* out = packed + (unit * 128 + (lane & 7) * 16) * BITS / 8;
+        if (BITS == 8) *reinterpret_cast<uint4*>(out) = make_uint4(w[0], w[1], w[2], w[3]);
+        else if (BITS == 4) *reinterpret_cast<uint2*>(out) = make_uint2(w[0], w[1]);
+        else *reinterpret_cast<uint32_t*>(out) = w[0];
       }
     }
     return;
@@ -147,22 +228,22 @@ __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, 
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    const float s = store_scale(amax, qmax, scale_f16, scales, unit, lane);
+    const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, lane == 0), qlo, qhi);
     word_t* out = reinterpret_cast<word_t*>(packed + static_cast<size_t>(n) * row_bytes + static_cast<size_t>(g) * G * BITS / 8);
     for (int i = lane * 4; i < G; i += 128) {
       const float4 v = i < 128 ? first : src.load4(n, k_first + i, unit);  // later steps come from L1/L2
-      out[i >> 2] = static_cast<word_t>(quantise4<BITS>(v, s, qmax));
+      out[i >> 2] = static_cast<word_t>(quantise4<BITS>(v, p));
     }
   }
 }
 
 template <typename Source>
-cudaError_t launch_quantise(const Source& src, int N, int K, int bits, int group, int scale_f16, uint8_t* packed,
-                            void* scales, cudaStream_t st) {
+cudaError_t launch_quantise(const Source& src, int N, int K, int bits, int group, int scale_f16, int full_range,
+                            uint8_t* packed, void* scales, cudaStream_t st) {
   const int G = group > 0 ? group : K;
   const int ngroups = K / G;
   const long long units = static_cast<long long>(N) * ngroups;
-  const long long warps_needed = G == 128 ? (units + UNITS - 1) / UNITS : units;
+  const long long warps_needed = G == 128 ? (units + 4 * STEPS - 1) / (4 * STEPS) : units;
   const int threads = 256;
   long long blocks = (warps_needed * 32 + threads - 1) / threads;
   const long long cap = 148LL * 8 * 4;  // a few waves of resident blocks; each warp then loops over its units
@@ -170,9 +251,9 @@ cudaError_t launch_quantise(const Source& src, int N, int K, int bits, int group
   if (blocks < 1) blocks = 1;
   const dim3 grid(static_cast<unsigned>(blocks));
   switch (bits) {
-    case 2: quantise_kernel<2, Source><<<grid, threads, 0, st>>>(src, N, K, G, ngroups, scale_f16, packed, scales); break;
-    case 4: quantise_kernel<4, Source><<<grid, threads, 0, st>>>(src, N, K, G, ngroups, scale_f16, packed, scales); break;
-    case 8: quantise_kernel<8, Source><<<grid, threads, 0, st>>>(src, N, K, G, ngroups, scale_f16, packed, scales); break;
+    case 2: quantise_kernel<2, Source><<<grid, threads, 0, st>>>(src, N, K, G, ngroups, scale_f16, full_range, packed, scales); break;
+    case 4: quantise_kernel<4, Source><<<grid, threads, 0, st>>>(src, N, K, G, ngroups, scale_f16, full_range, packed, scales); break;
+    case 8: quantise_kernel<8, Source><<<grid, threads, 0, st>>>(src, N, K, G, ngroups, scale_f16, full_range, packed, scales); break;
     default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
@@ -180,17 +261,17 @@ cudaError_t launch_quantise(const Source& src, int N, int K, int bits, int group
 
 }  // namespace
 
-cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int scale_f16, uint8_t* packed,
+cudaError_t launch_pack(const float* W, int N, int K, int bits, int group, int scale_f16, int full_range, uint8_t* packed,
                         void* scales, cudaStream_t st) {
-  return launch_quantise(SourceF32{W, K}, N, K, bits, group, scale_f16, packed, scales, st);
+  return launch_quantise(SourceF32{W, K}, N, K, bits, group, scale_f16, full_range, packed, scales, st);
 }
 
 cudaError_t launch_requant(const uint8_t* in_packed, const void* in_scales, int N, int K, int bits_in, int bits_out,
-                           int group, int scale_f16, uint8_t* packed, void* scales, cudaStream_t st) {
+                           int group, int scale_f16, int full_range, uint8_t* packed, void* scales, cudaStream_t st) {
   switch (bits_in) {
-    case 2: return launch_quantise(SourcePacked<2>{in_packed, in_scales, K, scale_f16}, N, K, bits_out, group, scale_f16, packed, scales, st);
-    case 4: return launch_quantise(SourcePacked<4>{in_packed, in_scales, K, scale_f16}, N, K, bits_out, group, scale_f16, packed, scales, st);
-    case 8: return launch_quantise(SourcePacked<8>{in_packed, in_scales, K, scale_f16}, N, K, bits_out, group, scale_f16, packed, scales, st);
+    case 2: return launch_quantise(SourcePacked<2>{in_packed, in_scales, K, scale_f16}, N, K, bits_out, group, scale_f16, full_range, packed, scales, st);
+    case 4: return launch_quantise(SourcePacked<4>{in_packed, in_scales, K, scale_f16}, N, K, bits_out, group, scale_f16, full_range, packed, scales, st);
+    case 8: return launch_quantise(SourcePacked<8>{in_packed, in_scales, K, scale_f16}, N, K, bits_out, group, scale_f16, full_range, packed, scales, st);
     default: return cudaErrorInvalidValue;
   }
 }

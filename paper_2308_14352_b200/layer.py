@@ -73,22 +73,22 @@ class MoELayer:
         self.ctx = None
 
     # -- packing -----------------------------------------------------------------------------
-    def pack_matrix(self, e: int, m: int, W_dev: torch.Tensor, stream: int = 0) -> None:
+    def pack_matrix(self, e: int, m: int, W_dev: torch.Tensor, stream: int = 0, full_range: bool = False) -> None:
         """Quantise + pack one fp32 device matrix [N][K] into this layer's storage."""
         N, K = self.shape.matrix_shape(m)
         assert W_dev.dtype == torch.float32 and W_dev.is_contiguous() and tuple(W_dev.shape) == (N, K)
-        B.emoe_pack_expert(self.ctx, W_dev.data_ptr(), N, K, self.bits[e], self.shape.group,
-                           _SDT[self.shape.scale_dtype], self.packed[e][m].data_ptr(), self.scales[e][m].data_ptr(),
-                           stream)
+        B.emoe_pack_expert_mode(self.ctx, W_dev.data_ptr(), N, K, self.bits[e], self.shape.group,
+                                _SDT[self.shape.scale_dtype], B.RANGE_FULL if full_range else B.RANGE_SYMMETRIC,
+                                self.packed[e][m].data_ptr(), self.scales[e][m].data_ptr(), stream)
 
-    def pack_from_host(self, W: Sequence[Sequence[np.ndarray]]) -> None:
+    def pack_from_host(self, W: Sequence[Sequence[np.ndarray]], full_range: bool = False) -> None:
         for e in range(self.shape.n_experts):
             for m in range(self.shape.n_matrices):
                 w = torch.from_numpy(np.ascontiguousarray(W[e][m], dtype=np.float32)).to(self.device)
-                self.pack_matrix(e, m, w)
+                self.pack_matrix(e, m, w, full_range=full_range)
         torch.cuda.synchronize(self.device)
 
-    def change_width(self, e: int, bits_out: int, stream: int = 0) -> None:
+    def change_width(self, e: int, bits_out: int, stream: int = 0, full_range: bool = False) -> None:
         """Moves expert `e` to `bits_out` on the device, from its stored codes and scales (no fp32
         original needed), and points the expert table at the new buffers."""
         b_in = self.bits[e]
@@ -97,9 +97,10 @@ class MoELayer:
             N, K = self.shape.matrix_shape(m)
             p = torch.empty(N * K * bits_out // 8, dtype=torch.uint8, device=self.device)
             s = torch.empty_like(self.scales[e][m])
-            B.emoe_requantize_expert(self.ctx, self.packed[e][m].data_ptr(), self.scales[e][m].data_ptr(), N, K, b_in,
-                                     bits_out, self.shape.group, _SDT[self.shape.scale_dtype], p.data_ptr(),
-                                     s.data_ptr(), stream)
+            B.emoe_requantize_expert_mode(self.ctx, self.packed[e][m].data_ptr(), self.scales[e][m].data_ptr(), N, K,
+                                          b_in, bits_out, self.shape.group, _SDT[self.shape.scale_dtype],
+                                          B.RANGE_FULL if full_range else B.RANGE_SYMMETRIC, p.data_ptr(),
+                                          s.data_ptr(), stream)
             new_packed.append(p)
             new_scales.append(s)
         torch.cuda.synchronize(self.device)  # the old buffers are released below

@@ -5,10 +5,11 @@ import oracle
 from paper_2308_14352_b200 import inputs
 
 
-def oracle_pack_layer(W, shape, bits):
+def oracle_pack_layer(W, shape, bits, full_range=False):
     packed, scales = [], []
     for e in range(shape.n_experts):
-        ps = [oracle.pack_expert(W[e][m], bits[e], shape.group, shape.scale_dtype) for m in range(shape.n_matrices)]
+        ps = [oracle.pack_expert(W[e][m], bits[e], shape.group, shape.scale_dtype, full_range)
+              for m in range(shape.n_matrices)]
         packed.append([p for p, _ in ps])
         scales.append([s for _, s in ps])
     return packed, scales

@@ -15,15 +15,16 @@ from tests.helpers import check_ids, oracle_pack_layer, output_tolerance, rel_to
 pytestmark = pytest.mark.gpu
 
 
-def _run_case(shape, bits, T, seed, path, bias=None, std=0.02, max_tokens=None, fused=True, want_y=False):
+def _run_case(shape, bits, T, seed, path, bias=None, std=0.02, max_tokens=None, fused=True, want_y=False,
+              full_range=False):
     W = inputs.expert_set(seed, 0, shape, std)
     x = inputs.activations(seed, 0, T, shape.d_model, shape.act_dtype)
     Wr = inputs.router_weight(seed, 0, shape.d_model, shape.n_experts, std=0.05)
-    packed, scales = oracle_pack_layer(W, shape, bits)
+    packed, scales = oracle_pack_layer(W, shape, bits, full_range)
     with layer.MoELayer(shape, bits, max_tokens=max_tokens or T) as moe:
         B.emoe_set_ffn_path(moe.ctx, path)
         B.emoe_set_fused_projections(moe.ctx, fused)
-        moe.pack_from_host(W)
+        moe.pack_from_host(W, full_range)
         for e in range(shape.n_experts):          # packed bytes and scales are bit-exact
             for m in range(shape.n_matrices):
                 assert np.array_equal(moe.packed_host(e, m), packed[e][m])
@@ -136,6 +137,28 @@ def test_int8_streaming_path_keeps_the_bf16_range():
         y_ref = oracle.moe_ffn_combine(x, shape.d_ff, shape.act, shape.group, True, bits, packed, scales, ids, gates)
         assert np.isfinite(y).all() and np.abs(y_ref).max() > 0
         assert rel_to_max(y, y_ref) <= 2e-3, (scale_x, std, rel_to_max(y, y_ref))
+
+
+FULL_RANGE_CASES = [
+    # path, act, act_dtype, group, sdt, d, f, E, k, gate, bits, T
+    (1, "relu", "f32", 64, "f32", 192, 320, 3, 2, "softmax_renorm", [2, 8, 4], 7),            # CUDA-core kernel
+    (2, "swiglu", "bf16", 128, "f16", 256, 384, 4, 2, "softmax", [2, 4, 8, 2], 9),              # register-staged mma.sync
+    (3, "relu", "bf16", 128, "f16", 512, 1024, 4, 1, "softmax", [2, 4, 8, 2], 12),              # streaming, offset codes
+    (3, "swiglu", "bf16", 128, "f16", 512, 1024, 4, 2, "softmax_renorm", [2, 2, 4, 8], 40),     # streaming, exact codes
+    (6, "relu", "bf16", 128, "f16", 512, 1024, 4, 1, "softmax", [2, 4, 8, 2], 12),              # int8 tcgen05 streaming
+    (6, "swiglu", "bf16", 128, "f16", 512, 1024, 4, 2, "softmax_renorm", [2, 2, 4, 8], 9),
+    (4, "relu", "bf16", 128, "f16", 512, 1024, 2, 1, "softmax", [2, 4], 300),                   # tcgen05 grouped GEMM
+    (4, "swiglu", "bf16", 128, "f16", 512, 1024, 2, 2, "softmax", [8, 2], 200),
+]
+
+
+@pytest.mark.parametrize("path,act,adt,group,sdt,d,f,E,k,gate,bits,T", FULL_RANGE_CASES)
+def test_forward_with_experts_packed_over_the_full_code_range(path, act, adt, group, sdt, d, f, E, k, gate, bits, T):
+    """Experts quantised with the reading that uses every code of the field (-2^(b-1) included: the
+    fourth INT2 level, -8, -128) run through every kernel family: the kernels decode whole
+    two's-complement fields, so only the quantiser differs."""
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, adt)
+    _run_case(shape, bits, T, seed=29, path=path, full_range=True)
 
 
 ROUTE_CASES = [

@@ -21,7 +21,7 @@ def ctx():
     B.emoe_destroy(c)
 
 
-def _gpu_pack(ctx, W, bits, group, sdt):
+def _gpu_pack(ctx, W, bits, group, sdt, full_range=False):
     N, K = W.shape
     G = group if group else K
     code, tdt = SDT[sdt]
@@ -29,7 +29,11 @@ def _gpu_pack(ctx, W, bits, group, sdt):
     packed = torch.zeros(B.emoe_packed_bytes(N, K, bits), dtype=torch.uint8, device="cuda")
     scales = torch.zeros(N * (K // G), dtype=tdt, device="cuda")
     assert B.emoe_scales_bytes(N, K, group, code) == scales.numel() * scales.element_size()
-    B.emoe_pack_expert(ctx, Wd.data_ptr(), N, K, bits, group, code, packed.data_ptr(), scales.data_ptr(), 0)
+    if full_range:
+        B.emoe_pack_expert_mode(ctx, Wd.data_ptr(), N, K, bits, group, code, B.RANGE_FULL, packed.data_ptr(),
+                                scales.data_ptr(), 0)
+    else:
+        B.emoe_pack_expert(ctx, Wd.data_ptr(), N, K, bits, group, code, packed.data_ptr(), scales.data_ptr(), 0)
     torch.cuda.synchronize()
     return packed.cpu().numpy().reshape(N, -1), scales.cpu().numpy().reshape(N, K // G)
 
@@ -75,3 +79,64 @@ def test_pack_argument_errors(ctx):
     assert call(W.data_ptr(), 0, 128, 4, 0, B.DTYPE_F32, out.data_ptr(), sc.data_ptr(), None) == B.ERR_INVALID_ARG
     assert call(W.data_ptr() + 4, 8, 128, 4, 0, B.DTYPE_F32, out.data_ptr(), sc.data_ptr(), None) == B.ERR_ALIGNMENT
     assert call(W.data_ptr(), 8, 128, 4, 0, B.DTYPE_BF16, out.data_ptr(), sc.data_ptr(), None) == B.ERR_UNSUPPORTED
+
+
+def _assert_same(p_gpu, s_gpu, p_ref, s_ref, sdt):
+    view = np.uint16 if sdt == "f16" else np.uint32
+    assert np.array_equal(s_gpu.view(view), oracle.scales_storage(s_ref, sdt).view(view))
+    assert np.array_equal(p_gpu, p_ref)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("group,sdt", [(0, "f32"), (128, "f16"), (32, "f16"), (128, "f32")])
+@pytest.mark.parametrize("N,K", [(37, 384), (130, 128)])
+def test_pack_full_range_bit_exact(ctx, bits, group, sdt, N, K):
+    """The reading that uses every code of the field (Section 3.2): bytes and scales bit for bit."""
+    rng = np.random.default_rng(bits * 77 + group + N)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    W[1, :] = 0.0
+    W[2, : K // 2] *= 1e-6
+    W[3, 5] = -np.abs(W[3]).max() * 2                # the negative extreme takes the extra code
+    W[4, 9] = np.abs(W[4]).max() * 2                 # the positive extreme is clamped
+    p_ref, s_ref = oracle.pack_expert(W, bits, group, sdt, full_range=True)
+    p_gpu, s_gpu = _gpu_pack(ctx, W, bits, group, sdt, full_range=True)
+    _assert_same(p_gpu, s_gpu, p_ref, s_ref, sdt)
+    q = oracle.unpack(p_gpu, K, bits)
+    assert q.min() == -(1 << (bits - 1)) and q.max() == (1 << (bits - 1)) - 1
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("group,sdt", [(128, "f16"), (128, "f32"), (0, "f32"), (64, "f16")])
+@pytest.mark.parametrize("full_range", [False, True])
+def test_pack_weights_on_and_next_to_rounding_ties(ctx, bits, group, sdt, full_range):
+    """The kernel forms w * (1/s) and falls back to the definition's division near a half-integer.
+    Weights placed on the ties of their group's stored scale and one to three fp32 steps on either
+    side of them, at ordinary, tiny and huge magnitudes, must still give the definition's codes."""
+    rng = np.random.default_rng(9 + bits + group)
+    N, K = 48, 512
+    G = group or K
+    half = 1 << (bits - 1)
+    W = np.zeros((N, K), dtype=np.float32)
+    for n in range(N):
+        mag = [0.02, 1.0, 3e-7, 1e-36, 3e34, 777.0][n % 6]
+        for g in range(K // G):
+            amax = np.float32(mag * (1.0 + rng.random()))
+            rng_div = np.float32(half if full_range else half - 1)
+            s = np.float32(amax / rng_div)
+            if sdt == "f16":
+                with np.errstate(over="ignore"):
+                    s = np.float32(np.float16(s))
+            if not np.isfinite(s) or s == 0:
+                s = np.float32(amax / rng_div)
+            h = rng.integers(-half, half, size=G).astype(np.float64) + 0.5      # half-integers in range
+            w = (h * np.float64(s)).astype(np.float32)
+            steps = rng.integers(-3, 4, size=G)
+            for i in range(G):
+                for _ in range(abs(int(steps[i]))):
+                    w[i] = np.nextafter(w[i], np.float32(np.inf if steps[i] > 0 else -np.inf))
+            w[0] = amax                                                          # fixes the group's max-abs
+            w = np.clip(w, -amax, amax)
+            W[n, g * G:(g + 1) * G] = w
+    p_ref, s_ref = oracle.pack_expert(W, bits, group, sdt, full_range)
+    p_gpu, s_gpu = _gpu_pack(ctx, W, bits, group, sdt, full_range)
+    _assert_same(p_gpu, s_gpu, p_ref, s_ref, sdt)

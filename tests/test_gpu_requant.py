@@ -22,7 +22,7 @@ def ctx():
     B.emoe_destroy(c)
 
 
-def _gpu_requant(ctx, packed, scales, K, bits_in, bits_out, group, sdt):
+def _gpu_requant(ctx, packed, scales, K, bits_in, bits_out, group, sdt, full_range=False):
     N = packed.shape[0]
     G = group if group else K
     code, tdt, _ = SDT[sdt]
@@ -30,8 +30,12 @@ def _gpu_requant(ctx, packed, scales, K, bits_in, bits_out, group, sdt):
     sin = torch.from_numpy(oracle.scales_storage(scales, sdt)).cuda()
     pout = torch.zeros(B.emoe_packed_bytes(N, K, bits_out), dtype=torch.uint8, device="cuda")
     sout = torch.zeros(N * (K // G), dtype=tdt, device="cuda")
-    B.emoe_requantize_expert(ctx, pin.data_ptr(), sin.data_ptr(), N, K, bits_in, bits_out, group, code,
-                             pout.data_ptr(), sout.data_ptr(), 0)
+    if full_range:
+        B.emoe_requantize_expert_mode(ctx, pin.data_ptr(), sin.data_ptr(), N, K, bits_in, bits_out, group, code,
+                                      B.RANGE_FULL, pout.data_ptr(), sout.data_ptr(), 0)
+    else:
+        B.emoe_requantize_expert(ctx, pin.data_ptr(), sin.data_ptr(), N, K, bits_in, bits_out, group, code,
+                                 pout.data_ptr(), sout.data_ptr(), 0)
     torch.cuda.synchronize()
     return pout.cpu().numpy().reshape(N, -1), sout.cpu().numpy().reshape(N, K // G)
 
@@ -149,3 +153,20 @@ def test_forward_after_lowering_the_width_of_two_experts():
         y, ids, gates, _ = moe.forward(x, Wr)
     y_ref = oracle.moe_ffn_combine(x, shape.d_ff, "swiglu", 128, True, new_bits, packed, scales, ids, gates)
     assert rel_to_max(y, y_ref) <= 2e-3
+
+
+@pytest.mark.parametrize("bits_in,bits_out", [(8, 4), (8, 2), (4, 2), (2, 2), (2, 8)])
+@pytest.mark.parametrize("group,sdt", [(0, "f32"), (128, "f16"), (32, "f16")])
+def test_requantize_full_range_bit_exact(ctx, bits_in, bits_out, group, sdt):
+    """A stored matrix (itself packed with the full code range) moved to another width, again with
+    the full range (Section 3.2): bytes and scales bit for bit."""
+    N, K = 37, 384
+    rng = np.random.default_rng(bits_in * 31 + bits_out + group)
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    W[1, :] = 0.0
+    packed, scales = oracle.pack_expert(W, bits_in, group, sdt, full_range=True)
+    p_ref, s_ref = oracle.requantize(packed, scales, K, bits_in, bits_out, group, sdt, full_range=True)
+    p_gpu, s_gpu = _gpu_requant(ctx, packed, scales, K, bits_in, bits_out, group, sdt, full_range=True)
+    view = SDT[sdt][2]
+    assert np.array_equal(s_gpu.view(view), oracle.scales_storage(s_ref, sdt).view(view))
+    assert np.array_equal(p_gpu, p_ref)
