@@ -26,6 +26,8 @@
 namespace emoe {
 namespace {
 
+constexpr float ROUND_MAGIC = 12582912.0f;  // 1.5 * 2^23, bit pattern 0x4B400000
+
 template <int BITS>
 struct PackWord;  // the codes of 4 consecutive weights
 template <>
@@ -38,29 +40,46 @@ struct PackWord<2> { typedef uint8_t type; };
 // Where the weights come from.  load4(n, k): weights k .. k+3 of row n (k a multiple of 4);
 // `unit` is the row's group index n * ngroups + g.
 struct SourceF32 {
+  static constexpr int IN_BITS = 32;
   const float* W;
   int K;
   __device__ __forceinline__ float4 load4(int n, int k, long long) const {
     return *reinterpret_cast<const float4*>(W + static_cast<size_t>(n) * K + k);
   }
-  // 16 consecutive weights from linear index w0 (a multiple of 16) of the dense matrix
-  __device__ __forceinline__ void load16(long long w0, long long, float (&v)[16]) const {
+  // 16 consecutive weights from linear index w0 (a multiple of 16) of the dense matrix: first the
+  // loads (several steps are requested before the first is used), then the values
+  static constexpr int STEPS = 2;  // four-unit steps a warp has in flight
+  struct Raw {
+    float4 f[4];
+  };
+  __device__ __forceinline__ void load_raw(long long w0, long long, Raw& r, float&) const {
     const float4* p = reinterpret_cast<const float4*>(W + w0);
 #pragma unroll
+    for (int i = 0; i < 4; ++i) r.f[i] = p[i];
+  }
+  __device__ __forceinline__ void zero_raw(Raw& r, float&) const {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r.f[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  __device__ __forceinline__ void decode(const Raw& r, float, float (&v)[16]) const {
+#pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const float4 f = p[i];
-      v[4 * i] = f.x;
-      v[4 * i + 1] = f.y;
-      v[4 * i + 2] = f.z;
-      v[4 * i + 3] = f.w;
+      v[4 * i] = r.f[i].x;
+      v[4 * i + 1] = r.f[i].y;
+      v[4 * i + 2] = r.f[i].z;
+      v[4 * i + 3] = r.f[i].w;
     }
   }
 };
 template <int BIN>
 struct SourcePacked {
+  static constexpr int IN_BITS = BIN;
   const uint8_t* packed;
   const void* scales;
   int K, scale_f16;
+  __device__ __forceinline__ float scale_of(long long unit) const {
+    return scale_f16 ? __half2float(reinterpret_cast<const __half*>(scales)[unit]) : reinterpret_cast<const float*>(scales)[unit];
+  }
   __device__ __forceinline__ float4 load4(int n, int k, long long unit) const {
     const uint8_t* row = packed + static_cast<size_t>(n) * (static_cast<size_t>(K) * BIN / 8);
     uint32_t w;  // the codes of the 4 weights, low fields first
@@ -77,26 +96,35 @@ struct SourcePacked {
     }
     return make_float4(v[0], v[1], v[2], v[3]);
   }
-  __device__ __forceinline__ void load16(long long w0, long long unit, float (&v)[16]) const {
-    uint32_t w[4];  // the 16 codes, low fields first
+  static constexpr int STEPS = 2;  // as measured: more steps in flight buy nothing here (the kernel is bound by its instruction count)
+  struct Raw {
+    uint32_t w[BIN / 2];  // the 16 codes, low fields first
+  };
+  __device__ __forceinline__ void load_raw(long long w0, long long unit, Raw& r, float& s) const {
     const uint8_t* p = packed + w0 * BIN / 8;
     if (BIN == 8) {
       const uint4 q = *reinterpret_cast<const uint4*>(p);
-      w[0] = q.x, w[1] = q.y, w[2] = q.z, w[3] = q.w;
+      r.w[0] = q.x, r.w[1] = q.y, r.w[2] = q.z, r.w[3] = q.w;
     } else if (BIN == 4) {
       const uint2 q = *reinterpret_cast<const uint2*>(p);
-      w[0] = q.x, w[1] = q.y;
+      r.w[0] = q.x, r.w[1] = q.y;
     } else {
-      w[0] = *reinterpret_cast<const uint32_t*>(p);
+      r.w[0] = *reinterpret_cast<const uint32_t*>(p);
     }
-    const float s = scale_f16 ? __half2float(reinterpret_cast<const __half*>(scales)[unit])
-                              : reinterpret_cast<const float*>(scales)[unit];
+    s = scale_of(unit);
+  }
+  __device__ __forceinline__ void zero_raw(Raw& r, float& s) const {
+#pragma unroll
+    for (int i = 0; i < BIN / 2; ++i) r.w[i] = 0u;
+    s = 0.0f;
+  }
+  __device__ __forceinline__ void decode(const Raw& r, float s, float (&v)[16]) const {
     constexpr int PER_WORD = 32 / BIN;
 #pragma unroll
     for (int c = 0; c < 16; ++c) {
-      const uint32_t word = w[c / PER_WORD];
+      const uint32_t word = r.w[c / PER_WORD];
       const int q = static_cast<int>(word << (32 - BIN * (c % PER_WORD + 1))) >> (32 - BIN);
-      v[c] = __fmul_rn(static_cast<float>(q), s);
+      v[c] = __fmul_rn(__int_as_float(0x4B400000 + q) - ROUND_MAGIC, s);  // the integer as a float, exactly
     }
   }
 };
@@ -123,19 +151,23 @@ struct QuantParams {
 __device__ __forceinline__ QuantParams quant_params(float s, float qlo, float qhi) {
   QuantParams p;
   p.s = s;
-  p.r = (s > 1e-30f && s < 1e30f) ? __frcp_rn(s) : __int_as_float(0x7fc00000);
+  // scale 0: reciprocal 0, every product is 0 and every code is 0, as the definition says
+  p.r = s == 0.0f ? 0.0f : ((s > 1e-30f && s < 1e30f) ? __frcp_rn(s) : __int_as_float(0x7fc00000));
   p.qlo = qlo;
   p.qhi = qhi;
   return p;
 }
-// one code: round-half-even of the fp32 quotient e / s, clamped (0 when the scale is 0)
-__device__ __forceinline__ int quantise1(float e, const QuantParams& p) {
-  const float t = e * p.r;
-  float q = rintf(t);
+// Adding and subtracting 1.5 * 2^23 rounds a float of magnitude below 2^22 to the nearest integer,
+// ties to even (the addition's own rounding); after the addition the integer sits in the low
+// mantissa bits in two's complement.
+// one code (its low bits are the field): round-half-even of the fp32 quotient e / s, clamped
+__device__ __forceinline__ uint32_t quantise1(float e, const QuantParams& p) {
+  const float t = __fmul_rn(e, p.r);  // never contracted into the addition below
+  float q = __fsub_rn(__fadd_rn(t, ROUND_MAGIC), ROUND_MAGIC);
   const float d = fabsf(fabsf(t - q) - 0.5f);
   if (!(d >= 1e-4f) || !(fabsf(t) < 200.0f)) q = rintf(__fdiv_rn(e, p.s));
   q = fminf(fmaxf(q, p.qlo), p.qhi);
-  return p.s != 0.0f ? static_cast<int>(q) : 0;
+  return __float_as_uint(__fadd_rn(q, ROUND_MAGIC));
 }
 
 // codes of 4 weights: round half to even on the quotient by the stored scale, clamp, pack
@@ -145,15 +177,13 @@ __device__ __forceinline__ uint32_t quantise4(const float4& v, const QuantParams
   const float e[4] = {v.x, v.y, v.z, v.w};
   uint32_t word = 0;
 #pragma unroll
-  for (int c = 0; c < 4; ++c) word |= static_cast<uint32_t>(quantise1(e[c], p) & MASK) << (BITS * c);
+  for (int c = 0; c < 4; ++c) word |= (quantise1(e[c], p) & MASK) << (BITS * c);
   return word;
 }
 
 __device__ __forceinline__ float amax4(const float4& v) {
   return fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
 }
-
-constexpr int STEPS = 2;  // four-unit steps a warp has in flight (groups of 128)
 
 template <int BITS, typename Source>
 __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, int K, int G, int ngroups, int scale_f16,
@@ -170,45 +200,98 @@ __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, 
   const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
   const size_t row_bytes = static_cast<size_t>(K) * BITS / 8;
 
+  if constexpr (Source::IN_BITS == 4 && BITS == 2) {
+    if (G == 128) {
+      // A 4-bit unit holds at most 16 different weights: the unit's 8 lanes quantise two of the 16
+      // possible codes each (with the very function every other path uses), share the results as a
+      // table of 16 x 2 bits, and every stored code is then a table lookup.  The unit's max-abs is
+      // s * max |q| (rounding is monotone), found on the integer codes.
+      constexpr int STEPS = Source::STEPS;
+      const long long n_steps = (n_units + 3) >> 2;
+      for (long long st0 = warp * STEPS; st0 < n_steps; st0 += warps * STEPS) {
+        typename Source::Raw raws[STEPS];
+        float s_ins[STEPS];
+#pragma unroll
+        for (int u = 0; u < STEPS; ++u) {
+          const long long unit = (st0 + u) * 4 + (lane >> 3);
+          if (unit < n_units) src.load_raw(unit * 128 + (lane & 7) * 16, unit, raws[u], s_ins[u]);
+          else src.zero_raw(raws[u], s_ins[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < STEPS; ++u) {
+          const long long unit = (st0 + u) * 4 + (lane >> 3);
+          const bool live = unit < n_units;
+          const uint32_t rx = raws[u].w[0], ry = raws[u].w[1];
+          const float s_in = s_ins[u];
+          int m = 0;
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const uint32_t word = c < 8 ? rx : ry;
+            const int q = static_cast<int>(word << (28 - 4 * (c & 7))) >> 28;
+            m = max(m, abs(q));
+          }
+#pragma unroll
+          for (int o = 4; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+          const float amax = __fmul_rn(static_cast<float>(m), s_in);
+          const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, live && (lane & 7) == 0), qlo, qhi);
+          uint32_t lut = 0;
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            const int nib = 2 * (lane & 7) + i;
+            const int q = (nib ^ 8) - 8;  // the field's value
+            lut |= (quantise1(__fmul_rn(static_cast<float>(q), s_in), p) & 3u) << (2 * nib);
+          }
+#pragma unroll
+          for (int o = 4; o > 0; o >>= 1) lut |= __shfl_xor_sync(0xffffffffu, lut, o);
+          uint32_t out = 0;
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const uint32_t word = c < 8 ? rx : ry;
+            const uint32_t nib2 = ((word >> (4 * (c & 7))) << 1) & 30u;
+            out |= ((lut >> nib2) & 3u) << (2 * c);
+          }
+          if (live) *reinterpret_cast<uint32_t*>(packed + (unit * 128 + (lane & 7) * 16) / 4) = out;
+        }
+      }
+      return;
+    }
+  }
   if (G == 128) {
     // K is a whole number of units, so unit u holds the weights 128 u .. 128 u + 127 of the dense
     // matrix and the bytes 16 b u .. of the packed one, whatever its row
+    constexpr int STEPS = Source::STEPS;
     const long long n_steps = (n_units + 3) >> 2;
     for (long long st0 = warp * STEPS; st0 < n_steps; st0 += warps * STEPS) {
-      float v[STEPS][16];
-      float amax[STEPS];
+      typename Source::Raw raws[STEPS];
+      float s_ins[STEPS];
 #pragma unroll
       for (int u = 0; u < STEPS; ++u) {
         const long long unit = (st0 + u) * 4 + (lane >> 3);
-        if (unit < n_units) {
-          src.load16(unit * 128 + (lane & 7) * 16, unit, v[u]);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 16; ++c) v[u][c] = 0.0f;
-        }
-        float m = 0.0f;
-#pragma unroll
-        for (int c = 0; c < 16; ++c) m = fmaxf(m, fabsf(v[u][c]));
-        amax[u] = m;
+        if (unit < n_units) src.load_raw(unit * 128 + (lane & 7) * 16, unit, raws[u], s_ins[u]);
+        else src.zero_raw(raws[u], s_ins[u]);
       }
 #pragma unroll
-      for (int o = 4; o > 0; o >>= 1)
-#pragma unroll
-        for (int u = 0; u < STEPS; ++u) amax[u] = fmaxf(amax[u], __shfl_xor_sync(0xffffffffu, amax[u], o));
-#pragma unroll
       for (int u = 0; u < STEPS; ++u) {
         const long long unit = (st0 + u) * 4 + (lane >> 3);
-        if (unit >= n_units) continue;
-        const QuantParams p = quant_params(store_scale(amax[u], range, scale_f16, scales, unit, (lane & 7) == 0), qlo, qhi);
+        const bool live = unit < n_units;
+        float v[16];
+        src.decode(raws[u], s_ins[u], v);
+        float amax = 0.0f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) amax = fmaxf(amax, fabsf(v[c]));
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, live && (lane & 7) == 0), qlo, qhi);
         uint32_t w[4] = {0u, 0u, 0u, 0u};
         constexpr int PER_WORD = 32 / BITS;
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-          w[c / PER_WORD] |= static_cast<uint32_t>(quantise1(v[u][c], p) & MASK) << (BITS * (c % PER_WORD));
-        uint8_t* out = packed + (unit * 128 + (lane & 7) * 16) * BITS / 8;
-        if (BITS == 8) *reinterpret_cast<uint4*>(out) = make_uint4(w[0], w[1], w[2], w[3]);
-        else if (BITS == 4) *reinterpret_cast<uint2*>(out) = make_uint2(w[0], w[1]);
-        else *reinterpret_cast<uint32_t*>(out) = w[0];
+        for (int c = 0; c < 16; ++c) w[c / PER_WORD] |= (quantise1(v[c], p) & MASK) << (BITS * (c % PER_WORD));
+        if (live) {
+          uint8_t* out = packed + (unit * 128 + (lane & 7) * 16) * BITS / 8;
+          if (BITS == 8) *reinterpret_cast<uint4*>(out) = make_uint4(w[0], w[1], w[2], w[3]);
+          else if (BITS == 4) *reinterpret_cast<uint2*>(out) = make_uint2(w[0], w[1]);
+          else *reinterpret_cast<uint32_t*>(out) = w[0];
+        }
       }
     }
     return;
@@ -243,7 +326,7 @@ cudaError_t launch_quantise(const Source& src, int N, int K, int bits, int group
   const int G = group > 0 ? group : K;
   const int ngroups = K / G;
   const long long units = static_cast<long long>(N) * ngroups;
-  const long long warps_needed = G == 128 ? (units + 4 * STEPS - 1) / (4 * STEPS) : units;
+  const long long warps_needed = G == 128 ? (units + 4 * Source::STEPS - 1) / (4 * Source::STEPS) : units;
   const int threads = 256;
   long long blocks = (warps_needed * 32 + threads - 1) / threads;
   const long long cap = 148LL * 8 * 4;  // a few waves of resident blocks; each warp then loops over its units
