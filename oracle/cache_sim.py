@@ -150,3 +150,41 @@ def rank_experts(prior, prev_ids):
     E = len(prior)
     score = [sum(float(prior[p][e]) for p in prev_ids) for e in range(E)]
     return sorted(range(E), key=lambda e: (-score[e], e))
+
+
+def build_profile2(trace, n_experts):
+    """The offline statistical profile of Section 3.3 ("Opportunistic preloading"): a dictionary
+    whose key is the activation status of the two previous MoE layers and whose value is the
+    probability of each expert of the next layer being activated.  trace[token][layer] lists the
+    experts a token activated in a layer.  Returned: table[n][a][b][e] for every layer n >= 2 =
+    (times e was active in layer n while a was active in layer n-2 and b in layer n-1) / (times a
+    and b were active in layers n-2 and n-1); keys never seen get the uniform distribution; layers
+    0 and 1 (no two previous layers) get all zeros.  With Top-K > 1 a key is every (a, b) pair of
+    the two layers' picks."""
+    n_layers = len(trace[0])
+    E = n_experts
+    table = [[[[0.0] * E for _ in range(E)] for _ in range(E)] for _ in range(n_layers)]
+    seen = [[[0] * E for _ in range(E)] for _ in range(n_layers)]
+    for row in trace:
+        for n in range(2, n_layers):
+            for a in row[n - 2]:
+                for b in row[n - 1]:
+                    seen[n][a][b] += 1
+                    for e in row[n]:
+                        table[n][a][b][e] += 1.0
+    for n in range(2, n_layers):
+        for a in range(E):
+            for b in range(E):
+                c = seen[n][a][b]
+                for e in range(E):
+                    table[n][a][b][e] = table[n][a][b][e] / c if c else 1.0 / E
+    return table
+
+
+def rank_experts2(table_n, prev2_ids, prev1_ids):
+    """Next layer's experts by descending estimated probability given the picks of the two previous
+    layers (table_n[a][b] = distribution for the key (a, b); several picks per layer: the rows of
+    every (a, b) pair are added), ties by lower index."""
+    E = len(table_n)
+    score = [sum(float(table_n[a][b][e]) for a in prev2_ids for b in prev1_ids) for e in range(E)]
+    return sorted(range(E), key=lambda e: (-score[e], e))

@@ -5,9 +5,10 @@ import itertools
 import random
 from collections import OrderedDict
 
+import numpy as np
 import pytest
 
-from oracle.cache_sim import ExpertBufferModel, rank_experts
+from oracle.cache_sim import ExpertBufferModel, build_profile2, rank_experts, rank_experts2
 
 
 def _fill(m, ids, layer_fn, acquires):
@@ -205,3 +206,55 @@ def test_rank_experts():
     assert rank_experts(prior, [0]) == [0, 1, 2]
     assert rank_experts(prior, [1]) == [2, 0, 1]            # tie between 0 and 1: lower index first
     assert rank_experts(prior, [0, 1]) == [2, 0, 1]         # sums 0.8, 0.3, 0.9
+
+
+def test_profile_keyed_on_two_previous_layers_hand_worked():
+    """Four tokens through three layers of three experts, top-1 (picks per layer):
+    (0,1,2) (0,1,2) (0,1,0) (1,1,2).  Key (0,1) was seen three times: expert 2 followed twice,
+    expert 0 once; key (1,1) once, followed by expert 2; every other key was never seen."""
+    trace = [[[0], [1], [2]], [[0], [1], [2]], [[0], [1], [0]], [[1], [1], [2]]]
+    t = build_profile2(trace, 3)
+    assert t[0] == [[[0.0] * 3] * 3] * 3 and t[1] == [[[0.0] * 3] * 3] * 3
+    assert t[2][0][1] == [1 / 3, 0.0, 2 / 3]
+    assert t[2][1][1] == [0.0, 0.0, 1.0]
+    assert t[2][2][0] == [1 / 3] * 3
+    assert rank_experts2(t[2], [0], [1]) == [2, 0, 1]
+    assert rank_experts2(t[2], [1], [1]) == [2, 0, 1]          # 0 and 1 tie at zero: lower index first
+    assert rank_experts2(t[2], [0, 1], [1]) == [2, 0, 1]       # sums 1/3, 0, 5/3
+
+
+def test_profile2_rows_are_distributions_and_reduce_to_first_order_when_layer_n_minus_2_is_constant():
+    """Closed forms: with Top-K = k every seen key's row sums to k; if layer n-2 always activates
+    the same expert, the table is the first-order conditional P(e | b) counted directly."""
+    rng = np.random.default_rng(2)
+    E, k, L = 5, 2, 4
+    trace = [[sorted(rng.choice(E, size=k, replace=False).tolist()) for _ in range(L)] for _ in range(300)]
+    t = build_profile2(trace, E)
+    for n in range(2, L):
+        for a in range(E):
+            for b in range(E):
+                assert abs(sum(t[n][a][b]) - k) < 1e-12 or t[n][a][b] == [1.0 / E] * E
+    trace1 = [[[0], [int(rng.integers(0, E))], [int(rng.integers(0, E))]] for _ in range(400)]
+    t1 = build_profile2(trace1, E)
+    for b in range(E):
+        nb = sum(1 for r in trace1 if r[1] == [b])
+        for e in range(E):
+            direct = sum(1 for r in trace1 if r[1] == [b] and r[2] == [e]) / nb
+            assert abs(t1[2][0][b][e] - direct) < 1e-12
+
+
+def test_rank_experts2_equals_brute_force_and_first_order_on_a_separable_table():
+    rng = np.random.default_rng(4)
+    E = 6
+    tab = rng.random((E, E, E))
+    for _ in range(20):
+        p2 = rng.integers(0, E, size=2).tolist()
+        p1 = rng.integers(0, E, size=2).tolist()
+        score = np.einsum("abe->e", tab[np.ix_(p2, p1)])
+        assert rank_experts2(tab.tolist(), p2, p1) == sorted(range(E), key=lambda e: (-score[e], e))
+    # a table that ignores layer n-2 ranks exactly as the first-order one
+    first = rng.random((E, E))
+    tab2 = np.broadcast_to(first[None, :, :], (E, E, E))
+    for _ in range(10):
+        p1 = rng.integers(0, E, size=2).tolist()
+        assert rank_experts2(tab2.tolist(), [3], p1) == rank_experts(first.tolist(), p1)
