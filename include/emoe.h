@@ -408,6 +408,21 @@ int emoe_policy_get_stats(emoe_policy* p, emoe_cache_stats* out);
  * experts by descending score, ties by lower index. */
 int emoe_rank_experts(const float* prior, int n_experts, const int32_t* prev_ids, int n_prev, int32_t* out_order);
 
+/* The statistical profile of Section 3.3 ("Opportunistic preloading") with the key the paper
+ * names: the activation status of the TWO previous MoE layers.
+ * emoe_build_profile2 (the offline phase): trace is a host array [n_tokens][n_layers][top_k] of
+ * the experts each token activated; out_prior2 (host, [n_layers][E][E][E] floats, E = n_experts)
+ * receives for every layer n >= 2 and key (a, b) the share of the tokens with a active in layer
+ * n-2 and b active in layer n-1 that activated e in layer n (with top_k > 1 every (a, b) pair of
+ * the two layers' picks is a key; a row sums to top_k); keys never seen get 1/E; layers 0 and 1
+ * get zeros.  An id outside [0, E) returns EMOE_ERR_INVALID_ARG.
+ * emoe_rank_experts2 (the online query): prior2_layer = the [E][E][E] block of the layer to be
+ * predicted; score[e] = sum over a in prev2_ids, b in prev1_ids of prior2_layer[a][b][e];
+ * out_order lists the experts by descending score, ties by lower index. */
+int emoe_build_profile2(const int32_t* trace, int n_tokens, int n_layers, int top_k, int n_experts, float* out_prior2);
+int emoe_rank_experts2(const float* prior2_layer, int n_experts, const int32_t* prev2_ids, int n_prev2,
+                       const int32_t* prev1_ids, int n_prev1, int32_t* out_order);
+
 #ifdef __cplusplus
 }
 #endif

@@ -42,6 +42,7 @@ EXPORTS = (
     "emoe_cache_create", "emoe_register_expert", "emoe_prefetch_experts", "emoe_cache_acquire", "emoe_cache_release",
     "emoe_cache_slot_of", "emoe_cache_get_stats", "emoe_policy_create", "emoe_policy_destroy", "emoe_policy_register",
     "emoe_policy_prefetch", "emoe_policy_acquire", "emoe_policy_release", "emoe_policy_get_stats", "emoe_rank_experts",
+    "emoe_build_profile2", "emoe_rank_experts2",
 )
 
 
@@ -133,6 +134,9 @@ def lib() -> ctypes.CDLL:
         L.emoe_policy_get_stats.argtypes = [vp, ctypes.POINTER(emoe_cache_stats)]
         L.emoe_rank_experts.argtypes = [ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(ctypes.c_int32), i32,
                                         ctypes.POINTER(ctypes.c_int32)]
+        pf, pi = ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)
+        L.emoe_build_profile2.argtypes = [pi, i32, i32, i32, i32, pf]
+        L.emoe_rank_experts2.argtypes = [pf, i32, pi, i32, pi, i32, pi]
         L.emoe_moe_forward_routed_static.argtypes = [i32, ctypes.POINTER(emoe_layer_desc), vp, i32, vp, vp,
                                                      ctypes.POINTER(emoe_expert), vp, vp]
         L.emoe_static_device_status.argtypes = [i32, vp]
@@ -396,4 +400,31 @@ def emoe_rank_experts(prior, prev_ids):
     _check(lib().emoe_rank_experts(prior.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), E,
                                    prev.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), len(prev),
                                    out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "emoe_rank_experts")
+    return out
+
+
+def emoe_build_profile2(trace, n_experts: int):
+    """trace: int array [n_tokens][n_layers][top_k]; returns float32 [n_layers][E][E][E]."""
+    import numpy as np
+
+    tr = np.ascontiguousarray(trace, dtype=np.int32)
+    n_tokens, n_layers, top_k = tr.shape
+    out = np.empty((n_layers, n_experts, n_experts, n_experts), dtype=np.float32)
+    _check(lib().emoe_build_profile2(tr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), n_tokens, n_layers, top_k,
+                                     n_experts, out.ctypes.data_as(ctypes.POINTER(ctypes.c_float))),
+           "emoe_build_profile2")
+    return out
+
+
+def emoe_rank_experts2(prior2_layer, prev2_ids, prev1_ids):
+    import numpy as np
+
+    tab = np.ascontiguousarray(prior2_layer, dtype=np.float32)
+    p2 = np.ascontiguousarray(prev2_ids, dtype=np.int32).reshape(-1)
+    p1 = np.ascontiguousarray(prev1_ids, dtype=np.int32).reshape(-1)
+    E = tab.shape[0]
+    out = np.empty(E, dtype=np.int32)
+    pi = ctypes.POINTER(ctypes.c_int32)
+    _check(lib().emoe_rank_experts2(tab.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), E, p2.ctypes.data_as(pi), len(p2),
+                                    p1.ctypes.data_as(pi), len(p1), out.ctypes.data_as(pi)), "emoe_rank_experts2")
     return out

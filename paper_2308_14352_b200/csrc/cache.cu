@@ -451,4 +451,64 @@ int emoe_rank_experts(const float* prior, int n_experts, const int32_t* prev_ids
   return EMOE_OK;
 }
 
+int emoe_build_profile2(const int32_t* trace, int n_tokens, int n_layers, int top_k, int n_experts, float* out_prior2) {
+  if (!trace || !out_prior2 || n_tokens <= 0 || n_layers <= 0 || top_k <= 0 || n_experts <= 0) return EMOE_ERR_INVALID_ARG;
+  if (n_experts > EMOE_MAX_EXPERTS || top_k > n_experts) return EMOE_ERR_INVALID_ARG;
+  const size_t E = static_cast<size_t>(n_experts);
+  const size_t per_layer = E * E * E;
+  std::vector<double> cnt(per_layer);
+  std::vector<long long> seen(E * E);
+  for (int n = 0; n < n_layers; ++n) {
+    float* out = out_prior2 + static_cast<size_t>(n) * per_layer;
+    if (n < 2) {  // no two previous layers
+      std::fill(out, out + per_layer, 0.0f);
+      continue;
+    }
+    std::fill(cnt.begin(), cnt.end(), 0.0);
+    std::fill(seen.begin(), seen.end(), 0LL);
+    for (int t = 0; t < n_tokens; ++t) {
+      const int32_t* row = trace + (static_cast<size_t>(t) * n_layers) * top_k;
+      const int32_t* l2 = row + static_cast<size_t>(n - 2) * top_k;
+      const int32_t* l1 = row + static_cast<size_t>(n - 1) * top_k;
+      const int32_t* l0 = row + static_cast<size_t>(n) * top_k;
+      for (int i = 0; i < top_k; ++i)
+        for (int j = 0; j < top_k; ++j) {
+          const int a = l2[i], b = l1[j];
+          if (a < 0 || a >= n_experts || b < 0 || b >= n_experts) return EMOE_ERR_INVALID_ARG;
+          ++seen[a * E + b];
+          for (int k = 0; k < top_k; ++k) {
+            const int e = l0[k];
+            if (e < 0 || e >= n_experts) return EMOE_ERR_INVALID_ARG;
+            cnt[(a * E + b) * E + e] += 1.0;
+          }
+        }
+    }
+    for (size_t ab = 0; ab < E * E; ++ab)
+      for (size_t e = 0; e < E; ++e)
+        out[ab * E + e] = seen[ab] ? static_cast<float>(cnt[ab * E + e] / static_cast<double>(seen[ab]))
+                                   : static_cast<float>(1.0 / static_cast<double>(E));
+  }
+  return EMOE_OK;
+}
+
+int emoe_rank_experts2(const float* prior2_layer, int n_experts, const int32_t* prev2_ids, int n_prev2,
+                       const int32_t* prev1_ids, int n_prev1, int32_t* out_order) {
+  if (!prior2_layer || !prev2_ids || !prev1_ids || !out_order || n_experts <= 0 || n_prev2 <= 0 || n_prev1 <= 0)
+    return EMOE_ERR_INVALID_ARG;
+  const size_t E = static_cast<size_t>(n_experts);
+  std::vector<double> score(E, 0.0);
+  for (int i = 0; i < n_prev2; ++i) {
+    if (prev2_ids[i] < 0 || prev2_ids[i] >= n_experts) return EMOE_ERR_INVALID_ARG;
+    for (int j = 0; j < n_prev1; ++j) {
+      if (prev1_ids[j] < 0 || prev1_ids[j] >= n_experts) return EMOE_ERR_INVALID_ARG;
+      const float* row = prior2_layer + (static_cast<size_t>(prev2_ids[i]) * E + static_cast<size_t>(prev1_ids[j])) * E;
+      for (size_t e = 0; e < E; ++e) score[e] += static_cast<double>(row[e]);
+    }
+  }
+  for (int e = 0; e < n_experts; ++e) out_order[e] = e;
+  std::stable_sort(out_order, out_order + n_experts,
+                   [&](int32_t a, int32_t b) { return score[static_cast<size_t>(a)] > score[static_cast<size_t>(b)]; });
+  return EMOE_OK;
+}
+
 }  // extern "C"

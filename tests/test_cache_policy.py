@@ -6,7 +6,7 @@ import random
 import numpy as np
 import pytest
 
-from oracle.cache_sim import ExpertBufferModel, rank_experts
+from oracle.cache_sim import ExpertBufferModel, build_profile2, rank_experts, rank_experts2
 from paper_2308_14352_b200 import binding as B
 
 RULES = [("forward", B.EVICT_FORWARD), ("printed", B.EVICT_PRINTED), ("lru", B.EVICT_LRU), ("lfu", B.EVICT_LFU),
@@ -86,3 +86,23 @@ def test_rank_experts_matches_the_model():
             prev = rng.integers(0, E, size=k)
             got = B.emoe_rank_experts(prior, prev)
             assert got.tolist() == rank_experts(prior.tolist(), prev.tolist())
+
+
+def test_profile_keyed_on_two_previous_layers_matches_the_model():
+    """emoe_build_profile2 / emoe_rank_experts2 (Section 3.3: key = the two previous layers)
+    against the model, entry by entry and rank by rank, incl. keys never seen and exact ties."""
+    rng = np.random.default_rng(6)
+    for E, k, L, n in ((4, 1, 5, 60), (6, 2, 4, 200), (3, 3, 3, 10)):
+        trace = np.stack([np.stack([np.sort(rng.choice(E, size=k, replace=False)) for _ in range(L)]) for _ in range(n)])
+        got = B.emoe_build_profile2(trace, E)
+        ref = np.array(build_profile2(trace.tolist(), E))
+        assert got.shape == ref.shape
+        np.testing.assert_allclose(got, ref, rtol=0, atol=1e-7)
+        for _ in range(20):
+            layer = int(rng.integers(2, L))
+            p2 = rng.choice(E, size=k, replace=False)
+            p1 = rng.choice(E, size=k, replace=False)
+            assert B.emoe_rank_experts2(got[layer], p2, p1).tolist() == rank_experts2(got[layer].astype(np.float64).tolist(),
+                                                                                    p2.tolist(), p1.tolist())
+    with pytest.raises(B.EmoeError):
+        B.emoe_build_profile2(np.full((2, 3, 1), 9, dtype=np.int32), 4)      # id outside [0, E)
