@@ -352,6 +352,10 @@ typedef struct emoe_cache_stats {
   int64_t prefetch_refused;   /* prefetch requests dropped because every slot was in use */
   int64_t evictions;
   int64_t bytes_copied;       /* host -> device bytes of all loads started */
+  int64_t exposed_copy_ns;    /* device time the compute stream stood still inside emoe_cache_acquire, waiting for
+                                 slot contents (loading not hidden under compute: Section 3.3, the pipeline's
+                                 failed-prediction case); counted only while emoe_cache_set_timing is on */
+  int64_t timed_acquires;     /* acquire calls that contributed to exposed_copy_ns */
 } emoe_cache_stats;
 
 /* Allocates the cache of a context: n_slots x slot_bytes of device memory and two events per
@@ -387,6 +391,20 @@ int emoe_cache_release(emoe_ctx* ctx, const int64_t* ids, int n, void* compute_s
 /* Slot that holds the expert, -1 if none. */
 int emoe_cache_slot_of(emoe_ctx* ctx, int64_t id);
 int emoe_cache_get_stats(emoe_ctx* ctx, emoe_cache_stats* out);
+
+/* Exposed-copy accounting (the paper reports compute and loading time separately, Section 4):
+ * while enabled, every emoe_cache_acquire records one CUDA event on compute_stream in front of
+ * its waits and one behind them; emoe_cache_get_stats waits for the recorded pairs, adds their
+ * distances to exposed_copy_ns and clears the record.  With every expert resident the waits return
+ * at once and the sum stays near zero; it can never exceed the time of loading on demand.  Off by
+ * default; not for use during stream capture. */
+int emoe_cache_set_timing(emoe_ctx* ctx, int enabled);
+
+/* Tokens per expert of the most recent forward call on this context (the "tokens per expert"
+ * counter): copies the call's per-expert pair counts (n_experts int32, host memory) after
+ * synchronising `stream`.  EMOE_ERR_INVALID_ARG before the first forward call or when n_experts
+ * differs from that call's. */
+int emoe_last_expert_counts(emoe_ctx* ctx, int32_t* out_counts, int n_experts, void* stream);
 
 /* The cache's bookkeeping alone, without a device (same code as behind the calls above): for
  * checking slot assignment, eviction order and counters on a host without a GPU.

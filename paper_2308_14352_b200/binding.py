@@ -40,7 +40,7 @@ EXPORTS = (
     "emoe_set_fused_projections", "emoe_set_fused_routing", "emoe_kernels_last_forward", "emoe_set_wait_limit",
     "emoe_debug_expect_extra_completions",
     "emoe_cache_create", "emoe_register_expert", "emoe_prefetch_experts", "emoe_cache_acquire", "emoe_cache_release",
-    "emoe_cache_slot_of", "emoe_cache_get_stats", "emoe_policy_create", "emoe_policy_destroy", "emoe_policy_register",
+    "emoe_cache_slot_of", "emoe_cache_get_stats", "emoe_cache_set_timing", "emoe_last_expert_counts", "emoe_policy_create", "emoe_policy_destroy", "emoe_policy_register",
     "emoe_policy_prefetch", "emoe_policy_acquire", "emoe_policy_release", "emoe_policy_get_stats", "emoe_rank_experts",
     "emoe_build_profile2", "emoe_rank_experts2",
 )
@@ -65,7 +65,7 @@ class emoe_layer_desc(ctypes.Structure):
 class emoe_cache_stats(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in
                 ("hits", "misses", "prefetch_hits", "prefetched", "prefetch_redundant", "prefetch_refused", "evictions",
-                 "bytes_copied")]
+                 "bytes_copied", "exposed_copy_ns", "timed_acquires")]
 
     def as_dict(self):
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -123,6 +123,8 @@ def lib() -> ctypes.CDLL:
         L.emoe_cache_release.argtypes = [vp, ctypes.POINTER(i64), i32, vp]
         L.emoe_cache_slot_of.argtypes = [vp, i64]
         L.emoe_cache_get_stats.argtypes = [vp, ctypes.POINTER(emoe_cache_stats)]
+        L.emoe_cache_set_timing.argtypes = [vp, i32]
+        L.emoe_last_expert_counts.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), i32, vp]
         L.emoe_policy_create.restype = vp
         L.emoe_policy_create.argtypes = [i32, i32, i32]
         L.emoe_policy_destroy.restype = None
@@ -344,6 +346,19 @@ def emoe_cache_get_stats(ctx) -> dict:
     st = emoe_cache_stats()
     _check(lib().emoe_cache_get_stats(ctx, ctypes.byref(st)), "emoe_cache_get_stats")
     return st.as_dict()
+
+
+def emoe_cache_set_timing(ctx, enabled: bool) -> None:
+    _check(lib().emoe_cache_set_timing(ctx, int(enabled)), "emoe_cache_set_timing")
+
+
+def emoe_last_expert_counts(ctx, n_experts: int, stream=0):
+    import numpy as np
+
+    out = np.empty(n_experts, dtype=np.int32)
+    _check(lib().emoe_last_expert_counts(ctx, out.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), n_experts, stream),
+           "emoe_last_expert_counts")
+    return out
 
 
 def emoe_policy_create(n_slots: int, n_layers: int, policy: int = EVICT_FORWARD):

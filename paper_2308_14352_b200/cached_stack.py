@@ -85,7 +85,7 @@ class CachedStack:
                    for _ in range(n_layers)]
         prior = rng.random((E, E)) ** 4          # peaked rows: a few likely successors per expert
         self.prior = (prior / prior.sum(axis=1, keepdims=True)).astype(np.float32)
-        self.exposed_events: List[tuple] = []
+        self._exposed_ns_seen = 0
         self.ids = torch.empty(max_tokens, shape.top_k, dtype=torch.int32, device=self.dev)
         self.gates = torch.empty(max_tokens, shape.top_k, dtype=torch.float32, device=self.dev)
         self.bias = torch.zeros(max_tokens, E, dtype=torch.float32, device=self.dev)
@@ -129,9 +129,9 @@ class CachedStack:
     def forward_stack(self, xs: Sequence[torch.Tensor], measure: bool = False, prefetch: bool = True,
                       outputs: Optional[list] = None):
         """One pass of the token batch through all layers.  xs[l]: [T][d] bf16 on the device.
-        Returns the picks of every layer (host arrays).  With measure=True every acquire is
-        bracketed by two events on the compute stream: their distance is the time the compute
-        stream stood still for a load (the exposed copy time).  If `outputs` is a list, every
+        Returns the picks of every layer (host arrays).  With measure=True the library brackets
+        every acquire by two events on the compute stream (emoe_cache_set_timing): their distance is
+        the time the compute stream stood still for a load (the exposed copy time).  If `outputs` is a list, every
         layer appends (gates, y) of the batch to it (device copies)."""
         sh, E = self.shape, self.shape.n_experts
         T = xs[0].shape[0]
@@ -157,13 +157,8 @@ class CachedStack:
                     n = E if T > 1 else self.n_prefetch
                     B.emoe_prefetch_experts(self.ctx, [self.expert_id(l + 1, int(e)) for e in order[:n]], l, cps)
                 eids = [self.expert_id(l, e) for e in active]
-                if measure:
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record(self.compute)
+                B.emoe_cache_set_timing(self.ctx, measure)
                 acq = B.emoe_cache_acquire(self.ctx, eids, l, cs, cps)
-                if measure:
-                    e1.record(self.compute)
-                    self.exposed_events.append((e0, e1))
                 by_e = {e: acq[i] for i, e in enumerate(active)}
                 first = acq[0]
                 table = (B.emoe_expert * E)()
@@ -185,8 +180,9 @@ class CachedStack:
         return picks
 
     def exposed_ms(self) -> float:
-        """Sum of the measured compute-stream stalls since the last call (synchronises)."""
+        """Sum of the compute-stream stalls the library measured since the last call (synchronises)."""
         self.compute.synchronize()
-        ms = sum(a.elapsed_time(b) for a, b in self.exposed_events)
-        self.exposed_events = []
+        ns = B.emoe_cache_get_stats(self.ctx)["exposed_copy_ns"]
+        ms = (ns - self._exposed_ns_seen) * 1e-6
+        self._exposed_ns_seen = ns
         return ms

@@ -5,6 +5,7 @@
 #include <climits>
 #include <cstring>
 #include <new>
+#include <unordered_map>
 #include <vector>
 
 #include "common.cuh"
@@ -108,6 +109,27 @@ struct emoe_ctx {
   bool timing = false;
   unsigned wait_limit = 0;  // polls before a wait inside the int8 streaming kernel gives up (0 = its default)
   int dep_extra = 0;        // test hook: extra completions the second projection waits for
+  const int32_t* last_counts = nullptr;  // device: per-expert pair counts of the last forward call
+  int last_counts_n = 0;
+  // tensor maps by what they describe: a matrix that comes back (a cache slot, a resident expert in a
+  // new table) is not encoded again
+  struct MapKey {
+    const void* ptr;
+    int a, b, c;
+    bool operator==(const MapKey& o) const { return ptr == o.ptr && a == o.a && b == o.b && c == o.c; }
+  };
+  struct MapKeyHash {
+    size_t operator()(const MapKey& k) const {
+      size_t h = reinterpret_cast<size_t>(k.ptr) * 0x9E3779B97F4A7C15ull;
+      h ^= (static_cast<size_t>(k.a) << 40) ^ (static_cast<size_t>(k.b) << 16) ^ static_cast<size_t>(k.c);
+      return h;
+    }
+  };
+  struct MapBytes {
+    char b[128];
+    int rc;
+  };
+  std::unordered_map<MapKey, MapBytes, MapKeyHash> map_cache;
   int resident_route_ctas = -1;  // CTAs of the one-launch routing kernel the device holds at once (-1 = not asked yet)
   int kernels_last = 0;  // kernels the last forward call enqueued
   ExpertCache* cache = nullptr;  // expert cache (cache.cu), optional
@@ -138,6 +160,22 @@ int cuda_fail(emoe_ctx* ctx, cudaError_t e) {
     EMOE_CUDA(ctx, call);      \
     ++(ctx)->kernels_last;     \
   } while (0)
+
+// encode_weight_tmap / encode_scale_tmap through the context's cache (kind 0: packed weights with
+// a = N, b = K, c = bits; kind 1: scale channel with a = N, b = row bytes)
+int cached_tmap(emoe_ctx* ctx, int kind, void* out, const void* ptr, int a, int b, int c) {
+  const emoe_ctx::MapKey key{ptr, a, b, kind == 0 ? c : -1};
+  auto it = ctx->map_cache.find(key);
+  if (it == ctx->map_cache.end()) {
+    if (ctx->map_cache.size() > 16384) ctx->map_cache.clear();
+    emoe_ctx::MapBytes mb;
+    std::memset(mb.b, 0, sizeof(mb.b));
+    mb.rc = kind == 0 ? encode_weight_tmap(mb.b, ptr, a, b, c) : encode_scale_tmap(mb.b, ptr, a, b);
+    it = ctx->map_cache.emplace(key, mb).first;
+  }
+  std::memcpy(out, it->second.b, 128);
+  return it->second.rc;
+}
 
 // Device copy of a host expert table (entries + tensor maps); uploaded on `st` the first time
 // its content is seen.  *tmaps is null when the shape has no TMA path.
@@ -188,13 +226,13 @@ int get_table(emoe_ctx* ctx, const LayerDims& L, const emoe_expert* host, cudaSt
     for (int m = 0; m < nmat && maps_ok; ++m) {
       const bool first = m < nmat - 1;
       const int N = first ? L.d_ff : L.d_model, K = first ? L.d_model : L.d_ff;
-      maps_ok = encode_weight_tmap(pin_block + TABLE_MAPS_OFFSET + TMAP_BYTES * (3 * e + m), host[e].packed[m], N, K,
-                                   host[e].bits) == 0;
+      maps_ok = cached_tmap(ctx, 0, pin_block + TABLE_MAPS_OFFSET + TMAP_BYTES * (3 * e + m), host[e].packed[m], N, K,
+                            host[e].bits) == 0;
       // the scale channel's map, where its rows allow one (long rows in multiples of 16 bytes)
       const int row_bytes = (L.group > 0 ? K / L.group : 1) * ssz;
       char* smap = pin_block + TABLE_SMAPS_OFFSET + TMAP_BYTES * (3 * e + m);
       if (!aligned(host[e].scales[m], 16)) scales16 = false;
-      else if (encode_scale_tmap(smap, host[e].scales[m], N, row_bytes) != 0) std::memset(smap, 0, TMAP_BYTES);
+      else if (cached_tmap(ctx, 1, smap, host[e].scales[m], N, row_bytes, 0) != 0) std::memset(smap, 0, TMAP_BYTES);
     }
   }
   char* dev = ctx->tables_dev + slot * TABLE_BLOCK_BYTES;
@@ -292,6 +330,8 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   float* hsc = reinterpret_cast<float*>(ws + w.hsc);
   float* o_part = reinterpret_cast<float*>(ws + w.o_part);
 
+  ctx->last_counts = counts;
+  ctx->last_counts_n = L.E;
   const int32_t* ids_use = routed ? ids_in : ids;
   const float* gates_use = routed ? gates_in : gates;
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
@@ -689,6 +729,15 @@ int emoe_read_timing(emoe_ctx* ctx, float* out_first_ms, float* out_second_ms, i
 int emoe_set_dependent_launch(emoe_ctx* ctx, int enabled) {
   if (!ctx) return EMOE_ERR_INVALID_ARG;
   ctx->pdl = enabled != 0;
+  return EMOE_OK;
+}
+
+int emoe_last_expert_counts(emoe_ctx* ctx, int32_t* out_counts, int n_experts, void* stream) {
+  if (!ctx || !out_counts || !ctx->last_counts || n_experts != ctx->last_counts_n) return EMOE_ERR_INVALID_ARG;
+  EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
+  EMOE_CUDA(ctx, cudaMemcpyAsync(out_counts, ctx->last_counts, sizeof(int32_t) * n_experts, cudaMemcpyDeviceToHost,
+                                 static_cast<cudaStream_t>(stream)));
+  EMOE_CUDA(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
   return EMOE_OK;
 }
 

@@ -185,6 +185,12 @@ struct ExpertCache {
   std::vector<cudaEvent_t> ready;  // contents of the slot are complete (recorded on the copy stream)
   std::vector<cudaEvent_t> idle;   // last reader of the slot is done (recorded on the compute stream)
   std::vector<char> idle_valid;
+  // exposed-copy accounting: event pairs around the waits of acquire calls, summed on request
+  bool timing = false;
+  std::vector<cudaEvent_t> timed;  // pairs (before, after), timing enabled
+  size_t timed_used = 0;
+  double exposed_ns = 0.0;
+  long long timed_acquires = 0;
   ExpertCache(int n_slots, int n_layers, int pol) : policy(n_slots, n_layers, pol), device(0), slot_bytes(0), base(nullptr) {}
 };
 
@@ -192,6 +198,7 @@ void cache_destroy(ExpertCache* c) {
   if (!c) return;
   for (cudaEvent_t e : c->ready) cudaEventDestroy(e);
   for (cudaEvent_t e : c->idle) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->timed) cudaEventDestroy(e);
   if (c->base) cudaFree(c->base);
   delete c;
 }
@@ -320,6 +327,19 @@ int emoe_cache_acquire(emoe_ctx* ctx, const int64_t* ids, int n, int current_lay
   for (int i = 0; i < n; ++i)  // nothing is touched unless every id is known
     if (c->policy.find(ids[i]) < 0) return EMOE_ERR_INVALID_ARG;
   int rc = EMOE_OK, done = 0;
+  cudaEvent_t t_after = nullptr;
+  if (c->timing) {
+    while (c->timed.size() < c->timed_used + 2) {
+      cudaEvent_t ev;
+      err = cudaEventCreate(&ev);
+      if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
+      c->timed.push_back(ev);
+    }
+    err = cudaEventRecord(c->timed[c->timed_used], static_cast<cudaStream_t>(compute_stream));
+    if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
+    t_after = c->timed[c->timed_used + 1];
+    c->timed_used += 2;
+  }
   for (; done < n && rc == EMOE_OK; ++done) {
     const int ei = c->policy.find(ids[done]);
     int load, evicted;
@@ -338,6 +358,10 @@ int emoe_cache_acquire(emoe_ctx* ctx, const int64_t* ids, int n, int current_lay
       if (err != cudaSuccess) rc = ctx_cuda_fail(ctx, err);
     }
     if (rc == EMOE_OK) expert_pointers(c, c->policy.expert(ei), &out_experts[done]);
+  }
+  if (t_after) {  // recorded even after a failure, so that every pair of the record is complete
+    err = cudaEventRecord(t_after, static_cast<cudaStream_t>(compute_stream));
+    if (err != cudaSuccess && rc == EMOE_OK) rc = ctx_cuda_fail(ctx, err);
   }
   if (rc != EMOE_OK) {
     // all or nothing: the experts acquired so far by this call are let go again, so that a failed
@@ -377,7 +401,25 @@ int emoe_cache_slot_of(emoe_ctx* ctx, int64_t id) {
 
 int emoe_cache_get_stats(emoe_ctx* ctx, emoe_cache_stats* out) {
   if (!ctx || !ctx_cache(ctx) || !out) return EMOE_ERR_INVALID_ARG;
-  *out = ctx_cache(ctx)->policy.stats();
+  ExpertCache* c = ctx_cache(ctx);
+  for (size_t i = 0; i + 1 < c->timed_used; i += 2) {
+    cudaError_t err = cudaEventSynchronize(c->timed[i + 1]);
+    float ms = 0.0f;
+    if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, c->timed[i], c->timed[i + 1]);
+    if (err != cudaSuccess) return ctx_cuda_fail(ctx, err);
+    c->exposed_ns += static_cast<double>(ms) * 1e6;
+    ++c->timed_acquires;
+  }
+  c->timed_used = 0;
+  *out = c->policy.stats();
+  out->exposed_copy_ns = static_cast<int64_t>(c->exposed_ns + 0.5);
+  out->timed_acquires = c->timed_acquires;
+  return EMOE_OK;
+}
+
+int emoe_cache_set_timing(emoe_ctx* ctx, int enabled) {
+  if (!ctx || !ctx_cache(ctx)) return EMOE_ERR_INVALID_ARG;
+  ctx_cache(ctx)->timing = enabled != 0;
   return EMOE_OK;
 }
 

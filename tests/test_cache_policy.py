@@ -9,6 +9,11 @@ import pytest
 from oracle.cache_sim import ExpertBufferModel, build_profile2, rank_experts, rank_experts2
 from paper_2308_14352_b200 import binding as B
 
+def _bookkeeping(stats):
+    """The counters the bookkeeping model has (the library adds its timing fields)."""
+    return {k: v for k, v in stats.items() if k not in ("exposed_copy_ns", "timed_acquires")}
+
+
 RULES = [("forward", B.EVICT_FORWARD), ("printed", B.EVICT_PRINTED), ("lru", B.EVICT_LRU), ("lfu", B.EVICT_LFU),
          ("fifo", B.EVICT_FIFO)]
 
@@ -51,8 +56,8 @@ def test_random_traces_agree(rule, code, n_slots, n_layers, per_layer, seed):
                 eid = held.pop(0)
                 assert B.emoe_policy_release(h, eid) == model.release(eid)
             if step % 97 == 0:
-                assert B.emoe_policy_get_stats(h) == model.counters
-        assert B.emoe_policy_get_stats(h) == model.counters
+                assert _bookkeeping(B.emoe_policy_get_stats(h)) == model.counters
+        assert _bookkeeping(B.emoe_policy_get_stats(h)) == model.counters
         assert model.counters["evictions"] > 0
     finally:
         B.emoe_policy_destroy(h)

@@ -60,6 +60,11 @@ class HostExperts:
                    for l in range(self.n_layers) for e in range(self.shape.n_experts))
 
 
+def _bookkeeping(stats):
+    """The counters the bookkeeping model has (the library adds its timing fields)."""
+    return {k: v for k, v in stats.items() if k not in ("exposed_copy_ns", "timed_acquires")}
+
+
 def _table_from(acquired, ids_active, bits):
     """Expert table of a layer: acquired pointers for the activated experts; the other entries
     (never touched by the kernels) borrow the pointers of the first activated one."""
@@ -131,7 +136,7 @@ def test_cached_forward_matches_checker_and_model(rule, code):
                     for e in range(shape.n_experts):
                         eid = host.expert_id(ll, e)
                         assert B.emoe_cache_slot_of(ctx, eid) == model.where.get(eid, -1)
-                assert B.emoe_cache_get_stats(ctx) == model.counters
+                assert _bookkeeping(B.emoe_cache_get_stats(ctx)) == model.counters
                 prev_active = active
         assert worst <= output_tolerance("bf16"), worst
         st = B.emoe_cache_get_stats(ctx)
@@ -298,3 +303,64 @@ def test_cached_stack_two_layers_at_the_mixtral_shape():
         assert st["bytes_copied"] > 0 and st["hits"] + st["misses"] > 0
     finally:
         stack.close()
+
+
+def test_exposed_copy_time_is_counted_by_the_library_and_vanishes_when_everything_is_resident():
+    """Section 3.3's pipeline invariants on the library's own counter: loading on demand leaves the
+    compute stream waiting (exposed time > 0, and about the copy time of the bytes); once every
+    expert sits in a slot the same acquires cost next to nothing; nothing is counted while the
+    accounting is off."""
+    shape = inputs.LayerShape(2048, 4096, 4, 2, "relu", "softmax_renorm", 128, "f16", "bf16")
+    host = HostExperts(shape, 1, lambda l: [8, 8, 8, 8], seed=37)
+    desc = layer.make_desc(shape)
+    dev = torch.device("cuda", 0)
+    torch.zeros(1, device=dev)
+    ctx = B.emoe_create(0, B.emoe_workspace_bytes(desc, 4))
+    compute, copy = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    model = ExpertBufferModel(4, 1, "forward")
+    try:
+        B.emoe_cache_create(ctx, 4, host.slot_bytes(), 1, B.EVICT_FORWARD)
+        host.register_all(ctx, model)
+        eids = [host.expert_id(0, e) for e in range(4)]
+        B.emoe_cache_acquire(ctx, eids[:1], 0, compute.cuda_stream, copy.cuda_stream)     # accounting off
+        B.emoe_cache_release(ctx, eids[:1], compute.cuda_stream)
+        compute.synchronize()
+        st = B.emoe_cache_get_stats(ctx)
+        assert st["exposed_copy_ns"] == 0 and st["timed_acquires"] == 0
+        B.emoe_cache_set_timing(ctx, True)
+        B.emoe_cache_acquire(ctx, eids[1:], 0, compute.cuda_stream, copy.cuda_stream)     # three loads on demand
+        B.emoe_cache_release(ctx, eids[1:], compute.cuda_stream)
+        compute.synchronize()
+        st1 = B.emoe_cache_get_stats(ctx)
+        nbytes = sum(sum(host.nbytes(0, e)) for e in range(1, 4))                         # 3 x 16.9 MB
+        assert st1["timed_acquires"] == 1
+        assert st1["exposed_copy_ns"] > nbytes / 100e9 * 1e9          # no host link moves 100 GB/s
+        assert st1["exposed_copy_ns"] < 1e9
+        for _ in range(3):                                                                # everything resident now
+            B.emoe_cache_acquire(ctx, eids, 0, compute.cuda_stream, copy.cuda_stream)
+            B.emoe_cache_release(ctx, eids, compute.cuda_stream)
+        compute.synchronize()
+        st2 = B.emoe_cache_get_stats(ctx)
+        assert st2["timed_acquires"] == 4 and st2["misses"] == st1["misses"]
+        assert st2["exposed_copy_ns"] - st1["exposed_copy_ns"] < 0.05 * st1["exposed_copy_ns"]
+    finally:
+        torch.cuda.synchronize()
+        B.emoe_destroy(ctx)
+
+
+def test_tokens_per_expert_of_the_last_forward_call():
+    shape = inputs.LayerShape(512, 1024, 8, 2, "relu", "softmax_renorm", 128, "f16", "bf16")
+    bits = [8, 4, 2, 4, 8, 4, 2, 4]
+    W = inputs.expert_set(39, 0, shape)
+    Wr = inputs.router_weight(39, 0, shape.d_model, shape.n_experts, std=0.05)
+    with layer.MoELayer(shape, bits, max_tokens=200) as moe:
+        with pytest.raises(B.EmoeError):
+            B.emoe_last_expert_counts(moe.ctx, shape.n_experts)      # no forward call yet
+        moe.pack_from_host(W)
+        for T in (1, 37, 200):                                        # streaming kernels and the grouped GEMM
+            x = inputs.activations(39, T, T, shape.d_model, "bf16")
+            _, ids, _, _ = moe.forward(x, Wr)
+            counts = B.emoe_last_expert_counts(moe.ctx, shape.n_experts)
+            assert np.array_equal(counts, np.bincount(ids.reshape(-1), minlength=shape.n_experts))
+        with pytest.raises(B.EmoeError):
+            B.emoe_last_expert_counts(moe.ctx, shape.n_experts + 1)
