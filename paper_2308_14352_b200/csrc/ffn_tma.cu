@@ -40,8 +40,20 @@
 namespace emoe {
 namespace {
 
-constexpr int TMA_CONSUMER_WARPS = 4;
-constexpr int TMA_THREADS = (TMA_CONSUMER_WARPS + 1) * 32;  // + the producer warp
+// Consumer warps of a CTA: four, each with two 16-row tiles of a stage's 128 rows; or (SPLIT) eight,
+// one tile each, in CTAs that are fewer per SM but bring more consumer warps to it in all: the
+// consumers are bound by the latency of their own instruction stream, which more warps hide.
+__host__ __device__ constexpr int consumer_warps(bool split) { return split ? 8 : 4; }
+__host__ __device__ constexpr int tma_threads(bool split) { return (consumer_warps(split) + 1) * 32; }  // + the producer warp
+#ifndef EMOE_TMA_SPLIT_NT1
+#define EMOE_TMA_SPLIT_NT1 0  // 1: 8-token tiles take the eight-warp variant (as measured: slower, see consumer_warps)
+#endif
+#ifndef EMOE_TMA_SPLIT_STAGES
+#define EMOE_TMA_SPLIT_STAGES 4
+#endif
+#ifndef EMOE_TMA_SPLIT_CTAS
+#define EMOE_TMA_SPLIT_CTAS 2
+#endif
 constexpr int TMA_SCALE_BYTES = 128 * 16;                   // raw scales of a stage: 16 bytes per row
 constexpr int TMA_BOX_ROWS = 64;
 constexpr int TMA_BOX_BYTES = TMA_BOX_ROWS * 128;  // 8 KB
@@ -157,10 +169,13 @@ constexpr int META_FIRST = 1, META_LAST = 2, META_STOP = 4, META_EMPTY = 8, META
 // How long the second projection of an expert waits for its hidden vectors (polls of ~0.1 us).
 constexpr unsigned DEP_WAIT_LIMIT = 1u << 20;
 
-template <int BITS, int NT>
+template <int BITS, int NT, bool SPLIT>
 __device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int rb, int k0, int ntok,
-                                              const unsigned char* st, int warp, int lane, uint32_t bar_empty,
+                                              const unsigned char* st, int warp_full, int lane, uint32_t bar_empty,
                                               float (&tot)[2][NT][4]) {
+  // SPLIT: warps 2p and 2p+1 share the 32 rows (or the w1 / w3 tiles) that warp p owns otherwise
+  const int warp = SPLIT ? warp_full >> 1 : warp_full;
+  const int mt_own = warp_full & 1;
   constexpr int KSPAN = 1024 / BITS;  // inputs per stage (128 bytes of a row)
   constexpr int SEGS = KSPAN / 128;   // scale segments per stage
   // one token tile: offset codes (fewest instructions per code); more: exact codes (no MMAs for
@@ -232,7 +247,8 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int r
       // accumulators so that consecutive MMAs do not depend on each other; the first starts from
       // the constant's share.
 #pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
+      for (int mi = 0; mi < (SPLIT ? 1 : 2); ++mi) {
+        const int mt = SPLIT ? mt_own : mi;  // which tile; its totals live in tot[mi]
         const Raw<BITS> raw0 = lds_raw<BITS>(row_base + mt * dmt, swz, sg, t);
         const Raw<BITS> raw1 = lds_raw<BITS>(row_base + mt * dmt + 8 * 128, swz, sg, t);
         const unsigned char* sc = sc_base + mt * (dmt >> 3) + sdelta;
@@ -271,10 +287,10 @@ __device__ __forceinline__ void consume_stage(const TmaArgs& a, int phase, int r
         }
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          tot[mt][nt][0] = fmaf(s0, pa[nt][0] + pb[nt][0], tot[mt][nt][0]);
-          tot[mt][nt][1] = fmaf(s0, pa[nt][1] + pb[nt][1], tot[mt][nt][1]);
-          tot[mt][nt][2] = fmaf(s1, pa[nt][2] + pb[nt][2], tot[mt][nt][2]);
-          tot[mt][nt][3] = fmaf(s1, pa[nt][3] + pb[nt][3], tot[mt][nt][3]);
+          tot[mi][nt][0] = fmaf(s0, pa[nt][0] + pb[nt][0], tot[mi][nt][0]);
+          tot[mi][nt][1] = fmaf(s0, pa[nt][1] + pb[nt][1], tot[mi][nt][1]);
+          tot[mi][nt][2] = fmaf(s1, pa[nt][2] + pb[nt][2], tot[mi][nt][2]);
+          tot[mi][nt][3] = fmaf(s1, pa[nt][3] + pb[nt][3], tot[mi][nt][3]);
         }
       }
     }
@@ -300,15 +316,44 @@ __device__ __forceinline__ __half hidden_value(float h, int* check_word) {
   return f32_to_f16_sat(hb);
 }
 
-// results of one item pass: lane holds rows (gp, gp+8) x tokens (2t, 2t+1) of every tile
-template <int BITS, int NT>
-__device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m, int warp, int lane,
-                                           const float (&tot)[2][NT][4]) {
+// results of one item pass: lane holds rows (gp, gp+8) x tokens (2t, 2t+1) of every tile.
+// SPLIT: a warp holds one tile (tot[0]); in a gated first projection the warp with the w3 tile
+// hands its totals to the warp with the w1 tile of the same rows through shared memory (xch, one
+// slot per warp pair, guarded by a full / free pair of barriers with bounded waits).
+template <int BITS, int NT, bool SPLIT>
+__device__ __forceinline__ bool store_item(const TmaArgs& a, const StageMeta& m, int warp_full, int lane,
+                                           float (&tot)[2][NT][4], float* xch, uint32_t bar_x, int& n_exchanged,
+                                           volatile int* abort_flag) {
   const LayerDims& L = a.L;
   const int N = m.phase == 0 ? L.d_ff : L.d_model;
   const bool swiglu_in = m.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const int warp = SPLIT ? warp_full >> 1 : warp_full;
+  const int mt_own = warp_full & 1;
   const int g = lane >> 2, t = lane & 3;
   const int gp = box_row_of<BITS>(g);
+  if (SPLIT && swiglu_in) {
+    float* slot = xch + warp * (NT * 4 * 32);
+    const uint32_t full = bar_x + 8 * (2 * warp), free_ = bar_x + 8 * (2 * warp + 1);
+    const uint32_t par = n_exchanged & 1;
+    ++n_exchanged;
+    if (mt_own == 1) {  // the w3 tile: hand over, nothing to store
+      if (!mbar_wait(free_, par ^ 1, a.check_word, abort_flag)) return false;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) slot[(nt * 4 + i) * 32 + lane] = tot[0][nt][i];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full);
+      return true;
+    }
+    if (!mbar_wait(full, par, a.check_word, abort_flag)) return false;
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) tot[1][nt][i] = slot[(nt * 4 + i) * 32 + lane];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(free_);
+  }
 #pragma unroll
   for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -324,38 +369,42 @@ __device__ __forceinline__ void store_item(const TmaArgs& a, const StageMeta& m,
         }
       } else {
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
+        for (int mi = 0; mi < (SPLIT ? 1 : 2); ++mi) {
+          const int mt = SPLIT ? mt_own : mi;
           const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
           if (n >= N) continue;
           if (m.phase == 0)
-            a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(fmaxf(tot[mt][nt][i], 0.0f), a.check_word);
+            a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(fmaxf(tot[mi][nt][i], 0.0f), a.check_word);
           else
-            a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + slot) * N + n] = tot[mt][nt][i];
+            a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + slot) * N + n] = tot[mi][nt][i];
         }
       }
     }
   }
+  return true;
 }
 
 // ring depth and CTAs per SM by token-tile count: more, smaller CTAs when registers allow, so
 // that every scheduler has several consumer warps to switch between
-template <int NT>
-__host__ __device__ constexpr int stages_for() { return NT == 1 ? EMOE_TMA_STAGES_NT1 : 3; }
-template <int NT>
-__host__ __device__ constexpr int ctas_per_sm_for() { return NT == 1 ? EMOE_TMA_CTAS_NT1 : (NT == 2 ? 2 : 1); }
+template <int NT, bool SPLIT>
+__host__ __device__ constexpr int stages_for() { return SPLIT ? EMOE_TMA_SPLIT_STAGES : (NT == 1 ? EMOE_TMA_STAGES_NT1 : 3); }
+template <int NT, bool SPLIT>
+__host__ __device__ constexpr int ctas_per_sm_for() { return SPLIT ? EMOE_TMA_SPLIT_CTAS : (NT == 1 ? EMOE_TMA_CTAS_NT1 : (NT == 2 ? 2 : 1)); }
 
-template <int NT>
+template <int NT, bool SPLIT>
 __host__ __device__ constexpr int smem_bytes_for() {
-  return stages_for<NT>() * stage_bytes_for(NT) + 1024;  // + slack to align the base to 1024
+  return stages_for<NT, SPLIT>() * stage_bytes_for(NT) + 1024;  // + slack to align the base to 1024
 }
 
-template <int NT>
-__global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_kernel(const __grid_constant__ TmaArgs a) {
-  constexpr int STAGES = stages_for<NT>();
+template <int NT, bool SPLIT>
+__global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>()) ffn_tma_kernel(const __grid_constant__ TmaArgs a) {
+  constexpr int TMA_CONSUMER_WARPS = consumer_warps(SPLIT);
+  constexpr int STAGES = stages_for<NT, SPLIT>();
   constexpr int STAGE_BYTES = stage_bytes_for(NT);
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * STAGES];  // full, empty
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 8];  // full, empty; SPLIT: (full, free) per warp pair of the w3 -> w1 hand-over
   __shared__ __align__(16) StageMeta meta[STAGES];
+  __shared__ float xch[SPLIT ? 4 * NT * 4 * 32 : 1];
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -367,6 +416,7 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
       mbar_init(smem_u32(bars + s), 33);  // full: lane 0's arrival (+ bulk-copy bytes) and every lane's scale copies
       mbar_init(smem_u32(bars + STAGES + s), TMA_CONSUMER_WARPS);  // empty: one arrival per consumer warp
     }
+    for (int i = 0; i < 8; ++i) mbar_init(smem_u32(bars + 2 * STAGES + i), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // Token rows of a stage that no copy fills keep whatever shared memory held.  That is
@@ -469,6 +519,15 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
           const uint32_t full = bar_full + 8 * stage;
           const int k0 = (step_begin + s) * kspan;
           const int klen = nsteps > 0 ? min(kspan, K - k0) : 0;
+          // Lanes 30 and 31 start the two weight boxes at once; lane 0 writes the record and announces
+          // the bytes.  The order among them is free: the stage cannot complete before all 33
+          // arrivals are in, and the byte count may run ahead of its announcement.
+          if (klen > 0 && lane >= 30) {
+            const int c0 = k0 * bits / 8;
+            const int bx = lane - 30;
+            if (swiglu_in) tma_load_2d(smem_u32(st + bx * TMA_BOX_BYTES), maps + bx, c0, row0, full);
+            else tma_load_2d(smem_u32(st + bx * TMA_BOX_BYTES), maps + mat_first, c0, row0 + bx * TMA_BOX_ROWS, full);
+          }
           if (lane == 0) {
             const int flags = (s == 0 ? META_FIRST : 0) | (s == nst - 1 ? META_LAST : 0) | (klen == 0 ? META_EMPTY : 0) |
                               (fused && phase == 0 && s == nst - 1 && pass == npass - 1 ? META_DONE : 0);
@@ -477,19 +536,8 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
             mq[0] = make_uint4(e, rb, z, begin);
             mq[1] = make_uint4(p0, ntok, k0, bits);
             mq[2] = make_uint4(flags, phase, ai, 0);
-            if (klen > 0) {
-              mbar_expect_tx(full, 2 * TMA_BOX_BYTES + ntok * klen * 2);
-              const int c0 = k0 * bits / 8;
-              if (swiglu_in) {
-                tma_load_2d(smem_u32(st), maps + 0, c0, row0, full);
-                tma_load_2d(smem_u32(st + TMA_BOX_BYTES), maps + 1, c0, row0, full);
-              } else {
-                tma_load_2d(smem_u32(st), maps + mat_first, c0, row0, full);
-                tma_load_2d(smem_u32(st + TMA_BOX_BYTES), maps + mat_first, c0, row0 + TMA_BOX_ROWS, full);
-              }
-            } else {
-              mbar_arrive(full);
-            }
+            if (klen > 0) mbar_expect_tx(full, 2 * TMA_BOX_BYTES + ntok * klen * 2);
+            else mbar_arrive(full);
           }
           __syncwarp();
           if (klen > 0) {
@@ -514,7 +562,9 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
               // in the making on other SMs.  Every lane acquires the counter itself, so that its
               // own copies below are ordered behind the writers' stores.
               need_dep = false;
-              const int expect = a.row_blocks[0] * TMA_CONSUMER_WARPS;
+              // every consumer warp that stores hidden values counts once per item (SPLIT, gated layer: the
+              // warps with the w1 tiles only)
+              const int expect = a.row_blocks[0] * ((SPLIT && L.act == EMOE_ACT_SWIGLU) ? 4 : TMA_CONSUMER_WARPS);
               const int* done = &recs[ai].done;
               bool ready = false;
               for (unsigned i = 0; i < DEP_WAIT_LIMIT; ++i) {
@@ -608,6 +658,8 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
   } else {
     // ---------------- consumer warps ----------------
     float tot[2][NT][4];
+    int n_exchanged = 0;
+    const uint32_t bar_x = smem_u32(bars + 2 * STAGES);
     // A finished first-projection item is counted one stage late: by then its stores have long
     // been acknowledged and the fence in front of the count costs nothing.  It is never held back
     // across a wait, because the stage waited for may be the one that waits for this count.
@@ -633,26 +685,29 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
       const unsigned char* st = smem + stage * STAGE_BYTES;
       if (!(m.flags & META_EMPTY)) {
         switch (m.bits) {
-          case 2: consume_stage<2, NT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
-          case 4: consume_stage<4, NT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
-          default: consume_stage<8, NT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          case 2: consume_stage<2, NT, SPLIT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          case 4: consume_stage<4, NT, SPLIT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
+          default: consume_stage<8, NT, SPLIT>(a, m.phase, m.rb, m.k0, m.ntok, st, warp, lane, bar_empty + 8 * stage, tot); break;
         }
       } else {
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_empty + 8 * stage);
       }
       if (m.flags & META_LAST) {
+        bool ok;
         switch (m.bits) {
-          case 2: store_item<2, NT>(a, m, warp, lane, tot); break;
-          case 4: store_item<4, NT>(a, m, warp, lane, tot); break;
-          default: store_item<8, NT>(a, m, warp, lane, tot); break;
+          case 2: ok = store_item<2, NT, SPLIT>(a, m, warp, lane, tot, xch, bar_x, n_exchanged, abort_flag); break;
+          case 4: ok = store_item<4, NT, SPLIT>(a, m, warp, lane, tot, xch, bar_x, n_exchanged, abort_flag); break;
+          default: ok = store_item<8, NT, SPLIT>(a, m, warp, lane, tot, xch, bar_x, n_exchanged, abort_flag); break;
         }
+        if (!ok) break;
       }
       if (pending_ai >= 0) {
         count_item_done(recs, pending_ai, lane);
         pending_ai = -1;
       }
-      if ((m.flags & META_LAST) && (m.flags & META_DONE)) pending_ai = m.ai;
+      // the warps that stored hidden values count the item (SPLIT, gated layer: not the w3 warps)
+      if ((m.flags & META_LAST) && (m.flags & META_DONE) && !(SPLIT && a.L.act == EMOE_ACT_SWIGLU && (warp & 1))) pending_ai = m.ai;
     }
     if (pending_ai >= 0) count_item_done(recs, pending_ai, lane);
   }
@@ -664,26 +719,27 @@ __global__ void __launch_bounds__(TMA_THREADS, ctas_per_sm_for<NT>()) ffn_tma_ke
   }
 }
 
-template <int NT>
+template <int NT, bool SPLIT>
 cudaError_t launch_nt(const TmaArgs& a, int max_items, cudaStream_t st) {
-  constexpr int SMEM = smem_bytes_for<NT>();
+  constexpr int SMEM = smem_bytes_for<NT, SPLIT>();
+  constexpr int TMA_THREADS = tma_threads(SPLIT);
   static int ctas_per_device[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (!ctas_per_device[dev]) {
-    e = cudaFuncSetAttribute(ffn_tma_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
+    e = cudaFuncSetAttribute(ffn_tma_kernel<NT, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
     if (e != cudaSuccess) return e;
     int per_sm = 0, sms = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ffn_tma_kernel<NT>, TMA_THREADS, SMEM);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ffn_tma_kernel<NT, SPLIT>, TMA_THREADS, SMEM);
     if (e != cudaSuccess) return e;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     ctas_per_device[dev] = (per_sm > 0 ? per_sm : 1) * sms;
   }
   const int grid = max_items < ctas_per_device[dev] ? max_items : ctas_per_device[dev];
-  return launch_chain(ffn_tma_kernel<NT>, dim3(grid), dim3(TMA_THREADS), SMEM, st, a);
+  return launch_chain(ffn_tma_kernel<NT, SPLIT>, dim3(grid), dim3(TMA_THREADS), SMEM, st, a);
 }
 
 }  // namespace
@@ -749,9 +805,9 @@ cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, c
   const long long items = active_max * per_expert;
   const int max_items = items > (1 << 30) ? (1 << 30) : static_cast<int>(items);
   const int nt = token_tiles > 0 ? token_tiles : ffn_token_tiles(L, T);
-  if (nt == 1) return launch_nt<1>(a, max_items, st);
-  if (nt == 2) return launch_nt<2>(a, max_items, st);
-  return launch_nt<4>(a, max_items, st);
+  if (nt == 1) return launch_nt<1, EMOE_TMA_SPLIT_NT1 != 0>(a, max_items, st);
+  if (nt == 2) return launch_nt<2, false>(a, max_items, st);
+  return launch_nt<4, false>(a, max_items, st);
 }
 
 // Host-side tensor-map encoder (driver entry point looked up once; no link against libcuda).
