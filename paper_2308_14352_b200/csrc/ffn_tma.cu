@@ -493,13 +493,13 @@ __global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>
       const int npass = (cnt + NT * 8 - 1) / (NT * 8);
       const int row0 = rb * pd.rows_per_item;
       bool need_dep = fused && phase == 1;
-      // scale rows of the item this lane copies (rows 4l .. 4l+3 of a stage, box-major): start
+      // scale rows of the item this lane copies (rows l, l+32, l+64, l+96 of a stage, box-major): start
       // of each row's scale channel as a byte offset from its 4-byte-aligned matrix base
       const char* srow_base[4];
       int srow_off[4];
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
-        const int row = 4 * lane + r;
+        const int row = lane + 32 * r;  // neighbouring lanes take neighbouring rows: their 4-byte copies spread over the banks
         const int n = min(swiglu_in ? row0 + (row & 63) : row0 + row, pd.N - 1);
         srow_base[r] = static_cast<const char*>(swiglu_in ? rec.scales[row >> 6] : rec.scales[mat_first]);
         srow_off[r] = n * ngroups_k * ssz;
@@ -541,7 +541,7 @@ __global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>
           }
           __syncwarp();
           if (klen > 0) {
-            // scales: lane l copies the windows of rows 4l .. 4l+3 of the stage (box-major)
+            // scales: lane l copies the windows of rows l, l+32, l+64, l+96 of the stage (box-major)
             const int nseg = klen / 128;
             const int g0 = group_of(k0, a.gshift, L.group, ngroups_k),
                       g1 = group_of(k0 + (nseg - 1) * 128, a.gshift, L.group, ngroups_k);
@@ -552,7 +552,7 @@ __global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>
               const int b1 = srow_off[r] + (g1 + 1) * ssz;
 #pragma unroll 1
               for (int w = 0; b0 + 4 * w < b1; ++w)
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + (4 * lane + r) * 16 + 4 * w),
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(sdst + (lane + 32 * r) * 16 + 4 * w),
                              "l"(srow_base[r] + b0 + 4 * w)
                              : "memory");
             }
