@@ -36,7 +36,7 @@ struct TableEntry {
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-  size_t ids, gates, counts, off, perm, slot_of_pair, plan, xs, hidden, xsc, hsc, o_part, total;
+  size_t ids, gates, counts, off, perm, slot_of_pair, plan, xs, hidden, xsc, hsc, o_part, um_scratch, um_scratch_bytes, total;
   int ksplit;
 };
 
@@ -84,6 +84,11 @@ WorkspaceLayout make_layout(const LayerDims& L, int T) {
   w.xsc = o;          o += align_up(ffn_i8_supported(L) ? P * (L.d_model / 128) * 4 : 0);
   w.hsc = o;          o += align_up(ffn_i8_supported(L) ? P * (L.d_ff / 128) * 4 : 0);
   w.o_part = o;       o += align_up(static_cast<size_t>(w.ksplit) * P * L.d_model * 4);
+  // scratch of the tcgen05 kernel's gated first projection: only calls with at least one full token tile of
+  // pairs can take that kernel's many-token shapes
+  w.um_scratch = o;
+  w.um_scratch_bytes = (ffn_umma_supported(L) && P >= 128) ? ffn_umma_scratch_bytes(L) : 0;
+  o += align_up(w.um_scratch_bytes);
   w.total = o;
   return w;
 }
@@ -329,6 +334,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   float* xsc = reinterpret_cast<float*>(ws + w.xsc);
   float* hsc = reinterpret_cast<float*>(ws + w.hsc);
   float* o_part = reinterpret_cast<float*>(ws + w.o_part);
+  float* um_scratch = w.um_scratch_bytes ? reinterpret_cast<float*>(ws + w.um_scratch) : nullptr;
 
   ctx->last_counts = counts;
   ctx->last_counts_n = L.E;
@@ -336,7 +342,8 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   const float* gates_use = routed ? gates_in : gates;
   const bool can_tma = ffn_tma_supported(L) && tmaps != nullptr;
   const bool can_i8 = ffn_i8_supported(L) && tmaps != nullptr;
-  const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr;
+  // (a gated layer needs the kernel's scratch block, which calls below one token tile of pairs do not carry)
+  const bool can_umma = ffn_umma_supported(L) && tmaps != nullptr && (L.act != EMOE_ACT_SWIGLU || um_scratch != nullptr);
   // many tokens per expert: the tcgen05 grouped GEMM; otherwise the weight-streaming kernels
   const bool many_tokens = ffn_many_tokens(L, T);
   // skewed loads: experts with few tokens stream through the TMA kernel, the others take the
@@ -406,8 +413,8 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
       EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
     }
-    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, P, ctx->check_word, st));
-    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, um_scratch, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, um_scratch, P, ctx->check_word, st));
     if (ev[1]) {  // one interval for the whole expert stage
       EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
       ctx->events_one_launch[ctx->events_used / 3 - 1] = 1;
@@ -416,9 +423,9 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   } else if (use_umma) {
     EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
-    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, um_scratch, P, ctx->check_word, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, um_scratch, P, ctx->check_word, st));
   } else if (use_i8) {
     ksplit = ffn_i8_ksplit(L, T);
     if (one_launch_route)

@@ -167,8 +167,9 @@ bool ffn_umma_supported(const LayerDims& L);
 cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, const void* x, const int32_t* ids,
                                const int32_t* perm, const int32_t* off, int* plan, void* xs16, int n_pairs,
                                int cnt_lo, int cnt_hi, int* check_word, cudaStream_t st);
+size_t ffn_umma_scratch_bytes(const LayerDims& L);  // scratch of the gated first projection (0 for other layers)
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
-                            void* hidden16, float* o, int n_pairs, int* check_word, cudaStream_t st);
+                            void* hidden16, float* o, float* scratch, int n_pairs, int* check_word, cudaStream_t st);
 
 // y[t] = sum_j gates[t][j] * sum_z o_part[z][slot_of_pair[t*k+j]]
 // o_part holds ksplit partial results, each [n_pairs_stride][d].

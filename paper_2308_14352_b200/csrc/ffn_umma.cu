@@ -2,24 +2,30 @@
 // many tokens (prefill, large decode batches).  Paper Sections 1/2.1 (each activated expert is
 // an independent FFN) on the Section 3.2 storage (b-bit codes + scale channel, w~ = q * s).
 //
-// Shape of one tile: 128 output channels (UMMA M, "swap-AB": the weight rows are the M side)
-// x a group of up to three 128-token tiles of one expert (UMMA N = 128 each, one accumulator in
-// tensor memory per token tile; two token tiles with two accumulators each for a gated first
-// projection) x all inputs.  The dequantised A stage, the expensive part, is shared by the whole
-// group: up to 384 tokens per dequantisation.
+// Shape of one work unit: 128 output channels (UMMA M, "swap-AB": the weight rows are the M side)
+// x a group of up to three 128-token tiles of one expert (one accumulator of 128 tensor-memory
+// columns per token tile, neighbouring tiles issued as one N = 256 MMA) x all inputs.  The
+// dequantised A operand, the expensive part, is shared by the whole group, and it never touches
+// shared memory: the dequantisation warps write it into TENSOR MEMORY (tcgen05.st, 32 columns per
+// 64-input stage, a ring of four stages behind the accumulators) and the MMA takes it from there
+// (the [a_tmem] operand form).  Shared memory then carries only the packed boxes and the
+// activation tiles: with A in shared memory too, the operand reads of the MMAs, the stores of the
+// dequantisation and the TMA writes together asked for more than the 128 bytes per cycle an SM
+// has, and the tensor pipe ran at a third of its rate.
 //   warp 0    TMA producer: packed code boxes (128 rows x 128 bytes, the decode kernel's tensor
 //             maps) into a 2-deep raw ring, and the tokens' activations (one box of 128 tokens x
-//             64 inputs per token tile, fp16, K-major, 128-byte swizzle) into a 2- or 3-deep operand ring;
+//             64 inputs per token tile, fp16, K-major, 128-byte swizzle) into a 4-deep ring;
 //   warps 2-9 two threads per output channel: read the channel's packed bytes from the raw ring,
 //             dequantise to fp16 (code -> exact fp16 integer by mantissa insertion, then one
 //             multiply by the group scale: |error| <= 2^-12 relative, the only approximation of
-//             this path), and write the row of the A operand in the canonical K-major
-//             swizzled layout; later the epilogue: tensor memory -> registers -> activation ->
-//             global memory;
-//   warp 1    one thread issues tcgen05.mma (M128 N128 K16, fp16 x fp16 -> fp32 in TMEM) per 16
-//             inputs and token tile and commits each stage back to the producers.
-// SwiGLU's first projection runs two accumulators (w1 and w3 rows of the same 128 channels
-// against the same activation tile), so that silu(a) * b needs no exchange between warps.
+//             this path), and store their 32 values as 16 columns of the channel's tensor-memory
+//             lane; later the epilogue: tensor memory -> registers -> activation -> global memory;
+//   warp 1    one thread issues tcgen05.mma (M128 N256/N128 K16, fp16 x fp16 -> fp32 in TMEM) per
+//             16 inputs and commits each stage back to the producers.
+// SwiGLU's first projection runs a unit twice, first against w1, then against w3 (all 384
+// accumulator columns for one matrix at a time keep the group at three token tiles): the first
+// pass parks its raw sums in a per-CTA scratch block in global memory (written and read back by
+// the same thread, L2-resident), the second pass's epilogue forms silu(a) * b.
 // Activations travel as fp16 (exact for bf16 values inside the fp16 range, saturated outside);
 // the hidden vector is rounded to bf16 first, as the definition asks, then stored as fp16.
 // The reduction index is enumerated in the order the unpack emits code pairs; the activation
@@ -38,26 +44,20 @@ namespace {
 constexpr int UM_TOK = 128;                // tokens per tile (UMMA N)
 constexpr int UM_ROWS = 128;               // output channels per tile (UMMA M)
 constexpr int UM_BK = 64;                  // inputs per operand stage: one 128-byte row of fp16
-constexpr int UM_AB_STAGES_MAX = 3;
+constexpr int UM_STAGES = 4;               // operand stages: A in tensor memory (32 columns each), B in shared memory
 constexpr int UM_RAW_STAGES = 2;
-constexpr int UM_TILE_BYTES = 128 * 128;   // a [128][64] fp16 operand tile, or a [128 rows][128 B] packed tile
-// One dequantised A stage is multiplied with a group of token tiles (each its own accumulator in
-// tensor memory), so that the dequantisation, the slowest step, is shared by up to 384 tokens
-// (256 with the two accumulators per token tile of a gated first projection).  Shared memory
-// decides the shapes: an operand stage holds the A tiles (1 or 2 matrices) and the group's B
-// tiles, a raw stage the packed tiles of 1 or 2 matrices.
-//   one matrix:   group 3, 3 operand stages of 4 tiles + 2 raw stages of 1 tile = 224 KB
-//   two matrices: group 2, 2 operand stages of 4 tiles + 2 raw stages of 2 tiles = 192 KB
-constexpr int UM_GROUP_SINGLE = 3;
-constexpr int UM_GROUP_DUAL = 2;
-constexpr int UM_STAGES_SINGLE = 3;
-constexpr int UM_STAGES_DUAL = 2;
-constexpr int UM_AB_STAGE_BYTES = 4 * UM_TILE_BYTES;
-constexpr int UM_SMEM_BYTES = 14 * UM_TILE_BYTES + 1024;
+constexpr int UM_TILE_BYTES = 128 * 128;   // a [128 tokens][64] fp16 operand tile, or a [128 rows][128 B] packed tile
+constexpr int UM_GROUP = 3;                // token tiles that share one dequantised A stage
+constexpr int UM_B_STAGE_BYTES = UM_GROUP * UM_TILE_BYTES;
+constexpr int UM_SMEM_BYTES = UM_RAW_STAGES * UM_TILE_BYTES + UM_STAGES * UM_B_STAGE_BYTES + 1024;  // 225 KB + alignment slack
+constexpr int UM_ACC_COLS = UM_GROUP * UM_TOK;  // accumulators: tensor-memory columns 0 .. 383
+constexpr int UM_A_COLS = UM_BK / 2;             // one A stage: 64 fp16 inputs = 32 columns; stages at 384, 416, 448, 480
+constexpr int UM_MAX_CTAS = 160;                 // grid limit (one CTA per SM): sizes the scratch of the gated first projection
 #ifndef EMOE_UM_UNPACK_WARPS
 #define EMOE_UM_UNPACK_WARPS 8
 #endif
-constexpr int UM_UNPACK_WARPS = EMOE_UM_UNPACK_WARPS;  // 8 or 16: two or four threads per output channel
+constexpr int UM_UNPACK_WARPS = EMOE_UM_UNPACK_WARPS;  // two threads per output channel
+static_assert(UM_UNPACK_WARPS == 8, "a thread stores its 32 values as one 16-column block of tensor memory");
 constexpr int UM_PARTS = UM_UNPACK_WARPS / 4;            // each dequantises its share of a stage and reads its share of the columns
 constexpr int UM_THREADS = (2 + UM_UNPACK_WARPS) * 32;
 constexpr int UM_TMEM_COLS = 512;
@@ -156,6 +156,7 @@ struct UmmaArgs {
   const int* plan;           // header + PlanRec per activated expert
   __half* hidden16;          // first projection's output (fp16, pair order)
   float* o;                  // second projection's output [n_pairs][d_model]
+  float* scratch;            // gated first projection: [gridDim.x][384 token columns][128 channels] raw sums of the w1 pass
   int* check_word;
 };
 
@@ -207,20 +208,21 @@ struct TileWalk {
 __global__ void __launch_bounds__(UM_THREADS, 1)
     ffn_umma_kernel(const UmmaArgs a, const __grid_constant__ CUtensorMap tmap_b) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * UM_RAW_STAGES + 3 * UM_AB_STAGES_MAX + 2];
+  __shared__ __align__(8) uint64_t bars[2 * UM_RAW_STAGES + 3 * UM_STAGES + 2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_word;
   volatile int* abort_flag = &abort_word;
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* raw_ring = smem;
+  unsigned char* b_ring = smem + UM_RAW_STAGES * UM_TILE_BYTES;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
   const uint32_t bar_raw_full = smem_u32(bars);
   const uint32_t bar_raw_empty = smem_u32(bars + UM_RAW_STAGES);
   const uint32_t bar_b_full = smem_u32(bars + 2 * UM_RAW_STAGES);
-  const uint32_t bar_a_full = smem_u32(bars + 2 * UM_RAW_STAGES + UM_AB_STAGES_MAX);
-  const uint32_t bar_ab_empty = smem_u32(bars + 2 * UM_RAW_STAGES + 2 * UM_AB_STAGES_MAX);
-  const uint32_t bar_acc_full = smem_u32(bars + 2 * UM_RAW_STAGES + 3 * UM_AB_STAGES_MAX);
+  const uint32_t bar_a_full = smem_u32(bars + 2 * UM_RAW_STAGES + UM_STAGES);
+  const uint32_t bar_ab_empty = smem_u32(bars + 2 * UM_RAW_STAGES + 2 * UM_STAGES);
+  const uint32_t bar_acc_full = smem_u32(bars + 2 * UM_RAW_STAGES + 3 * UM_STAGES);
   const uint32_t bar_acc_empty = bar_acc_full + 8;
 
   if (threadIdx.x == 0) {
@@ -229,7 +231,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       mbar_init(bar_raw_full + 8 * s, 1);
       mbar_init(bar_raw_empty + 8 * s, UM_UNPACK_WARPS);
     }
-    for (int s = 0; s < UM_AB_STAGES_MAX; ++s) {
+    for (int s = 0; s < UM_STAGES; ++s) {
       mbar_init(bar_b_full + 8 * s, 1);
       mbar_init(bar_a_full + 8 * s, UM_UNPACK_WARPS);
       mbar_init(bar_ab_empty + 8 * s, 1);
@@ -238,15 +240,10 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
     mbar_init(bar_acc_empty, UM_UNPACK_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {  // tensor memory for the accumulators (two of 128 columns)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                 "r"(UM_TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  if (warp == 1) tmem_alloc(smem_u32(&tmem_base_slot), UM_TMEM_COLS);  // three accumulators + four A stages
+  tc_fence_before();
   __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   pdl_wait();  // barrier set-up and the tensor-memory allocation overlap the kernel in front
   pdl_trigger();
@@ -254,19 +251,14 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
   const LayerDims& L = a.L;
   const int N = a.phase == 0 ? L.d_ff : L.d_model;
   const int K = a.phase == 0 ? L.d_model : L.d_ff;
-  const bool dual = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
-  const int n_mats = dual ? 2 : 1;
+  const bool gated = a.phase == 0 && L.act == EMOE_ACT_SWIGLU;
+  const int npass = gated ? 2 : 1;  // a gated unit runs against w1, then against w3
   const int mat_first = a.phase == 0 ? 0 : (L.act == EMOE_ACT_SWIGLU ? 2 : 1);
   const int row_blocks = (N + UM_ROWS - 1) / UM_ROWS;
   const int kb_total = K / UM_BK;
 
-  const int group_max = dual ? UM_GROUP_DUAL : UM_GROUP_SINGLE;  // token tiles that may share one dequantised A stage
-  const int ab_stages = dual ? UM_STAGES_DUAL : UM_STAGES_SINGLE;
-  const int raw_stage_bytes = n_mats * UM_TILE_BYTES;
-  unsigned char* ab_ring = smem + UM_RAW_STAGES * raw_stage_bytes;
-  const int b_off = n_mats * UM_TILE_BYTES;                   // B tiles follow the A tiles inside an operand stage
   TileWalk walk;
-  walk.init(a.plan, row_blocks, group_max);
+  walk.init(a.plan, row_blocks, UM_GROUP);
   const int group = walk.group;
   int tt, rb;
 
@@ -282,34 +274,34 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
         const int row0 = rb * UM_ROWS;
         const int tok0 = rec.begin + tt * group * UM_TOK;
         const int ntt = min(group, (rec.cnt - tt * group * UM_TOK + UM_TOK - 1) / UM_TOK);  // token tiles of this group
-        for (int kb = 0; kb < kb_total && ok;) {
-          const int rs = raw_it % UM_RAW_STAGES;
-          if (!mbar_wait(bar_raw_empty + 8 * rs, ((raw_it / UM_RAW_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
-            ok = false;
-            break;
-          }
-          const uint32_t rfull = bar_raw_full + 8 * rs;
-          mbar_expect_tx(rfull, n_mats * UM_TILE_BYTES);
-          const int c0 = (kb / kbs) * 128;
-          for (int m = 0; m < n_mats; ++m) {
-            const uint32_t dst = smem_u32(raw_ring + rs * raw_stage_bytes + m * UM_TILE_BYTES);
-            const CUtensorMap* mp = maps + (dual ? m : mat_first);
-            tma_load_2d(dst, mp, c0, row0, rfull);
-            tma_load_2d(dst + UM_TILE_BYTES / 2, mp, c0, row0 + 64, rfull);
-          }
-          ++raw_it;
-          for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb) {
-            const int s = ab_it % ab_stages;
-            if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / ab_stages) & 1) ^ 1, a.check_word, abort_flag)) {
+        for (int pass = 0; pass < npass && ok; ++pass) {
+          const CUtensorMap* mp = maps + (gated ? pass : mat_first);
+          for (int kb = 0; kb < kb_total && ok;) {
+            const int rs = raw_it % UM_RAW_STAGES;
+            if (!mbar_wait(bar_raw_empty + 8 * rs, ((raw_it / UM_RAW_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
               ok = false;
               break;
             }
-            const uint32_t bfull = bar_b_full + 8 * s;
-            mbar_expect_tx(bfull, ntt * UM_TILE_BYTES);
-            for (int j = 0; j < ntt; ++j)
-              tma_load_2d(smem_u32(ab_ring + s * UM_AB_STAGE_BYTES + b_off + j * UM_TILE_BYTES), &tmap_b, kb * UM_BK,
-                          tok0 + j * UM_TOK, bfull);
-            ++ab_it;
+            const uint32_t rfull = bar_raw_full + 8 * rs;
+            mbar_expect_tx(rfull, UM_TILE_BYTES);
+            const int c0 = (kb / kbs) * 128;
+            const uint32_t dst = smem_u32(raw_ring + rs * UM_TILE_BYTES);
+            tma_load_2d(dst, mp, c0, row0, rfull);
+            tma_load_2d(dst + UM_TILE_BYTES / 2, mp, c0, row0 + 64, rfull);
+            ++raw_it;
+            for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb) {
+              const int s = ab_it % UM_STAGES;
+              if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
+                ok = false;
+                break;
+              }
+              const uint32_t bfull = bar_b_full + 8 * s;
+              mbar_expect_tx(bfull, ntt * UM_TILE_BYTES);
+              for (int t = 0; t < ntt; ++t)
+                tma_load_2d(smem_u32(b_ring + s * UM_B_STAGE_BYTES + t * UM_TILE_BYTES), &tmap_b, kb * UM_BK, tok0 + t * UM_TOK,
+                            bfull);
+              ++ab_it;
+            }
           }
         }
       }
@@ -317,165 +309,189 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
   } else if (warp == 1) {
     // ---------------- MMA issuer (one lane) ----------------
     if (lane == 0) {
-      // kind::f16, fp16 x fp16 -> fp32, both operands K-major, M = 128, N = 128
+      // kind::f16, fp16 x fp16 -> fp32, A from tensor memory, B K-major from shared memory, M = 128, N = 128
       const uint32_t idesc = (1u << 4) | ((UM_TOK >> 3) << 17) | ((UM_ROWS >> 4) << 24);
-      // two neighbouring token tiles as one N = 256 MMA: the A tile is read from shared memory once
-      // for both (at N = 128 the operand reads alone take the whole shared-memory bandwidth)
+      // two neighbouring token tiles as one N = 256 MMA
       const uint32_t idesc2 = (1u << 4) | (((2 * UM_TOK) >> 3) << 17) | ((UM_ROWS >> 4) << 24);
-      int ab_it = 0, tile_it = 0;
+      int ab_it = 0, unit_it = 0;
       bool ok = true;
       while (ok && walk.next(tt, rb)) {
         const int ntt = min(group, (walk.rec.cnt - tt * group * UM_TOK + UM_TOK - 1) / UM_TOK);
-        if (!mbar_wait(bar_acc_empty, ((tile_it & 1) ^ 1), a.check_word, abort_flag)) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        for (int kb = 0; kb < kb_total; ++kb, ++ab_it) {
-          const int s = ab_it % ab_stages;
-          const uint32_t par = (ab_it / ab_stages) & 1;
-          if (!mbar_wait(bar_a_full + 8 * s, par, a.check_word, abort_flag) ||
-              !mbar_wait(bar_b_full + 8 * s, par, a.check_word, abort_flag)) {
+        for (int pass = 0; pass < npass && ok; ++pass, ++unit_it) {
+          if (!mbar_wait(bar_acc_empty, ((unit_it & 1) ^ 1), a.check_word, abort_flag)) {
             ok = false;
             break;
           }
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t st = smem_u32(ab_ring + s * UM_AB_STAGE_BYTES);
-          const uint64_t da0 = umma_desc(st), da1 = umma_desc(st + UM_TILE_BYTES);
-          // accumulator of token tile j of matrix m: columns (m * group + j) * 128; the B tiles of a
-          // group lie back to back, so tiles j and j+1 form one 256-token operand
-          for (int j = 0; j < ntt; j += 2) {
-            const bool two = j + 1 < ntt;
-            const uint64_t db = umma_desc(st + b_off + j * UM_TILE_BYTES);
-            const uint32_t acc_col = tmem_base + j * UM_TOK;
-            const uint32_t id = two ? idesc2 : idesc;
-#pragma unroll
-            for (int k4 = 0; k4 < UM_BK / 16; ++k4) {  // 16 inputs = 32 bytes = 2 descriptor units per step
-              const uint32_t acc = (kb > 0 || k4 > 0) ? 1u : 0u;
-              umma_f16(acc_col, da0 + 2 * k4, db + 2 * k4, id, acc);
-              if (dual) umma_f16(acc_col + group * UM_TOK, da1 + 2 * k4, db + 2 * k4, id, acc);
+          tc_fence_after();
+          for (int kb = 0; kb < kb_total; ++kb, ++ab_it) {
+            const int s = ab_it % UM_STAGES;
+            const uint32_t par = (ab_it / UM_STAGES) & 1;
+            if (!mbar_wait(bar_a_full + 8 * s, par, a.check_word, abort_flag) ||
+                !mbar_wait(bar_b_full + 8 * s, par, a.check_word, abort_flag)) {
+              ok = false;
+              break;
             }
+            tc_fence_after();
+            const uint32_t a_t = tmem_base + UM_ACC_COLS + s * UM_A_COLS;
+            const uint32_t bs = smem_u32(b_ring + s * UM_B_STAGE_BYTES);
+            // accumulator of token tile j: columns j * 128; the B tiles of a group lie back to back, so
+            // tiles j and j+1 form one 256-token operand
+            for (int j = 0; j < ntt; j += 2) {
+              const bool two = j + 1 < ntt;
+              const uint64_t db = umma_desc(bs + j * UM_TILE_BYTES);
+              const uint32_t acc_col = tmem_base + j * UM_TOK;
+              const uint32_t id = two ? idesc2 : idesc;
+#pragma unroll
+              for (int k4 = 0; k4 < UM_BK / 16; ++k4)  // 16 inputs: 8 columns of A, 32 bytes (2 descriptor units) of B
+                umma_f16_ts(acc_col, a_t + 8 * k4, db + 2 * k4, id, (kb > 0 || k4 > 0) ? 1u : 0u);
+            }
+            umma_commit(bar_ab_empty + 8 * s);  // the stage may be refilled once these MMAs have read it
           }
-          umma_commit(bar_ab_empty + 8 * s);  // the stage may be refilled once these MMAs have read it
+          if (ok) umma_commit(bar_acc_full);
         }
-        if (ok) umma_commit(bar_acc_full);
-        ++tile_it;
       }
     }
   } else {
-    // ---------------- dequantise (one thread per output channel), then epilogue ----------------
-    const int quarter = warp & 3;          // TMEM lanes this warp may read: 32 * quarter ...
-    const int part = (warp - 2) >> 2;      // which share of a stage's chunks (and of the token columns) is this warp's
+    // ---------------- dequantise (two threads per output channel), then epilogue ----------------
+    const int quarter = warp & 3;          // TMEM lanes this warp may access: 32 * quarter ...
+    const int part = (warp - 2) >> 2;      // which half of a stage's inputs (and of the token columns) is this warp's
     const int r = 32 * quarter + lane;     // channel of the tile = row of the operand = TMEM lane
     const int box = r >> 6, rin = r & 63;
     const int G = L.group > 0 ? L.group : K;
     const int ngroups = K / G;
     const bool sf16 = L.scale_f16 != 0;
-    int raw_it = 0, ab_it = 0, tile_it = 0;
+    const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16);
+    // scratch block of this CTA, token-column major: [384 columns][128 channels], so that the 32 lanes of a warp
+    // (32 neighbouring channels) touch 128 contiguous bytes per column
+    float* park = a.scratch + static_cast<size_t>(blockIdx.x) * UM_ROWS * UM_ACC_COLS + r;
+    int raw_it = 0, ab_it = 0, unit_it = 0;
     bool ok = true;
     while (ok && walk.next(tt, rb)) {
       const PlanRec rec = walk.rec;
       const int bits = rec.bits;
       const int kbs = (1024 / bits) / UM_BK;
       const int n = min(rb * UM_ROWS + r, N - 1);
-      const void* sp[2] = {dual ? rec.scales[0] : rec.scales[mat_first], dual ? rec.scales[1] : rec.scales[mat_first]};
       const size_t srow = static_cast<size_t>(n) * ngroups;
-      float sv[2], sv_next[2];
-      for (int m = 0; m < n_mats; ++m) sv[m] = load_scale_ro(sp[m], sf16, srow);
-      bool tiny_scale = false;  // q * s below the smallest normal fp16 number would lose bits in the fp16 operand
-      for (int kb = 0; kb < kb_total && ok;) {
-        const int rs = raw_it % UM_RAW_STAGES;
-        if (!mbar_wait(bar_raw_full + 8 * rs, (raw_it / UM_RAW_STAGES) & 1, a.check_word, abort_flag)) {
-          ok = false;
-          break;
-        }
-        for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb, ++ab_it) {
-          const int s = ab_it % ab_stages;
-          if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / ab_stages) & 1) ^ 1, a.check_word, abort_flag)) {
+      for (int pass = 0; pass < npass && ok; ++pass, ++unit_it) {
+        const void* sp = rec.scales[gated ? pass : mat_first];
+        float sv = load_scale_ro(sp, sf16, srow), sv_next;
+        bool tiny_scale = false;  // q * s below the smallest normal fp16 number would lose bits in the fp16 operand
+        for (int kb = 0; kb < kb_total && ok;) {
+          const int rs = raw_it % UM_RAW_STAGES;
+          if (!mbar_wait(bar_raw_full + 8 * rs, (raw_it / UM_RAW_STAGES) & 1, a.check_word, abort_flag)) {
             ok = false;
             break;
           }
-          const int g_next = min(((kb + 1) * UM_BK) / G, ngroups - 1);
-          for (int m = 0; m < n_mats; ++m) {
-            sv_next[m] = load_scale_ro(sp[m], sf16, srow + g_next);
-            tiny_scale |= sv[m] != 0.0f && fabsf(sv[m]) < 6.104e-5f;
-          }
-          for (int m = 0; m < n_mats; ++m) {
-            const __half sh = __float2half_rn(sv[m]);
-            const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
-            const unsigned char* rrow = raw_ring + rs * raw_stage_bytes + m * UM_TILE_BYTES + box * (UM_TILE_BYTES / 2) + rin * 128;
-            unsigned char* arow = ab_ring + s * UM_AB_STAGE_BYTES + m * UM_TILE_BYTES + r * 128;
-#pragma unroll
-            for (int pp = part * (4 / UM_PARTS); pp < (part + 1) * (4 / UM_PARTS); ++pp) {
-              uint4 o[2];
-              dequant_pair(bits, rrow, rin, j, pp, s2, o);
-              *reinterpret_cast<uint4*>(arow + (((2 * pp) ^ (r & 7)) << 4)) = o[0];
-              *reinterpret_cast<uint4*>(arow + (((2 * pp + 1) ^ (r & 7)) << 4)) = o[1];
+          const unsigned char* rrow = raw_ring + rs * UM_TILE_BYTES + box * (UM_TILE_BYTES / 2) + rin * 128;
+          for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb, ++ab_it) {
+            const int s = ab_it % UM_STAGES;
+            if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
+              ok = false;
+              break;
             }
-          }
-          for (int m = 0; m < n_mats; ++m) sv[m] = sv_next[m];
-          // generic-proxy writes of the operand must be visible to the tensor core's async reads
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_a_full + 8 * s);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_raw_empty + 8 * rs);
-        ++raw_it;
-      }
-      if (!ok) break;
-      if (tiny_scale) atomicOr(a.check_word, CHECK_F16_RANGE);
-      // ---- epilogue: this warp's 32 channels x its share of the token columns ----
-      if (!mbar_wait(bar_acc_full, tile_it & 1, a.check_word, abort_flag)) break;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int nrow = rb * UM_ROWS + r;
-      const int tok_first = tt * group * UM_TOK;
-      const int ntt = min(group, (rec.cnt - tok_first + UM_TOK - 1) / UM_TOK);
-      const int hpos = a.phase == 0 ? pair_pos_rt(bits, min(nrow, N - 1)) : 0;
-#pragma unroll 1
-      for (int jc = 0; jc < ntt * (UM_TOK / UM_PARTS / 32); ++jc) {
-        // token tile j of the group, 32 columns from cc on (this warp's share of the tile's columns)
-        const int j = jc / (UM_TOK / UM_PARTS / 32);
-        const int cc = (UM_TOK / UM_PARTS) * part + 32 * (jc % (UM_TOK / UM_PARTS / 32));
-        const int tokens = min(UM_TOK, rec.cnt - tok_first - j * UM_TOK);
-        const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tok_first) + static_cast<size_t>(j) * UM_TOK;
-        uint32_t va[32], vb[32];
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(32 * quarter) << 16) + j * UM_TOK + cc;
-        tmem_ld32(taddr, va);
-        if (dual) tmem_ld32(taddr + group * UM_TOK, vb);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (nrow < N) {
+            tc_fence_after();  // the MMAs that read this stage's columns are complete
+            const int g_next = min(((kb + 1) * UM_BK) / G, ngroups - 1);
+            sv_next = load_scale_ro(sp, sf16, srow + g_next);
+            tiny_scale |= sv != 0.0f && fabsf(sv) < 6.104e-5f;
+            const __half sh = __float2half_rn(sv);
+            const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
+            uint32_t v[16];  // inputs 32 * part .. 32 * part + 31 of the stage, two per register
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (cc + j < tokens) {
-              const float x = __uint_as_float(va[j]);
-              if (a.phase == 0) {
-                float h;
-                if (dual) h = x / (1.0f + expf(-x)) * __uint_as_float(vb[j]);
-                else h = fmaxf(x, 0.0f);
-                h = __bfloat162float(__float2bfloat16_rn(h));  // the hidden vector is a bf16 tensor
-                if (beyond_f16(h)) atomicOr(a.check_word, CHECK_F16_RANGE);  // saturated below: reported, not silent
-                h = fminf(fmaxf(h, -65504.0f), 65504.0f);
-                a.hidden16[(slot0 + cc + j) * N + hpos] = __float2half_rn(h);
-              } else {
-                a.o[(slot0 + cc + j) * N + nrow] = x;
+            for (int q = 0; q < 2; ++q) {
+              uint4 o[2];
+              dequant_pair(bits, rrow, rin, j, 2 * part + q, s2, o);
+              v[8 * q + 0] = o[0].x, v[8 * q + 1] = o[0].y, v[8 * q + 2] = o[0].z, v[8 * q + 3] = o[0].w;
+              v[8 * q + 4] = o[1].x, v[8 * q + 5] = o[1].y, v[8 * q + 6] = o[1].z, v[8 * q + 7] = o[1].w;
+            }
+            tmem_st16(lane_base + UM_ACC_COLS + s * UM_A_COLS + 16 * part, v);
+            tmem_st_wait();
+            sv = sv_next;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_a_full + 8 * s);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_raw_empty + 8 * rs);
+          ++raw_it;
+        }
+        if (!ok) break;
+        if (tiny_scale) atomicOr(a.check_word, CHECK_F16_RANGE);
+        // ---- epilogue: this warp's 32 channels x its half of the token columns ----
+        if (!mbar_wait(bar_acc_full, unit_it & 1, a.check_word, abort_flag)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const int nrow = rb * UM_ROWS + r;
+        const int tok_first = tt * group * UM_TOK;
+        const int ntt = min(group, (rec.cnt - tok_first + UM_TOK - 1) / UM_TOK);
+        const int hpos = a.phase == 0 ? pair_pos_rt(bits, min(nrow, N - 1)) : 0;
+#pragma unroll 1
+        for (int jc = 0; jc < ntt * (UM_TOK / UM_PARTS / 32); ++jc) {
+          // token tile j of the group, 32 columns from cc on (this warp's share of the tile's columns)
+          const int j = jc / (UM_TOK / UM_PARTS / 32);
+          const int cc = (UM_TOK / UM_PARTS) * part + 32 * (jc % (UM_TOK / UM_PARTS / 32));
+          const int tokens = min(UM_TOK, rec.cnt - tok_first - j * UM_TOK);
+          const size_t slot0 = static_cast<size_t>(rec.begin) + static_cast<size_t>(tok_first) + static_cast<size_t>(j) * UM_TOK;
+          uint32_t va[32];
+          tmem_ld32(lane_base + j * UM_TOK + cc, va);
+          tmem_ld_wait();
+          float* pk = park + static_cast<size_t>(j * UM_TOK + cc) * UM_ROWS;
+          if (gated && pass == 0) {
+            // the w1 sums wait in the scratch block for the w3 pass of the same unit
+#pragma unroll
+            for (int c = 0; c < 32; ++c) pk[c * UM_ROWS] = __uint_as_float(va[c]);
+            continue;
+          }
+          // one compact unrolled loop per case (the conditions are uniform; a single loop with all cases
+          // inside was several times the code, fetched anew at every unit's end)
+          if (nrow >= N) continue;
+          const int live = min(32, tokens - cc);  // token columns of this chunk that exist
+          if (a.phase != 0) {
+            float* dst = a.o + (slot0 + cc) * N + nrow;
+#pragma unroll
+            for (int c = 0; c < 32; ++c)
+              if (c < live) dst[static_cast<size_t>(c) * N] = __uint_as_float(va[c]);
+          } else {
+            __half* dst = a.hidden16 + (slot0 + cc) * N + hpos;
+            bool beyond = false;
+            if (gated) {
+              float av[32];
+#pragma unroll
+              for (int c = 0; c < 32; ++c) av[c] = pk[c * UM_ROWS];  // all loads first: one round trip to L2, not 32
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                // the hidden vector is a bf16 tensor
+                const float h = __bfloat162float(__float2bfloat16_rn(av[c] / (1.0f + expf(-av[c])) * __uint_as_float(va[c])));
+                beyond |= beyond_f16(h);
+                if (c < live) dst[static_cast<size_t>(c) * N] = __float2half_rn(fminf(fmaxf(h, -65504.0f), 65504.0f));
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                const float h = __bfloat162float(__float2bfloat16_rn(fmaxf(__uint_as_float(va[c]), 0.0f)));
+                beyond |= beyond_f16(h);
+                if (c < live) dst[static_cast<size_t>(c) * N] = __float2half_rn(fminf(h, 65504.0f));
               }
             }
+            if (beyond) atomicOr(a.check_word, CHECK_F16_RANGE);  // saturated above: reported, not silent
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_acc_empty);
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_acc_empty);
-      ++tile_it;
     }
   }
 
   // wind-down: everybody meets, then the allocating warp releases tensor memory
   if (*abort_flag)
     for (int i = 0; i < 2000; ++i) __nanosleep(100);  // let copies in flight land
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(UM_TMEM_COLS) : "memory");
+    tc_fence_after();
+    tmem_dealloc(tmem_base, UM_TMEM_COLS);
   }
 }
 
@@ -551,8 +567,13 @@ cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, con
                       perm, off, L.E, plan, L.top_k, L.d_model, n_pairs, cnt_lo, cnt_hi, reinterpret_cast<__half*>(xs16), check_word);
 }
 
+size_t ffn_umma_scratch_bytes(const LayerDims& L) {
+  return L.act == EMOE_ACT_SWIGLU ? static_cast<size_t>(UM_MAX_CTAS) * UM_ROWS * UM_ACC_COLS * sizeof(float) : 0;
+}
+
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
-                            void* hidden16, float* o, int n_pairs, int* check_word, cudaStream_t st) {
+                            void* hidden16, float* o, float* scratch, int n_pairs, int* check_word, cudaStream_t st) {
+  if (phase == 0 && L.act == EMOE_ACT_SWIGLU && !scratch) return cudaErrorInvalidValue;
   const int N = phase == 0 ? L.d_ff : L.d_model;
   const int K = phase == 0 ? L.d_model : L.d_ff;
   CUtensorMap tmap_b;
@@ -573,7 +594,8 @@ cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, co
   const long long row_blocks = (N + UM_ROWS - 1) / UM_ROWS;
   // upper bound of the tile count: every pair alone in a token tile
   long long tiles = row_blocks * (static_cast<long long>(n_pairs < L.E ? n_pairs : L.E) + n_pairs / UM_TOK);
-  const int grid = static_cast<int>(tiles < sms_of_device[dev] ? tiles : sms_of_device[dev]);
+  const int cap = sms_of_device[dev] < UM_MAX_CTAS ? sms_of_device[dev] : UM_MAX_CTAS;
+  const int grid = static_cast<int>(tiles < cap ? tiles : cap);
   UmmaArgs a;
   a.phase = phase;
   a.L = L;
@@ -581,6 +603,7 @@ cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, co
   a.plan = plan;
   a.hidden16 = reinterpret_cast<__half*>(hidden16);
   a.o = o;
+  a.scratch = scratch;
   a.check_word = check_word;
   return launch_chain(ffn_umma_kernel, dim3(grid), dim3(UM_THREADS), UM_SMEM_BYTES, st, a, tmap_b);
 }

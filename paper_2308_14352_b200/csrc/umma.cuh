@@ -24,6 +24,15 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t da, uint64_t 
       : "r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// ... or A from tensor memory (row i of A in lane i, two fp16 inputs per 32-bit column)
+__device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      :
+      : "r"(d_tmem), "r"(a_tmem), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 // 8-bit integers -> int32: A from shared memory ...
 __device__ __forceinline__ void umma_i8_ss(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
