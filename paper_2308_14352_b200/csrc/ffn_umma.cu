@@ -56,8 +56,8 @@ constexpr int UM_MAX_CTAS = 160;                 // grid limit (one CTA per SM):
 #ifndef EMOE_UM_UNPACK_WARPS
 #define EMOE_UM_UNPACK_WARPS 8
 #endif
-constexpr int UM_UNPACK_WARPS = EMOE_UM_UNPACK_WARPS;  // two threads per output channel
-static_assert(UM_UNPACK_WARPS == 8, "a thread stores its 32 values as one 16-column block of tensor memory");
+constexpr int UM_UNPACK_WARPS = EMOE_UM_UNPACK_WARPS;  // two (or four) threads per output channel
+static_assert(UM_UNPACK_WARPS == 8 || UM_UNPACK_WARPS == 16, "a thread stores its 32 or 16 values as one block of 16 or 8 tensor-memory columns");
 constexpr int UM_PARTS = UM_UNPACK_WARPS / 4;            // each dequantises its share of a stage and reads its share of the columns
 constexpr int UM_THREADS = (2 + UM_UNPACK_WARPS) * 32;
 constexpr int UM_TMEM_COLS = 512;
@@ -148,6 +148,9 @@ __device__ __forceinline__ void dequant_pair(int bits, const unsigned char* rrow
     dequant_word2(pick_word(raw, pp), s2, out);
   }
 }
+
+__device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t (&r)[16]) { tmem_st16(taddr, r); }
+__device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t (&r)[8]) { tmem_st8(taddr, r); }
 
 struct UmmaArgs {
   int phase;
@@ -395,15 +398,16 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
             tiny_scale |= sv != 0.0f && fabsf(sv) < 6.104e-5f;
             const __half sh = __float2half_rn(sv);
             const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
-            uint32_t v[16];  // inputs 32 * part .. 32 * part + 31 of the stage, two per register
+            constexpr int QN = 4 / UM_PARTS;  // 16-input pieces of the stage per thread
+            uint32_t v[8 * QN];               // this thread's inputs of the stage, two per register
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
+            for (int q = 0; q < QN; ++q) {
               uint4 o[2];
-              dequant_pair(bits, rrow, rin, j, 2 * part + q, s2, o);
+              dequant_pair(bits, rrow, rin, j, QN * part + q, s2, o);
               v[8 * q + 0] = o[0].x, v[8 * q + 1] = o[0].y, v[8 * q + 2] = o[0].z, v[8 * q + 3] = o[0].w;
               v[8 * q + 4] = o[1].x, v[8 * q + 5] = o[1].y, v[8 * q + 6] = o[1].z, v[8 * q + 7] = o[1].w;
             }
-            tmem_st16(lane_base + UM_ACC_COLS + s * UM_A_COLS + 16 * part, v);
+            tmem_st_cols(lane_base + UM_ACC_COLS + s * UM_A_COLS + 8 * QN * part, v);
             tmem_st_wait();
             sv = sv_next;
             tc_fence_before();
