@@ -377,7 +377,12 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       const size_t srow = static_cast<size_t>(n) * ngroups;
       for (int pass = 0; pass < npass && ok; ++pass, ++unit_it) {
         const void* sp = rec.scales[gated ? pass : mat_first];
-        float sv = load_scale_ro(sp, sf16, srow), sv_next;
+        // scales of this step, the next one and the one after: a load has two steps to come back from L2
+        float sv = load_scale_ro(sp, sf16, srow), sv_n1 = load_scale_ro(sp, sf16, srow + min(UM_BK / G, ngroups - 1)), sv_n2;
+        // group of the step two ahead, kept by counting (a division by the group size per step was a
+        // third of the step's instructions)
+        const int spg = G / UM_BK;  // steps per scale group (G is a multiple of 128, or the whole row)
+        int g2 = 2 / spg, c2 = 2 % spg;
         bool tiny_scale = false;  // q * s below the smallest normal fp16 number would lose bits in the fp16 operand
         for (int kb = 0; kb < kb_total && ok;) {
           const int rs = raw_it % UM_RAW_STAGES;
@@ -393,8 +398,11 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
               break;
             }
             tc_fence_after();  // the MMAs that read this stage's columns are complete
-            const int g_next = min(((kb + 1) * UM_BK) / G, ngroups - 1);
-            sv_next = load_scale_ro(sp, sf16, srow + g_next);
+            sv_n2 = load_scale_ro(sp, sf16, srow + min(g2, ngroups - 1));
+            if (++c2 == spg) {
+              c2 = 0;
+              ++g2;
+            }
             tiny_scale |= sv != 0.0f && fabsf(sv) < 6.104e-5f;
             const __half sh = __float2half_rn(sv);
             const uint32_t s2 = static_cast<uint32_t>(__half_as_ushort(sh)) * 0x00010001u;
@@ -409,7 +417,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
             }
             tmem_st_cols(lane_base + UM_ACC_COLS + s * UM_A_COLS + 8 * QN * part, v);
             tmem_st_wait();
-            sv = sv_next;
+            sv = sv_n1;
+            sv_n1 = sv_n2;
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_a_full + 8 * s);
