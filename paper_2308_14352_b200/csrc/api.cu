@@ -399,7 +399,9 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     constexpr int HYBRID_STREAM_TOKENS = EMOE_HYBRID_TOKENS;
     int* plan_heavy = reinterpret_cast<int*>(reinterpret_cast<char*>(plan) + align_up(plan_bytes(L.E)));
     __nv_bfloat16* hid = reinterpret_cast<__nv_bfloat16*>(hidden);
-    ksplit = ffn_tma_ksplit(L, T);
+    // many tokens in the call: the streaming family's tail matters little, every further split-K plane costs a
+    // cleared and a re-read [P][d] fp32 array
+    ksplit = ffn_tma_ksplit(L, T) < 2 ? ffn_tma_ksplit(L, T) : 2;
     EMOE_LAUNCH(ctx, launch_scatter_x(L, table, x, ids_use, perm, off, plan, xs, nullptr, P, 1, 1, HYBRID_STREAM_TOKENS, ctx->check_word, st));
     EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan_heavy, xs, P, HYBRID_STREAM_TOKENS + 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
