@@ -136,12 +136,19 @@ struct TmaArgs {
   int gshift;         // log2(group size) if it is a power of two, else -1
   int n_pairs;
   int* check_word;
+  // floor(2^32 / d) + 1 for the divisors of the item index, per projection: n / d = umulhi(n, magic) for the
+  // small n and d met here (n * d < 2^32), instead of an integer division in front of every item's first copy
+  uint32_t mg_units[2], mg_ksplit[2], mg_rb[2];
 };
+
+__host__ __device__ inline uint32_t div_magic(uint32_t d) { return d <= 1 ? 0u : static_cast<uint32_t>((1ull << 32) / d) + 1u; }
+__device__ __forceinline__ int fast_div(int n, int d, uint32_t magic) { return d <= 1 ? n : static_cast<int>(__umulhi(static_cast<uint32_t>(n), magic)); }
 
 // what differs between the two projections
 struct PhaseDims {
   int K, N, rows_per_item, row_blocks, ksplit, mat_first;
   bool swiglu_in;
+  uint32_t mg_units, mg_ksplit, mg_rb;
 };
 __device__ __forceinline__ PhaseDims phase_dims(const TmaArgs& a, int phase) {
   PhaseDims d;
@@ -152,6 +159,9 @@ __device__ __forceinline__ PhaseDims phase_dims(const TmaArgs& a, int phase) {
   d.row_blocks = a.row_blocks[phase];
   d.ksplit = phase == 0 ? 1 : a.ksplit;
   d.mat_first = phase == 0 ? 0 : (a.L.act == EMOE_ACT_SWIGLU ? 2 : 1);
+  d.mg_units = a.mg_units[phase];
+  d.mg_ksplit = a.mg_ksplit[phase];
+  d.mg_rb = a.mg_rb[phase];
   return d;
 }
 
@@ -475,19 +485,21 @@ __global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>
       const bool swiglu_in = pd.swiglu_in;
       const int mat_first = pd.mat_first;
       const int ngroups_k = a.ngroups[phase];
-      const int ai = li / (pd.ksplit * pd.row_blocks);
+      const int ai = fast_div(li, pd.ksplit * pd.row_blocks, pd.mg_units);
       const PlanRec rec = (it == 0 && ai == ai_guess) ? rec_guess : recs[ai];
       const __half* in = phase == 0 ? a.xs : a.hidden;
-      const int z = li % pd.ksplit;
-      const int rb = (li / pd.ksplit) % pd.row_blocks;
+      const int lz = fast_div(li, pd.ksplit, pd.mg_ksplit);  // (expert, row block) index
+      const int z = li - lz * pd.ksplit;
+      const int rb = lz - fast_div(lz, pd.row_blocks, pd.mg_rb) * pd.row_blocks;
       const int e = rec.e;
       const int begin = rec.begin;
       const int cnt = rec.cnt;
       const CUtensorMap* maps = a.tmaps + static_cast<size_t>(e) * 3;
       const int bits = rec.bits;
-      const int kspan = 1024 / bits;
-      const int steps_total = (K + kspan - 1) / kspan;
-      const int spz = (steps_total + pd.ksplit - 1) / pd.ksplit;
+      const int kshift = bits == 8 ? 7 : (bits == 4 ? 8 : 9);  // log2 of the inputs per stage
+      const int kspan = 1 << kshift;
+      const int steps_total = (K + kspan - 1) >> kshift;
+      const int spz = fast_div(steps_total + pd.ksplit - 1, pd.ksplit, pd.mg_ksplit);
       const int step_begin = z * spz;
       const int nsteps = max(0, min(steps_total, step_begin + spz) - step_begin);
       const int npass = (cnt + NT * 8 - 1) / (NT * 8);
@@ -620,8 +632,9 @@ __global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>
         const int phn = item_cur < n_items0 ? 0 : 1;
         const int lin = item_cur - (phn == 0 ? 0 : n_items0);
         const PhaseDims pn = phase_dims(a, phn);
-        const PlanRec rn = recs[lin / (pn.ksplit * pn.row_blocks)];
-        const int rbn = (lin / pn.ksplit) % pn.row_blocks;
+        const PlanRec rn = recs[fast_div(lin, pn.ksplit * pn.row_blocks, pn.mg_units)];
+        const int lzn = fast_div(lin, pn.ksplit, pn.mg_ksplit);
+        const int rbn = lzn - fast_div(lzn, pn.row_blocks, pn.mg_rb) * pn.row_blocks;
         const int ngroups = a.ngroups[phn];
         const int rows = min(pn.rows_per_item, pn.N - rbn * pn.rows_per_item);
         const int lines = (rows * ngroups * ssz + 127) / 128;
@@ -798,6 +811,12 @@ cudaError_t launch_ffn_tma(int phase_begin, int phase_end, const LayerDims& L, c
     if (L.group == (1 << b)) a.gshift = b;
   a.n_pairs = n_pairs;
   a.check_word = check_word;
+  for (int p = 0; p < 2; ++p) {
+    const int ks = p == 0 ? 1 : ksplit;
+    a.mg_units[p] = div_magic(static_cast<uint32_t>(ks * a.row_blocks[p]));
+    a.mg_ksplit[p] = div_magic(static_cast<uint32_t>(ks));
+    a.mg_rb[p] = div_magic(static_cast<uint32_t>(a.row_blocks[p]));
+  }
   const long long active_max = n_pairs < L.E ? n_pairs : L.E;
   long long per_expert = 0;
   if (phase_begin == 0) per_expert += a.row_blocks[0];
