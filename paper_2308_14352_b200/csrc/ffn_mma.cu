@@ -276,12 +276,7 @@ __global__ void __launch_bounds__(128)
     }
     if (bad) atomicOr(check_word, CHECK_BAD_EXPERT_ID);
     __syncthreads();
-    if (tid == 0) {
-      for (int ee = 0; ee < E; ++ee) {
-        counts[ee] = s_off[ee + 1];
-        s_off[ee + 1] += s_off[ee];
-      }
-    }
+    if (warp == 0) counts_to_offsets(s_off, counts, E, lane);
     __syncthreads();
     for (int ee = tid; ee <= E; ee += blockDim.x) off[ee] = s_off[ee];
     if (warp == 0) build_plan(plan, experts, s_off, E, 1, 0x7fffffff, lane);

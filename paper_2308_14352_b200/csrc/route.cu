@@ -45,7 +45,7 @@ __device__ __forceinline__ void router_logits(float* smem, const void* __restric
     const int dc = min(ROUTER_DC, d - c0);
     __syncthreads();
     for (int idx = tid; idx < TT * dc; idx += ROUTER_THREADS) {
-      const int tt = idx / dc, i = idx - tt * dc;
+      const int tt = TT == 1 ? 0 : idx / dc, i = idx - tt * dc;
       const int t = t0 + tt;
       float v = 0.0f;
       if (t < T) {
@@ -259,12 +259,7 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
     __syncthreads();
     for (int q = tid; q < n_pairs; q += ROUTER_THREADS) atomicAdd(&s_off[s_ids[q] + 1], 1);
     __syncthreads();
-    if (tid == 0) {
-      for (int ee = 0; ee < E; ++ee) {
-        counts[ee] = s_off[ee + 1];
-        s_off[ee + 1] += s_off[ee];
-      }
-    }
+    if (warp == 0) counts_to_offsets(s_off, counts, E, lane);
     __syncthreads();
     for (int ee = tid; ee <= E; ee += ROUTER_THREADS) off[ee] = s_off[ee];
     if (warp == 0) build_plan(plan, experts, s_off, E, 1, 0x7fffffff, lane);

@@ -42,6 +42,27 @@ __device__ __forceinline__ void build_plan(int* plan, const ExpertDev* __restric
   }
 }
 
+// Per-expert counts -> exclusive offsets, by one warp: s_off[e + 1] holds the count of expert e on
+// entry (s_off[0] = 0) and the offset of expert e + 1 on exit; the counts go to counts_out.
+__device__ __forceinline__ void counts_to_offsets(int* s_off, int32_t* __restrict__ counts_out, int E, int lane) {
+  int carry = 0;
+  for (int e0 = 0; e0 < E; e0 += 32) {
+    const int e = e0 + lane;
+    const int c = e < E ? s_off[e + 1] : 0;
+    int incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (e < E) {
+      counts_out[e] = c;
+      s_off[e + 1] = carry + incl;
+    }
+    carry += __shfl_sync(0xffffffffu, incl, 31);
+  }
+}
+
 // One activation row into the layout of the owning expert's bitwidth (optionally as fp16).
 __device__ __forceinline__ void scatter_row(const __nv_bfloat16* __restrict__ src_row, __nv_bfloat16* __restrict__ dst_row,
                                             int d, int bits, int to_f16, int* __restrict__ check_word) {
