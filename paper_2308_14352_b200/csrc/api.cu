@@ -348,7 +348,10 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   const bool many_tokens = ffn_many_tokens(L, T);
   // skewed loads: experts with few tokens stream through the TMA kernel, the others take the
   // tcgen05 grouped GEMM, in the same forward call
-  const bool use_hybrid = can_umma && can_tma && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens));
+  // ... unless the experts hold hundreds of tokens each on average: then next to nobody is left for the streaming
+  // family, whose launch, cleared split-K plane and second plan would only cost
+  const bool dense_tokens = static_cast<double>(T) * L.top_k / L.E >= 256.0;
+  const bool use_hybrid = can_umma && can_tma && (ctx->ffn_path == 5 || (ctx->ffn_path == 0 && many_tokens && !dense_tokens));
   const bool use_umma = !use_hybrid && can_umma && (ctx->ffn_path == 4 || (ctx->ffn_path == 0 && many_tokens));
   // the weight-streaming kernels: the fp16 mma.sync one by default (the faster of the two as measured), the
   // one on int8 tcgen05 operands on request
