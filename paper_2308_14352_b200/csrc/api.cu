@@ -418,19 +418,25 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       EMOE_LAUNCH(ctx, launch_ffn_tma(0, 1, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
       EMOE_LAUNCH(ctx, launch_ffn_tma(1, 2, L, table, tmaps, xs, off, plan, hid, o_part, ksplit, P, T, EMOE_HYBRID_TILES, ctx->check_word, st));
     }
-    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, um_scratch, P, ctx->check_word, st));
-    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, um_scratch, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan_heavy, xs, hidden, o_part, um_scratch, P, 1, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan_heavy, hidden, hidden, o_part, um_scratch, P, 1, ctx->check_word, st));
     if (ev[1]) {  // one interval for the whole expert stage
       EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
       ctx->events_one_launch[ctx->events_used / 3 - 1] = 1;
       ev[2] = nullptr;
     }
   } else if (use_umma) {
+    {  // the second projection's units may be halves of the inputs, summed by the combine step like any split-K
+      int sms = 0;
+      EMOE_CUDA(ctx, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device));
+      ksplit = ffn_umma_zsplit(L, T, sms);
+      if (ksplit > w.ksplit) ksplit = w.ksplit;  // the workspace holds w.ksplit planes
+    }
     EMOE_LAUNCH(ctx, launch_scatter_x16(L, table, x, ids_use, perm, off, plan, xs, P, 1, INT_MAX, ctx->check_word, st));
     if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
-    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, um_scratch, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(0, L, tmaps, plan, xs, hidden, o_part, um_scratch, P, 1, ctx->check_word, st));
     if (ev[1]) EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
-    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, um_scratch, P, ctx->check_word, st));
+    EMOE_LAUNCH(ctx, launch_ffn_umma(1, L, tmaps, plan, hidden, hidden, o_part, um_scratch, P, ksplit, ctx->check_word, st));
   } else if (use_i8) {
     ksplit = ffn_i8_ksplit(L, T);
     if (one_launch_route)

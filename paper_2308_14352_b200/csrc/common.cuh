@@ -169,7 +169,9 @@ cudaError_t launch_scatter_x16(const LayerDims& L, const ExpertDev* experts, con
                                int cnt_lo, int cnt_hi, int* check_word, cudaStream_t st);
 size_t ffn_umma_scratch_bytes(const LayerDims& L);  // scratch of the gated first projection (0 for other layers)
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
-                            void* hidden16, float* o, float* scratch, int n_pairs, int* check_word, cudaStream_t st);
+                            void* hidden16, float* o, float* scratch, int n_pairs, int zsplit, int* check_word,
+                            cudaStream_t st);
+int ffn_umma_zsplit(const LayerDims& L, int T, int sms);  // 1 or 2 slices of the second projection's inputs per unit
 
 // y[t] = sum_j gates[t][j] * sum_z o_part[z][slot_of_pair[t*k+j]]
 // o_part holds ksplit partial results, each [n_pairs_stride][d].

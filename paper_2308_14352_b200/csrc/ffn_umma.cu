@@ -159,6 +159,8 @@ struct UmmaArgs {
   const int* plan;           // header + PlanRec per activated expert
   __half* hidden16;          // first projection's output (fp16, pair order)
   float* o;                  // second projection's output [n_pairs][d_model]
+  int zsplit;                // second projection: slices of the inputs per unit (1 or 2), slice z into plane z of o
+  size_t plane_stride;       // floats between the planes of o
   float* scratch;            // gated first projection: [gridDim.x][384 token columns][128 channels] raw sums of the w1 pass
   int* check_word;
 };
@@ -167,10 +169,11 @@ struct UmmaArgs {
 // (activated expert, group of `group` token tiles, row block) with the row block running fastest
 struct TileWalk {
   const PlanRec* recs;
-  int n_active, row_blocks, lin, a, base, group;
+  int n_active, row_blocks, lin, a, base, group, zs;
   PlanRec rec;
   int tiles_of_a;
-  __device__ __forceinline__ void init(const int* plan, int rb, int token_tiles_per_group) {
+  __device__ __forceinline__ void init(const int* plan, int rb, int token_tiles_per_group, int zsplit) {
+    zs = zsplit;
     n_active = *reinterpret_cast<const volatile int*>(plan);
     recs = reinterpret_cast<const PlanRec*>(reinterpret_cast<const char*>(plan) + PLAN_HEADER_BYTES);
     row_blocks = rb;
@@ -181,7 +184,7 @@ struct TileWalk {
     for (int g = token_tiles_per_group; g > 1; --g) {
       long long units = 0;
       for (int i = 0; i < n_active; ++i) units += (recs[i].cnt + g * UM_TOK - 1) / (g * UM_TOK);
-      if (units * rb >= static_cast<long long>(gridDim.x)) {
+      if (units * rb * zs >= static_cast<long long>(gridDim.x)) {
         group = g;
         break;
       }
@@ -192,17 +195,19 @@ struct TileWalk {
     tiles_of_a = 0;
   }
   // advances to the CTA's next tile (tt = index of its token group); false when there is none
-  __device__ __forceinline__ bool next(int& tt, int& rb) {
+  __device__ __forceinline__ bool next(int& tt, int& rb, int& z) {
     while (a < 0 || lin >= base + tiles_of_a) {
       base += tiles_of_a;
       ++a;
       if (a >= n_active) return false;
       rec = recs[a];
-      tiles_of_a = row_blocks * ((rec.cnt + group * UM_TOK - 1) / (group * UM_TOK));
+      tiles_of_a = row_blocks * zs * ((rec.cnt + group * UM_TOK - 1) / (group * UM_TOK));
     }
     const int local = lin - base;
-    tt = local / row_blocks;
-    rb = local - tt * row_blocks;
+    tt = local / (row_blocks * zs);
+    const int rz = local - tt * row_blocks * zs;  // the slices of a row block lie next to each other
+    rb = rz / zs;
+    z = rz - rb * zs;
     lin += gridDim.x;
     return true;
   }
@@ -261,16 +266,18 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
   const int kb_total = K / UM_BK;
 
   TileWalk walk;
-  walk.init(a.plan, row_blocks, UM_GROUP);
+  const int zs = a.phase == 0 ? 1 : a.zsplit;
+  const int kb_len = kb_total / zs;  // steps of a unit
+  walk.init(a.plan, row_blocks, UM_GROUP, zs);
   const int group = walk.group;
-  int tt, rb;
+  int tt, rb, z;
 
   if (warp == 0) {
     // ---------------- TMA producer (one lane) ----------------
     if (lane == 0) {
       int raw_it = 0, ab_it = 0;
       bool ok = true;
-      while (ok && walk.next(tt, rb)) {
+      while (ok && walk.next(tt, rb, z)) {
         const PlanRec rec = walk.rec;
         const CUtensorMap* maps = a.wmaps + static_cast<size_t>(rec.e) * 3;
         const int kbs = (1024 / rec.bits) / UM_BK;  // operand stages per packed box (128 bytes of a row)
@@ -279,7 +286,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
         const int ntt = min(group, (rec.cnt - tt * group * UM_TOK + UM_TOK - 1) / UM_TOK);  // token tiles of this group
         for (int pass = 0; pass < npass && ok; ++pass) {
           const CUtensorMap* mp = maps + (gated ? pass : mat_first);
-          for (int kb = 0; kb < kb_total && ok;) {
+          const int kb_end = (z + 1) * kb_len;
+          for (int kb = z * kb_len; kb < kb_end && ok;) {
             const int rs = raw_it % UM_RAW_STAGES;
             if (!mbar_wait(bar_raw_empty + 8 * rs, ((raw_it / UM_RAW_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
               ok = false;
@@ -292,7 +300,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
             tma_load_2d(dst, mp, c0, row0, rfull);
             tma_load_2d(dst + UM_TILE_BYTES / 2, mp, c0, row0 + 64, rfull);
             ++raw_it;
-            for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb) {
+            for (int j = 0; j < kbs && kb < kb_end; ++j, ++kb) {
               const int s = ab_it % UM_STAGES;
               if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
                 ok = false;
@@ -318,7 +326,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       const uint32_t idesc2 = (1u << 4) | (((2 * UM_TOK) >> 3) << 17) | ((UM_ROWS >> 4) << 24);
       int ab_it = 0, unit_it = 0;
       bool ok = true;
-      while (ok && walk.next(tt, rb)) {
+      while (ok && walk.next(tt, rb, z)) {
         const int ntt = min(group, (walk.rec.cnt - tt * group * UM_TOK + UM_TOK - 1) / UM_TOK);
         for (int pass = 0; pass < npass && ok; ++pass, ++unit_it) {
           if (!mbar_wait(bar_acc_empty, ((unit_it & 1) ^ 1), a.check_word, abort_flag)) {
@@ -326,7 +334,8 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
             break;
           }
           tc_fence_after();
-          for (int kb = 0; kb < kb_total; ++kb, ++ab_it) {
+          const int kb0 = z * kb_len;
+          for (int kb = kb0; kb < kb0 + kb_len; ++kb, ++ab_it) {
             const int s = ab_it % UM_STAGES;
             const uint32_t par = (ab_it / UM_STAGES) & 1;
             if (!mbar_wait(bar_a_full + 8 * s, par, a.check_word, abort_flag) ||
@@ -346,7 +355,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
               const uint32_t id = two ? idesc2 : idesc;
 #pragma unroll
               for (int k4 = 0; k4 < UM_BK / 16; ++k4)  // 16 inputs: 8 columns of A, 32 bytes (2 descriptor units) of B
-                umma_f16_ts(acc_col, a_t + 8 * k4, db + 2 * k4, id, (kb > 0 || k4 > 0) ? 1u : 0u);
+                umma_f16_ts(acc_col, a_t + 8 * k4, db + 2 * k4, id, (kb > kb0 || k4 > 0) ? 1u : 0u);
             }
             umma_commit(bar_ab_empty + 8 * s);  // the stage may be refilled once these MMAs have read it
           }
@@ -369,7 +378,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
     float* park = a.scratch + static_cast<size_t>(blockIdx.x) * UM_ROWS * UM_ACC_COLS + r;
     int raw_it = 0, ab_it = 0, unit_it = 0;
     bool ok = true;
-    while (ok && walk.next(tt, rb)) {
+    while (ok && walk.next(tt, rb, z)) {
       const PlanRec rec = walk.rec;
       const int bits = rec.bits;
       const int kbs = (1024 / bits) / UM_BK;
@@ -378,20 +387,23 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
       for (int pass = 0; pass < npass && ok; ++pass, ++unit_it) {
         const void* sp = rec.scales[gated ? pass : mat_first];
         // scales of this step, the next one and the one after: a load has two steps to come back from L2
-        float sv = load_scale_ro(sp, sf16, srow), sv_n1 = load_scale_ro(sp, sf16, srow + min(UM_BK / G, ngroups - 1)), sv_n2;
+        const int spg = G / UM_BK;  // steps per scale group (G is a multiple of 128, or the whole row)
+        const int kb_first = z * kb_len;
+        float sv = load_scale_ro(sp, sf16, srow + min(kb_first / spg, ngroups - 1)),
+              sv_n1 = load_scale_ro(sp, sf16, srow + min((kb_first + 1) / spg, ngroups - 1)), sv_n2;
         // group of the step two ahead, kept by counting (a division by the group size per step was a
         // third of the step's instructions)
-        const int spg = G / UM_BK;  // steps per scale group (G is a multiple of 128, or the whole row)
-        int g2 = 2 / spg, c2 = 2 % spg;
+        int g2 = (kb_first + 2) / spg, c2 = (kb_first + 2) % spg;
         bool tiny_scale = false;  // q * s below the smallest normal fp16 number would lose bits in the fp16 operand
-        for (int kb = 0; kb < kb_total && ok;) {
+        const int kb_end = (z + 1) * kb_len;
+        for (int kb = z * kb_len; kb < kb_end && ok;) {
           const int rs = raw_it % UM_RAW_STAGES;
           if (!mbar_wait(bar_raw_full + 8 * rs, (raw_it / UM_RAW_STAGES) & 1, a.check_word, abort_flag)) {
             ok = false;
             break;
           }
           const unsigned char* rrow = raw_ring + rs * UM_TILE_BYTES + box * (UM_TILE_BYTES / 2) + rin * 128;
-          for (int j = 0; j < kbs && kb < kb_total; ++j, ++kb, ++ab_it) {
+          for (int j = 0; j < kbs && kb < kb_end; ++j, ++kb, ++ab_it) {
             const int s = ab_it % UM_STAGES;
             if (!mbar_wait(bar_ab_empty + 8 * s, ((ab_it / UM_STAGES) & 1) ^ 1, a.check_word, abort_flag)) {
               ok = false;
@@ -461,7 +473,7 @@ __global__ void __launch_bounds__(UM_THREADS, 1)
           if (nrow >= N) continue;
           const int live = min(32, tokens - cc);  // token columns of this chunk that exist
           if (a.phase != 0) {
-            float* dst = a.o + (slot0 + cc) * N + nrow;
+            float* dst = a.o + z * a.plane_stride + (slot0 + cc) * N + nrow;
 #pragma unroll
             for (int c = 0; c < 32; ++c)
               if (c < live) dst[static_cast<size_t>(c) * N] = __uint_as_float(va[c]);
@@ -584,8 +596,23 @@ size_t ffn_umma_scratch_bytes(const LayerDims& L) {
   return L.act == EMOE_ACT_SWIGLU ? static_cast<size_t>(UM_MAX_CTAS) * UM_ROWS * UM_ACC_COLS * sizeof(float) : 0;
 }
 
+// Slices of the second projection's inputs per unit: two when whole units alone would leave the last round of
+// CTAs mostly idle (the estimate assumes uniform routing; the kernel is right for any routing).
+int ffn_umma_zsplit(const LayerDims& L, int T, int sms) {
+  const long long per_expert = (static_cast<long long>(T) * L.top_k + L.E - 1) / L.E;
+  const long long units = static_cast<long long>(L.E) * ((per_expert + UM_GROUP * UM_TOK - 1) / (UM_GROUP * UM_TOK)) *
+                          ((L.d_model + UM_ROWS - 1) / UM_ROWS);
+  if (sms <= 0 || units < sms) return 1;
+  const bool halves_ok = (L.d_ff / UM_BK / 2) % 8 == 0;  // a slice starts on a packed box at every width
+  // share of the CTA rounds that does work, with whole units and with halves
+  const double whole = static_cast<double>(units) / (((units + sms - 1) / sms) * sms);
+  const double halves = static_cast<double>(2 * units) / (((2 * units + sms - 1) / sms) * sms);
+  return (halves_ok && halves > whole + 0.03) ? 2 : 1;
+}
+
 cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, const int* plan, const void* in16,
-                            void* hidden16, float* o, float* scratch, int n_pairs, int* check_word, cudaStream_t st) {
+                            void* hidden16, float* o, float* scratch, int n_pairs, int zsplit, int* check_word,
+                            cudaStream_t st) {
   if (phase == 0 && L.act == EMOE_ACT_SWIGLU && !scratch) return cudaErrorInvalidValue;
   const int N = phase == 0 ? L.d_ff : L.d_model;
   const int K = phase == 0 ? L.d_model : L.d_ff;
@@ -606,7 +633,7 @@ cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, co
   }
   const long long row_blocks = (N + UM_ROWS - 1) / UM_ROWS;
   // upper bound of the tile count: every pair alone in a token tile
-  long long tiles = row_blocks * (static_cast<long long>(n_pairs < L.E ? n_pairs : L.E) + n_pairs / UM_TOK);
+  long long tiles = row_blocks * (static_cast<long long>(n_pairs < L.E ? n_pairs : L.E) + n_pairs / UM_TOK) * (phase == 1 ? zsplit : 1);
   const int cap = sms_of_device[dev] < UM_MAX_CTAS ? sms_of_device[dev] : UM_MAX_CTAS;
   const int grid = static_cast<int>(tiles < cap ? tiles : cap);
   UmmaArgs a;
@@ -617,6 +644,8 @@ cudaError_t launch_ffn_umma(int phase, const LayerDims& L, const void* wmaps, co
   a.hidden16 = reinterpret_cast<__half*>(hidden16);
   a.o = o;
   a.scratch = scratch;
+  a.zsplit = zsplit < 1 ? 1 : zsplit;
+  a.plane_stride = static_cast<size_t>(n_pairs) * L.d_model;
   a.check_word = check_word;
   return launch_chain(ffn_umma_kernel, dim3(grid), dim3(UM_THREADS), UM_SMEM_BYTES, st, a, tmap_b);
 }
