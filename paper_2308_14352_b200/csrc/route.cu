@@ -19,7 +19,9 @@ namespace emoe {
 namespace {
 
 constexpr int ROUTER_THREADS = 256;
-constexpr int ROUTER_DC = 1024;  // d_model chunk held in shared memory
+constexpr int ROUTER_DC = 1024;  // d_model chunk held in shared memory (1 and 8 tokens per CTA)
+// tokens per CTA -> chunk: 32 tokens take chunks of 256 so that their rows still fit shared memory
+__host__ __device__ constexpr int router_dc(int tt) { return tt > 8 ? 256 : ROUTER_DC; }
 
 // Logits of the CTA's TT tokens into zs[TT][EP] (shared memory).  x and the router weights are
 // inputs of the call: the logits are computed while the kernels in front drain; the wait on
@@ -28,8 +30,9 @@ template <int TT>
 __device__ __forceinline__ void router_logits(float* smem, const void* __restrict__ x, int x_bf16, int T, int d,
                                               const float* __restrict__ Wr, const float* __restrict__ bias,
                                               int bias_stride, int E, int EP, int ep_shift, float* __restrict__ logits) {
-  float* xs = smem;                          // [TT][ROUTER_DC]
-  float* red = xs + TT * ROUTER_DC;          // [S][TT][EP]
+  constexpr int DC = router_dc(TT);
+  float* xs = smem;                          // [TT][DC]
+  float* red = xs + TT * DC;                 // [S][TT][EP]
   float* zs = red + ROUTER_THREADS * TT;     // [TT][EP]
   const int tid = threadIdx.x;
   const int e = tid & (EP - 1);
@@ -41,19 +44,20 @@ __device__ __forceinline__ void router_logits(float* smem, const void* __restric
 #pragma unroll
   for (int tt = 0; tt < TT; ++tt) acc[tt] = 0.0f;
 
-  for (int c0 = 0; c0 < d; c0 += ROUTER_DC) {
-    const int dc = min(ROUTER_DC, d - c0);
+  for (int c0 = 0; c0 < d; c0 += DC) {
+    const int dc = min(DC, d - c0);
     __syncthreads();
-    for (int idx = tid; idx < TT * dc; idx += ROUTER_THREADS) {
-      const int tt = TT == 1 ? 0 : idx / dc, i = idx - tt * dc;
+    for (int tt = 0; tt < TT; ++tt) {
       const int t = t0 + tt;
-      float v = 0.0f;
-      if (t < T) {
-        const size_t src = static_cast<size_t>(t) * d + c0 + i;
-        v = x_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(x)[src])
-                   : reinterpret_cast<const float*>(x)[src];
+      for (int i = tid; i < dc; i += ROUTER_THREADS) {
+        float v = 0.0f;
+        if (t < T) {
+          const size_t src = static_cast<size_t>(t) * d + c0 + i;
+          v = x_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(x)[src])
+                     : reinterpret_cast<const float*>(x)[src];
+        }
+        xs[tt * DC + i] = v;
       }
-      xs[tt * ROUTER_DC + i] = v;
     }
     __syncthreads();
     if (e < E) {
@@ -71,7 +75,7 @@ __device__ __forceinline__ void router_logits(float* smem, const void* __restric
         for (int u = 0; u < U; ++u) {
           const int ii = min(i + u * S, dc - 1);
 #pragma unroll
-          for (int tt = 0; tt < TT; ++tt) acc[tt] = fmaf(xs[tt * ROUTER_DC + ii], w[u], acc[tt]);
+          for (int tt = 0; tt < TT; ++tt) acc[tt] = fmaf(xs[tt * DC + ii], w[u], acc[tt]);
         }
       }
     }
@@ -169,17 +173,18 @@ __global__ void __launch_bounds__(ROUTER_THREADS)
   extern __shared__ float smem[];
   pdl_trigger();
   router_logits<TT>(smem, x, x_bf16, T, d, Wr, bias, bias_stride, E, EP, ep_shift, logits);
-  const float* zs = smem + TT * ROUTER_DC + ROUTER_THREADS * TT;
+  const float* zs = smem + TT * router_dc(TT) + ROUTER_THREADS * TT;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp >= TT) return;
-  const int t = blockIdx.x * TT + warp;
-  if (t >= T) return;
-  int my_id;
-  float my_gate;
-  router_pick(zs + warp * EP, E, top_k, renorm, lane, my_id, my_gate);
-  if (lane < top_k) {
-    ids[static_cast<size_t>(t) * top_k + lane] = my_id;
-    gates[static_cast<size_t>(t) * top_k + lane] = my_gate;
+  for (int tt = warp; tt < TT; tt += ROUTER_THREADS / 32) {  // a warp per token, in turns when the CTA owns more tokens than warps
+    const int t = blockIdx.x * TT + tt;
+    if (t >= T) return;
+    int my_id;
+    float my_gate;
+    router_pick(zs + tt * EP, E, top_k, renorm, lane, my_id, my_gate);
+    if (lane < top_k) {
+      ids[static_cast<size_t>(t) * top_k + lane] = my_id;
+      gates[static_cast<size_t>(t) * top_k + lane] = my_gate;
+    }
   }
 }
 
@@ -382,7 +387,9 @@ cudaError_t launch_router_topk(const void* x, int x_bf16, int T, int d, const fl
     EP <<= 1;
     ++sh;
   }
-  // 8 tokens per CTA once there are enough tokens to fill the GPU that way, else 1
+  // 8 tokens per CTA once there are enough tokens to fill the GPU that way, else 1 (32 tokens per CTA, which
+  // would cut the re-reads of the router matrix from L2, was measured three times slower at 2048 tokens: 64 CTAs,
+  // each bound by its shared-memory reads)
   if (T >= 8 * 64) {
     constexpr int TT = 8;
     const size_t smem = sizeof(float) * (TT * ROUTER_DC + ROUTER_THREADS * TT + TT * EP);  // <= 48 KB

@@ -52,6 +52,9 @@ CASES = [
     (515, 1100, 7, 2, True, False, "tok"),         # d not a multiple of the chunk, odd E, per-token bias
     (9, 96, 1, 1, False, False, None),
     (4, 128, 8, 8, True, True, None),
+    (2048, 1024, 128, 1, False, True, "vec"),     # long batches
+    (1037, 1100, 200, 2, True, False, "tok"),      # ... ragged last CTA, d not a multiple of the chunk, E above 128
+    (1500, 4096, 8, 2, True, True, None),
 ]
 
 
