@@ -34,6 +34,9 @@ __device__ __forceinline__ void load_x8(const void* base, bool bf16, size_t idx,
   }
 }
 
+// a small integer as fp32 without the conversion unit: 1.5 * 2^23 + i has i in its low mantissa bits
+__device__ __forceinline__ float small_int_to_float(int i) { return __int_as_float(0x4B400000 + i) - 12582912.0f; }
+
 // codes 8*blk .. 8*blk+7 of a 128-bit load, as fp32 (two's-complement fields, low bits first)
 template <int BITS>
 __device__ __forceinline__ void unpack8(const uint32_t (&w)[4], int blk, float (&q)[8]);
@@ -43,20 +46,20 @@ __device__ __forceinline__ void unpack8<8>(const uint32_t (&w)[4], int blk, floa
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const uint32_t word = w[2 * blk + (i >> 2)];
-    q[i] = static_cast<float>(static_cast<int>(word << (24 - 8 * (i & 3))) >> 24);
+    q[i] = small_int_to_float(static_cast<int>(word << (24 - 8 * (i & 3))) >> 24);
   }
 }
 template <>
 __device__ __forceinline__ void unpack8<4>(const uint32_t (&w)[4], int blk, float (&q)[8]) {
   const uint32_t word = w[blk];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) q[i] = static_cast<float>(static_cast<int>(word << (28 - 4 * i)) >> 28);
+  for (int i = 0; i < 8; ++i) q[i] = small_int_to_float(static_cast<int>(word << (28 - 4 * i)) >> 28);
 }
 template <>
 __device__ __forceinline__ void unpack8<2>(const uint32_t (&w)[4], int blk, float (&q)[8]) {
   const uint32_t word = w[blk >> 1] >> (16 * (blk & 1));
 #pragma unroll
-  for (int i = 0; i < 8; ++i) q[i] = static_cast<float>(static_cast<int>(word << (30 - 2 * i)) >> 30);
+  for (int i = 0; i < 8; ++i) q[i] = small_int_to_float(static_cast<int>(word << (30 - 2 * i)) >> 30);
 }
 
 __device__ __forceinline__ float load_scale(const void* scales, bool f16, size_t idx) {
@@ -71,12 +74,14 @@ __device__ __forceinline__ void row_dot(const uint8_t* __restrict__ packed, cons
   constexpr int WPV = 128 / BITS;  // weights per 128-bit load
   const int nvec = K / WPV;
   const int ngroups = K / G;
+  const int gshift = (G & (G - 1)) == 0 ? 31 - __clz(G) : -1;  // log2(G) when G is a power of two
   const uint4* row = reinterpret_cast<const uint4*>(packed + static_cast<size_t>(n) * (static_cast<size_t>(K) * BITS / 8));
   for (int j = lane; j < nvec; j += 32) {
     const uint4 r = __ldg(row + j);
     const uint32_t w[4] = {r.x, r.y, r.z, r.w};
     const int k0 = j * WPV;
-    const float s = load_scale(scales, scale_f16, static_cast<size_t>(n) * ngroups + k0 / G);
+    const int g = ngroups == 1 ? 0 : (gshift >= 0 ? k0 >> gshift : k0 / G);
+    const float s = load_scale(scales, scale_f16, static_cast<size_t>(n) * ngroups + g);
     float part[GEMV_MTOK];
 #pragma unroll
     for (int m = 0; m < GEMV_MTOK; ++m) part[m] = 0.0f;
@@ -117,7 +122,7 @@ __device__ __forceinline__ void expert_rows(int phase, const LayerDims& L, const
 #pragma unroll
     for (int m = 0; m < GEMV_MTOK; ++m) {
       const int slot = begin + c0 + min(m, ntok - 1);
-      const size_t r = phase == 0 ? static_cast<size_t>(perm[slot] / L.top_k) : static_cast<size_t>(slot);
+      const size_t r = phase == 0 ? static_cast<size_t>(L.top_k == 1 ? perm[slot] : perm[slot] / L.top_k) : static_cast<size_t>(slot);
       const char* base = reinterpret_cast<const char*>(phase == 0 ? x : hidden);
       xrow[m] = base + r * static_cast<size_t>(K) * xsz;
     }
