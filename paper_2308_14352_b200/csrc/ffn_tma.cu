@@ -513,7 +513,9 @@ __global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>
       for (int r = 0; r < 4; ++r) {
         const int row = lane + 32 * r;  // neighbouring lanes take neighbouring rows: their 4-byte copies spread over the banks
         const int n = min(swiglu_in ? row0 + (row & 63) : row0 + row, pd.N - 1);
-        srow_base[r] = static_cast<const char*>(swiglu_in ? rec.scales[row >> 6] : rec.scales[mat_first]);
+        // constant indices only: a record indexed by a variable would live in local memory
+        const void* sc_first = mat_first == 0 ? rec.scales[0] : (mat_first == 1 ? rec.scales[1] : rec.scales[2]);
+        srow_base[r] = static_cast<const char*>(swiglu_in ? ((row >> 6) ? rec.scales[1] : rec.scales[0]) : sc_first);
         srow_off[r] = n * ngroups_k * ssz;
       }
       for (int pass = 0; pass < npass && ok; ++pass) {
@@ -641,8 +643,9 @@ __global__ void __launch_bounds__(tma_threads(SPLIT), ctas_per_sm_for<NT, SPLIT>
         const size_t offs = static_cast<size_t>(rbn) * pn.rows_per_item * ngroups * ssz;
         const int nm = pn.swiglu_in ? 2 : 1;
         for (int i = lane; i < nm * lines; i += 32) {
-          const char* base = static_cast<const char*>(rn.scales[pn.swiglu_in ? i / lines : pn.mat_first]) + offs;
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(base + static_cast<size_t>(i % lines) * 128));
+          const int second = i >= lines ? 1 : 0;  // nm is 1 or 2: no division needed
+          const char* base = static_cast<const char*>(pn.swiglu_in ? (second ? rn.scales[1] : rn.scales[0]) : (pn.mat_first == 0 ? rn.scales[0] : (pn.mat_first == 1 ? rn.scales[1] : rn.scales[2]))) + offs;
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(base + static_cast<size_t>(i - second * lines) * 128));
         }
       }
     }
