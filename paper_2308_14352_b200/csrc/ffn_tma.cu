@@ -319,12 +319,11 @@ __device__ __forceinline__ void count_item_done(PlanRec* recs, int ai, int lane)
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(&recs[ai].done), "r"(1) : "memory");
 }
 
-// the hidden vector is rounded to bf16 (the layer's activation type), then carried as fp16
-__device__ __forceinline__ __half hidden_value(float h, int* check_word) {
-  const float hb = __bfloat162float(__float2bfloat16_rn(h));
-  if (beyond_f16(hb)) atomicOr(check_word, CHECK_F16_RANGE);  // saturated below: reported, not silent
-  return f32_to_f16_sat(hb);
-}
+// the hidden vector is rounded to bf16 (the layer's activation type), then carried as fp16;
+// the same without the report: a saturated value is recognised afterwards by its bit pattern (+-65504 is
+// not a bf16 number, so a hidden value can only be there by saturation), for the positions that are stored
+__device__ __forceinline__ __half hidden_half(float h) { return f32_to_f16_sat(__bfloat162float(__float2bfloat16_rn(h))); }
+__device__ __forceinline__ bool half_saturated(__half v) { return (__half_as_ushort(v) & 0x7fffu) == 0x7bffu; }
 
 // results of one item pass: lane holds rows (gp, gp+8) x tokens (2t, 2t+1) of every tile.
 // SPLIT: a warp holds one tile (tot[0]); in a gated first projection the warp with the w3 tile
@@ -364,33 +363,66 @@ __device__ __forceinline__ bool store_item(const TmaArgs& a, const StageMeta& m,
     __syncwarp();
     if (lane == 0) mbar_arrive(free_);
   }
+  // Values first, for all positions at once (independent instruction streams), then the stores under
+  // their predicates: a position-by-position loop with early exits ran as one long dependent chain.
+  bool beyond = false;
+  if (swiglu_in) {
+    __half hv[NT][4];
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
+    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int tok = nt * 8 + 2 * t + (i & 1);
-      if (tok >= m.ntok) continue;
-      const size_t slot = static_cast<size_t>(m.begin + m.p0 + tok);
-      if (swiglu_in) {
+      for (int i = 0; i < 4; ++i) {
+        const float av = tot[0][nt][i], bv = tot[1][nt][i];
+        hv[nt][i] = hidden_half(av / (1.0f + expf(-av)) * bv);
+      }
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int tok = nt * 8 + 2 * t + (i & 1);
         const int n = m.rb * TMA_BOX_ROWS + 16 * warp + gp + 8 * (i >> 1);
-        if (n < N) {
-          const float av = tot[0][nt][i], bv = tot[1][nt][i];
-          a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(av / (1.0f + expf(-av)) * bv, a.check_word);
-        }
-      } else {
-#pragma unroll
-        for (int mi = 0; mi < (SPLIT ? 1 : 2); ++mi) {
-          const int mt = SPLIT ? mt_own : mi;
-          const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
-          if (n >= N) continue;
-          if (m.phase == 0)
-            a.hidden[slot * N + act_pos<BITS>(n)] = hidden_value(fmaxf(tot[mi][nt][i], 0.0f), a.check_word);
-          else
-            a.o_part[(static_cast<size_t>(m.z) * a.n_pairs + slot) * N + n] = tot[mi][nt][i];
+        if (tok < m.ntok && n < N) {
+          a.hidden[static_cast<size_t>(m.begin + m.p0 + tok) * N + act_pos<BITS>(n)] = hv[nt][i];
+          beyond |= half_saturated(hv[nt][i]);
         }
       }
-    }
+  } else if (m.phase == 0) {
+    __half hv[2][NT][4];
+#pragma unroll
+    for (int mi = 0; mi < (SPLIT ? 1 : 2); ++mi)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) hv[mi][nt][i] = hidden_half(fmaxf(tot[mi][nt][i], 0.0f));
+#pragma unroll
+    for (int mi = 0; mi < (SPLIT ? 1 : 2); ++mi)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int mt = SPLIT ? mt_own : mi;
+          const int tok = nt * 8 + 2 * t + (i & 1);
+          const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
+          if (tok < m.ntok && n < N) {
+            a.hidden[static_cast<size_t>(m.begin + m.p0 + tok) * N + act_pos<BITS>(n)] = hv[mi][nt][i];
+            beyond |= half_saturated(hv[mi][nt][i]);
+          }
+        }
+  } else {
+    float* plane = a.o_part + static_cast<size_t>(m.z) * a.n_pairs * N;
+#pragma unroll
+    for (int mi = 0; mi < (SPLIT ? 1 : 2); ++mi)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int mt = SPLIT ? mt_own : mi;
+          const int tok = nt * 8 + 2 * t + (i & 1);
+          const int n = m.rb * 2 * TMA_BOX_ROWS + 32 * warp + 16 * mt + gp + 8 * (i >> 1);
+          if (tok < m.ntok && n < N) plane[static_cast<size_t>(m.begin + m.p0 + tok) * N + n] = tot[mi][nt][i];
+        }
   }
+  if (beyond) atomicOr(a.check_word, CHECK_F16_RANGE);  // saturated above: reported, not silent
   return true;
 }
 
