@@ -37,7 +37,7 @@ EXPORTS = (
     "emoe_router_topk",
     "emoe_permute", "emoe_moe_forward", "emoe_moe_forward_routed", "emoe_set_ffn_path", "emoe_set_timing",
     "emoe_read_timing", "emoe_moe_forward_routed_static", "emoe_static_device_status", "emoe_set_dependent_launch",
-    "emoe_set_fused_projections", "emoe_set_fused_routing", "emoe_kernels_last_forward", "emoe_set_wait_limit",
+    "emoe_set_fused_projections", "emoe_set_fused_routing", "emoe_set_fused_layer", "emoe_kernels_last_forward", "emoe_set_wait_limit",
     "emoe_debug_expect_extra_completions",
     "emoe_cache_create", "emoe_register_expert", "emoe_prefetch_experts", "emoe_cache_acquire", "emoe_cache_release",
     "emoe_cache_slot_of", "emoe_cache_get_stats", "emoe_cache_set_timing", "emoe_last_expert_counts", "emoe_policy_create", "emoe_policy_destroy", "emoe_policy_register",
@@ -112,6 +112,7 @@ def lib() -> ctypes.CDLL:
         L.emoe_set_dependent_launch.argtypes = [vp, i32]
         L.emoe_set_fused_projections.argtypes = [vp, i32]
         L.emoe_set_fused_routing.argtypes = [vp, i32]
+        L.emoe_set_fused_layer.argtypes = [vp, i32]
         L.emoe_kernels_last_forward.argtypes = [vp]
         L.emoe_set_wait_limit.argtypes = [vp, ctypes.c_uint]
         L.emoe_debug_expect_extra_completions.argtypes = [vp, i32]
@@ -288,6 +289,10 @@ def emoe_set_fused_projections(ctx, enabled: bool) -> None:
 
 def emoe_set_fused_routing(ctx, enabled: bool) -> None:
     _check(lib().emoe_set_fused_routing(ctx, int(enabled)), "emoe_set_fused_routing")
+
+
+def emoe_set_fused_layer(ctx, enabled: bool) -> None:
+    _check(lib().emoe_set_fused_layer(ctx, int(enabled)), "emoe_set_fused_layer")
 
 
 def emoe_set_wait_limit(ctx, polls: int) -> None:

@@ -114,6 +114,9 @@ struct emoe_ctx {
   bool timing = false;
   unsigned wait_limit = 0;  // polls before a wait inside the int8 streaming kernel gives up (0 = its default)
   int dep_extra = 0;        // test hook: extra completions the second projection waits for
+  bool fuse_layer = false;  // small layer, a handful of tokens: the whole layer in one launch
+  int resident_layer_ctas = -1;  // CTAs of the one-launch layer kernel the device holds at once (-1: not asked yet)
+  int sms = 0;
   const int32_t* last_counts = nullptr;  // device: per-expert pair counts of the last forward call
   int last_counts_n = 0;
   // tensor maps by what they describe: a matrix that comes back (a cache slot, a resident expert in a
@@ -369,12 +372,21 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
   if (ctx->resident_route_ctas < 0) ctx->resident_route_ctas = route_permute_scatter_resident_ctas(ctx->device);
   const bool one_launch_route =
       ctx->fuse_routing && one_launch_permute && !routed && route_permute_scatter_supported(L, T, ctx->resident_route_ctas);
-  if (!routed && !one_launch_route)
+  // a handful of tokens on a small layer: router, both projections and the gate-weighted sum in one launch
+  bool one_launch_layer = false;
+  if (ctx->fuse_layer && ctx->ffn_path == 0 && decode_layer_supported(L, T)) {
+    if (ctx->resident_layer_ctas < 0) {
+      ctx->resident_layer_ctas = decode_layer_resident_ctas(ctx->device);
+      EMOE_CUDA(ctx, cudaDeviceGetAttribute(&ctx->sms, cudaDevAttrMultiProcessorCount, ctx->device));
+    }
+    one_launch_layer = ctx->sms > 0 && ctx->resident_layer_ctas >= 2 * ctx->sms;
+  }
+  if (!routed && !one_launch_route && !one_launch_layer)
     EMOE_LAUNCH(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,
                                       L.top_k, L.gate_mode == EMOE_GATE_SOFTMAX_RENORM, ids, gates, nullptr, st));
   unsigned* route_sync = reinterpret_cast<unsigned*>(ctx->check_word + 1);
   const unsigned route_wait = ctx->wait_limit ? ctx->wait_limit : (1u << 22);
-  if (!one_launch_permute)
+  if (!one_launch_permute && !one_launch_layer)
     EMOE_LAUNCH(ctx, launch_permute(ids_use, P, L.E, counts, off, perm, slot_of_pair, ctx->check_word, st));
   int ksplit = 1;
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -388,6 +400,21 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
     if (ctx->events_one_launch.size() < ctx->events_used / 3 + 1) ctx->events_one_launch.resize(ctx->events_used / 3 + 1);
     ctx->events_one_launch[ctx->events_used / 3] = 0;
     ctx->events_used += 3;
+  }
+  if (one_launch_layer) {
+    if (ev[0]) EMOE_CUDA(ctx, cudaEventRecord(ev[0], st));
+    EMOE_LAUNCH(ctx, launch_decode_layer(L, table, x, T, routed ? nullptr : router_W, router_bias, bias_token_stride, ids_in, gates_in,
+                                         ids, gates, counts, off, perm, slot_of_pair, hidden, y, ctx->resident_layer_ctas, ctx->sms,
+                                         reinterpret_cast<unsigned*>(ctx->check_word + 4), route_wait, ctx->dep_extra,
+                                         ctx->check_word, st));
+    if (ev[1]) {  // one interval for the whole layer
+      EMOE_CUDA(ctx, cudaEventRecord(ev[1], st));
+      ctx->events_one_launch[ctx->events_used / 3 - 1] = 1;
+    }
+    if (out_ids) EMOE_CUDA(ctx, cudaMemcpyAsync(out_ids, ids_use, sizeof(int32_t) * P, cudaMemcpyDeviceToDevice, st));
+    if (out_gates) EMOE_CUDA(ctx, cudaMemcpyAsync(out_gates, gates_use, sizeof(float) * P, cudaMemcpyDeviceToDevice, st));
+    if (out_perm) EMOE_CUDA(ctx, cudaMemcpyAsync(out_perm, perm, sizeof(int32_t) * P, cudaMemcpyDeviceToDevice, st));
+    return EMOE_OK;
   }
   if (use_hybrid) {
     // experts with up to HYBRID_STREAM_TOKENS tokens: passes of 8-token tiles through the streaming
@@ -536,8 +563,8 @@ emoe_ctx* emoe_create(int device, size_t workspace_bytes, int* status) {
   ctx->device = device;
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess && workspace_bytes > 0) e = cudaMalloc(&ctx->workspace, workspace_bytes);
-  if (e == cudaSuccess) e = cudaMalloc(&ctx->check_word, 4 * sizeof(int));  // + the routing kernel's two grid counters
-  if (e == cudaSuccess) e = cudaMemset(ctx->check_word, 0, 4 * sizeof(int));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->check_word, 8 * sizeof(int));  // + the grid counters of the routing kernel (2) and of the one-launch layer (3)
+  if (e == cudaSuccess) e = cudaMemset(ctx->check_word, 0, 8 * sizeof(int));
   if (e == cudaSuccess) e = cudaMallocHost(&ctx->check_host, sizeof(int));
   if (e == cudaSuccess) e = cudaMalloc(&ctx->tables_dev, TABLE_BLOCK_BYTES * MAX_TABLES);
   if (e == cudaSuccess) e = cudaMallocHost(&ctx->tables_pin, TABLE_BLOCK_BYTES * MAX_TABLES);
@@ -586,7 +613,7 @@ int emoe_device_status(emoe_ctx* ctx, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   EMOE_CUDA(ctx, cudaSetDevice(ctx->device));
   EMOE_CUDA(ctx, cudaMemcpyAsync(ctx->check_host, ctx->check_word, sizeof(int), cudaMemcpyDeviceToHost, st));
-  EMOE_CUDA(ctx, cudaMemsetAsync(ctx->check_word, 0, 4 * sizeof(int), st));  // also the grid counters a timed-out wait left behind
+  EMOE_CUDA(ctx, cudaMemsetAsync(ctx->check_word, 0, 8 * sizeof(int), st));  // also the grid counters a timed-out wait left behind
   EMOE_CUDA(ctx, cudaStreamSynchronize(st));
   if (*ctx->check_host & CHECK_WAIT_TIMEOUT) return EMOE_ERR_TIMEOUT;
   if (*ctx->check_host & CHECK_BAD_EXPERT_ID) return EMOE_ERR_DEVICE_CHECK;
@@ -770,6 +797,12 @@ int emoe_set_fused_projections(emoe_ctx* ctx, int enabled) {
 int emoe_set_fused_routing(emoe_ctx* ctx, int enabled) {
   if (!ctx) return EMOE_ERR_INVALID_ARG;
   ctx->fuse_routing = enabled != 0;
+  return EMOE_OK;
+}
+
+int emoe_set_fused_layer(emoe_ctx* ctx, int enabled) {
+  if (!ctx) return EMOE_ERR_INVALID_ARG;
+  ctx->fuse_layer = enabled != 0;
   return EMOE_OK;
 }
 

@@ -1,0 +1,369 @@
+// A whole MoE layer in ONE launch for a handful of tokens on a small layer (paper Sections 2.1 and
+// 3.2: router, Top-K, the activated experts' FFNs on their packed codes, gate-weighted sum; the
+// paper's target is single-request decoding, where every step of the layer is a few microseconds
+// of work and the launches and dependencies between kernels are most of the time).
+//
+// The grid is resident at once (the host sizes it from the device's capacity), so its CTAs may
+// wait for one another; every such wait is bounded.
+//   1. CTA t < T computes token t's logits and picks (the device functions of the router kernel)
+//      and counts itself in; every CTA waits until all T have done so and reads the picks.
+//   2. First projection: one warp per (pair, hidden channel) streams the packed row with 128-bit
+//      loads, decodes in registers, accumulates in fp32 and stores the activated value in the
+//      activation type.  The CTAs then meet at a grid-wide arrival counter.
+//   3. Second projection and gate-weighted sum: four warps share one (token, output channel),
+//      each takes a quarter of the hidden axis of every expert of the token; the quarters are
+//      added in a fixed order, so the result does not depend on timing.
+// CTA 0 also writes the bookkeeping the library keeps per call (counts, offsets, permutation).
+// sync[0] counts the routing arrivals, sync[1] the arrivals after the first projection, sync[2]
+// the departures; the last CTA to leave sets all three back to zero for the next launch.
+#include "common.cuh"
+#include "router.cuh"
+
+namespace emoe {
+namespace {
+
+constexpr int DL_THREADS = ROUTER_THREADS;
+constexpr int DL_WARPS = DL_THREADS / 32;
+constexpr int DL_MAX_PAIRS = 16;
+constexpr int DL_WPR = 4;                    // warps per output row in the second projection
+constexpr int DL_ROWS = DL_WARPS / DL_WPR;   // output rows a CTA works on at a time
+constexpr long long DL_MAX_WEIGHTS = 8LL << 20;  // per matrix: beyond this a layer is bandwidth-bound and streams better
+
+struct DecodeLayerArgs {
+  LayerDims L;
+  const ExpertDev* experts;
+  const void* x;
+  int T;
+  const float* Wr;       // null: the picks are given (ids_in / gates_in)
+  const float* bias;
+  int bias_stride, EP, ep_shift, renorm;
+  const int32_t* ids_in;
+  const float* gates_in;
+  int32_t* ids;
+  float* gates;
+  int32_t *counts, *off, *perm, *slot_of_pair;
+  void* hidden;  // [pairs][d_ff], activation type
+  float* y;      // [T][d_model]
+  unsigned* sync;
+  unsigned wait_limit;
+  int extra_arrivals;  // test hook: arrivals the grid-wide wait expects beyond the grid's CTAs
+  int* check_word;
+};
+
+// 8 consecutive activations as fp32
+__device__ __forceinline__ void x8(const void* row, bool bf16, int k, bool coherent, float (&v)[8]) {
+  if (bf16) {
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(row) + k);
+    const uint4 r = coherent ? __ldcg(p) : __ldg(p);
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  } else {
+    const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(row) + k);
+    const float4 a = coherent ? __ldcg(p) : __ldg(p);
+    const float4 b = coherent ? __ldcg(p + 1) : __ldg(p + 1);
+    v[0] = a.x, v[1] = a.y, v[2] = a.z, v[3] = a.w;
+    v[4] = b.x, v[5] = b.y, v[6] = b.z, v[7] = b.w;
+  }
+}
+
+// The lane's share of  sum_k q[k] * s[k / G] * x[k]  over the 128-bit words j0 .. j1-1 of one packed
+// row (two's-complement fields, low bits first); the caller adds the lanes up.  `coherent`: x was
+// written by other CTAs of this launch and must not come from the read-only cache.
+template <int BITS>
+__device__ __forceinline__ float dot_slice(const uint8_t* __restrict__ row, const void* __restrict__ srow, bool scale_f16,
+                                           int gshift, const void* xrow, bool x_bf16, bool coherent, int j0, int j1,
+                                           int lane) {
+  constexpr int WPV = 128 / BITS;  // weights per 128-bit word
+  constexpr int PER32 = 32 / BITS;
+  float acc = 0.0f;
+#pragma unroll 2
+  for (int j = j0 + lane; j < j1; j += 32) {
+    const uint4 r = __ldg(reinterpret_cast<const uint4*>(row) + j);
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    const int k0 = j * WPV;
+    const int g = gshift < 0 ? 0 : k0 >> gshift;
+    const float s = scale_f16 ? __half2float(reinterpret_cast<const __half*>(srow)[g]) : reinterpret_cast<const float*>(srow)[g];
+    float part = 0.0f;
+#pragma unroll
+    for (int blk = 0; blk < WPV / 8; ++blk) {
+      float xv[8];
+      x8(xrow, x_bf16, k0 + 8 * blk, coherent, xv);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int c = 8 * blk + i;  // code index inside the 128-bit word
+        const int q = static_cast<int>(w[c / PER32] << (32 - BITS * (c % PER32 + 1))) >> (32 - BITS);
+        // the integer as a float without the conversion unit: 1.5 * 2^23 + q has q in its low mantissa bits
+        part = fmaf(__int_as_float(0x4B400000 + q) - 12582912.0f, xv[i], part);
+      }
+    }
+    acc = fmaf(s, part, acc);
+  }
+  return acc;
+}
+
+__device__ __forceinline__ float dot_bits(int bits, const uint8_t* row, const void* srow, bool scale_f16, int gshift,
+                                          const void* xrow, bool x_bf16, bool coherent, int j0, int j1, int lane) {
+  switch (bits) {
+    case 8: return dot_slice<8>(row, srow, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane);
+    case 4: return dot_slice<4>(row, srow, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane);
+    default: return dot_slice<2>(row, srow, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane);
+  }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Thread 0 of the CTA counts the CTA in and polls until `target` CTAs have arrived (at most
+// `limit` polls); the CTA's earlier global writes are visible to whoever sees its arrival.
+// Returns to every thread whether the wait ended in time.
+__device__ __forceinline__ bool grid_arrive_wait(unsigned* counter, unsigned target, bool arrive, unsigned limit,
+                                                 int* check_word, int* s_flag) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    if (arrive) {
+      __threadfence();
+      atomicAdd(counter, 1u);
+    }
+    unsigned seen = 0, polls = 0;
+    int ok = 1;
+    for (;;) {
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+      if (seen >= target) break;
+      if (++polls > limit) {
+        ok = 0;
+        atomicOr(check_word, CHECK_WAIT_TIMEOUT);
+        break;
+      }
+      __nanosleep(40);
+    }
+    *s_flag = ok;
+  }
+  __syncthreads();
+  return *s_flag != 0;
+}
+
+__global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLayerArgs a) {
+  extern __shared__ float smem[];
+  __shared__ int s_ids[DL_MAX_PAIRS];
+  __shared__ float s_gates[DL_MAX_PAIRS];
+  __shared__ float s_part[DL_ROWS][DL_WPR];
+  __shared__ int s_flag;
+  const LayerDims& L = a.L;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int P = a.T * L.top_k;
+  const bool bf16 = L.act_bf16 != 0;
+  const size_t xsz = bf16 ? 2 : 4;
+  const int gshift = L.group > 0 ? 31 - __clz(L.group) : -1;
+  // The next kernel of the chain is scheduled once every CTA of this grid has executed this, i.e.
+  // once the whole grid is resident: it cannot take the room of a CTA the waits below need.
+  pdl_trigger();
+
+  // ---- 1. routing ----
+  const int32_t* ids = a.ids_in;
+  const float* gates = a.gates_in;
+  if (a.Wr) {
+    if (static_cast<int>(blockIdx.x) < a.T) {
+      router_logits<1>(smem, a.x, L.act_bf16, a.T, L.d_model, a.Wr, a.bias, a.bias_stride, L.E, a.EP, a.ep_shift,
+                       nullptr);  // waits on the kernels in front before its first global write
+      if (warp == 0) {
+        int my_id;
+        float my_gate;
+        router_pick(smem + ROUTER_DC + ROUTER_THREADS, L.E, L.top_k, a.renorm, lane, my_id, my_gate);
+        if (lane < L.top_k) {
+          a.ids[static_cast<size_t>(blockIdx.x) * L.top_k + lane] = my_id;
+          a.gates[static_cast<size_t>(blockIdx.x) * L.top_k + lane] = my_gate;
+        }
+      }
+    } else {
+      pdl_wait();
+    }
+    if (!grid_arrive_wait(a.sync, static_cast<unsigned>(a.T + a.extra_arrivals), static_cast<int>(blockIdx.x) < a.T,
+                          a.wait_limit, a.check_word, &s_flag))
+      return;
+    ids = a.ids;
+    gates = a.gates;
+  } else {
+    pdl_wait();
+  }
+  if (tid < P) {
+    int id = __ldcg(ids + tid);
+    if (id < 0 || id >= L.E) {  // only a caller's picks can be out of range
+      atomicOr(a.check_word, CHECK_BAD_EXPERT_ID);
+      id = -1;
+    }
+    s_ids[tid] = id;
+    s_gates[tid] = __ldcg(gates + tid);
+  }
+  __syncthreads();
+
+  if (blockIdx.x == 0 && tid == 0) {
+    // per-call bookkeeping: counts, exclusive offsets, pairs in expert order (stable) and its inverse
+    int run = 0;
+    for (int e = 0; e < L.E; ++e) {
+      a.off[e] = run;
+      int c = 0;
+      for (int p = 0; p < P; ++p)
+        if (s_ids[p] == e) {
+          a.perm[run + c] = p;
+          a.slot_of_pair[p] = run + c;
+          ++c;
+        }
+      a.counts[e] = c;
+      run += c;
+    }
+    a.off[L.E] = run;
+  }
+
+  // ---- 2. first projection: hidden[p][n] = act(W1[e_p][n] . x_t) ----
+  {
+    const int N = L.d_ff, K = L.d_model;
+    const int ngroups = gshift < 0 ? 1 : K >> gshift;
+    const long long units = static_cast<long long>(P) * N;
+    const long long stride = static_cast<long long>(gridDim.x) * DL_WARPS;
+    for (long long u = static_cast<long long>(blockIdx.x) * DL_WARPS + warp; u < units; u += stride) {
+      const int p = static_cast<int>(u / N);
+      const int n = static_cast<int>(u - static_cast<long long>(p) * N);
+      const int e = s_ids[p];
+      float h = 0.0f;
+      if (e >= 0) {
+        const ExpertDev ex = a.experts[e];
+        const int nvec = K * ex.bits / 128;
+        const size_t row_bytes = static_cast<size_t>(K) * ex.bits / 8;
+        const size_t srow = static_cast<size_t>(n) * ngroups * (L.scale_f16 ? 2 : 4);
+        const void* xrow = static_cast<const char*>(a.x) + static_cast<size_t>(p / L.top_k) * K * xsz;
+        const float v1 = warp_sum(dot_bits(ex.bits, ex.packed[0] + n * row_bytes, static_cast<const char*>(ex.scales[0]) + srow,
+                                           L.scale_f16, gshift, xrow, bf16, false, 0, nvec, lane));
+        if (L.act == EMOE_ACT_RELU) {
+          h = fmaxf(v1, 0.0f);
+        } else {
+          const float v3 = warp_sum(dot_bits(ex.bits, ex.packed[1] + n * row_bytes, static_cast<const char*>(ex.scales[1]) + srow,
+                                             L.scale_f16, gshift, xrow, bf16, false, 0, nvec, lane));
+          h = v1 / (1.0f + expf(-v1)) * v3;
+        }
+      }
+      if (lane == 0) {
+        if (bf16) reinterpret_cast<__nv_bfloat16*>(a.hidden)[u] = __float2bfloat16_rn(h);
+        else reinterpret_cast<float*>(a.hidden)[u] = h;
+      }
+    }
+  }
+  if (!grid_arrive_wait(a.sync + 1, gridDim.x + static_cast<unsigned>(a.extra_arrivals), true, a.wait_limit, a.check_word,
+                        &s_flag))
+    return;
+
+  // ---- 3. second projection and gate-weighted sum: y[t][n] = sum_j gate_j * (W2[e_j][n] . hidden_j) ----
+  {
+    const int N = L.d_model, K = L.d_ff;
+    const int ngroups = gshift < 0 ? 1 : K >> gshift;
+    const int m_last = L.act == EMOE_ACT_RELU ? 1 : 2;
+    const long long units = static_cast<long long>(a.T) * N;
+    const long long stride = static_cast<long long>(gridDim.x) * DL_ROWS;
+    const int rs = warp / DL_WPR, sub = warp % DL_WPR;
+    for (long long u0 = static_cast<long long>(blockIdx.x) * DL_ROWS; u0 < units; u0 += stride) {  // same trip count for the whole CTA
+      const long long u = u0 + rs;
+      float acc = 0.0f;
+      int t = 0, n = 0;
+      if (u < units) {
+        t = static_cast<int>(u / N);
+        n = static_cast<int>(u - static_cast<long long>(t) * N);
+        for (int j = 0; j < L.top_k; ++j) {
+          const int p = t * L.top_k + j;
+          const int e = s_ids[p];
+          if (e < 0) continue;
+          const ExpertDev ex = a.experts[e];
+          const int nvec = K * ex.bits / 128;
+          const int j0 = static_cast<int>(static_cast<long long>(nvec) * sub / DL_WPR);
+          const int j1 = static_cast<int>(static_cast<long long>(nvec) * (sub + 1) / DL_WPR);
+          const size_t row_bytes = static_cast<size_t>(K) * ex.bits / 8;
+          const size_t srow = static_cast<size_t>(n) * ngroups * (L.scale_f16 ? 2 : 4);
+          const void* hrow = static_cast<const char*>(a.hidden) + static_cast<size_t>(p) * K * xsz;
+          const float d = dot_bits(ex.bits, ex.packed[m_last] + n * row_bytes, static_cast<const char*>(ex.scales[m_last]) + srow,
+                                   L.scale_f16, gshift, hrow, bf16, true, j0, j1, lane);
+          acc = fmaf(s_gates[p], d, acc);
+        }
+      }
+      acc = warp_sum(acc);
+      if (lane == 0) s_part[rs][sub] = acc;
+      __syncthreads();
+      if (sub == 0 && lane == 0 && u < units)
+        a.y[u] = ((s_part[rs][0] + s_part[rs][1]) + s_part[rs][2]) + s_part[rs][3];
+      __syncthreads();
+    }
+  }
+  // the last CTA to leave clears the counters for the next launch
+  if (tid == 0 && atomicAdd(a.sync + 2, 1u) == gridDim.x - 1u) {
+    a.sync[0] = 0;
+    a.sync[1] = 0;
+    a.sync[2] = 0;
+    __threadfence();
+  }
+}
+
+size_t decode_layer_smem() { return sizeof(float) * (ROUTER_DC + ROUTER_THREADS + EMOE_MAX_EXPERTS); }
+
+}  // namespace
+
+bool decode_layer_supported(const LayerDims& L, int T) {
+  const bool group_ok = L.group == 0 || L.group == 64 || L.group == 128;
+  return T * L.top_k <= DL_MAX_PAIRS && L.E <= EMOE_MAX_EXPERTS && L.d_model % 64 == 0 && L.d_ff % 64 == 0 && group_ok &&
+         static_cast<long long>(L.d_model) * L.d_ff <= DL_MAX_WEIGHTS;
+}
+
+int decode_layer_resident_ctas(int device) {
+  int per_sm = 0, sms = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_layer_kernel, DL_THREADS, decode_layer_smem()) != cudaSuccess)
+    return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return 0;
+  return per_sm * sms;
+}
+
+cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, const void* x, int T, const float* Wr,
+                                const float* bias, int bias_stride, const int32_t* ids_in, const float* gates_in,
+                                int32_t* ids, float* gates, int32_t* counts, int32_t* off, int32_t* perm,
+                                int32_t* slot_of_pair, void* hidden, float* y, int resident_ctas, int sms, unsigned* sync,
+                                unsigned wait_limit, int extra_arrivals, int* check_word, cudaStream_t st) {
+  DecodeLayerArgs a;
+  a.L = L;
+  a.experts = experts;
+  a.x = x;
+  a.T = T;
+  a.Wr = Wr;
+  a.bias = bias;
+  a.bias_stride = bias_stride;
+  a.EP = 1;
+  a.ep_shift = 0;
+  while (a.EP < L.E) {
+    a.EP <<= 1;
+    ++a.ep_shift;
+  }
+  a.renorm = L.gate_mode == EMOE_GATE_SOFTMAX_RENORM;
+  a.ids_in = ids_in;
+  a.gates_in = gates_in;
+  a.ids = ids;
+  a.gates = gates;
+  a.counts = counts;
+  a.off = off;
+  a.perm = perm;
+  a.slot_of_pair = slot_of_pair;
+  a.hidden = hidden;
+  a.y = y;
+  a.sync = sync;
+  a.wait_limit = wait_limit;
+  a.extra_arrivals = extra_arrivals;
+  a.check_word = check_word;
+  // every CTA must be resident at once; four CTAs per SM are as many as the two projections can
+  // use, and every further CTA makes the grid-wide waits longer
+  int grid = 4 * sms;
+  if (grid > resident_ctas) grid = resident_ctas;
+  if (grid < T) return cudaErrorInvalidConfiguration;
+  return launch_chain(decode_layer_kernel, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
+}
+
+}  // namespace emoe

@@ -204,6 +204,91 @@ def test_router_topk_permutation_and_scatter_in_one_launch(act, d, f, E, k, gate
             assert np.array_equal(one[3], perm_ref)
 
 
+LAYER_CASES = [
+    # act, act_dtype, group, scale_dtype, d, f, E, k, gate, T list (one context, calls back to back)
+    ("relu", "bf16", 128, "f16", 768, 3072, 32, 1, "softmax", [1, 4, 16, 1, 2]),
+    ("swiglu", "bf16", 128, "f16", 512, 1536, 8, 2, "softmax_renorm", [1, 8, 3]),
+    ("relu", "f32", 0, "f32", 128, 256, 4, 1, "softmax", [5, 1]),
+    ("swiglu", "f32", 64, "f16", 192, 320, 3, 2, "softmax_renorm", [7, 2]),
+    ("relu", "bf16", 64, "f16", 512, 512, 128, 1, "softmax", [3, 16]),
+]
+
+
+@pytest.mark.parametrize("act,adt,group,sdt,d,f,E,k,gate,Ts", LAYER_CASES)
+def test_whole_layer_in_one_launch(act, adt, group, sdt, d, f, E, k, gate, Ts):
+    """A handful of tokens on a small layer: router, Top-K, both projections and the gate-weighted
+    sum in ONE launch.  ids, gates and permutation are bit-identical to the chain of launches; the
+    output matches the CPU checker within the path's tolerance and the chain's output within the
+    difference of two fp32 summation orders; the same through the call with given picks; call
+    after call on one context (the grid counters must come back to zero)."""
+    shape = inputs.LayerShape(d, f, E, k, act, gate, group, sdt, adt)
+    bits = ([8, 4, 2, 4] * E)[:E]
+    W = inputs.expert_set(47, 0, shape)
+    Wr = inputs.router_weight(47, 0, d, E, std=0.05)
+    packed, scales = oracle_pack_layer(W, shape, bits)
+    with layer.MoELayer(shape, bits, max_tokens=max(Ts)) as moe:
+        moe.pack_from_host(W)
+        for i, T in enumerate(Ts):
+            x = inputs.activations(47, i, T, d, adt)
+            B.emoe_set_fused_layer(moe.ctx, True)
+            y, ids, gates, perm = moe.forward(x, Wr)
+            assert B.emoe_kernels_last_forward(moe.ctx) == 1
+            y_r, perm_r = moe.forward_routed(x, ids, gates)
+            assert B.emoe_kernels_last_forward(moe.ctx) == 1
+            B.emoe_set_fused_layer(moe.ctx, False)
+            y_c, ids_c, gates_c, perm_c = moe.forward(x, Wr)
+            assert B.emoe_kernels_last_forward(moe.ctx) > 1
+            assert np.array_equal(ids, ids_c) and np.array_equal(gates, gates_c) and np.array_equal(perm, perm_c)
+            assert np.array_equal(perm_r, perm) and np.array_equal(y_r, y)
+            y_ref = oracle.moe_ffn_combine(x, f, act, group, adt == "bf16", bits, packed, scales, ids, gates)
+            assert rel_to_max(y, y_ref) <= output_tolerance(adt)
+            assert rel_to_max(y, y_c) <= output_tolerance(adt)
+            assert np.array_equal(B.emoe_last_expert_counts(moe.ctx, E), np.bincount(ids.ravel(), minlength=E))
+
+
+def test_one_launch_layer_leaves_larger_calls_to_the_other_kernels():
+    """Calls beyond 16 token-expert pairs, or with a forced kernel family, run as before."""
+    shape = inputs.LayerShape(512, 1024, 8, 2, "relu", "softmax", 128, "f16", "bf16")
+    bits = [8, 4, 2, 4] * 2
+    W = inputs.expert_set(49, 0, shape)
+    Wr = inputs.router_weight(49, 0, 512, 8, std=0.05)
+    with layer.MoELayer(shape, bits, max_tokens=16) as moe:
+        moe.pack_from_host(W)
+        B.emoe_set_fused_layer(moe.ctx, True)
+        moe.forward(inputs.activations(49, 0, 8, 512, "bf16"), Wr)
+        assert B.emoe_kernels_last_forward(moe.ctx) == 1
+        moe.forward(inputs.activations(49, 1, 9, 512, "bf16"), Wr)
+        assert B.emoe_kernels_last_forward(moe.ctx) > 1
+        B.emoe_set_ffn_path(moe.ctx, 3)
+        moe.forward(inputs.activations(49, 0, 8, 512, "bf16"), Wr)
+        assert B.emoe_kernels_last_forward(moe.ctx) > 1
+
+
+def test_grid_wide_waits_of_the_one_launch_layer_run_out_without_a_hang():
+    """The CTAs are told to wait for one more arrival than will ever come, with a short limit: the
+    waits give up, the kernel returns, the status call says "timeout", and the next call on the
+    context is right again."""
+    shape = inputs.LayerShape(512, 1024, 8, 1, "relu", "softmax", 128, "f16", "bf16")
+    bits, T = [8, 4, 2, 4] * 2, 4
+    W = inputs.expert_set(51, 0, shape)
+    x = inputs.activations(51, 0, T, 512, "bf16")
+    Wr = inputs.router_weight(51, 0, 512, 8, std=0.05)
+    with layer.MoELayer(shape, bits, max_tokens=T) as moe:
+        moe.pack_from_host(W)
+        B.emoe_set_fused_layer(moe.ctx, True)
+        good = moe.forward(x, Wr)
+        B.emoe_set_wait_limit(moe.ctx, 2000)
+        B.emoe_debug_expect_extra_completions(moe.ctx, 1)
+        with pytest.raises(B.EmoeError) as ei:
+            moe.forward(x, Wr)
+        assert ei.value.status == B.ERR_TIMEOUT
+        B.emoe_set_wait_limit(moe.ctx, 0)
+        B.emoe_debug_expect_extra_completions(moe.ctx, 0)
+        again = moe.forward(x, Wr)
+        for a, b in zip(good, again):
+            assert np.array_equal(a, b)
+
+
 def test_grid_wide_wait_of_the_one_launch_routing_runs_out_without_a_hang():
     """The CTAs are told to wait for one more arrival than the grid has, with a short limit: every
     wait gives up, every kernel still returns, the status call says "timeout", and the next call on
