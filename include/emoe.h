@@ -281,16 +281,20 @@ int emoe_set_fused_routing(emoe_ctx* ctx, int enabled);
  * packed codes, gate-weighted sum) in ONE launch, for calls of at most 16 token-expert pairs on
  * layers whose matrices hold at most 8 Mi weights each (single-request decoding, the paper's
  * target, on a Switch-base-sized layer): such a call is a few microseconds of work and the chain
- * of dependent launches is most of its time.  One resident grid; CTA t routes token t, all CTAs
- * then share the rows of the first projection (one warp per row, packed codes decoded in
+ * of dependent launches is most of its time.  One resident grid; a few CTAs per token form the
+ * router product, every CTA makes the picks from it, all CTAs then share the rows of the first projection (one warp per row, packed codes decoded in
  * registers, fp32 accumulation), meet at a bounded grid-wide wait, and share the rows of the
  * second projection, whose sums over the token's experts are formed in a fixed order.  Applies
  * to emoe_moe_forward and emoe_moe_forward_routed when no kernel family was forced
- * (emoe_set_ffn_path 0); calls outside the limits run as before.  ids, gates and permutation are
- * identical to the other paths', y agrees within the accumulation-order difference (fp32 sums
- * of the same products).  A wait that runs out reports EMOE_ERR_TIMEOUT through
- * emoe_device_status (limit: emoe_set_wait_limit). */
-int emoe_set_fused_layer(emoe_ctx* ctx, int enabled);
+ * (emoe_set_ffn_path 0); calls outside the limits run as before.  The router product is summed
+ * in slices of the d_model axis here, so logits and gates agree with the other paths' to fp32
+ * rounding (picks can differ only between experts whose logits agree that closely), and y
+ * within the accumulation-order difference (fp32 sums of the same products).  A wait that runs out reports EMOE_ERR_TIMEOUT through
+ * emoe_device_status (limit: emoe_set_wait_limit).
+ * mode 0: never; 1: every call inside the limits; 2 (the default): calls of one or two pairs,
+ * where it was measured faster than the chain of launches (1.5 x for one pair on a Switch-base-
+ * sized layer; from four pairs on the chain wins).  Other values: EMOE_ERR_INVALID_ARG. */
+int emoe_set_fused_layer(emoe_ctx* ctx, int mode);
 
 /* Number of kernels the last emoe_moe_forward / emoe_moe_forward_routed call on this context
  * enqueued (router + Top-K, permutation, scatter, expert FFNs, combine: Sections 2.1 and 3.2 name

@@ -291,8 +291,9 @@ def emoe_set_fused_routing(ctx, enabled: bool) -> None:
     _check(lib().emoe_set_fused_routing(ctx, int(enabled)), "emoe_set_fused_routing")
 
 
-def emoe_set_fused_layer(ctx, enabled: bool) -> None:
-    _check(lib().emoe_set_fused_layer(ctx, int(enabled)), "emoe_set_fused_layer")
+def emoe_set_fused_layer(ctx, mode) -> None:
+    """0 / False: never; 1 / True: every call inside the limits; 2: the default (one or two pairs)."""
+    _check(lib().emoe_set_fused_layer(ctx, int(mode)), "emoe_set_fused_layer")
 
 
 def emoe_set_wait_limit(ctx, polls: int) -> None:

@@ -120,8 +120,9 @@ int decode_layer_resident_ctas(int device);
 cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, const void* x, int T, const float* Wr,
                                 const float* bias, int bias_stride, const int32_t* ids_in, const float* gates_in,
                                 int32_t* ids, float* gates, int32_t* counts, int32_t* off, int32_t* perm,
-                                int32_t* slot_of_pair, void* hidden, float* y, int resident_ctas, int sms, unsigned* sync,
-                                unsigned wait_limit, int extra_arrivals, int* check_word, cudaStream_t st);
+                                int32_t* slot_of_pair, void* hidden, float* y, float* zpart, size_t zpart_floats,
+                                int resident_ctas, int sms, unsigned* sync, unsigned wait_limit, int extra_arrivals,
+                                int* check_word, cudaStream_t st);
 bool route_permute_scatter_supported(const LayerDims& L, int T, int resident_ctas);
 int route_permute_scatter_resident_ctas(int device);
 cudaError_t launch_route_permute_scatter(const LayerDims& L, const ExpertDev* experts, const void* x, int T, const float* Wr,

@@ -5,15 +5,18 @@
 //
 // The grid is resident at once (the host sizes it from the device's capacity), so its CTAs may
 // wait for one another; every such wait is bounded.
-//   1. CTA t < T computes token t's logits and picks (the device functions of the router kernel)
-//      and counts itself in; every CTA waits until all T have done so and reads the picks.
+//   1. The d_model axis of every token's router product is cut into slices, one CTA each; a CTA
+//      writes its partial logits and counts itself in.  Every CTA waits until all slices have
+//      arrived, adds the partial logits up in slice order and makes the picks itself (the Top-K
+//      device function of the router kernel), so that no second wait is needed to spread them.
+//      Each warp then asks for the rows of the second projection it will need (L2 prefetch).
 //   2. First projection: one warp per (pair, hidden channel) streams the packed row with 128-bit
 //      loads, decodes in registers, accumulates in fp32 and stores the activated value in the
 //      activation type.  The CTAs then meet at a grid-wide arrival counter.
 //   3. Second projection and gate-weighted sum: four warps share one (token, output channel),
 //      each takes a quarter of the hidden axis of every expert of the token; the quarters are
 //      added in a fixed order, so the result does not depend on timing.
-// CTA 0 also writes the bookkeeping the library keeps per call (counts, offsets, permutation).
+// The last CTA also writes the bookkeeping the library keeps per call (counts, offsets, permutation).
 // sync[0] counts the routing arrivals, sync[1] the arrivals after the first projection, sync[2]
 // the departures; the last CTA to leave sets all three back to zero for the next launch.
 #include "common.cuh"
@@ -37,6 +40,8 @@ struct DecodeLayerArgs {
   const float* Wr;       // null: the picks are given (ids_in / gates_in)
   const float* bias;
   int bias_stride, EP, ep_shift, renorm;
+  int rsplit;            // slices of the d_model axis per token in the router product
+  float* zpart;          // [T][rsplit][EP] partial logits
   const int32_t* ids_in;
   const float* gates_in;
   int32_t* ids;
@@ -150,10 +155,11 @@ __device__ __forceinline__ bool grid_arrive_wait(unsigned* counter, unsigned tar
 }
 
 __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLayerArgs a) {
-  extern __shared__ float smem[];
   __shared__ int s_ids[DL_MAX_PAIRS];
   __shared__ float s_gates[DL_MAX_PAIRS];
   __shared__ float s_part[DL_ROWS][DL_WPR];
+  __shared__ float s_red[DL_THREADS];            // router product: [parts][EP]
+  __shared__ float s_z[DL_WARPS][EMOE_MAX_EXPERTS];  // logits of the token a warp picks for
   __shared__ int s_flag;
   const LayerDims& L = a.L;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -166,59 +172,128 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
   pdl_trigger();
 
   // ---- 1. routing ----
-  const int32_t* ids = a.ids_in;
-  const float* gates = a.gates_in;
   if (a.Wr) {
-    if (static_cast<int>(blockIdx.x) < a.T) {
-      router_logits<1>(smem, a.x, L.act_bf16, a.T, L.d_model, a.Wr, a.bias, a.bias_stride, L.E, a.EP, a.ep_shift,
-                       nullptr);  // waits on the kernels in front before its first global write
-      if (warp == 0) {
-        int my_id;
-        float my_gate;
-        router_pick(smem + ROUTER_DC + ROUTER_THREADS, L.E, L.top_k, a.renorm, lane, my_id, my_gate);
-        if (lane < L.top_k) {
-          a.ids[static_cast<size_t>(blockIdx.x) * L.top_k + lane] = my_id;
-          a.gates[static_cast<size_t>(blockIdx.x) * L.top_k + lane] = my_gate;
+    const int RS = a.rsplit, EP = a.EP, d = L.d_model;
+    const int n_route = a.T * RS;
+    if (static_cast<int>(blockIdx.x) < n_route) {
+      // partial logits of one token over one slice of the d_model axis: thread = (expert, interleaved part of the slice)
+      const int t = static_cast<int>(blockIdx.x) / RS, r = static_cast<int>(blockIdx.x) - t * RS;
+      const int kb = static_cast<int>(static_cast<long long>(d) * r / RS), ke = static_cast<int>(static_cast<long long>(d) * (r + 1) / RS);
+      const int e = tid & (EP - 1), part = tid >> a.ep_shift, S = DL_THREADS >> a.ep_shift;
+      float acc = 0.0f;
+      if (e < L.E) {
+        constexpr int U = 8;  // independent loads in flight per thread
+        for (int i = kb + part; i < ke; i += U * S) {
+          float w[U], xv[U];
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            const int ii = i + u * S;
+            const bool in = ii < ke;
+            w[u] = in ? __ldg(a.Wr + static_cast<size_t>(ii) * L.E + e) : 0.0f;
+            const size_t xi = static_cast<size_t>(t) * d + (in ? ii : kb);
+            xv[u] = bf16 ? __bfloat162float(__ldg(reinterpret_cast<const __nv_bfloat16*>(a.x) + xi))
+                         : __ldg(reinterpret_cast<const float*>(a.x) + xi);
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u) acc = fmaf(xv[u], w[u], acc);
         }
+      }
+      s_red[part * EP + e] = acc;
+      __syncthreads();
+      pdl_wait();  // the kernels in front may still read what is written from here on
+      if (tid < EP) {
+        float z = 0.0f;
+        for (int sidx = 0; sidx < S; ++sidx) z += s_red[sidx * EP + tid];
+        a.zpart[(static_cast<size_t>(t) * RS + r) * EP + tid] = z;
       }
     } else {
       pdl_wait();
     }
-    if (!grid_arrive_wait(a.sync, static_cast<unsigned>(a.T + a.extra_arrivals), static_cast<int>(blockIdx.x) < a.T,
+    if (!grid_arrive_wait(a.sync, static_cast<unsigned>(n_route + a.extra_arrivals), static_cast<int>(blockIdx.x) < n_route,
                           a.wait_limit, a.check_word, &s_flag))
       return;
-    ids = a.ids;
-    gates = a.gates;
+    // every CTA makes the picks of every token from the same numbers in the same order
+    for (int t = warp; t < a.T; t += DL_WARPS) {
+      float* zrow = s_z[warp];
+      for (int e = lane; e < EP; e += 32) {
+        float z = 0.0f;
+        if (e < L.E) {
+          for (int r = 0; r < RS; ++r) z += __ldcg(a.zpart + (static_cast<size_t>(t) * RS + r) * EP + e);
+          if (a.bias) z += a.bias[static_cast<size_t>(t) * a.bias_stride + e];
+        }
+        zrow[e] = z;
+      }
+      __syncwarp();
+      int my_id;
+      float my_gate;
+      router_pick(zrow, L.E, L.top_k, a.renorm, lane, my_id, my_gate);
+      if (lane < L.top_k) {
+        s_ids[t * L.top_k + lane] = my_id;
+        s_gates[t * L.top_k + lane] = my_gate;
+        if (blockIdx.x == 0) {
+          a.ids[static_cast<size_t>(t) * L.top_k + lane] = my_id;
+          a.gates[static_cast<size_t>(t) * L.top_k + lane] = my_gate;
+        }
+      }
+      __syncwarp();
+    }
   } else {
     pdl_wait();
-  }
-  if (tid < P) {
-    int id = __ldcg(ids + tid);
-    if (id < 0 || id >= L.E) {  // only a caller's picks can be out of range
-      atomicOr(a.check_word, CHECK_BAD_EXPERT_ID);
-      id = -1;
+    if (tid < P) {
+      int id = __ldcg(a.ids_in + tid);
+      if (id < 0 || id >= L.E) {  // only a caller's picks can be out of range
+        atomicOr(a.check_word, CHECK_BAD_EXPERT_ID);
+        id = -1;
+      }
+      s_ids[tid] = id;
+      s_gates[tid] = __ldcg(a.gates_in + tid);
     }
-    s_ids[tid] = id;
-    s_gates[tid] = __ldcg(gates + tid);
   }
   __syncthreads();
 
-  if (blockIdx.x == 0 && tid == 0) {
-    // per-call bookkeeping: counts, exclusive offsets, pairs in expert order (stable) and its inverse
-    int run = 0;
-    for (int e = 0; e < L.E; ++e) {
-      a.off[e] = run;
-      int c = 0;
-      for (int p = 0; p < P; ++p)
-        if (s_ids[p] == e) {
-          a.perm[run + c] = p;
-          a.slot_of_pair[p] = run + c;
-          ++c;
-        }
-      a.counts[e] = c;
-      run += c;
+  // the rows of the second projection this warp will read: ask for them now, so that they are in
+  // L2 by the time the first projection is done
+  {
+    const int N = L.d_model, K = L.d_ff;
+    const int m_last = L.act == EMOE_ACT_RELU ? 1 : 2;
+    const long long units = static_cast<long long>(a.T) * N;
+    const long long stride = static_cast<long long>(gridDim.x) * DL_ROWS;
+    const int rs = warp / DL_WPR, sub = warp % DL_WPR;
+    for (long long u = static_cast<long long>(blockIdx.x) * DL_ROWS + rs; u < units; u += stride) {
+      const int t = static_cast<int>(u / N);
+      const int n = static_cast<int>(u - static_cast<long long>(t) * N);
+      for (int j = 0; j < L.top_k; ++j) {
+        const int e = s_ids[t * L.top_k + j];
+        if (e < 0) continue;
+        const ExpertDev ex = a.experts[e];
+        const int nvec = K * ex.bits / 128;
+        const size_t b0 = static_cast<size_t>(static_cast<long long>(nvec) * sub / DL_WPR) * 16;
+        const size_t b1 = static_cast<size_t>(static_cast<long long>(nvec) * (sub + 1) / DL_WPR) * 16;
+        const uint8_t* row = ex.packed[m_last] + static_cast<size_t>(n) * (static_cast<size_t>(K) * ex.bits / 8);
+        for (size_t b = (b0 & ~static_cast<size_t>(127)) + 128 * lane; b < b1; b += 128 * 32)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(row + b));
+      }
     }
-    a.off[L.E] = run;
+  }
+
+  if (blockIdx.x == gridDim.x - 1) {
+    // per-call bookkeeping, by the CTA with the least work in the projections: counts, exclusive
+    // offsets, pairs in expert order (stable) and the inverse; every entry on its own
+    for (int e = tid; e <= L.E; e += DL_THREADS) {
+      int below = 0, same = 0;
+      for (int p = 0; p < P; ++p) {
+        below += s_ids[p] >= 0 && s_ids[p] < e;
+        same += s_ids[p] == e;
+      }
+      a.off[e] = below;
+      if (e < L.E) a.counts[e] = same;
+    }
+    if (tid < P && s_ids[tid] >= 0) {
+      int slot = 0;
+      for (int q = 0; q < P; ++q) slot += s_ids[q] >= 0 && (s_ids[q] < s_ids[tid] || (s_ids[q] == s_ids[tid] && q < tid));
+      a.perm[slot] = tid;
+      a.slot_of_pair[tid] = slot;
+    }
   }
 
   // ---- 2. first projection: hidden[p][n] = act(W1[e_p][n] . x_t) ----
@@ -306,7 +381,7 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
   }
 }
 
-size_t decode_layer_smem() { return sizeof(float) * (ROUTER_DC + ROUTER_THREADS + EMOE_MAX_EXPERTS); }
+size_t decode_layer_smem() { return 0; }
 
 }  // namespace
 
@@ -327,8 +402,9 @@ int decode_layer_resident_ctas(int device) {
 cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, const void* x, int T, const float* Wr,
                                 const float* bias, int bias_stride, const int32_t* ids_in, const float* gates_in,
                                 int32_t* ids, float* gates, int32_t* counts, int32_t* off, int32_t* perm,
-                                int32_t* slot_of_pair, void* hidden, float* y, int resident_ctas, int sms, unsigned* sync,
-                                unsigned wait_limit, int extra_arrivals, int* check_word, cudaStream_t st) {
+                                int32_t* slot_of_pair, void* hidden, float* y, float* zpart, size_t zpart_floats,
+                                int resident_ctas, int sms, unsigned* sync, unsigned wait_limit, int extra_arrivals,
+                                int* check_word, cudaStream_t st) {
   DecodeLayerArgs a;
   a.L = L;
   a.experts = experts;
@@ -344,6 +420,11 @@ cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, co
     ++a.ep_shift;
   }
   a.renorm = L.gate_mode == EMOE_GATE_SOFTMAX_RENORM;
+  // slices of the router product: as many as the scratch array holds and as leave a slice 64 inputs or more
+  a.rsplit = 8;
+  while (a.rsplit > 1 && (static_cast<size_t>(T) * a.rsplit * a.EP > zpart_floats || L.d_model / a.rsplit < 64)) a.rsplit >>= 1;
+  if (Wr && static_cast<size_t>(T) * a.rsplit * a.EP > zpart_floats) return cudaErrorInvalidValue;
+  a.zpart = zpart;
   a.ids_in = ids_in;
   a.gates_in = gates_in;
   a.ids = ids;
@@ -362,7 +443,7 @@ cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, co
   // use, and every further CTA makes the grid-wide waits longer
   int grid = 4 * sms;
   if (grid > resident_ctas) grid = resident_ctas;
-  if (grid < T) return cudaErrorInvalidConfiguration;
+  if (grid < T * a.rsplit) return cudaErrorInvalidConfiguration;
   return launch_chain(decode_layer_kernel, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
 }
 

@@ -217,7 +217,8 @@ LAYER_CASES = [
 @pytest.mark.parametrize("act,adt,group,sdt,d,f,E,k,gate,Ts", LAYER_CASES)
 def test_whole_layer_in_one_launch(act, adt, group, sdt, d, f, E, k, gate, Ts):
     """A handful of tokens on a small layer: router, Top-K, both projections and the gate-weighted
-    sum in ONE launch.  ids, gates and permutation are bit-identical to the chain of launches; the
+    sum in ONE launch.  Picks and permutation are those of the chain of launches, the gates agree
+    to rounding (the router product is summed in another order); the
     output matches the CPU checker within the path's tolerance and the chain's output within the
     difference of two fp32 summation orders; the same through the call with given picks; call
     after call on one context (the grid counters must come back to zero)."""
@@ -238,7 +239,11 @@ def test_whole_layer_in_one_launch(act, adt, group, sdt, d, f, E, k, gate, Ts):
             B.emoe_set_fused_layer(moe.ctx, False)
             y_c, ids_c, gates_c, perm_c = moe.forward(x, Wr)
             assert B.emoe_kernels_last_forward(moe.ctx) > 1
-            assert np.array_equal(ids, ids_c) and np.array_equal(gates, gates_c) and np.array_equal(perm, perm_c)
+            # the router product is summed slice by slice here: same picks, gates equal to rounding
+            assert np.array_equal(ids, ids_c) and np.array_equal(perm, perm_c)
+            np.testing.assert_allclose(gates, gates_c, rtol=2e-5, atol=1e-7)
+            _, _, logits_ref = oracle.route(x, Wr, None, k, gate == "softmax_renorm")
+            check_ids(ids, logits_ref, k)
             assert np.array_equal(perm_r, perm) and np.array_equal(y_r, y)
             y_ref = oracle.moe_ffn_combine(x, f, act, group, adt == "bf16", bits, packed, scales, ids, gates)
             assert rel_to_max(y, y_ref) <= output_tolerance(adt)
@@ -261,6 +266,13 @@ def test_one_launch_layer_leaves_larger_calls_to_the_other_kernels():
         assert B.emoe_kernels_last_forward(moe.ctx) > 1
         B.emoe_set_ffn_path(moe.ctx, 3)
         moe.forward(inputs.activations(49, 0, 8, 512, "bf16"), Wr)
+        assert B.emoe_kernels_last_forward(moe.ctx) > 1
+        # the default: only calls of one or two pairs, where the single launch was measured faster
+        B.emoe_set_ffn_path(moe.ctx, 0)
+        B.emoe_set_fused_layer(moe.ctx, 2)
+        moe.forward(inputs.activations(49, 2, 1, 512, "bf16"), Wr)
+        assert B.emoe_kernels_last_forward(moe.ctx) == 1
+        moe.forward(inputs.activations(49, 3, 2, 512, "bf16"), Wr)
         assert B.emoe_kernels_last_forward(moe.ctx) > 1
 
 
