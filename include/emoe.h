@@ -291,9 +291,10 @@ int emoe_set_fused_routing(emoe_ctx* ctx, int enabled);
  * rounding (picks can differ only between experts whose logits agree that closely), and y
  * within the accumulation-order difference (fp32 sums of the same products).  A wait that runs out reports EMOE_ERR_TIMEOUT through
  * emoe_device_status (limit: emoe_set_wait_limit).
- * mode 0: never; 1: every call inside the limits; 2 (the default): calls of one or two pairs,
- * where it was measured faster than the chain of launches (1.5 x for one pair on a Switch-base-
- * sized layer; from four pairs on the chain wins).  Other values: EMOE_ERR_INVALID_ARG. */
+ * mode 0: never; 1: every call inside the limits; 2 (the default): calls of up to eight pairs,
+ * where it was measured faster than the chain of launches (about 1.5 x for one to four pairs on
+ * a Switch-base-sized layer, 1.1 x for eight; for sixteen the chain wins).  Other values:
+ * EMOE_ERR_INVALID_ARG. */
 int emoe_set_fused_layer(emoe_ctx* ctx, int mode);
 
 /* Number of kernels the last emoe_moe_forward / emoe_moe_forward_routed call on this context

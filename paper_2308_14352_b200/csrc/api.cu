@@ -374,9 +374,9 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       ctx->fuse_routing && one_launch_permute && !routed && route_permute_scatter_supported(L, T, ctx->resident_route_ctas);
   // a handful of tokens on a small layer: router, both projections and the gate-weighted sum in one launch
   bool one_launch_layer = false;
-  // as measured on a Switch-base-sized layer: 1.5 x faster than the chain of launches for one pair, 1.17 x for two,
-  // slower from four pairs on (the first projection then takes several rows per warp, one after the other)
-  const bool layer_wanted = ctx->fuse_layer == 1 || (ctx->fuse_layer == 2 && P <= 2);
+  // as measured on a Switch-base-sized layer: 1.5 x faster than the chain of launches for one to four pairs, 1.1 x
+  // for eight, slower for sixteen (the projections then take several passes of dependent loads per warp)
+  const bool layer_wanted = ctx->fuse_layer == 1 || (ctx->fuse_layer == 2 && P <= 8);
   if (layer_wanted && ctx->ffn_path == 0 && decode_layer_supported(L, T)) {
     if (ctx->resident_layer_ctas < 0) {
       ctx->resident_layer_ctas = decode_layer_resident_ctas(ctx->device);

@@ -10,12 +10,13 @@
 //      arrived, adds the partial logits up in slice order and makes the picks itself (the Top-K
 //      device function of the router kernel), so that no second wait is needed to spread them.
 //      Each warp then asks for the rows of the second projection it will need (L2 prefetch).
-//   2. First projection: one warp per (pair, hidden channel) streams the packed row with 128-bit
-//      loads, decodes in registers, accumulates in fp32 and stores the activated value in the
-//      activation type.  The CTAs then meet at a grid-wide arrival counter.
-//   3. Second projection and gate-weighted sum: four warps share one (token, output channel),
-//      each takes a quarter of the hidden axis of every expert of the token; the quarters are
-//      added in a fixed order, so the result does not depend on timing.
+//   2. First projection: one warp per (pair, one or four hidden channels) streams its packed rows
+//      with 128-bit loads, all started before the first is used, decodes in registers, reads
+//      the activations once for all of them, accumulates in fp32 and stores the activated values
+//      in the activation type.  The CTAs then meet at a grid-wide arrival counter.
+//   3. Second projection and gate-weighted sum: four warps share one (token, one or four output
+//      channels), each takes a quarter of the hidden axis of every expert of the token; the
+//      quarters are added in a fixed order, so the result does not depend on timing.
 // The last CTA also writes the bookkeeping the library keeps per call (counts, offsets, permutation).
 // sync[0] counts the routing arrivals, sync[1] the arrivals after the first projection, sync[2]
 // the departures; the last CTA to leave sets all three back to zero for the next launch.
@@ -29,7 +30,8 @@ constexpr int DL_THREADS = ROUTER_THREADS;
 constexpr int DL_WARPS = DL_THREADS / 32;
 constexpr int DL_MAX_PAIRS = 16;
 constexpr int DL_WPR = 4;                    // warps per output row in the second projection
-constexpr int DL_ROWS = DL_WARPS / DL_WPR;   // output rows a CTA works on at a time
+constexpr int DL_ROWS = DL_WARPS / DL_WPR;   // row blocks of the second projection a CTA works on at a time
+constexpr int DL_R_MAX = 4;                  // consecutive rows of a matrix one warp takes at once: 1 or this
 constexpr long long DL_MAX_WEIGHTS = 8LL << 20;  // per matrix: beyond this a layer is bandwidth-bound and streams better
 
 struct DecodeLayerArgs {
@@ -75,47 +77,58 @@ __device__ __forceinline__ void x8(const void* row, bool bf16, int k, bool coher
   }
 }
 
-// The lane's share of  sum_k q[k] * s[k / G] * x[k]  over the 128-bit words j0 .. j1-1 of one packed
-// row (two's-complement fields, low bits first); the caller adds the lanes up.  `coherent`: x was
-// written by other CTAs of this launch and must not come from the read-only cache.
-template <int BITS>
-__device__ __forceinline__ float dot_slice(const uint8_t* __restrict__ row, const void* __restrict__ srow, bool scale_f16,
-                                           int gshift, const void* xrow, bool x_bf16, bool coherent, int j0, int j1,
-                                           int lane) {
+// The lane's share of  sum_k q[r][k] * s[r][k / G] * x[k]  for DL_R consecutive rows r of one packed
+// matrix over their 128-bit words j0 .. j1-1 (two's-complement fields, low bits first); the caller
+// adds the lanes up.  The rows' loads are all started before the first is used, and the
+// activations are read once for all of them.  `coherent`: x was written by other CTAs of this
+// launch and must not come from the read-only cache.
+template <int BITS, int DL_R>
+__device__ __forceinline__ void dot_rows(const uint8_t* __restrict__ row0, size_t row_bytes, const char* __restrict__ srow0,
+                                         size_t srow_bytes, bool scale_f16, int gshift, const void* xrow, bool x_bf16,
+                                         bool coherent, int j0, int j1, int lane, float (&acc)[DL_R]) {
   constexpr int WPV = 128 / BITS;  // weights per 128-bit word
   constexpr int PER32 = 32 / BITS;
-  float acc = 0.0f;
-#pragma unroll 2
   for (int j = j0 + lane; j < j1; j += 32) {
-    const uint4 r = __ldg(reinterpret_cast<const uint4*>(row) + j);
-    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    uint32_t w[DL_R][4];
+    float sc[DL_R], part[DL_R];
     const int k0 = j * WPV;
     const int g = gshift < 0 ? 0 : k0 >> gshift;
-    const float s = scale_f16 ? __half2float(reinterpret_cast<const __half*>(srow)[g]) : reinterpret_cast<const float*>(srow)[g];
-    float part = 0.0f;
+#pragma unroll
+    for (int r = 0; r < DL_R; ++r) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(row0 + r * row_bytes) + j);
+      w[r][0] = v.x, w[r][1] = v.y, w[r][2] = v.z, w[r][3] = v.w;
+      const char* sp = srow0 + r * srow_bytes;
+      sc[r] = scale_f16 ? __half2float(reinterpret_cast<const __half*>(sp)[g]) : reinterpret_cast<const float*>(sp)[g];
+      part[r] = 0.0f;
+    }
 #pragma unroll
     for (int blk = 0; blk < WPV / 8; ++blk) {
       float xv[8];
       x8(xrow, x_bf16, k0 + 8 * blk, coherent, xv);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int c = 8 * blk + i;  // code index inside the 128-bit word
-        const int q = static_cast<int>(w[c / PER32] << (32 - BITS * (c % PER32 + 1))) >> (32 - BITS);
-        // the integer as a float without the conversion unit: 1.5 * 2^23 + q has q in its low mantissa bits
-        part = fmaf(__int_as_float(0x4B400000 + q) - 12582912.0f, xv[i], part);
+      for (int r = 0; r < DL_R; ++r) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int c = 8 * blk + i;  // code index inside the 128-bit word
+          const int q = static_cast<int>(w[r][c / PER32] << (32 - BITS * (c % PER32 + 1))) >> (32 - BITS);
+          // the integer as a float without the conversion unit: 1.5 * 2^23 + q has q in its low mantissa bits
+          part[r] = fmaf(__int_as_float(0x4B400000 + q) - 12582912.0f, xv[i], part[r]);
+        }
       }
     }
-    acc = fmaf(s, part, acc);
+#pragma unroll
+    for (int r = 0; r < DL_R; ++r) acc[r] = fmaf(sc[r], part[r], acc[r]);
   }
-  return acc;
 }
 
-__device__ __forceinline__ float dot_bits(int bits, const uint8_t* row, const void* srow, bool scale_f16, int gshift,
-                                          const void* xrow, bool x_bf16, bool coherent, int j0, int j1, int lane) {
+template <int DL_R>
+__device__ __forceinline__ void dot_bits(int bits, const uint8_t* row0, size_t row_bytes, const char* srow0, size_t srow_bytes,
+                                         bool scale_f16, int gshift, const void* xrow, bool x_bf16, bool coherent, int j0,
+                                         int j1, int lane, float (&acc)[DL_R]) {
   switch (bits) {
-    case 8: return dot_slice<8>(row, srow, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane);
-    case 4: return dot_slice<4>(row, srow, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane);
-    default: return dot_slice<2>(row, srow, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane);
+    case 8: dot_rows<8, DL_R>(row0, row_bytes, srow0, srow_bytes, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane, acc); break;
+    case 4: dot_rows<4, DL_R>(row0, row_bytes, srow0, srow_bytes, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane, acc); break;
+    default: dot_rows<2, DL_R>(row0, row_bytes, srow0, srow_bytes, scale_f16, gshift, xrow, x_bf16, coherent, j0, j1, lane, acc); break;
   }
 }
 
@@ -154,10 +167,11 @@ __device__ __forceinline__ bool grid_arrive_wait(unsigned* counter, unsigned tar
   return *s_flag != 0;
 }
 
+template <int DL_R>
 __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLayerArgs a) {
   __shared__ int s_ids[DL_MAX_PAIRS];
   __shared__ float s_gates[DL_MAX_PAIRS];
-  __shared__ float s_part[DL_ROWS][DL_WPR];
+  __shared__ float s_part[DL_ROWS][DL_WPR][DL_R_MAX];
   __shared__ float s_red[DL_THREADS];            // router product: [parts][EP]
   __shared__ float s_z[DL_WARPS][EMOE_MAX_EXPERTS];  // logits of the token a warp picks for
   __shared__ int s_flag;
@@ -256,12 +270,13 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
   {
     const int N = L.d_model, K = L.d_ff;
     const int m_last = L.act == EMOE_ACT_RELU ? 1 : 2;
-    const long long units = static_cast<long long>(a.T) * N;
+    const int NB = N / DL_R;  // blocks of DL_R rows
+    const long long units = static_cast<long long>(a.T) * NB;
     const long long stride = static_cast<long long>(gridDim.x) * DL_ROWS;
     const int rs = warp / DL_WPR, sub = warp % DL_WPR;
     for (long long u = static_cast<long long>(blockIdx.x) * DL_ROWS + rs; u < units; u += stride) {
-      const int t = static_cast<int>(u / N);
-      const int n = static_cast<int>(u - static_cast<long long>(t) * N);
+      const int t = static_cast<int>(u / NB);
+      const int n = static_cast<int>(u - static_cast<long long>(t) * NB) * DL_R;
       for (int j = 0; j < L.top_k; ++j) {
         const int e = s_ids[t * L.top_k + j];
         if (e < 0) continue;
@@ -269,9 +284,12 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
         const int nvec = K * ex.bits / 128;
         const size_t b0 = static_cast<size_t>(static_cast<long long>(nvec) * sub / DL_WPR) * 16;
         const size_t b1 = static_cast<size_t>(static_cast<long long>(nvec) * (sub + 1) / DL_WPR) * 16;
-        const uint8_t* row = ex.packed[m_last] + static_cast<size_t>(n) * (static_cast<size_t>(K) * ex.bits / 8);
-        for (size_t b = (b0 & ~static_cast<size_t>(127)) + 128 * lane; b < b1; b += 128 * 32)
-          asm volatile("prefetch.global.L2 [%0];" ::"l"(row + b));
+        const size_t row_bytes = static_cast<size_t>(K) * ex.bits / 8;
+        for (int r = 0; r < DL_R; ++r) {
+          const uint8_t* row = ex.packed[m_last] + static_cast<size_t>(n + r) * row_bytes;
+          for (size_t b = (b0 & ~static_cast<size_t>(127)) + 128 * lane; b < b1; b += 128 * 32)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(row + b));
+        }
       }
     }
   }
@@ -296,36 +314,53 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
     }
   }
 
-  // ---- 2. first projection: hidden[p][n] = act(W1[e_p][n] . x_t) ----
+  // ---- 2. first projection: hidden[p][n] = act(W1[e_p][n] . x_t), DL_R hidden channels per warp ----
   {
-    const int N = L.d_ff, K = L.d_model;
+    const int N = L.d_ff, K = L.d_model, NB = N / DL_R;
     const int ngroups = gshift < 0 ? 1 : K >> gshift;
-    const long long units = static_cast<long long>(P) * N;
+    const size_t srow_bytes = static_cast<size_t>(ngroups) * (L.scale_f16 ? 2 : 4);
+    const long long units = static_cast<long long>(P) * NB;
     const long long stride = static_cast<long long>(gridDim.x) * DL_WARPS;
     for (long long u = static_cast<long long>(blockIdx.x) * DL_WARPS + warp; u < units; u += stride) {
-      const int p = static_cast<int>(u / N);
-      const int n = static_cast<int>(u - static_cast<long long>(p) * N);
+      const int p = static_cast<int>(u / NB);
+      const int n = static_cast<int>(u - static_cast<long long>(p) * NB) * DL_R;
       const int e = s_ids[p];
-      float h = 0.0f;
+      float h[DL_R];
+#pragma unroll
+      for (int r = 0; r < DL_R; ++r) h[r] = 0.0f;
       if (e >= 0) {
         const ExpertDev ex = a.experts[e];
         const int nvec = K * ex.bits / 128;
         const size_t row_bytes = static_cast<size_t>(K) * ex.bits / 8;
-        const size_t srow = static_cast<size_t>(n) * ngroups * (L.scale_f16 ? 2 : 4);
         const void* xrow = static_cast<const char*>(a.x) + static_cast<size_t>(p / L.top_k) * K * xsz;
-        const float v1 = warp_sum(dot_bits(ex.bits, ex.packed[0] + n * row_bytes, static_cast<const char*>(ex.scales[0]) + srow,
-                                           L.scale_f16, gshift, xrow, bf16, false, 0, nvec, lane));
+        float v1[DL_R];
+#pragma unroll
+        for (int r = 0; r < DL_R; ++r) v1[r] = 0.0f;
+        dot_bits<DL_R>(ex.bits, ex.packed[0] + n * row_bytes, row_bytes, static_cast<const char*>(ex.scales[0]) + n * srow_bytes, srow_bytes,
+                 L.scale_f16, gshift, xrow, bf16, false, 0, nvec, lane, v1);
         if (L.act == EMOE_ACT_RELU) {
-          h = fmaxf(v1, 0.0f);
+#pragma unroll
+          for (int r = 0; r < DL_R; ++r) h[r] = fmaxf(warp_sum(v1[r]), 0.0f);
         } else {
-          const float v3 = warp_sum(dot_bits(ex.bits, ex.packed[1] + n * row_bytes, static_cast<const char*>(ex.scales[1]) + srow,
-                                             L.scale_f16, gshift, xrow, bf16, false, 0, nvec, lane));
-          h = v1 / (1.0f + expf(-v1)) * v3;
+          float v3[DL_R];
+#pragma unroll
+          for (int r = 0; r < DL_R; ++r) v3[r] = 0.0f;
+          dot_bits<DL_R>(ex.bits, ex.packed[1] + n * row_bytes, row_bytes, static_cast<const char*>(ex.scales[1]) + n * srow_bytes, srow_bytes,
+                   L.scale_f16, gshift, xrow, bf16, false, 0, nvec, lane, v3);
+#pragma unroll
+          for (int r = 0; r < DL_R; ++r) {
+            const float g1 = warp_sum(v1[r]), g3 = warp_sum(v3[r]);
+            h[r] = g1 / (1.0f + expf(-g1)) * g3;
+          }
         }
       }
       if (lane == 0) {
-        if (bf16) reinterpret_cast<__nv_bfloat16*>(a.hidden)[u] = __float2bfloat16_rn(h);
-        else reinterpret_cast<float*>(a.hidden)[u] = h;
+        const size_t o = static_cast<size_t>(p) * N + n;
+#pragma unroll
+        for (int r = 0; r < DL_R; ++r) {
+          if (bf16) reinterpret_cast<__nv_bfloat16*>(a.hidden)[o + r] = __float2bfloat16_rn(h[r]);
+          else reinterpret_cast<float*>(a.hidden)[o + r] = h[r];
+        }
       }
     }
   }
@@ -333,21 +368,25 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
                         &s_flag))
     return;
 
-  // ---- 3. second projection and gate-weighted sum: y[t][n] = sum_j gate_j * (W2[e_j][n] . hidden_j) ----
+  // ---- 3. second projection and gate-weighted sum: y[t][n] = sum_j gate_j * (W2[e_j][n] . hidden_j),
+  //         DL_R output channels per group of DL_WPR warps ----
   {
-    const int N = L.d_model, K = L.d_ff;
+    const int N = L.d_model, K = L.d_ff, NB = N / DL_R;
     const int ngroups = gshift < 0 ? 1 : K >> gshift;
+    const size_t srow_bytes = static_cast<size_t>(ngroups) * (L.scale_f16 ? 2 : 4);
     const int m_last = L.act == EMOE_ACT_RELU ? 1 : 2;
-    const long long units = static_cast<long long>(a.T) * N;
+    const long long units = static_cast<long long>(a.T) * NB;
     const long long stride = static_cast<long long>(gridDim.x) * DL_ROWS;
     const int rs = warp / DL_WPR, sub = warp % DL_WPR;
     for (long long u0 = static_cast<long long>(blockIdx.x) * DL_ROWS; u0 < units; u0 += stride) {  // same trip count for the whole CTA
       const long long u = u0 + rs;
-      float acc = 0.0f;
+      float acc[DL_R];
+#pragma unroll
+      for (int r = 0; r < DL_R; ++r) acc[r] = 0.0f;
       int t = 0, n = 0;
       if (u < units) {
-        t = static_cast<int>(u / N);
-        n = static_cast<int>(u - static_cast<long long>(t) * N);
+        t = static_cast<int>(u / NB);
+        n = static_cast<int>(u - static_cast<long long>(t) * NB) * DL_R;
         for (int j = 0; j < L.top_k; ++j) {
           const int p = t * L.top_k + j;
           const int e = s_ids[p];
@@ -357,18 +396,25 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
           const int j0 = static_cast<int>(static_cast<long long>(nvec) * sub / DL_WPR);
           const int j1 = static_cast<int>(static_cast<long long>(nvec) * (sub + 1) / DL_WPR);
           const size_t row_bytes = static_cast<size_t>(K) * ex.bits / 8;
-          const size_t srow = static_cast<size_t>(n) * ngroups * (L.scale_f16 ? 2 : 4);
           const void* hrow = static_cast<const char*>(a.hidden) + static_cast<size_t>(p) * K * xsz;
-          const float d = dot_bits(ex.bits, ex.packed[m_last] + n * row_bytes, static_cast<const char*>(ex.scales[m_last]) + srow,
-                                   L.scale_f16, gshift, hrow, bf16, true, j0, j1, lane);
-          acc = fmaf(s_gates[p], d, acc);
+          float d[DL_R];
+#pragma unroll
+          for (int r = 0; r < DL_R; ++r) d[r] = 0.0f;
+          dot_bits<DL_R>(ex.bits, ex.packed[m_last] + n * row_bytes, row_bytes, static_cast<const char*>(ex.scales[m_last]) + n * srow_bytes,
+                   srow_bytes, L.scale_f16, gshift, hrow, bf16, true, j0, j1, lane, d);
+#pragma unroll
+          for (int r = 0; r < DL_R; ++r) acc[r] = fmaf(s_gates[p], d[r], acc[r]);
         }
       }
-      acc = warp_sum(acc);
-      if (lane == 0) s_part[rs][sub] = acc;
+#pragma unroll
+      for (int r = 0; r < DL_R; ++r) {
+        const float v = warp_sum(acc[r]);
+        if (lane == 0) s_part[rs][sub][r] = v;
+      }
       __syncthreads();
-      if (sub == 0 && lane == 0 && u < units)
-        a.y[u] = ((s_part[rs][0] + s_part[rs][1]) + s_part[rs][2]) + s_part[rs][3];
+      if (sub == 0 && lane < DL_R && u < units)
+        a.y[static_cast<size_t>(t) * N + n + lane] =
+            ((s_part[rs][0][lane] + s_part[rs][1][lane]) + s_part[rs][2][lane]) + s_part[rs][3][lane];
       __syncthreads();
     }
   }
@@ -393,8 +439,12 @@ bool decode_layer_supported(const LayerDims& L, int T) {
 
 int decode_layer_resident_ctas(int device) {
   int per_sm = 0, sms = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_layer_kernel, DL_THREADS, decode_layer_smem()) != cudaSuccess)
+  int per_sm1 = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_layer_kernel<DL_R_MAX>, DL_THREADS, decode_layer_smem()) != cudaSuccess)
     return 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm1, decode_layer_kernel<1>, DL_THREADS, decode_layer_smem()) != cudaSuccess)
+    return 0;
+  if (per_sm1 < per_sm) per_sm = per_sm1;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return 0;
   return per_sm * sms;
 }
@@ -444,7 +494,12 @@ cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, co
   int grid = 4 * sms;
   if (grid > resident_ctas) grid = resident_ctas;
   if (grid < T * a.rsplit) return cudaErrorInvalidConfiguration;
-  return launch_chain(decode_layer_kernel, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
+  // one row per warp while every row of the first projection then finds a warp of its own (most loads in flight);
+  // beyond that four rows per warp, whose loads are in flight together and share the activations
+  const long long rows = static_cast<long long>(T) * L.top_k * L.d_ff;
+  if (rows <= static_cast<long long>(grid) * DL_WARPS)
+    return launch_chain(decode_layer_kernel<1>, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
+  return launch_chain(decode_layer_kernel<DL_R_MAX>, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
 }
 
 }  // namespace emoe

@@ -267,12 +267,14 @@ def test_one_launch_layer_leaves_larger_calls_to_the_other_kernels():
         B.emoe_set_ffn_path(moe.ctx, 3)
         moe.forward(inputs.activations(49, 0, 8, 512, "bf16"), Wr)
         assert B.emoe_kernels_last_forward(moe.ctx) > 1
-        # the default: only calls of one or two pairs, where the single launch was measured faster
+        # the default: only calls of up to eight pairs, where the single launch was measured faster
         B.emoe_set_ffn_path(moe.ctx, 0)
         B.emoe_set_fused_layer(moe.ctx, 2)
         moe.forward(inputs.activations(49, 2, 1, 512, "bf16"), Wr)
         assert B.emoe_kernels_last_forward(moe.ctx) == 1
-        moe.forward(inputs.activations(49, 3, 2, 512, "bf16"), Wr)
+        moe.forward(inputs.activations(49, 3, 4, 512, "bf16"), Wr)
+        assert B.emoe_kernels_last_forward(moe.ctx) == 1
+        moe.forward(inputs.activations(49, 4, 5, 512, "bf16"), Wr)
         assert B.emoe_kernels_last_forward(moe.ctx) > 1
 
 
