@@ -251,6 +251,49 @@ def test_whole_layer_in_one_launch(act, adt, group, sdt, d, f, E, k, gate, Ts):
             assert np.array_equal(B.emoe_last_expert_counts(moe.ctx, E), np.bincount(ids.ravel(), minlength=E))
 
 
+def test_whole_layer_in_one_launch_with_a_router_bias_and_with_a_bad_pick():
+    """A per-token router bias (the form the skewed workloads use) goes into the picks of the
+    one-launch layer as it does into the router kernel's; a pick outside [0, E) in the call with
+    given picks is reported by the device check, contributes nothing, and the context stays usable."""
+    shape = inputs.LayerShape(512, 1024, 8, 2, "relu", "softmax_renorm", 128, "f16", "bf16")
+    bits = [8, 4, 2, 4] * 2
+    T = 4
+    W = inputs.expert_set(53, 0, shape)
+    Wr = inputs.router_weight(53, 0, 512, 8, std=0.05)
+    x = inputs.activations(53, 0, T, 512, "bf16")
+    bias = np.random.default_rng(53).normal(0.0, 2.0, size=(T, 8)).astype(np.float32)
+    packed, scales = oracle_pack_layer(W, shape, bits)
+    with layer.MoELayer(shape, bits, max_tokens=T) as moe:
+        moe.pack_from_host(W)
+        y, ids, gates, perm = moe.forward(x, Wr, bias)
+        assert B.emoe_kernels_last_forward(moe.ctx) == 1
+        ids_ref, gates_ref, logits_ref = oracle.route(x, Wr, bias, 2, True)
+        check_ids(ids, logits_ref, 2)
+        assert not np.array_equal(ids_ref, oracle.route(x, Wr, None, 2, True)[0])   # the bias decides picks here
+        same = np.all(ids == ids_ref, axis=1)
+        np.testing.assert_allclose(gates[same], gates_ref[same], rtol=2e-5, atol=1e-7)
+        y_ref = oracle.moe_ffn_combine(x, 1024, "relu", 128, True, bits, packed, scales, ids, gates)
+        assert rel_to_max(y, y_ref) <= 2e-3
+        bad = ids.copy()
+        bad[1, 0] = 8
+        xd = moe.to_device_x(x)
+        idd = torch.from_numpy(bad).to(moe.device)
+        gd = torch.from_numpy(gates).to(moe.device)
+        yd = torch.empty(T, 512, dtype=torch.float32, device=moe.device)
+        B.emoe_moe_forward_routed(moe.ctx, moe.desc, xd.data_ptr(), T, idd.data_ptr(), gd.data_ptr(), moe.table,
+                                  yd.data_ptr(), None, 0)
+        torch.cuda.synchronize(moe.device)
+        assert B.emoe_kernels_last_forward(moe.ctx) == 1
+        assert B.emoe_device_status(moe.ctx) == B.ERR_DEVICE_CHECK
+        # the other tokens are untouched by the bad pick, and token 1 keeps its valid expert's share
+        g2 = gates.copy()
+        g2[1, 0] = 0.0
+        y_ref2 = oracle.moe_ffn_combine(x, 1024, "relu", 128, True, bits, packed, scales, ids, g2)
+        assert rel_to_max(yd.cpu().numpy(), y_ref2) <= 2e-3
+        y3, ids3, _, _ = moe.forward(x, Wr, bias)
+        assert np.array_equal(y3, y) and np.array_equal(ids3, ids)
+
+
 def test_one_launch_layer_leaves_larger_calls_to_the_other_kernels():
     """Calls beyond 16 token-expert pairs, or with a forced kernel family, run as before."""
     shape = inputs.LayerShape(512, 1024, 8, 2, "relu", "softmax", 128, "f16", "bf16")
