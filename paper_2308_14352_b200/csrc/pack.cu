@@ -120,11 +120,22 @@ struct SourcePacked {
   }
   __device__ __forceinline__ void decode(const Raw& r, float s, float (&v)[16]) const {
     constexpr int PER_WORD = 32 / BIN;
+    if constexpr (BIN == 8) {
+      // a byte with its sign bit flipped is q + 128; dropped into the low mantissa byte of
+      // 1.5 * 2^23 it is the float 12582912 + 128 + q, exactly
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
-      const uint32_t word = r.w[c / PER_WORD];
-      const int q = static_cast<int>(word << (32 - BIN * (c % PER_WORD + 1))) >> (32 - BIN);
-      v[c] = __fmul_rn(__int_as_float(0x4B400000 + q) - ROUND_MAGIC, s);  // the integer as a float, exactly
+      for (int c = 0; c < 16; ++c) {
+        const uint32_t word = r.w[c >> 2] ^ 0x80808080u;
+        const uint32_t f = __byte_perm(word, 0x4B400000u, 0x7640u | (c & 3));
+        v[c] = __fmul_rn(__uint_as_float(f) - (ROUND_MAGIC + 128.0f), s);
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint32_t word = r.w[c / PER_WORD];
+        const int q = static_cast<int>(word << (32 - BIN * (c % PER_WORD + 1))) >> (32 - BIN);
+        v[c] = __fmul_rn(__int_as_float(0x4B400000 + q) - ROUND_MAGIC, s);  // the integer as a float, exactly
+      }
     }
   }
 };
@@ -148,11 +159,15 @@ __device__ __forceinline__ float store_scale(float amax, float range, int scale_
 struct QuantParams {
   float s, r, qlo, qhi;
 };
-__device__ __forceinline__ QuantParams quant_params(float s, float qlo, float qhi) {
+__device__ __forceinline__ QuantParams quant_params(float s, float amax, float qlo, float qhi) {
   QuantParams p;
   p.s = s;
   // scale 0: reciprocal 0, every product is 0 and every code is 0, as the definition says
   p.r = s == 0.0f ? 0.0f : ((s > 1e-30f && s < 1e30f) ? __frcp_rn(s) : __int_as_float(0x7fc00000));
+  // The rounding by addition needs |w * r| well below 2^22.  No weight of the unit exceeds its
+  // max-abs and the product is monotone, so one test per unit covers them all (it fails only
+  // where the stored scale lost its precision to fp16's subnormal range).
+  if (!(__fmul_rn(amax, p.r) < 200.0f)) p.r = __int_as_float(0x7fc00000);
   p.qlo = qlo;
   p.qhi = qhi;
   return p;
@@ -165,7 +180,7 @@ __device__ __forceinline__ uint32_t quantise1(float e, const QuantParams& p) {
   const float t = __fmul_rn(e, p.r);  // never contracted into the addition below
   float q = __fsub_rn(__fadd_rn(t, ROUND_MAGIC), ROUND_MAGIC);
   const float d = fabsf(fabsf(t - q) - 0.5f);
-  if (!(d >= 1e-4f) || !(fabsf(t) < 200.0f)) q = rintf(__fdiv_rn(e, p.s));
+  if (!(d >= 1e-4f)) q = rintf(__fdiv_rn(e, p.s));  // also every weight of a unit whose reciprocal is NaN
   q = fminf(fmaxf(q, p.qlo), p.qhi);
   return __float_as_uint(__fadd_rn(q, ROUND_MAGIC));
 }
@@ -233,7 +248,7 @@ __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, 
 #pragma unroll
           for (int o = 4; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
           const float amax = __fmul_rn(static_cast<float>(m), s_in);
-          const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, live && (lane & 7) == 0), qlo, qhi);
+          const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, live && (lane & 7) == 0), amax, qlo, qhi);
           uint32_t lut = 0;
 #pragma unroll
           for (int i = 0; i < 2; ++i) {
@@ -281,7 +296,7 @@ __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, 
         for (int c = 0; c < 16; ++c) amax = fmaxf(amax, fabsf(v[c]));
 #pragma unroll
         for (int o = 4; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-        const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, live && (lane & 7) == 0), qlo, qhi);
+        const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, live && (lane & 7) == 0), amax, qlo, qhi);
         uint32_t w[4] = {0u, 0u, 0u, 0u};
         constexpr int PER_WORD = 32 / BITS;
 #pragma unroll
@@ -311,7 +326,7 @@ __global__ void __launch_bounds__(256) quantise_kernel(const Source src, int N, 
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-    const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, lane == 0), qlo, qhi);
+    const QuantParams p = quant_params(store_scale(amax, range, scale_f16, scales, unit, lane == 0), amax, qlo, qhi);
     word_t* out = reinterpret_cast<word_t*>(packed + static_cast<size_t>(n) * row_bytes + static_cast<size_t>(g) * G * BITS / 8);
     for (int i = lane * 4; i < G; i += 128) {
       const float4 v = i < 128 ? first : src.load4(n, k_first + i, unit);  // later steps come from L1/L2
