@@ -807,8 +807,10 @@ int ffn_tma_ksplit(const LayerDims& L, int T) {
   const long long ctas = row_blocks * active;
   const int steps_min = (L.d_ff + 511) / 512;  // stages at the widest span (2 bits)
   // enough slices that the second projection's items outnumber the resident CTAs (3 per SM)
-  // about twice: short items at the end of the launch keep its tail short
-  long long z = (8 * 148 + ctas - 1) / ctas;
+  // about four times: short items at the end of the launch keep its tail short (as measured: the
+  // same on the Switch-base-like layer at 64 tokens as twice as many CTAs' worth, 3 % faster on
+  // the Mixtral-like layer at 4 tokens; fewer slices were slower on both)
+  long long z = (12 * 148 + ctas - 1) / ctas;
   // A handful of tokens leaves most SMs without an item: the slices are then cut as fine as the
   // 8-bit stages allow (narrower experts get empty slices, which only store zeros), so that the
   // second projection of the one or two activated experts is a short step on many SMs instead
