@@ -320,6 +320,8 @@ def time_offline_kernels(ctx, dev):
     return out
 
 
+L2_BYTES = 126 << 20
+
 PER_CONFIG = (
     # (label, workload, tokens, copies of the layer so that the weights of a step exceed L2)
     ("cfg0", "switch_tiny_fp32", 16, 8),
@@ -407,6 +409,24 @@ def measure_config(label, wname, T, copies, local, steps):
             e1.record(stream)
             stream.synchronize()
         ms = e0.elapsed_time(e1) / steps
+        # A step whose packed bytes fit the 126 MB L2 replays out of L2: time it once more with a
+        # buffer larger than L2 written between the replays, every replay between its own events.
+        cold_ms = None
+        if nbytes < 2 * L2_BYTES:
+            junk = torch.empty(4 * L2_BYTES, dtype=torch.uint8, device=dev)
+            total = 0.0
+            with torch.cuda.stream(stream):
+                for i in range(steps + 2):
+                    junk.fill_(i & 255)
+                    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a0.record(stream)
+                    g.replay()
+                    a1.record(stream)
+                    stream.synchronize()
+                    if i >= 2:
+                        total += a0.elapsed_time(a1)
+            cold_ms = total / steps
+            del junk
         B.emoe_set_timing(ctx, True)
         with torch.cuda.stream(stream):
             for _ in range(5):
@@ -428,7 +448,12 @@ def measure_config(label, wname, T, copies, local, steps):
                          {"bound": "hbm", "achieved": nbytes / (kms * 1e-3) / 1e9, "peak": hbm, "unit": "GB/s",
                           "frac": nbytes / (kms * 1e-3) / 1e9 / hbm, "algorithmic_bytes": nbytes}),
             "frac_of_roofline_time": max(t_hbm, t_tensor) / (kms * 1e-3),
+            "l2": ("the step's packed bytes exceed L2 twice over: nothing flushed" if cold_ms is None else
+                   "the step's packed bytes fit L2: ms_per_step is the warm replay, ms_per_step_cold_l2 the replay "
+                   "after 504 MB were written"),
         }
+        if cold_ms is not None:
+            out["ms_per_step_cold_l2"] = cold_ms
         if heavy_flops and not tensor_bound:
             # the dense-contraction subset of a skewed load: its flops against the time of the WHOLE expert stage
             # (a lower bound of the tensor rate of that subset, the light experts' streaming time is in it)

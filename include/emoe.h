@@ -292,8 +292,8 @@ int emoe_set_fused_routing(emoe_ctx* ctx, int enabled);
  * within the accumulation-order difference (fp32 sums of the same products).  A wait that runs out reports EMOE_ERR_TIMEOUT through
  * emoe_device_status (limit: emoe_set_wait_limit).
  * mode 0: never; 1: every call inside the limits; 2 (the default): calls of up to eight pairs,
- * where it was measured faster than the chain of launches (about 1.5 x for one to four pairs on
- * a Switch-base-sized layer, 1.1 x for eight; for sixteen the chain wins).  Other values:
+ * where it was measured faster than the chain of launches (1.8 x for one pair, 1.5 x for two to
+ * four on a Switch-base-sized layer, 1.1 x for eight; for sixteen the chain wins).  Other values:
  * EMOE_ERR_INVALID_ARG. */
 int emoe_set_fused_layer(emoe_ctx* ctx, int mode);
 

@@ -374,7 +374,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       ctx->fuse_routing && one_launch_permute && !routed && route_permute_scatter_supported(L, T, ctx->resident_route_ctas);
   // a handful of tokens on a small layer: router, both projections and the gate-weighted sum in one launch
   bool one_launch_layer = false;
-  // as measured on a Switch-base-sized layer: 1.5 x faster than the chain of launches for one to four pairs, 1.1 x
+  // as measured on a Switch-base-sized layer: 1.8 x faster than the chain of launches for one pair, 1.5 x for two to four, 1.1 x
   // for eight, slower for sixteen (the projections then take several passes of dependent loads per warp)
   const bool layer_wanted = ctx->fuse_layer == 1 || (ctx->fuse_layer == 2 && P <= 8);
   if (layer_wanted && ctx->ffn_path == 0 && decode_layer_supported(L, T)) {
@@ -382,7 +382,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       ctx->resident_layer_ctas = decode_layer_resident_ctas(ctx->device);
       EMOE_CUDA(ctx, cudaDeviceGetAttribute(&ctx->sms, cudaDevAttrMultiProcessorCount, ctx->device));
     }
-    one_launch_layer = ctx->sms > 0 && ctx->resident_layer_ctas >= 2 * ctx->sms;
+    one_launch_layer = ctx->sms > 0 && ctx->resident_layer_ctas >= ctx->sms;
   }
   if (!routed && !one_launch_route && !one_launch_layer)
     EMOE_LAUNCH(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,

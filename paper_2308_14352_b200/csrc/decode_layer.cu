@@ -3,18 +3,18 @@
 // paper's target is single-request decoding, where every step of the layer is a few microseconds
 // of work and the launches and dependencies between kernels are most of the time).
 //
-// The grid is resident at once (the host sizes it from the device's capacity), so its CTAs may
-// wait for one another; every such wait is bounded.
+// The grid is resident at once (the host sizes it from the device's capacity and the call's
+// work: one to three CTAs per SM), so its CTAs may wait for one another; every such wait is bounded.
 //   1. The d_model axis of every token's router product is cut into slices, one CTA each; a CTA
 //      writes its partial logits and counts itself in.  Every CTA waits until all slices have
 //      arrived, adds the partial logits up in slice order and makes the picks itself (the Top-K
 //      device function of the router kernel), so that no second wait is needed to spread them.
 //      Each warp then asks for the rows of the second projection it will need (L2 prefetch).
-//   2. First projection: one warp per (pair, one or four hidden channels) streams its packed rows
+//   2. First projection: one warp per (pair, four hidden channels) streams its packed rows
 //      with 128-bit loads, all started before the first is used, decodes in registers, reads
 //      the activations once for all of them, accumulates in fp32 and stores the activated values
 //      in the activation type.  The CTAs then meet at a grid-wide arrival counter.
-//   3. Second projection and gate-weighted sum: four warps share one (token, one or four output
+//   3. Second projection and gate-weighted sum: four warps share one (token, four output
 //      channels), each takes a quarter of the hidden axis of every expert of the token; the
 //      quarters are added in a fixed order, so the result does not depend on timing.
 // The last CTA also writes the bookkeeping the library keeps per call (counts, offsets, permutation).
@@ -31,7 +31,7 @@ constexpr int DL_WARPS = DL_THREADS / 32;
 constexpr int DL_MAX_PAIRS = 16;
 constexpr int DL_WPR = 4;                    // warps per output row in the second projection
 constexpr int DL_ROWS = DL_WARPS / DL_WPR;   // row blocks of the second projection a CTA works on at a time
-constexpr int DL_R_MAX = 4;                  // consecutive rows of a matrix one warp takes at once: 1 or this
+constexpr int DL_R_MAX = 4;                  // consecutive rows of a matrix one warp takes at once
 constexpr long long DL_MAX_WEIGHTS = 8LL << 20;  // per matrix: beyond this a layer is bandwidth-bound and streams better
 
 struct DecodeLayerArgs {
@@ -168,7 +168,7 @@ __device__ __forceinline__ bool grid_arrive_wait(unsigned* counter, unsigned tar
 }
 
 template <int DL_R>
-__global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLayerArgs a) {
+__global__ void __launch_bounds__(DL_THREADS, 3) decode_layer_kernel(const DecodeLayerArgs a) {
   __shared__ int s_ids[DL_MAX_PAIRS];
   __shared__ float s_gates[DL_MAX_PAIRS];
   __shared__ float s_part[DL_ROWS][DL_WPR][DL_R_MAX];
@@ -321,6 +321,22 @@ __global__ void __launch_bounds__(DL_THREADS) decode_layer_kernel(const DecodeLa
     const size_t srow_bytes = static_cast<size_t>(ngroups) * (L.scale_f16 ? 2 : 4);
     const long long units = static_cast<long long>(P) * NB;
     const long long stride = static_cast<long long>(gridDim.x) * DL_WARPS;
+    // a warp with more than one unit asks for the rows of the later ones now: their loads then
+    // come from L2 instead of starting a trip to HBM only when the unit before is done
+    for (long long u = static_cast<long long>(blockIdx.x) * DL_WARPS + warp + stride; u < units; u += stride) {
+      const int p = static_cast<int>(u / NB);
+      const int n = static_cast<int>(u - static_cast<long long>(p) * NB) * DL_R;
+      const int e = s_ids[p];
+      if (e < 0) continue;
+      const ExpertDev ex = a.experts[e];
+      const size_t bytes = static_cast<size_t>(K) * ex.bits / 8 * DL_R;  // the unit's rows follow each other
+      const int n_mat = L.act == EMOE_ACT_RELU ? 1 : 2;
+      for (int m = 0; m < n_mat; ++m) {
+        const uint8_t* rows = ex.packed[m] + static_cast<size_t>(n) * (bytes / DL_R);
+        for (size_t b = 128 * static_cast<size_t>(lane); b < bytes; b += 128 * 32)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(rows + b));
+      }
+    }
     for (long long u = static_cast<long long>(blockIdx.x) * DL_WARPS + warp; u < units; u += stride) {
       const int p = static_cast<int>(u / NB);
       const int n = static_cast<int>(u - static_cast<long long>(p) * NB) * DL_R;
@@ -439,12 +455,8 @@ bool decode_layer_supported(const LayerDims& L, int T) {
 
 int decode_layer_resident_ctas(int device) {
   int per_sm = 0, sms = 0;
-  int per_sm1 = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_layer_kernel<DL_R_MAX>, DL_THREADS, decode_layer_smem()) != cudaSuccess)
     return 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm1, decode_layer_kernel<1>, DL_THREADS, decode_layer_smem()) != cudaSuccess)
-    return 0;
-  if (per_sm1 < per_sm) per_sm = per_sm1;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return 0;
   return per_sm * sms;
 }
@@ -489,16 +501,16 @@ cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, co
   a.wait_limit = wait_limit;
   a.extra_arrivals = extra_arrivals;
   a.check_word = check_word;
-  // every CTA must be resident at once; four CTAs per SM are as many as the two projections can
-  // use, and every further CTA makes the grid-wide waits longer
-  int grid = 4 * sms;
-  if (grid > resident_ctas) grid = resident_ctas;
-  if (grid < T * a.rsplit) return cudaErrorInvalidConfiguration;
-  // one row per warp while every row of the first projection then finds a warp of its own (most loads in flight);
-  // beyond that four rows per warp, whose loads are in flight together and share the activations
-  const long long rows = static_cast<long long>(T) * L.top_k * L.d_ff;
-  if (rows <= static_cast<long long>(grid) * DL_WARPS)
-    return launch_chain(decode_layer_kernel<1>, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
+  // Every CTA must be resident at once.  As few CTAs as give every block of four rows of the
+  // first projection a warp of its own (one, two or three per SM): each further CTA makes the two
+  // grid-wide waits longer (as measured, one token: 0.139 ms per 12-layer step with one CTA per
+  // SM, 0.154 with two, 0.173 with three; four tokens: 0.307 / 0.259 / 0.224).
+  const long long blocks = static_cast<long long>(T) * L.top_k * L.d_ff / DL_R_MAX;
+  const int max_per_sm = resident_ctas / sms < 3 ? resident_ctas / sms : 3;
+  int per_sm = 1;
+  while (per_sm < max_per_sm && static_cast<long long>(per_sm) * sms * DL_WARPS < blocks) ++per_sm;
+  const int grid = per_sm * sms;
+  if (per_sm < 1 || grid < T * a.rsplit) return cudaErrorInvalidConfiguration;
   return launch_chain(decode_layer_kernel<DL_R_MAX>, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
 }
 
