@@ -719,7 +719,9 @@ def run_emoe(args, w, T, n_layers, rank, world, local):
                             "calls and copy out one after the other on one stream"},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": {
-                "kernel": "expert-FFN kernels (both projections of every layer)", "bound": "hbm",
+                "kernel": ("the one-launch layer kernel (router, both projections, weighted sum of every layer)"
+                           if kernels_per_layer == 1 else "expert-FFN kernels (both projections of every layer)"),
+                "bound": "hbm",
                 "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_8TBs": achieved / 8000.0,
                 "traffic": (ncu_traffic_per_layer(w.name, T) * n_layers
