@@ -293,7 +293,7 @@ int emoe_set_fused_routing(emoe_ctx* ctx, int enabled);
  * emoe_device_status (limit: emoe_set_wait_limit).
  * mode 0: never; 1: every call inside the limits; 2 (the default): calls of up to eight pairs,
  * where it was measured faster than the chain of launches (1.8 x for one pair, 1.5 x for two to
- * four on a Switch-base-sized layer, 1.1 x for eight; for sixteen the chain wins).  Other values:
+ * four on a Switch-base-sized layer, 1.25 x for eight; for sixteen the chain wins).  Other values:
  * EMOE_ERR_INVALID_ARG. */
 int emoe_set_fused_layer(emoe_ctx* ctx, int mode);
 

@@ -374,7 +374,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       ctx->fuse_routing && one_launch_permute && !routed && route_permute_scatter_supported(L, T, ctx->resident_route_ctas);
   // a handful of tokens on a small layer: router, both projections and the gate-weighted sum in one launch
   bool one_launch_layer = false;
-  // as measured on a Switch-base-sized layer: 1.8 x faster than the chain of launches for one pair, 1.5 x for two to four, 1.1 x
+  // as measured on a Switch-base-sized layer: 1.8 x faster than the chain of launches for one pair, 1.5 x for two to four, 1.25 x
   // for eight, slower for sixteen (the projections then take several passes of dependent loads per warp)
   const bool layer_wanted = ctx->fuse_layer == 1 || (ctx->fuse_layer == 2 && P <= 8);
   if (layer_wanted && ctx->ffn_path == 0 && decode_layer_supported(L, T)) {
