@@ -382,7 +382,7 @@ int forward_impl(emoe_ctx* ctx, const emoe_layer_desc* desc, const void* x, int 
       ctx->resident_layer_ctas = decode_layer_resident_ctas(ctx->device);
       EMOE_CUDA(ctx, cudaDeviceGetAttribute(&ctx->sms, cudaDevAttrMultiProcessorCount, ctx->device));
     }
-    one_launch_layer = ctx->sms > 0 && ctx->resident_layer_ctas >= ctx->sms;
+    one_launch_layer = ctx->sms >= T && ctx->resident_layer_ctas >= ctx->sms;  // at least one CTA per SM, one per token
   }
   if (!routed && !one_launch_route && !one_launch_layer)
     EMOE_LAUNCH(ctx, launch_router_topk(x, L.act_bf16, T, L.d_model, router_W, router_bias, bias_token_stride, L.E,

@@ -518,7 +518,8 @@ cudaError_t launch_decode_layer(const LayerDims& L, const ExpertDev* experts, co
   // one pass; else two, else one (eight tokens: 0.361 -> 0.304 ms per 12-layer step with two)
   a.wpr = DL_WPR_MAX;
   while (a.wpr > 1 && static_cast<long long>(T) * (L.d_model / DL_R_MAX) > static_cast<long long>(grid) * (DL_WARPS / a.wpr)) a.wpr >>= 1;
-  if (per_sm < 1 || grid < T * a.rsplit) return cudaErrorInvalidConfiguration;
+  while (a.rsplit > 1 && T * a.rsplit > grid) a.rsplit >>= 1;  // a small device: fewer slices than CTAs
+  if (per_sm < 1 || grid < T) return cudaErrorInvalidConfiguration;
   return launch_chain(decode_layer_kernel<DL_R_MAX>, dim3(grid), dim3(DL_THREADS), decode_layer_smem(), st, a);
 }
 
