@@ -326,6 +326,7 @@ PER_CONFIG = (
     # (label, workload, tokens, copies of the layer so that the weights of a step exceed L2)
     ("cfg0", "switch_tiny_fp32", 16, 8),
     ("cfg1 T=1", "switch_base_decode", 1, 12),
+    ("cfg1 T=4", "switch_base_decode", 4, 12),
     ("cfg1 T=8", "switch_base_decode", 8, 12),
     ("cfg2", "switch_large_prefill", 2048, 2),
     ("cfg3 T=1", "mixtral_decode", 1, 2),
